@@ -1,0 +1,339 @@
+"""fp64 CPU oracle for the MiniCache hot path.  TEST INFRASTRUCTURE ONLY.
+
+This file is the yardstick the CUDA kernels are measured against.  It is a
+plain, slow, step-by-step numpy restatement of the method in double precision
+and shares no code, table or helper with the CUDA path.  Only the tests, the
+smoke check and the CPU-baseline leg of the benchmark may import it; the
+product never does.
+
+What each function follows (MiniCache, arXiv 2405.14366):
+
+* ``merge_rows``            Eq. 3 (SLERP of unit directions), the angle defined
+                            right below Eq. 3, the distance d = Omega / pi of
+                            Sec. 4.2 "Unmergeable token retention", Algorithm 2
+                            "MiniCache Merge".
+* ``store_direction``       Sec. 4.3: the cache is stored in 16-bit floats.
+* ``retention_indices``     Eq. 4 / Algorithm 2 "MiniCache Prefill".
+* ``merge_pair``            Algorithm 2 "MiniCache Prefill" for one layer pair.
+* ``restore``               Eq. 2 and Sec. 4.2 "Cache restoration";
+                            Algorithm 2 "MiniCache Decoding" (rescale, then
+                            put the retained rows back).
+* ``attention`` / ``decode_attention`` / ``decode_attention_compressed``
+                            Algorithm 2 "MiniCache Decoding": concatenate the
+                            new token, softmax(q K^T) V.
+* ``append_rows``           Algorithm 2 "MiniCache Decoding", the branch that
+                            merges the new token pair and appends it.
+* ``merge_rows_fmax`` / ``merge_rows_mean``
+                            Eq. A (Sec. "Alternative merging function") and the
+                            averaging baseline of Sec. 3.1.
+
+Readings taken where the paper is silent or inconsistent (each is a keyword
+argument so the other reading can be run):
+
+* ``convention="eq3"``: t weights layer l (t = 0 gives the direction of layer
+  l-1, t = 1 that of layer l), as Eq. 3 prints it and as the prose around the
+  default t = 0.6 says ("smaller rotation angle to the next layer").
+  ``"alg2"`` swaps the two coefficients, as Algorithm 2's Merge prints them.
+* ``mode="distinct"``: keep tokens with d > d_max - (d_max - d_min) * gamma,
+  i.e. Eq. 4 applied to angular similarity 1 - d, which is what every sentence
+  around Eq. 4 describes (the most distinct pairs are kept).  ``"literal"`` is
+  Eq. 4 exactly as printed; ``"topk"`` keeps the ceil(gamma * n) largest d.
+* one vector = one (token, kv head) row of 128 channels; d_min / d_max are
+  taken per (tensor, sequence, kv head) over that sequence's tokens.
+* sin(Omega) -> 0: same direction  -> normalised linear interpolation (the
+  limit of Eq. 3); opposite direction -> layer l's direction if t >= 0.5 else
+  layer l-1's.  A zero row has angle 0 and contributes no direction.
+* restore divides by the length of the *stored* (16-bit rounded) direction,
+  exactly as Eq. 2 is written.
+
+Parity unpinned: none of the functions here.  What stays unpinned is outside
+this file: whether merging preserves a real model's accuracy needs trained
+weights and datasets and is not claimed anywhere.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+F64 = np.float64
+# arccos of a rounded cosine is only good to about 1e-8 rad next to 0 and pi;
+# below this value of sin(Omega) the limit forms of Eq. 3 are used instead.
+SIN_GUARD = 1e-6
+
+
+# --------------------------------------------------------------------------
+# 16-bit storage formats (bit patterns <-> exact doubles)
+# --------------------------------------------------------------------------
+def decode_bits(bits: np.ndarray, dtype: str) -> np.ndarray:
+    """uint16 bit patterns of IEEE binary16 ("f16") or bfloat16 ("bf16") -> exact float64."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    if dtype == "f16":
+        return bits.view(np.float16).astype(F64)
+    if dtype == "bf16":
+        with np.errstate(invalid="ignore"):
+            return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(F64)
+    raise ValueError(dtype)
+
+
+def encode_bits(x: np.ndarray, dtype: str) -> np.ndarray:
+    """Round float64 to the nearest 16-bit float (ties to even), once, and return its bits."""
+    x = np.asarray(x, dtype=F64)
+    if dtype == "f16":
+        with np.errstate(over="ignore"):
+            return x.astype(np.float16).view(np.uint16)
+    if dtype == "bf16":
+        # bfloat16 = 8 significant bits, binary32 exponent range.  Round on the
+        # bfloat16 grid directly from the double (no intermediate binary32 step).
+        _, ex = np.frexp(x)  # |x| in [2^(ex-1), 2^ex)
+        ex = np.maximum(ex - 1, -126)  # subnormal grid below 2^-126
+        quantum = np.ldexp(1.0, ex - 7)
+        r = np.rint(x / quantum) * quantum  # exact scaling by a power of two; rint = ties to even
+        r = np.where(np.isfinite(x), r, x)
+        r32 = r.astype(np.float32)  # exact: r is on the bfloat16 grid
+        return (r32.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+    raise ValueError(dtype)
+
+
+# --------------------------------------------------------------------------
+# Merge (Eq. 3), distance, alternative merge functions
+# --------------------------------------------------------------------------
+def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") -> Dict[str, np.ndarray]:
+    """SLERP-merge rows a (layer l-1) and c (layer l); both [..., D] float64.
+
+    Returns e (unit direction, float64, not yet rounded for storage), n_a, n_c
+    (the two magnitudes), omega (angle in [0, pi]) and d = omega / pi."""
+    a = np.asarray(a, F64)
+    c = np.asarray(c, F64)
+    n_a = np.sqrt(np.sum(a * a, axis=-1))
+    n_c = np.sqrt(np.sum(c * c, axis=-1))
+    za = n_a == 0.0
+    zc = n_c == 0.0
+    u = a / np.where(za, 1.0, n_a)[..., None]
+    v = c / np.where(zc, 1.0, n_c)[..., None]
+    cosw = np.clip(np.sum(u * v, axis=-1), -1.0, 1.0)
+    omega = np.arccos(cosw)
+    omega = np.where(za | zc, 0.0, omega)
+    sinw = np.sin(omega)
+    if convention == "eq3":
+        ta, tc = 1.0 - t, t
+    elif convention == "alg2":
+        ta, tc = t, 1.0 - t
+    else:
+        raise ValueError(convention)
+    safe = np.where(sinw < SIN_GUARD, 1.0, sinw)
+    w_a = np.sin(ta * omega) / safe
+    w_c = np.sin(tc * omega) / safe
+    e = w_a[..., None] * u + w_c[..., None] * v
+    # sin(Omega) -> 0 with the same direction: limit of Eq. 3, renormalised.
+    same = (sinw < SIN_GUARD) & (cosw > 0.0) & ~(za | zc)
+    if np.any(same):
+        lin = ta * u + tc * v
+        lin = lin / np.sqrt(np.sum(lin * lin, axis=-1))[..., None]
+        e = np.where(same[..., None], lin, e)
+    # opposite directions: Eq. 3 is undefined; take the endpoint t is closer to.
+    opp = (sinw < SIN_GUARD) & (cosw <= 0.0) & ~(za | zc)
+    if np.any(opp):
+        pick = v if tc >= 0.5 else u
+        e = np.where(opp[..., None], pick, e)
+    # zero rows carry no direction: use the other row's (zero vector if both).
+    e = np.where((za & ~zc)[..., None], v, e)
+    e = np.where((zc & ~za)[..., None], u, e)
+    e = np.where((za & zc)[..., None], 0.0, e)
+    return {"e": e, "n_a": n_a, "n_c": n_c, "omega": omega, "d": omega / math.pi}
+
+
+def merge_rows_fmax(a: np.ndarray, c: np.ndarray) -> np.ndarray:
+    """Maximum-norm-preserving interpolation, Eq. A: mean direction x max magnitude."""
+    a = np.asarray(a, F64)
+    c = np.asarray(c, F64)
+    mean = 0.5 * (a + c)
+    nm = np.sqrt(np.sum(mean * mean, axis=-1))
+    big = np.maximum(np.sqrt(np.sum(a * a, -1)), np.sqrt(np.sum(c * c, -1)))
+    return mean / np.where(nm == 0.0, 1.0, nm)[..., None] * big[..., None]
+
+
+def merge_rows_mean(a: np.ndarray, c: np.ndarray) -> np.ndarray:
+    """The averaging baseline of Sec. 3.1: plain mean of the two rows."""
+    return 0.5 * (np.asarray(a, F64) + np.asarray(c, F64))
+
+
+def store_direction(e: np.ndarray, dtype: str) -> np.ndarray:
+    """Round the merged direction to the cache's 16-bit storage format (bits)."""
+    return encode_bits(e, dtype)
+
+
+# --------------------------------------------------------------------------
+# Retention (Eq. 4)
+# --------------------------------------------------------------------------
+def retention_threshold(d: np.ndarray, gamma: float, mode: str = "distinct") -> float:
+    d = np.asarray(d, F64)
+    dmin, dmax = float(np.min(d)), float(np.max(d))
+    if mode == "distinct":
+        return dmax - (dmax - dmin) * gamma
+    if mode == "literal":
+        return dmin + (dmax - dmin) * gamma
+    raise ValueError(mode)
+
+
+def retention_indices(d: np.ndarray, gamma: float, mode: str = "distinct") -> np.ndarray:
+    """Ascending token indices kept unmerged for one segment's distances d [n]."""
+    d = np.asarray(d, F64)
+    n = d.shape[0]
+    if n == 0:
+        return np.zeros(0, np.int64)
+    if mode == "distinct":
+        return np.nonzero(d > retention_threshold(d, gamma, mode))[0].astype(np.int64)
+    if mode == "literal":
+        return np.nonzero(d < retention_threshold(d, gamma, mode))[0].astype(np.int64)
+    if mode == "topk":
+        k = min(n, int(math.ceil(gamma * n - 1e-12)))
+        order = np.lexsort((np.arange(n), -d))  # largest d first, ties -> lower index
+        return np.sort(order[:k]).astype(np.int64)
+    raise ValueError(mode)
+
+
+# --------------------------------------------------------------------------
+# One layer pair (Algorithm 2, "MiniCache Prefill")
+# --------------------------------------------------------------------------
+def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[int], dtype: str,
+               t: float, gamma: float, mode: str = "distinct", convention: str = "eq3",
+               do_retention: bool = True) -> Dict[str, object]:
+    """Compress one tensor (K or V) of a layer pair.
+
+    x_*_bits: uint16 [B][S][H][D] logical rows (layer l-1, layer l).
+    Returns e_bits [B][S][H][D], e (float64, before storage rounding), n_lm1,
+    n_l, d [B][S][H] (float64), ``retained``: dict (b, h) -> ascending indices.
+    The retained raw rows are the input bits at those indices."""
+    a = decode_bits(x_lm1_bits, dtype)
+    c = decode_bits(x_l_bits, dtype)
+    m = merge_rows(a, c, t, convention)
+    e_bits = store_direction(m["e"], dtype)
+    B, S, H, _ = a.shape
+    retained = {}
+    for b in range(B):
+        n = int(seq_lens[b])
+        for h in range(H):
+            if do_retention and n > 0:
+                retained[(b, h)] = retention_indices(m["d"][b, :n, h], gamma, mode)
+            else:
+                retained[(b, h)] = np.zeros(0, np.int64)
+    return {"e_bits": e_bits, "e": m["e"], "n_lm1": m["n_a"], "n_l": m["n_c"], "d": m["d"],
+            "omega": m["omega"], "retained": retained}
+
+
+def append_rows(a_bits: np.ndarray, c_bits: np.ndarray, dtype: str, t: float,
+                convention: str = "eq3") -> Dict[str, np.ndarray]:
+    """Merge the decode step's new token pair (no retention decision for it)."""
+    m = merge_rows(decode_bits(a_bits, dtype), decode_bits(c_bits, dtype), t, convention)
+    m["e_bits"] = store_direction(m["e"], dtype)
+    return m
+
+
+# --------------------------------------------------------------------------
+# Restore (Eq. 2) and attention (Algorithm 2, "MiniCache Decoding")
+# --------------------------------------------------------------------------
+def restore(e_bits: np.ndarray, norms: np.ndarray, dtype: str,
+            retained_idx: Optional[np.ndarray] = None,
+            retained_rows_bits: Optional[np.ndarray] = None) -> np.ndarray:
+    """Restore one layer's rows of one segment.
+
+    e_bits [n][D] stored directions, norms [n] that layer's magnitudes,
+    retained_idx [r] with retained_rows_bits [r][D] that layer's raw rows.
+    Returns float64 [n][D]: e * (norm / ||e||), retained rows put back."""
+    e = decode_bits(e_bits, dtype)
+    len_e = np.sqrt(np.sum(e * e, axis=-1))
+    scale = np.asarray(norms, F64) / np.where(len_e == 0.0, 1.0, len_e)
+    x = e * scale[..., None]
+    if retained_idx is not None and len(retained_idx):
+        x[np.asarray(retained_idx)] = decode_bits(retained_rows_bits, dtype)
+    return x
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, sm_scale: float):
+    """Single-query softmax attention: q [D], k [n][D], v [n][D] -> (o [D], lse)."""
+    s = (k @ q) * sm_scale
+    m = np.max(s)
+    p = np.exp(s - m)
+    z = np.sum(p)
+    return (p @ v) / z, m + math.log(z)
+
+
+def decode_attention(q_bits: np.ndarray, e_k_bits: np.ndarray, e_v_bits: np.ndarray,
+                     n_k: np.ndarray, n_v: np.ndarray, dtype: str, sm_scale: float,
+                     idx_k=None, rows_k_bits=None, idx_v=None, rows_v_bits=None,
+                     k_new_bits=None, v_new_bits=None):
+    """One (sequence, q head) of decode attention for one layer of a pair:
+    restore K and V densely, append the new token, then plain attention."""
+    k_hat = restore(e_k_bits, n_k, dtype, idx_k, rows_k_bits)
+    v_hat = restore(e_v_bits, n_v, dtype, idx_v, rows_v_bits)
+    if k_new_bits is not None:
+        k_hat = np.concatenate([k_hat, decode_bits(k_new_bits, dtype).reshape(1, -1)], axis=0)
+        v_hat = np.concatenate([v_hat, decode_bits(v_new_bits, dtype).reshape(1, -1)], axis=0)
+    return attention(decode_bits(q_bits, dtype), k_hat, v_hat, sm_scale)
+
+
+def decode_attention_compressed(q_bits, e_k_bits, e_v_bits, n_k, n_v, dtype, sm_scale,
+                                idx_k=None, rows_k_bits=None, idx_v=None, rows_v_bits=None,
+                                k_new_bits=None, v_new_bits=None):
+    """Same result as ``decode_attention`` computed without materialising the
+    restored cache: the magnitude is applied to the score (K) and to the
+    probability (V), and retained rows replace single terms.  Kept as a second
+    code path so the two can be checked against each other."""
+    q = decode_bits(q_bits, dtype)
+    ek = decode_bits(e_k_bits, dtype)
+    ev = decode_bits(e_v_bits, dtype)
+    gk = np.asarray(n_k, F64) / np.sqrt(np.sum(ek * ek, -1))
+    gv = np.asarray(n_v, F64) / np.sqrt(np.sum(ev * ev, -1))
+    s = gk * (ek @ q)
+    if idx_k is not None and len(idx_k):
+        s[np.asarray(idx_k)] = decode_bits(rows_k_bits, dtype) @ q
+    s_new = None
+    if k_new_bits is not None:
+        s_new = float(decode_bits(k_new_bits, dtype).reshape(-1) @ q)
+        s = np.concatenate([s, [s_new]])
+    s = s * sm_scale
+    m = np.max(s)
+    p = np.exp(s - m)
+    z = np.sum(p)
+    n = ek.shape[0]
+    coef = p[:n] * gv
+    keep = np.ones(n, bool)
+    o = np.zeros_like(q)
+    if idx_v is not None and len(idx_v):
+        keep[np.asarray(idx_v)] = False
+        o += p[np.asarray(idx_v)] @ decode_bits(rows_v_bits, dtype)
+    o += (coef * keep) @ ev
+    if v_new_bits is not None:
+        o += p[n] * decode_bits(v_new_bits, dtype).reshape(-1)
+    return o / z, m + math.log(z)
+
+
+def lse_combine(parts: List):
+    """Combine partial attention results [(o_j, lse_j)] of disjoint token sets."""
+    lses = np.array([p[1] for p in parts], F64)
+    m = np.max(lses)
+    w = np.exp(lses - m)
+    o = sum(wj * p[0] for wj, p in zip(w, parts)) / np.sum(w)
+    return o, m + math.log(np.sum(w))
+
+
+# --------------------------------------------------------------------------
+# Footprint (Sec. 4.3, Appendix "Detailed Efficiency Derivation")
+# --------------------------------------------------------------------------
+def footprint_bytes(n_layers: int, start_layer: int, tokens_heads: int, head_dim: int,
+                    retained_rows: int, elem_bytes: int = 2) -> Dict[str, float]:
+    """First-principles byte count of the cache, full versus compressed.
+
+    tokens_heads = number of (token, kv head) rows per layer and tensor;
+    retained_rows = total retained (row, tensor) entries over all pairs."""
+    row = head_dim * elem_bytes
+    full = 2 * n_layers * tokens_heads * row
+    n_pairs = (n_layers - start_layer) // 2
+    lower = 2 * (n_layers - 2 * n_pairs) * tokens_heads * row
+    shared = 2 * n_pairs * tokens_heads * row
+    scalars = 2 * n_pairs * tokens_heads * 3 * 4  # two magnitudes and the distance, fp32
+    kept = retained_rows * (2 * row + 4)
+    comp = lower + shared + scalars + kept
+    return {"full": float(full), "compressed": float(comp), "ratio": comp / full}
