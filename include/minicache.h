@@ -1,0 +1,213 @@
+/*
+ * minicache.h -- C ABI of the MiniCache hot path for NVIDIA B200 (sm_100a).
+ *
+ * MiniCache (arXiv 2405.14366) compresses the KV cache in the depth dimension:
+ * for every adjacent layer pair (l-1, l) from the start layer S = L/2 upwards
+ * (Sec. 4.1), each key and value vector of both layers is split into magnitude
+ * and unit direction (Eq. 2), the two directions are merged by spherical
+ * interpolation with parameter t (Eq. 3), both magnitudes are kept, and the
+ * token pairs whose angular distance d = Omega / pi stands out are kept
+ * unmerged (Eq. 4).  At decode time a layer's K/V is the shared direction
+ * times that layer's magnitude with the retained rows put back (Sec. 4.2
+ * "Cache restoration"; Algorithm 2 "MiniCache Decoding").
+ *
+ * One "vector" here is one (token, kv head) row of 128 channels.  d_min and
+ * d_max of Eq. 4 are taken per segment = (tensor K or V, sequence, kv head).
+ *
+ * General conventions
+ * -------------------
+ * - Every pointer inside the structs below is DEVICE memory owned by the caller
+ *   unless a comment says "host".  The library never allocates or frees device
+ *   memory.  Struct arguments themselves live in host memory and are read
+ *   before the call returns.
+ * - All compute calls only enqueue work on `stream` (a cudaStream_t passed as
+ *   void*, NULL = default stream) and return; they never synchronise.
+ * - Pools are paged: [n_pages][n_kv_heads][page_size][128] elements of the
+ *   16-bit storage type, base addresses 256-byte aligned.  One block table
+ *   ([batch][max_pages_per_seq], int32 page ids) addresses every pool of a
+ *   batch: page id p names slot p of the layer pools and of the pair cache
+ *   alike.  Token i of sequence b lives in page block_table[b][i / page_size]
+ *   at row i % page_size.
+ * - Argument errors are reported synchronously through the return code and
+ *   launch nothing.  Data-dependent conditions (retained-row pool too small,
+ *   a bounded wait inside a kernel running out) are recorded in the pair
+ *   cache's device status words and read back with mc_read_status.
+ * - Results are deterministic: identical inputs give bit-identical outputs.
+ */
+#ifndef MINICACHE_H_
+#define MINICACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MC_OK = 0,
+  MC_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum value */
+  MC_ERR_SHAPE = 2,       /* head_dim != 128, page_size not 16/32/64, head ratio not supported */
+  MC_ERR_DTYPE = 3,
+  MC_ERR_ALIGN = 4,       /* a pool base is not 256-byte aligned */
+  MC_ERR_CAPACITY = 5,    /* workspace too small / retained pool overflowed (from mc_read_status) */
+  MC_ERR_UNSUPPORTED = 6,
+  MC_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed; see mc_last_cuda_error */
+  MC_ERR_DEVICE_STATUS = 8 /* a kernel recorded a failure in the status words */
+} mc_status;
+
+typedef enum { MC_F16 = 0, MC_BF16 = 1 } mc_dtype;
+
+/* Which tokens Eq. 4 keeps unmerged.
+ * DISTINCT: d_i > d_max - (d_max - d_min) * gamma  (Eq. 4 applied to similarity 1 - d: the most
+ *           distinct pairs are kept, as the text around Eq. 4 describes; gamma = 0 keeps none).
+ * LITERAL : d_i < d_min + (d_max - d_min) * gamma  (Eq. 4 exactly as printed).
+ * TOPK    : the ceil(gamma * n) largest d (ties: lower index first). */
+typedef enum { MC_RETAIN_DISTINCT = 0, MC_RETAIN_LITERAL = 1, MC_RETAIN_TOPK = 2 } mc_retain_mode;
+
+/* Which layer of the pair a call restores / attends for. BOTH = the two layers at once
+ * (two query sets, one pass over the shared directions). */
+typedef enum { MC_LAYER_LM1 = 0, MC_LAYER_L = 1, MC_LAYER_BOTH = 2 } mc_layer_sel;
+
+/* Operations whose scratch need mc_workspace_bytes reports. */
+typedef enum { MC_OP_MERGE = 0, MC_OP_DECODE_ATTN = 1 } mc_op;
+
+/* Status word indices (mc_read_status). */
+enum {
+  MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out */
+  MC_STATUS_RETAINED_TOTAL = 1, /* retained entries the last merge selected (K and V segments together) */
+  MC_STATUS_RESERVED0 = 2,
+  MC_STATUS_RESERVED1 = 3,
+  MC_STATUS_WORDS = 4
+};
+#define MC_FLAG_RETAIN_OVERFLOW 1
+#define MC_FLAG_WAIT_TIMEOUT 2
+
+/* Method parameters and tensor geometry (Sec. 4.1-4.2, Sec. 5 defaults t = 0.6, gamma = 0.05). */
+typedef struct mc_config {
+  int32_t n_kv_heads;  /* kv heads per layer */
+  int32_t n_q_heads;   /* query heads; n_q_heads / n_kv_heads must be 1, 2, 4 or 8 (at most 4 with MC_LAYER_BOTH) */
+  int32_t head_dim;    /* must be 128 */
+  int32_t page_size;   /* tokens per page: 16, 32 or 64 */
+  int32_t dtype;       /* mc_dtype of K/V/q/out storage */
+  int32_t retain_mode; /* mc_retain_mode */
+  double t;            /* interpolation parameter of Eq. 3: 0 -> direction of layer l-1, 1 -> of layer l */
+  double gamma;        /* retention threshold of Eq. 4 */
+} mc_config;
+
+/* Batch geometry shared by the layer pools and the pair cache. */
+typedef struct mc_batch {
+  const int32_t* block_table; /* [batch][max_pages_per_seq] page ids; entries past a sequence's pages are ignored */
+  const int32_t* seq_lens;    /* [batch] cached tokens per sequence */
+  int32_t batch;
+  int32_t max_pages_per_seq;
+  int32_t max_seq_len;        /* host-known upper bound of seq_lens (sizes grids and workspaces) */
+  int32_t reserved;
+  int64_t n_pages;            /* pages in every pool */
+} mc_batch;
+
+/* One layer's K and V pools: [n_pages][n_kv_heads][page_size][128], 16-bit. */
+typedef struct mc_layer_kv {
+  void* k_pool;
+  void* v_pool;
+} mc_layer_kv;
+
+/* The shared cache C^{l,l-1} of one layer pair (Sec. 4.2: [E, R^l, R^{l-1}, |X^{l-1}|, |X^l|, I]).
+ *
+ * e_k / e_v  shared directions E, rounded to the storage type, every token position kept.
+ * scale      [n_pages][n_kv_heads][4][page_size] fp32; slot 0: K of layer l-1, 1: K of layer l,
+ *            2: V of layer l-1, 3: V of layer l.  The stored number is |x| / |e_stored|, the
+ *            magnitude of Eq. 2 already divided by the length of the rounded direction, so
+ *            that restore is one multiply: x_hat = e_stored * scale.
+ * dist       [n_pages][n_kv_heads][2][page_size] fp32 angular distance d = Omega / pi; slot 0: K, 1: V.
+ * Retention, per segment seg = (tensor * batch + b) * n_kv_heads + head (tensor 0 = K, 1 = V):
+ * ret_count  [2 * batch * n_kv_heads] retained tokens of the segment
+ * ret_offset [2 * batch * n_kv_heads + 1] exclusive prefix of ret_count = first slot of the segment
+ * ret_index  [ret_capacity] token indices, ascending inside a segment
+ * ret_rows   [ret_capacity][2][128] raw 16-bit rows: [.][0] layer l-1, [.][1] layer l (bit copies)
+ * seg_minmax [2 * batch * n_kv_heads][2] fp32 d_min, d_max of the prefill tokens
+ * status     [MC_STATUS_WORDS] int32 */
+typedef struct mc_pair_cache {
+  void* e_k;
+  void* e_v;
+  float* scale;
+  float* dist;
+  int32_t* ret_count;
+  int32_t* ret_offset;
+  int32_t* ret_index;
+  void* ret_rows;
+  int64_t ret_capacity;
+  float* seg_minmax;
+  int32_t* status;
+} mc_pair_cache;
+
+/* Library version (major * 10000 + minor * 100 + patch). No device work. */
+int32_t mc_version(void);
+
+/* Human-readable name of a status code (static string). */
+const char* mc_status_str(int32_t status);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* mc_last_cuda_error(void);
+
+/* Scratch bytes `op` needs for this geometry (a multiple of 256).  Pure host arithmetic.
+ * `n_query_sets` is 2 for MC_LAYER_BOTH decode attention, else 1 (ignored for MC_OP_MERGE). */
+mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_t op,
+                             int32_t n_query_sets, size_t* bytes);
+
+/* Algorithm 2 "MiniCache Prefill" for one layer pair: Eq. 3 merge of every cached token of
+ * every sequence (K and V), magnitudes (Eq. 2), distances, and -- if do_retention -- the
+ * retention set of Eq. 4 with the raw rows of both layers gathered into `out`.
+ * lm1 / l : the two layers' pools (read only; they may be released once the stream has run
+ *           the call).  out: all fields written; status words are cleared first.
+ * With do_retention == 0 every ret_count is set to 0.
+ * If the selection needs more than ret_capacity entries the overflow flag is set, no retained
+ * entry is written and every ret_count is 0 (the merged directions are still valid).
+ * workspace: at least mc_workspace_bytes(MC_OP_MERGE) bytes, 256-byte aligned, contents
+ * irrelevant on entry, must stay untouched until the call has run on the stream. */
+mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1,
+                        const mc_layer_kv* l, const mc_pair_cache* out, int32_t do_retention,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 2 "MiniCache Decoding", the branch that compresses the step's new token pair:
+ * merges k/v_new_lm1 with k/v_new_l ([batch][n_kv_heads][128], 16-bit) by Eq. 3 and writes
+ * direction, scales and distance at token position seq_lens[b] of every sequence (the block
+ * table must already hold a page for it).  No retention decision is taken for new tokens.
+ * seq_lens is not modified: the caller advances it once all layers of the step are done. */
+mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                         const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l,
+                         const void* v_new_l, void* stream);
+
+/* Eq. 2 + Sec. 4.2 "Cache restoration": writes the dense restored K and V of one layer
+ * (layer_sel = MC_LAYER_LM1 or MC_LAYER_L) into dst pools of the same paged layout and type:
+ * x_hat = e * scale, then retained rows overwritten with their raw copies. */
+mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                     int32_t layer_sel, const mc_layer_kv* dst, void* stream);
+
+/* Algorithm 2 "MiniCache Decoding": single-query attention of every sequence over the restored
+ * cache of one layer, computed straight from the compressed pair (restore fused; the dense K/V
+ * is never materialised), split along the token axis and combined by log-sum-exp.
+ * layer_sel   MC_LAYER_LM1 / MC_LAYER_L: one query set.  MC_LAYER_BOTH: two query sets, set 0
+ *             attends layer l-1 and set 1 layer l, sharing one pass over the directions.
+ * q           [n_sets][batch][n_q_heads][128] 16-bit
+ * k_new,v_new [n_sets][batch][n_kv_heads][128] 16-bit raw rows of the step's new token, attended
+ *             as one extra token after the cached ones; both NULL to attend the cache alone.
+ * sm_scale    multiplies q.k before the softmax (Algorithm 2 prints none; pass 1/sqrt(128)).
+ * out         [n_sets][batch][n_q_heads][128] 16-bit
+ * lse         [n_sets][batch][n_q_heads] fp32 natural-log sum of exponentials, or NULL
+ * workspace   at least mc_workspace_bytes(MC_OP_DECODE_ATTN, n_sets) bytes, 256-byte aligned.
+ * A sequence with seq_lens[b] == 0 and no new token yields zeros (lse = -inf). */
+mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                         int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
+                         float sm_scale, void* out, float* lse, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/* Copies the pair's status words to host memory `out_words[MC_STATUS_WORDS]` after synchronising
+ * `stream`.  Returns MC_ERR_CAPACITY if the overflow flag is set, MC_ERR_DEVICE_STATUS for any
+ * other flag, MC_OK otherwise. */
+mc_status mc_read_status(const mc_pair_cache* pair, void* stream, int32_t* out_words);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MINICACHE_H_ */

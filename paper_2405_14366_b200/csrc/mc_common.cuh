@@ -1,0 +1,129 @@
+// Shared device/host helpers of the MiniCache CUDA path (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "minicache.h"
+
+namespace mc {
+
+constexpr int kHeadDim = 128;
+constexpr int kRowBytes = kHeadDim * 2;  // one 16-bit row
+constexpr float kInvPi = 0.31830988618379067154f;
+
+// Host-side launch plumbing ---------------------------------------------------
+void set_cuda_error(cudaError_t e, const char* where);
+#define MC_CUDA_CHECK(expr)            \
+  do {                                 \
+    cudaError_t _e = (expr);           \
+    if (_e != cudaSuccess) {           \
+      ::mc::set_cuda_error(_e, #expr); \
+      return MC_ERR_CUDA;              \
+    }                                  \
+  } while (0)
+
+// Geometry handed to every kernel by value.
+struct Geom {
+  const int32_t* block_table;
+  const int32_t* seq_lens;
+  int batch;
+  int max_pages_per_seq;
+  int n_kv_heads;
+  int page_size;
+  int page_shift;  // log2(page_size)
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// 16-bit storage types ---------------------------------------------------------
+template <int DT>
+struct Elem;
+template <>
+struct Elem<MC_F16> {
+  static __device__ __forceinline__ float2 unpack(uint32_t w) {
+    return __half22float2(*reinterpret_cast<const __half2*>(&w));
+  }
+  static __device__ __forceinline__ uint32_t pack(float x, float y) {
+    __half2 h = __floats2half2_rn(x, y);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+};
+template <>
+struct Elem<MC_BF16> {
+  static __device__ __forceinline__ float2 unpack(uint32_t w) {
+    // bfloat16 is the upper half of a binary32
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+  }
+  static __device__ __forceinline__ uint32_t pack(float x, float y) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
+};
+
+// Streaming 16-byte global accesses (read once / write once data).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream16(void* p, const uint4& v) {
+  asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y),
+               "r"(v.z), "r"(v.w)
+               : "memory");
+}
+
+// Sum over the 16 lanes that share one row (lane ^ 8, 4, 2, 1 stay inside a half-warp).
+__device__ __forceinline__ float sum16(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 8);
+  v += __shfl_xor_sync(0xffffffffu, v, 4);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v;
+}
+
+// Per-row scalars of the merge (Eq. 3 weights folded with 1/|x|, both magnitudes, distance).
+struct RowScalars {
+  float fa, fc;  // e = fa * a + fc * c
+  float na, nc;  // |a|, |c|
+  float d;       // Omega / pi
+};
+
+// Angle and SLERP weights from |a|^2, |c|^2, |u - v|^2, |u + v|^2 (u, v the unit directions).
+// Omega = 2 atan2(|u - v|, |u + v|) is well conditioned at both ends of [0, pi], where arccos
+// of a rounded cosine is not.  ta weights layer l-1, tc layer l (Eq. 3: ta = 1 - t, tc = t).
+__device__ __forceinline__ RowScalars slerp_scalars(float aa, float cc, float sm, float sp, float ta,
+                                                    float tc) {
+  RowScalars r;
+  r.na = sqrtf(aa);
+  r.nc = sqrtf(cc);
+  const float ra = aa > 0.f ? 1.0f / r.na : 0.f;
+  const float rc = cc > 0.f ? 1.0f / r.nc : 0.f;
+  if (aa > 0.f && cc > 0.f) {
+    const float omega = 2.0f * atan2f(sqrtf(sm), sqrtf(sp));
+    const float sinw = sinf(omega);
+    r.d = omega * kInvPi;
+    if (sinw >= 1e-6f) {
+      const float inv = 1.0f / sinw;
+      r.fa = sinf(ta * omega) * inv * ra;
+      r.fc = sinf(tc * omega) * inv * rc;
+    } else if (sp > sm) {  // same direction: limit of Eq. 3
+      r.fa = ta * ra;
+      r.fc = tc * rc;
+    } else {  // opposite directions: the endpoint t is closer to
+      r.fa = tc >= 0.5f ? 0.f : ra;
+      r.fc = tc >= 0.5f ? rc : 0.f;
+    }
+  } else {  // a zero row has no direction: take the other one's
+    r.d = 0.f;
+    r.fa = ra;
+    r.fc = rc;
+  }
+  return r;
+}
+
+}  // namespace mc
