@@ -1,0 +1,229 @@
+"""ctypes binding of libminicache.so: argument marshalling only.
+
+Every function here has the name of the C entry point it wraps (``include/minicache.h``)
+and hands raw device pointers of torch tensors to it.  Nothing is computed in Python, and
+there is no fallback: without the compiled library every call raises."""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+import os
+from typing import Optional
+
+import torch
+
+MC_F16, MC_BF16 = 0, 1
+MC_RETAIN_DISTINCT, MC_RETAIN_LITERAL, MC_RETAIN_TOPK = 0, 1, 2
+MC_LAYER_LM1, MC_LAYER_L, MC_LAYER_BOTH = 0, 1, 2
+MC_OP_MERGE, MC_OP_DECODE_ATTN = 0, 1
+MC_STATUS_WORDS = 4
+MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT = 1, 2
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libminicache.so")
+
+
+class McError(RuntimeError):
+    def __init__(self, code: int, name: str, detail: str = ""):
+        super().__init__(f"{name} ({code}){': ' + detail if detail else ''}")
+        self.code = code
+        self.name = name
+
+
+class _Config(C.Structure):
+    _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("page_size", C.c_int32), ("dtype", C.c_int32), ("retain_mode", C.c_int32),
+                ("t", C.c_double), ("gamma", C.c_double)]
+
+
+class _Batch(C.Structure):
+    _fields_ = [("block_table", C.c_void_p), ("seq_lens", C.c_void_p), ("batch", C.c_int32),
+                ("max_pages_per_seq", C.c_int32), ("max_seq_len", C.c_int32), ("reserved", C.c_int32),
+                ("n_pages", C.c_int64)]
+
+
+class _LayerKV(C.Structure):
+    _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p)]
+
+
+class _PairCache(C.Structure):
+    _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("scale", C.c_void_p), ("dist", C.c_void_p),
+                ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
+                ("ret_rows", C.c_void_p), ("ret_capacity", C.c_int64), ("seg_minmax", C.c_void_p),
+                ("status", C.c_void_p)]
+
+
+EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+           "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+@dataclasses.dataclass
+class McConfig:
+    n_kv_heads: int
+    n_q_heads: int
+    page_size: int
+    dtype: str  # "f16" | "bf16"
+    t: float = 0.6
+    gamma: float = 0.05
+    retain_mode: int = MC_RETAIN_DISTINCT
+    head_dim: int = 128
+
+    def c(self) -> _Config:
+        return _Config(self.n_kv_heads, self.n_q_heads, self.head_dim, self.page_size,
+                       {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma))
+
+    @property
+    def torch_dtype(self):
+        return {"f16": torch.float16, "bf16": torch.bfloat16}[self.dtype]
+
+
+@dataclasses.dataclass
+class Batch:
+    """Device block table / sequence lengths plus the host-known bounds."""
+    block_table: torch.Tensor  # int32 [batch][max_pages_per_seq]
+    seq_lens: torch.Tensor  # int32 [batch]
+    max_seq_len: int
+    n_pages: int
+
+    def c(self) -> _Batch:
+        assert self.block_table.dtype == torch.int32 and self.seq_lens.dtype == torch.int32
+        assert self.block_table.is_contiguous() and self.seq_lens.is_contiguous()
+        b = self.seq_lens.shape[0]
+        mp = self.block_table.shape[1] if self.block_table.dim() == 2 else 0
+        return _Batch(_ptr(self.block_table), _ptr(self.seq_lens), b, mp, int(self.max_seq_len), 0, int(self.n_pages))
+
+
+class PairCache:
+    """Caller-owned device buffers of one compressed layer pair (allocated with torch)."""
+
+    def __init__(self, cfg: McConfig, batch: int, n_pages: int, ret_capacity: int, device="cuda"):
+        H, ps = cfg.n_kv_heads, cfg.page_size
+        dt = cfg.torch_dtype
+        self.cfg = cfg
+        self.e_k = torch.zeros(n_pages, H, ps, 128, dtype=dt, device=device)
+        self.e_v = torch.zeros(n_pages, H, ps, 128, dtype=dt, device=device)
+        self.scale = torch.zeros(n_pages, H, 4, ps, dtype=torch.float32, device=device)
+        self.dist = torch.zeros(n_pages, H, 2, ps, dtype=torch.float32, device=device)
+        nseg = 2 * batch * H
+        self.ret_count = torch.zeros(nseg, dtype=torch.int32, device=device)
+        self.ret_offset = torch.zeros(nseg + 1, dtype=torch.int32, device=device)
+        self.ret_index = torch.zeros(max(ret_capacity, 1), dtype=torch.int32, device=device)
+        self.ret_rows = torch.zeros(max(ret_capacity, 1), 2, 128, dtype=dt, device=device)
+        self.ret_capacity = int(ret_capacity)
+        self.seg_minmax = torch.zeros(nseg, 2, dtype=torch.float32, device=device)
+        self.status = torch.zeros(MC_STATUS_WORDS, dtype=torch.int32, device=device)
+
+    def c(self) -> _PairCache:
+        return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.scale), _ptr(self.dist), _ptr(self.ret_count),
+                          _ptr(self.ret_offset), _ptr(self.ret_index), _ptr(self.ret_rows), self.ret_capacity,
+                          _ptr(self.seg_minmax), _ptr(self.status))
+
+    def nbytes(self) -> int:
+        ts = (self.e_k, self.e_v, self.scale, self.dist, self.ret_count, self.ret_offset, self.ret_index,
+              self.ret_rows, self.seg_minmax, self.status)
+        return sum(t.numel() * t.element_size() for t in ts)
+
+
+class MiniCacheLib:
+    """Loads libminicache.so and exposes its entry points under their C names."""
+
+    def __init__(self, path: str = _LIB_PATH):
+        if not os.path.exists(path):
+            raise McError(-1, "library missing",
+                          f"{path} not built; run `python -m paper_2405_14366_b200.build` (there is no fallback path)")
+        self.path = path
+        self._lib = C.CDLL(path)
+        L = self._lib
+        L.mc_version.restype = C.c_int32
+        L.mc_status_str.restype = C.c_char_p
+        L.mc_status_str.argtypes = [C.c_int32]
+        L.mc_last_cuda_error.restype = C.c_char_p
+        P, V = C.POINTER, C.c_void_p
+        L.mc_workspace_bytes.argtypes = [P(_Config), P(_Batch), C.c_int32, C.c_int32, P(C.c_size_t)]
+        L.mc_merge_pair.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_PairCache), C.c_int32, V,
+                                    C.c_size_t, V]
+        L.mc_append_pair.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, V, V, V, V]
+        L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), V]
+        L.mc_decode_attn.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V,
+                                     C.c_size_t, V]
+        L.mc_read_status.argtypes = [P(_PairCache), V, P(C.c_int32)]
+        for f in ("mc_workspace_bytes", "mc_merge_pair", "mc_append_pair", "mc_restore", "mc_decode_attn",
+                  "mc_read_status"):
+            getattr(L, f).restype = C.c_int32
+
+    # -- helpers ------------------------------------------------------------------------------
+    def _check(self, code: int):
+        if code != 0:
+            name = self._lib.mc_status_str(code).decode()
+            detail = self._lib.mc_last_cuda_error().decode() if code == 7 else ""
+            raise McError(code, name, detail)
+
+    def has_symbol(self, name: str) -> bool:
+        return hasattr(self._lib, name)
+
+    # -- entry points ---------------------------------------------------------------------------
+    def mc_version(self) -> int:
+        return self._lib.mc_version()
+
+    def mc_status_str(self, code: int) -> str:
+        return self._lib.mc_status_str(code).decode()
+
+    def mc_workspace_bytes(self, cfg: McConfig, batch: Batch, op: int, n_query_sets: int = 1) -> int:
+        out = C.c_size_t(0)
+        c, b = cfg.c(), batch.c()
+        self._check(self._lib.mc_workspace_bytes(C.byref(c), C.byref(b), op, n_query_sets, C.byref(out)))
+        return out.value
+
+    def mc_merge_pair(self, cfg: McConfig, batch: Batch, k_lm1, v_lm1, k_l, v_l, pair: PairCache,
+                      do_retention: bool, workspace: torch.Tensor, stream=None):
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        a, l = _LayerKV(_ptr(k_lm1), _ptr(v_lm1)), _LayerKV(_ptr(k_l), _ptr(v_l))
+        self._check(self._lib.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(l), C.byref(pc),
+                                            1 if do_retention else 0, _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_append_pair(self, cfg: McConfig, batch: Batch, pair: PairCache, k_new_lm1, v_new_lm1, k_new_l, v_new_l,
+                       stream=None):
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        self._check(self._lib.mc_append_pair(C.byref(c), C.byref(b), C.byref(pc), _ptr(k_new_lm1), _ptr(v_new_lm1),
+                                             _ptr(k_new_l), _ptr(v_new_l), _stream(stream)))
+
+    def mc_restore(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, dst_k, dst_v, stream=None):
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        d = _LayerKV(_ptr(dst_k), _ptr(dst_v))
+        self._check(self._lib.mc_restore(C.byref(c), C.byref(b), C.byref(pc), layer_sel, C.byref(d), _stream(stream)))
+
+    def mc_decode_attn(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q, k_new, v_new,
+                       sm_scale: float, out, lse, workspace: torch.Tensor, stream=None):
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        self._check(self._lib.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q), _ptr(k_new),
+                                             _ptr(v_new), float(sm_scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                             workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_read_status(self, pair: PairCache, stream=None, check: bool = True):
+        words = (C.c_int32 * MC_STATUS_WORDS)()
+        pc = pair.c()
+        code = self._lib.mc_read_status(C.byref(pc), _stream(stream), words)
+        if check:
+            self._check(code)
+        return list(words), code
+
+
+_LIB: Optional[MiniCacheLib] = None
+
+
+def lib() -> MiniCacheLib:
+    """The process-wide library handle (raises if the shared object has not been built)."""
+    global _LIB
+    if _LIB is None:
+        _LIB = MiniCacheLib()
+    return _LIB

@@ -1,0 +1,187 @@
+// C-ABI entry points: argument validation and dispatch to the kernel launchers.
+#include <stdio.h>
+#include <string.h>
+
+#include "mc_common.cuh"
+#include "mc_kernels.h"
+
+namespace mc {
+
+static thread_local char g_cuda_error[256] = "";
+
+void set_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+  (void)cudaGetLastError();  // clear the sticky-free error state
+}
+
+static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+static mc_status check_config(const mc_config* cfg) {
+  if (cfg == nullptr) return MC_ERR_INVALID_ARG;
+  if (cfg->head_dim != kHeadDim) return MC_ERR_SHAPE;
+  if (cfg->page_size != 16 && cfg->page_size != 32 && cfg->page_size != 64) return MC_ERR_SHAPE;
+  if (cfg->n_kv_heads <= 0 || cfg->n_q_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads != 0) return MC_ERR_SHAPE;
+  const int nq = cfg->n_q_heads / cfg->n_kv_heads;
+  if (nq != 1 && nq != 2 && nq != 4 && nq != 8) return MC_ERR_SHAPE;
+  if (cfg->dtype != MC_F16 && cfg->dtype != MC_BF16) return MC_ERR_DTYPE;
+  if (cfg->retain_mode < MC_RETAIN_DISTINCT || cfg->retain_mode > MC_RETAIN_TOPK) return MC_ERR_INVALID_ARG;
+  if (!(cfg->t >= 0.0 && cfg->t <= 1.0) || !(cfg->gamma >= 0.0 && cfg->gamma <= 1.0)) return MC_ERR_INVALID_ARG;
+  return MC_OK;
+}
+
+static mc_status check_batch(const mc_config* cfg, const mc_batch* bt) {
+  if (bt == nullptr) return MC_ERR_INVALID_ARG;
+  if (bt->batch < 0 || bt->max_pages_per_seq < 0 || bt->max_seq_len < 0 || bt->n_pages < 0) return MC_ERR_INVALID_ARG;
+  if (bt->batch > 0 && (bt->block_table == nullptr || bt->seq_lens == nullptr)) return MC_ERR_INVALID_ARG;
+  if ((long long)bt->max_pages_per_seq * cfg->page_size < bt->max_seq_len) return MC_ERR_SHAPE;
+  if (2LL * bt->batch * cfg->n_kv_heads > 65535) return MC_ERR_SHAPE;  // one grid row per segment
+  if (bt->n_pages * cfg->n_kv_heads * cfg->page_size > 0x7fffffffLL) return MC_ERR_SHAPE;
+  return MC_OK;
+}
+
+static mc_status check_pair(const mc_pair_cache* pc) {
+  if (pc == nullptr) return MC_ERR_INVALID_ARG;
+  if (!pc->e_k || !pc->e_v || !pc->scale || !pc->dist || !pc->ret_count || !pc->ret_offset || !pc->seg_minmax ||
+      !pc->status)
+    return MC_ERR_INVALID_ARG;
+  if (pc->ret_capacity < 0) return MC_ERR_INVALID_ARG;
+  if (pc->ret_capacity > 0 && (!pc->ret_index || !pc->ret_rows)) return MC_ERR_INVALID_ARG;
+  if (!aligned256(pc->e_k) || !aligned256(pc->e_v) || !aligned256(pc->scale) || !aligned256(pc->dist)) return MC_ERR_ALIGN;
+  if (pc->ret_rows && !aligned256(pc->ret_rows)) return MC_ERR_ALIGN;
+  return MC_OK;
+}
+
+static Geom make_geom(const mc_config* cfg, const mc_batch* bt) {
+  Geom g;
+  g.block_table = bt->block_table;
+  g.seq_lens = bt->seq_lens;
+  g.batch = bt->batch;
+  g.max_pages_per_seq = bt->max_pages_per_seq;
+  g.n_kv_heads = cfg->n_kv_heads;
+  g.page_size = cfg->page_size;
+  g.page_shift = cfg->page_size == 16 ? 4 : (cfg->page_size == 32 ? 5 : 6);
+  return g;
+}
+
+}  // namespace mc
+
+using namespace mc;
+
+extern "C" {
+
+int32_t mc_version(void) { return 100; }
+
+const char* mc_status_str(int32_t s) {
+  switch (s) {
+    case MC_OK: return "MC_OK";
+    case MC_ERR_INVALID_ARG: return "MC_ERR_INVALID_ARG";
+    case MC_ERR_SHAPE: return "MC_ERR_SHAPE";
+    case MC_ERR_DTYPE: return "MC_ERR_DTYPE";
+    case MC_ERR_ALIGN: return "MC_ERR_ALIGN";
+    case MC_ERR_CAPACITY: return "MC_ERR_CAPACITY";
+    case MC_ERR_UNSUPPORTED: return "MC_ERR_UNSUPPORTED";
+    case MC_ERR_CUDA: return "MC_ERR_CUDA";
+    case MC_ERR_DEVICE_STATUS: return "MC_ERR_DEVICE_STATUS";
+    default: return "MC_ERR_UNKNOWN";
+  }
+}
+
+const char* mc_last_cuda_error(void) { return g_cuda_error; }
+
+mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_t op, int32_t n_query_sets,
+                             size_t* bytes) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (batch == nullptr || bytes == nullptr) return MC_ERR_INVALID_ARG;
+  if (batch->batch < 0 || batch->max_seq_len < 0) return MC_ERR_INVALID_ARG;
+  if (op == MC_OP_MERGE) {
+    *bytes = merge_workspace_bytes(cfg, batch) + 256;
+  } else if (op == MC_OP_DECODE_ATTN) {
+    if (n_query_sets != 1 && n_query_sets != 2) return MC_ERR_INVALID_ARG;
+    *bytes = attn_workspace_bytes(cfg, batch, n_query_sets) + 256;
+  } else {
+    return MC_ERR_INVALID_ARG;
+  }
+  return MC_OK;
+}
+
+mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1, const mc_layer_kv* l,
+                        const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(out);
+  if (st != MC_OK) return st;
+  if (!lm1 || !l || !lm1->k_pool || !lm1->v_pool || !l->k_pool || !l->v_pool) return MC_ERR_INVALID_ARG;
+  if (!aligned256(lm1->k_pool) || !aligned256(lm1->v_pool) || !aligned256(l->k_pool) || !aligned256(l->v_pool))
+    return MC_ERR_ALIGN;
+  if (do_retention && cfg->retain_mode == MC_RETAIN_TOPK) return MC_ERR_UNSUPPORTED;
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
+  return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, out, do_retention ? 1 : 0, workspace,
+                      (cudaStream_t)stream);
+}
+
+mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, const void* k_new_lm1,
+                         const void* v_new_lm1, const void* k_new_l, const void* v_new_l, void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(pair);
+  if (st != MC_OK) return st;
+  if (!k_new_lm1 || !v_new_lm1 || !k_new_l || !v_new_l) return MC_ERR_INVALID_ARG;
+  const uintptr_t al = (uintptr_t)k_new_lm1 | (uintptr_t)v_new_lm1 | (uintptr_t)k_new_l | (uintptr_t)v_new_l;
+  if (al & 15u) return MC_ERR_ALIGN;
+  return launch_append(cfg, batch, make_geom(cfg, batch), pair, k_new_lm1, v_new_lm1, k_new_l, v_new_l,
+                       (cudaStream_t)stream);
+}
+
+mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
+                     const mc_layer_kv* dst, void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(pair);
+  if (st != MC_OK) return st;
+  if (layer_sel != MC_LAYER_LM1 && layer_sel != MC_LAYER_L) return MC_ERR_INVALID_ARG;
+  if (!dst || !dst->k_pool || !dst->v_pool) return MC_ERR_INVALID_ARG;
+  if (!aligned256(dst->k_pool) || !aligned256(dst->v_pool)) return MC_ERR_ALIGN;
+  return launch_restore(cfg, batch, make_geom(cfg, batch), pair, layer_sel, dst, (cudaStream_t)stream);
+}
+
+mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
+                         const void* q, const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(pair);
+  if (st != MC_OK) return st;
+  if (layer_sel < MC_LAYER_LM1 || layer_sel > MC_LAYER_BOTH) return MC_ERR_INVALID_ARG;
+  const int n_sets = layer_sel == MC_LAYER_BOTH ? 2 : 1;
+  if (n_sets * (cfg->n_q_heads / cfg->n_kv_heads) > 8) return MC_ERR_SHAPE;
+  if (!q || !out) return MC_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return MC_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15u) return MC_ERR_ALIGN;
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  if (workspace_bytes < attn_workspace_bytes(cfg, batch, n_sets)) return MC_ERR_CAPACITY;
+  return launch_decode_attn(cfg, batch, make_geom(cfg, batch), pair, layer_sel, q, k_new, v_new, sm_scale, out, lse,
+                            workspace, (cudaStream_t)stream);
+}
+
+mc_status mc_read_status(const mc_pair_cache* pair, void* stream, int32_t* out_words) {
+  if (pair == nullptr || pair->status == nullptr || out_words == nullptr) return MC_ERR_INVALID_ARG;
+  MC_CUDA_CHECK(cudaMemcpyAsync(out_words, pair->status, MC_STATUS_WORDS * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                                (cudaStream_t)stream));
+  MC_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  if (out_words[MC_STATUS_FLAGS] & MC_FLAG_RETAIN_OVERFLOW) return MC_ERR_CAPACITY;
+  if (out_words[MC_STATUS_FLAGS] != 0) return MC_ERR_DEVICE_STATUS;
+  return MC_OK;
+}
+
+}  // extern "C"

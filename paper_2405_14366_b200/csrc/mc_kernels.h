@@ -1,0 +1,22 @@
+// Internal launch interface between the C-ABI dispatch (mc_api.cu) and the kernel files.
+#pragma once
+#include "mc_common.cuh"
+
+namespace mc {
+
+size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt);
+mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
+                       const mc_layer_kv* l, const mc_pair_cache* out, int do_retention, void* workspace,
+                       cudaStream_t stream);
+mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
+                        const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
+                        cudaStream_t stream);
+mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
+                         int layer, const mc_layer_kv* dst, cudaStream_t stream);
+
+size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets);
+mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
+                             int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,
+                             void* out, float* lse, void* workspace, cudaStream_t stream);
+
+}  // namespace mc

@@ -1,0 +1,502 @@
+// Cross-layer merge of one layer pair (Algorithm 2 "MiniCache Prefill"):
+//   merge_kernel      Eq. 2 magnitudes, angle, Eq. 3 SLERP direction, distance d = Omega / pi,
+//                     per-segment d_min / d_max
+//   retain_*          Eq. 4 retention set: count, scan, ordered compaction + raw-row gather
+//   append_kernel     the decode-time merge of one new token per sequence
+#include "mc_common.cuh"
+#include "mc_kernels.h"
+
+namespace mc {
+
+constexpr int kMergeThreads = 256;
+constexpr int kRowsPerItem = 64;  // rows of one page handled by one CTA
+constexpr int kRowsPerHalfWarp = 4;
+
+struct MergeParams {
+  Geom g;
+  const char* a_pool[2];  // layer l-1: K, V
+  const char* c_pool[2];  // layer l:   K, V
+  char* e_pool[2];
+  float* scale;
+  float* dist;
+  unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
+  float ta, tc;
+  int items_per_page;
+};
+
+// One merged row: 16 lanes hold 8 channels each of a (layer l-1) and c (layer l).
+template <int DT>
+__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, uint4& e_out,
+                                          float& g_a, float& g_c, float& d_out) {
+  float a[8], c[8];
+  {
+    const uint32_t wa[4] = {ra.x, ra.y, ra.z, ra.w};
+    const uint32_t wc[4] = {rc.x, rc.y, rc.z, rc.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 fa = Elem<DT>::unpack(wa[i]);
+      float2 fc = Elem<DT>::unpack(wc[i]);
+      a[2 * i] = fa.x;
+      a[2 * i + 1] = fa.y;
+      c[2 * i] = fc.x;
+      c[2 * i + 1] = fc.y;
+    }
+  }
+  float aa = 0.f, cc = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    aa = fmaf(a[i], a[i], aa);
+    cc = fmaf(c[i], c[i], cc);
+  }
+  aa = sum16(aa);
+  cc = sum16(cc);
+  const float ia = aa > 0.f ? rsqrtf(aa) : 0.f;
+  const float ic = cc > 0.f ? rsqrtf(cc) : 0.f;
+  // |u - v|^2 and |u + v|^2 formed channel by channel: no cancellation at small or large angles
+  float sm = 0.f, sp = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float u = a[i] * ia;
+    const float dm = fmaf(-c[i], ic, u);
+    const float dp = fmaf(c[i], ic, u);
+    sm = fmaf(dm, dm, sm);
+    sp = fmaf(dp, dp, sp);
+  }
+  sm = sum16(sm);
+  sp = sum16(sp);
+  const RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
+  uint32_t w[4];
+  float ee = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float x = fmaf(s.fa, a[2 * i], s.fc * c[2 * i]);
+    const float y = fmaf(s.fa, a[2 * i + 1], s.fc * c[2 * i + 1]);
+    w[i] = Elem<DT>::pack(x, y);
+    const float2 r = Elem<DT>::unpack(w[i]);  // the stored value: Eq. 2 divides by its length
+    ee = fmaf(r.x, r.x, ee);
+    ee = fmaf(r.y, r.y, ee);
+  }
+  ee = sum16(ee);
+  const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
+  e_out = make_uint4(w[0], w[1], w[2], w[3]);
+  g_a = s.na * il;
+  g_c = s.nc * il;
+  d_out = s.d;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams p) {
+  __shared__ unsigned s_min[4], s_max[4];
+  const int ipp = p.items_per_page;
+  int bid = blockIdx.x;
+  const int item = bid % ipp;
+  bid /= ipp;
+  const int pslot = bid % p.g.max_pages_per_seq;
+  bid /= p.g.max_pages_per_seq;
+  const int b = bid % p.g.batch;
+  const int tensor = bid / p.g.batch;
+
+  const int n = p.g.seq_lens[b];
+  const int ps = p.g.page_size;
+  if (pslot * ps >= n) return;
+  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + pslot];
+  const int H = p.g.n_kv_heads;
+  const int rows_in_page = H * ps;
+
+  if (threadIdx.x < 4) {
+    s_min[threadIdx.x] = 0x7f800000u;
+    s_max[threadIdx.x] = 0u;
+  }
+  __syncthreads();
+
+  const int hw = threadIdx.x >> 4;
+  const int l16 = threadIdx.x & 15;
+  const int row0 = item * kRowsPerItem + hw * kRowsPerHalfWarp;  // 4 consecutive rows, one head
+  const int head = row0 >> p.g.page_shift;
+  const int tk0 = row0 & (ps - 1);
+  const int tok0 = pslot * ps + tk0;
+  const size_t page_off = (size_t)page * rows_in_page;
+  const char* pa = p.a_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
+  const char* pc = p.c_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
+  char* pe = p.e_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
+
+  uint4 va[kRowsPerHalfWarp], vc[kRowsPerHalfWarp];
+  bool valid[kRowsPerHalfWarp];
+#pragma unroll
+  for (int j = 0; j < kRowsPerHalfWarp; ++j) {
+    valid[j] = (row0 + j < rows_in_page) && (tok0 + j < n);
+    if (valid[j]) {
+      va[j] = ld_stream16(pa + j * kRowBytes);
+      vc[j] = ld_stream16(pc + j * kRowBytes);
+    } else {
+      va[j] = make_uint4(0, 0, 0, 0);
+      vc[j] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  float dmin = __int_as_float(0x7f800000), dmax = 0.f;
+  float ga[kRowsPerHalfWarp], gc[kRowsPerHalfWarp], dd[kRowsPerHalfWarp];
+#pragma unroll
+  for (int j = 0; j < kRowsPerHalfWarp; ++j) {
+    uint4 e;
+    merge_row<DT>(va[j], vc[j], p.ta, p.tc, e, ga[j], gc[j], dd[j]);
+    if (valid[j]) {
+      st_stream16(pe + j * kRowBytes, e);
+      dmin = fminf(dmin, dd[j]);
+      dmax = fmaxf(dmax, dd[j]);
+    }
+  }
+  // lane j of the half-warp writes token j's three scalars (consecutive tokens -> 16-byte runs)
+  if (l16 < kRowsPerHalfWarp && row0 < rows_in_page) {
+    float g_a = ga[0], g_c = gc[0], d = dd[0];
+    bool ok = valid[0];
+#pragma unroll
+    for (int j = 1; j < kRowsPerHalfWarp; ++j)
+      if (l16 == j) {
+        g_a = ga[j];
+        g_c = gc[j];
+        d = dd[j];
+        ok = valid[j];
+      }
+    if (ok) {
+      const size_t ph = (size_t)page * H + head;
+      float* sc = p.scale + (ph * 4 + tensor * 2) * ps + tk0 + l16;
+      sc[0] = g_a;
+      sc[ps] = g_c;
+      p.dist[(ph * 2 + tensor) * ps + tk0 + l16] = d;
+    }
+  }
+  if (l16 == 0 && valid[0]) {
+    const int hl = (hw * kRowsPerHalfWarp) >> p.g.page_shift;  // head inside the item
+    atomicMin(&s_min[hl], __float_as_uint(dmin));
+    atomicMax(&s_max[hl], __float_as_uint(dmax));
+  }
+  __syncthreads();
+  const int heads_per_item = kRowsPerItem >> p.g.page_shift;
+  if ((int)threadIdx.x < heads_per_item) {
+    const int h = (item * kRowsPerItem >> p.g.page_shift) + threadIdx.x;
+    if (h < H && s_min[threadIdx.x] != 0x7f800000u) {
+      const size_t seg = ((size_t)tensor * p.g.batch + b) * H + h;
+      atomicMin(&p.seg_minmax[seg * 2], s_min[threadIdx.x]);
+      atomicMax(&p.seg_minmax[seg * 2 + 1], s_max[threadIdx.x]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Retention (Eq. 4)
+// ---------------------------------------------------------------------------------------------
+constexpr int kChunk = 1024;  // tokens per retention work item
+constexpr int kRetThreads = 256;
+
+struct RetainParams {
+  Geom g;
+  const char* a_pool[2];
+  const char* c_pool[2];
+  const float* dist;
+  const float* seg_minmax;
+  int32_t* chunk_count;   // workspace [nseg][chunks_per_seg]
+  int32_t* chunk_offset;  // workspace [nseg][chunks_per_seg]
+  int32_t* ret_count;
+  int32_t* ret_offset;
+  int32_t* ret_index;
+  char* ret_rows;
+  int64_t ret_capacity;
+  int32_t* status;
+  int chunks_per_seg;
+  int nseg;
+  int mode;
+  int do_retention;
+  double gamma;
+};
+
+__global__ void merge_init_kernel(unsigned* seg_minmax, int nseg, int32_t* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < nseg) {
+    seg_minmax[2 * i] = 0x7f800000u;
+    seg_minmax[2 * i + 1] = 0u;
+  }
+  if (i < MC_STATUS_WORDS) status[i] = 0;
+}
+
+// Retention decision of one token; the threshold is formed in double from the fp32 extremes.
+__device__ __forceinline__ bool keep_token(float d, float dmin, float dmax, double gamma, int mode) {
+  const double lo = dmin, hi = dmax;
+  if (mode == MC_RETAIN_DISTINCT) return (double)d > hi - (hi - lo) * gamma;
+  return (double)d < lo + (hi - lo) * gamma;
+}
+
+__device__ __forceinline__ float load_dist(const RetainParams& p, int tensor, int b, int h, int tok) {
+  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+  return p.dist[(((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok & (p.g.page_size - 1))];
+}
+
+__global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainParams p) {
+  __shared__ int s_cnt[kRetThreads / 32];
+  const int seg = blockIdx.y, chunk = blockIdx.x;
+  const int h = seg % p.g.n_kv_heads;
+  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
+  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  const int n = p.g.seq_lens[b];
+  int cnt = 0;
+  if (p.do_retention && chunk * kChunk < n) {
+    const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
+    for (int i = threadIdx.x; i < kChunk; i += kRetThreads) {
+      const int tok = chunk * kChunk + i;
+      if (tok < n) cnt += keep_token(load_dist(p, tensor, b, h, tok), dmin, dmax, p.gamma, p.mode) ? 1 : 0;
+    }
+  }
+  for (int o = 16; o; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if ((threadIdx.x & 31) == 0) s_cnt[threadIdx.x >> 5] = cnt;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = 0;
+    for (int w = 0; w < kRetThreads / 32; ++w) t += s_cnt[w];
+    p.chunk_count[(size_t)seg * p.chunks_per_seg + chunk] = t;
+  }
+}
+
+// One CTA: exclusive scan of the chunk counts in (segment, chunk) order.
+__global__ void __launch_bounds__(1024) retain_scan_kernel(const RetainParams p) {
+  __shared__ int s_warp[32];
+  __shared__ int s_carry;
+  const int total = p.nseg * p.chunks_per_seg;
+  if (threadIdx.x == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < total; base += 1024) {
+    const int i = base + threadIdx.x;
+    const int v = i < total ? p.chunk_count[i] : 0;
+    int x = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if ((threadIdx.x & 31) >= o) x += y;
+    }
+    if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int w = s_warp[threadIdx.x];
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, w, o);
+        if ((int)threadIdx.x >= o) w += y;
+      }
+      s_warp[threadIdx.x] = w;  // inclusive over warps
+    }
+    __syncthreads();
+    const int warp_excl = (threadIdx.x >> 5) ? s_warp[(threadIdx.x >> 5) - 1] : 0;
+    const int excl = s_carry + warp_excl + x - v;
+    if (i < total) {
+      p.chunk_offset[i] = excl;
+      if (i % p.chunks_per_seg == 0) p.ret_offset[i / p.chunks_per_seg] = excl;
+    }
+    __syncthreads();
+    if (threadIdx.x == 1023) s_carry = excl + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const int sum = s_carry;
+    p.ret_offset[p.nseg] = sum;
+    p.status[MC_STATUS_RETAINED_TOTAL] = sum;
+    if ((int64_t)sum > p.ret_capacity) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_RETAIN_OVERFLOW);
+  }
+}
+
+// Per (segment, chunk): ordered compaction of the kept token indices, then bit copies of both
+// layers' rows.  Writes ret_count per segment from the chunk offsets.
+__global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const RetainParams p) {
+  __shared__ int s_warp[kRetThreads / 32];
+  __shared__ int s_base;
+  const int seg = blockIdx.y, chunk = blockIdx.x;
+  const int h = seg % p.g.n_kv_heads;
+  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
+  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  const int n = p.g.seq_lens[b];
+  const bool overflow = (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
+  if (chunk == 0 && threadIdx.x == 0)
+    p.ret_count[seg] = overflow ? 0 : p.ret_offset[seg + 1] - p.ret_offset[seg];
+  if (overflow || !p.do_retention || chunk * kChunk >= n) return;
+  const size_t ci = (size_t)seg * p.chunks_per_seg + chunk;
+  const int my_count = p.chunk_count[ci];
+  if (my_count == 0) return;
+  const int out0 = p.chunk_offset[ci];
+  const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
+  if (threadIdx.x == 0) s_base = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int r = 0; r < kChunk; r += kRetThreads) {
+    const int tok = chunk * kChunk + r + threadIdx.x;
+    const bool keep = tok < n && keep_token(load_dist(p, tensor, b, h, tok), dmin, dmax, p.gamma, p.mode);
+    const unsigned m = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) s_warp[warp] = __popc(m);
+    __syncthreads();
+    int before = s_base;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+    if (keep) p.ret_index[out0 + before + __popc(m & ((1u << lane) - 1))] = tok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = s_base;
+      for (int w = 0; w < kRetThreads / 32; ++w) t += s_warp[w];
+      s_base = t;
+    }
+    __syncthreads();
+  }
+  // gather: one half-warp per (entry, layer) row of 256 bytes
+  const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+  for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
+    const int ent = r >> 1, layer = r & 1;
+    const int tok = p.ret_index[out0 + ent];
+    const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+    const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
+    const char* src = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kRowBytes + l16 * 16;
+    char* dst = p.ret_rows + ((size_t)(out0 + ent) * 2 + layer) * kRowBytes + l16 * 16;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode-time append (Algorithm 2 "MiniCache Decoding": merge of the new token pair)
+// ---------------------------------------------------------------------------------------------
+struct AppendParams {
+  Geom g;
+  const char* a_new[2];  // [batch][H][128]: K, V of layer l-1
+  const char* c_new[2];
+  char* e_pool[2];
+  float* scale;
+  float* dist;
+  float ta, tc;
+  int total_rows;  // 2 * batch * H
+};
+
+template <int DT>
+__global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
+  const int r = blockIdx.x * (128 / 16) + (threadIdx.x >> 4);
+  const int l16 = threadIdx.x & 15;
+  const bool ok = r < p.total_rows;
+  const int rr = ok ? r : 0;
+  const int H = p.g.n_kv_heads;
+  const int h = rr % H;
+  const int b = (rr / H) % p.g.batch;
+  const int tensor = rr / (H * p.g.batch);
+  uint4 va = make_uint4(0, 0, 0, 0), vc = va;
+  if (ok) {
+    const size_t off = ((size_t)b * H + h) * kRowBytes + l16 * 16;
+    va = *reinterpret_cast<const uint4*>(p.a_new[tensor] + off);
+    vc = *reinterpret_cast<const uint4*>(p.c_new[tensor] + off);
+  }
+  uint4 e;
+  float ga, gc, d;
+  merge_row<DT>(va, vc, p.ta, p.tc, e, ga, gc, d);
+  if (!ok) return;
+  const int tok = p.g.seq_lens[b];
+  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+  const int tk = tok & (p.g.page_size - 1);
+  const size_t ph = (size_t)page * H + h;
+  *reinterpret_cast<uint4*>(p.e_pool[tensor] + (ph * p.g.page_size + tk) * kRowBytes + l16 * 16) = e;
+  if (l16 == 0) {
+    float* sc = p.scale + (ph * 4 + tensor * 2) * p.g.page_size + tk;
+    sc[0] = ga;
+    sc[p.g.page_size] = gc;
+    p.dist[(ph * 2 + tensor) * p.g.page_size + tk] = d;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------------------------
+static inline int chunks_per_seg(int max_seq_len) { return max_seq_len > 0 ? (max_seq_len + kChunk - 1) / kChunk : 1; }
+
+size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
+  const size_t nseg = (size_t)2 * bt->batch * cfg->n_kv_heads;
+  return align_up(nseg * chunks_per_seg(bt->max_seq_len) * sizeof(int32_t), 256) * 2;
+}
+
+mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
+                       const mc_layer_kv* l, const mc_pair_cache* out, int do_retention, void* workspace,
+                       cudaStream_t stream) {
+  const int nseg = 2 * bt->batch * cfg->n_kv_heads;
+  merge_init_kernel<<<(max(nseg, MC_STATUS_WORDS) + 255) / 256, 256, 0, stream>>>(
+      reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status);
+  MC_CUDA_CHECK(cudaGetLastError());
+  if (bt->batch == 0) return MC_OK;
+
+  MergeParams mp;
+  mp.g = g;
+  mp.a_pool[0] = (const char*)lm1->k_pool;
+  mp.a_pool[1] = (const char*)lm1->v_pool;
+  mp.c_pool[0] = (const char*)l->k_pool;
+  mp.c_pool[1] = (const char*)l->v_pool;
+  mp.e_pool[0] = (char*)out->e_k;
+  mp.e_pool[1] = (char*)out->e_v;
+  mp.scale = out->scale;
+  mp.dist = out->dist;
+  mp.seg_minmax = reinterpret_cast<unsigned*>(out->seg_minmax);
+  mp.ta = (float)(1.0 - cfg->t);
+  mp.tc = (float)cfg->t;
+  mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
+  const long long blocks = 2LL * bt->batch * bt->max_pages_per_seq * mp.items_per_page;
+  if (blocks > 0) {
+    if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
+    if (cfg->dtype == MC_F16)
+      merge_kernel<MC_F16><<<(unsigned)blocks, kMergeThreads, 0, stream>>>(mp);
+    else
+      merge_kernel<MC_BF16><<<(unsigned)blocks, kMergeThreads, 0, stream>>>(mp);
+    MC_CUDA_CHECK(cudaGetLastError());
+  }
+
+  RetainParams rp;
+  rp.g = g;
+  rp.a_pool[0] = mp.a_pool[0];
+  rp.a_pool[1] = mp.a_pool[1];
+  rp.c_pool[0] = mp.c_pool[0];
+  rp.c_pool[1] = mp.c_pool[1];
+  rp.dist = out->dist;
+  rp.seg_minmax = out->seg_minmax;
+  rp.chunks_per_seg = chunks_per_seg(bt->max_seq_len);
+  rp.nseg = nseg;
+  rp.chunk_count = reinterpret_cast<int32_t*>(workspace);
+  rp.chunk_offset = reinterpret_cast<int32_t*>((char*)workspace +
+                                               align_up((size_t)nseg * rp.chunks_per_seg * sizeof(int32_t), 256));
+  rp.ret_count = out->ret_count;
+  rp.ret_offset = out->ret_offset;
+  rp.ret_index = out->ret_index;
+  rp.ret_rows = (char*)out->ret_rows;
+  rp.ret_capacity = out->ret_capacity;
+  rp.status = out->status;
+  rp.mode = cfg->retain_mode;
+  rp.do_retention = do_retention;
+  rp.gamma = cfg->gamma;
+  dim3 grid(rp.chunks_per_seg, nseg);
+  retain_count_kernel<<<grid, kRetThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(cudaGetLastError());
+  retain_scan_kernel<<<1, 1024, 0, stream>>>(rp);
+  MC_CUDA_CHECK(cudaGetLastError());
+  retain_compact_kernel<<<grid, kRetThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(cudaGetLastError());
+  return MC_OK;
+}
+
+mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
+                        const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
+                        cudaStream_t stream) {
+  AppendParams ap;
+  ap.g = g;
+  ap.a_new[0] = (const char*)k_new_lm1;
+  ap.a_new[1] = (const char*)v_new_lm1;
+  ap.c_new[0] = (const char*)k_new_l;
+  ap.c_new[1] = (const char*)v_new_l;
+  ap.e_pool[0] = (char*)pair->e_k;
+  ap.e_pool[1] = (char*)pair->e_v;
+  ap.scale = pair->scale;
+  ap.dist = pair->dist;
+  ap.ta = (float)(1.0 - cfg->t);
+  ap.tc = (float)cfg->t;
+  ap.total_rows = 2 * bt->batch * cfg->n_kv_heads;
+  if (ap.total_rows == 0) return MC_OK;
+  const int blocks = (ap.total_rows + 7) / 8;
+  if (cfg->dtype == MC_F16)
+    append_kernel<MC_F16><<<blocks, 128, 0, stream>>>(ap);
+  else
+    append_kernel<MC_BF16><<<blocks, 128, 0, stream>>>(ap);
+  MC_CUDA_CHECK(cudaGetLastError());
+  return MC_OK;
+}
+
+}  // namespace mc

@@ -1,0 +1,295 @@
+"""Shared test plumbing: builds a seeded problem, runs the CUDA path through the C ABI, runs the
+fp64 oracle on the same bits and compares the two.  Used by the gpu-marked tests and by the
+smoke check.  The oracle side only ever sees generator output and, for the stage-wise checks,
+buffers read back from the device; no expected value is stored from the CUDA path."""
+from __future__ import annotations
+
+import math
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+import gen
+from gen import WorkloadConfig, as_bits
+from oracle import minicache_oracle as orc
+
+ULP_REL = {"f16": 2.0 ** -10, "bf16": 2.0 ** -7}  # spacing of neighbouring values relative to the value
+
+
+class Problem:
+    """One layer pair of a workload, paged on the device, plus the logical host copies."""
+
+    def __init__(self, cfg: WorkloadConfig, pair: int = 0, device="cuda", seq_lens=None, gamma=None, t=None,
+                 retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
+                 tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None):
+        import paper_2405_14366_b200 as mc
+        self.mc = mc
+        self.lib = mc.lib()
+        self.wl = cfg
+        self.device = device
+        self.dtype = cfg.dtype
+        self.t = cfg.t if t is None else t
+        self.gamma = cfg.gamma if gamma is None else gamma
+        self.ps = cfg.page_size if page_size is None else page_size
+        self.H, self.Hq = cfg.n_kv_heads, cfg.n_q_heads
+        if tensors is None:
+            tensors = gen.make_pair_tensors(cfg, pair, device="cpu")
+        self.logical = {k: v for k, v in tensors.items() if k in ("k_lm1", "k_l", "v_lm1", "v_l")}
+        B, S = self.logical["k_l"].shape[:2]
+        self.B, self.S = B, S
+        if seq_lens is None:
+            seq_lens = np.full(B, S, np.int32)
+        self.seq_lens_host = np.asarray(seq_lens, np.int32)
+        cap = self.seq_lens_host + decode_room
+        bt, n_pages = gen.make_block_table(np.maximum(cap, 1), self.ps, seed=1234 + cfg.index)
+        self.n_pages = n_pages
+        self.block_table = torch.from_numpy(bt).to(device)
+        self.seq_lens = torch.from_numpy(self.seq_lens_host.copy()).to(device)
+        self.max_seq_len = int(self.seq_lens_host.max()) if B else 0
+        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode)
+        self.pools = {}
+        for name, x in self.logical.items():
+            xm = x.clone()
+            for b in range(B):  # rows past a sequence's length never reach the device pools as data
+                xm[b, self.seq_lens_host[b]:] = 0
+            self.pools[name] = gen.to_paged(xm.to(device), self.block_table, self.ps, n_pages)
+        total = int(self.seq_lens_host.sum()) * self.H * 2
+        self.ret_capacity = total if ret_capacity is None else ret_capacity
+        self.pair = mc.PairCache(self.cfg, B, n_pages, self.ret_capacity, device=device)
+        self.bits = {k: as_bits(v) for k, v in self.logical.items()}
+
+    # ------------------------------------------------------------------ device side
+    def batch(self, extra: int = 0):
+        return self.mc.Batch(self.block_table, self.seq_lens, self.max_seq_len + extra, self.n_pages)
+
+    def workspace(self, op: int, n_sets: int = 1, extra: int = 0):
+        n = self.lib.mc_workspace_bytes(self.cfg, self.batch(extra), op, n_sets)
+        return torch.empty(n, dtype=torch.uint8, device=self.device)
+
+    def run_merge(self, do_retention: bool = True):
+        ws = self.workspace(0)
+        self.lib.mc_merge_pair(self.cfg, self.batch(), self.pools["k_lm1"], self.pools["v_lm1"], self.pools["k_l"],
+                               self.pools["v_l"], self.pair, do_retention, ws)
+        torch.cuda.synchronize()
+        return self.lib.mc_read_status(self.pair, check=False)
+
+    def run_restore(self, layer: int):
+        dk = torch.zeros_like(self.pair.e_k)
+        dv = torch.zeros_like(self.pair.e_v)
+        self.lib.mc_restore(self.cfg, self.batch(), self.pair, layer, dk, dv)
+        torch.cuda.synchronize()
+        return dk, dv
+
+    def run_attn(self, layer_sel: int, q: torch.Tensor, k_new=None, v_new=None, want_lse=True):
+        n_sets = 2 if layer_sel == 2 else 1
+        out = torch.zeros(n_sets, self.B, self.Hq, 128, dtype=self.cfg.torch_dtype, device=self.device)
+        lse = torch.zeros(n_sets, self.B, self.Hq, dtype=torch.float32, device=self.device) if want_lse else None
+        ws = self.workspace(1, n_sets)
+        self.lib.mc_decode_attn(self.cfg, self.batch(), self.pair, layer_sel, q, k_new, v_new,
+                                1.0 / math.sqrt(128.0), out, lse, ws)
+        torch.cuda.synchronize()
+        return out, lse
+
+    # ------------------------------------------------------------------ read-back helpers
+    def logical_of(self, pool: torch.Tensor, seq_len: Optional[int] = None) -> torch.Tensor:
+        return gen.from_paged(pool, self.block_table, self.S if seq_len is None else seq_len).cpu()
+
+    def device_cache(self, extra_tokens: int = 0) -> Dict[str, np.ndarray]:
+        """The compressed pair read back into logical numpy arrays."""
+        S = self.S + extra_tokens
+        pc = self.pair
+        out = {"e_k": as_bits(self.logical_of(pc.e_k, S)), "e_v": as_bits(self.logical_of(pc.e_v, S))}
+        sc = gen.from_paged(pc.scale.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()  # [B][S][H][4]
+        ds = gen.from_paged(pc.dist.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()   # [B][S][H][2]
+        out["scale"], out["dist"] = sc.astype(np.float64), ds.astype(np.float64)
+        out["ret_count"] = pc.ret_count.cpu().numpy().reshape(2, self.B, self.H)
+        out["ret_offset"] = pc.ret_offset.cpu().numpy()
+        out["ret_index"] = pc.ret_index.cpu().numpy()
+        out["ret_rows"] = as_bits(pc.ret_rows.cpu())
+        out["seg_minmax"] = pc.seg_minmax.cpu().numpy().reshape(2, self.B, self.H, 2).astype(np.float64)
+        return out
+
+    def retained(self, dc, tensor: int, b: int, h: int):
+        seg = (tensor * self.B + b) * self.H + h
+        off, cnt = int(dc["ret_offset"][seg]), int(dc["ret_count"][tensor, b, h])
+        return dc["ret_index"][off:off + cnt].astype(np.int64), dc["ret_rows"][off:off + cnt]
+
+    # ------------------------------------------------------------------ oracle side
+    def oracle_merge(self, mode: str = "distinct", do_retention: bool = True):
+        out = {}
+        for ti, tn in enumerate(("k", "v")):
+            out[tn] = orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype,
+                                     self.t, self.gamma, mode=mode, do_retention=do_retention)
+        return out
+
+
+def _mask_valid(p: Problem):
+    m = np.zeros((p.B, p.S), bool)
+    for b in range(p.B):
+        m[b, :p.seq_lens_host[b]] = True
+    return m
+
+
+def compare_merge(p: Problem, om, dc, mode: str = "distinct", do_retention: bool = True) -> Dict[str, float]:
+    """Element-by-element comparison of the merge outputs.  Returns statistics; asserts the bars."""
+    stats: Dict[str, float] = {}
+    valid = _mask_valid(p)
+    ulp = ULP_REL[p.dtype]
+    for ti, tn in enumerate(("k", "v")):
+        o = om[tn]
+        e_gpu = orc.decode_bits(dc["e_" + tn], p.dtype)
+        e_orc = orc.decode_bits(o["e_bits"], p.dtype)
+        vm = valid[:, :, None, None]
+        # stored directions: identical codes, except elements whose unrounded value sits on a rounding
+        # boundary (fp32 vs fp64 arithmetic lands on different sides): at most one unit in the last place
+        diff = np.abs(e_gpu - e_orc) * vm
+        flips = (dc["e_" + tn] != o["e_bits"]) & np.broadcast_to(vm, diff.shape)
+        nflip = int(flips.sum())
+        if nflip:
+            spacing = np.maximum(np.abs(e_orc), 2.0 ** -14) * ulp * 1.01
+            assert np.all(diff[flips] <= spacing[flips]), "direction differs by more than one ulp"
+            # ... and the oracle's unrounded value is close to the midpoint between the two codes
+            mid_dist = np.abs(np.abs(o["e"] - e_orc) - 0.5 * np.abs(e_gpu - e_orc))
+            assert np.all(mid_dist[flips] <= 3e-7), "flip not at a rounding boundary"
+        total = int(valid.sum()) * p.H * 128
+        stats[f"{tn}_flip_frac"] = nflip / max(total, 1)
+        assert nflip <= max(8, 5e-3 * total), f"too many rounding flips: {nflip}/{total}"
+        # scales: |x| / |e_stored| with the oracle's own stored direction
+        len_e = np.sqrt(np.sum(e_orc * e_orc, -1))
+        len_e = np.where(len_e == 0, 1.0, len_e)
+        row_flip = flips.any(-1)
+        for li, nm in enumerate(("n_lm1", "n_l")):
+            want = o[nm] / len_e
+            got = dc["scale"][..., ti * 2 + li]
+            rel = np.abs(got - want) / np.maximum(np.abs(want), 1e-30) * valid[:, :, None]
+            clean = rel * ~row_flip
+            stats[f"{tn}_scale_rel"] = max(stats.get(f"{tn}_scale_rel", 0.0), float(clean.max(initial=0.0)))
+            assert clean.max(initial=0.0) < 2e-6, f"scale mismatch {clean.max()}"
+            assert rel.max(initial=0.0) < 4 * ulp, "scale of a row with a rounding flip is off"
+        # distances
+        dd = np.abs(dc["dist"][..., ti] - o["d"]) * valid[:, :, None]
+        stats[f"{tn}_dist_abs"] = float(dd.max(initial=0.0))
+        assert dd.max(initial=0.0) < 5e-7, f"distance mismatch {dd.max()}"
+        # retention sets
+        near = 0
+        mism = 0
+        for b in range(p.B):
+            n = int(p.seq_lens_host[b])
+            for h in range(p.H):
+                want = o["retained"][(b, h)]
+                got, rows = p.retained(dc, ti, b, h)
+                assert np.all(np.diff(got) > 0), "retained indices not ascending"
+                if n == 0:
+                    assert len(got) == 0
+                    continue
+                d = o["d"][b, :n, h]
+                if not do_retention:
+                    assert len(got) == 0
+                    continue
+                mm = dc["seg_minmax"][ti, b, h]
+                assert abs(mm[0] - d.min()) < 5e-7 and abs(mm[1] - d.max()) < 5e-7
+                thr = orc.retention_threshold(d, p.gamma, mode)
+                sym = np.setxor1d(want, got)
+                # exact, except tokens whose distance lies within 1e-6 of the threshold
+                assert np.all(np.abs(d[sym] - thr) < 1e-6), f"retained set differs away from the threshold: {sym}"
+                mism += len(sym)
+                near += int(np.sum(np.abs(d - thr) < 1e-6))
+                # raw rows are bit copies of both layers' inputs
+                assert np.array_equal(rows[:, 0], p.bits[tn + "_lm1"][b, got, h])
+                assert np.array_equal(rows[:, 1], p.bits[tn + "_l"][b, got, h])
+        stats[f"{tn}_near_threshold"] = near
+        stats[f"{tn}_set_mismatch"] = mism
+    return stats
+
+
+def oracle_restore_from_device(p: Problem, dc, layer: int, tensor: str, b: int, h: int, n: Optional[int] = None):
+    """Oracle restore fed with the device's compressed cache (stage-wise check)."""
+    ti = 0 if tensor == "k" else 1
+    n = int(p.seq_lens_host[b]) if n is None else n
+    e_bits = dc["e_" + tensor][b, :n, h]
+    e = orc.decode_bits(e_bits, p.dtype)
+    norms = dc["scale"][b, :n, h, ti * 2 + layer] * np.sqrt(np.sum(e * e, -1))
+    idx, rows = p.retained(dc, ti, b, h)
+    return orc.restore(e_bits, norms, p.dtype, idx, rows[:, layer] if len(idx) else None)
+
+
+def compare_restore(p: Problem, om, dc, layer: int, dk: torch.Tensor, dv: torch.Tensor) -> Dict[str, float]:
+    stats = {}
+    lname = ("n_lm1", "n_l")[layer]
+    src = ("_lm1", "_l")[layer]
+    for ti, (tn, pool) in enumerate((("k", dk), ("v", dv))):
+        got = orc.decode_bits(as_bits(p.logical_of(pool)), p.dtype)
+        o = om[tn]
+        err_e2e, ref_max, err_stage = 0.0, 0.0, 0.0
+        for b in range(p.B):
+            n = int(p.seq_lens_host[b])
+            for h in range(p.H):
+                idx = o["retained"][(b, h)]
+                want = orc.restore(o["e_bits"][b, :n, h], o[lname][b, :n, h], p.dtype, idx,
+                                   p.bits[tn + src][b, idx, h] if len(idx) else None)
+                g = got[b, :n, h]
+                didx, _ = p.retained(dc, ti, b, h)
+                same_set = np.setdiff1d(np.arange(n), np.setxor1d(idx, didx))  # rows both sides treat alike
+                flips = (dc["e_" + tn][b, :n, h] != o["e_bits"][b, :n, h])
+                dif = np.abs(g - want)
+                dif[flips] = 0.0  # one-ulp rounding flips of the stored direction are counted in compare_merge
+                err_e2e = max(err_e2e, float(dif[same_set].max(initial=0.0)))
+                ref_max = max(ref_max, float(np.abs(want).max(initial=0.0)))
+                # retained rows come back bit-exactly
+                if len(didx):
+                    assert np.array_equal(as_bits(p.logical_of(pool))[b, didx, h], p.bits[tn + src][b, didx, h])
+                # stage-wise: oracle restore of the device's own cache; only the final 16-bit rounding differs
+                want2 = oracle_restore_from_device(p, dc, layer, tn, b, h)
+                # (0.505 ulp of the value, plus half the subnormal spacing of binary16)
+                bound = 0.505 * ULP_REL[p.dtype] * np.abs(want2) + 3.1e-8
+                err_stage = max(err_stage, float((np.abs(g - want2) / bound).max(initial=0.0)))
+        rel = err_e2e / max(ref_max, 1e-30)
+        stats[f"{tn}_restore_rel"] = rel
+        stats[f"{tn}_restore_stage"] = err_stage
+        assert rel < 2e-3, f"restored {tn} off by {rel} (max-abs relative)"
+        assert err_stage <= 1.0, f"restore of the device cache off by {err_stage} rounding bounds"
+    return stats
+
+
+def oracle_attention(p: Problem, om, layer: int, q_bits, b: int, hq: int, k_new_bits=None, v_new_bits=None):
+    g = hq // (p.Hq // p.H)
+    n = int(p.seq_lens_host[b])
+    lname = ("n_lm1", "n_l")[layer]
+    src = ("_lm1", "_l")[layer]
+    ik, iv = om["k"]["retained"][(b, g)], om["v"]["retained"][(b, g)]
+    return orc.decode_attention(
+        q_bits, om["k"]["e_bits"][b, :n, g], om["v"]["e_bits"][b, :n, g], om["k"][lname][b, :n, g],
+        om["v"][lname][b, :n, g], p.dtype, 1.0 / math.sqrt(128.0),
+        idx_k=ik, rows_k_bits=p.bits["k" + src][b, ik, g] if len(ik) else None,
+        idx_v=iv, rows_v_bits=p.bits["v" + src][b, iv, g] if len(iv) else None,
+        k_new_bits=k_new_bits, v_new_bits=v_new_bits)
+
+
+def compare_attention(p: Problem, om, layer_sel: int, q: torch.Tensor, out: torch.Tensor, lse, k_new=None, v_new=None,
+                      sample=None) -> Dict[str, float]:
+    """out [n_sets][B][Hq][128] against the oracle (restore + dense attention in fp64)."""
+    qb = as_bits(q)
+    ob = orc.decode_bits(as_bits(out), p.dtype)
+    knb = as_bits(k_new) if k_new is not None else None
+    vnb = as_bits(v_new) if v_new is not None else None
+    layers = (0, 1) if layer_sel == 2 else (layer_sel,)
+    err, lerr = 0.0, 0.0
+    nq = p.Hq // p.H
+    items = [(b, h) for b in range(p.B) for h in range(p.Hq)] if sample is None else sample
+    for si, layer in enumerate(layers):
+        for b, hq in items:
+            g = hq // nq
+            kn = knb[si, b, g] if knb is not None else None
+            vn = vnb[si, b, g] if vnb is not None else None
+            n = int(p.seq_lens_host[b])
+            if n == 0 and kn is None:
+                assert np.all(ob[si, b, hq] == 0)
+                continue
+            o, l = oracle_attention(p, om, layer, qb[si, b, hq], b, hq, kn, vn)
+            err = max(err, float(np.abs(ob[si, b, hq] - o).max()))
+            if lse is not None:
+                lerr = max(lerr, abs(float(lse[si, b, hq]) - l))
+    assert err < 1e-2, f"attention output off by {err} (max-abs)"
+    assert lerr < 1e-3, f"log-sum-exp off by {lerr}"
+    return {"attn_abs": err, "lse_abs": lerr}

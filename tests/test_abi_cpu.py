@@ -1,0 +1,118 @@
+"""Host-only checks of the C ABI: the library loads, exports what the header declares, and
+rejects bad arguments before touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2405_14366_b200 as mc
+from paper_2405_14366_b200 import binding as B
+from paper_2405_14366_b200.build import build_library
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_library()
+    return mc.lib()
+
+
+def test_exports_match_header(lib, repo_root):
+    text = open(os.path.join(repo_root, "include", "minicache.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(mc_[a-z_]+)\s*\(", text))
+    assert declared, "no declarations found"
+    for name in declared:
+        assert lib.has_symbol(name), f"{name} declared in minicache.h but not exported"
+    assert set(B.EXPORTS) <= declared | {"mc_version"}
+    assert lib.mc_version() >= 100
+
+
+def test_status_strings(lib):
+    assert lib.mc_status_str(0) == "MC_OK"
+    assert lib.mc_status_str(5) == "MC_ERR_CAPACITY"
+    assert lib.mc_status_str(99) == "MC_ERR_UNKNOWN"
+
+
+def _cfg(**kw):
+    d = dict(n_kv_heads=8, n_q_heads=32, head_dim=128, page_size=16, dtype=0, retain_mode=0, t=0.6, gamma=0.05)
+    d.update(kw)
+    return B._Config(d["n_kv_heads"], d["n_q_heads"], d["head_dim"], d["page_size"], d["dtype"], d["retain_mode"],
+                     d["t"], d["gamma"])
+
+
+def _batch(batch=2, mpps=4, max_len=64, n_pages=10, bt=0x1000, sl=0x2000):
+    return B._Batch(bt, sl, batch, mpps, max_len, 0, n_pages)
+
+
+def test_workspace_bytes_is_host_arithmetic(lib):
+    out = C.c_size_t(0)
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b), 0, 1, C.byref(out)) == 0 and out.value % 256 == 0 and out.value > 0
+    m = out.value
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b), 1, 2, C.byref(out)) == 0 and out.value % 256 == 0
+    b2 = _batch(max_len=64 * 1024, mpps=4096)
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b2), 0, 1, C.byref(out)) == 0 and out.value > m
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b), 7, 1, C.byref(out)) == 1
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b), 1, 3, C.byref(out)) == 1
+    assert L.mc_workspace_bytes(None, C.byref(b), 0, 1, C.byref(out)) == 1
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(head_dim=64), 2), (dict(page_size=8), 2), (dict(n_q_heads=12), 2), (dict(n_q_heads=24), 2),
+    (dict(dtype=5), 3), (dict(retain_mode=9), 1), (dict(t=1.5), 1), (dict(gamma=-0.1), 1),
+])
+def test_bad_config_rejected(lib, kw, code):
+    out = C.c_size_t(0)
+    c, b = _cfg(**kw), _batch()
+    assert lib._lib.mc_workspace_bytes(C.byref(c), C.byref(b), 0, 1, C.byref(out)) == code
+
+
+def test_merge_rejects_bad_arguments_without_launching(lib):
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    a = B._LayerKV(0x10000, 0x20000)
+    pc = B._PairCache(0x30000, 0x40000, 0x50000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    ws = 0x100000
+    # null layer pool
+    bad = B._LayerKV(0, 0x20000)
+    assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(bad), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 1
+    # misaligned pool
+    mis = B._LayerKV(0x10010, 0x20000)
+    assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(mis), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 4
+    # workspace too small
+    assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 16, None) == 5
+    # block table narrower than max_seq_len
+    b2 = _batch(mpps=2, max_len=64)
+    assert L.mc_merge_pair(C.byref(c), C.byref(b2), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 2
+    # top-k retention is not built on the device
+    ck = _cfg(retain_mode=2)
+    assert L.mc_merge_pair(C.byref(ck), C.byref(b), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 6
+    # pair cache with a missing buffer
+    pc2 = B._PairCache(0x30000, 0, 0x50000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(a), C.byref(pc2), 1, ws, 1 << 20, None) == 1
+
+
+def test_attn_and_restore_reject_bad_arguments(lib):
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    pc = B._PairCache(0x30000, 0x40000, 0x50000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    d = B._LayerKV(0x10000, 0x20000)
+    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 2, C.byref(d), None) == 1  # BOTH is not a restore target
+    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 0, None, None) == 1
+    ws = 0x100000
+    # pair mode with 4 query heads per kv head needs 8 rows: allowed; with 8 per kv head it does not fit
+    c8 = _cfg(n_kv_heads=4, n_q_heads=32)
+    assert L.mc_decode_attn(C.byref(c8), C.byref(b), C.byref(pc), 2, 0x1000, None, None, 1.0, 0x2000, None, ws, 1 << 24, None) == 2
+    # k_new without v_new
+    assert L.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), 0, 0x1000, 0x3000, None, 1.0, 0x2000, None, ws, 1 << 24, None) == 1
+    # null q
+    assert L.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), 0, None, None, None, 1.0, 0x2000, None, ws, 1 << 24, None) == 1
+    # workspace too small
+    assert L.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), 0, 0x1000, None, None, 1.0, 0x2000, None, ws, 8, None) == 5
+
+
+def test_binding_fails_loudly_without_library(tmp_path):
+    with pytest.raises(mc.McError):
+        B.MiniCacheLib(str(tmp_path / "nope.so"))

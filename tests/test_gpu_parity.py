@@ -1,0 +1,200 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle on the same seeded bits.
+
+Bars: retained sets exact except tokens within 1e-6 of the threshold; restored K/V within 2e-3
+max-abs relative; attention output within 1e-2 max-abs; integer/bit work (indices, raw rows) exact."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+from gen import CONFIGS
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2405_14366_b200.build import build_library
+    build_library()
+    import mc_harness
+    return mc_harness
+
+
+def _full_cycle(H, p, mode="distinct", do_retention=True, new_token=True, pair_mode=True, steps_q=1):
+    words, code = p.run_merge(do_retention)
+    assert code == 0, words
+    om = p.oracle_merge(mode, do_retention)
+    dc = p.device_cache()
+    stats = H.compare_merge(p, om, dc, mode, do_retention)
+    for layer in (0, 1):
+        dk, dv = p.run_restore(layer)
+        stats.update({f"l{layer}_{k}": v for k, v in H.compare_restore(p, om, dc, layer, dk, dv).items()})
+    wl = dataclasses.replace(p.wl, batch=p.B)
+    q = gen.make_queries(wl, 0, device="cpu", n_sets=2).to(p.device)
+    nt = gen.make_new_tokens(wl, 0, 0, device="cpu")
+    for layer in (0, 1):
+        out, lse = p.run_attn(layer, q[layer:layer + 1].contiguous())
+        stats.update({f"a{layer}_{k}": v for k, v in
+                      H.compare_attention(p, om, layer, q[layer:layer + 1].cpu(), out.cpu(), lse.cpu()).items()})
+    if new_token:
+        kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()  # [2][B][H][128]
+        vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+        out, lse = p.run_attn(1, q[1:2].contiguous(), kn[1:2].contiguous().to(p.device), vn[1:2].contiguous().to(p.device))
+        stats.update({f"anew_{k}": v for k, v in
+                      H.compare_attention(p, om, 1, q[1:2].cpu(), out.cpu(), lse.cpu(), kn[1:2], vn[1:2]).items()})
+        if pair_mode and 2 * (p.Hq // p.H) <= 8:
+            out, lse = p.run_attn(2, q.contiguous(), kn.to(p.device), vn.to(p.device))
+            stats.update({f"apair_{k}": v for k, v in
+                          H.compare_attention(p, om, 2, q.cpu(), out.cpu(), lse.cpu(), kn, vn).items()})
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 0, words
+    return stats
+
+
+def test_config1_full_parity(H):
+    """Single pair, 32 heads x 128, batch 1, 512 tokens, fp16: every output element compared."""
+    p = H.Problem(CONFIGS["c1"])
+    stats = _full_cycle(H, p)
+    print(stats)
+    # the planted outliers (3 % of tokens, large angles) are what retention keeps
+    dc = p.device_cache()
+    kept = dc["ret_count"].sum() / (2 * 512 * 32)
+    assert 0.002 < kept < 0.06
+
+
+@pytest.mark.parametrize("n", [1, 2, 15, 16, 17, 33, 100])
+@pytest.mark.parametrize("dtype,hkv,hq,ps", [("f16", 2, 2, 16), ("bf16", 2, 8, 16), ("f16", 1, 2, 32), ("bf16", 2, 4, 64)])
+def test_tiny_shapes(H, n, dtype, hkv, hq, ps):
+    wl = CONFIGS["c1"].scaled("tiny", n_kv_heads=hkv, n_q_heads=hq, dtype=dtype, batch=3, seq_len=n, page_size=ps,
+                              outlier_frac=0.15, index=40 + n)
+    lens = np.array([n, max(1, n // 2), max(1, n - 1)], np.int32)
+    p = H.Problem(wl, seq_lens=lens, gamma=0.1)
+    _full_cycle(H, p)
+
+
+@pytest.mark.parametrize("gamma,mode", [(0.0, "distinct"), (1.0, "distinct"), (0.2, "distinct"), (0.05, "literal"), (0.5, "literal")])
+def test_retention_modes(H, gamma, mode):
+    wl = CONFIGS["c1"].scaled("ret", n_kv_heads=4, n_q_heads=4, batch=2, seq_len=300, outlier_frac=0.05, index=77)
+    p = H.Problem(wl, gamma=gamma, retain_mode={"distinct": 0, "literal": 1}[mode], seq_lens=[300, 211])
+    stats = _full_cycle(H, p, mode=mode)
+    dc = p.device_cache()
+    if gamma == 0.0:
+        assert dc["ret_count"].sum() == 0  # gamma = 0: everything merged
+    if gamma == 1.0 and mode == "distinct":
+        assert dc["ret_count"].sum() >= 2 * 4 * (300 + 211) - 2 * 2 * 4  # all but the least distinct token(s)
+
+
+def test_no_retention_flag(H):
+    wl = CONFIGS["c1"].scaled("noret", n_kv_heads=4, n_q_heads=4, batch=1, seq_len=130, index=78)
+    p = H.Problem(wl)
+    _full_cycle(H, p, do_retention=False)
+    assert p.device_cache()["ret_count"].sum() == 0
+
+
+def test_degenerate_rows(H):
+    """Identical, antipodal and zero rows (the cases Eq. 3 leaves undefined) and t at both ends."""
+    wl = CONFIGS["c1"].scaled("deg", n_kv_heads=2, n_q_heads=2, batch=1, seq_len=48, index=79)
+    t = gen.make_pair_tensors(wl, 0)
+    for name in ("k", "v"):
+        a, c = t[name + "_lm1"], t[name + "_l"]
+        a[0, 0:4] = c[0, 0:4]                 # identical rows: d = 0, passthrough
+        a[0, 4:8] = -2 * c[0, 4:8]            # antipodal
+        a[0, 8:10] = 0                        # zero row in layer l-1
+        c[0, 10:12] = 0                       # zero row in layer l
+        a[0, 12] = 0
+        c[0, 12] = 0                          # both zero
+    for tt in (0.6, 0.4, 0.0, 1.0):
+        p = H.Problem(wl, tensors=t, t=tt, gamma=0.3)
+        _full_cycle(H, p, new_token=False)
+        dc = p.device_cache()
+        assert np.all(dc["dist"][0, 0:4] < 1e-6) and np.all(np.abs(dc["dist"][0, 4:8] - 1) < 1e-6)
+        assert np.all(np.isfinite(dc["scale"][0, :48])) and np.all(dc["dist"][0, 8:13] == 0)
+        dk, dv = p.run_restore(1)
+        x = p.logical_of(dk)
+        assert torch.all(x[0, 10:13] == 0) and torch.all(torch.isfinite(x.float()))
+
+
+def test_retained_pool_overflow_is_reported(H):
+    wl = CONFIGS["c1"].scaled("ovf", n_kv_heads=2, n_q_heads=2, batch=2, seq_len=200, outlier_frac=0.1, index=80)
+    p = H.Problem(wl, gamma=0.5, ret_capacity=3)
+    words, code = p.run_merge()
+    assert code == 5 and (words[0] & 1) and words[1] > 3
+    dc = p.device_cache()
+    assert dc["ret_count"].sum() == 0  # nothing half-written: the pair falls back to "everything merged"
+    om = p.oracle_merge(do_retention=False)
+    H.compare_merge(p, om, dc, do_retention=False)
+
+
+def test_append_then_attend(H):
+    """Decode steps: attend with the new raw token, merge-append it, attend again over n + 1."""
+    wl = CONFIGS["c1"].scaled("app", n_kv_heads=4, n_q_heads=8, dtype="bf16", batch=3, seq_len=61, index=81)
+    lens = np.array([61, 16, 31], np.int32)
+    p = H.Problem(wl, seq_lens=lens, decode_room=8)
+    words, code = p.run_merge()
+    assert code == 0
+    om = p.oracle_merge()
+    import mc_harness as M
+    from oracle import minicache_oracle as orc
+    for step in range(3):
+        nt = gen.make_new_tokens(dataclasses.replace(wl, batch=3), 0, step)
+        dev = {k: v[:, 0].contiguous().to(p.device) for k, v in nt.items()}
+        p.lib.mc_append_pair(p.cfg, p.batch(), p.pair, dev["k_lm1"], dev["v_lm1"], dev["k_l"], dev["v_l"])
+        torch.cuda.synchronize()
+        # oracle: append to its own logical cache
+        for tn in ("k", "v"):
+            m = orc.append_rows(gen.as_bits(nt[tn + "_lm1"][:, 0]), gen.as_bits(nt[tn + "_l"][:, 0]), p.dtype, p.t)
+            o = om[tn]
+            if o["e_bits"].shape[1] < p.S + step + 1:
+                padn = p.S + 8 - o["e_bits"].shape[1]
+                for key in ("e_bits", "n_lm1", "n_l", "d"):
+                    shp = list(o[key].shape)
+                    shp[1] = padn
+                    o[key] = np.concatenate([o[key], np.zeros(shp, o[key].dtype)], axis=1)
+            for b in range(3):
+                pos = int(p.seq_lens_host[b])
+                o["e_bits"][b, pos] = m["e_bits"][b]
+                o["n_lm1"][b, pos] = m["n_a"][b]
+                o["n_l"][b, pos] = m["n_c"][b]
+        p.seq_lens_host = p.seq_lens_host + 1
+        p.seq_lens += 1
+        p.max_seq_len += 1
+        q = gen.make_queries(dataclasses.replace(wl, batch=3), 10 + step, n_sets=1)
+        out, lse = p.run_attn(0, q.to(p.device))
+        M.compare_attention(p, om, 0, q, out.cpu(), lse.cpu())
+    # appended directions equal the oracle's (up to boundary flips) and carry no retention decision
+    dc = p.device_cache(extra_tokens=3)
+    for b in range(3):
+        n = int(p.seq_lens_host[b])
+        e_gpu = orc.decode_bits(dc["e_k"][b, n - 3:n], p.dtype)
+        e_orc = orc.decode_bits(om["k"]["e_bits"][b, n - 3:n], p.dtype)
+        assert np.max(np.abs(e_gpu - e_orc)) <= 2.0 ** -7 * 0.51
+    assert dc["ret_count"].sum() == sum(len(v) for v in om["k"]["retained"].values()) + sum(len(v) for v in om["v"]["retained"].values())
+
+
+@pytest.mark.parametrize("name", ["c2_s", "c3_s", "c5_s"])
+def test_scaled_configs_sampled(H, name):
+    """1/16-scale replicas of the throughput configs: merge compared on every row, restore on
+    every row, attention on a seeded sample of (sequence, head) items spanning several splits."""
+    wl = CONFIGS[name]
+    pair = wl.n_pairs - 1
+    p = H.Problem(wl, pair=pair)
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge()
+    dc = p.device_cache()
+    stats = H.compare_merge(p, om, dc)
+    dk, dv = p.run_restore(1)
+    stats.update(H.compare_restore(p, om, dc, 1, dk, dv))
+    rs = np.random.RandomState(5)
+    sample = [(int(rs.randint(p.B)), int(rs.randint(p.Hq))) for _ in range(6)]
+    q = gen.make_queries(dataclasses.replace(wl, batch=p.B), 0, n_sets=2)
+    for sel in ((0, 1, 2) if 2 * (p.Hq // p.H) <= 8 else (0, 1)):
+        qq = q if sel == 2 else q[sel:sel + 1].contiguous()
+        out, lse = p.run_attn(sel, qq.to(p.device))
+        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample))
+    print(name, stats)
