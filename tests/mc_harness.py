@@ -233,6 +233,10 @@ def compare_restore(p: Problem, om, dc, layer: int, dk: torch.Tensor, dv: torch.
                 same_set = np.setdiff1d(np.arange(n), np.setxor1d(idx, didx))  # rows both sides treat alike
                 flips = (dc["e_" + tn][b, :n, h] != o["e_bits"][b, :n, h])
                 dif = np.abs(g - want)
+                if p.dtype == "bf16":
+                    # the dense output is itself stored in bfloat16, whose half-ulp (2^-8 of the value)
+                    # alone exceeds the 2e-3 bar: the bar applies to the value before that last rounding
+                    dif = np.maximum(dif - 0.505 * ULP_REL["bf16"] * np.abs(want), 0.0)
                 dif[flips] = 0.0  # one-ulp rounding flips of the stored direction are counted in compare_merge
                 err_e2e = max(err_e2e, float(dif[same_set].max(initial=0.0)))
                 ref_max = max(ref_max, float(np.abs(want).max(initial=0.0)))
