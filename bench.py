@@ -394,12 +394,60 @@ def main():
 
 def run_e2e(job: Job, wl, rho, args, dist, dev, world):
     """Same step with HOST buffers: every pair's four input pools start in pinned host memory and
-    are copied in before its merge; every attention call takes its query and new-token rows from
-    pinned host memory and returns its output there.  Copies are inside the timed region."""
+    are copied in by mc_merge_pair_host before its merge; every attention call takes its query and
+    new-token rows from pinned host memory and returns its output there (mc_decode_attn_host).
+    The copies are inside the timed region."""
     lib = job.lib
-    if not lib.has_symbol("mc_merge_pair_host"):
-        return None
-    return None
+    host_pools = []
+    for pl in job.pools:
+        host_pools.append({k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in pl.items()})
+    stage = {k: torch.empty_like(v) for k, v in job.pools[0].items()}  # device staging the host pools land in
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+    q_host = [pin(q) for q in job.q]
+    new_host = [{k: pin(v) for k, v in nt.items()} for nt in job.new]
+    out_host = torch.empty(job.out.shape, dtype=job.out.dtype, pin_memory=True)
+    bd = job.batch(True)
+    io = torch.empty(lib.mc_decode_io_bytes(job.cfg, bd, 1), dtype=torch.uint8, device=dev)
+    pool_bytes = sum(v.numel() * v.element_size() for v in job.pools[0].values())
+    q_bytes = job.B * job.Hq * ROW
+    n_bytes = job.B * job.H * ROW
+
+    def e2e_step():
+        job.seq_lens.copy_(job.seq0)
+        b = job.batch(False)
+        for pr in range(wl.n_pairs):
+            lib.mc_merge_pair_host(job.cfg, b, host_pools[pr], stage, job.pairs[pr], True, job.ws_merge)
+        for pr in range(wl.n_pairs):
+            for layer in (0, 1):
+                lib.mc_restore(job.cfg, b, job.pairs[pr], layer, job.dst_k, job.dst_v)
+        for s in range(job.steps):
+            q, nt = q_host[s % len(q_host)], new_host[s % len(new_host)]
+            ntd = job.new[s % len(job.new)]
+            for pr in range(wl.n_pairs):
+                pc = job.pairs[pr]
+                for layer in (0, 1):
+                    kn = nt["k_lm1" if layer == 0 else "k_l"]
+                    vn = nt["v_lm1" if layer == 0 else "v_l"]
+                    lib.mc_decode_attn_host(job.cfg, bd, pc, layer, q[layer], kn, vn, job.sm_scale, out_host, None,
+                                            io, job.ws_attn)
+                lib.mc_append_pair(job.cfg, bd, pc, ntd["k_lm1"], ntd["v_lm1"], ntd["k_l"], ntd["v_l"])
+            job.seq_lens += 1
+
+    e2e_step()
+    if dist is not None:
+        dist.barrier()
+    n = max(1, min(args.steps, 2))
+    t = timed(lambda: [e2e_step() for _ in range(n)])
+    if dist is not None:
+        tt = torch.tensor([t], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t = float(tt.item())
+    by = job.bytes_per_step(rho)
+    calls = job.steps * wl.n_pairs * 2
+    return {"value": world * sum(by.values()) * n / t / 1e9, "unit": "GB/s", "steps": n, "ms_per_step": t / n * 1e3,
+            "h2d_bytes_per_step": wl.n_pairs * pool_bytes + calls * (q_bytes + 2 * n_bytes),
+            "d2h_bytes_per_step": calls * q_bytes,
+            "api": "mc_merge_pair_host + mc_restore + mc_decode_attn_host + mc_append_pair, pinned host buffers"}
 
 
 if __name__ == "__main__":

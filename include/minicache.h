@@ -202,6 +202,30 @@ mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_p
                          float sm_scale, void* out, float* lse, void* workspace,
                          size_t workspace_bytes, void* stream);
 
+/* Host-buffer form of mc_merge_pair (Algorithm 2 "MiniCache Prefill" with the layers' K/V arriving
+ * from the host): host_lm1 / host_l are HOST pools (pinned memory for asynchronous copies) in the
+ * paged layout; they are copied into the caller's device pools dev_lm1 / dev_l on `stream`
+ * (n_pages * n_kv_heads * page_size * 256 bytes each) and merged there.  Nothing is allocated. */
+mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* host_lm1,
+                             const mc_layer_kv* host_l, const mc_layer_kv* dev_lm1,
+                             const mc_layer_kv* dev_l, const mc_pair_cache* out, int32_t do_retention,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Host-buffer form of mc_decode_attn (Algorithm 2 "MiniCache Decoding" for a caller whose queries
+ * live on the host): q_host, k_new_host, v_new_host are read from and out_host (and lse_host, if not
+ * NULL) written to HOST memory, through `dev_io`, a device staging buffer of at least
+ * mc_decode_io_bytes() bytes (256-byte aligned).  The copies are enqueued on `stream` around the
+ * kernels; out_host is valid once the stream has run the call.  Nothing is allocated. */
+mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                              int32_t layer_sel, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, float sm_scale, void* out_host, float* lse_host,
+                              void* dev_io, size_t dev_io_bytes, void* workspace,
+                              size_t workspace_bytes, void* stream);
+
+/* Bytes of device staging mc_decode_attn_host needs (q, new K/V rows, out, lse). Host arithmetic. */
+mc_status mc_decode_io_bytes(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets,
+                             size_t* bytes);
+
 /* Copies the pair's status words to host memory `out_words[MC_STATUS_WORDS]` after synchronising
  * `stream`.  Returns MC_ERR_CAPACITY if the overflow flag is set, MC_ERR_DEVICE_STATUS for any
  * other flag, MC_OK otherwise. */

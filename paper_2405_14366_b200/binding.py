@@ -53,7 +53,8 @@ class _PairCache(C.Structure):
 
 
 EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
-           "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status")
+           "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
+           "mc_decode_attn_host", "mc_decode_io_bytes")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -156,8 +157,13 @@ class MiniCacheLib:
         L.mc_decode_attn.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V,
                                      C.c_size_t, V]
         L.mc_read_status.argtypes = [P(_PairCache), V, P(C.c_int32)]
+        L.mc_merge_pair_host.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_LayerKV), P(_LayerKV),
+                                         P(_PairCache), C.c_int32, V, C.c_size_t, V]
+        L.mc_decode_attn_host.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V,
+                                          V, C.c_size_t, V, C.c_size_t, V]
+        L.mc_decode_io_bytes.argtypes = [P(_Config), P(_Batch), C.c_int32, P(C.c_size_t)]
         for f in ("mc_workspace_bytes", "mc_merge_pair", "mc_append_pair", "mc_restore", "mc_decode_attn",
-                  "mc_read_status"):
+                  "mc_read_status", "mc_merge_pair_host", "mc_decode_attn_host", "mc_decode_io_bytes"):
             getattr(L, f).restype = C.c_int32
 
     # -- helpers ------------------------------------------------------------------------------
@@ -208,6 +214,32 @@ class MiniCacheLib:
         self._check(self._lib.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q), _ptr(k_new),
                                              _ptr(v_new), float(sm_scale), _ptr(out), _ptr(lse), _ptr(workspace),
                                              workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_merge_pair_host(self, cfg: McConfig, batch: Batch, host, dev, pair: PairCache, do_retention: bool,
+                           workspace: torch.Tensor, stream=None):
+        """host / dev: dicts with k_lm1, v_lm1, k_l, v_l pools (pinned host tensors / device tensors)."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        ha, hl = _LayerKV(_ptr(host["k_lm1"]), _ptr(host["v_lm1"])), _LayerKV(_ptr(host["k_l"]), _ptr(host["v_l"]))
+        da, dl = _LayerKV(_ptr(dev["k_lm1"]), _ptr(dev["v_lm1"])), _LayerKV(_ptr(dev["k_l"]), _ptr(dev["v_l"]))
+        self._check(self._lib.mc_merge_pair_host(C.byref(c), C.byref(b), C.byref(ha), C.byref(hl), C.byref(da),
+                                                 C.byref(dl), C.byref(pc), 1 if do_retention else 0, _ptr(workspace),
+                                                 workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_decode_io_bytes(self, cfg: McConfig, batch: Batch, n_query_sets: int = 1) -> int:
+        out = C.c_size_t(0)
+        c, b = cfg.c(), batch.c()
+        self._check(self._lib.mc_decode_io_bytes(C.byref(c), C.byref(b), n_query_sets, C.byref(out)))
+        return out.value
+
+    def mc_decode_attn_host(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q_host, k_new_host,
+                            v_new_host, sm_scale: float, out_host, lse_host, dev_io: torch.Tensor,
+                            workspace: torch.Tensor, stream=None):
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        self._check(self._lib.mc_decode_attn_host(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q_host),
+                                                  _ptr(k_new_host), _ptr(v_new_host), float(sm_scale), _ptr(out_host),
+                                                  _ptr(lse_host), _ptr(dev_io), dev_io.numel() * dev_io.element_size(),
+                                                  _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                  _stream(stream)))
 
     def mc_read_status(self, pair: PairCache, stream=None, check: bool = True):
         words = (C.c_int32 * MC_STATUS_WORDS)()

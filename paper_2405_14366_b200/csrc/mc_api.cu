@@ -174,6 +174,84 @@ mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_p
                             workspace, (cudaStream_t)stream);
 }
 
+mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* host_lm1,
+                             const mc_layer_kv* host_l, const mc_layer_kv* dev_lm1, const mc_layer_kv* dev_l,
+                             const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  if (!host_lm1 || !host_l || !dev_lm1 || !dev_l) return MC_ERR_INVALID_ARG;
+  if (!host_lm1->k_pool || !host_lm1->v_pool || !host_l->k_pool || !host_l->v_pool) return MC_ERR_INVALID_ARG;
+  if (!dev_lm1->k_pool || !dev_lm1->v_pool || !dev_l->k_pool || !dev_l->v_pool) return MC_ERR_INVALID_ARG;
+  const size_t pool_bytes = (size_t)batch->n_pages * cfg->n_kv_heads * cfg->page_size * kRowBytes;
+  cudaStream_t s = (cudaStream_t)stream;
+  MC_CUDA_CHECK(cudaMemcpyAsync(dev_lm1->k_pool, host_lm1->k_pool, pool_bytes, cudaMemcpyHostToDevice, s));
+  MC_CUDA_CHECK(cudaMemcpyAsync(dev_lm1->v_pool, host_lm1->v_pool, pool_bytes, cudaMemcpyHostToDevice, s));
+  MC_CUDA_CHECK(cudaMemcpyAsync(dev_l->k_pool, host_l->k_pool, pool_bytes, cudaMemcpyHostToDevice, s));
+  MC_CUDA_CHECK(cudaMemcpyAsync(dev_l->v_pool, host_l->v_pool, pool_bytes, cudaMemcpyHostToDevice, s));
+  return mc_merge_pair(cfg, batch, dev_lm1, dev_l, out, do_retention, workspace, workspace_bytes, stream);
+}
+
+static void decode_io_layout(const mc_config* cfg, const mc_batch* bt, int n_sets, size_t off[6]) {
+  const size_t qb = align_up((size_t)n_sets * bt->batch * cfg->n_q_heads * kRowBytes, 256);
+  const size_t nb = align_up((size_t)n_sets * bt->batch * cfg->n_kv_heads * kRowBytes, 256);
+  const size_t lb = align_up((size_t)n_sets * bt->batch * cfg->n_q_heads * sizeof(float), 256);
+  off[0] = 0;            // q
+  off[1] = qb;           // k_new
+  off[2] = qb + nb;      // v_new
+  off[3] = qb + 2 * nb;  // out
+  off[4] = 2 * qb + 2 * nb;  // lse
+  off[5] = 2 * qb + 2 * nb + lb;
+}
+
+mc_status mc_decode_io_bytes(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets, size_t* bytes) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (!batch || !bytes || batch->batch < 0 || (n_query_sets != 1 && n_query_sets != 2)) return MC_ERR_INVALID_ARG;
+  size_t off[6];
+  decode_io_layout(cfg, batch, n_query_sets, off);
+  *bytes = off[5];
+  return MC_OK;
+}
+
+mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                              int32_t layer_sel, const void* q_host, const void* k_new_host, const void* v_new_host,
+                              float sm_scale, void* out_host, float* lse_host, void* dev_io, size_t dev_io_bytes,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  if (layer_sel < MC_LAYER_LM1 || layer_sel > MC_LAYER_BOTH) return MC_ERR_INVALID_ARG;
+  if (!q_host || !out_host || !dev_io) return MC_ERR_INVALID_ARG;
+  if ((k_new_host == nullptr) != (v_new_host == nullptr)) return MC_ERR_INVALID_ARG;
+  if (!aligned256(dev_io)) return MC_ERR_ALIGN;
+  const int n_sets = layer_sel == MC_LAYER_BOTH ? 2 : 1;
+  size_t off[6];
+  decode_io_layout(cfg, batch, n_sets, off);
+  if (dev_io_bytes < off[5]) return MC_ERR_CAPACITY;
+  char* io = (char*)dev_io;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t qb = (size_t)n_sets * batch->batch * cfg->n_q_heads * kRowBytes;
+  const size_t nb = (size_t)n_sets * batch->batch * cfg->n_kv_heads * kRowBytes;
+  MC_CUDA_CHECK(cudaMemcpyAsync(io + off[0], q_host, qb, cudaMemcpyHostToDevice, s));
+  if (k_new_host) {
+    MC_CUDA_CHECK(cudaMemcpyAsync(io + off[1], k_new_host, nb, cudaMemcpyHostToDevice, s));
+    MC_CUDA_CHECK(cudaMemcpyAsync(io + off[2], v_new_host, nb, cudaMemcpyHostToDevice, s));
+  }
+  st = mc_decode_attn(cfg, batch, pair, layer_sel, io + off[0], k_new_host ? io + off[1] : nullptr,
+                      k_new_host ? io + off[2] : nullptr, sm_scale, io + off[3],
+                      lse_host ? (float*)(io + off[4]) : nullptr, workspace, workspace_bytes, stream);
+  if (st != MC_OK) return st;
+  MC_CUDA_CHECK(cudaMemcpyAsync(out_host, io + off[3], qb, cudaMemcpyDeviceToHost, s));
+  if (lse_host)
+    MC_CUDA_CHECK(cudaMemcpyAsync(lse_host, io + off[4], (size_t)n_sets * batch->batch * cfg->n_q_heads * sizeof(float),
+                                  cudaMemcpyDeviceToHost, s));
+  return MC_OK;
+}
+
 mc_status mc_read_status(const mc_pair_cache* pair, void* stream, int32_t* out_words) {
   if (pair == nullptr || pair->status == nullptr || out_words == nullptr) return MC_ERR_INVALID_ARG;
   MC_CUDA_CHECK(cudaMemcpyAsync(out_words, pair->status, MC_STATUS_WORDS * sizeof(int32_t), cudaMemcpyDeviceToHost,
