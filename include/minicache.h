@@ -226,6 +226,32 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
 mc_status mc_decode_io_bytes(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets,
                              size_t* bytes);
 
+/* Largest split-partial scratch mc_decode_attn_static can serve (bytes of its built-in array). */
+#define MC_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+
+/* mc_decode_attn without a workspace argument.  (The paper has no counterpart: this exists for
+ * integration reasons only.)  Some callers cannot hand the library scratch memory: a serving
+ * engine that has already given every free byte of HBM to its KV-cache pool, a plugin that is
+ * only passed its input and output tensors, or a decode loop that must not call cudaMalloc
+ * because an allocation synchronises the device and stalls every stream.  For them the split
+ * partials live in an array that is part of the library image: MC_STATIC_SCRATCH_BYTES of device
+ * memory on every GPU that loads the library, held until the process exits.
+ *
+ * Arguments, results and numerics are those of mc_decode_attn (same kernels).  Differences:
+ * - A geometry whose partials need more than MC_STATIC_SCRATCH_BYTES (what
+ *   mc_workspace_bytes(MC_OP_DECODE_ATTN) reports) is refused with MC_ERR_CAPACITY before anything
+ *   is launched; mc_last_cuda_error() then names both sizes.
+ * - The first call on each device looks up the array's device address (one runtime query, no
+ *   allocation).  Make that first call outside any stream capture.
+ * - All calls on a device share the one array.  Nothing in it has to start at zero: every slot a
+ *   call reads was written earlier by the same call.  But two calls that may run at the same time
+ *   on the GPU (different streams, no ordering between them) overwrite each other's partials:
+ *   order them on one stream or with events.
+ * The call allocates and frees nothing, on the device or through any library. */
+mc_status mc_decode_attn_static(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                                int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
+                                float sm_scale, void* out, float* lse, void* stream);
+
 /* Copies the pair's status words to host memory `out_words[MC_STATUS_WORDS]` after synchronising
  * `stream`.  Returns MC_ERR_CAPACITY if the overflow flag is set, MC_ERR_DEVICE_STATUS for any
  * other flag, MC_OK otherwise. */

@@ -54,7 +54,7 @@ class _PairCache(C.Structure):
 
 EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
-           "mc_decode_attn_host", "mc_decode_io_bytes")
+           "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -162,6 +162,8 @@ class MiniCacheLib:
         L.mc_decode_attn_host.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V,
                                           V, C.c_size_t, V, C.c_size_t, V]
         L.mc_decode_io_bytes.argtypes = [P(_Config), P(_Batch), C.c_int32, P(C.c_size_t)]
+        L.mc_decode_attn_static.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V]
+        L.mc_decode_attn_static.restype = C.c_int32
         for f in ("mc_workspace_bytes", "mc_merge_pair", "mc_append_pair", "mc_restore", "mc_decode_attn",
                   "mc_read_status", "mc_merge_pair_host", "mc_decode_attn_host", "mc_decode_io_bytes"):
             getattr(L, f).restype = C.c_int32
@@ -240,6 +242,17 @@ class MiniCacheLib:
                                                   _ptr(lse_host), _ptr(dev_io), dev_io.numel() * dev_io.element_size(),
                                                   _ptr(workspace), workspace.numel() * workspace.element_size(),
                                                   _stream(stream)))
+
+    def mc_decode_attn_static(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q, k_new, v_new,
+                              sm_scale: float, out, lse, stream=None):
+        """mc_decode_attn for callers with no scratch memory to give: the split partials go to the
+        library's built-in device array (at most MC_STATIC_SCRATCH_BYTES; larger geometries raise)."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        code = self._lib.mc_decode_attn_static(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q), _ptr(k_new),
+                                               _ptr(v_new), float(sm_scale), _ptr(out), _ptr(lse), _stream(stream))
+        if code == 5:
+            raise McError(code, "MC_ERR_CAPACITY", self._lib.mc_last_cuda_error().decode())
+        self._check(code)
 
     def mc_read_status(self, pair: PairCache, stream=None, check: bool = True):
         words = (C.c_int32 * MC_STATUS_WORDS)()

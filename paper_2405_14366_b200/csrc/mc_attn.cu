@@ -609,3 +609,52 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
 }
 
 }  // namespace mc
+
+// ---------------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot supply scratch memory: the split partials live in a
+// device array that is part of the library image.
+// ---------------------------------------------------------------------------------------------------
+#include <mutex>
+#include <stdio.h>
+
+static __device__ __align__(256) unsigned char g_static_scratch[MC_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};  // device address of g_static_scratch, per device
+}  // namespace
+
+extern "C" mc_status mc_decode_attn_static(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                                           int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
+                                           float sm_scale, void* out, float* lse, void* stream) {
+  if (layer_sel < MC_LAYER_LM1 || layer_sel > MC_LAYER_BOTH) return MC_ERR_INVALID_ARG;
+  const int n_sets = layer_sel == MC_LAYER_BOTH ? 2 : 1;
+  size_t need = 0;
+  const mc_status st = mc_workspace_bytes(cfg, batch, MC_OP_DECODE_ATTN, n_sets, &need);  // validates cfg, host only
+  if (st != MC_OK) return st;
+  if (need > (size_t)MC_STATIC_SCRATCH_BYTES) {
+    char msg[160];
+    snprintf(msg, sizeof(msg), "mc_decode_attn_static: partials need %zu bytes, built-in scratch holds %u", need,
+             (unsigned)MC_STATIC_SCRATCH_BYTES);
+    mc::set_cuda_error(cudaSuccess, msg);
+    return MC_ERR_CAPACITY;
+  }
+  int dev = -1;
+  MC_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return MC_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+      // In host code `g_static_scratch` is only a handle for the symbol; the address the kernels
+      // must be given comes from the runtime, separately for each device.
+      void* ptr = nullptr;
+      MC_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_scratch));
+      g_scratch_addr[dev] = ptr;
+    }
+    scratch = g_scratch_addr[dev];
+  }
+  return mc_decode_attn(cfg, batch, pair, layer_sel, q, k_new, v_new, sm_scale, out, lse, scratch,
+                        (size_t)MC_STATIC_SCRATCH_BYTES, stream);
+}
