@@ -306,7 +306,10 @@ def main():
 
     job = Job(wl, dev)
     warm = max(3, args.warmup)
-    for _ in range(warm):
+    sampler = None
+    for i in range(warm):
+        if i == warm - 1 and rank == 0:
+            sampler = ClockSampler(local)  # started one step early: nvidia-smi takes a moment to begin sampling
         job.step()
     torch.cuda.synchronize()
     rho = job.retained_fraction()
@@ -318,7 +321,6 @@ def main():
     # ---- device-resident timed region: exactly K steps ----------------------------------------
     job.launches = 0
     job.attn_events = []
-    sampler = ClockSampler(local) if rank == 0 else None
     if dist is not None:
         dist.barrier()
     t_total = timed(lambda: [job.step(sample_events=True) for _ in range(args.steps)])

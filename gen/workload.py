@@ -90,6 +90,9 @@ def _mk() -> Dict[str, WorkloadConfig]:
     c["c3_s"] = c["c3"].scaled("c3_s", batch=4, seq_len=2048, n_layers=20, decode_steps=4)
     c["c4_s"] = c["c4"].scaled("c4_s", batch=8, seq_len=512, n_layers=18, decode_steps=8)
     c["c5_s"] = c["c5"].scaled("c5_s", batch=1, seq_len=8192, n_layers=18, decode_steps=4)
+    # one pair of config 2 / 3 at full batch and length (larger than L2, ~2 GB): profiler captures
+    c["c2_p1"] = c["c2"].scaled("c2_p1", n_layers=18, decode_steps=2)
+    c["c3_p1"] = c["c3"].scaled("c3_p1", n_layers=18, decode_steps=2)
     return c
 
 
