@@ -277,12 +277,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--page-size", type=int, default=None, help="override the workload's page size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     wl = gen.CONFIGS[args.workload]
     if args.decode_steps is not None:
         wl = dataclasses.replace(wl, decode_steps=args.decode_steps)
+    if args.page_size is not None:
+        wl = dataclasses.replace(wl, page_size=args.page_size)
     if args.impl == "reference":
         run_reference(args, wl)
         return
