@@ -114,11 +114,15 @@ typedef struct mc_layer_kv {
 
 /* The shared cache C^{l,l-1} of one layer pair (Sec. 4.2: [E, R^l, R^{l-1}, |X^{l-1}|, |X^l|, I]).
  *
- * e_k / e_v  shared directions E, rounded to the storage type, every token position kept.
- * scale      [n_pages][n_kv_heads][4][page_size] fp32; slot 0: K of layer l-1, 1: K of layer l,
- *            2: V of layer l-1, 3: V of layer l.  The stored number is |x| / |e_stored|, the
- *            magnitude of Eq. 2 already divided by the length of the rounded direction, so
- *            that restore is one multiply: x_hat = e_stored * scale.
+ * e_k / e_v  [n_pages][n_kv_heads][tile] bytes, tile = page_size * 256 + 2 * page_size * 4 bytes: the
+ *            shared directions E of one (page, head) -- page_size rows of 128 values of the 16-bit
+ *            storage type, every token position kept -- followed by the two layers' scales
+ *            [2][page_size] fp32 ([0]: layer l-1, [1]: layer l).  Inside a row the sixteen 16-byte
+ *            chunks are permuted: chunk c of row r is stored at chunk position
+ *            (c & 8) | ((c & 7) ^ (r & 7)), the order the attention kernel wants in shared memory.
+ *            A scale is |x| / |e_stored|, the magnitude of Eq. 2 already divided by the length of
+ *            the rounded direction, so that restore is one multiply: x_hat = e_stored * scale.
+ *            The scales of a retained token are zero (its rows are kept raw in ret_rows).
  * dist       [n_pages][n_kv_heads][2][page_size] fp32 angular distance d = Omega / pi; slot 0: K, 1: V.
  * Retention, per segment seg = (tensor * batch + b) * n_kv_heads + head (tensor 0 = K, 1 = V):
  * ret_count  [2 * batch * n_kv_heads] retained tokens of the segment
@@ -130,7 +134,6 @@ typedef struct mc_layer_kv {
 typedef struct mc_pair_cache {
   void* e_k;
   void* e_v;
-  float* scale;
   float* dist;
   int32_t* ret_count;
   int32_t* ret_offset;

@@ -46,7 +46,7 @@ class _LayerKV(C.Structure):
 
 
 class _PairCache(C.Structure):
-    _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("scale", C.c_void_p), ("dist", C.c_void_p),
+    _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("dist", C.c_void_p),
                 ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
                 ("ret_rows", C.c_void_p), ("ret_capacity", C.c_int64), ("seg_minmax", C.c_void_p),
                 ("status", C.c_void_p)]
@@ -110,9 +110,9 @@ class PairCache:
         H, ps = cfg.n_kv_heads, cfg.page_size
         dt = cfg.torch_dtype
         self.cfg = cfg
-        self.e_k = torch.zeros(n_pages, H, ps, 128, dtype=dt, device=device)
-        self.e_v = torch.zeros(n_pages, H, ps, 128, dtype=dt, device=device)
-        self.scale = torch.zeros(n_pages, H, 4, ps, dtype=torch.float32, device=device)
+        self.tile_bytes = ps * 256 + 2 * ps * 4
+        self.e_k = torch.zeros(n_pages, H, self.tile_bytes, dtype=torch.uint8, device=device)
+        self.e_v = torch.zeros(n_pages, H, self.tile_bytes, dtype=torch.uint8, device=device)
         self.dist = torch.zeros(n_pages, H, 2, ps, dtype=torch.float32, device=device)
         nseg = 2 * batch * H
         self.ret_count = torch.zeros(nseg, dtype=torch.int32, device=device)
@@ -124,12 +124,34 @@ class PairCache:
         self.status = torch.zeros(MC_STATUS_WORDS, dtype=torch.int32, device=device)
 
     def c(self) -> _PairCache:
-        return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.scale), _ptr(self.dist), _ptr(self.ret_count),
+        return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.dist), _ptr(self.ret_count),
                           _ptr(self.ret_offset), _ptr(self.ret_index), _ptr(self.ret_rows), self.ret_capacity,
                           _ptr(self.seg_minmax), _ptr(self.status))
 
+    # -- decoding the tile layout (pure re-indexing, no arithmetic) ------------------------------
+    def directions(self, tensor: str) -> torch.Tensor:
+        """Stored directions of "k" or "v" as [n_pages][H][page_size][128] in the storage type
+        (the 16-byte chunk permutation of the tile format undone)."""
+        pool = self.e_k if tensor == "k" else self.e_v
+        ps = self.cfg.page_size
+        n_pages, H = pool.shape[:2]
+        rows = pool[:, :, :ps * 256].reshape(n_pages, H, ps, 16, 16)  # [..][row][chunk position][16 bytes]
+        r = torch.arange(ps, device=pool.device)[:, None]
+        c = torch.arange(16, device=pool.device)[None, :]
+        pos = (c & 8) | ((c & 7) ^ (r & 7))  # where chunk c of row r is stored
+        idx = pos[None, None, :, :, None].expand(n_pages, H, ps, 16, 16)
+        plain = torch.gather(rows, 3, idx).reshape(n_pages, H, ps, 256)
+        return plain.view(self.cfg.torch_dtype)
+
+    def scales(self, tensor: str) -> torch.Tensor:
+        """Scales of "k" or "v" as [n_pages][H][2][page_size] fp32 ([..][0]: layer l-1, [1]: layer l)."""
+        pool = self.e_k if tensor == "k" else self.e_v
+        ps = self.cfg.page_size
+        n_pages, H = pool.shape[:2]
+        return pool[:, :, ps * 256:].contiguous().view(torch.float32).reshape(n_pages, H, 2, ps)
+
     def nbytes(self) -> int:
-        ts = (self.e_k, self.e_v, self.scale, self.dist, self.ret_count, self.ret_offset, self.ret_index,
+        ts = (self.e_k, self.e_v, self.dist, self.ret_count, self.ret_offset, self.ret_index,
               self.ret_rows, self.seg_minmax, self.status)
         return sum(t.numel() * t.element_size() for t in ts)
 

@@ -41,12 +41,12 @@ static mc_status check_batch(const mc_config* cfg, const mc_batch* bt) {
 
 static mc_status check_pair(const mc_pair_cache* pc) {
   if (pc == nullptr) return MC_ERR_INVALID_ARG;
-  if (!pc->e_k || !pc->e_v || !pc->scale || !pc->dist || !pc->ret_count || !pc->ret_offset || !pc->seg_minmax ||
+  if (!pc->e_k || !pc->e_v || !pc->dist || !pc->ret_count || !pc->ret_offset || !pc->seg_minmax ||
       !pc->status)
     return MC_ERR_INVALID_ARG;
   if (pc->ret_capacity < 0) return MC_ERR_INVALID_ARG;
   if (pc->ret_capacity > 0 && (!pc->ret_index || !pc->ret_rows)) return MC_ERR_INVALID_ARG;
-  if (!aligned256(pc->e_k) || !aligned256(pc->e_v) || !aligned256(pc->scale) || !aligned256(pc->dist)) return MC_ERR_ALIGN;
+  if (!aligned256(pc->e_k) || !aligned256(pc->e_v) || !aligned256(pc->dist)) return MC_ERR_ALIGN;
   if (pc->ret_rows && !aligned256(pc->ret_rows)) return MC_ERR_ALIGN;
   return MC_OK;
 }

@@ -2,19 +2,25 @@
 // (Algorithm 2 "MiniCache Decoding": rescale by the layer's magnitude, put the retained rows
 // back, append the new token, softmax(q K^T) V), with the restore folded into the kernel:
 //
-//   q . (g_i e_i) = g_i (q . e_i)            the K magnitude scales the score
-//   sum_i p_i (g_i e_i) = sum_i (p_i g_i) e_i  the V magnitude scales the probability
+//   q . (g_i e_i) = g_i (q . e_i)              the K scale multiplies the score
+//   sum_i p_i (g_i e_i) = sum_i (p_i g_i) e_i  the V scale multiplies the probability
 //
-// so the shared direction rows are streamed once, untouched, and a retained token only
-// replaces one score (K) or one term of the sum (V).
+// so the shared direction rows are streamed once, untouched; a retained token (whose scales the
+// merge left at zero) only replaces one score (K) or adds one term to the sum (V).
 //
-// Work item = (sequence, kv head, split of the token axis).  One producer thread streams the
-// page tiles of the split with TMA (128-byte swizzled boxes, mbarrier pipeline): first all K
-// tiles, then all V tiles.  Four consumer warps run both contractions on the tensor cores with
-// the query rows of the kv head's group (and, in pair mode, of both layers) as the padded M
-// tile: scores -> shared memory -> split-local softmax -> P V.  Partial (m, l, o) per split are
-// merged by attn_combine_kernel.
-#include <cuda.h>
+// Work item = (sequence, split of the token axis, kv head).  The kernel is persistent: two CTAs
+// per SM walk the item list with a fixed stride.  In each CTA
+//   - the producer warp streams the compressed tiles of its items, one bulk copy (TMA engine,
+//     cp.async.bulk + mbarrier) per (page, head, tensor) tile, all K tiles of an item and then
+//     all its V tiles, through a ring of stages, running ahead into the next item;
+//   - four consumer warps run both contractions on the tensor cores, the query rows of the kv
+//     head's group (and of both layers in pair mode) being the padded M tile: scores x K scale
+//     -> shared memory -> split-local softmax -> (P x V scale) V;
+//   - the auxiliary warp does the irregular part in the shadow of the streaming: it finds the
+//     item's range of the retained lists, computes the retained rows' and the new token's
+//     scores while the K tiles stream, and adds their V terms while the V tiles stream.
+// Partial (m, l, o) per split are merged by attn_combine_kernel.  Every wait is bounded.
+#include <algorithm>
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
@@ -25,17 +31,18 @@ constexpr int kTile = 64;  // tokens per pipeline stage
 constexpr int kStages = 4;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kAttnThreads = kConsumerThreads + 64;  // + producer warp + lookup warp
+constexpr int kAttnThreads = kConsumerThreads + 64;  // + producer warp + auxiliary warp
 constexpr int kMaxRows = 8;                          // query rows per work item (M tile rows used)
-constexpr int kTileBytes = kTile * kRowBytes;        // 16 KB
-constexpr int kStageScaleBytes = 1024;
-constexpr int kStageBytes = kTileBytes + kStageScaleBytes;
-constexpr int kMaxSplit = 1024;
+constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
+constexpr int kMaxSplit = 512;
+constexpr int kFixCap = 128;  // retained-K entries per item whose scores the auxiliary warp pre-computes
+constexpr int kMaxBatchSmem = 1024;
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr int kCtasPerSm = 2;
 
 struct AttnParams {
   Geom g;
-  const float* scale;
+  const char* e_pool[2];  // compressed tiles: K, V
   const int32_t* ret_count;
   const int32_t* ret_offset;
   const int32_t* ret_index;
@@ -76,13 +83,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          dst),
-      "l"(tm), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
+// Bulk asynchronous copy global -> shared (TMA engine), completion counted in bytes on an mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
@@ -98,8 +99,7 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
 }
-// D += A(16x16, rows 8..15 zero) * B(16x8); only the two accumulator registers of rows 0..7 matter
-// to the caller but the instruction carries all four.
+// D += A(16x16, rows 8..15 zero) * B(16x8); only the accumulator registers of rows 0..7 matter.
 template <int DT>
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
   const uint32_t z = 0u;
@@ -118,7 +118,7 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
 
 // Bounded wait: gives up after kWaitLimit polls, records it, and makes every later wait of the
-// CTA (and of CTAs that start afterwards) return at once.
+// CTA (and of CTAs that look at the status word afterwards) return at once.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
   if (*s_abort) return false;
   for (uint32_t it = 0; it < kWaitLimit; ++it) {
@@ -131,353 +131,487 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
-// Address of 16-byte chunk `chunk` (0..15 over the 128 channels) of tile row `tk` inside a stage.
-// A stage holds, per page j and channel half, one TMA box [page_size rows][128 bytes] written
-// with the 128-byte swizzle: chunk c of row r sits at chunk position c ^ (r & 7).
-__device__ __forceinline__ uint32_t tile_addr(uint32_t stage, int tk, int chunk, int page_shift) {
+// Shared-memory address of 16-byte chunk `chunk` (0..15) of token row `tk` (0..63) of a stage.
+// A stage holds 64 / page_size tiles back to back, each as in global memory (see tile_bytes).
+__device__ __forceinline__ uint32_t tile_addr(uint32_t stage, int tk, int chunk, int page_shift, int tbytes) {
   const int j = tk >> page_shift;
   const int r = tk & ((1 << page_shift) - 1);
-  const int half = chunk >> 3;
-  return stage + (uint32_t)(((j * 2 + half) << page_shift) * 128 + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
+  return stage + (uint32_t)(j * tbytes + r * kRowBytes + (chunk_pos(r, chunk) << 4));
+}
+
+// One work item.
+struct Item {
+  int b, g, split;
+  int split_start;
+  int n_tok;    // cached tokens of this split
+  int T;        // 64-token tiles
+  bool has_new;
+  bool valid;
+};
+
+// Item `i` of the flattened list (sequence-major, then split, then kv head) from the per-sequence
+// prefix of split counts in shared memory.
+__device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, const AttnParams& p) {
+  Item it;
+  it.valid = i < total;
+  if (!it.valid) {
+    it.b = it.g = it.split = it.split_start = it.n_tok = it.T = 0;
+    it.has_new = false;
+    return it;
+  }
+  const int H = p.g.n_kv_heads;
+  int lo = 0, hi = p.g.batch - 1;  // last b with pre_s[b] * H <= i
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (pre_s[mid] * H <= i) lo = mid; else hi = mid - 1;
+  }
+  it.b = lo;
+  const int local = i - pre_s[lo] * H;
+  it.split = local / H;
+  it.g = local - it.split * H;
+  const int n = p.g.seq_lens[lo];
+  const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
+  it.split_start = it.split * p.split_len;
+  it.n_tok = max(0, min(n, it.split_start + p.split_len) - it.split_start);
+  it.T = (it.n_tok + kTile - 1) / kTile;
+  it.has_new = (p.k_new != nullptr) && (it.split == nsp - 1);
+  return it;
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const __grid_constant__ CUtensorMap tm_k,
-                                                                 const __grid_constant__ CUtensorMap tm_v,
-                                                                 const AttnParams p) {
-  const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
-  const int n = p.g.seq_lens[b];
-  const int n_splits_b = max(1, (n + p.split_len - 1) / p.split_len);
-  if (split >= n_splits_b) return;
-  const int split_start = split * p.split_len;
-  const int n_tok = max(0, min(n, split_start + p.split_len) - split_start);  // cached tokens of this split
-  const bool has_new = (p.k_new != nullptr) && (split == n_splits_b - 1);
-  const int n_cols = n_tok + (has_new ? 1 : 0);
-  const int T = (n_tok + kTile - 1) / kTile;
+__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnParams p) {
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
+  const int tbytes = tile_bytes(ps);
   const int nslots = p.n_sets;
   const int rows = p.rows;
   const int s_stride = p.split_len + 8;
 
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
-  float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);       // [kMaxRows][s_stride]
-  float* O_s = S + kMaxRows * s_stride;                                    // [kMaxRows][128]
-  uint32_t* q_s = reinterpret_cast<uint32_t*>(O_s + kMaxRows * kHeadDim);  // [kMaxRows][64] packed pairs
-  int* pages_s = reinterpret_cast<int*>(q_s + kMaxRows * 64);              // [kMaxSplit / 16]
-  float* m_s = reinterpret_cast<float*>(pages_s + kMaxSplit / 16);         // [kMaxRows]
-  float* l_s = m_s + kMaxRows;
-  int* look_s = reinterpret_cast<int*>(l_s + kMaxRows);  // k_lo, k_hi, v_lo, v_hi
-  volatile int* s_abort = look_s + 4;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(look_s + 8);  // full[kStages], empty[kStages], lookup
-  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages, lookbar = full0 + 16 * kStages;
+  float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);  // [kMaxRows][s_stride]
+  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kMaxRows * s_stride);  // [2][kMaxRows][64] packed pairs
+  float* kfix_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);     // [kFixCap][kMaxRows]
+  int* kcol_s = reinterpret_cast<int*>(kfix_s + kFixCap * kMaxRows);     // [kFixCap]
+  float* knew_s = reinterpret_cast<float*>(kcol_s + kFixCap);            // [kMaxRows]
+  float* oaux_s = knew_s + kMaxRows;                                     // [kMaxRows][128]
+  float* m_s = oaux_s + kMaxRows * kHeadDim;                             // [kMaxRows]
+  float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
+  float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
+  int* aux_info = reinterpret_cast<int*>(red_s + kMaxRows * kConsumerWarps);  // n_fast, k_lo, k_hi, pad
+  int* pre_s = aux_info + 4;                                                  // [batch + 1] split-count prefix
+  volatile int* s_abort = pre_s + kMaxBatchSmem + 1;
+  uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
+  const uint32_t kfix_bar = full0 + 16 * kStages, pready_bar = kfix_bar + 8, oaux_bar = kfix_bar + 16;
   const uint32_t stage0 = smem_u32(stages);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  // ---- prologue: barriers, page ids, query rows -------------------------------------------------
+  // ---- prologue -----------------------------------------------------------------------------------
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, kConsumerWarps);
     }
-    mbar_init(lookbar, 1);
+    mbar_init(kfix_bar, 1);
+    mbar_init(pready_bar, 1);
+    mbar_init(oaux_bar, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  {
-    const int first_slot = split_start >> shift;
-    const int n_pg = (n_tok + ps - 1) >> shift;
-    for (int i = tid; i < n_pg; i += kAttnThreads)
-      pages_s[i] = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + first_slot + i];
-    // query rows: row r = set * nq + rq  ->  q[set][b][g * nq + rq][:]
-    for (int i = tid; i < kMaxRows * 64; i += kAttnThreads) {
-      const int r = i >> 6, w = i & 63;
-      uint32_t v = 0;
-      if (r < rows) {
-        const int set = r / p.nq, rq = r - set * p.nq;
-        const size_t qrow = ((size_t)set * p.g.batch + b) * p.n_q_heads + g * p.nq + rq;
-        v = reinterpret_cast<const uint32_t*>(p.q)[qrow * 64 + w];
-      }
-      q_s[i] = v;
+    // prefix of per-sequence split counts (a sequence always owns at least one split)
+    int acc = 0;
+    for (int b = 0; b < p.g.batch; ++b) {
+      pre_s[b] = acc;
+      acc += max(1, (p.g.seq_lens[b] + p.split_len - 1) / p.split_len);
     }
+    pre_s[p.g.batch] = acc;
   }
   __syncthreads();
-
-  const int seg_k = b * H + g;
-  const int seg_v = (p.g.batch + b) * H + g;
+  const int total_items = pre_s[p.g.batch] * H;
+  const int first = blockIdx.x, stride = gridDim.x;
 
   if (warp == kConsumerWarps) {
     // ===================== producer =====================
-    if (lane == 0) {
-      const uint32_t page_bytes = (uint32_t)ps * kRowBytes + (uint32_t)nslots * ps * 4;
-      for (int it = 0; it < 2 * T; ++it) {
-        const int phase = it >= T ? 1 : 0;
-        const int t = it - phase * T;
-        const int s = it % kStages;
-        if (it >= kStages && !mbar_wait(empty0 + 8 * s, ((it / kStages) - 1) & 1, s_abort, p.status)) break;
-        const int tok0 = t * kTile;
-        const int n_pg = min(kTile >> shift, (n_tok - tok0 + ps - 1) >> shift);
-        const uint32_t bar = full0 + 8 * s;
-        const uint32_t sbase = stage0 + s * kStageBytes;
-        mbar_expect_tx(bar, n_pg * page_bytes);
-        const CUtensorMap* tm = phase ? &tm_v : &tm_k;
-        for (int j = 0; j < n_pg; ++j) {
-          const int page = pages_s[(tok0 >> shift) + j];
-          const int y = (page * H + g) * ps;
-          tma_load_2d(sbase + (uint32_t)((j * 2) << shift) * 128, tm, 0, y, bar);
-          tma_load_2d(sbase + (uint32_t)((j * 2 + 1) << shift) * 128, tm, 64, y, bar);
-          const int slot = phase * 2 + (nslots == 2 ? 0 : p.layer_sel);
-          const float* src = p.scale + (((size_t)page * H + g) * 4 + slot) * ps;
-          bulk_load(sbase + kTileBytes + (uint32_t)j * nslots * ps * 4, src, (uint32_t)nslots * ps * 4, bar);
+    int it = 0;  // running stage counter, same sequence as the consumers'
+    for (int i = first; i < total_items; i += stride) {
+      const Item w = get_item(i, total_items, pre_s, p);
+      // page ids of the item's pages, one per lane (split_len / page_size <= 32)
+      const int n_pages_item = (w.n_tok + ps - 1) >> shift;
+      int my_page = 0;
+      if (lane < n_pages_item)
+        my_page = p.g.block_table[(size_t)w.b * p.g.max_pages_per_seq + (w.split_start >> shift) + lane];
+      bool ok = true;
+      for (int ph = 0; ph < 2 && ok; ++ph) {
+        for (int t = 0; t < w.T; ++t, ++it) {
+          const int s = it % kStages;
+          if (it >= kStages) {
+            int good = 1;
+            if (lane == 0) good = mbar_wait(empty0 + 8 * s, ((it / kStages) - 1) & 1, s_abort, p.status) ? 1 : 0;
+            good = __shfl_sync(0xffffffffu, good, 0);
+            if (!good) { ok = false; break; }
+          }
+          const int pg0 = (t * kTile) >> shift;
+          const int n_pg = min(kTile >> shift, n_pages_item - pg0);
+          const uint32_t bar = full0 + 8 * s;
+          if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_pg * tbytes));
+          __syncwarp();
+          // lane pg0 + j copies tile j of the stage (it holds that page's id)
+          const int j = lane - pg0;
+          if (j >= 0 && j < n_pg) {
+            const char* src = p.e_pool[ph] + ((size_t)my_page * H + w.g) * tbytes;
+            bulk_load(stage0 + s * kStageBytes + j * tbytes, src, (uint32_t)tbytes, bar);
+          }
         }
       }
+      if (!ok) break;
     }
     return;
   }
+
   if (warp == kConsumerWarps + 1) {
-    // ===================== retained-list lookup =====================
-    // lane 0: K segment, lane 1: V segment.  Range of list entries whose token lies in this split.
-    if (lane < 2) {
-      const int seg = lane == 0 ? seg_k : seg_v;
-      const int cnt = p.ret_count[seg];
-      const int off = p.ret_offset[seg];
-      int lo = 0, hi = cnt;  // first entry with token >= split_start
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (p.ret_index[off + mid] < split_start) lo = mid + 1; else hi = mid;
+    // ===================== auxiliary warp: retained rows and the new token =====================
+    int n_item = 0;
+    for (int i = first; i < total_items; i += stride, ++n_item) {
+      const Item w = get_item(i, total_items, pre_s, p);
+      const uint32_t par = n_item & 1;
+      const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
+      // ranges of the retained lists whose tokens lie in this split (all lanes search alike)
+      int rng[2][2];
+#pragma unroll
+      for (int tz = 0; tz < 2; ++tz) {
+        const int seg = tz ? seg_v : seg_k;
+        const int cnt = p.ret_count[seg], off = p.ret_offset[seg];
+        int lo = 0, hi = cnt;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (p.ret_index[off + mid] < w.split_start) lo = mid + 1; else hi = mid;
+        }
+        const int firstp = lo;
+        hi = cnt;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (p.ret_index[off + mid] < w.split_start + w.n_tok) lo = mid + 1; else hi = mid;
+        }
+        rng[tz][0] = off + firstp;
+        rng[tz][1] = off + lo;
       }
-      const int first = lo;
-      hi = cnt;  // first entry with token >= split_start + n_tok
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (p.ret_index[off + mid] < split_start + n_tok) lo = mid + 1; else hi = mid;
+      const int n_k = rng[0][1] - rng[0][0], n_v = rng[1][1] - rng[1][0];
+      const int n_fast = min(n_k, kFixCap);
+      // query rows, 4 channels per lane
+      float qf[kMaxRows][4];
+      if (n_k > 0 || w.has_new) {
+#pragma unroll
+        for (int r = 0; r < kMaxRows; ++r) {
+          if (r < rows) {
+            const int set = r / p.nq, rq = r - set * p.nq;
+            const size_t qrow = ((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq;
+            const uint2 v = *reinterpret_cast<const uint2*>(p.q + qrow * kRowBytes + lane * 8);
+            const float2 a = Elem<DT>::unpack(v.x), c = Elem<DT>::unpack(v.y);
+            qf[r][0] = a.x; qf[r][1] = a.y; qf[r][2] = c.x; qf[r][3] = c.y;
+          }
+        }
       }
-      look_s[lane * 2] = off + first;
-      look_s[lane * 2 + 1] = off + lo;
+      // ---- K part: scores of retained rows (first kFixCap of them) and of the new token
+      for (int e = 0; e < n_fast + (w.has_new ? 1 : 0); ++e) {
+        const bool is_new = e >= n_fast;
+        const int col = is_new ? w.n_tok : p.ret_index[rng[0][0] + e] - w.split_start;
+#pragma unroll
+        for (int r = 0; r < kMaxRows; ++r) {
+          if (r < rows) {
+            const int set = r / p.nq;
+            const char* src = is_new ? p.k_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
+                                     : p.ret_rows + ((size_t)(rng[0][0] + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
+            const uint2 kv = *reinterpret_cast<const uint2*>(src + lane * 8);
+            const float2 k0 = Elem<DT>::unpack(kv.x), k1 = Elem<DT>::unpack(kv.y);
+            float d = qf[r][0] * k0.x + qf[r][1] * k0.y + qf[r][2] * k1.x + qf[r][3] * k1.y;
+            for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            if (lane == 0) {
+              if (is_new) knew_s[r] = d * p.scale_log2; else kfix_s[e * kMaxRows + r] = d * p.scale_log2;
+            }
+          }
+        }
+        if (lane == 0 && !is_new) kcol_s[e] = col;
+      }
+      if (lane == 0) {
+        aux_info[0] = n_fast;
+        aux_info[1] = rng[0][0];
+        aux_info[2] = rng[0][1];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(kfix_bar);
+      // ---- V part: after the softmax, add the retained V rows' and the new token's terms
+      int good = 1;
+      if (lane == 0) good = mbar_wait(pready_bar, par, s_abort, p.status) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      float oa[kMaxRows][4];
+#pragma unroll
+      for (int r = 0; r < kMaxRows; ++r) oa[r][0] = oa[r][1] = oa[r][2] = oa[r][3] = 0.f;
+      for (int e = 0; e < n_v + (w.has_new ? 1 : 0); ++e) {
+        const bool is_new = e >= n_v;
+        const int col = is_new ? w.n_tok : p.ret_index[rng[1][0] + e] - w.split_start;
+        float val[2][4];
+#pragma unroll
+        for (int set = 0; set < 2; ++set) {
+          if (set < nslots) {
+            const char* src = is_new ? p.v_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
+                                     : p.ret_rows + ((size_t)(rng[1][0] + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
+            const uint2 vv = *reinterpret_cast<const uint2*>(src + lane * 8);
+            const float2 a = Elem<DT>::unpack(vv.x), c = Elem<DT>::unpack(vv.y);
+            val[set][0] = a.x; val[set][1] = a.y; val[set][2] = c.x; val[set][3] = c.y;
+          } else {
+            val[set][0] = val[set][1] = val[set][2] = val[set][3] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < kMaxRows; ++r) {
+          if (r < rows) {
+            const float pr = S[r * s_stride + col];
+            const int set = nslots == 2 ? r / p.nq : 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) oa[r][k] = fmaf(pr, set ? val[1][k] : val[0][k], oa[r][k]);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < kMaxRows; ++r)
+        if (r < rows) *reinterpret_cast<float4*>(oaux_s + r * kHeadDim + lane * 4) = make_float4(oa[r][0], oa[r][1], oa[r][2], oa[r][3]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(oaux_bar);
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(lookbar);  // release: the writes above are visible to waiters
     return;
   }
 
   // ===================== consumers =====================
-  const int row = lane >> 2;         // M-tile row of this thread's fragments
-  const int colp = (lane & 3) * 2;   // column pair inside an 8-wide n tile
-  const int slot_row = (nslots == 2 && row < rows) ? row / p.nq : 0;
+  const int row = lane >> 2;        // M-tile row of this thread's fragments
+  const int colp = (lane & 3) * 2;  // column pair inside an 8-wide n tile
+  const int slot_row = (nslots == 2 && row < rows) ? row / p.nq : (nslots == 2 ? 0 : p.layer_sel);
+  const int mi = lane >> 3, mr = lane & 7;
+  int it = 0, n_item = 0;
 
-  // ---- K phase: S[r][i] = log2e * sm_scale * g_i * (q_r . e_i) -----------------------------------
-  {
-    uint32_t qa0[8], qa2[8];
+  // query rows of the first item
+  auto load_q_words = [&](const Item& w, uint32_t (&qw)[4]) {
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      qa0[ks] = q_s[row * 64 + ks * 8 + (lane & 3)];
-      qa2[ks] = q_s[row * 64 + ks * 8 + 4 + (lane & 3)];
-    }
-    const int tk_w = warp * 16;  // this warp's 16 tokens of every tile
-    const int mi = lane >> 3, mr = lane & 7;
-    for (int t = 0; t < T; ++t) {
-      const int it = t, s = it % kStages;
-      if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) break;
-      const uint32_t sbase = stage0 + s * kStageBytes;
-      const int valid = min(kTile, n_tok - t * kTile);
-      if (tk_w < valid) {
-        float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-        const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          uint32_t r0, r1, r2, r3;
-          ldsm_x4(tile_addr(sbase, tk_m, ks * 2 + (mi & 1), shift), r0, r1, r2, r3);
-          mma_16816<DT>(acc0, qa0[ks], qa2[ks], r0, r1);
-          mma_16816<DT>(acc1, qa0[ks], qa2[ks], r2, r3);
-        }
-        if (row < rows) {
-          const float* sc = reinterpret_cast<const float*>(stages + s * kStageBytes + kTileBytes);
-          const int j = tk_w >> shift, r = tk_w & (ps - 1);
-          const float* scj = sc + (j * nslots + slot_row) * ps + r;
-          float* srow = S + row * s_stride + t * kTile + tk_w;
-          const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
-          const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
-          *reinterpret_cast<float2*>(srow + colp) =
-              make_float2(acc0[0] * g0.x * p.scale_log2, acc0[1] * g0.y * p.scale_log2);
-          *reinterpret_cast<float2*>(srow + 8 + colp) =
-              make_float2(acc1[0] * g1.x * p.scale_log2, acc1[1] * g1.y * p.scale_log2);
-        }
+    for (int k = 0; k < 4; ++k) {
+      const int i = tid + k * kConsumerThreads;  // 512 words = 8 rows x 64
+      const int r = i >> 6, wd = i & 63;
+      uint32_t v = 0;
+      if (w.valid && r < rows) {
+        const int set = r / p.nq, rq = r - set * p.nq;
+        const size_t qrow = ((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq;
+        v = reinterpret_cast<const uint32_t*>(p.q)[qrow * 64 + wd];
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      qw[k] = v;
     }
+  };
+  {
+    uint32_t qw[4];
+    load_q_words(get_item(first, total_items, pre_s, p), qw);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
   consumer_sync();
 
-  // ---- retained K rows and the new token replace / add single scores ----------------------------
-  const bool any_list = (p.ret_count[seg_k] | p.ret_count[seg_v]) != 0;
-  int k_lo = 0, k_hi = 0, v_lo = 0, v_hi = 0;
-  if (any_list) {
-    mbar_wait(lookbar, 0, s_abort, p.status);
-    k_lo = look_s[0];
-    k_hi = look_s[1];
-    v_lo = look_s[2];
-    v_hi = look_s[3];
-  }
-  {
-    const int n_extra = (k_hi - k_lo) + (has_new ? 1 : 0);
-    for (int e = warp; e < n_extra; e += kConsumerWarps) {
-      const bool is_new = e >= (k_hi - k_lo);
-      const int col = is_new ? n_tok : p.ret_index[k_lo + e] - split_start;
+  for (int i = first; i < total_items; i += stride, ++n_item) {
+    const Item w = get_item(i, total_items, pre_s, p);
+    const uint32_t par = n_item & 1;
+    const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
+    const int n_cols = w.n_tok + (w.has_new ? 1 : 0);
+    bool ok = true;
+
+    // ---- K phase: S[r][i] = log2e * sm_scale * g_i * (q_r . e_i) ---------------------------------
+    {
+      uint32_t qa0[8], qa2[8];
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qa0[ks] = qcur[row * 64 + ks * 8 + (lane & 3)];
+        qa2[ks] = qcur[row * 64 + ks * 8 + 4 + (lane & 3)];
+      }
+      const int tk_w = warp * 16;  // this warp's 16 tokens of every tile
+      for (int t = 0; t < w.T; ++t, ++it) {
+        const int s = it % kStages;
+        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const uint32_t sbase = stage0 + s * kStageBytes;
+        const int valid = min(kTile, w.n_tok - t * kTile);
+        if (tk_w < valid) {
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+          const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
+          const uint32_t rowaddr = tile_addr(sbase, tk_m, 0, shift, tbytes) - (chunk_pos(tk_m & (ps - 1), 0) << 4);
+          const int rsw = tk_m & 7;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t r0, r1, r2, r3;
+            const int c = ks * 2 + (mi & 1);
+            ldsm_x4(rowaddr + ((uint32_t)((c & 8) | ((c & 7) ^ rsw)) << 4), r0, r1, r2, r3);
+            mma_16816<DT>(acc0, qa0[ks], qa2[ks], r0, r1);
+            mma_16816<DT>(acc1, qa0[ks], qa2[ks], r2, r3);
+          }
+          if (row < rows) {
+            const int j = tk_w >> shift, r = tk_w & (ps - 1);
+            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + j * tbytes + ps * kRowBytes) +
+                               slot_row * ps + r;
+            float* srow = S + row * s_stride + t * kTile + tk_w;
+            const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
+            const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
+            *reinterpret_cast<float2*>(srow + colp) =
+                make_float2(acc0[0] * g0.x * p.scale_log2, acc0[1] * g0.y * p.scale_log2);
+            *reinterpret_cast<float2*>(srow + 8 + colp) =
+                make_float2(acc1[0] * g1.x * p.scale_log2, acc1[1] * g1.y * p.scale_log2);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      }
+    }
+    consumer_sync();
+
+    // ---- retained K rows and the new token replace / add single scores ----------------------------
+    if (ok && !mbar_wait(kfix_bar, par, s_abort, p.status)) ok = false;
+    if (ok) {
+      const int n_fast = aux_info[0], k_lo = aux_info[1], k_hi = aux_info[2];
+      for (int e = tid; e < n_fast; e += kConsumerThreads) {
+        const int col = kcol_s[e];
+        for (int r = 0; r < rows; ++r) S[r * s_stride + col] = kfix_s[e * kMaxRows + r];
+      }
+      if (w.has_new && tid < rows) S[tid * s_stride + w.n_tok] = knew_s[tid];
+      // more retained rows than the auxiliary warp pre-computes: finish them here
+      for (int e = k_lo + n_fast + warp; e < k_hi; e += kConsumerWarps) {
+        const int col = p.ret_index[e] - w.split_start;
+        for (int r = 0; r < rows; ++r) {
+          const int set = r / p.nq;
+          const char* src = p.ret_rows + ((size_t)e * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
+          const uint2 kv = *reinterpret_cast<const uint2*>(src + lane * 8);
+          const uint2 qv = *reinterpret_cast<const uint2*>(qcur + r * 64 + lane * 2);
+          const float2 k0 = Elem<DT>::unpack(kv.x), k1 = Elem<DT>::unpack(kv.y);
+          const float2 q0 = Elem<DT>::unpack(qv.x), q1 = Elem<DT>::unpack(qv.y);
+          float d = q0.x * k0.x + q0.y * k0.y + q1.x * k1.x + q1.y * k1.y;
+          for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+          if (lane == 0) S[r * s_stride + col] = d * p.scale_log2;
+        }
+      }
+    }
+    consumer_sync();
+
+    // ---- split-local softmax: S <- 2^(S - m), row sums; every warp takes a quarter of the columns ----
+    {
+      const int c_lo = (n_cols * warp) / kConsumerWarps, c_hi = (n_cols * (warp + 1)) / kConsumerWarps;
       for (int r = 0; r < rows; ++r) {
-        const int set = r / p.nq;
-        const char* src;
-        if (is_new)
-          src = p.k_new + (((size_t)set * p.g.batch + b) * H + g) * kRowBytes;
-        else
-          src = p.ret_rows + ((size_t)(k_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-        const uint2 kv = *reinterpret_cast<const uint2*>(src + lane * 8);
-        const uint2 qv = *reinterpret_cast<const uint2*>(q_s + r * 64 + lane * 2);
-        const float2 k0 = Elem<DT>::unpack(kv.x), k1 = Elem<DT>::unpack(kv.y);
-        const float2 q0 = Elem<DT>::unpack(qv.x), q1 = Elem<DT>::unpack(qv.y);
-        float d = q0.x * k0.x + q0.y * k0.y + q1.x * k1.x + q1.y * k1.y;
-        for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-        if (lane == 0) S[r * s_stride + col] = d * p.scale_log2;
-      }
-    }
-  }
-  consumer_sync();
-
-  // ---- split-local softmax: S <- 2^(S - m), row sums --------------------------------------------
-  for (int r = warp; r < rows; r += kConsumerWarps) {
-    float* srow = S + r * s_stride;
-    float m = -INFINITY;
-    for (int c = lane; c < n_cols; c += 32) m = fmaxf(m, srow[c]);
-    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float l = 0.f;
-    for (int c = lane; c < n_cols; c += 32) {
-      const float e = exp2f(srow[c] - m);
-      srow[c] = e;
-      l += e;
-    }
-    for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (lane == 0) {
-      m_s[r] = m;
-      l_s[r] = l;
-    }
-  }
-  consumer_sync();
-
-  // ---- retained V rows and the new token: their terms are added outside the tile loop ------------
-  float o_ret[kMaxRows];
-#pragma unroll
-  for (int r = 0; r < kMaxRows; ++r) o_ret[r] = 0.f;
-  {
-    const int n_extra = (v_hi - v_lo) + (has_new ? 1 : 0);
-    const unsigned short* rr = reinterpret_cast<const unsigned short*>(p.ret_rows);
-    for (int e = 0; e < n_extra; ++e) {
-      const bool is_new = e >= (v_hi - v_lo);
-      const int col = is_new ? n_tok : p.ret_index[v_lo + e] - split_start;
-      float val[2];
-#pragma unroll
-      for (int set = 0; set < 2; ++set) {
-        unsigned short bits = 0;
-        if (set < nslots) {
-          if (is_new)
-            bits = reinterpret_cast<const unsigned short*>(p.v_new)[(((size_t)set * p.g.batch + b) * H + g) * kHeadDim + tid];
-          else
-            bits = rr[((size_t)(v_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kHeadDim + tid];
-        }
-        val[set] = Elem<DT>::unpack((uint32_t)bits).x;
-      }
-#pragma unroll
-      for (int r = 0; r < kMaxRows; ++r)
-        if (r < rows) o_ret[r] = fmaf(S[r * s_stride + col], val[nslots == 2 ? r / p.nq : 0], o_ret[r]);
-    }
-    if (v_hi > v_lo) {
-      consumer_sync();
-      for (int e = tid; e < (v_hi - v_lo); e += kConsumerThreads) {
-        const int col = p.ret_index[v_lo + e] - split_start;
-        for (int r = 0; r < rows; ++r) S[r * s_stride + col] = 0.f;
+        float m = -INFINITY;
+        for (int c = c_lo + lane; c < c_hi; c += 32) m = fmaxf(m, S[r * s_stride + c]);
+        for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) red_s[r * kConsumerWarps + warp] = m;
       }
       consumer_sync();
-    }
-  }
-
-  // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
-  float acc[4][4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int k = 0; k < 4; ++k) acc[i][k] = 0.f;
-  {
-    const int mi = lane >> 3, mr = lane & 7;
-    const int chunk0 = warp * 4;  // this warp owns channels [32 warp, 32 warp + 32)
-    for (int t = 0; t < T; ++t) {
-      const int it = T + t, s = it % kStages;
-      if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) break;
-      const uint32_t sbase = stage0 + s * kStageBytes;
-      const int valid = min(kTile, n_tok - t * kTile);
-      const int ksteps = (valid + 15) >> 4;
-      // rows past the last cached token may hold anything (page tail, unloaded page): zero this
-      // warp's channels there so that 0 * x stays 0 in the contraction
-      for (int rz = valid + (lane >> 2); rz < ksteps * 16; rz += 8) {
-        const uint32_t a = tile_addr(sbase, rz, chunk0 + (lane & 3), shift);
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-      }
-      __syncwarp();
-      const float* sc = reinterpret_cast<const float*>(stages + s * kStageBytes + kTileBytes);
-      for (int kk = 0; kk < ksteps; ++kk) {
-        // A fragment: probabilities times the V magnitude, rounded to the storage type
-        uint32_t a0 = 0u, a2 = 0u;
-        if (row < rows) {
-          const int tk = kk * 16;
-          const int j = tk >> shift, r = tk & (ps - 1);
-          const float* scj = sc + (j * nslots + slot_row) * ps + r;
-          const float* srow = S + row * s_stride + t * kTile + tk;
-          const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
-          const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
-          const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
-          const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
-          const int c0 = tk + colp;
-          a0 = Elem<DT>::pack(c0 < valid ? p0.x * g0.x : 0.f, c0 + 1 < valid ? p0.y * g0.y : 0.f);
-          a2 = Elem<DT>::pack(c0 + 8 < valid ? p1.x * g1.x : 0.f, c0 + 9 < valid ? p1.y * g1.y : 0.f);
+      for (int r = 0; r < rows; ++r) {
+        const float4 mm = *reinterpret_cast<const float4*>(red_s + r * kConsumerWarps);
+        const float m = fmaxf(fmaxf(mm.x, mm.y), fmaxf(mm.z, mm.w));
+        float l = 0.f;
+        for (int c = c_lo + lane; c < c_hi; c += 32) {
+          const float e = exp2f(S[r * s_stride + c] - m);
+          S[r * s_stride + c] = e;
+          l += e;
         }
-        const int tk_m = kk * 16 + (mi & 1) * 8 + mr;
-#pragma unroll
-        for (int np = 0; np < 2; ++np) {
-          uint32_t r0, r1, r2, r3;
-          ldsm_x4_t(tile_addr(sbase, tk_m, chunk0 + np * 2 + (mi >> 1), shift), r0, r1, r2, r3);
-          mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
-          mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
+        for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (lane == 0) {
+          l_s[r * kConsumerWarps + warp] = l;
+          if (warp == 0) m_s[r] = m;
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      consumer_sync();
+      if (tid == 0) mbar_arrive(pready_bar);  // the probabilities are final: the auxiliary warp may read them
     }
-  }
-  if (row < rows) {
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-      *reinterpret_cast<float2*>(O_s + row * kHeadDim + warp * 32 + nt * 8 + colp) = make_float2(acc[nt][0], acc[nt][1]);
-  }
-  consumer_sync();
 
-  // ---- partial results of this split --------------------------------------------------------------
+    // query rows of the next item travel while the V tiles stream
+    uint32_t qnext[4];
+    load_q_words(get_item(i + stride, total_items, pre_s, p), qnext);
+
+    // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
+    float acc[4][4];
 #pragma unroll
-  for (int r = 0; r < kMaxRows; ++r) {
-    if (r < rows) {
-      const int set = r / p.nq, rq = r - set * p.nq;
-      const size_t prow = (((size_t)set * p.g.batch + b) * p.n_q_heads + g * p.nq + rq) * p.n_splits + split;
-      p.part_o[prow * kHeadDim + tid] = O_s[r * kHeadDim + tid] + o_ret[r];
-      if (tid == 0) {
-        p.part_ml[prow * 2] = m_s[r];
-        p.part_ml[prow * 2 + 1] = l_s[r];
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[a][k] = 0.f;
+    if (ok) {
+      const int chunk0 = warp * 4;  // this warp owns channels [32 warp, 32 warp + 32)
+      for (int t = 0; t < w.T; ++t, ++it) {
+        const int s = it % kStages;
+        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const uint32_t sbase = stage0 + s * kStageBytes;
+        const int valid = min(kTile, w.n_tok - t * kTile);
+        const int ksteps = (valid + 15) >> 4;
+        // rows past the last cached token may hold anything (page tail, page not copied): zero this
+        // warp's channels there so that 0 * x stays 0 in the contraction
+        bool wrote = false;
+        for (int rz = valid + (lane >> 2); rz < ksteps * 16; rz += 8) {
+          const uint32_t a = tile_addr(sbase, rz, chunk0 + (lane & 3), shift, tbytes);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+          wrote = true;
+        }
+        __syncwarp();
+        for (int kk = 0; kk < ksteps; ++kk) {
+          // A fragment: probabilities times the V scale, rounded to the storage type
+          uint32_t a0 = 0u, a2 = 0u;
+          if (row < rows) {
+            const int tk = kk * 16;
+            const int j = tk >> shift, r = tk & (ps - 1);
+            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + j * tbytes + ps * kRowBytes) +
+                               slot_row * ps + r;
+            const float* srow = S + row * s_stride + t * kTile + tk;
+            const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
+            const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
+            const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
+            const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
+            const int c0 = tk + colp;
+            a0 = Elem<DT>::pack(c0 < valid ? p0.x * g0.x : 0.f, c0 + 1 < valid ? p0.y * g0.y : 0.f);
+            a2 = Elem<DT>::pack(c0 + 8 < valid ? p1.x * g1.x : 0.f, c0 + 9 < valid ? p1.y * g1.y : 0.f);
+          }
+          const int tk_m = kk * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+          for (int np = 0; np < 2; ++np) {
+            uint32_t r0, r1, r2, r3;
+            ldsm_x4_t(tile_addr(sbase, tk_m, chunk0 + np * 2 + (mi >> 1), shift, tbytes), r0, r1, r2, r3);
+            mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
+            mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
+          }
+        }
+        if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
     }
+
+    // ---- partial results of this split: tensor-core part + the auxiliary warp's terms --------------
+    if (ok && !mbar_wait(oaux_bar, par, s_abort, p.status)) ok = false;
+    if (row < rows) {
+      const int set = row / p.nq, rq = row - set * p.nq;
+      const size_t prow = (((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
+      float* dst = p.part_o + prow * kHeadDim + warp * 32 + colp;
+      const float* oa = oaux_s + row * kHeadDim + warp * 32 + colp;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const float2 x = *reinterpret_cast<const float2*>(oa + nt * 8);
+        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(acc[nt][0] + x.x, acc[nt][1] + x.y);
+      }
+      if (warp == 0 && (lane & 3) == 0) {
+        const float4 ll = *reinterpret_cast<const float4*>(l_s + row * kConsumerWarps);
+        p.part_ml[prow * 2] = m_s[row];
+        p.part_ml[prow * 2 + 1] = (ll.x + ll.y) + (ll.z + ll.w);
+      }
+    }
+    // next item's query rows into the other buffer (nobody reads that buffer any more)
+    {
+      uint32_t* qn = q_s + ((n_item + 1) & 1) * kMaxRows * 64;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) qn[tid + k * kConsumerThreads] = qnext[k];
+    }
+    consumer_sync();
+    if (*s_abort) break;  // read after the barrier: the same answer in every consumer thread
   }
   if (*s_abort) {
     // give copies that may still be in flight time to land before the CTA's memory is released
-    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    for (int k = 0; k < 2000; ++k) __nanosleep(1000);
   }
 }
 
@@ -506,63 +640,49 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, u
 }
 
 // ---- host side ------------------------------------------------------------------------------------
+// Split length: the candidate that minimises rounds of the persistent grid x (tokens + fixed cost).
 static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
-  const long long items = (long long)bt->batch * cfg->n_kv_heads;
-  int len = kMaxSplit;
-  while (len > 128 && items * ((bt->max_seq_len + len - 1) / len) < 148 * 4) len >>= 1;
-  return len;
+  const long long per_split = (long long)bt->batch * cfg->n_kv_heads;
+  const int slots = 148 * kCtasPerSm;
+  int best = 128;
+  double best_cost = 1e300;
+  for (int len = 128; len <= kMaxSplit; len <<= 1) {
+    const long long items = per_split * std::max(1, (bt->max_seq_len + len - 1) / len);
+    const double rounds = (double)((items + slots - 1) / slots);
+    const double cost = rounds * (std::min(len, std::max(bt->max_seq_len, 1)) + 40.0);
+    if (cost < best_cost * 0.999) {
+      best_cost = cost;
+      best = len;
+    }
+  }
+  return best;
 }
 
 static size_t attn_smem_bytes(int split_len) {
-  return 1024 + (size_t)kStages * kStageBytes + (size_t)kMaxRows * (split_len + 8) * 4 + kMaxRows * kHeadDim * 4 +
-         kMaxRows * 64 * 4 + (kMaxSplit / 16) * 4 + 2 * kMaxRows * 4 + 8 * 4 + (2 * kStages + 1) * 8 + 64;
+  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kMaxRows * (split_len + 8) * 4;  // stages, S
+  b += 2 * kMaxRows * 64 * 4;                                                                // q_s
+  b += (size_t)kFixCap * kMaxRows * 4 + kFixCap * 4 + kMaxRows * 4;                          // kfix, kcol, knew
+  b += kMaxRows * kHeadDim * 4 + kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;           // oaux, m, l, red
+  b += 4 * 4 + (kMaxBatchSmem + 1) * 4 + 4 + 8 + (2 * kStages + 3) * 8 + 64;
+  return b;
 }
 
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets) {
   const int split_len = pick_split_len(cfg, bt);
-  const size_t n_splits = (size_t)max(1, (bt->max_seq_len + split_len - 1) / split_len);
+  const size_t n_splits = (size_t)std::max(1, (bt->max_seq_len + split_len - 1) / split_len);
   const size_t prow = (size_t)n_sets * bt->batch * cfg->n_q_heads * n_splits;
   return align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256);
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static mc_status encode_pool_map(CUtensorMap* tm, const void* pool, int dtype, int64_t n_rows, int page_size) {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    MC_CUDA_CHECK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr));
-    if (sym == nullptr || qr != cudaDriverEntryPointSuccess) {
-      set_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled entry point not found");
-      return MC_ERR_CUDA;
-    }
-    fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
-  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
-  const cuuint32_t box[2] = {64u, (cuuint32_t)page_size};
-  const cuuint32_t estr[2] = {1u, 1u};
-  const CUresult r = fn(tm, dtype == MC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                        const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled failed");
-    return MC_ERR_CUDA;
-  }
-  return MC_OK;
 }
 
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                              int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,
                              void* out, float* lse, void* workspace, cudaStream_t stream) {
   if (bt->batch == 0) return MC_OK;
+  if (bt->batch > kMaxBatchSmem) return MC_ERR_SHAPE;
   AttnParams ap;
   ap.g = g;
-  ap.scale = pair->scale;
+  ap.e_pool[0] = (const char*)pair->e_k;
+  ap.e_pool[1] = (const char*)pair->e_v;
   ap.ret_count = pair->ret_count;
   ap.ret_offset = pair->ret_offset;
   ap.ret_index = pair->ret_index;
@@ -578,29 +698,29 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.rows = ap.n_sets * ap.nq;
   ap.n_q_heads = cfg->n_q_heads;
   ap.split_len = pick_split_len(cfg, bt);
-  ap.n_splits = max(1, (bt->max_seq_len + ap.split_len - 1) / ap.split_len);
+  ap.n_splits = std::max(1, (bt->max_seq_len + ap.split_len - 1) / ap.split_len);
   const size_t prow = (size_t)ap.n_sets * bt->batch * cfg->n_q_heads * ap.n_splits;
   ap.part_o = reinterpret_cast<float*>(workspace);
   ap.part_ml = reinterpret_cast<float*>((char*)workspace + align_up(prow * kHeadDim * 4, 256));
 
-  CUtensorMap tm_k, tm_v;
-  const int64_t n_rows = bt->n_pages * cfg->n_kv_heads * cfg->page_size;
-  mc_status st = encode_pool_map(&tm_k, pair->e_k, cfg->dtype, n_rows, cfg->page_size);
-  if (st != MC_OK) return st;
-  st = encode_pool_map(&tm_v, pair->e_v, cfg->dtype, n_rows, cfg->page_size);
-  if (st != MC_OK) return st;
-
+  static int n_sm = 0;  // persistent grid: kCtasPerSm CTAs per SM of the current device
+  if (n_sm == 0) {
+    int dev = 0;
+    MC_CUDA_CHECK(cudaGetDevice(&dev));
+    MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const long long max_items = (long long)bt->batch * ap.n_splits * cfg->n_kv_heads;
+  const int grid = (int)std::min<long long>((long long)n_sm * kCtasPerSm, std::max<long long>(max_items, 1));
   const size_t smem = attn_smem_bytes(ap.split_len);
-  dim3 grid(ap.n_splits, cfg->n_kv_heads, bt->batch);
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_split_kernel<MC_F16><<<grid, kAttnThreads, smem, stream>>>(tm_k, tm_v, ap);
+    attn_split_kernel<MC_F16><<<grid, kAttnThreads, smem, stream>>>(ap);
     MC_CUDA_CHECK(cudaGetLastError());
     attn_combine_kernel<MC_F16><<<cgrid, 128, 0, stream>>>(ap, (unsigned short*)out, lse);
   } else {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_split_kernel<MC_BF16><<<grid, kAttnThreads, smem, stream>>>(tm_k, tm_v, ap);
+    attn_split_kernel<MC_BF16><<<grid, kAttnThreads, smem, stream>>>(ap);
     MC_CUDA_CHECK(cudaGetLastError());
     attn_combine_kernel<MC_BF16><<<cgrid, 128, 0, stream>>>(ap, (unsigned short*)out, lse);
   }

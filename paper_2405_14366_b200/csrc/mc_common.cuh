@@ -38,6 +38,15 @@ struct Geom {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Compressed tile of one (page, kv head, tensor) in the pair cache: page_size direction rows of
+// 256 bytes, then the two layers' scales [2][page_size] fp32.  Inside a row the sixteen 16-byte
+// chunks are permuted: chunk c of row r sits at position (c & 8) | ((c & 7) ^ (r & 7)).  A tile is
+// thus one contiguous block that a single bulk copy brings into shared memory in a layout where
+// eight consecutive rows of one chunk column fall into eight different bank groups (ldmatrix
+// without conflicts), and the scales a layer needs arrive with it.
+__host__ __device__ inline int tile_bytes(int page_size) { return page_size * kRowBytes + 2 * page_size * 4; }
+__host__ __device__ inline int chunk_pos(int r, int c) { return (c & 8) | ((c & 7) ^ (r & 7)); }
+
 // 16-bit storage types ---------------------------------------------------------
 template <int DT>
 struct Elem;

@@ -16,8 +16,7 @@ struct MergeParams {
   Geom g;
   const char* a_pool[2];  // layer l-1: K, V
   const char* c_pool[2];  // layer l:   K, V
-  char* e_pool[2];
-  float* scale;
+  char* e_pool[2];  // compressed tiles (see tile_bytes)
   float* dist;
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
   float ta, tc;
@@ -118,7 +117,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams 
   const size_t page_off = (size_t)page * rows_in_page;
   const char* pa = p.a_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
   const char* pc = p.c_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
-  char* pe = p.e_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
+  char* tile = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
 
   uint4 va[kRowsPerHalfWarp], vc[kRowsPerHalfWarp];
   bool valid[kRowsPerHalfWarp];
@@ -140,7 +139,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams 
     uint4 e;
     merge_row<DT>(va[j], vc[j], p.ta, p.tc, e, ga[j], gc[j], dd[j]);
     if (valid[j]) {
-      st_stream16(pe + j * kRowBytes, e);
+      st_stream16(tile + (tk0 + j) * kRowBytes + chunk_pos(tk0 + j, l16) * 16, e);
       dmin = fminf(dmin, dd[j]);
       dmax = fmaxf(dmax, dd[j]);
     }
@@ -159,7 +158,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams 
       }
     if (ok) {
       const size_t ph = (size_t)page * H + head;
-      float* sc = p.scale + (ph * 4 + tensor * 2) * ps + tk0 + l16;
+      float* sc = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk0 + l16;
       sc[0] = g_a;
       sc[ps] = g_c;
       p.dist[(ph * 2 + tensor) * ps + tk0 + l16] = d;
@@ -192,6 +191,7 @@ struct RetainParams {
   Geom g;
   const char* a_pool[2];
   const char* c_pool[2];
+  char* e_pool[2];
   const float* dist;
   const float* seg_minmax;
   int32_t* chunk_count;   // workspace [nseg][chunks_per_seg]
@@ -329,7 +329,16 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     __syncthreads();
     int before = s_base;
     for (int w = 0; w < warp; ++w) before += s_warp[w];
-    if (keep) p.ret_index[out0 + before + __popc(m & ((1u << lane) - 1))] = tok;
+    if (keep) {
+      p.ret_index[out0 + before + __popc(m & ((1u << lane) - 1))] = tok;
+      // a retained token is served from its raw rows: its scales are never read again, and zero
+      // makes the shared direction contribute nothing for it wherever scales are applied blindly
+      const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+      float* sc = reinterpret_cast<float*>(p.e_pool[tensor] + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
+                                           p.g.page_size * kRowBytes) + (tok & (p.g.page_size - 1));
+      sc[0] = 0.f;
+      sc[p.g.page_size] = 0.f;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
       int t = s_base;
@@ -359,7 +368,6 @@ struct AppendParams {
   const char* a_new[2];  // [batch][H][128]: K, V of layer l-1
   const char* c_new[2];
   char* e_pool[2];
-  float* scale;
   float* dist;
   float ta, tc;
   int total_rows;  // 2 * batch * H
@@ -389,9 +397,10 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
   const int tk = tok & (p.g.page_size - 1);
   const size_t ph = (size_t)page * H + h;
-  *reinterpret_cast<uint4*>(p.e_pool[tensor] + (ph * p.g.page_size + tk) * kRowBytes + l16 * 16) = e;
+  char* tile = p.e_pool[tensor] + ph * tile_bytes(p.g.page_size);
+  *reinterpret_cast<uint4*>(tile + tk * kRowBytes + chunk_pos(tk, l16) * 16) = e;
   if (l16 == 0) {
-    float* sc = p.scale + (ph * 4 + tensor * 2) * p.g.page_size + tk;
+    float* sc = reinterpret_cast<float*>(tile + p.g.page_size * kRowBytes) + tk;
     sc[0] = ga;
     sc[p.g.page_size] = gc;
     p.dist[(ph * 2 + tensor) * p.g.page_size + tk] = d;
@@ -425,7 +434,6 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   mp.c_pool[1] = (const char*)l->v_pool;
   mp.e_pool[0] = (char*)out->e_k;
   mp.e_pool[1] = (char*)out->e_v;
-  mp.scale = out->scale;
   mp.dist = out->dist;
   mp.seg_minmax = reinterpret_cast<unsigned*>(out->seg_minmax);
   mp.ta = (float)(1.0 - cfg->t);
@@ -447,6 +455,8 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.a_pool[1] = mp.a_pool[1];
   rp.c_pool[0] = mp.c_pool[0];
   rp.c_pool[1] = mp.c_pool[1];
+  rp.e_pool[0] = mp.e_pool[0];
+  rp.e_pool[1] = mp.e_pool[1];
   rp.dist = out->dist;
   rp.seg_minmax = out->seg_minmax;
   rp.chunks_per_seg = chunks_per_seg(bt->max_seq_len);
@@ -484,7 +494,6 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   ap.c_new[1] = (const char*)v_new_l;
   ap.e_pool[0] = (char*)pair->e_k;
   ap.e_pool[1] = (char*)pair->e_v;
-  ap.scale = pair->scale;
   ap.dist = pair->dist;
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;

@@ -14,7 +14,6 @@ struct RestoreParams {
   Geom g;
   const char* e_pool[2];
   char* dst_pool[2];
-  const float* scale;
   const int32_t* ret_count;
   const int32_t* ret_offset;
   const int32_t* ret_index;
@@ -46,15 +45,15 @@ __global__ void __launch_bounds__(kRestoreThreads) restore_scale_kernel(const Re
   const int tk0 = row0 & (ps - 1);
   const int tok0 = pslot * ps + tk0;
   const size_t page_off = (size_t)page * rows_in_page;
-  const char* pe = p.e_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
+  const char* tile = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
   char* pd = p.dst_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
-  const float* sc = p.scale + (((size_t)page * H + head) * 4 + tensor * 2 + p.layer) * ps + tk0;
+  const float* sc = reinterpret_cast<const float*>(tile + ps * kRowBytes) + p.layer * ps + tk0;
   uint4 v[kRowsPerHalfWarp];
   float g[kRowsPerHalfWarp];
 #pragma unroll
   for (int j = 0; j < kRowsPerHalfWarp; ++j)
     if (tok0 + j < n) {
-      v[j] = ld_stream16(pe + j * kRowBytes);
+      v[j] = ld_stream16(tile + (tk0 + j) * kRowBytes + chunk_pos(tk0 + j, l16) * 16);
       g[j] = __ldg(sc + j);
     }
 #pragma unroll
@@ -99,7 +98,6 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
   rp.e_pool[1] = (const char*)pair->e_v;
   rp.dst_pool[0] = (char*)dst->k_pool;
   rp.dst_pool[1] = (char*)dst->v_pool;
-  rp.scale = pair->scale;
   rp.ret_count = pair->ret_count;
   rp.ret_offset = pair->ret_offset;
   rp.ret_index = pair->ret_index;

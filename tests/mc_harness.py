@@ -75,8 +75,8 @@ class Problem:
         return self.lib.mc_read_status(self.pair, check=False)
 
     def run_restore(self, layer: int):
-        dk = torch.zeros_like(self.pair.e_k)
-        dv = torch.zeros_like(self.pair.e_v)
+        dk = torch.zeros(self.n_pages, self.H, self.ps, 128, dtype=self.cfg.torch_dtype, device=self.device)
+        dv = torch.zeros_like(dk)
         self.lib.mc_restore(self.cfg, self.batch(), self.pair, layer, dk, dv)
         torch.cuda.synchronize()
         return dk, dv
@@ -99,8 +99,9 @@ class Problem:
         """The compressed pair read back into logical numpy arrays."""
         S = self.S + extra_tokens
         pc = self.pair
-        out = {"e_k": as_bits(self.logical_of(pc.e_k, S)), "e_v": as_bits(self.logical_of(pc.e_v, S))}
-        sc = gen.from_paged(pc.scale.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()  # [B][S][H][4]
+        out = {"e_k": as_bits(self.logical_of(pc.directions("k"), S)), "e_v": as_bits(self.logical_of(pc.directions("v"), S))}
+        scale = torch.cat([pc.scales("k"), pc.scales("v")], dim=2)  # [n_pages][H][4][ps]: K l-1, K l, V l-1, V l
+        sc = gen.from_paged(scale.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()  # [B][S][H][4]
         ds = gen.from_paged(pc.dist.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()   # [B][S][H][2]
         out["scale"], out["dist"] = sc.astype(np.float64), ds.astype(np.float64)
         out["ret_count"] = pc.ret_count.cpu().numpy().reshape(2, self.B, self.H)
@@ -155,14 +156,20 @@ def compare_merge(p: Problem, om, dc, mode: str = "distinct", do_retention: bool
         total = int(valid.sum()) * p.H * 128
         stats[f"{tn}_flip_frac"] = nflip / max(total, 1)
         assert nflip <= max(8, 5e-3 * total), f"too many rounding flips: {nflip}/{total}"
-        # scales: |x| / |e_stored| with the oracle's own stored direction
+        # scales: |x| / |e_stored| with the oracle's own stored direction; zero where the device retained
+        # the token (its raw rows serve it instead)
+        ret_mask = np.zeros((p.B, p.S, p.H), bool)
+        for b in range(p.B):
+            for h in range(p.H):
+                ret_mask[b, p.retained(dc, ti, b, h)[0], h] = True
         len_e = np.sqrt(np.sum(e_orc * e_orc, -1))
         len_e = np.where(len_e == 0, 1.0, len_e)
         row_flip = flips.any(-1)
         for li, nm in enumerate(("n_lm1", "n_l")):
             want = o[nm] / len_e
             got = dc["scale"][..., ti * 2 + li]
-            rel = np.abs(got - want) / np.maximum(np.abs(want), 1e-30) * valid[:, :, None]
+            assert np.all(got[ret_mask] == 0.0), "scale of a retained token must be zero"
+            rel = np.abs(got - want) / np.maximum(np.abs(want), 1e-30) * valid[:, :, None] * ~ret_mask
             clean = rel * ~row_flip
             stats[f"{tn}_scale_rel"] = max(stats.get(f"{tn}_scale_rel", 0.0), float(clean.max(initial=0.0)))
             assert clean.max(initial=0.0) < 2e-6, f"scale mismatch {clean.max()}"
