@@ -129,6 +129,10 @@ typedef struct mc_layer_kv {
  * ret_offset [2 * batch * n_kv_heads + 1] exclusive prefix of ret_count = first slot of the segment
  * ret_index  [ret_capacity] token indices, ascending inside a segment
  * ret_rows   [ret_capacity][2][128] raw 16-bit rows: [.][0] layer l-1, [.][1] layer l (bit copies)
+ * ret_prefix [2 * batch * n_kv_heads][ret_prefix_stride]: entry j = how many of the segment's retained
+ *            tokens lie before token 128 * j (so a token range maps to a range of the segment's list
+ *            without searching).  ret_prefix_stride (a host-side number, fixed when the pair is merged)
+ *            must be at least ceil(max_seq_len at merge / 128) + 1.
  * seg_minmax [2 * batch * n_kv_heads][2] fp32 d_min, d_max of the prefill tokens
  * status     [MC_STATUS_WORDS] int32 */
 typedef struct mc_pair_cache {
@@ -140,6 +144,8 @@ typedef struct mc_pair_cache {
   int32_t* ret_index;
   void* ret_rows;
   int64_t ret_capacity;
+  int32_t* ret_prefix;
+  int64_t ret_prefix_stride;
   float* seg_minmax;
   int32_t* status;
 } mc_pair_cache;

@@ -48,7 +48,8 @@ class _LayerKV(C.Structure):
 class _PairCache(C.Structure):
     _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("dist", C.c_void_p),
                 ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
-                ("ret_rows", C.c_void_p), ("ret_capacity", C.c_int64), ("seg_minmax", C.c_void_p),
+                ("ret_rows", C.c_void_p), ("ret_capacity", C.c_int64), ("ret_prefix", C.c_void_p),
+                ("ret_prefix_stride", C.c_int64), ("seg_minmax", C.c_void_p),
                 ("status", C.c_void_p)]
 
 
@@ -106,7 +107,8 @@ class Batch:
 class PairCache:
     """Caller-owned device buffers of one compressed layer pair (allocated with torch)."""
 
-    def __init__(self, cfg: McConfig, batch: int, n_pages: int, ret_capacity: int, device="cuda"):
+    def __init__(self, cfg: McConfig, batch: int, n_pages: int, ret_capacity: int, device="cuda",
+                 max_merge_len: Optional[int] = None):
         H, ps = cfg.n_kv_heads, cfg.page_size
         dt = cfg.torch_dtype
         self.cfg = cfg
@@ -120,13 +122,17 @@ class PairCache:
         self.ret_index = torch.zeros(max(ret_capacity, 1), dtype=torch.int32, device=device)
         self.ret_rows = torch.zeros(max(ret_capacity, 1), 2, 128, dtype=dt, device=device)
         self.ret_capacity = int(ret_capacity)
+        if max_merge_len is None:  # bound of the sequence length at merge time: what the pages can hold at most
+            max_merge_len = n_pages * ps
+        self.ret_prefix_stride = (int(max_merge_len) + 127) // 128 + 1
+        self.ret_prefix = torch.zeros(nseg, self.ret_prefix_stride, dtype=torch.int32, device=device)
         self.seg_minmax = torch.zeros(nseg, 2, dtype=torch.float32, device=device)
         self.status = torch.zeros(MC_STATUS_WORDS, dtype=torch.int32, device=device)
 
     def c(self) -> _PairCache:
         return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.dist), _ptr(self.ret_count),
                           _ptr(self.ret_offset), _ptr(self.ret_index), _ptr(self.ret_rows), self.ret_capacity,
-                          _ptr(self.seg_minmax), _ptr(self.status))
+                          _ptr(self.ret_prefix), self.ret_prefix_stride, _ptr(self.seg_minmax), _ptr(self.status))
 
     # -- decoding the tile layout (pure re-indexing, no arithmetic) ------------------------------
     def directions(self, tensor: str) -> torch.Tensor:
@@ -152,7 +158,7 @@ class PairCache:
 
     def nbytes(self) -> int:
         ts = (self.e_k, self.e_v, self.dist, self.ret_count, self.ret_offset, self.ret_index,
-              self.ret_rows, self.seg_minmax, self.status)
+              self.ret_rows, self.ret_prefix, self.seg_minmax, self.status)
         return sum(t.numel() * t.element_size() for t in ts)
 
 

@@ -44,7 +44,7 @@ static mc_status check_pair(const mc_pair_cache* pc) {
   if (!pc->e_k || !pc->e_v || !pc->dist || !pc->ret_count || !pc->ret_offset || !pc->seg_minmax ||
       !pc->status)
     return MC_ERR_INVALID_ARG;
-  if (pc->ret_capacity < 0) return MC_ERR_INVALID_ARG;
+  if (pc->ret_capacity < 0 || pc->ret_prefix == nullptr || pc->ret_prefix_stride < 2) return MC_ERR_INVALID_ARG;
   if (pc->ret_capacity > 0 && (!pc->ret_index || !pc->ret_rows)) return MC_ERR_INVALID_ARG;
   if (!aligned256(pc->e_k) || !aligned256(pc->e_v) || !aligned256(pc->dist)) return MC_ERR_ALIGN;
   if (pc->ret_rows && !aligned256(pc->ret_rows)) return MC_ERR_ALIGN;
@@ -120,6 +120,7 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
   if (do_retention && cfg->retain_mode == MC_RETAIN_TOPK) return MC_ERR_UNSUPPORTED;
   if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
   if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
+  if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
   return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, out, do_retention ? 1 : 0, workspace,
                       (cudaStream_t)stream);
 }

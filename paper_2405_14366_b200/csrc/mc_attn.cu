@@ -36,7 +36,7 @@ constexpr int kMaxRows = 8;                          // query rows per work item
 constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
 constexpr int kMaxSplit = 512;
 constexpr int kFixCap = 128;  // retained-K entries per item whose scores the auxiliary warp pre-computes
-constexpr int kMaxBatchSmem = 1024;
+constexpr int kMaxBatchSmem = 512;
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kCtasPerSm = 2;
 
@@ -46,6 +46,8 @@ struct AttnParams {
   const int32_t* ret_count;
   const int32_t* ret_offset;
   const int32_t* ret_index;
+  const int32_t* ret_prefix;
+  int ret_prefix_stride;
   const char* ret_rows;
   const char* q;
   const char* k_new;
@@ -151,7 +153,7 @@ struct Item {
 
 // Item `i` of the flattened list (sequence-major, then split, then kv head) from the per-sequence
 // prefix of split counts in shared memory.
-__device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, const AttnParams& p) {
+__device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, const int* len_s, const AttnParams& p) {
   Item it;
   it.valid = i < total;
   if (!it.valid) {
@@ -169,7 +171,7 @@ __device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, con
   const int local = i - pre_s[lo] * H;
   it.split = local / H;
   it.g = local - it.split * H;
-  const int n = p.g.seq_lens[lo];
+  const int n = len_s[lo];
   const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
   it.split_start = it.split * p.split_len;
   it.n_tok = max(0, min(n, it.split_start + p.split_len) - it.split_start);
@@ -178,8 +180,127 @@ __device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, con
   return it;
 }
 
+// Shared-memory views and loop constants the auxiliary warp's K part needs.
+struct AuxCtx {
+  float* kfix_s;
+  int* kcol_s;
+  float* knew_s;
+  float* aq_s;
+  int* aux_info;
+  const int* pre_s;
+  const int* len_s;
+  uint32_t kfix_bar;
+  int total_items, H, rows, nslots, lane;
+};
+
+// K part of the auxiliary warp for item i (the n-th item of this CTA): scores of the split's retained
+// K rows and of the new token into buffer n & 1, then the buffer's barrier.
 template <int DT>
-__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnParams p) {
+__device__ __noinline__ void aux_k_part(const AttnParams& p, const AuxCtx& x, int i, int n) {
+  float* const kfix_s = x.kfix_s;
+  int* const kcol_s = x.kcol_s;
+  float* const knew_s = x.knew_s;
+  float* const aq_s = x.aq_s;
+  int* const aux_info = x.aux_info;
+  const int* pre_s = x.pre_s;
+  const int* len_s = x.len_s;
+  const uint32_t kfix_bar = x.kfix_bar;
+  const int total_items = x.total_items, H = x.H, rows = x.rows, nslots = x.nslots, lane = x.lane;
+    const Item w = get_item(i, total_items, pre_s, len_s, p);
+    if (!w.valid) return;
+    const int buf = n & 1;
+    float* kfix = kfix_s + buf * kFixCap * kMaxRows;
+    int* kcol = kcol_s + buf * kFixCap;
+    const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
+    // ranges of the two retained lists whose tokens lie in this split: two table entries each
+    // (split boundaries are multiples of 128; no retained token lies past the merged length)
+    const int pj0 = min(w.split_start >> 7, p.ret_prefix_stride - 1);
+    const int pj1 = min((w.split_start + w.n_tok + 127) >> 7, p.ret_prefix_stride - 1);
+    const int32_t* pk = p.ret_prefix + (size_t)seg_k * p.ret_prefix_stride;
+    const int32_t* pv = p.ret_prefix + (size_t)seg_v * p.ret_prefix_stride;
+    const int off_k = __ldg(p.ret_offset + seg_k), off_v = __ldg(p.ret_offset + seg_v);
+    const int k_lo = off_k + __ldg(pk + pj0), k_hi = off_k + __ldg(pk + pj1);
+    const int v_lo = off_v + __ldg(pv + pj0), v_hi = off_v + __ldg(pv + pj1);
+    const int n_fast = min(k_hi - k_lo, kFixCap);
+    const int n_new = w.has_new ? 1 : 0;
+    if (n_fast + n_new > 0) {
+      // one lane per retained row (or the new token): full 128-channel dot products
+#pragma unroll
+      for (int r = 0; r < kMaxRows; ++r) {
+        if (r < rows) {
+          const int set = r / p.nq, rq = r - set * p.nq;
+          const size_t qrow = ((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq;
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(p.q + qrow * kRowBytes + lane * 8));
+          const float2 a = Elem<DT>::unpack(v.x), c = Elem<DT>::unpack(v.y);
+          *reinterpret_cast<float4*>(aq_s + r * kHeadDim + lane * 4) = make_float4(a.x, a.y, c.x, c.y);
+        }
+      }
+      __syncwarp();
+      for (int base = 0; base < n_fast + n_new; base += 32) {
+        const int e = base + lane;
+        const bool act = e < n_fast + n_new;
+        const bool is_new = e >= n_fast;
+        if (act) {
+          const int col = is_new ? w.n_tok : __ldg(p.ret_index + k_lo + e) - w.split_start;
+          float dots[kMaxRows];
+#pragma unroll
+          for (int r = 0; r < kMaxRows; ++r) dots[r] = 0.f;
+#pragma unroll
+          for (int set = 0; set < 2; ++set) {
+            if (set < nslots) {
+              const char* src = is_new ? p.k_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
+                                       : p.ret_rows + ((size_t)(k_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
+              const int r_lo = nslots == 2 ? set * p.nq : 0, r_hi = nslots == 2 ? r_lo + p.nq : rows;
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                uint4 kv[8];  // half a row in flight at once
+#pragma unroll
+                for (int c = 0; c < 8; ++c) kv[c] = ld_stream16(src + (half * 8 + c) * 16);
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                  const int c = half * 8 + cc;
+                  const float2 x0 = Elem<DT>::unpack(kv[cc].x), x1 = Elem<DT>::unpack(kv[cc].y);
+                  const float2 x2 = Elem<DT>::unpack(kv[cc].z), x3 = Elem<DT>::unpack(kv[cc].w);
+#pragma unroll
+                  for (int r = 0; r < kMaxRows; ++r) {
+                    if (r >= r_lo && r < r_hi) {
+                      const float4 q0 = *reinterpret_cast<const float4*>(aq_s + r * kHeadDim + c * 8);
+                      const float4 q1 = *reinterpret_cast<const float4*>(aq_s + r * kHeadDim + c * 8 + 4);
+                      dots[r] += x0.x * q0.x + x0.y * q0.y + x1.x * q0.z + x1.y * q0.w + x2.x * q1.x +
+                                 x2.y * q1.y + x3.x * q1.z + x3.y * q1.w;
+                    }
+                  }
+                }
+              }
+            }
+          }
+          if (is_new) {
+#pragma unroll
+            for (int r = 0; r < kMaxRows; ++r)
+              if (r < rows) knew_s[buf * kMaxRows + r] = dots[r] * p.scale_log2;
+          } else {
+            kcol[e] = col;
+#pragma unroll
+            for (int r = 0; r < kMaxRows; ++r)
+              if (r < rows) kfix[e * kMaxRows + r] = dots[r] * p.scale_log2;
+          }
+        }
+      }
+    }
+    if (lane == 0) {
+      int* info = aux_info + buf * 8;
+      info[0] = n_fast;
+      info[1] = k_lo;
+      info[2] = k_hi;
+      info[3] = v_lo;
+      info[4] = v_hi;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(kfix_bar + 8 * buf);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(const AttnParams p) {
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
   const int tbytes = tile_bytes(ps);
@@ -192,19 +313,21 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
   unsigned char* stages = smem;
   float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);  // [kMaxRows][s_stride]
   uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kMaxRows * s_stride);  // [2][kMaxRows][64] packed pairs
-  float* kfix_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);     // [kFixCap][kMaxRows]
-  int* kcol_s = reinterpret_cast<int*>(kfix_s + kFixCap * kMaxRows);     // [kFixCap]
-  float* knew_s = reinterpret_cast<float*>(kcol_s + kFixCap);            // [kMaxRows]
-  float* oaux_s = knew_s + kMaxRows;                                     // [kMaxRows][128]
+  float* kfix_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);     // [2][kFixCap][kMaxRows]
+  int* kcol_s = reinterpret_cast<int*>(kfix_s + 2 * kFixCap * kMaxRows);  // [2][kFixCap]
+  float* knew_s = reinterpret_cast<float*>(kcol_s + 2 * kFixCap);        // [2][kMaxRows]
+  float* oaux_s = knew_s + 2 * kMaxRows;                                 // [kMaxRows][128]
   float* m_s = oaux_s + kMaxRows * kHeadDim;                             // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
-  int* aux_info = reinterpret_cast<int*>(red_s + kMaxRows * kConsumerWarps);  // n_fast, k_lo, k_hi, pad
-  int* pre_s = aux_info + 4;                                                  // [batch + 1] split-count prefix
-  volatile int* s_abort = pre_s + kMaxBatchSmem + 1;
+  float* aq_s = red_s + kMaxRows * kConsumerWarps;                       // [kMaxRows][128] query rows of the auxiliary warp
+  int* aux_info = reinterpret_cast<int*>(aq_s + kMaxRows * kHeadDim);    // [2][8]: n_fast, k_lo, k_hi, v_lo, v_hi
+  int* pre_s = aux_info + 16;                                            // [batch + 1] split-count prefix
+  int* len_s = pre_s + kMaxBatchSmem + 1;                                // [batch] sequence lengths
+  volatile int* s_abort = len_s + kMaxBatchSmem;
   uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
-  const uint32_t kfix_bar = full0 + 16 * kStages, pready_bar = kfix_bar + 8, oaux_bar = kfix_bar + 16;
+  const uint32_t kfix_bar = full0 + 16 * kStages, pready_bar = kfix_bar + 16, oaux_bar = kfix_bar + 24;  // kfix_bar[2]
   const uint32_t stage0 = smem_u32(stages);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -216,6 +339,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
       mbar_init(empty0 + 8 * s, kConsumerWarps);
     }
     mbar_init(kfix_bar, 1);
+    mbar_init(kfix_bar + 8, 1);
     mbar_init(pready_bar, 1);
     mbar_init(oaux_bar, 1);
     *s_abort = 0;
@@ -223,8 +347,10 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
     // prefix of per-sequence split counts (a sequence always owns at least one split)
     int acc = 0;
     for (int b = 0; b < p.g.batch; ++b) {
+      const int n = p.g.seq_lens[b];
+      len_s[b] = n;
       pre_s[b] = acc;
-      acc += max(1, (p.g.seq_lens[b] + p.split_len - 1) / p.split_len);
+      acc += max(1, (n + p.split_len - 1) / p.split_len);
     }
     pre_s[p.g.batch] = acc;
   }
@@ -236,7 +362,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
     // ===================== producer =====================
     int it = 0;  // running stage counter, same sequence as the consumers'
     for (int i = first; i < total_items; i += stride) {
-      const Item w = get_item(i, total_items, pre_s, p);
+      const Item w = get_item(i, total_items, pre_s, len_s, p);
       // page ids of the item's pages, one per lane (split_len / page_size <= 32)
       const int n_pages_item = (w.n_tok + ps - 1) >> shift;
       int my_page = 0;
@@ -272,106 +398,66 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
 
   if (warp == kConsumerWarps + 1) {
     // ===================== auxiliary warp: retained rows and the new token =====================
+    // Software pipeline over this CTA's items n = 0, 1, 2, ...:
+    //   K part of item n + 2 (scores of its retained K rows and of its new token; needs nothing
+    //   from the consumers, so it runs two items ahead into a double buffer), then, once the
+    //   consumers have published item n's probabilities, the V part of item n.
+    // All global loads here are latency-bound while the copy engine saturates the memory system,
+    // which is why nothing the consumers wait for is started late.
+    AuxCtx ax;
+    ax.kfix_s = kfix_s; ax.kcol_s = kcol_s; ax.knew_s = knew_s; ax.aq_s = aq_s; ax.aux_info = aux_info;
+    ax.pre_s = pre_s; ax.len_s = len_s; ax.kfix_bar = kfix_bar;
+    ax.total_items = total_items; ax.H = H; ax.rows = rows; ax.nslots = nslots; ax.lane = lane;
+    auto k_part = [&](int i, int n) { aux_k_part<DT>(p, ax, i, n); };
+    k_part(first, 0);
+    k_part(first + stride, 1);
     int n_item = 0;
     for (int i = first; i < total_items; i += stride, ++n_item) {
-      const Item w = get_item(i, total_items, pre_s, p);
-      const uint32_t par = n_item & 1;
-      const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
-      // ranges of the retained lists whose tokens lie in this split (all lanes search alike)
-      int rng[2][2];
-#pragma unroll
-      for (int tz = 0; tz < 2; ++tz) {
-        const int seg = tz ? seg_v : seg_k;
-        const int cnt = p.ret_count[seg], off = p.ret_offset[seg];
-        int lo = 0, hi = cnt;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (p.ret_index[off + mid] < w.split_start) lo = mid + 1; else hi = mid;
-        }
-        const int firstp = lo;
-        hi = cnt;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (p.ret_index[off + mid] < w.split_start + w.n_tok) lo = mid + 1; else hi = mid;
-        }
-        rng[tz][0] = off + firstp;
-        rng[tz][1] = off + lo;
-      }
-      const int n_k = rng[0][1] - rng[0][0], n_v = rng[1][1] - rng[1][0];
-      const int n_fast = min(n_k, kFixCap);
-      // query rows, 4 channels per lane
-      float qf[kMaxRows][4];
-      if (n_k > 0 || w.has_new) {
-#pragma unroll
-        for (int r = 0; r < kMaxRows; ++r) {
-          if (r < rows) {
-            const int set = r / p.nq, rq = r - set * p.nq;
-            const size_t qrow = ((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq;
-            const uint2 v = *reinterpret_cast<const uint2*>(p.q + qrow * kRowBytes + lane * 8);
-            const float2 a = Elem<DT>::unpack(v.x), c = Elem<DT>::unpack(v.y);
-            qf[r][0] = a.x; qf[r][1] = a.y; qf[r][2] = c.x; qf[r][3] = c.y;
-          }
-        }
-      }
-      // ---- K part: scores of retained rows (first kFixCap of them) and of the new token
-      for (int e = 0; e < n_fast + (w.has_new ? 1 : 0); ++e) {
-        const bool is_new = e >= n_fast;
-        const int col = is_new ? w.n_tok : p.ret_index[rng[0][0] + e] - w.split_start;
-#pragma unroll
-        for (int r = 0; r < kMaxRows; ++r) {
-          if (r < rows) {
-            const int set = r / p.nq;
-            const char* src = is_new ? p.k_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
-                                     : p.ret_rows + ((size_t)(rng[0][0] + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-            const uint2 kv = *reinterpret_cast<const uint2*>(src + lane * 8);
-            const float2 k0 = Elem<DT>::unpack(kv.x), k1 = Elem<DT>::unpack(kv.y);
-            float d = qf[r][0] * k0.x + qf[r][1] * k0.y + qf[r][2] * k1.x + qf[r][3] * k1.y;
-            for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-            if (lane == 0) {
-              if (is_new) knew_s[r] = d * p.scale_log2; else kfix_s[e * kMaxRows + r] = d * p.scale_log2;
-            }
-          }
-        }
-        if (lane == 0 && !is_new) kcol_s[e] = col;
-      }
-      if (lane == 0) {
-        aux_info[0] = n_fast;
-        aux_info[1] = rng[0][0];
-        aux_info[2] = rng[0][1];
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(kfix_bar);
-      // ---- V part: after the softmax, add the retained V rows' and the new token's terms
+      const Item w = get_item(i, total_items, pre_s, len_s, p);
+      const int v_lo = aux_info[(n_item & 1) * 8 + 3], v_hi = aux_info[(n_item & 1) * 8 + 4];
+      const int n_v = v_hi - v_lo, n_new = w.has_new ? 1 : 0;
+      // ---- V part: after the softmax, add the retained V rows' and the new token's terms (lane = 4 channels)
+      int my_col = 0;  // first batch of token columns, loaded before the wait
+      if (lane < min(32, n_v + n_new)) my_col = lane >= n_v ? w.n_tok : __ldg(p.ret_index + v_lo + lane) - w.split_start;
       int good = 1;
-      if (lane == 0) good = mbar_wait(pready_bar, par, s_abort, p.status) ? 1 : 0;
+      if (lane == 0) good = mbar_wait(pready_bar, n_item & 1, s_abort, p.status) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
       float oa[kMaxRows][4];
 #pragma unroll
       for (int r = 0; r < kMaxRows; ++r) oa[r][0] = oa[r][1] = oa[r][2] = oa[r][3] = 0.f;
-      for (int e = 0; e < n_v + (w.has_new ? 1 : 0); ++e) {
-        const bool is_new = e >= n_v;
-        const int col = is_new ? w.n_tok : p.ret_index[rng[1][0] + e] - w.split_start;
-        float val[2][4];
-#pragma unroll
-        for (int set = 0; set < 2; ++set) {
-          if (set < nslots) {
-            const char* src = is_new ? p.v_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
-                                     : p.ret_rows + ((size_t)(rng[1][0] + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-            const uint2 vv = *reinterpret_cast<const uint2*>(src + lane * 8);
-            const float2 a = Elem<DT>::unpack(vv.x), c = Elem<DT>::unpack(vv.y);
-            val[set][0] = a.x; val[set][1] = a.y; val[set][2] = c.x; val[set][3] = c.y;
-          } else {
-            val[set][0] = val[set][1] = val[set][2] = val[set][3] = 0.f;
-          }
+      for (int base = 0; base < n_v + n_new; base += 32) {
+        const int cnt = min(32, n_v + n_new - base);
+        if (base > 0) {
+          my_col = 0;
+          if (lane < cnt) my_col = (base + lane) >= n_v ? w.n_tok : __ldg(p.ret_index + v_lo + base + lane) - w.split_start;
         }
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+          const int e = base + j;
+          const bool is_new = e >= n_v;
+          const int col = __shfl_sync(0xffffffffu, my_col, j);
+          float val[2][4];
 #pragma unroll
-        for (int r = 0; r < kMaxRows; ++r) {
-          if (r < rows) {
-            const float pr = S[r * s_stride + col];
-            const int set = nslots == 2 ? r / p.nq : 0;
+          for (int set = 0; set < 2; ++set) {
+            if (set < nslots) {
+              const char* src = is_new ? p.v_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
+                                       : p.ret_rows + ((size_t)(v_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
+              const uint2 vv = __ldg(reinterpret_cast<const uint2*>(src + lane * 8));
+              const float2 a = Elem<DT>::unpack(vv.x), c = Elem<DT>::unpack(vv.y);
+              val[set][0] = a.x; val[set][1] = a.y; val[set][2] = c.x; val[set][3] = c.y;
+            } else {
+              val[set][0] = val[set][1] = val[set][2] = val[set][3] = 0.f;
+            }
+          }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) oa[r][k] = fmaf(pr, set ? val[1][k] : val[0][k], oa[r][k]);
+          for (int r = 0; r < kMaxRows; ++r) {
+            if (r < rows) {
+              const float pr = S[r * s_stride + col];
+              const bool second = nslots == 2 && r >= p.nq;
+#pragma unroll
+              for (int k = 0; k < 4; ++k) oa[r][k] = fmaf(pr, second ? val[1][k] : val[0][k], oa[r][k]);
+            }
           }
         }
       }
@@ -380,6 +466,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
         if (r < rows) *reinterpret_cast<float4*>(oaux_s + r * kHeadDim + lane * 4) = make_float4(oa[r][0], oa[r][1], oa[r][2], oa[r][3]);
       __syncwarp();
       if (lane == 0) mbar_arrive(oaux_bar);
+      k_part(i + 2 * stride, n_item + 2);
     }
     return;
   }
@@ -408,14 +495,14 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
   };
   {
     uint32_t qw[4];
-    load_q_words(get_item(first, total_items, pre_s, p), qw);
+    load_q_words(get_item(first, total_items, pre_s, len_s, p), qw);
 #pragma unroll
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
   consumer_sync();
 
   for (int i = first; i < total_items; i += stride, ++n_item) {
-    const Item w = get_item(i, total_items, pre_s, p);
+    const Item w = get_item(i, total_items, pre_s, len_s, p);
     const uint32_t par = n_item & 1;
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
     const int n_cols = w.n_tok + (w.has_new ? 1 : 0);
@@ -468,14 +555,15 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
     consumer_sync();
 
     // ---- retained K rows and the new token replace / add single scores ----------------------------
-    if (ok && !mbar_wait(kfix_bar, par, s_abort, p.status)) ok = false;
+    const int kb = n_item & 1;
+    if (ok && !mbar_wait(kfix_bar + 8 * kb, (n_item >> 1) & 1, s_abort, p.status)) ok = false;
     if (ok) {
-      const int n_fast = aux_info[0], k_lo = aux_info[1], k_hi = aux_info[2];
+      const int n_fast = aux_info[kb * 8], k_lo = aux_info[kb * 8 + 1], k_hi = aux_info[kb * 8 + 2];
       for (int e = tid; e < n_fast; e += kConsumerThreads) {
-        const int col = kcol_s[e];
-        for (int r = 0; r < rows; ++r) S[r * s_stride + col] = kfix_s[e * kMaxRows + r];
+        const int col = kcol_s[kb * kFixCap + e];
+        for (int r = 0; r < rows; ++r) S[r * s_stride + col] = kfix_s[(kb * kFixCap + e) * kMaxRows + r];
       }
-      if (w.has_new && tid < rows) S[tid * s_stride + w.n_tok] = knew_s[tid];
+      if (w.has_new && tid < rows) S[tid * s_stride + w.n_tok] = knew_s[kb * kMaxRows + tid];
       // more retained rows than the auxiliary warp pre-computes: finish them here
       for (int e = k_lo + n_fast + warp; e < k_hi; e += kConsumerWarps) {
         const int col = p.ret_index[e] - w.split_start;
@@ -525,7 +613,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const AttnPara
 
     // query rows of the next item travel while the V tiles stream
     uint32_t qnext[4];
-    load_q_words(get_item(i + stride, total_items, pre_s, p), qnext);
+    load_q_words(get_item(i + stride, total_items, pre_s, len_s, p), qnext);
 
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
     float acc[4][4];
@@ -661,9 +749,9 @@ static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
 static size_t attn_smem_bytes(int split_len) {
   size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kMaxRows * (split_len + 8) * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                                // q_s
-  b += (size_t)kFixCap * kMaxRows * 4 + kFixCap * 4 + kMaxRows * 4;                          // kfix, kcol, knew
-  b += kMaxRows * kHeadDim * 4 + kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;           // oaux, m, l, red
-  b += 4 * 4 + (kMaxBatchSmem + 1) * 4 + 4 + 8 + (2 * kStages + 3) * 8 + 64;
+  b += 2 * ((size_t)kFixCap * kMaxRows * 4 + kFixCap * 4 + kMaxRows * 4);                    // kfix, kcol, knew (x2)
+  b += 2 * kMaxRows * kHeadDim * 4 + kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;       // oaux, aq, m, l, red
+  b += 16 * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + (2 * kStages + 4) * 8 + 64;
   return b;
 }
 
@@ -686,6 +774,8 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.ret_count = pair->ret_count;
   ap.ret_offset = pair->ret_offset;
   ap.ret_index = pair->ret_index;
+  ap.ret_prefix = pair->ret_prefix;
+  ap.ret_prefix_stride = (int)pair->ret_prefix_stride;
   ap.ret_rows = (const char*)pair->ret_rows;
   ap.q = (const char*)q;
   ap.k_new = (const char*)k_new;

@@ -360,6 +360,22 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   }
 }
 
+// ret_prefix[seg][j] = number of the segment's retained tokens before token 128 * j.
+__global__ void __launch_bounds__(256) retain_prefix_kernel(const int32_t* ret_count, const int32_t* ret_offset,
+                                                           const int32_t* ret_index, int32_t* ret_prefix, int stride) {
+  const int seg = blockIdx.x;
+  const int cnt = ret_count[seg], off = ret_offset[seg];
+  for (int j = threadIdx.x; j < stride; j += blockDim.x) {
+    const int key = j * 128;
+    int lo = 0, hi = cnt;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (ret_index[off + mid] < key) lo = mid + 1; else hi = mid;
+    }
+    ret_prefix[(size_t)seg * stride + j] = lo;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Decode-time append (Algorithm 2 "MiniCache Decoding": merge of the new token pair)
 // ---------------------------------------------------------------------------------------------
@@ -479,6 +495,9 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   retain_scan_kernel<<<1, 1024, 0, stream>>>(rp);
   MC_CUDA_CHECK(cudaGetLastError());
   retain_compact_kernel<<<grid, kRetThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(cudaGetLastError());
+  retain_prefix_kernel<<<nseg, 256, 0, stream>>>(out->ret_count, out->ret_offset, out->ret_index, out->ret_prefix,
+                                                 (int)out->ret_prefix_stride);
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }

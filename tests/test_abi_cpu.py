@@ -73,7 +73,7 @@ def test_merge_rejects_bad_arguments_without_launching(lib):
     L = lib._lib
     c, b = _cfg(), _batch()
     a = B._LayerKV(0x10000, 0x20000)
-    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
     ws = 0x100000
     # null layer pool
     bad = B._LayerKV(0, 0x20000)
@@ -90,14 +90,14 @@ def test_merge_rejects_bad_arguments_without_launching(lib):
     ck = _cfg(retain_mode=2)
     assert L.mc_merge_pair(C.byref(ck), C.byref(b), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 6
     # pair cache with a missing buffer
-    pc2 = B._PairCache(0x30000, 0, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    pc2 = B._PairCache(0x30000, 0, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
     assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(a), C.byref(pc2), 1, ws, 1 << 20, None) == 1
 
 
 def test_attn_and_restore_reject_bad_arguments(lib):
     L = lib._lib
     c, b = _cfg(), _batch()
-    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xB0000, 0xC0000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
     d = B._LayerKV(0x10000, 0x20000)
     assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 2, C.byref(d), None) == 1  # BOTH is not a restore target
     assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 0, None, None) == 1
