@@ -128,7 +128,9 @@ typedef struct mc_layer_kv {
  * ret_count  [2 * batch * n_kv_heads] retained tokens of the segment
  * ret_offset [2 * batch * n_kv_heads + 1] exclusive prefix of ret_count = first slot of the segment
  * ret_index  [ret_capacity] token indices, ascending inside a segment
- * ret_rows   [ret_capacity][2][128] raw 16-bit rows: [.][0] layer l-1, [.][1] layer l (bit copies)
+ * ret_rows   [2][ret_capacity][272 bytes]: [0] layer l-1, [1] layer l; an entry is the raw 16-bit row
+ *            (256 bytes, a bit copy of the input), the token's index (int32) and 12 bytes of padding,
+ *            so that a run of entries is one contiguous, 16-byte aligned block for a bulk copy
  * ret_prefix [2 * batch * n_kv_heads][ret_prefix_stride]: entry j = how many of the segment's retained
  *            tokens lie before token 128 * j (so a token range maps to a range of the segment's list
  *            without searching).  ret_prefix_stride (a host-side number, fixed when the pair is merged)

@@ -120,7 +120,7 @@ class PairCache:
         self.ret_count = torch.zeros(nseg, dtype=torch.int32, device=device)
         self.ret_offset = torch.zeros(nseg + 1, dtype=torch.int32, device=device)
         self.ret_index = torch.zeros(max(ret_capacity, 1), dtype=torch.int32, device=device)
-        self.ret_rows = torch.zeros(max(ret_capacity, 1), 2, 128, dtype=dt, device=device)
+        self.ret_rows = torch.zeros(2, max(ret_capacity, 1), 272, dtype=torch.uint8, device=device)
         self.ret_capacity = int(ret_capacity)
         if max_merge_len is None:  # bound of the sequence length at merge time: what the pages can hold at most
             max_merge_len = n_pages * ps
@@ -155,6 +155,14 @@ class PairCache:
         ps = self.cfg.page_size
         n_pages, H = pool.shape[:2]
         return pool[:, :, ps * 256:].contiguous().view(torch.float32).reshape(n_pages, H, 2, ps)
+
+    def retained_rows(self, layer: int) -> torch.Tensor:
+        """Raw retained rows of one layer (0: l-1, 1: l) as [ret_capacity][128] in the storage type."""
+        return self.ret_rows[layer, :, :256].contiguous().view(self.cfg.torch_dtype)
+
+    def retained_tokens(self, layer: int) -> torch.Tensor:
+        """Token index stored with each retained entry of one layer: [ret_capacity] int32."""
+        return self.ret_rows[layer, :, 256:260].contiguous().view(torch.int32).reshape(-1)
 
     def nbytes(self) -> int:
         ts = (self.e_k, self.e_v, self.dist, self.ret_count, self.ret_offset, self.ret_index,

@@ -10,15 +10,17 @@
 //
 // Work item = (sequence, split of the token axis, kv head).  The kernel is persistent: two CTAs
 // per SM walk the item list with a fixed stride.  In each CTA
-//   - the producer warp streams the compressed tiles of its items, one bulk copy (TMA engine,
-//     cp.async.bulk + mbarrier) per (page, head, tensor) tile, all K tiles of an item and then
-//     all its V tiles, through a ring of stages, running ahead into the next item;
-//   - four consumer warps run both contractions on the tensor cores, the query rows of the kv
+//   - the producer warp streams everything the item needs through one ring of stages with bulk
+//     asynchronous copies (TMA engine, cp.async.bulk + mbarrier): one copy per (page, head, tensor)
+//     tile, all K tiles of an item, then "extra" stages holding the split's retained K rows and
+//     the step's new K row, then the V tiles and the V extras; it runs ahead into the next item,
+//     and loads page ids and retained ranges one item early (a demand load takes microseconds
+//     while the copy engine saturates the memory system, so nothing irregular is left on any
+//     critical path);
+//   - four consumer warps run every contraction on the tensor cores, the query rows of the kv
 //     head's group (and of both layers in pair mode) being the padded M tile: scores x K scale
-//     -> shared memory -> split-local softmax -> (P x V scale) V;
-//   - the auxiliary warp does the irregular part in the shadow of the streaming: it finds the
-//     item's range of the retained lists, computes the retained rows' and the new token's
-//     scores while the K tiles stream, and adds their V terms while the V tiles stream.
+//     -> shared memory, scores of retained rows scattered over them -> split-local softmax ->
+//     (P x V scale) V, plus gathered P times the retained V rows.
 // Partial (m, l, o) per split are merged by attn_combine_kernel.  Every wait is bounded.
 #include <algorithm>
 
@@ -31,11 +33,11 @@ constexpr int kTile = 64;  // tokens per pipeline stage
 constexpr int kStages = 4;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kAttnThreads = kConsumerThreads + 64;  // + producer warp + auxiliary warp
+constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
 constexpr int kMaxRows = 8;                          // query rows per work item (M tile rows used)
 constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
 constexpr int kMaxSplit = 512;
-constexpr int kFixCap = 128;  // retained-K entries per item whose scores the auxiliary warp pre-computes
+constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kCtasPerSm = 2;
@@ -48,7 +50,8 @@ struct AttnParams {
   const int32_t* ret_index;
   const int32_t* ret_prefix;
   int ret_prefix_stride;
-  const char* ret_rows;
+  const char* ret_rows;  // [2 layers][ret_capacity][kEntryBytes]
+  int64_t ret_capacity;
   const char* q;
   const char* k_new;
   const char* v_new;
@@ -180,123 +183,30 @@ __device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, con
   return it;
 }
 
-// Shared-memory views and loop constants the auxiliary warp's K part needs.
-struct AuxCtx {
-  float* kfix_s;
-  int* kcol_s;
-  float* knew_s;
-  float* aq_s;
-  int* aux_info;
-  const int* pre_s;
-  const int* len_s;
-  uint32_t kfix_bar;
-  int total_items, H, rows, nslots, lane;
+// Where an item's retained entries sit in the pair's lists (first entry, count) for K and V.
+struct Ranges {
+  int k_lo, n_k, v_lo, n_v;
 };
 
-// K part of the auxiliary warp for item i (the n-th item of this CTA): scores of the split's retained
-// K rows and of the new token into buffer n & 1, then the buffer's barrier.
-template <int DT>
-__device__ __noinline__ void aux_k_part(const AttnParams& p, const AuxCtx& x, int i, int n) {
-  float* const kfix_s = x.kfix_s;
-  int* const kcol_s = x.kcol_s;
-  float* const knew_s = x.knew_s;
-  float* const aq_s = x.aq_s;
-  int* const aux_info = x.aux_info;
-  const int* pre_s = x.pre_s;
-  const int* len_s = x.len_s;
-  const uint32_t kfix_bar = x.kfix_bar;
-  const int total_items = x.total_items, H = x.H, rows = x.rows, nslots = x.nslots, lane = x.lane;
-    const Item w = get_item(i, total_items, pre_s, len_s, p);
-    if (!w.valid) return;
-    const int buf = n & 1;
-    float* kfix = kfix_s + buf * kFixCap * kMaxRows;
-    int* kcol = kcol_s + buf * kFixCap;
-    const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
-    // ranges of the two retained lists whose tokens lie in this split: two table entries each
-    // (split boundaries are multiples of 128; no retained token lies past the merged length)
-    const int pj0 = min(w.split_start >> 7, p.ret_prefix_stride - 1);
-    const int pj1 = min((w.split_start + w.n_tok + 127) >> 7, p.ret_prefix_stride - 1);
-    const int32_t* pk = p.ret_prefix + (size_t)seg_k * p.ret_prefix_stride;
-    const int32_t* pv = p.ret_prefix + (size_t)seg_v * p.ret_prefix_stride;
-    const int off_k = __ldg(p.ret_offset + seg_k), off_v = __ldg(p.ret_offset + seg_v);
-    const int k_lo = off_k + __ldg(pk + pj0), k_hi = off_k + __ldg(pk + pj1);
-    const int v_lo = off_v + __ldg(pv + pj0), v_hi = off_v + __ldg(pv + pj1);
-    const int n_fast = min(k_hi - k_lo, kFixCap);
-    const int n_new = w.has_new ? 1 : 0;
-    if (n_fast + n_new > 0) {
-      // one lane per retained row (or the new token): full 128-channel dot products
-#pragma unroll
-      for (int r = 0; r < kMaxRows; ++r) {
-        if (r < rows) {
-          const int set = r / p.nq, rq = r - set * p.nq;
-          const size_t qrow = ((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq;
-          const uint2 v = __ldg(reinterpret_cast<const uint2*>(p.q + qrow * kRowBytes + lane * 8));
-          const float2 a = Elem<DT>::unpack(v.x), c = Elem<DT>::unpack(v.y);
-          *reinterpret_cast<float4*>(aq_s + r * kHeadDim + lane * 4) = make_float4(a.x, a.y, c.x, c.y);
-        }
-      }
-      __syncwarp();
-      for (int base = 0; base < n_fast + n_new; base += 32) {
-        const int e = base + lane;
-        const bool act = e < n_fast + n_new;
-        const bool is_new = e >= n_fast;
-        if (act) {
-          const int col = is_new ? w.n_tok : __ldg(p.ret_index + k_lo + e) - w.split_start;
-          float dots[kMaxRows];
-#pragma unroll
-          for (int r = 0; r < kMaxRows; ++r) dots[r] = 0.f;
-#pragma unroll
-          for (int set = 0; set < 2; ++set) {
-            if (set < nslots) {
-              const char* src = is_new ? p.k_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
-                                       : p.ret_rows + ((size_t)(k_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-              const int r_lo = nslots == 2 ? set * p.nq : 0, r_hi = nslots == 2 ? r_lo + p.nq : rows;
-#pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                uint4 kv[8];  // half a row in flight at once
-#pragma unroll
-                for (int c = 0; c < 8; ++c) kv[c] = ld_stream16(src + (half * 8 + c) * 16);
-#pragma unroll
-                for (int cc = 0; cc < 8; ++cc) {
-                  const int c = half * 8 + cc;
-                  const float2 x0 = Elem<DT>::unpack(kv[cc].x), x1 = Elem<DT>::unpack(kv[cc].y);
-                  const float2 x2 = Elem<DT>::unpack(kv[cc].z), x3 = Elem<DT>::unpack(kv[cc].w);
-#pragma unroll
-                  for (int r = 0; r < kMaxRows; ++r) {
-                    if (r >= r_lo && r < r_hi) {
-                      const float4 q0 = *reinterpret_cast<const float4*>(aq_s + r * kHeadDim + c * 8);
-                      const float4 q1 = *reinterpret_cast<const float4*>(aq_s + r * kHeadDim + c * 8 + 4);
-                      dots[r] += x0.x * q0.x + x0.y * q0.y + x1.x * q0.z + x1.y * q0.w + x2.x * q1.x +
-                                 x2.y * q1.y + x3.x * q1.z + x3.y * q1.w;
-                    }
-                  }
-                }
-              }
-            }
-          }
-          if (is_new) {
-#pragma unroll
-            for (int r = 0; r < kMaxRows; ++r)
-              if (r < rows) knew_s[buf * kMaxRows + r] = dots[r] * p.scale_log2;
-          } else {
-            kcol[e] = col;
-#pragma unroll
-            for (int r = 0; r < kMaxRows; ++r)
-              if (r < rows) kfix[e * kMaxRows + r] = dots[r] * p.scale_log2;
-          }
-        }
-      }
-    }
-    if (lane == 0) {
-      int* info = aux_info + buf * 8;
-      info[0] = n_fast;
-      info[1] = k_lo;
-      info[2] = k_hi;
-      info[3] = v_lo;
-      info[4] = v_hi;
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(kfix_bar + 8 * buf);
+// Two table entries per list: split boundaries are multiples of 128 and no retained token lies
+// past the length the pair was merged at.
+__device__ __forceinline__ Ranges load_ranges(const Item& w, const AttnParams& p) {
+  Ranges r;
+  r.k_lo = r.n_k = r.v_lo = r.n_v = 0;
+  if (!w.valid) return r;
+  const int H = p.g.n_kv_heads;
+  const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
+  const int pj0 = min(w.split_start >> 7, p.ret_prefix_stride - 1);
+  const int pj1 = min((w.split_start + w.n_tok + 127) >> 7, p.ret_prefix_stride - 1);
+  const int32_t* pk = p.ret_prefix + (size_t)seg_k * p.ret_prefix_stride;
+  const int32_t* pv = p.ret_prefix + (size_t)seg_v * p.ret_prefix_stride;
+  const int off_k = __ldg(p.ret_offset + seg_k), off_v = __ldg(p.ret_offset + seg_v);
+  const int k0 = __ldg(pk + pj0), k1 = __ldg(pk + pj1), v0 = __ldg(pv + pj0), v1 = __ldg(pv + pj1);
+  r.k_lo = off_k + k0;
+  r.n_k = k1 - k0;
+  r.v_lo = off_v + v0;
+  r.n_v = v1 - v0;
+  return r;
 }
 
 template <int DT>
@@ -307,27 +217,23 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   const int nslots = p.n_sets;
   const int rows = p.rows;
   const int s_stride = p.split_len + 8;
+  const int cap_e = nslots == 2 ? 16 : 32;  // retained entries (per layer) in one extra stage
+  const int set_bytes = cap_e * kEntryBytes;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
-  float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);  // [kMaxRows][s_stride]
+  float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);     // [kMaxRows][s_stride]
   uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kMaxRows * s_stride);  // [2][kMaxRows][64] packed pairs
-  float* kfix_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);     // [2][kFixCap][kMaxRows]
-  int* kcol_s = reinterpret_cast<int*>(kfix_s + 2 * kFixCap * kMaxRows);  // [2][kFixCap]
-  float* knew_s = reinterpret_cast<float*>(kcol_s + 2 * kFixCap);        // [2][kMaxRows]
-  float* oaux_s = knew_s + 2 * kMaxRows;                                 // [kMaxRows][128]
-  float* m_s = oaux_s + kMaxRows * kHeadDim;                             // [kMaxRows]
+  float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
-  float* aq_s = red_s + kMaxRows * kConsumerWarps;                       // [kMaxRows][128] query rows of the auxiliary warp
-  int* aux_info = reinterpret_cast<int*>(aq_s + kMaxRows * kHeadDim);    // [2][8]: n_fast, k_lo, k_hi, v_lo, v_hi
-  int* pre_s = aux_info + 16;                                            // [batch + 1] split-count prefix
+  int* info_s = reinterpret_cast<int*>(red_s + kMaxRows * kConsumerWarps);  // [kStages][2]: entries, extra stages of the phase
+  int* pre_s = info_s + 2 * kStages;                                     // [batch + 1] split-count prefix
   int* len_s = pre_s + kMaxBatchSmem + 1;                                // [batch] sequence lengths
   volatile int* s_abort = len_s + kMaxBatchSmem;
   uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
-  const uint32_t kfix_bar = full0 + 16 * kStages, pready_bar = kfix_bar + 16, oaux_bar = kfix_bar + 24;  // kfix_bar[2]
   const uint32_t stage0 = smem_u32(stages);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -338,10 +244,6 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, kConsumerWarps);
     }
-    mbar_init(kfix_bar, 1);
-    mbar_init(kfix_bar + 8, 1);
-    mbar_init(pready_bar, 1);
-    mbar_init(oaux_bar, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // prefix of per-sequence split counts (a sequence always owns at least one split)
@@ -360,17 +262,28 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
   if (warp == kConsumerWarps) {
     // ===================== producer =====================
+    // Everything an item needs from global memory before its copies can be issued (page ids,
+    // retained ranges) is loaded one item ahead: such loads take microseconds while the copy
+    // engine saturates the memory system.
     int it = 0;  // running stage counter, same sequence as the consumers'
-    for (int i = first; i < total_items; i += stride) {
-      const Item w = get_item(i, total_items, pre_s, len_s, p);
-      // page ids of the item's pages, one per lane (split_len / page_size <= 32)
+    Item w = get_item(first, total_items, pre_s, len_s, p);
+    Ranges rg = load_ranges(w, p);
+    int my_page = 0;
+    if (w.valid && lane < ((w.n_tok + ps - 1) >> shift))
+      my_page = p.g.block_table[(size_t)w.b * p.g.max_pages_per_seq + (w.split_start >> shift) + lane];
+    bool ok = true;
+    for (int i = first; i < total_items && ok; i += stride) {
+      const Item wn = get_item(i + stride, total_items, pre_s, len_s, p);
+      const Ranges rgn = load_ranges(wn, p);
+      int next_page = 0;
+      if (wn.valid && lane < ((wn.n_tok + ps - 1) >> shift))
+        next_page = p.g.block_table[(size_t)wn.b * p.g.max_pages_per_seq + (wn.split_start >> shift) + lane];
       const int n_pages_item = (w.n_tok + ps - 1) >> shift;
-      int my_page = 0;
-      if (lane < n_pages_item)
-        my_page = p.g.block_table[(size_t)w.b * p.g.max_pages_per_seq + (w.split_start >> shift) + lane];
-      bool ok = true;
+      const int n_new = w.has_new ? 1 : 0;
       for (int ph = 0; ph < 2 && ok; ++ph) {
-        for (int t = 0; t < w.T; ++t, ++it) {
+        const int n_r = ph ? rg.n_v : rg.n_k, r_lo = ph ? rg.v_lo : rg.k_lo;
+        const int X = (n_r + n_new + cap_e - 1) / cap_e;  // extra stages: retained rows and the new token
+        for (int t = 0; t < w.T + X; ++t, ++it) {
           const int s = it % kStages;
           if (it >= kStages) {
             int good = 1;
@@ -378,95 +291,53 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) { ok = false; break; }
           }
-          const int pg0 = (t * kTile) >> shift;
-          const int n_pg = min(kTile >> shift, n_pages_item - pg0);
           const uint32_t bar = full0 + 8 * s;
-          if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_pg * tbytes));
-          __syncwarp();
-          // lane pg0 + j copies tile j of the stage (it holds that page's id)
-          const int j = lane - pg0;
-          if (j >= 0 && j < n_pg) {
-            const char* src = p.e_pool[ph] + ((size_t)my_page * H + w.g) * tbytes;
-            bulk_load(stage0 + s * kStageBytes + j * tbytes, src, (uint32_t)tbytes, bar);
-          }
-        }
-      }
-      if (!ok) break;
-    }
-    return;
-  }
-
-  if (warp == kConsumerWarps + 1) {
-    // ===================== auxiliary warp: retained rows and the new token =====================
-    // Software pipeline over this CTA's items n = 0, 1, 2, ...:
-    //   K part of item n + 2 (scores of its retained K rows and of its new token; needs nothing
-    //   from the consumers, so it runs two items ahead into a double buffer), then, once the
-    //   consumers have published item n's probabilities, the V part of item n.
-    // All global loads here are latency-bound while the copy engine saturates the memory system,
-    // which is why nothing the consumers wait for is started late.
-    AuxCtx ax;
-    ax.kfix_s = kfix_s; ax.kcol_s = kcol_s; ax.knew_s = knew_s; ax.aq_s = aq_s; ax.aux_info = aux_info;
-    ax.pre_s = pre_s; ax.len_s = len_s; ax.kfix_bar = kfix_bar;
-    ax.total_items = total_items; ax.H = H; ax.rows = rows; ax.nslots = nslots; ax.lane = lane;
-    auto k_part = [&](int i, int n) { aux_k_part<DT>(p, ax, i, n); };
-    k_part(first, 0);
-    k_part(first + stride, 1);
-    int n_item = 0;
-    for (int i = first; i < total_items; i += stride, ++n_item) {
-      const Item w = get_item(i, total_items, pre_s, len_s, p);
-      const int v_lo = aux_info[(n_item & 1) * 8 + 3], v_hi = aux_info[(n_item & 1) * 8 + 4];
-      const int n_v = v_hi - v_lo, n_new = w.has_new ? 1 : 0;
-      // ---- V part: after the softmax, add the retained V rows' and the new token's terms (lane = 4 channels)
-      int my_col = 0;  // first batch of token columns, loaded before the wait
-      if (lane < min(32, n_v + n_new)) my_col = lane >= n_v ? w.n_tok : __ldg(p.ret_index + v_lo + lane) - w.split_start;
-      int good = 1;
-      if (lane == 0) good = mbar_wait(pready_bar, n_item & 1, s_abort, p.status) ? 1 : 0;
-      good = __shfl_sync(0xffffffffu, good, 0);
-      if (!good) break;
-      float oa[kMaxRows][4];
-#pragma unroll
-      for (int r = 0; r < kMaxRows; ++r) oa[r][0] = oa[r][1] = oa[r][2] = oa[r][3] = 0.f;
-      for (int base = 0; base < n_v + n_new; base += 32) {
-        const int cnt = min(32, n_v + n_new - base);
-        if (base > 0) {
-          my_col = 0;
-          if (lane < cnt) my_col = (base + lane) >= n_v ? w.n_tok : __ldg(p.ret_index + v_lo + base + lane) - w.split_start;
-        }
-#pragma unroll 4
-        for (int j = 0; j < cnt; ++j) {
-          const int e = base + j;
-          const bool is_new = e >= n_v;
-          const int col = __shfl_sync(0xffffffffu, my_col, j);
-          float val[2][4];
-#pragma unroll
-          for (int set = 0; set < 2; ++set) {
-            if (set < nslots) {
-              const char* src = is_new ? p.v_new + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes
-                                       : p.ret_rows + ((size_t)(v_lo + e) * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-              const uint2 vv = __ldg(reinterpret_cast<const uint2*>(src + lane * 8));
-              const float2 a = Elem<DT>::unpack(vv.x), c = Elem<DT>::unpack(vv.y);
-              val[set][0] = a.x; val[set][1] = a.y; val[set][2] = c.x; val[set][3] = c.y;
-            } else {
-              val[set][0] = val[set][1] = val[set][2] = val[set][3] = 0.f;
+          const uint32_t sbase = stage0 + s * kStageBytes;
+          if (t < w.T) {
+            // ---- one 64-token tile: a bulk copy per page
+            const int pg0 = (t * kTile) >> shift;
+            const int n_pg = min(kTile >> shift, n_pages_item - pg0);
+            if (lane == 0) {
+              info_s[2 * s] = 0;
+              info_s[2 * s + 1] = X;
+              mbar_expect_tx(bar, (uint32_t)(n_pg * tbytes));
             }
-          }
-#pragma unroll
-          for (int r = 0; r < kMaxRows; ++r) {
-            if (r < rows) {
-              const float pr = S[r * s_stride + col];
-              const bool second = nslots == 2 && r >= p.nq;
-#pragma unroll
-              for (int k = 0; k < 4; ++k) oa[r][k] = fmaf(pr, second ? val[1][k] : val[0][k], oa[r][k]);
+            __syncwarp();
+            const int j = lane - pg0;  // lane pg0 + j holds the id of the stage's page j
+            if (j >= 0 && j < n_pg)
+              bulk_load(sbase + j * tbytes, p.e_pool[ph] + ((size_t)my_page * H + w.g) * tbytes, (uint32_t)tbytes, bar);
+          } else {
+            // ---- an extra stage: up to cap_e retained entries per layer, the new token last
+            const int x0 = (t - w.T) * cap_e;
+            const int cnt_ret = max(0, min(n_r, x0 + cap_e) - x0);
+            const bool add_new = n_new && n_r >= x0 && n_r < x0 + cap_e;
+            if (lane == 0) {
+              info_s[2 * s] = cnt_ret + (add_new ? 1 : 0);
+              info_s[2 * s + 1] = X;
+              if (add_new) {
+                for (int set = 0; set < nslots; ++set)
+                  *reinterpret_cast<int*>(stages + s * kStageBytes + set * set_bytes + cnt_ret * kEntryBytes + kRowBytes) =
+                      w.split_start + w.n_tok;  // the new token's index
+              }
+              mbar_expect_tx(bar, (uint32_t)(nslots * (cnt_ret * kEntryBytes + (add_new ? kRowBytes : 0))));
+            }
+            __syncwarp();
+            if (lane < nslots && cnt_ret > 0) {
+              const int layer = nslots == 2 ? lane : p.layer_sel;
+              bulk_load(sbase + lane * set_bytes, p.ret_rows + ((size_t)layer * p.ret_capacity + r_lo + x0) * kEntryBytes,
+                        (uint32_t)(cnt_ret * kEntryBytes), bar);
+            }
+            if (lane >= 2 && lane < 2 + nslots && add_new) {
+              const int set = lane - 2;
+              const char* src = (ph ? p.v_new : p.k_new) + (((size_t)set * p.g.batch + w.b) * H + w.g) * kRowBytes;
+              bulk_load(sbase + set * set_bytes + cnt_ret * kEntryBytes, src, (uint32_t)kRowBytes, bar);
             }
           }
         }
       }
-#pragma unroll
-      for (int r = 0; r < kMaxRows; ++r)
-        if (r < rows) *reinterpret_cast<float4*>(oaux_s + r * kHeadDim + lane * 4) = make_float4(oa[r][0], oa[r][1], oa[r][2], oa[r][3]);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(oaux_bar);
-      k_part(i + 2 * stride, n_item + 2);
+      w = wn;
+      rg = rgn;
+      my_page = next_page;
     }
     return;
   }
@@ -474,11 +345,11 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   // ===================== consumers =====================
   const int row = lane >> 2;        // M-tile row of this thread's fragments
   const int colp = (lane & 3) * 2;  // column pair inside an 8-wide n tile
-  const int slot_row = (nslots == 2 && row < rows) ? row / p.nq : (nslots == 2 ? 0 : p.layer_sel);
+  const int set_row = (nslots == 2 && row < rows) ? row / p.nq : 0;  // which layer this row attends (pair mode)
+  const int slot_row = nslots == 2 ? set_row : p.layer_sel;          // which of the tile's two scales it uses
   const int mi = lane >> 3, mr = lane & 7;
   int it = 0, n_item = 0;
 
-  // query rows of the first item
   auto load_q_words = [&](const Item& w, uint32_t (&qw)[4]) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -503,9 +374,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
   for (int i = first; i < total_items; i += stride, ++n_item) {
     const Item w = get_item(i, total_items, pre_s, len_s, p);
-    const uint32_t par = n_item & 1;
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
-    const int n_cols = w.n_tok + (w.has_new ? 1 : 0);
+    const int n_new = w.has_new ? 1 : 0;
+    const int n_cols = w.n_tok + n_new;
     bool ok = true;
 
     // ---- K phase: S[r][i] = log2e * sm_scale * g_i * (q_r . e_i) ---------------------------------
@@ -517,15 +388,17 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         qa2[ks] = qcur[row * 64 + ks * 8 + 4 + (lane & 3)];
       }
       const int tk_w = warp * 16;  // this warp's 16 tokens of every tile
+      int xk = n_new;              // extra stages after the tiles (an item without tiles has no retained rows)
       for (int t = 0; t < w.T; ++t, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const uint32_t sbase = stage0 + s * kStageBytes;
         const int valid = min(kTile, w.n_tok - t * kTile);
+        xk = info_s[2 * s + 1];
         if (tk_w < valid) {
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
           const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
-          const uint32_t rowaddr = tile_addr(sbase, tk_m, 0, shift, tbytes) - (chunk_pos(tk_m & (ps - 1), 0) << 4);
+          const uint32_t rowaddr = sbase + (uint32_t)((tk_m >> shift) * tbytes + (tk_m & (ps - 1)) * kRowBytes);
           const int rsw = tk_m & 7;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
@@ -551,33 +424,40 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
-    }
-    consumer_sync();
-
-    // ---- retained K rows and the new token replace / add single scores ----------------------------
-    const int kb = n_item & 1;
-    if (ok && !mbar_wait(kfix_bar + 8 * kb, (n_item >> 1) & 1, s_abort, p.status)) ok = false;
-    if (ok) {
-      const int n_fast = aux_info[kb * 8], k_lo = aux_info[kb * 8 + 1], k_hi = aux_info[kb * 8 + 2];
-      for (int e = tid; e < n_fast; e += kConsumerThreads) {
-        const int col = kcol_s[kb * kFixCap + e];
-        for (int r = 0; r < rows; ++r) S[r * s_stride + col] = kfix_s[(kb * kFixCap + e) * kMaxRows + r];
-      }
-      if (w.has_new && tid < rows) S[tid * s_stride + w.n_tok] = knew_s[kb * kMaxRows + tid];
-      // more retained rows than the auxiliary warp pre-computes: finish them here
-      for (int e = k_lo + n_fast + warp; e < k_hi; e += kConsumerWarps) {
-        const int col = p.ret_index[e] - w.split_start;
-        for (int r = 0; r < rows; ++r) {
-          const int set = r / p.nq;
-          const char* src = p.ret_rows + ((size_t)e * 2 + (nslots == 2 ? set : p.layer_sel)) * kRowBytes;
-          const uint2 kv = *reinterpret_cast<const uint2*>(src + lane * 8);
-          const uint2 qv = *reinterpret_cast<const uint2*>(qcur + r * 64 + lane * 2);
-          const float2 k0 = Elem<DT>::unpack(kv.x), k1 = Elem<DT>::unpack(kv.y);
-          const float2 q0 = Elem<DT>::unpack(qv.x), q1 = Elem<DT>::unpack(qv.y);
-          float d = q0.x * k0.x + q0.y * k0.y + q1.x * k1.x + q1.y * k1.y;
-          for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-          if (lane == 0) S[r * s_stride + col] = d * p.scale_log2;
+      // ---- retained K rows and the new token: their scores replace / add single columns of S.
+      // (A barrier first: the tile that wrote a column may have been handled by another warp.)
+      if (xk > 0) consumer_sync();
+      for (int x = 0; x < xk && ok; ++x, ++it) {
+        const int s = it % kStages;
+        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const int cnt = info_s[2 * s];
+        // single layer: warp w takes entries 8w..8w+7; pair mode: warps 0,1 layer l-1, warps 2,3 layer l
+        const int set = nslots == 2 ? (warp >> 1) : 0;
+        const int e_w = nslots == 2 ? (warp & 1) * 8 : warp * 8;
+        if (e_w < cnt) {
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f};
+          const unsigned char* sb = stages + s * kStageBytes + set * set_bytes;
+          const uint32_t rowaddr = smem_u32(sb) + (uint32_t)((e_w + mr) * kEntryBytes);
+#pragma unroll
+          for (int k2 = 0; k2 < 4; ++k2) {
+            uint32_t r0, r1, r2, r3;  // (k step 2 k2: chunks lo, hi), (k step 2 k2 + 1: lo, hi)
+            ldsm_x4(rowaddr + (uint32_t)((k2 * 4 + mi) << 4), r0, r1, r2, r3);
+            mma_16816<DT>(acc0, qa0[2 * k2], qa2[2 * k2], r0, r1);
+            mma_16816<DT>(acc0, qa0[2 * k2 + 1], qa2[2 * k2 + 1], r2, r3);
+          }
+          if (row < rows && set_row == set) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              const int e = e_w + colp + k;
+              if (e < cnt) {
+                const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
+                S[row * s_stride + col] = acc0[k] * p.scale_log2;
+              }
+            }
+          }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
     }
     consumer_sync();
@@ -608,7 +488,6 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         }
       }
       consumer_sync();
-      if (tid == 0) mbar_arrive(pready_bar);  // the probabilities are final: the auxiliary warp may read them
     }
 
     // query rows of the next item travel while the V tiles stream
@@ -623,12 +502,14 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       for (int k = 0; k < 4; ++k) acc[a][k] = 0.f;
     if (ok) {
       const int chunk0 = warp * 4;  // this warp owns channels [32 warp, 32 warp + 32)
+      int xv = n_new;
       for (int t = 0; t < w.T; ++t, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const uint32_t sbase = stage0 + s * kStageBytes;
         const int valid = min(kTile, w.n_tok - t * kTile);
         const int ksteps = (valid + 15) >> 4;
+        xv = info_s[2 * s + 1];
         // rows past the last cached token may hold anything (page tail, page not copied): zero this
         // warp's channels there so that 0 * x stays 0 in the contraction
         bool wrote = false;
@@ -668,20 +549,61 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
+      // ---- retained V rows and the new token: raw rows weighted by their tokens' probabilities
+      for (int x = 0; x < xv && ok; ++x, ++it) {
+        const int s = it % kStages;
+        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const int cnt = info_s[2 * s];
+        const int ksteps = (cnt + 15) >> 4;
+        bool wrote = false;
+        for (int set = 0; set < nslots; ++set) {
+          const unsigned char* sb = stages + s * kStageBytes + set * set_bytes;
+          const uint32_t sba = smem_u32(sb);
+          for (int rz = cnt + (lane >> 2); rz < ksteps * 16; rz += 8) {  // entries past the last one: zero our channels
+            const uint32_t a = sba + (uint32_t)(rz * kEntryBytes + ((chunk0 + (lane & 3)) << 4));
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+            wrote = true;
+          }
+          __syncwarp();
+          for (int kk = 0; kk < ksteps; ++kk) {
+            uint32_t a0 = 0u, a2 = 0u;
+            if (row < rows && set_row == set) {
+              float pv[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const int e = kk * 16 + colp + (k & 1) + (k >> 1) * 8;
+                pv[k] = 0.f;
+                if (e < cnt) {
+                  const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
+                  pv[k] = S[row * s_stride + col];
+                }
+              }
+              a0 = Elem<DT>::pack(pv[0], pv[1]);
+              a2 = Elem<DT>::pack(pv[2], pv[3]);
+            }
+            const int e_m = kk * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+              uint32_t r0, r1, r2, r3;
+              ldsm_x4_t(sba + (uint32_t)(e_m * kEntryBytes + ((chunk0 + np * 2 + (mi >> 1)) << 4)), r0, r1, r2, r3);
+              mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
+              mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
+            }
+          }
+        }
+        if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      }
     }
 
-    // ---- partial results of this split: tensor-core part + the auxiliary warp's terms --------------
-    if (ok && !mbar_wait(oaux_bar, par, s_abort, p.status)) ok = false;
+    // ---- partial results of this split ---------------------------------------------------------------
     if (row < rows) {
-      const int set = row / p.nq, rq = row - set * p.nq;
-      const size_t prow = (((size_t)set * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
+      const int rq = row - set_row * p.nq;
+      const size_t prow = (((size_t)set_row * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
       float* dst = p.part_o + prow * kHeadDim + warp * 32 + colp;
-      const float* oa = oaux_s + row * kHeadDim + warp * 32 + colp;
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) {
-        const float2 x = *reinterpret_cast<const float2*>(oa + nt * 8);
-        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(acc[nt][0] + x.x, acc[nt][1] + x.y);
-      }
+      for (int nt = 0; nt < 4; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(acc[nt][0], acc[nt][1]);
       if (warp == 0 && (lane & 3) == 0) {
         const float4 ll = *reinterpret_cast<const float4*>(l_s + row * kConsumerWarps);
         p.part_ml[prow * 2] = m_s[row];
@@ -749,9 +671,8 @@ static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
 static size_t attn_smem_bytes(int split_len) {
   size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kMaxRows * (split_len + 8) * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                                // q_s
-  b += 2 * ((size_t)kFixCap * kMaxRows * 4 + kFixCap * 4 + kMaxRows * 4);                    // kfix, kcol, knew (x2)
-  b += 2 * kMaxRows * kHeadDim * 4 + kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;       // oaux, aq, m, l, red
-  b += 16 * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + (2 * kStages + 4) * 8 + 64;
+  b += kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;                                     // m, l, red
+  b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + 2 * kStages * 8 + 64;
   return b;
 }
 
@@ -777,6 +698,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.ret_prefix = pair->ret_prefix;
   ap.ret_prefix_stride = (int)pair->ret_prefix_stride;
   ap.ret_rows = (const char*)pair->ret_rows;
+  ap.ret_capacity = pair->ret_capacity;
   ap.q = (const char*)q;
   ap.k_new = (const char*)k_new;
   ap.v_new = (const char*)v_new;

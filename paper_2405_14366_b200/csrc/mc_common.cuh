@@ -12,6 +12,7 @@ namespace mc {
 
 constexpr int kHeadDim = 128;
 constexpr int kRowBytes = kHeadDim * 2;  // one 16-bit row
+constexpr int kRetEntryBytes = 272;      // retained entry: raw 16-bit row, int32 token index, 12 bytes of padding
 constexpr float kInvPi = 0.31830988618379067154f;
 
 // Host-side launch plumbing ---------------------------------------------------

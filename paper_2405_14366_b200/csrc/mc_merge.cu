@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     }
     __syncthreads();
   }
-  // gather: one half-warp per (entry, layer) row of 256 bytes
+  // gather: one half-warp per (entry, layer): the raw row and the token index behind it
   const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
   for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
     const int ent = r >> 1, layer = r & 1;
@@ -355,8 +355,9 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
     const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
     const char* src = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kRowBytes + l16 * 16;
-    char* dst = p.ret_rows + ((size_t)(out0 + ent) * 2 + layer) * kRowBytes + l16 * 16;
-    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
+    *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
+    if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok, 0, 0, 0);
   }
 }
 

@@ -18,6 +18,7 @@ struct RestoreParams {
   const int32_t* ret_offset;
   const int32_t* ret_index;
   const char* ret_rows;
+  int64_t ret_capacity;
   int layer;  // 0: l-1, 1: l
   int items_per_page;
 };
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kRestoreThreads) restore_scatter_kernel(const 
     const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
     const size_t row = ((size_t)page * H + h) * p.g.page_size + (tok & (p.g.page_size - 1));
     const uint4 v =
-        *reinterpret_cast<const uint4*>(p.ret_rows + ((size_t)(off + e) * 2 + p.layer) * kRowBytes + l16 * 16);
+        *reinterpret_cast<const uint4*>(p.ret_rows + ((size_t)p.layer * p.ret_capacity + off + e) * kRetEntryBytes + l16 * 16);
     *reinterpret_cast<uint4*>(p.dst_pool[tensor] + row * kRowBytes + l16 * 16) = v;
   }
 }
@@ -102,6 +103,7 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
   rp.ret_offset = pair->ret_offset;
   rp.ret_index = pair->ret_index;
   rp.ret_rows = (const char*)pair->ret_rows;
+  rp.ret_capacity = pair->ret_capacity;
   rp.layer = layer;
   rp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
   const long long blocks = 2LL * bt->batch * bt->max_pages_per_seq * rp.items_per_page;

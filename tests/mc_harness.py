@@ -107,14 +107,18 @@ class Problem:
         out["ret_count"] = pc.ret_count.cpu().numpy().reshape(2, self.B, self.H)
         out["ret_offset"] = pc.ret_offset.cpu().numpy()
         out["ret_index"] = pc.ret_index.cpu().numpy()
-        out["ret_rows"] = as_bits(pc.ret_rows.cpu())
+        out["ret_rows"] = np.stack([as_bits(pc.retained_rows(0).cpu()), as_bits(pc.retained_rows(1).cpu())], axis=1)  # [cap][2][128]
+        out["ret_tokens"] = np.stack([pc.retained_tokens(0).cpu().numpy(), pc.retained_tokens(1).cpu().numpy()], axis=1)
         out["seg_minmax"] = pc.seg_minmax.cpu().numpy().reshape(2, self.B, self.H, 2).astype(np.float64)
         return out
 
     def retained(self, dc, tensor: int, b: int, h: int):
         seg = (tensor * self.B + b) * self.H + h
         off, cnt = int(dc["ret_offset"][seg]), int(dc["ret_count"][tensor, b, h])
-        return dc["ret_index"][off:off + cnt].astype(np.int64), dc["ret_rows"][off:off + cnt]
+        idx = dc["ret_index"][off:off + cnt].astype(np.int64)
+        # every entry carries its token index next to the row, for both layers
+        assert np.array_equal(dc["ret_tokens"][off:off + cnt, 0], idx) and np.array_equal(dc["ret_tokens"][off:off + cnt, 1], idx)
+        return idx, dc["ret_rows"][off:off + cnt]
 
     # ------------------------------------------------------------------ oracle side
     def oracle_merge(self, mode: str = "distinct", do_retention: bool = True):
