@@ -10,7 +10,6 @@ namespace mc {
 
 constexpr int kMergeThreads = 256;
 constexpr int kRowsPerItem = 64;  // rows of one page handled by one CTA
-constexpr int kRowsPerHalfWarp = 4;
 
 struct MergeParams {
   Geom g;
@@ -83,6 +82,97 @@ __device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, floa
   d_out = s.d;
 }
 
+// Sum of squares of the two 16-bit values of a packed word, accumulated in fp32 by the
+// mixed-precision FMA of sm_100 (no conversion instructions).
+template <int DT>
+__device__ __forceinline__ float sq_acc(uint32_t w, float acc) {
+  unsigned short lo, hi;
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(w));
+  if (DT == MC_F16) {
+    asm("fma.rn.f32.f16 %0, %1, %1, %0;" : "+f"(acc) : "h"(lo));
+    asm("fma.rn.f32.f16 %0, %1, %1, %0;" : "+f"(acc) : "h"(hi));
+  } else {
+    asm("fma.rn.f32.bf16 %0, %1, %1, %0;" : "+f"(acc) : "h"(lo));
+    asm("fma.rn.f32.bf16 %0, %1, %1, %0;" : "+f"(acc) : "h"(hi));
+  }
+  return acc;
+}
+
+// Sum over the 4 lanes that share one row.
+__device__ __forceinline__ float sum4(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  return v;
+}
+
+// One merged row held by a quad of lanes: lane k owns the 16-byte chunks k, k + 4, k + 8, k + 12 of
+// a (layer l-1) and c (layer l), 32 channels each.  Arithmetic in fp32, two channels per
+// instruction (packed f32x2).  Every lane of the quad returns the row's scalars.
+template <int DT>
+__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc,
+                                               uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
+  float2 a[16], c[16];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[4 * i] = Elem<DT>::unpack(ra[i].x);
+    a[4 * i + 1] = Elem<DT>::unpack(ra[i].y);
+    a[4 * i + 2] = Elem<DT>::unpack(ra[i].z);
+    a[4 * i + 3] = Elem<DT>::unpack(ra[i].w);
+    c[4 * i] = Elem<DT>::unpack(rc[i].x);
+    c[4 * i + 1] = Elem<DT>::unpack(rc[i].y);
+    c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
+    c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
+  }
+  float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    aa2 = __ffma2_rn(a[i], a[i], aa2);
+    cc2 = __ffma2_rn(c[i], c[i], cc2);
+  }
+  const float aa = sum4(aa2.x + aa2.y), cc = sum4(cc2.x + cc2.y);
+  const float ia = aa > 0.f ? rsqrtf(aa) : 0.f;
+  const float ic = cc > 0.f ? rsqrtf(cc) : 0.f;
+  // |u - v|^2 formed channel by channel (no cancellation at small angles); |u + v|^2 = 4 - |u - v|^2
+  // is as good until the two directions come close to opposite, where it is formed the same way
+  const float2 ia2 = make_float2(ia, ia), nic2 = make_float2(-ic, -ic);
+  float2 sm2 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float2 dm = __ffma2_rn(c[i], nic2, __fmul2_rn(a[i], ia2));
+    sm2 = __ffma2_rn(dm, dm, sm2);
+  }
+  const float sm = sum4(sm2.x + sm2.y);
+  float sp = 4.0f - sm;
+  if (__any_sync(0xffffffffu, sm > 3.5f)) {
+    const float2 ic2 = make_float2(ic, ic);
+    float2 sp2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float2 dp = __ffma2_rn(c[i], ic2, __fmul2_rn(a[i], ia2));
+      sp2 = __ffma2_rn(dp, dp, sp2);
+    }
+    const float spx = sum4(sp2.x + sp2.y);
+    if (sm > 3.5f) sp = spx;
+  }
+  const RowScalars s = slerp_scalars(aa, cc, sm, fmaxf(sp, 0.f), ta, tc);
+  const float2 fa2 = make_float2(s.fa, s.fa), fc2 = make_float2(s.fc, s.fc);
+  float ee = 0.f;
+  uint32_t w[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float2 x = __ffma2_rn(a[i], fa2, __fmul2_rn(c[i], fc2));
+    w[i] = Elem<DT>::pack(x.x, x.y);
+    ee = sq_acc<DT>(w[i], ee);  // the stored value: Eq. 2 divides by its length
+  }
+  ee = sum4(ee);
+  const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) e_out[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  g_a = s.na * il;
+  g_c = s.nc * il;
+  d_out = s.d;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams p) {
   __shared__ unsigned s_min[4], s_max[4];
@@ -108,64 +198,50 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams 
   }
   __syncthreads();
 
-  const int hw = threadIdx.x >> 4;
-  const int l16 = threadIdx.x & 15;
-  const int row0 = item * kRowsPerItem + hw * kRowsPerHalfWarp;  // 4 consecutive rows, one head
-  const int head = row0 >> p.g.page_shift;
-  const int tk0 = row0 & (ps - 1);
-  const int tok0 = pslot * ps + tk0;
-  const size_t page_off = (size_t)page * rows_in_page;
-  const char* pa = p.a_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
-  const char* pc = p.c_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
-  char* tile = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
+  const int quad = threadIdx.x >> 2, k = threadIdx.x & 3;
+  const int row = item * kRowsPerItem + quad;  // one row per quad of lanes; a warp = 8 consecutive rows of one head
+  const int head = row >> p.g.page_shift;
+  const int tk = row & (ps - 1);
+  const bool valid = row < rows_in_page && pslot * ps + tk < n;
+  const size_t in_off = ((size_t)page * rows_in_page + row) * kRowBytes + k * 16;
+  const char* pa = (tensor ? p.a_pool[1] : p.a_pool[0]) + in_off;
+  const char* pc = (tensor ? p.c_pool[1] : p.c_pool[0]) + in_off;
+  char* tile = (tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + head) * tile_bytes(ps);
 
-  uint4 va[kRowsPerHalfWarp], vc[kRowsPerHalfWarp];
-  bool valid[kRowsPerHalfWarp];
+  uint4 va[4], vc[4];
 #pragma unroll
-  for (int j = 0; j < kRowsPerHalfWarp; ++j) {
-    valid[j] = (row0 + j < rows_in_page) && (tok0 + j < n);
-    if (valid[j]) {
-      va[j] = ld_stream16(pa + j * kRowBytes);
-      vc[j] = ld_stream16(pc + j * kRowBytes);
+  for (int i = 0; i < 4; ++i) {
+    if (valid) {
+      va[i] = ld_stream16(pa + i * 64);
+      vc[i] = ld_stream16(pc + i * 64);
     } else {
-      va[j] = make_uint4(0, 0, 0, 0);
-      vc[j] = make_uint4(0, 0, 0, 0);
+      va[i] = make_uint4(0, 0, 0, 0);
+      vc[i] = make_uint4(0, 0, 0, 0);
     }
   }
+  uint4 e[4];
+  float g_a, g_c, d;
+  merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
   float dmin = __int_as_float(0x7f800000), dmax = 0.f;
-  float ga[kRowsPerHalfWarp], gc[kRowsPerHalfWarp], dd[kRowsPerHalfWarp];
+  if (valid) {
 #pragma unroll
-  for (int j = 0; j < kRowsPerHalfWarp; ++j) {
-    uint4 e;
-    merge_row<DT>(va[j], vc[j], p.ta, p.tc, e, ga[j], gc[j], dd[j]);
-    if (valid[j]) {
-      st_stream16(tile + (tk0 + j) * kRowBytes + chunk_pos(tk0 + j, l16) * 16, e);
-      dmin = fminf(dmin, dd[j]);
-      dmax = fmaxf(dmax, dd[j]);
-    }
-  }
-  // lane j of the half-warp writes token j's three scalars (consecutive tokens -> 16-byte runs)
-  if (l16 < kRowsPerHalfWarp && row0 < rows_in_page) {
-    float g_a = ga[0], g_c = gc[0], d = dd[0];
-    bool ok = valid[0];
-#pragma unroll
-    for (int j = 1; j < kRowsPerHalfWarp; ++j)
-      if (l16 == j) {
-        g_a = ga[j];
-        g_c = gc[j];
-        d = dd[j];
-        ok = valid[j];
-      }
-    if (ok) {
-      const size_t ph = (size_t)page * H + head;
-      float* sc = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk0 + l16;
+    for (int i = 0; i < 4; ++i) st_stream16(tile + tk * kRowBytes + chunk_pos(tk, i * 4 + k) * 16, e[i]);
+    if (k == 0) {
+      float* sc = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk;
       sc[0] = g_a;
       sc[ps] = g_c;
-      p.dist[(ph * 2 + tensor) * ps + tk0 + l16] = d;
+      p.dist[(((size_t)page * H + head) * 2 + tensor) * ps + tk] = d;
     }
+    dmin = d;
+    dmax = d;
   }
-  if (l16 == 0 && valid[0]) {
-    const int hl = (hw * kRowsPerHalfWarp) >> p.g.page_shift;  // head inside the item
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
+    dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+  }
+  if ((threadIdx.x & 31) == 0 && dmin != __int_as_float(0x7f800000)) {
+    const int hl = ((threadIdx.x >> 5) * 8) >> p.g.page_shift;  // head inside the item
     atomicMin(&s_min[hl], __float_as_uint(dmin));
     atomicMax(&s_max[hl], __float_as_uint(dmax));
   }
