@@ -211,6 +211,8 @@ __device__ __forceinline__ Ranges load_ranges(const Item& w, const AttnParams& p
 
 template <int DT>
 __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(const AttnParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
   const int tbytes = tile_bytes(ps);
@@ -628,6 +630,8 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 // Log-sum-exp merge of the split partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
 template <int DT>
 __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
   const int n = p.g.seq_lens[b];
   const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
@@ -727,14 +731,14 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_split_kernel<MC_F16><<<grid, kAttnThreads, smem, stream>>>(ap);
+    MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_F16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    attn_combine_kernel<MC_F16><<<cgrid, 128, 0, stream>>>(ap, (unsigned short*)out, lse);
+    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_F16>, dim3(cgrid), dim3(128), 0, stream, ap, (unsigned short*)out, lse));
   } else {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_split_kernel<MC_BF16><<<grid, kAttnThreads, smem, stream>>>(ap);
+    MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_BF16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    attn_combine_kernel<MC_BF16><<<cgrid, 128, 0, stream>>>(ap, (unsigned short*)out, lse);
+    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_BF16>, dim3(cgrid), dim3(128), 0, stream, ap, (unsigned short*)out, lse));
   }
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;

@@ -26,6 +26,31 @@ void set_cuda_error(cudaError_t e, const char* where);
     }                                  \
   } while (0)
 
+// Every kernel of the library is launched with programmatic dependent launch allowed and begins
+// with grid_dep_wait(): its blocks may be placed on the SMs while the previous kernel of the stream
+// drains, but touch no memory before that kernel has completed.  grid_dep_launch() right after lets
+// the next kernel do the same.  This removes the launch gap between the many short kernels of a
+// merge and of a decode step.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#if defined(__CUDACC__)
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 // Geometry handed to every kernel by value.
 struct Geom {
   const int32_t* block_table;

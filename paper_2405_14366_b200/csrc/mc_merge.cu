@@ -3,6 +3,8 @@
 //                     per-segment d_min / d_max
 //   retain_*          Eq. 4 retention set: count, scan, ordered compaction + raw-row gather
 //   append_kernel     the decode-time merge of one new token per sequence
+#include <algorithm>
+
 #include "mc_common.cuh"
 #include "mc_kernels.h"
 
@@ -175,6 +177,8 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
 
 template <int DT>
 __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ unsigned s_min[4], s_max[4];
   const int ipp = p.items_per_page;
   int bid = blockIdx.x;
@@ -286,6 +290,8 @@ struct RetainParams {
 };
 
 __global__ void merge_init_kernel(unsigned* seg_minmax, int nseg, int32_t* status) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < nseg) {
     seg_minmax[2 * i] = 0x7f800000u;
@@ -307,6 +313,8 @@ __device__ __forceinline__ float load_dist(const RetainParams& p, int tensor, in
 }
 
 __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ int s_cnt[kRetThreads / 32];
   const int seg = blockIdx.y, chunk = blockIdx.x;
   const int h = seg % p.g.n_kv_heads;
@@ -333,6 +341,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainP
 
 // One CTA: exclusive scan of the chunk counts in (segment, chunk) order.
 __global__ void __launch_bounds__(1024) retain_scan_kernel(const RetainParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ int s_warp[32];
   __shared__ int s_carry;
   const int total = p.nseg * p.chunks_per_seg;
@@ -378,6 +388,8 @@ __global__ void __launch_bounds__(1024) retain_scan_kernel(const RetainParams p)
 // Per (segment, chunk): ordered compaction of the kept token indices, then bit copies of both
 // layers' rows.  Writes ret_count per segment from the chunk offsets.
 __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const RetainParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ int s_warp[kRetThreads / 32];
   __shared__ int s_base;
   const int seg = blockIdx.y, chunk = blockIdx.x;
@@ -440,6 +452,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
 // ret_prefix[seg][j] = number of the segment's retained tokens before token 128 * j.
 __global__ void __launch_bounds__(256) retain_prefix_kernel(const int32_t* ret_count, const int32_t* ret_offset,
                                                            const int32_t* ret_index, int32_t* ret_prefix, int stride) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int seg = blockIdx.x;
   const int cnt = ret_count[seg], off = ret_offset[seg];
   for (int j = threadIdx.x; j < stride; j += blockDim.x) {
@@ -468,6 +482,8 @@ struct AppendParams {
 
 template <int DT>
 __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int r = blockIdx.x * (128 / 16) + (threadIdx.x >> 4);
   const int l16 = threadIdx.x & 15;
   const bool ok = r < p.total_rows;
@@ -514,8 +530,7 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
                        const mc_layer_kv* l, const mc_pair_cache* out, int do_retention, void* workspace,
                        cudaStream_t stream) {
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
-  merge_init_kernel<<<(max(nseg, MC_STATUS_WORDS) + 255) / 256, 256, 0, stream>>>(
-      reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status);
+  MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256), dim3(256), 0, stream, reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status));
   MC_CUDA_CHECK(cudaGetLastError());
   if (bt->batch == 0) return MC_OK;
 
@@ -536,9 +551,9 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   if (blocks > 0) {
     if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
     if (cfg->dtype == MC_F16)
-      merge_kernel<MC_F16><<<(unsigned)blocks, kMergeThreads, 0, stream>>>(mp);
+      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_F16>, dim3((unsigned)blocks), dim3(kMergeThreads), 0, stream, mp));
     else
-      merge_kernel<MC_BF16><<<(unsigned)blocks, kMergeThreads, 0, stream>>>(mp);
+      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_BF16>, dim3((unsigned)blocks), dim3(kMergeThreads), 0, stream, mp));
     MC_CUDA_CHECK(cudaGetLastError());
   }
 
@@ -567,14 +582,14 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.do_retention = do_retention;
   rp.gamma = cfg->gamma;
   dim3 grid(rp.chunks_per_seg, nseg);
-  retain_count_kernel<<<grid, kRetThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
   MC_CUDA_CHECK(cudaGetLastError());
-  retain_scan_kernel<<<1, 1024, 0, stream>>>(rp);
+  MC_CUDA_CHECK(launch_pdl(retain_scan_kernel, dim3(1), dim3(1024), 0, stream, rp));
   MC_CUDA_CHECK(cudaGetLastError());
-  retain_compact_kernel<<<grid, kRetThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
   MC_CUDA_CHECK(cudaGetLastError());
-  retain_prefix_kernel<<<nseg, 256, 0, stream>>>(out->ret_count, out->ret_offset, out->ret_index, out->ret_prefix,
-                                                 (int)out->ret_prefix_stride);
+  MC_CUDA_CHECK(launch_pdl(retain_prefix_kernel, dim3(nseg), dim3(256), 0, stream, out->ret_count, out->ret_offset, out->ret_index, out->ret_prefix,
+                                                 (int)out->ret_prefix_stride));
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }
@@ -597,9 +612,9 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   if (ap.total_rows == 0) return MC_OK;
   const int blocks = (ap.total_rows + 7) / 8;
   if (cfg->dtype == MC_F16)
-    append_kernel<MC_F16><<<blocks, 128, 0, stream>>>(ap);
+    MC_CUDA_CHECK(launch_pdl(append_kernel<MC_F16>, dim3(blocks), dim3(128), 0, stream, ap));
   else
-    append_kernel<MC_BF16><<<blocks, 128, 0, stream>>>(ap);
+    MC_CUDA_CHECK(launch_pdl(append_kernel<MC_BF16>, dim3(blocks), dim3(128), 0, stream, ap));
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }

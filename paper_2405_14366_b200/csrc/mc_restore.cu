@@ -25,6 +25,8 @@ struct RestoreParams {
 
 template <int DT>
 __global__ void __launch_bounds__(kRestoreThreads) restore_scale_kernel(const RestoreParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int ipp = p.items_per_page;
   int bid = blockIdx.x;
   const int item = bid % ipp;
@@ -72,6 +74,8 @@ __global__ void __launch_bounds__(kRestoreThreads) restore_scale_kernel(const Re
 }
 
 __global__ void __launch_bounds__(kRestoreThreads) restore_scatter_kernel(const RestoreParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   const int seg = blockIdx.y;
   const int H = p.g.n_kv_heads;
   const int h = seg % H;
@@ -110,14 +114,14 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
   if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
   if (blocks > 0) {
     if (cfg->dtype == MC_F16)
-      restore_scale_kernel<MC_F16><<<(unsigned)blocks, kRestoreThreads, 0, stream>>>(rp);
+      MC_CUDA_CHECK(launch_pdl(restore_scale_kernel<MC_F16>, dim3((unsigned)blocks), dim3(kRestoreThreads), 0, stream, rp));
     else
-      restore_scale_kernel<MC_BF16><<<(unsigned)blocks, kRestoreThreads, 0, stream>>>(rp);
+      MC_CUDA_CHECK(launch_pdl(restore_scale_kernel<MC_BF16>, dim3((unsigned)blocks), dim3(kRestoreThreads), 0, stream, rp));
     MC_CUDA_CHECK(cudaGetLastError());
   }
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
   dim3 grid(4, nseg);
-  restore_scatter_kernel<<<grid, kRestoreThreads, 0, stream>>>(rp);
+  MC_CUDA_CHECK(launch_pdl(restore_scatter_kernel, dim3(grid), dim3(kRestoreThreads), 0, stream, rp));
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }
