@@ -30,7 +30,7 @@
 namespace mc {
 
 constexpr int kTile = 64;  // tokens per pipeline stage
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
@@ -512,9 +512,45 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         const int valid = min(kTile, w.n_tok - t * kTile);
         const int ksteps = (valid + 15) >> 4;
         xv = info_s[2 * s + 1];
+        bool wrote = false;
+        if (valid == kTile) {
+          // full tile: all four 16-token steps unrolled, loads first, no masks
+          uint32_t a0[4], a2[4];
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            a0[kk] = a2[kk] = 0u;
+            if (row < rows) {
+              const int tk = kk * 16;
+              const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk >> shift) * tbytes +
+                                                                ps * kRowBytes) + slot_row * ps + (tk & (ps - 1));
+              const float* srow = S + row * s_stride + t * kTile + tk;
+              const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
+              const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
+              const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
+              const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
+              a0[kk] = Elem<DT>::pack(p0.x * g0.x, p0.y * g0.y);
+              a2[kk] = Elem<DT>::pack(p1.x * g1.x, p1.y * g1.y);
+            }
+          }
+          // token row (kk * 16 + (mi & 1) * 8 + mr): its swizzle term is mr for every kk
+          const uint32_t lane_base = sbase + (uint32_t)(((mi & 1) * 8 + mr) * kRowBytes);
+          const uint32_t pos0 = (uint32_t)chunk_pos(mr, chunk0 + (mi >> 1)) << 4;
+          const uint32_t pos1 = (uint32_t)chunk_pos(mr, chunk0 + 2 + (mi >> 1)) << 4;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const int tk = kk * 16;
+            const uint32_t rowa = lane_base + (uint32_t)((tk >> shift) * tbytes + (tk & (ps - 1)) * kRowBytes);
+            uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+            ldsm_x4_t(rowa + pos0, r0, r1, r2, r3);
+            ldsm_x4_t(rowa + pos1, r4, r5, r6, r7);
+            mma_16816<DT>(acc[0], a0[kk], a2[kk], r0, r1);
+            mma_16816<DT>(acc[1], a0[kk], a2[kk], r2, r3);
+            mma_16816<DT>(acc[2], a0[kk], a2[kk], r4, r5);
+            mma_16816<DT>(acc[3], a0[kk], a2[kk], r6, r7);
+          }
+        } else {
         // rows past the last cached token may hold anything (page tail, page not copied): zero this
         // warp's channels there so that 0 * x stays 0 in the contraction
-        bool wrote = false;
         for (int rz = valid + (lane >> 2); rz < ksteps * 16; rz += 8) {
           const uint32_t a = tile_addr(sbase, rz, chunk0 + (lane & 3), shift, tbytes);
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
@@ -546,6 +582,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
             mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
           }
+        }
         }
         if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
