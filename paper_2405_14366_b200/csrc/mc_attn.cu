@@ -26,6 +26,7 @@
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
+#include "mc_pipe.cuh"
 
 namespace mc {
 
@@ -39,7 +40,6 @@ constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64
 constexpr int kMaxSplit = 512;
 constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
-constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kCtasPerSm = 2;
 
 struct AttnParams {
@@ -68,32 +68,7 @@ struct AttnParams {
   int n_splits;
 };
 
-// ---- PTX wrappers -----------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bulk asynchronous copy global -> shared (TMA engine), completion counted in bytes on an mbarrier.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
+// ---- PTX wrappers (tensor-core side; the copy/barrier wrappers live in mc_pipe.cuh) ---------------
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
@@ -121,20 +96,6 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
   }
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
-
-// Bounded wait: gives up after kWaitLimit polls, records it, and makes every later wait of the
-// CTA (and of CTAs that look at the status word afterwards) return at once.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
-  if (*s_abort) return false;
-  for (uint32_t it = 0; it < kWaitLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (it > 64) __nanosleep(40);
-    if ((it & 1023) == 1023 && (*s_abort || (*(volatile int32_t*)status & MC_FLAG_WAIT_TIMEOUT))) break;
-  }
-  *s_abort = 1;
-  atomicOr(status, MC_FLAG_WAIT_TIMEOUT);
-  return false;
-}
 
 // Shared-memory address of 16-byte chunk `chunk` (0..15) of token row `tk` (0..63) of a stage.
 // A stage holds 64 / page_size tiles back to back, each as in global memory (see tile_bytes).

@@ -7,11 +7,17 @@
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
+#include "mc_pipe.cuh"
 
 namespace mc {
 
-constexpr int kMergeThreads = 256;
-constexpr int kRowsPerItem = 64;  // rows of one page handled by one CTA
+constexpr int kRowsPerItem = 64;  // rows of one page per work item
+constexpr int kMergeStages = 3;
+constexpr int kMergeStageBytes = 2 * kRowsPerItem * kRowBytes;  // the item's rows of layer l-1, then of layer l
+constexpr int kMergeConsumerWarps = 8;
+constexpr int kMergeThreads = kMergeConsumerWarps * 32 + 32;  // + producer warp
+constexpr int kMergeCtasPerSm = 2;
+constexpr int kMergeMaxBatchSmem = 1024;
 
 struct MergeParams {
   Geom g;
@@ -22,6 +28,9 @@ struct MergeParams {
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
   float ta, tc;
   int items_per_page;
+  int pages_used;   // page slots per sequence that can hold tokens
+  int total_items;  // 2 * batch * pages_used * items_per_page
+  int32_t* status;
 };
 
 // One merged row: 16 lanes hold 8 channels each of a (layer l-1) and c (layer l).
@@ -175,89 +184,161 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
   d_out = s.d;
 }
 
+// Work item of the merge: 64 consecutive rows of one page (rows of a page are [head][token], so an
+// item is a contiguous 16 KB block in each layer's pool).  Flattened order: tensor, sequence, page
+// slot, row group -- row group fastest.
+struct MergeItem {
+  int tensor, b, pslot, grp;
+};
+__device__ __forceinline__ bool merge_item(int i, const MergeParams& p, const int* lens, MergeItem& m) {
+  m.grp = i % p.items_per_page;
+  i /= p.items_per_page;
+  m.pslot = i % p.pages_used;
+  i /= p.pages_used;
+  m.b = i % p.g.batch;
+  m.tensor = i / p.g.batch;
+  return m.pslot * p.g.page_size < lens[m.b];
+}
+
+// Persistent merge kernel.  A producer warp streams the items' rows of both layers into a ring of
+// shared-memory stages with bulk asynchronous copies (two 16 KB copies per stage); eight consumer
+// warps take a row per quad of lanes out of shared memory, release the stage, and do Eq. 2 / Eq. 3
+// in registers.  The bytes in flight are set by the ring, not by registers or occupancy.
 template <int DT>
-__global__ void __launch_bounds__(kMergeThreads) merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const MergeParams p) {
   grid_dep_wait();
   grid_dep_launch();
-  __shared__ unsigned s_min[4], s_max[4];
-  const int ipp = p.items_per_page;
-  int bid = blockIdx.x;
-  const int item = bid % ipp;
-  bid /= ipp;
-  const int pslot = bid % p.g.max_pages_per_seq;
-  bid /= p.g.max_pages_per_seq;
-  const int b = bid % p.g.batch;
-  const int tensor = bid / p.g.batch;
-
-  const int n = p.g.seq_lens[b];
-  const int ps = p.g.page_size;
-  if (pslot * ps >= n) return;
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + pslot];
-  const int H = p.g.n_kv_heads;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  unsigned char* stages = smem;
+  int* page_s = reinterpret_cast<int*>(smem + kMergeStages * kMergeStageBytes);  // [kMergeStages] page id of the staged item
+  int* len_s = page_s + kMergeStages;                                            // [min(batch, kMergeMaxBatchSmem)]
+  volatile int* s_abort = len_s + kMergeMaxBatchSmem;
+  uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMergeStages;
+  const uint32_t stage0 = smem_u32(stages);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ps = p.g.page_size, H = p.g.n_kv_heads;
   const int rows_in_page = H * ps;
 
-  if (threadIdx.x < 4) {
-    s_min[threadIdx.x] = 0x7f800000u;
-    s_max[threadIdx.x] = 0u;
+  if (tid == 0) {
+    for (int s = 0; s < kMergeStages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, kMergeConsumerWarps);
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  const bool lens_in_smem = p.g.batch <= kMergeMaxBatchSmem;
+  if (lens_in_smem)
+    for (int b = tid; b < p.g.batch; b += kMergeThreads) len_s[b] = p.g.seq_lens[b];
   __syncthreads();
+  const int* lens = lens_in_smem ? len_s : p.g.seq_lens;
+  const int total = p.total_items;
+  const int stride = gridDim.x;
+  MergeItem m;
+  int i = blockIdx.x;
+  while (i < total && !merge_item(i, p, lens, m)) i += stride;  // first item with tokens
 
-  const int quad = threadIdx.x >> 2, k = threadIdx.x & 3;
-  const int row = item * kRowsPerItem + quad;  // one row per quad of lanes; a warp = 8 consecutive rows of one head
-  const int head = row >> p.g.page_shift;
-  const int tk = row & (ps - 1);
-  const bool valid = row < rows_in_page && pslot * ps + tk < n;
-  const size_t in_off = ((size_t)page * rows_in_page + row) * kRowBytes + k * 16;
-  const char* pa = (tensor ? p.a_pool[1] : p.a_pool[0]) + in_off;
-  const char* pc = (tensor ? p.c_pool[1] : p.c_pool[0]) + in_off;
-  char* tile = (tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + head) * tile_bytes(ps);
+  if (warp == kMergeConsumerWarps) {
+    // ===================== producer =====================
+    int page = 0;
+    if (i < total) page = p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot];
+    for (int it = 0; i < total; ++it) {
+      // the next item and its page id are looked up one item ahead of use
+      MergeItem mn;
+      int j = i + stride;
+      while (j < total && !merge_item(j, p, lens, mn)) j += stride;
+      int next_page = 0;
+      if (j < total) next_page = p.g.block_table[(size_t)mn.b * p.g.max_pages_per_seq + mn.pslot];
+      const int s = it % kMergeStages;
+      int good = 1;
+      if (it >= kMergeStages && lane == 0)
+        good = mbar_wait(empty0 + 8 * s, ((it / kMergeStages) - 1) & 1, s_abort, p.status) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
+      const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
+      const uint32_t bar = full0 + 8 * s;
+      if (lane == 0) {
+        page_s[s] = page;
+        mbar_expect_tx(bar, 2 * bytes);
+      }
+      __syncwarp();
+      if (lane < 2) {
+        const char* pool = lane ? (m.tensor ? p.c_pool[1] : p.c_pool[0]) : (m.tensor ? p.a_pool[1] : p.a_pool[0]);
+        const char* src = pool + ((size_t)page * rows_in_page + m.grp * kRowsPerItem) * kRowBytes;
+        bulk_load(stage0 + s * kMergeStageBytes + lane * (kRowsPerItem * kRowBytes), src, bytes, bar);
+      }
+      i = j;
+      m = mn;
+      page = next_page;
+    }
+    return;
+  }
 
-  uint4 va[4], vc[4];
+  // ===================== consumers =====================
+  const int quad = tid >> 2, k = tid & 3;
+  for (int it = 0; i < total; ++it) {
+    const int s = it % kMergeStages;
+    if (!mbar_wait(full0 + 8 * s, (it / kMergeStages) & 1, s_abort, p.status)) break;
+    const int page = page_s[s];
+    const int n = lens[m.b];
+    const int row = m.grp * kRowsPerItem + quad;  // one row per quad of lanes; a warp = 8 consecutive rows of one head
+    const int head = row >> p.g.page_shift;
+    const int tk = row & (ps - 1);
+    const bool valid = row < rows_in_page && m.pslot * ps + tk < n;
+    // lane k owns the 16-byte chunks k, k + 4, k + 8, k + 12; odd rows fetch them in the order that
+    // keeps the two rows of a quarter-warp in different bank groups
+    const unsigned char* sa = stages + s * kMergeStageBytes + quad * kRowBytes;
+    const unsigned char* sc = sa + kRowsPerItem * kRowBytes;
+    uint4 va[4], vc[4];
+    int ci[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+    for (int x = 0; x < 4; ++x) {
+      ci[x] = ((x ^ (quad & 1)) << 2) + k;
+      va[x] = *reinterpret_cast<const uint4*>(sa + ci[x] * 16);
+      vc[x] = *reinterpret_cast<const uint4*>(sc + ci[x] * 16);
+    }
+    if (!valid) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x) va[x] = vc[x] = make_uint4(0, 0, 0, 0);  // never computed on: page tail
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
+
+    uint4 e[4];
+    float g_a, g_c, d;
+    merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
+    float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
-      va[i] = ld_stream16(pa + i * 64);
-      vc[i] = ld_stream16(pc + i * 64);
-    } else {
-      va[i] = make_uint4(0, 0, 0, 0);
-      vc[i] = make_uint4(0, 0, 0, 0);
-    }
-  }
-  uint4 e[4];
-  float g_a, g_c, d;
-  merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
-  float dmin = __int_as_float(0x7f800000), dmax = 0.f;
-  if (valid) {
+      char* tile = (m.tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + head) * tile_bytes(ps);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) st_stream16(tile + tk * kRowBytes + chunk_pos(tk, i * 4 + k) * 16, e[i]);
-    if (k == 0) {
-      float* sc = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk;
-      sc[0] = g_a;
-      sc[ps] = g_c;
-      p.dist[(((size_t)page * H + head) * 2 + tensor) * ps + tk] = d;
+      for (int x = 0; x < 4; ++x) st_stream16(tile + tk * kRowBytes + chunk_pos(tk, ci[x]) * 16, e[x]);
+      if (k == 0) {
+        float* scp = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk;
+        scp[0] = g_a;
+        scp[ps] = g_c;
+        p.dist[(((size_t)page * H + head) * 2 + m.tensor) * ps + tk] = d;
+      }
+      dmin = d;
+      dmax = d;
     }
-    dmin = d;
-    dmax = d;
-  }
 #pragma unroll
-  for (int o = 4; o < 32; o <<= 1) {
-    dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
-    dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
-  }
-  if ((threadIdx.x & 31) == 0 && dmin != __int_as_float(0x7f800000)) {
-    const int hl = ((threadIdx.x >> 5) * 8) >> p.g.page_shift;  // head inside the item
-    atomicMin(&s_min[hl], __float_as_uint(dmin));
-    atomicMax(&s_max[hl], __float_as_uint(dmax));
-  }
-  __syncthreads();
-  const int heads_per_item = kRowsPerItem >> p.g.page_shift;
-  if ((int)threadIdx.x < heads_per_item) {
-    const int h = (item * kRowsPerItem >> p.g.page_shift) + threadIdx.x;
-    if (h < H && s_min[threadIdx.x] != 0x7f800000u) {
-      const size_t seg = ((size_t)tensor * p.g.batch + b) * H + h;
-      atomicMin(&p.seg_minmax[seg * 2], s_min[threadIdx.x]);
-      atomicMax(&p.seg_minmax[seg * 2 + 1], s_max[threadIdx.x]);
+    for (int o = 4; o < 32; o <<= 1) {
+      dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
+      dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
     }
+    if (lane == 0 && dmin != __int_as_float(0x7f800000)) {  // the warp's 8 rows belong to one head
+      const size_t seg = ((size_t)m.tensor * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
+      atomicMin(&p.seg_minmax[seg * 2], __float_as_uint(dmin));
+      atomicMax(&p.seg_minmax[seg * 2 + 1], __float_as_uint(dmax));
+    }
+    i += stride;
+    while (i < total && !merge_item(i, p, lens, m)) i += stride;
+  }
+  if (*s_abort) {
+    for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
   }
 }
 
@@ -547,14 +628,28 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
-  const long long blocks = 2LL * bt->batch * bt->max_pages_per_seq * mp.items_per_page;
-  if (blocks > 0) {
-    if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
-    if (cfg->dtype == MC_F16)
-      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_F16>, dim3((unsigned)blocks), dim3(kMergeThreads), 0, stream, mp));
-    else
-      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_BF16>, dim3((unsigned)blocks), dim3(kMergeThreads), 0, stream, mp));
-    MC_CUDA_CHECK(cudaGetLastError());
+  mp.pages_used = (bt->max_seq_len + cfg->page_size - 1) / cfg->page_size;
+  const long long total = 2LL * bt->batch * mp.pages_used * mp.items_per_page;
+  if (total > 0x7fffffffLL) return MC_ERR_SHAPE;
+  mp.total_items = (int)total;
+  mp.status = out->status;
+  if (total > 0) {
+    static int n_sm = 0;
+    if (n_sm == 0) {
+      int dev = 0;
+      MC_CUDA_CHECK(cudaGetDevice(&dev));
+      MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    }
+    const int grid = (int)std::min<long long>((long long)n_sm * kMergeCtasPerSm, total);
+    const size_t smem = 128 + (size_t)kMergeStages * kMergeStageBytes + (kMergeStages + kMergeMaxBatchSmem + 2) * 4 + 8 +
+                        2 * kMergeStages * 8 + 64;
+    if (cfg->dtype == MC_F16) {
+      MC_CUDA_CHECK(cudaFuncSetAttribute(merge_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_F16>, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
+    } else {
+      MC_CUDA_CHECK(cudaFuncSetAttribute(merge_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_BF16>, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
+    }
   }
 
   RetainParams rp;
