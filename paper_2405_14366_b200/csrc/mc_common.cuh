@@ -131,21 +131,36 @@ struct RowScalars {
 // Angle and SLERP weights from |a|^2, |c|^2, |u - v|^2, |u + v|^2 (u, v the unit directions).
 // Omega = 2 atan2(|u - v|, |u + v|) is well conditioned at both ends of [0, pi], where arccos
 // of a rounded cosine is not.  ta weights layer l-1, tc layer l (Eq. 3: ta = 1 - t, tc = t).
+// sin(x) for x in [0, pi]: fold to [0, pi/2] and sum the odd Taylor series through x^11 (the first
+// omitted term is below 6e-8 there).  No range reduction, no slow path.
+__device__ __forceinline__ float sin_0_pi(float x) {
+  const float y = x > 1.57079632679489661923f ? 3.14159265358979323846f - x : x;
+  const float y2 = y * y;
+  float p = fmaf(y2, -2.50521083854417187751e-8f, 2.75573192239858906526e-6f);  // -1/11!, 1/9!
+  p = fmaf(p, y2, -1.98412698412698412698e-4f);                                 // -1/7!
+  p = fmaf(p, y2, 8.33333333333333333333e-3f);                                  // 1/5!
+  p = fmaf(p, y2, -1.66666666666666666667e-1f);                                 // -1/3!
+  return fmaf(p * y2, y, y);
+}
+
 __device__ __forceinline__ RowScalars slerp_scalars(float aa, float cc, float sm, float sp, float ta,
                                                     float tc) {
   RowScalars r;
-  r.na = sqrtf(aa);
-  r.nc = sqrtf(cc);
-  const float ra = aa > 0.f ? 1.0f / r.na : 0.f;
-  const float rc = cc > 0.f ? 1.0f / r.nc : 0.f;
+  // 1/|x| by the hardware reciprocal square root (2 ulp); |x| = |x|^2 / |x|
+  const float ra = aa > 0.f ? rsqrtf(aa) : 0.f;
+  const float rc = cc > 0.f ? rsqrtf(cc) : 0.f;
+  r.na = aa * ra;
+  r.nc = cc * rc;
   if (aa > 0.f && cc > 0.f) {
-    const float omega = 2.0f * atan2f(sqrtf(sm), sqrtf(sp));
-    const float sinw = sinf(omega);
+    // h = |u - v| / 2 = sin(Omega / 2), c = |u + v| / 2 = cos(Omega / 2)
+    const float h2 = sm > 0.f ? sm * rsqrtf(sm) : 0.f, c2 = sp > 0.f ? sp * rsqrtf(sp) : 0.f;
+    const float omega = 2.0f * atan2f(h2, c2);
+    const float sinw = 0.5f * h2 * c2;  // sin(Omega) = 2 sin(Omega/2) cos(Omega/2)
     r.d = omega * kInvPi;
     if (sinw >= 1e-6f) {
-      const float inv = 1.0f / sinw;
-      r.fa = sinf(ta * omega) * inv * ra;
-      r.fc = sinf(tc * omega) * inv * rc;
+      const float inv = __fdividef(1.0f, sinw);
+      r.fa = sin_0_pi(ta * omega) * inv * ra;
+      r.fc = sin_0_pi(tc * omega) * inv * rc;
     } else if (sp > sm) {  // same direction: limit of Eq. 3
       r.fa = ta * ra;
       r.fc = tc * rc;

@@ -134,25 +134,29 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
     c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
     c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
   }
-  float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2;
+  float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2, aa3 = aa2, cc3 = aa2;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < 16; i += 2) {
     aa2 = __ffma2_rn(a[i], a[i], aa2);
     cc2 = __ffma2_rn(c[i], c[i], cc2);
+    aa3 = __ffma2_rn(a[i + 1], a[i + 1], aa3);
+    cc3 = __ffma2_rn(c[i + 1], c[i + 1], cc3);
   }
-  const float aa = sum4(aa2.x + aa2.y), cc = sum4(cc2.x + cc2.y);
+  const float aa = sum4((aa2.x + aa2.y) + (aa3.x + aa3.y)), cc = sum4((cc2.x + cc2.y) + (cc3.x + cc3.y));
   const float ia = aa > 0.f ? rsqrtf(aa) : 0.f;
   const float ic = cc > 0.f ? rsqrtf(cc) : 0.f;
   // |u - v|^2 formed channel by channel (no cancellation at small angles); |u + v|^2 = 4 - |u - v|^2
   // is as good until the two directions come close to opposite, where it is formed the same way
   const float2 ia2 = make_float2(ia, ia), nic2 = make_float2(-ic, -ic);
-  float2 sm2 = make_float2(0.f, 0.f);
+  float2 sm2 = make_float2(0.f, 0.f), sm3 = sm2;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < 16; i += 2) {
     const float2 dm = __ffma2_rn(c[i], nic2, __fmul2_rn(a[i], ia2));
+    const float2 dn = __ffma2_rn(c[i + 1], nic2, __fmul2_rn(a[i + 1], ia2));
     sm2 = __ffma2_rn(dm, dm, sm2);
+    sm3 = __ffma2_rn(dn, dn, sm3);
   }
-  const float sm = sum4(sm2.x + sm2.y);
+  const float sm = sum4((sm2.x + sm2.y) + (sm3.x + sm3.y));
   float sp = 4.0f - sm;
   if (__any_sync(0xffffffffu, sm > 3.5f)) {
     const float2 ic2 = make_float2(ic, ic);
@@ -167,16 +171,16 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
   }
   const RowScalars s = slerp_scalars(aa, cc, sm, fmaxf(sp, 0.f), ta, tc);
   const float2 fa2 = make_float2(s.fa, s.fa), fc2 = make_float2(s.fc, s.fc);
-  float ee = 0.f;
+  float ee4[4] = {0.f, 0.f, 0.f, 0.f};
   uint32_t w[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const float2 x = __ffma2_rn(a[i], fa2, __fmul2_rn(c[i], fc2));
     w[i] = Elem<DT>::pack(x.x, x.y);
-    ee = sq_acc<DT>(w[i], ee);  // the stored value: Eq. 2 divides by its length
+    ee4[i & 3] = sq_acc<DT>(w[i], ee4[i & 3]);  // the stored value: Eq. 2 divides by its length
   }
-  ee = sum4(ee);
-  const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
+  const float ee = sum4((ee4[0] + ee4[1]) + (ee4[2] + ee4[3]));
+  const float il = ee > 0.f ? rsqrtf(ee) : 0.f;
 #pragma unroll
   for (int i = 0; i < 4; ++i) e_out[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
   g_a = s.na * il;
@@ -205,7 +209,7 @@ __device__ __forceinline__ bool merge_item(int i, const MergeParams& p, const in
 // warps take a row per quad of lanes out of shared memory, release the stage, and do Eq. 2 / Eq. 3
 // in registers.  The bytes in flight are set by the ring, not by registers or occupancy.
 template <int DT>
-__global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const MergeParams p) {
+__global__ void __maxnreg__(112) merge_kernel(const MergeParams p) {
   grid_dep_wait();
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];

@@ -306,5 +306,7 @@ def compare_attention(p: Problem, om, layer_sel: int, q: torch.Tensor, out: torc
             if lse is not None:
                 lerr = max(lerr, abs(float(lse[si, b, hq]) - l))
     assert err < 1e-2, f"attention output off by {err} (max-abs)"
-    assert lerr < 1e-3, f"log-sum-exp off by {lerr}"
+    # a one-ulp rounding flip of one stored direction element (counted in compare_merge) moves that token's
+    # score by |q_i| * ulp * scale * sm_scale: about 1e-3 in binary16 and 8 times that in bfloat16
+    assert lerr < (2e-3 if p.dtype == "f16" else 1e-2), f"log-sum-exp off by {lerr}"
     return {"attn_abs": err, "lse_abs": lerr}
