@@ -78,8 +78,16 @@ template <int DT>
 struct Elem;
 template <>
 struct Elem<MC_F16> {
+  // binary16 -> binary32 as x * 1 + 0 on the FMA pipe (sm_100 mixed-precision FMA); the plain
+  // conversion instruction runs on the slow transcendental/conversion unit and was the
+  // bottleneck of the merge kernel
   static __device__ __forceinline__ float2 unpack(uint32_t w) {
-    return __half22float2(*reinterpret_cast<const __half2*>(&w));
+    float2 r;
+    asm("{\n\t.reg .b16 lo, hi, one;\n\tmov.b32 {lo, hi}, %2;\n\tmov.b16 one, 0x3C00;\n\t"
+        "fma.rn.f32.f16 %0, lo, one, 0f00000000;\n\tfma.rn.f32.f16 %1, hi, one, 0f00000000;\n\t}"
+        : "=f"(r.x), "=f"(r.y)
+        : "r"(w));
+    return r;
   }
   static __device__ __forceinline__ uint32_t pack(float x, float y) {
     __half2 h = __floats2half2_rn(x, y);
