@@ -178,6 +178,24 @@ class Job:
             self.seq_lens += 1
         self.launches += steps * self.wl.n_pairs * 5
 
+    def decode_pair_all(self, steps):
+        """Pair mode: both layers of a pair in one call (two query sets, one pass over the directions)."""
+        if not hasattr(self, "ws_attn2"):
+            bd = self.batch(True)
+            self.ws_attn2 = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bd, 1, 2), dtype=torch.uint8, device=self.dev)
+            self.out2 = torch.empty(2, self.B, self.Hq, 128, dtype=self.cfg.torch_dtype, device=self.dev)
+            self.new2 = [{"k": torch.stack([nt["k_lm1"], nt["k_l"]]).contiguous(),
+                          "v": torch.stack([nt["v_lm1"], nt["v_l"]]).contiguous()} for nt in self.new]
+        b = self.batch(True)
+        for s in range(steps):
+            q, nt, n2 = self.q[s % len(self.q)], self.new[s % len(self.new)], self.new2[s % len(self.new)]
+            for pr in range(self.wl.n_pairs):
+                pc = self.pairs[pr]
+                self.lib.mc_decode_attn(self.cfg, b, pc, 2, q, n2["k"], n2["v"], self.sm_scale, self.out2, None,
+                                        self.ws_attn2)
+                self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
+            self.seq_lens += 1
+
     def step(self, sample_events=False):
         self.merge_all()
         self.restore_all()
@@ -359,6 +377,20 @@ def main():
     tok_steps = job.steps * float(job.prompt.sum()) + job.B * job.steps * (job.steps - 1) / 2
     phases["decode"] = {"ms": t_d * 1e3, "GB/s": (by["attn"] + by["append"]) / t_d / 1e9,
                         "kv_tokens_per_s": tok_steps * 2 * wl.n_pairs / t_d, "ms_per_decode_step": t_d * 1e3 / job.steps}
+    if 2 * (wl.n_q_heads // wl.n_kv_heads) <= 8:
+        # pair mode (both layers' queries known up front: a replay or speculative setting, not a real
+        # model's layer-by-layer decode): the shared directions are read once for two layers
+        job.merge_all()
+        psteps = min(job.steps, 64)
+        t_p = timed(lambda: job.decode_pair_all(psteps))
+        th_steps = psteps * job.tok_heads + job.B * job.H * psteps * (psteps - 1) // 2
+        pair_bytes = wl.n_pairs * th_steps * (2 * ROW + 16 + 4 * rho * (ROW + 4)) + by["append"] * psteps / job.steps
+        phases["decode_pair_mode"] = {"ms_per_decode_step": t_p * 1e3 / psteps, "GB/s": pair_bytes / t_p / 1e9,
+                                      "kv_tokens_per_s": (psteps * float(job.prompt.sum()) + job.B * psteps * (psteps - 1) / 2)
+                                      * 2 * wl.n_pairs / t_p, "steps": psteps}
+    peak0, _ = measured_hbm_peak()
+    for ph in phases.values():
+        ph["frac_of_measured_hbm"] = ph["GB/s"] / peak0
 
     # ---- end to end: host buffers, copies inside the timed region ----------------------------------
     e2e = None
