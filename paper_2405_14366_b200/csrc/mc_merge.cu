@@ -14,8 +14,8 @@ namespace mc {
 constexpr int kRowsPerItem = 64;  // rows of one page per work item
 constexpr int kMergeStages = 3;
 constexpr int kMergeStageBytes = 2 * kRowsPerItem * kRowBytes;  // the item's rows of layer l-1, then of layer l
-constexpr int kMergeConsumerWarps = 8;
-constexpr int kMergeThreads = kMergeConsumerWarps * 32 + 32;  // + producer warp
+constexpr int kMergeWarps = 8;
+constexpr int kMergeThreads = kMergeWarps * 32;
 constexpr int kMergeCtasPerSm = 2;
 constexpr int kMergeMaxBatchSmem = 1024;
 
@@ -204,12 +204,14 @@ __device__ __forceinline__ bool merge_item(int i, const MergeParams& p, const in
   return m.pslot * p.g.page_size < lens[m.b];
 }
 
-// Persistent merge kernel.  A producer warp streams the items' rows of both layers into a ring of
-// shared-memory stages with bulk asynchronous copies (two 16 KB copies per stage); eight consumer
-// warps take a row per quad of lanes out of shared memory, release the stage, and do Eq. 2 / Eq. 3
-// in registers.  The bytes in flight are set by the ring, not by registers or occupancy.
+// Persistent merge kernel.  The items' rows of both layers are streamed into a ring of shared-memory
+// stages with bulk asynchronous copies (two 16 KB copies per stage), issued two items ahead by lane 0
+// of warp 0; the eight warps take a row per quad of lanes out of shared memory, release the stage,
+// and do Eq. 2 / Eq. 3 in registers.  The bytes in flight are set by the ring, not by registers or
+// occupancy.  (Eight warps, not nine with a dedicated producer: two CTAs of nine warps do not fit
+// the register file of an SM sub-partition.)
 template <int DT>
-__global__ void __maxnreg__(112) merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const MergeParams p) {
   grid_dep_wait();
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];
@@ -228,7 +230,7 @@ __global__ void __maxnreg__(112) merge_kernel(const MergeParams p) {
   if (tid == 0) {
     for (int s = 0; s < kMergeStages; ++s) {
       mbar_init(full0 + 8 * s, 1);
-      mbar_init(empty0 + 8 * s, kMergeConsumerWarps);
+      mbar_init(empty0 + 8 * s, kMergeWarps);
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -240,50 +242,63 @@ __global__ void __maxnreg__(112) merge_kernel(const MergeParams p) {
   const int* lens = lens_in_smem ? len_s : p.g.seq_lens;
   const int total = p.total_items;
   const int stride = gridDim.x;
-  MergeItem m;
-  int i = blockIdx.x;
-  while (i < total && !merge_item(i, p, lens, m)) i += stride;  // first item with tokens
 
-  if (warp == kMergeConsumerWarps) {
-    // ===================== producer =====================
-    int page = 0;
-    if (i < total) page = p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot];
-    for (int it = 0; i < total; ++it) {
-      // the next item and its page id are looked up one item ahead of use
-      MergeItem mn;
-      int j = i + stride;
-      while (j < total && !merge_item(j, p, lens, mn)) j += stride;
-      int next_page = 0;
-      if (j < total) next_page = p.g.block_table[(size_t)mn.b * p.g.max_pages_per_seq + mn.pslot];
-      const int s = it % kMergeStages;
-      int good = 1;
-      if (it >= kMergeStages && lane == 0)
-        good = mbar_wait(empty0 + 8 * s, ((it / kMergeStages) - 1) & 1, s_abort, p.status) ? 1 : 0;
-      good = __shfl_sync(0xffffffffu, good, 0);
-      if (!good) break;
-      const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
-      const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
-      const uint32_t bar = full0 + 8 * s;
-      if (lane == 0) {
-        page_s[s] = page;
-        mbar_expect_tx(bar, 2 * bytes);
-      }
-      __syncwarp();
-      if (lane < 2) {
-        const char* pool = lane ? (m.tensor ? p.c_pool[1] : p.c_pool[0]) : (m.tensor ? p.a_pool[1] : p.a_pool[0]);
-        const char* src = pool + ((size_t)page * rows_in_page + m.grp * kRowsPerItem) * kRowBytes;
-        bulk_load(stage0 + s * kMergeStageBytes + lane * (kRowsPerItem * kRowBytes), src, bytes, bar);
-      }
-      i = j;
-      m = mn;
-      page = next_page;
+  auto next_valid = [&](int i, MergeItem& m) {
+    while (i < total && !merge_item(i, p, lens, m)) i += stride;
+    return i;
+  };
+  auto page_of = [&](int i, const MergeItem& m) {
+    return i < total ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
+  };
+  // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kMergeStages
+  auto issue = [&](int j, const MergeItem& m, int page) -> bool {
+    const int s = j % kMergeStages;
+    if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, p.status)) return false;
+    const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
+    const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
+    const uint32_t bar = full0 + 8 * s;
+    page_s[s] = page;
+    mbar_expect_tx(bar, 2 * bytes);
+    const size_t off = ((size_t)page * rows_in_page + m.grp * kRowsPerItem) * kRowBytes;
+    bulk_load(stage0 + s * kMergeStageBytes, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + off, bytes, bar);
+    bulk_load(stage0 + s * kMergeStageBytes + kRowsPerItem * kRowBytes, (m.tensor ? p.c_pool[1] : p.c_pool[0]) + off, bytes,
+              bar);
+    return true;
+  };
+
+  MergeItem m;
+  int i = next_valid(blockIdx.x, m);
+  // warp 0 looks two items ahead (and loads page ids three ahead: a demand load takes microseconds
+  // while the copies saturate the memory system)
+  MergeItem m1 = m, m2 = m, m3 = m;
+  int i1 = total, i2 = total, i3 = total, pg2 = 0, pg3 = 0;
+  if (warp == 0) {
+    i1 = i < total ? next_valid(i + stride, m1) : total;
+    i2 = i1 < total ? next_valid(i1 + stride, m2) : total;
+    i3 = i2 < total ? next_valid(i2 + stride, m3) : total;
+    const int pg0 = page_of(i, m), pg1 = page_of(i1, m1);
+    pg2 = page_of(i2, m2);
+    pg3 = page_of(i3, m3);
+    if (lane == 0) {
+      if (i < total) issue(0, m, pg0);
+      if (i1 < total) issue(1, m1, pg1);
     }
-    return;
   }
 
-  // ===================== consumers =====================
   const int quad = tid >> 2, k = tid & 3;
   for (int it = 0; i < total; ++it) {
+    if (warp == 0) {
+      // item it + 2 goes into the stage that item it - 1 has just left
+      int good = 1;
+      if (lane == 0 && i2 < total) good = issue(it + 2, m2, pg2) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      i2 = i3;
+      m2 = m3;
+      pg2 = pg3;
+      i3 = i2 < total ? next_valid(i2 + stride, m3) : total;
+      pg3 = page_of(i3, m3);
+    }
     const int s = it % kMergeStages;
     if (!mbar_wait(full0 + 8 * s, (it / kMergeStages) & 1, s_abort, p.status)) break;
     const int page = page_s[s];
@@ -338,8 +353,7 @@ __global__ void __maxnreg__(112) merge_kernel(const MergeParams p) {
       atomicMin(&p.seg_minmax[seg * 2], __float_as_uint(dmin));
       atomicMax(&p.seg_minmax[seg * 2 + 1], __float_as_uint(dmax));
     }
-    i += stride;
-    while (i < total && !merge_item(i, p, lens, m)) i += stride;
+    i = next_valid(i + stride, m);
   }
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
