@@ -146,7 +146,7 @@ class Job:
             pl = self.pools[pr]
             self.lib.mc_merge_pair(self.cfg, b, pl["k_lm1"], pl["v_lm1"], pl["k_l"], pl["v_l"], self.pairs[pr], True,
                                    self.ws_merge)
-        self.launches += 5 * self.wl.n_pairs
+        self.launches += 4 * self.wl.n_pairs  # init, merge, count(+scan), compact
 
     def restore_all(self):
         b = self.batch(False)

@@ -381,6 +381,8 @@ struct RetainParams {
   char* ret_rows;
   int64_t ret_capacity;
   int32_t* status;
+  int32_t* ret_prefix;
+  int ret_prefix_stride;
   int chunks_per_seg;
   int nseg;
   int mode;
@@ -406,134 +408,152 @@ __device__ __forceinline__ bool keep_token(float d, float dmin, float dmax, doub
   return (double)d < lo + (hi - lo) * gamma;
 }
 
-__device__ __forceinline__ float load_dist(const RetainParams& p, int tensor, int b, int h, int tok) {
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
-  return p.dist[(((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok & (p.g.page_size - 1))];
+// The four consecutive distances of thread `t` of a chunk (tokens tok0 .. tok0 + 3 lie in one page).
+__device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, int b, int h, int tok0) {
+  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
+  return *reinterpret_cast<const float4*>(
+      p.dist + (((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok0 & (p.g.page_size - 1)));
 }
 
+// Bit j set = token tok0 + j is kept.
+__device__ __forceinline__ unsigned keep_mask4(const RetainParams& p, int tensor, int b, int h, int tok0, int n, float dmin,
+                                               float dmax) {
+  if (tok0 >= n) return 0u;
+  const float4 d = load_dist4(p, tensor, b, h, tok0);
+  unsigned m = 0u;
+  if (keep_token(d.x, dmin, dmax, p.gamma, p.mode)) m |= 1u;
+  if (tok0 + 1 < n && keep_token(d.y, dmin, dmax, p.gamma, p.mode)) m |= 2u;
+  if (tok0 + 2 < n && keep_token(d.z, dmin, dmax, p.gamma, p.mode)) m |= 4u;
+  if (tok0 + 3 < n && keep_token(d.w, dmin, dmax, p.gamma, p.mode)) m |= 8u;
+  return m;
+}
+
+// Per (segment, 1024-token chunk): how many tokens Eq. 4 keeps.  The block that finishes last
+// (ticket in a status word) turns the counts into offsets: exclusive scan in (segment, chunk) order.
 __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainParams p) {
   grid_dep_wait();
   grid_dep_launch();
   __shared__ int s_cnt[kRetThreads / 32];
+  __shared__ int s_last;
+  __shared__ int s_carry;
   const int seg = blockIdx.y, chunk = blockIdx.x;
   const int h = seg % p.g.n_kv_heads;
   const int b = (seg / p.g.n_kv_heads) % p.g.batch;
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
   const int n = p.g.seq_lens[b];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int cnt = 0;
   if (p.do_retention && chunk * kChunk < n) {
     const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
-    for (int i = threadIdx.x; i < kChunk; i += kRetThreads) {
-      const int tok = chunk * kChunk + i;
-      if (tok < n) cnt += keep_token(load_dist(p, tensor, b, h, tok), dmin, dmax, p.gamma, p.mode) ? 1 : 0;
-    }
+    cnt = __popc(keep_mask4(p, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, dmin, dmax));
   }
   for (int o = 16; o; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-  if ((threadIdx.x & 31) == 0) s_cnt[threadIdx.x >> 5] = cnt;
+  if (lane == 0) s_cnt[warp] = cnt;
   __syncthreads();
   if (threadIdx.x == 0) {
     int t = 0;
     for (int w = 0; w < kRetThreads / 32; ++w) t += s_cnt[w];
     p.chunk_count[(size_t)seg * p.chunks_per_seg + chunk] = t;
+    __threadfence();
+    const int ticket = atomicAdd(&p.status[MC_STATUS_RESERVED1], 1);
+    s_last = ticket == (int)(gridDim.x * gridDim.y) - 1;
+    s_carry = 0;
   }
-}
-
-// One CTA: exclusive scan of the chunk counts in (segment, chunk) order.
-__global__ void __launch_bounds__(1024) retain_scan_kernel(const RetainParams p) {
-  grid_dep_wait();
-  grid_dep_launch();
-  __shared__ int s_warp[32];
-  __shared__ int s_carry;
-  const int total = p.nseg * p.chunks_per_seg;
-  if (threadIdx.x == 0) s_carry = 0;
   __syncthreads();
-  for (int base = 0; base < total; base += 1024) {
+  if (!s_last) return;
+  __threadfence();
+  // ---- last block: exclusive scan of all chunk counts
+  const int total = p.nseg * p.chunks_per_seg;
+  for (int base = 0; base < total; base += kRetThreads) {
     const int i = base + threadIdx.x;
-    const int v = i < total ? p.chunk_count[i] : 0;
+    const int v = i < total ? __ldcg(p.chunk_count + i) : 0;
     int x = v;
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, x, o);
-      if ((threadIdx.x & 31) >= o) x += y;
+      if (lane >= o) x += y;
     }
-    if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = x;
+    if (lane == 31) s_cnt[warp] = x;
     __syncthreads();
-    if (threadIdx.x < 32) {
-      int w = s_warp[threadIdx.x];
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, w, o);
-        if ((int)threadIdx.x >= o) w += y;
-      }
-      s_warp[threadIdx.x] = w;  // inclusive over warps
-    }
-    __syncthreads();
-    const int warp_excl = (threadIdx.x >> 5) ? s_warp[(threadIdx.x >> 5) - 1] : 0;
+    int warp_excl = 0;
+    for (int w = 0; w < warp; ++w) warp_excl += s_cnt[w];
     const int excl = s_carry + warp_excl + x - v;
     if (i < total) {
       p.chunk_offset[i] = excl;
       if (i % p.chunks_per_seg == 0) p.ret_offset[i / p.chunks_per_seg] = excl;
     }
     __syncthreads();
-    if (threadIdx.x == 1023) s_carry = excl + v;
+    if (threadIdx.x == kRetThreads - 1) s_carry = excl + v;
     __syncthreads();
   }
   if (threadIdx.x == 0) {
     const int sum = s_carry;
     p.ret_offset[p.nseg] = sum;
     p.status[MC_STATUS_RETAINED_TOTAL] = sum;
+    p.status[MC_STATUS_RESERVED1] = 0;
     if ((int64_t)sum > p.ret_capacity) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_RETAIN_OVERFLOW);
   }
 }
 
-// Per (segment, chunk): ordered compaction of the kept token indices, then bit copies of both
-// layers' rows.  Writes ret_count per segment from the chunk offsets.
+// Per (segment, chunk): ordered compaction of the kept token indices, their scales zeroed, bit copies
+// of both layers' rows, and the chunk's eight entries of the prefix table (one per 128 tokens =
+// one warp).  Writes ret_count per segment.
 __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const RetainParams p) {
   grid_dep_wait();
   grid_dep_launch();
   __shared__ int s_warp[kRetThreads / 32];
-  __shared__ int s_base;
   const int seg = blockIdx.y, chunk = blockIdx.x;
   const int h = seg % p.g.n_kv_heads;
   const int b = (seg / p.g.n_kv_heads) % p.g.batch;
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
   const int n = p.g.seq_lens[b];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool overflow = (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
-  if (chunk == 0 && threadIdx.x == 0)
-    p.ret_count[seg] = overflow ? 0 : p.ret_offset[seg + 1] - p.ret_offset[seg];
-  if (overflow || !p.do_retention || chunk * kChunk >= n) return;
+  const int seg_off = p.ret_offset[seg];
+  const int seg_cnt = overflow ? 0 : p.ret_offset[seg + 1] - seg_off;
+  if (chunk == 0 && threadIdx.x == 0) p.ret_count[seg] = seg_cnt;
+  int32_t* prefix = p.ret_prefix + (size_t)seg * p.ret_prefix_stride;
+  if (chunk == 0)  // table entries past the last chunk: everything lies before them
+    for (int j = p.chunks_per_seg * (kChunk / 128) + threadIdx.x; j < p.ret_prefix_stride; j += kRetThreads) prefix[j] = seg_cnt;
+  const int pj = chunk * (kChunk / 128) + warp;  // this warp's 128 tokens start at table entry pj
+  const bool active = !overflow && p.do_retention && chunk * kChunk < n;
+  if (!active) {
+    if (lane == 0 && pj < p.ret_prefix_stride) prefix[pj] = seg_cnt;  // chunk past the sequence (or nothing retained)
+    return;
+  }
   const size_t ci = (size_t)seg * p.chunks_per_seg + chunk;
   const int my_count = p.chunk_count[ci];
-  if (my_count == 0) return;
   const int out0 = p.chunk_offset[ci];
   const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
-  if (threadIdx.x == 0) s_base = 0;
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int r = 0; r < kChunk; r += kRetThreads) {
-    const int tok = chunk * kChunk + r + threadIdx.x;
-    const bool keep = tok < n && keep_token(load_dist(p, tensor, b, h, tok), dmin, dmax, p.gamma, p.mode);
-    const unsigned m = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) s_warp[warp] = __popc(m);
-    __syncthreads();
-    int before = s_base;
-    for (int w = 0; w < warp; ++w) before += s_warp[w];
-    if (keep) {
-      p.ret_index[out0 + before + __popc(m & ((1u << lane) - 1))] = tok;
-      // a retained token is served from its raw rows: its scales are never read again, and zero
-      // makes the shared direction contribute nothing for it wherever scales are applied blindly
-      const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
-      float* sc = reinterpret_cast<float*>(p.e_pool[tensor] + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
-                                           p.g.page_size * kRowBytes) + (tok & (p.g.page_size - 1));
-      sc[0] = 0.f;
-      sc[p.g.page_size] = 0.f;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int t = s_base;
-      for (int w = 0; w < kRetThreads / 32; ++w) t += s_warp[w];
-      s_base = t;
-    }
-    __syncthreads();
+  const int tok0 = chunk * kChunk + 4 * threadIdx.x;
+  const unsigned m = keep_mask4(p, tensor, b, h, tok0, n, dmin, dmax);
+  const int c = __popc(m);
+  int x = c;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
   }
+  if (lane == 31) s_warp[warp] = x;
+  __syncthreads();
+  int before = 0;
+  for (int w = 0; w < warp; ++w) before += s_warp[w];
+  if (lane == 0 && pj < p.ret_prefix_stride) prefix[pj] = out0 - seg_off + before;
+  int pos = out0 + before + x - c;
+  if (m) {
+    const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
+    float* sc = reinterpret_cast<float*>(p.e_pool[tensor] + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
+                                         p.g.page_size * kRowBytes) + (tok0 & (p.g.page_size - 1));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (m & (1u << j)) {
+        p.ret_index[pos++] = tok0 + j;
+        // a retained token is served from its raw rows: its scales are never read again, and zero
+        // makes the shared direction contribute nothing for it wherever scales are applied blindly
+        sc[j] = 0.f;
+        sc[p.g.page_size + j] = 0.f;
+      }
+    }
+  }
+  __syncthreads();
   // gather: one half-warp per (entry, layer): the raw row and the token index behind it
   const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
   for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
@@ -545,24 +565,6 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
     *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
     if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok, 0, 0, 0);
-  }
-}
-
-// ret_prefix[seg][j] = number of the segment's retained tokens before token 128 * j.
-__global__ void __launch_bounds__(256) retain_prefix_kernel(const int32_t* ret_count, const int32_t* ret_offset,
-                                                           const int32_t* ret_index, int32_t* ret_prefix, int stride) {
-  grid_dep_wait();
-  grid_dep_launch();
-  const int seg = blockIdx.x;
-  const int cnt = ret_count[seg], off = ret_offset[seg];
-  for (int j = threadIdx.x; j < stride; j += blockDim.x) {
-    const int key = j * 128;
-    int lo = 0, hi = cnt;
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if (ret_index[off + mid] < key) lo = mid + 1; else hi = mid;
-    }
-    ret_prefix[(size_t)seg * stride + j] = lo;
   }
 }
 
@@ -691,19 +693,14 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.ret_rows = (char*)out->ret_rows;
   rp.ret_capacity = out->ret_capacity;
   rp.status = out->status;
+  rp.ret_prefix = out->ret_prefix;
+  rp.ret_prefix_stride = (int)out->ret_prefix_stride;
   rp.mode = cfg->retain_mode;
   rp.do_retention = do_retention;
   rp.gamma = cfg->gamma;
   dim3 grid(rp.chunks_per_seg, nseg);
   MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
-  MC_CUDA_CHECK(cudaGetLastError());
-  MC_CUDA_CHECK(launch_pdl(retain_scan_kernel, dim3(1), dim3(1024), 0, stream, rp));
-  MC_CUDA_CHECK(cudaGetLastError());
   MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
-  MC_CUDA_CHECK(cudaGetLastError());
-  MC_CUDA_CHECK(launch_pdl(retain_prefix_kernel, dim3(nseg), dim3(256), 0, stream, out->ret_count, out->ret_offset, out->ret_index, out->ret_prefix,
-                                                 (int)out->ret_prefix_stride));
-  MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }
 
