@@ -33,6 +33,10 @@ for _p in (ROOT, os.path.join(ROOT, "tests")):
 import gen  # noqa: E402
 
 ROW = 256  # bytes of one 16-bit row of 128 channels
+# DRAM bytes (read + written) per algorithmic byte of the split attention kernel, from the ncu capture
+# summarised in profiles/attn_split_kernel_c2_one_pair.md (563.3 MB for 547.8 MB).  Set to None when
+# the kernel changes until it is captured again.
+ATTN_TRAFFIC_RATIO = 1.028
 
 
 # ---------------------------------------------------------------------------------------------
@@ -363,7 +367,8 @@ def main():
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
     roofline = {"kernel": "attn_split_kernel (+attn_combine_kernel)", "bound": "hbm", "achieved": achieved,
                 "peak": peak, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0,
-                "peak_source": peak_src, "traffic": None, "launch_ms": attn_ms, "launches_timed": len(ev_ms),
+                "peak_source": peak_src,
+                "traffic": (float(attn_bytes) * ATTN_TRAFFIC_RATIO if ATTN_TRAFFIC_RATIO and wl.name.startswith("c2") else None), "launch_ms": attn_ms, "launches_timed": len(ev_ms),
                 "algorithmic_bytes_per_launch": float(attn_bytes)}
 
     # ---- per-phase breakdown (outside the headline region) ----------------------------------------
