@@ -62,7 +62,7 @@ typedef enum { MC_F16 = 0, MC_BF16 = 1 } mc_dtype;
  * DISTINCT: d_i > d_max - (d_max - d_min) * gamma  (Eq. 4 applied to similarity 1 - d: the most
  *           distinct pairs are kept, as the text around Eq. 4 describes; gamma = 0 keeps none).
  * LITERAL : d_i < d_min + (d_max - d_min) * gamma  (Eq. 4 exactly as printed).
- * TOPK    : the ceil(gamma * n) largest d (ties: lower index first). */
+ * TOPK    : the ceil(gamma * n) largest d of the segment (ties: lower index first). */
 typedef enum { MC_RETAIN_DISTINCT = 0, MC_RETAIN_LITERAL = 1, MC_RETAIN_TOPK = 2 } mc_retain_mode;
 
 /* Which layer of the pair a call restores / attends for. BOTH = the two layers at once

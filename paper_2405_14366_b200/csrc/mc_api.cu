@@ -117,7 +117,6 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
   if (!lm1 || !l || !lm1->k_pool || !lm1->v_pool || !l->k_pool || !l->v_pool) return MC_ERR_INVALID_ARG;
   if (!aligned256(lm1->k_pool) || !aligned256(lm1->v_pool) || !aligned256(l->k_pool) || !aligned256(l->v_pool))
     return MC_ERR_ALIGN;
-  if (do_retention && cfg->retain_mode == MC_RETAIN_TOPK) return MC_ERR_UNSUPPORTED;
   if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
   if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
   if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;

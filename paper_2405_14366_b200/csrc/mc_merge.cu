@@ -375,6 +375,8 @@ struct RetainParams {
   const float* seg_minmax;
   int32_t* chunk_count;   // workspace [nseg][chunks_per_seg]
   int32_t* chunk_offset;  // workspace [nseg][chunks_per_seg]
+  int32_t* chunk_eq;      // workspace [nseg][chunks_per_seg], top-k mode: tokens equal to the k-th largest d (count, then count before the chunk)
+  uint32_t* seg_sel;      // workspace [nseg][2], top-k mode: bits of the k-th largest d, how many tokens equal to it are kept
   int32_t* ret_count;
   int32_t* ret_offset;
   int32_t* ret_index;
@@ -415,17 +417,90 @@ __device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, 
       p.dist + (((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok0 & (p.g.page_size - 1)));
 }
 
-// Bit j set = token tok0 + j is kept.
-__device__ __forceinline__ unsigned keep_mask4(const RetainParams& p, int tensor, int b, int h, int tok0, int n, float dmin,
-                                               float dmax) {
-  if (tok0 >= n) return 0u;
-  const float4 d = load_dist4(p, tensor, b, h, tok0);
-  unsigned m = 0u;
-  if (keep_token(d.x, dmin, dmax, p.gamma, p.mode)) m |= 1u;
-  if (tok0 + 1 < n && keep_token(d.y, dmin, dmax, p.gamma, p.mode)) m |= 2u;
-  if (tok0 + 2 < n && keep_token(d.z, dmin, dmax, p.gamma, p.mode)) m |= 4u;
-  if (tok0 + 3 < n && keep_token(d.w, dmin, dmax, p.gamma, p.mode)) m |= 8u;
-  return m;
+// Masks over the thread's four tokens: `sure` = kept whatever the ties do, `eq` = kept only while the
+// segment's quota of ties lasts (top-k mode: d equal to the k-th largest; ties go to lower indices).
+__device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
+                                            unsigned& sure, unsigned& eq) {
+  sure = eq = 0u;
+  if (tok0 >= n) return;
+  const float4 d4 = load_dist4(p, tensor, b, h, tok0);
+  const float d[4] = {d4.x, d4.y, d4.z, d4.w};
+  if (p.mode == MC_RETAIN_TOPK) {
+    const uint32_t v = p.seg_sel[2 * seg];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (tok0 + j < n) {
+        const uint32_t key = __float_as_uint(d[j]);
+        if (key > v) sure |= 1u << j;
+        if (key == v) eq |= 1u << j;
+      }
+    }
+  } else {
+    const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (tok0 + j < n && keep_token(d[j], dmin, dmax, p.gamma, p.mode)) sure |= 1u << j;
+  }
+}
+
+// Top-k reading of the retention rule: per segment, the k-th largest distance (k = ceil(gamma n)) by a
+// radix select over the float bits (d >= 0, so unsigned order is float order), and how many of the
+// tokens equal to it belong to the k largest.
+__global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const RetainParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
+  __shared__ int hist[256];
+  __shared__ uint32_t s_prefix, s_mask;
+  __shared__ int s_remaining;
+  const int seg = blockIdx.x;
+  const int h = seg % p.g.n_kv_heads;
+  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
+  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  const int n = p.g.seq_lens[b];
+  const int k = min(n, (int)ceil(p.gamma * (double)n - 1e-12));
+  if (k <= 0 || !p.do_retention) {
+    if (threadIdx.x == 0) {
+      p.seg_sel[2 * seg] = 0xffffffffu;  // nothing is larger, nothing is equal
+      p.seg_sel[2 * seg + 1] = 0u;
+    }
+    return;
+  }
+  if (threadIdx.x == 0) {
+    s_prefix = 0u;
+    s_mask = 0u;
+    s_remaining = k;
+  }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix, mask = s_mask;
+    for (int tok0 = 4 * threadIdx.x; tok0 < n; tok0 += 4 * kRetThreads) {
+      const float4 d4 = load_dist4(p, tensor, b, h, tok0);
+      const float d[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t key = __float_as_uint(d[j]);
+        if (tok0 + j < n && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int remaining = s_remaining, bin = 255;
+      for (; bin > 0; --bin) {  // from the largest digit down: the bin holding the `remaining`-th largest key
+        if (hist[bin] >= remaining) break;
+        remaining -= hist[bin];
+      }
+      s_remaining = remaining;
+      s_prefix = prefix | ((uint32_t)bin << shift);
+      s_mask = mask | (255u << shift);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    p.seg_sel[2 * seg] = s_prefix;                  // the k-th largest distance
+    p.seg_sel[2 * seg + 1] = (uint32_t)s_remaining;  // of the tokens equal to it, this many (the lowest indices) are kept
+  }
 }
 
 // Per (segment, 1024-token chunk): how many tokens Eq. 4 keeps.  The block that finishes last
@@ -433,7 +508,7 @@ __device__ __forceinline__ unsigned keep_mask4(const RetainParams& p, int tensor
 __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainParams p) {
   grid_dep_wait();
   grid_dep_launch();
-  __shared__ int s_cnt[kRetThreads / 32];
+  __shared__ int s_cnt[kRetThreads / 32], s_eq[kRetThreads / 32];
   __shared__ int s_last;
   __shared__ int s_carry;
   const int seg = blockIdx.y, chunk = blockIdx.x;
@@ -442,18 +517,30 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainP
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
   const int n = p.g.seq_lens[b];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int cnt = 0;
+  int cnt = 0, cnt_eq = 0;
   if (p.do_retention && chunk * kChunk < n) {
-    const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
-    cnt = __popc(keep_mask4(p, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, dmin, dmax));
+    unsigned sure, eq;
+    keep_masks4(p, seg, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, sure, eq);
+    cnt = __popc(sure);
+    cnt_eq = __popc(eq);
   }
-  for (int o = 16; o; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-  if (lane == 0) s_cnt[warp] = cnt;
+  for (int o = 16; o; o >>= 1) {
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, o);
+  }
+  if (lane == 0) {
+    s_cnt[warp] = cnt;
+    s_eq[warp] = cnt_eq;
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
-    int t = 0;
-    for (int w = 0; w < kRetThreads / 32; ++w) t += s_cnt[w];
+    int t = 0, te = 0;
+    for (int w = 0; w < kRetThreads / 32; ++w) {
+      t += s_cnt[w];
+      te += s_eq[w];
+    }
     p.chunk_count[(size_t)seg * p.chunks_per_seg + chunk] = t;
+    p.chunk_eq[(size_t)seg * p.chunks_per_seg + chunk] = te;
     __threadfence();
     const int ticket = atomicAdd(&p.status[MC_STATUS_RESERVED1], 1);
     s_last = ticket == (int)(gridDim.x * gridDim.y) - 1;
@@ -462,7 +549,24 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainP
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // ---- last block: exclusive scan of all chunk counts
+  // ---- last block.  Top-k mode first: the ties are handed out in token order, so per segment the
+  // chunks take from the quota one after the other; chunk_eq becomes "ties before this chunk".
+  if (p.mode == MC_RETAIN_TOPK) {
+    for (int sg = threadIdx.x; sg < p.nseg; sg += kRetThreads) {
+      const int quota = (int)p.seg_sel[2 * sg + 1];
+      int eq_run = 0;
+      for (int c = 0; c < p.chunks_per_seg; ++c) {
+        const size_t ci = (size_t)sg * p.chunks_per_seg + c;
+        const int e = __ldcg(p.chunk_eq + ci);
+        p.chunk_count[ci] = __ldcg(p.chunk_count + ci) + max(0, min(e, quota - eq_run));
+        p.chunk_eq[ci] = eq_run;
+        eq_run += e;
+      }
+    }
+    __threadfence();
+    __syncthreads();
+  }
+  // exclusive scan of all chunk counts
   const int total = p.nseg * p.chunks_per_seg;
   for (int base = 0; base < total; base += kRetThreads) {
     const int i = base + threadIdx.x;
@@ -523,9 +627,30 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   const size_t ci = (size_t)seg * p.chunks_per_seg + chunk;
   const int my_count = p.chunk_count[ci];
   const int out0 = p.chunk_offset[ci];
-  const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
   const int tok0 = chunk * kChunk + 4 * threadIdx.x;
-  const unsigned m = keep_mask4(p, tensor, b, h, tok0, n, dmin, dmax);
+  unsigned m, m_eq;
+  keep_masks4(p, seg, tensor, b, h, tok0, n, m, m_eq);
+  if (p.mode == MC_RETAIN_TOPK) {
+    // ties: kept while the segment's quota lasts, in token order (ordered count of the ties before each)
+    const int ce = __popc(m_eq);
+    int xe = ce;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, xe, o);
+      if (lane >= o) xe += y;
+    }
+    if (lane == 31) s_warp[warp] = xe;
+    __syncthreads();
+    int seen = p.chunk_eq[ci] + xe - ce;
+    for (int w = 0; w < warp; ++w) seen += s_warp[w];
+    const int quota = (int)p.seg_sel[2 * seg + 1];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (m_eq & (1u << j)) {
+        if (seen < quota) m |= 1u << j;
+        ++seen;
+      }
+    __syncthreads();
+  }
   const int c = __popc(m);
   int x = c;
   for (int o = 1; o < 32; o <<= 1) {
@@ -624,7 +749,7 @@ static inline int chunks_per_seg(int max_seq_len) { return max_seq_len > 0 ? (ma
 
 size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
   const size_t nseg = (size_t)2 * bt->batch * cfg->n_kv_heads;
-  return align_up(nseg * chunks_per_seg(bt->max_seq_len) * sizeof(int32_t), 256) * 2;
+  return align_up(nseg * chunks_per_seg(bt->max_seq_len) * sizeof(int32_t), 256) * 3 + align_up(nseg * 2 * sizeof(uint32_t), 256);
 }
 
 mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
@@ -685,8 +810,10 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.chunks_per_seg = chunks_per_seg(bt->max_seq_len);
   rp.nseg = nseg;
   rp.chunk_count = reinterpret_cast<int32_t*>(workspace);
-  rp.chunk_offset = reinterpret_cast<int32_t*>((char*)workspace +
-                                               align_up((size_t)nseg * rp.chunks_per_seg * sizeof(int32_t), 256));
+  const size_t arr = align_up((size_t)nseg * rp.chunks_per_seg * sizeof(int32_t), 256);
+  rp.chunk_offset = reinterpret_cast<int32_t*>((char*)workspace + arr);
+  rp.chunk_eq = reinterpret_cast<int32_t*>((char*)workspace + 2 * arr);
+  rp.seg_sel = reinterpret_cast<uint32_t*>((char*)workspace + 3 * arr);
   rp.ret_count = out->ret_count;
   rp.ret_offset = out->ret_offset;
   rp.ret_index = out->ret_index;
@@ -699,6 +826,8 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.do_retention = do_retention;
   rp.gamma = cfg->gamma;
   dim3 grid(rp.chunks_per_seg, nseg);
+  if (cfg->retain_mode == MC_RETAIN_TOPK)
+    MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg), dim3(kRetThreads), 0, stream, rp));
   MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
   MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
   return MC_OK;

@@ -86,9 +86,6 @@ def test_merge_rejects_bad_arguments_without_launching(lib):
     # block table narrower than max_seq_len
     b2 = _batch(mpps=2, max_len=64)
     assert L.mc_merge_pair(C.byref(c), C.byref(b2), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 2
-    # top-k retention is not built on the device
-    ck = _cfg(retain_mode=2)
-    assert L.mc_merge_pair(C.byref(ck), C.byref(b), C.byref(a), C.byref(a), C.byref(pc), 1, ws, 1 << 20, None) == 6
     # pair cache with a missing buffer
     pc2 = B._PairCache(0x30000, 0, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
     assert L.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(a), C.byref(pc2), 1, ws, 1 << 20, None) == 1

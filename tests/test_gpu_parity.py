@@ -77,16 +77,40 @@ def test_tiny_shapes(H, n, dtype, hkv, hq, ps):
     _full_cycle(H, p)
 
 
-@pytest.mark.parametrize("gamma,mode", [(0.0, "distinct"), (1.0, "distinct"), (0.2, "distinct"), (0.05, "literal"), (0.5, "literal")])
+@pytest.mark.parametrize("gamma,mode", [(0.0, "distinct"), (1.0, "distinct"), (0.2, "distinct"), (0.05, "literal"), (0.5, "literal"),
+                                        (0.05, "topk"), (0.3, "topk"), (0.0, "topk"), (1.0, "topk")])
 def test_retention_modes(H, gamma, mode):
     wl = CONFIGS["c1"].scaled("ret", n_kv_heads=4, n_q_heads=4, batch=2, seq_len=300, outlier_frac=0.05, index=77)
-    p = H.Problem(wl, gamma=gamma, retain_mode={"distinct": 0, "literal": 1}[mode], seq_lens=[300, 211])
+    p = H.Problem(wl, gamma=gamma, retain_mode={"distinct": 0, "literal": 1, "topk": 2}[mode], seq_lens=[300, 211])
     stats = _full_cycle(H, p, mode=mode)
     dc = p.device_cache()
     if gamma == 0.0:
         assert dc["ret_count"].sum() == 0  # gamma = 0: everything merged
+    if mode == "topk":  # exactly ceil(gamma n) tokens per segment
+        for b, n in enumerate((300, 211)):
+            assert np.all(dc["ret_count"][:, b] == math.ceil(gamma * n - 1e-12))
     if gamma == 1.0 and mode == "distinct":
         assert dc["ret_count"].sum() >= 2 * 4 * (300 + 211) - 2 * 2 * 4  # all but the least distinct token(s)
+
+
+def test_topk_ties_go_to_lower_indices(H):
+    """Many token pairs with exactly equal distance (a zero row has d = 0 by definition on both sides):
+    the k largest include some of them, and which ones is decided by token index."""
+    wl = CONFIGS["c1"].scaled("ties", n_kv_heads=2, n_q_heads=2, batch=1, seq_len=1500, index=83, outlier_frac=0.02)
+    t = gen.make_pair_tensors(wl, 0)
+    keep_distinct = np.arange(1500) % 5 == 0  # every fifth token keeps its planted angle, the rest get d = 0
+    for name in ("k", "v"):
+        t[name + "_lm1"][0, ~torch.from_numpy(keep_distinct)] = 0
+    p = H.Problem(wl, tensors=t, gamma=0.5, retain_mode=2)
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge("topk")
+    dc = p.device_cache()
+    H.compare_merge(p, om, dc, "topk")
+    got, _ = p.retained(dc, 0, 0, 0)
+    assert len(got) == 750
+    zeros = np.nonzero(~keep_distinct)[0]
+    assert set(got) == set(np.nonzero(keep_distinct)[0]) | set(zeros[:750 - keep_distinct.sum()])
 
 
 def test_no_retention_flag(H):
