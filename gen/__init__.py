@@ -18,4 +18,5 @@ from .workload import (  # noqa: F401
     from_paged,
     torch_dtype,
     as_bits,
+    quantise_q4,
 )

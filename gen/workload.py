@@ -239,3 +239,32 @@ def from_paged(pool: torch.Tensor, block_table: torch.Tensor, seq_len: int) -> t
     perm = (0, 1, 3, 2) + tuple(range(4, 4 + len(rest)))
     g = g.permute(*perm).reshape(bt.shape[0], npg * ps, H, *rest)
     return g[:, :seq_len]
+
+
+def quantise_q4(x: torch.Tensor, kind: str) -> Dict[str, torch.Tensor]:
+    """4-bit input layers for the serving-mix workload (data preparation, KIVI's asymmetric scheme,
+    groups of 32): x [B][S][H][128] 16-bit, S a multiple of 32.
+
+    kind "k": per channel, a group = 32 consecutive tokens; meta [B][S/32][H][128][2] (scale, zero).
+    kind "v": per token, a group = 32 consecutive channels; meta [B][S][H][4][2].
+    codes [B][S][H][64] uint8, channel 2i in the low nibble of byte i, channel 2i+1 in the high one.
+    scale = (max - min) / 15 and zero = min are stored in binary16; a constant group gets scale 1."""
+    B, S, H, D = x.shape
+    assert S % 32 == 0 and D == 128
+    xf = x.double()
+    if kind == "k":
+        g = xf.view(B, S // 32, 32, H, D)
+        lo, hi = g.amin(2), g.amax(2)  # [B][S/32][H][D]
+    else:
+        g = xf.view(B, S, H, 4, 32)
+        lo, hi = g.amin(-1), g.amax(-1)  # [B][S][H][4]
+    scale = ((hi - lo) / 15.0).to(torch.float16)
+    zero = lo.to(torch.float16)
+    scale = torch.where(scale == 0, torch.ones_like(scale), scale)
+    if kind == "k":
+        q = torch.clamp(torch.round((g - zero.double()[:, :, None]) / scale.double()[:, :, None]), 0, 15).view(B, S, H, D)
+    else:
+        q = torch.clamp(torch.round((g - zero.double()[..., None]) / scale.double()[..., None]), 0, 15).view(B, S, H, D)
+    q = q.to(torch.uint8)
+    codes = (q[..., 0::2] | (q[..., 1::2] << 4)).contiguous()
+    return {"codes": codes, "meta": torch.stack([scale, zero], dim=-1).contiguous()}

@@ -112,6 +112,22 @@ typedef struct mc_layer_kv {
   void* v_pool;
 } mc_layer_kv;
 
+/* One layer's K and V stored in 4 bits (Sec. 5: MiniCache on top of 4-bit KIVI quantisation; the
+ * paper names the scheme only, the layout is ours).  Asymmetric round-to-nearest, groups of 32:
+ * value = code * scale + zero, scale and zero in binary16.  page_size must be 32 (one key group =
+ * the page's tokens).
+ * k_codes, v_codes  [n_pages][n_kv_heads][page_size][64] bytes; channel 2i in the low, 2i+1 in the high nibble of byte i
+ * k_meta            [n_pages][n_kv_heads][128][2] binary16 (scale, zero): keys are quantised per channel,
+ *                   a group = the 32 tokens of the page
+ * v_meta            [n_pages][n_kv_heads][page_size][4][2] binary16: values per token, a group = 32 channels
+ * All four 256-byte aligned. */
+typedef struct mc_layer_q4 {
+  const void* k_codes;
+  const void* k_meta;
+  const void* v_codes;
+  const void* v_meta;
+} mc_layer_q4;
+
 /* The shared cache C^{l,l-1} of one layer pair (Sec. 4.2: [E, R^l, R^{l-1}, |X^{l-1}|, |X^l|, I]).
  *
  * e_k / e_v  [n_pages][n_kv_heads][tile] bytes, tile = page_size * 256 + 2 * page_size * 4 bytes: the
@@ -179,6 +195,14 @@ mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_
 mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1,
                         const mc_layer_kv* l, const mc_pair_cache* out, int32_t do_retention,
                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* mc_merge_pair for layers stored in 4 bits: the rows are de-quantised inside the merge kernel
+ * (code * scale + zero in fp32) and merged exactly as in mc_merge_pair; the pair cache it writes is
+ * the same 16-bit format (cfg->dtype).  The raw rows of retained tokens are the de-quantised values
+ * rounded once to cfg->dtype.  cfg->page_size must be 32. */
+mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc_layer_q4* lm1,
+                           const mc_layer_q4* l, const mc_pair_cache* out, int32_t do_retention,
+                           void* workspace, size_t workspace_bytes, void* stream);
 
 /* Algorithm 2 "MiniCache Decoding", the branch that compresses the step's new token pair:
  * merges k/v_new_lm1 with k/v_new_l ([batch][n_kv_heads][128], 16-bit) by Eq. 3 and writes

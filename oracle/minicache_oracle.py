@@ -207,8 +207,14 @@ def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[
     Returns e_bits [B][S][H][D], e (float64, before storage rounding), n_lm1,
     n_l, d [B][S][H] (float64), ``retained``: dict (b, h) -> ascending indices.
     The retained raw rows are the input bits at those indices."""
-    a = decode_bits(x_lm1_bits, dtype)
-    c = decode_bits(x_l_bits, dtype)
+    return merge_pair_values(decode_bits(x_lm1_bits, dtype), decode_bits(x_l_bits, dtype), seq_lens, dtype, t, gamma,
+                             mode, convention, do_retention)
+
+
+def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dtype: str, t: float, gamma: float,
+                      mode: str = "distinct", convention: str = "eq3", do_retention: bool = True) -> Dict[str, object]:
+    """``merge_pair`` on rows given as float64 values (e.g. de-quantised 4-bit layers); `dtype` is
+    the storage type of the merged direction."""
     m = merge_rows(a, c, t, convention)
     e_bits = store_direction(m["e"], dtype)
     B, S, H, _ = a.shape
@@ -318,6 +324,44 @@ def lse_combine(parts: List):
     w = np.exp(lses - m)
     o = sum(wj * p[0] for wj, p in zip(w, parts)) / np.sum(w)
     return o, m + math.log(np.sum(w))
+
+
+# --------------------------------------------------------------------------
+# 4-bit storage (Sec. 5: MiniCache on top of 4-bit KIVI quantisation)
+# --------------------------------------------------------------------------
+# The paper only names the scheme; the reading taken here is KIVI's asymmetric round-to-nearest
+# quantisation with groups of 32: keys per channel (a group = 32 consecutive tokens of one
+# channel), values per token (a group = 32 consecutive channels of one token):
+#   scale = (max - min) / 15, zero = min, both stored in binary16;
+#   code = clamp(rint((x - zero) / scale), 0, 15) with the *stored* scale and zero;
+#   a constant group stores scale = 1 and code 0.
+Q4_GROUP = 32
+
+
+def q4_quantise(x: np.ndarray, axis: int):
+    """Quantise float64 x along `axis` in groups of 32 (its length must be a multiple of 32).
+
+    Returns (codes uint8, same shape; scale, zero: float64 values that are exactly representable in
+    binary16, shape of x with `axis` divided by 32)."""
+    x = np.moveaxis(np.asarray(x, F64), axis, -1)
+    shp = x.shape
+    assert shp[-1] % Q4_GROUP == 0
+    g = x.reshape(shp[:-1] + (shp[-1] // Q4_GROUP, Q4_GROUP))
+    lo, hi = g.min(-1), g.max(-1)
+    scale = decode_bits(encode_bits((hi - lo) / 15.0, "f16"), "f16")
+    zero = decode_bits(encode_bits(lo, "f16"), "f16")
+    scale = np.where(scale == 0.0, 1.0, scale)
+    codes = np.clip(np.rint((g - zero[..., None]) / scale[..., None]), 0, 15).astype(np.uint8)
+    codes = np.moveaxis(codes.reshape(shp), -1, axis)
+    return codes, np.moveaxis(scale, -1, axis), np.moveaxis(zero, -1, axis)
+
+
+def q4_dequantise(codes: np.ndarray, scale: np.ndarray, zero: np.ndarray, axis: int) -> np.ndarray:
+    """value = code * scale + zero, the group's scale and zero repeated over its 32 members."""
+    c = np.moveaxis(np.asarray(codes, F64), axis, -1)
+    s = np.repeat(np.moveaxis(np.asarray(scale, F64), axis, -1), Q4_GROUP, axis=-1)
+    z = np.repeat(np.moveaxis(np.asarray(zero, F64), axis, -1), Q4_GROUP, axis=-1)
+    return np.moveaxis(c * s + z, -1, axis)
 
 
 # --------------------------------------------------------------------------

@@ -45,6 +45,10 @@ class _LayerKV(C.Structure):
     _fields_ = [("k_pool", C.c_void_p), ("v_pool", C.c_void_p)]
 
 
+class _LayerQ4(C.Structure):
+    _fields_ = [("k_codes", C.c_void_p), ("k_meta", C.c_void_p), ("v_codes", C.c_void_p), ("v_meta", C.c_void_p)]
+
+
 class _PairCache(C.Structure):
     _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("dist", C.c_void_p),
                 ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
@@ -55,7 +59,7 @@ class _PairCache(C.Structure):
 
 EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
-           "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static")
+           "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -200,6 +204,9 @@ class MiniCacheLib:
         L.mc_decode_io_bytes.argtypes = [P(_Config), P(_Batch), C.c_int32, P(C.c_size_t)]
         L.mc_decode_attn_static.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V]
         L.mc_decode_attn_static.restype = C.c_int32
+        L.mc_merge_pair_q4.argtypes = [P(_Config), P(_Batch), P(_LayerQ4), P(_LayerQ4), P(_PairCache), C.c_int32, V,
+                                       C.c_size_t, V]
+        L.mc_merge_pair_q4.restype = C.c_int32
         for f in ("mc_workspace_bytes", "mc_merge_pair", "mc_append_pair", "mc_restore", "mc_decode_attn",
                   "mc_read_status", "mc_merge_pair_host", "mc_decode_attn_host", "mc_decode_io_bytes"):
             getattr(L, f).restype = C.c_int32
@@ -234,6 +241,16 @@ class MiniCacheLib:
         self._check(self._lib.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(l), C.byref(pc),
                                             1 if do_retention else 0, _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_merge_pair_q4(self, cfg: McConfig, batch: Batch, q_lm1, q_l, pair: PairCache, do_retention: bool,
+                         workspace: torch.Tensor, stream=None):
+        """q_lm1 / q_l: dicts with k_codes, k_meta, v_codes, v_meta device tensors (4-bit layers)."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        a = _LayerQ4(_ptr(q_lm1["k_codes"]), _ptr(q_lm1["k_meta"]), _ptr(q_lm1["v_codes"]), _ptr(q_lm1["v_meta"]))
+        l = _LayerQ4(_ptr(q_l["k_codes"]), _ptr(q_l["k_meta"]), _ptr(q_l["v_codes"]), _ptr(q_l["v_meta"]))
+        self._check(self._lib.mc_merge_pair_q4(C.byref(c), C.byref(b), C.byref(a), C.byref(l), C.byref(pc),
+                                               1 if do_retention else 0, _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _stream(stream)))
 
     def mc_append_pair(self, cfg: McConfig, batch: Batch, pair: PairCache, k_new_lm1, v_new_lm1, k_new_l, v_new_l,
                        stream=None):

@@ -120,7 +120,30 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
   if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
   if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
   if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
-  return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, out, do_retention ? 1 : 0, workspace,
+  return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, nullptr, nullptr, out, do_retention ? 1 : 0, workspace,
+                      (cudaStream_t)stream);
+}
+
+mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc_layer_q4* lm1, const mc_layer_q4* l,
+                           const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (cfg->page_size != 32) return MC_ERR_SHAPE;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(out);
+  if (st != MC_OK) return st;
+  if (!lm1 || !l) return MC_ERR_INVALID_ARG;
+  const void* ptrs[8] = {lm1->k_codes, lm1->k_meta, lm1->v_codes, lm1->v_meta, l->k_codes, l->k_meta, l->v_codes, l->v_meta};
+  for (const void* q : ptrs) {
+    if (q == nullptr) return MC_ERR_INVALID_ARG;
+    if (!aligned256(q)) return MC_ERR_ALIGN;
+  }
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
+  if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
+  return launch_merge(cfg, batch, make_geom(cfg, batch), nullptr, nullptr, lm1, l, out, do_retention ? 1 : 0, workspace,
                       (cudaStream_t)stream);
 }
 

@@ -6,8 +6,8 @@ namespace mc {
 
 size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt);
 mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
-                       const mc_layer_kv* l, const mc_pair_cache* out, int do_retention, void* workspace,
-                       cudaStream_t stream);
+                       const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
+                       int do_retention, void* workspace, cudaStream_t stream);
 mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                         const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
                         cudaStream_t stream);

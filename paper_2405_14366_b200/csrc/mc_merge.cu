@@ -18,11 +18,16 @@ constexpr int kMergeWarps = 8;
 constexpr int kMergeThreads = kMergeWarps * 32;
 constexpr int kMergeCtasPerSm = 2;
 constexpr int kMergeMaxBatchSmem = 1024;
+constexpr int kQ4RowBytes = 64;                              // 128 four-bit codes
+constexpr int kQ4CodesBytes = kRowsPerItem * kQ4RowBytes;    // one layer's codes of an item
+constexpr int kQ4MetaBytes = kRowsPerItem * 16;              // one layer's (scale, zero) pairs of an item
 
 struct MergeParams {
   Geom g;
   const char* a_pool[2];  // layer l-1: K, V
   const char* c_pool[2];  // layer l:   K, V
+  const char* a_meta[2];  // 4-bit layers: (scale, zero) pairs; a_pool / c_pool then hold the codes
+  const char* c_meta[2];
   char* e_pool[2];  // compressed tiles (see tile_bytes)
   float* dist;
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
@@ -120,20 +125,8 @@ __device__ __forceinline__ float sum4(float v) {
 // a (layer l-1) and c (layer l), 32 channels each.  Arithmetic in fp32, two channels per
 // instruction (packed f32x2).  Every lane of the quad returns the row's scalars.
 template <int DT>
-__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc,
+__device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const float2 (&c)[16], float ta, float tc,
                                                uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
-  float2 a[16], c[16];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    a[4 * i] = Elem<DT>::unpack(ra[i].x);
-    a[4 * i + 1] = Elem<DT>::unpack(ra[i].y);
-    a[4 * i + 2] = Elem<DT>::unpack(ra[i].z);
-    a[4 * i + 3] = Elem<DT>::unpack(ra[i].w);
-    c[4 * i] = Elem<DT>::unpack(rc[i].x);
-    c[4 * i + 1] = Elem<DT>::unpack(rc[i].y);
-    c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
-    c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
-  }
   float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2, aa3 = aa2, cc3 = aa2;
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
@@ -211,6 +204,45 @@ __device__ __forceinline__ bool merge_item(int i, const MergeParams& p, const in
 // occupancy.  (Eight warps, not nine with a dedicated producer: two CTAs of nine warps do not fit
 // the register file of an SM sub-partition.)
 template <int DT>
+__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc,
+                                               uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
+  float2 a[16], c[16];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[4 * i] = Elem<DT>::unpack(ra[i].x);
+    a[4 * i + 1] = Elem<DT>::unpack(ra[i].y);
+    a[4 * i + 2] = Elem<DT>::unpack(ra[i].z);
+    a[4 * i + 3] = Elem<DT>::unpack(ra[i].w);
+    c[4 * i] = Elem<DT>::unpack(rc[i].x);
+    c[4 * i + 1] = Elem<DT>::unpack(rc[i].y);
+    c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
+    c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
+  }
+  merge_row_core<DT>(a, c, ta, tc, e_out, g_a, g_c, d_out);
+}
+
+// 32 consecutive 4-bit codes (16 bytes; channel 2i in the low nibble of byte i) to values
+// code * scale + zero.  `meta` points at the (scale, zero) binary16 pairs: one pair per channel
+// (keys, per_channel) or a single pair for all 32 (values, one group per token).  The nibble becomes a
+// float through the 2^23 trick on the integer pipe (the integer-to-float conversion unit is slow).
+__device__ __forceinline__ void dequant32(const uint4& codes, const uint32_t* meta, bool per_channel, float2 (&out)[16]) {
+  const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
+  float2 sz = Elem<MC_F16>::unpack(meta[0]);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint32_t two = w[i >> 2] >> (8 * (i & 3));
+    const float c0 = __uint_as_float(0x4B000000u | (two & 15u)) - 8388608.0f;
+    const float c1 = __uint_as_float(0x4B000000u | ((two >> 4) & 15u)) - 8388608.0f;
+    if (per_channel) {
+      const float2 s0 = Elem<MC_F16>::unpack(meta[2 * i]), s1 = Elem<MC_F16>::unpack(meta[2 * i + 1]);
+      out[i] = make_float2(fmaf(c0, s0.x, s0.y), fmaf(c1, s1.x, s1.y));
+    } else {
+      out[i] = make_float2(fmaf(c0, sz.x, sz.y), fmaf(c1, sz.x, sz.y));
+    }
+  }
+}
+
+template <int DT, bool Q4IN>
 __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const MergeParams p) {
   grid_dep_wait();
   grid_dep_launch();
@@ -255,14 +287,28 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     const int s = j % kMergeStages;
     if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, p.status)) return false;
     const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
-    const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
     const uint32_t bar = full0 + 8 * s;
     page_s[s] = page;
-    mbar_expect_tx(bar, 2 * bytes);
-    const size_t off = ((size_t)page * rows_in_page + m.grp * kRowsPerItem) * kRowBytes;
-    bulk_load(stage0 + s * kMergeStageBytes, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + off, bytes, bar);
-    bulk_load(stage0 + s * kMergeStageBytes + kRowsPerItem * kRowBytes, (m.tensor ? p.c_pool[1] : p.c_pool[0]) + off, bytes,
-              bar);
+    const size_t row0 = (size_t)page * rows_in_page + m.grp * kRowsPerItem;
+    if (!Q4IN) {
+      const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
+      mbar_expect_tx(bar, 2 * bytes);
+      bulk_load(stage0 + s * kMergeStageBytes, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + row0 * kRowBytes, bytes, bar);
+      bulk_load(stage0 + s * kMergeStageBytes + kRowsPerItem * kRowBytes,
+                (m.tensor ? p.c_pool[1] : p.c_pool[0]) + row0 * kRowBytes, bytes, bar);
+    } else {
+      // 4-bit layers: 64 bytes of codes per row; (scale, zero) pairs per channel and head (keys, a
+      // group = the page's 32 tokens) or per token and 32 channels (values)
+      const uint32_t cbytes = (uint32_t)rows_item * kQ4RowBytes;
+      const uint32_t mbytes = m.tensor ? (uint32_t)rows_item * 16u : (uint32_t)(rows_item / 32) * 512u;
+      const size_t moff = m.tensor ? row0 * 16 : (row0 / 32) * 512;
+      mbar_expect_tx(bar, 2 * (cbytes + mbytes));
+      const uint32_t sb = stage0 + s * kMergeStageBytes;
+      bulk_load(sb, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + row0 * kQ4RowBytes, cbytes, bar);
+      bulk_load(sb + kQ4CodesBytes, (m.tensor ? p.c_pool[1] : p.c_pool[0]) + row0 * kQ4RowBytes, cbytes, bar);
+      bulk_load(sb + 2 * kQ4CodesBytes, (m.tensor ? p.a_meta[1] : p.a_meta[0]) + moff, mbytes, bar);
+      bulk_load(sb + 2 * kQ4CodesBytes + kQ4MetaBytes, (m.tensor ? p.c_meta[1] : p.c_meta[0]) + moff, mbytes, bar);
+    }
     return true;
   };
 
@@ -307,28 +353,50 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     const int head = row >> p.g.page_shift;
     const int tk = row & (ps - 1);
     const bool valid = row < rows_in_page && m.pslot * ps + tk < n;
-    // lane k owns the 16-byte chunks k, k + 4, k + 8, k + 12; odd rows fetch them in the order that
-    // keeps the two rows of a quarter-warp in different bank groups
-    const unsigned char* sa = stages + s * kMergeStageBytes + quad * kRowBytes;
-    const unsigned char* sc = sa + kRowsPerItem * kRowBytes;
-    uint4 va[4], vc[4];
-    int ci[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      ci[x] = ((x ^ (quad & 1)) << 2) + k;
-      va[x] = *reinterpret_cast<const uint4*>(sa + ci[x] * 16);
-      vc[x] = *reinterpret_cast<const uint4*>(sc + ci[x] * 16);
-    }
-    if (!valid) {
-#pragma unroll
-      for (int x = 0; x < 4; ++x) va[x] = vc[x] = make_uint4(0, 0, 0, 0);  // never computed on: page tail
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
-
     uint4 e[4];
     float g_a, g_c, d;
-    merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
+    int ci[4];
+    if (!Q4IN) {
+      // lane k owns the 16-byte chunks k, k + 4, k + 8, k + 12; odd rows fetch them in the order that
+      // keeps the two rows of a quarter-warp in different bank groups
+      const unsigned char* sa = stages + s * kMergeStageBytes + quad * kRowBytes;
+      const unsigned char* sc = sa + kRowsPerItem * kRowBytes;
+      uint4 va[4], vc[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        ci[x] = ((x ^ (quad & 1)) << 2) + k;
+        va[x] = *reinterpret_cast<const uint4*>(sa + ci[x] * 16);
+        vc[x] = *reinterpret_cast<const uint4*>(sc + ci[x] * 16);
+      }
+      if (!valid) {
+#pragma unroll
+        for (int x = 0; x < 4; ++x) va[x] = vc[x] = make_uint4(0, 0, 0, 0);  // never computed on: page tail
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
+      merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
+    } else {
+      // lane k owns channels [32 k, 32 k + 32): 16 bytes of codes = the 16-byte chunks 4 k .. 4 k + 3 of the output row
+      const unsigned char* sb = stages + s * kMergeStageBytes;
+      const uint4 qa = *reinterpret_cast<const uint4*>(sb + quad * kQ4RowBytes + k * 16);
+      const uint4 qc = *reinterpret_cast<const uint4*>(sb + kQ4CodesBytes + quad * kQ4RowBytes + k * 16);
+      const bool per_channel = m.tensor == 0;
+      const int mo = per_channel ? ((quad >> 5) * 128 + 32 * k) : (quad * 4 + k);  // in (scale, zero) pairs
+      const uint32_t* ma = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes) + mo;
+      const uint32_t* mc = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes + kQ4MetaBytes) + mo;
+      float2 a[16], c[16];
+      dequant32(qa, ma, per_channel, a);
+      dequant32(qc, mc, per_channel, c);
+      if (!valid) {
+#pragma unroll
+        for (int x = 0; x < 16; ++x) a[x] = c[x] = make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x) ci[x] = 4 * k + x;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      merge_row_core<DT>(a, c, p.ta, p.tc, e, g_a, g_c, d);
+    }
     float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
       char* tile = (m.tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + head) * tile_bytes(ps);
@@ -370,6 +438,10 @@ struct RetainParams {
   Geom g;
   const char* a_pool[2];
   const char* c_pool[2];
+  const char* a_meta[2];  // 4-bit layers only
+  const char* c_meta[2];
+  int q4;                 // the layers are 4-bit: raw rows are de-quantised (exactly) into the storage type
+  int dtype;
   char* e_pool[2];
   const float* dist;
   const float* seg_minmax;
@@ -686,9 +758,39 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     const int tok = p.ret_index[out0 + ent];
     const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
     const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
-    const char* src = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kRowBytes + l16 * 16;
     char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
-    *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
+    if (!p.q4) {
+      const char* src = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kRowBytes + l16 * 16;
+      *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
+    } else {
+      // lane l16: channels [8 l16, 8 l16 + 8).  code * scale + zero is formed in double (exact) and
+      // rounded once to the storage type, so the row is the same bits on any machine.
+      const char* codes = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kQ4RowBytes;
+      const char* meta = layer ? p.c_meta[tensor] : p.a_meta[tensor];
+      const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + l16 * 4);
+      const __half2* mp = tensor == 0 ? reinterpret_cast<const __half2*>(meta) + (row / p.g.page_size) * 128 + 8 * l16
+                                      : reinterpret_cast<const __half2*>(meta) + row * 4 + (l16 >> 2);
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        unsigned short hb[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int ch = 2 * j + q;
+          const __half2 sz = tensor == 0 ? mp[ch] : mp[0];
+          const double v = (double)((w >> (4 * ch)) & 15u) * (double)__low2float(sz) + (double)__high2float(sz);
+          if (p.dtype == MC_F16) {
+            const __half hv = __double2half(v);
+            hb[q] = *reinterpret_cast<const unsigned short*>(&hv);
+          } else {
+            const __nv_bfloat16 bv = __double2bfloat16(v);
+            hb[q] = *reinterpret_cast<const unsigned short*>(&bv);
+          }
+        }
+        o[j] = (uint32_t)hb[0] | ((uint32_t)hb[1] << 16);
+      }
+      *reinterpret_cast<uint4*>(dst + l16 * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
     if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok, 0, 0, 0);
   }
 }
@@ -753,8 +855,9 @@ size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
 }
 
 mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
-                       const mc_layer_kv* l, const mc_pair_cache* out, int do_retention, void* workspace,
-                       cudaStream_t stream) {
+                       const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
+                       int do_retention, void* workspace, cudaStream_t stream) {
+  const bool q4 = q_lm1 != nullptr;
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
   MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256), dim3(256), 0, stream, reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status));
   MC_CUDA_CHECK(cudaGetLastError());
@@ -762,10 +865,14 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
 
   MergeParams mp;
   mp.g = g;
-  mp.a_pool[0] = (const char*)lm1->k_pool;
-  mp.a_pool[1] = (const char*)lm1->v_pool;
-  mp.c_pool[0] = (const char*)l->k_pool;
-  mp.c_pool[1] = (const char*)l->v_pool;
+  mp.a_pool[0] = (const char*)(q4 ? q_lm1->k_codes : lm1->k_pool);
+  mp.a_pool[1] = (const char*)(q4 ? q_lm1->v_codes : lm1->v_pool);
+  mp.c_pool[0] = (const char*)(q4 ? q_l->k_codes : l->k_pool);
+  mp.c_pool[1] = (const char*)(q4 ? q_l->v_codes : l->v_pool);
+  mp.a_meta[0] = (const char*)(q4 ? q_lm1->k_meta : nullptr);
+  mp.a_meta[1] = (const char*)(q4 ? q_lm1->v_meta : nullptr);
+  mp.c_meta[0] = (const char*)(q4 ? q_l->k_meta : nullptr);
+  mp.c_meta[1] = (const char*)(q4 ? q_l->v_meta : nullptr);
   mp.e_pool[0] = (char*)out->e_k;
   mp.e_pool[1] = (char*)out->e_v;
   mp.dist = out->dist;
@@ -788,13 +895,11 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
     const int grid = (int)std::min<long long>((long long)n_sm * kMergeCtasPerSm, total);
     const size_t smem = 128 + (size_t)kMergeStages * kMergeStageBytes + (kMergeStages + kMergeMaxBatchSmem + 2) * 4 + 8 +
                         2 * kMergeStages * 8 + 64;
-    if (cfg->dtype == MC_F16) {
-      MC_CUDA_CHECK(cudaFuncSetAttribute(merge_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_F16>, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
-    } else {
-      MC_CUDA_CHECK(cudaFuncSetAttribute(merge_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      MC_CUDA_CHECK(launch_pdl(merge_kernel<MC_BF16>, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
-    }
+    void (*kern)(const MergeParams) =
+        cfg->dtype == MC_F16 ? (q4 ? merge_kernel<MC_F16, true> : merge_kernel<MC_F16, false>)
+                             : (q4 ? merge_kernel<MC_BF16, true> : merge_kernel<MC_BF16, false>);
+    MC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MC_CUDA_CHECK(launch_pdl(kern, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
   }
 
   RetainParams rp;
@@ -803,6 +908,12 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   rp.a_pool[1] = mp.a_pool[1];
   rp.c_pool[0] = mp.c_pool[0];
   rp.c_pool[1] = mp.c_pool[1];
+  rp.a_meta[0] = mp.a_meta[0];
+  rp.a_meta[1] = mp.a_meta[1];
+  rp.c_meta[0] = mp.c_meta[0];
+  rp.c_meta[1] = mp.c_meta[1];
+  rp.q4 = q4 ? 1 : 0;
+  rp.dtype = cfg->dtype;
   rp.e_pool[0] = mp.e_pool[0];
   rp.e_pool[1] = mp.e_pool[1];
   rp.dist = out->dist;

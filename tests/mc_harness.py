@@ -22,7 +22,8 @@ class Problem:
 
     def __init__(self, cfg: WorkloadConfig, pair: int = 0, device="cuda", seq_lens=None, gamma=None, t=None,
                  retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
-                 tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None):
+                 tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None,
+                 q4: bool = False):
         import paper_2405_14366_b200 as mc
         self.mc = mc
         self.lib = mc.lib()
@@ -49,15 +50,44 @@ class Problem:
         self.max_seq_len = int(self.seq_lens_host.max()) if B else 0
         self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode)
         self.pools = {}
+        self.q4 = q4
+        self.q4_pools: Dict[str, Dict[str, torch.Tensor]] = {}
+        self.values: Dict[str, np.ndarray] = {}
         for name, x in self.logical.items():
             xm = x.clone()
             for b in range(B):  # rows past a sequence's length never reach the device pools as data
                 xm[b, self.seq_lens_host[b]:] = 0
-            self.pools[name] = gen.to_paged(xm.to(device), self.block_table, self.ps, n_pages)
+            if not q4:
+                self.pools[name] = gen.to_paged(xm.to(device), self.block_table, self.ps, n_pages)
+                continue
+            # 4-bit layers: quantise the logical rows (data preparation), page codes and meta, and keep
+            # the exact de-quantised values for the oracle
+            assert self.ps == 32 and S % 32 == 0
+            kind = name[0]
+            qd = gen.quantise_q4(xm, kind)
+            codes, meta = qd["codes"], qd["meta"]
+            axis = 1 if kind == "k" else 3
+            cn = codes.numpy()
+            full = np.empty((B, S, self.H, 128), np.uint8)
+            full[..., 0::2], full[..., 1::2] = cn & 15, cn >> 4
+            mt = meta.double().numpy()
+            self.values[name] = orc.q4_dequantise(full, mt[..., 0], mt[..., 1], axis)
+            pc = gen.to_paged(codes.to(device), self.block_table, self.ps, n_pages)
+            if kind == "k":
+                pm = torch.zeros(n_pages, self.H, 128, 2, dtype=torch.float16, device=device)
+                btl = self.block_table[:, :S // 32].long()
+                ok = btl >= 0
+                pm[btl[ok]] = meta.to(device)[ok]
+            else:
+                pm = gen.to_paged(meta.reshape(B, S, self.H, 8).to(device), self.block_table, self.ps, n_pages)
+            self.q4_pools[name] = {"codes": pc, "meta": pm.contiguous()}
         total = int(self.seq_lens_host.sum()) * self.H * 2
         self.ret_capacity = total if ret_capacity is None else ret_capacity
         self.pair = mc.PairCache(self.cfg, B, n_pages, self.ret_capacity, device=device)
-        self.bits = {k: as_bits(v) for k, v in self.logical.items()}
+        if q4:  # the rows the cache can hold: the de-quantised values rounded once to the storage type
+            self.bits = {k: orc.encode_bits(v, self.dtype) for k, v in self.values.items()}
+        else:
+            self.bits = {k: as_bits(v) for k, v in self.logical.items()}
 
     # ------------------------------------------------------------------ device side
     def batch(self, extra: int = 0):
@@ -69,6 +99,12 @@ class Problem:
 
     def run_merge(self, do_retention: bool = True):
         ws = self.workspace(0)
+        if self.q4:
+            lay = lambda sfx: {"k_codes": self.q4_pools["k" + sfx]["codes"], "k_meta": self.q4_pools["k" + sfx]["meta"],
+                               "v_codes": self.q4_pools["v" + sfx]["codes"], "v_meta": self.q4_pools["v" + sfx]["meta"]}
+            self.lib.mc_merge_pair_q4(self.cfg, self.batch(), lay("_lm1"), lay("_l"), self.pair, do_retention, ws)
+            torch.cuda.synchronize()
+            return self.lib.mc_read_status(self.pair, check=False)
         self.lib.mc_merge_pair(self.cfg, self.batch(), self.pools["k_lm1"], self.pools["v_lm1"], self.pools["k_l"],
                                self.pools["v_l"], self.pair, do_retention, ws)
         torch.cuda.synchronize()
@@ -124,6 +160,10 @@ class Problem:
     def oracle_merge(self, mode: str = "distinct", do_retention: bool = True):
         out = {}
         for ti, tn in enumerate(("k", "v")):
+            if self.q4:
+                out[tn] = orc.merge_pair_values(self.values[tn + "_lm1"], self.values[tn + "_l"], self.seq_lens_host,
+                                                self.dtype, self.t, self.gamma, mode=mode, do_retention=do_retention)
+                continue
             out[tn] = orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype,
                                      self.t, self.gamma, mode=mode, do_retention=do_retention)
         return out

@@ -20,7 +20,7 @@ def lib():
 def test_exports_match_header(lib, repo_root):
     text = open(os.path.join(repo_root, "include", "minicache.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    declared = set(re.findall(r"\b(mc_[a-z_]+)\s*\(", text))
+    declared = set(re.findall(r"\b(mc_[a-z0-9_]+)\s*\(", text))
     assert declared, "no declarations found"
     for name in declared:
         assert lib.has_symbol(name), f"{name} declared in minicache.h but not exported"

@@ -222,3 +222,39 @@ def test_scaled_configs_sampled(H, name):
         out, lse = p.run_attn(sel, qq.to(p.device))
         stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample))
     print(name, stats)
+
+
+@pytest.mark.parametrize("q4", [False, True], ids=["f16_inputs", "q4_inputs"])
+def test_serving_mix_ragged(H, q4):
+    """Scaled serving mix: ragged log-normal lengths, pages of 32 tokens; with `q4` the two layers
+    arrive in 4 bits (keys per channel, values per token, groups of 32) and are de-quantised inside
+    the merge; the oracle merges the exact de-quantised values."""
+    wl = CONFIGS["c4_s"]
+    lens, _ = gen.make_lengths(wl)
+    assert len(set(lens.tolist())) > 3 and lens.max() <= wl.seq_len
+    p = H.Problem(wl, pair=wl.n_pairs - 1, seq_lens=lens, q4=q4)
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge()
+    dc = p.device_cache()
+    stats = H.compare_merge(p, om, dc)
+    for layer in (0, 1):
+        dk, dv = p.run_restore(layer)
+        stats.update(H.compare_restore(p, om, dc, layer, dk, dv))
+    q = gen.make_queries(dataclasses.replace(wl, batch=p.B), 0, n_sets=2)
+    rs = np.random.RandomState(11)
+    sample = [(int(b), int(rs.randint(p.Hq))) for b in range(p.B)]
+    for sel in (0, 1, 2):
+        qq = q if sel == 2 else q[sel:sel + 1].contiguous()
+        out, lse = p.run_attn(sel, qq.to(p.device))
+        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample))
+    print("c4_s", "q4" if q4 else "f16", stats)
+
+
+def test_q4_rejects_other_page_sizes(H):
+    wl = CONFIGS["c1"]
+    p = H.Problem(wl)  # page size 16
+    ws = p.workspace(0)
+    dummy = {k: ws for k in ("k_codes", "k_meta", "v_codes", "v_meta")}
+    with pytest.raises(Exception):
+        p.lib.mc_merge_pair_q4(p.cfg, p.batch(), dummy, dummy, p.pair, True, ws)

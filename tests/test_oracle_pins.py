@@ -394,3 +394,58 @@ def test_footprint_near_paper_formula():
     kept = int(0.05 * th * 2 * 8)
     r = orc.footprint_bytes(32, 16, th, 128, kept)["ratio"]
     assert abs(r - 3.1 / 4) < 0.02  # (3.1 h + 2) / 4h of Sec. 4.3, within the slack of its derivation
+
+
+# ---------------------------------------------------------------- 4-bit storage (Sec. 5, KIVI scheme)
+def test_q4_roundtrip_error_bound_and_codes():
+    x = rng.standard_normal((3, 64, 128)) * np.exp(rng.standard_normal((3, 64, 1)))
+    for axis in (1, 2):  # per-channel groups run along tokens (axis 1), per-token groups along channels (axis 2)
+        codes, scale, zero = orc.q4_quantise(x, axis)
+        assert codes.dtype == np.uint8 and codes.min() >= 0 and codes.max() <= 15
+        assert scale.shape[axis] == x.shape[axis] // 32
+        y = orc.q4_dequantise(codes, scale, zero, axis)
+        s_full = np.repeat(scale, 32, axis=axis)
+        rng_full = 15.0 * s_full
+        # half a step, plus what the binary16 rounding of scale (15 steps) and zero can add
+        assert np.all(np.abs(y - x) <= 0.5 * s_full + rng_full * 2.0 ** -10 + 1e-12)
+        # scale and zero are binary16 values
+        assert np.array_equal(orc.decode_bits(orc.encode_bits(scale, "f16"), "f16"), scale)
+        assert np.array_equal(orc.decode_bits(orc.encode_bits(zero, "f16"), "f16"), zero)
+        # both ends of every group are hit (codes 0 and 15 occur) unless the group is constant
+        c = np.moveaxis(codes, axis, -1).reshape(-1, 32)
+        assert np.all(c.min(-1) == 0) and np.all(c.max(-1) >= 14)
+
+
+def test_q4_constant_group_and_brute_force():
+    x = np.full((1, 32, 4), 0.375)
+    codes, scale, zero = orc.q4_quantise(x, 1)
+    assert np.all(codes == 0) and np.all(scale == 1.0) and np.all(zero == 0.375)
+    assert np.array_equal(orc.q4_dequantise(codes, scale, zero, 1), x)
+    # pure-Python restatement on one group
+    g = [float(v) for v in rng.standard_normal(32)]
+    lo, hi = min(g), max(g)
+    s = float(np.float16((hi - lo) / 15.0))
+    z = float(np.float16(lo))
+    want = [min(15, max(0, int(np.rint((v - z) / s)))) for v in g]
+    codes, scale, zero = orc.q4_quantise(np.array(g)[None, :], 1)
+    assert list(codes[0]) == want and scale[0, 0] == s and zero[0, 0] == z
+    assert np.allclose(orc.q4_dequantise(codes, scale, zero, 1)[0], [c * s + z for c in want], atol=0)
+
+
+def test_input_quantiser_matches_oracle_quantiser():
+    """The seeded input generator's 4-bit quantiser (data preparation) and the oracle's produce the
+    same codes, scales and zeros: the device is fed what the oracle de-quantises."""
+    import torch
+    from gen import workload as W
+    g = torch.Generator().manual_seed(3)
+    x = (torch.randn(2, 64, 3, 128, generator=g) * 2).to(torch.float16)
+    xv = x.double().numpy()
+    for kind, axis in (("k", 1), ("v", 3)):
+        q = W.quantise_q4(x, kind)
+        codes, scale, zero = orc.q4_quantise(xv, axis)
+        cn = q["codes"].numpy()
+        full = np.empty(xv.shape, np.uint8)
+        full[..., 0::2], full[..., 1::2] = cn & 15, cn >> 4
+        assert np.array_equal(full, codes)
+        m = q["meta"].double().numpy()
+        assert np.array_equal(m[..., 0], scale) and np.array_equal(m[..., 1], zero)
