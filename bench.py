@@ -95,9 +95,9 @@ class ClockSampler:
 class Job:
     """All device state of one rank's workload."""
 
-    def __init__(self, wl: gen.WorkloadConfig, device):
+    def __init__(self, wl: gen.WorkloadConfig, device, q4: bool = False):
         import paper_2405_14366_b200 as mc
-        self.mc, self.lib, self.wl, self.dev = mc, mc.lib(), wl, device
+        self.mc, self.lib, self.wl, self.dev, self.q4 = mc, mc.lib(), wl, device, q4
         self.B, self.S, self.H, self.Hq, self.ps = wl.batch, wl.seq_len, wl.n_kv_heads, wl.n_q_heads, wl.page_size
         self.steps = wl.decode_steps
         prompt, _ = gen.make_lengths(wl)
@@ -118,7 +118,10 @@ class Job:
                 for b in range(self.B):
                     for v in t.values():
                         v[b, prompt[b]:] = 0
-            self.pools.append({k: gen.to_paged(v, self.block_table, self.ps, self.n_pages) for k, v in t.items()})
+            if q4:
+                self.pools.append(self._q4_layers(t))
+            else:
+                self.pools.append({k: gen.to_paged(v, self.block_table, self.ps, self.n_pages) for k, v in t.items()})
             del t
             self.pairs.append(mc.PairCache(self.cfg, self.B, self.n_pages, cap_rows, device=device))
         dt = self.cfg.torch_dtype
@@ -138,6 +141,27 @@ class Job:
         self.launches = 0
         self.attn_events = []
 
+    def _q4_layers(self, t):
+        """The pair's two layers as 4-bit pools (keys per channel, values per token, groups of 32)."""
+        assert self.ps == 32 and self.S % 32 == 0, "4-bit layers need pages of 32 tokens"
+        npg = self.S // 32
+        btl = self.block_table[:, :npg].long()
+        ok = btl >= 0
+        out = {}
+        for sfx in ("_lm1", "_l"):
+            lay = {}
+            for kind in ("k", "v"):
+                qd = gen.quantise_q4(t[kind + sfx], kind)
+                lay[kind + "_codes"] = gen.to_paged(qd["codes"], self.block_table, self.ps, self.n_pages)
+                if kind == "k":
+                    pm = torch.zeros(self.n_pages, self.H, 128, 2, dtype=torch.float16, device=self.dev)
+                    pm[btl[ok]] = qd["meta"][ok]
+                else:
+                    pm = gen.to_paged(qd["meta"].reshape(self.B, self.S, self.H, 8), self.block_table, self.ps, self.n_pages)
+                lay[kind + "_meta"] = pm.contiguous()
+            out[sfx] = lay
+        return out
+
     def batch(self, decode: bool):
         mx = self.max_prefill + (self.steps + 1 if decode else 0)
         return self.mc.Batch(self.block_table, self.seq_lens, mx, self.n_pages)
@@ -148,6 +172,9 @@ class Job:
         b = self.batch(False)
         for pr in range(self.wl.n_pairs):
             pl = self.pools[pr]
+            if self.q4:
+                self.lib.mc_merge_pair_q4(self.cfg, b, pl["_lm1"], pl["_l"], self.pairs[pr], True, self.ws_merge)
+                continue
             self.lib.mc_merge_pair(self.cfg, b, pl["k_lm1"], pl["v_lm1"], pl["k_l"], pl["v_l"], self.pairs[pr], True,
                                    self.ws_merge)
         self.launches += 4 * self.wl.n_pairs  # init, merge, count(+scan), compact
@@ -212,7 +239,8 @@ class Job:
 
     def bytes_per_step(self, rho: float):
         th, npairs, steps = self.tok_heads, self.wl.n_pairs, self.steps
-        merge = npairs * 2 * th * (3 * ROW + 12 + 4 + rho * (4 * ROW + 4))
+        in_row = 64 + 16 if self.q4 else ROW  # 4-bit codes + the row's share of the group meta
+        merge = npairs * 2 * th * (2 * in_row + ROW + 12 + 4 + rho * (2 * in_row + 2 * ROW + 4))
         restore = npairs * 2 * 2 * th * (2 * ROW + 4 + rho * 2 * ROW)
         # decode: token-heads grow by batch*H per step
         th_steps = steps * th + self.B * self.H * steps * (steps - 1) // 2
@@ -302,6 +330,7 @@ def main():
     ap.add_argument("--page-size", type=int, default=None, help="override the workload's page size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--q4", action="store_true", help="the layers arrive in 4 bits (page size 32; no host-buffer leg)")
     args = ap.parse_args()
     wl = gen.CONFIGS[args.workload]
     if args.decode_steps is not None:
@@ -329,7 +358,9 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    job = Job(wl, dev)
+    job = Job(wl, dev, q4=args.q4)
+    if args.q4:
+        args.no_e2e = True  # the host-buffer entry points take 16-bit layers only
     warm = max(3, args.warmup)
     sampler = None
     for i in range(warm):
@@ -421,7 +452,7 @@ def main():
                 "steps": args.steps, "warmup": warm, "ms_per_step": t_total / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": wl.name, "batch": wl.batch, "seq_len": wl.seq_len, "kv_heads": wl.n_kv_heads,
-                           "q_heads": wl.n_q_heads, "storage": wl.dtype, "page_size": wl.page_size,
+                           "q_heads": wl.n_q_heads, "storage": wl.dtype, "input_layers": "4-bit, de-quantised in the merge" if args.q4 else wl.dtype, "page_size": wl.page_size,
                            "pairs": wl.n_pairs, "decode_steps": wl.decode_steps, "t": wl.t, "gamma": wl.gamma,
                            "retained_fraction": rho, "attention_mode": "single-layer calls (2 per pair per step)",
                            "l2": "inputs larger than L2: every launch streams >= 0.5 GB"},

@@ -425,29 +425,48 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     }
     consumer_sync();
 
-    // ---- split-local softmax: S <- 2^(S - m), row sums; every warp takes a quarter of the columns ----
+    // ---- split-local softmax: S <- 2^(S - m), row sums ----------------------------------------------
+    // A unit of work = (row, part of the columns): one row is cut into four parts (one per warp), two
+    // rows into two parts each, more rows are taken whole (no exchange between warps then).
     {
-      const int c_lo = (n_cols * warp) / kConsumerWarps, c_hi = (n_cols * (warp + 1)) / kConsumerWarps;
-      for (int r = 0; r < rows; ++r) {
+      const int P = rows == 1 ? 4 : (rows == 2 ? 2 : 1);
+      const int units = rows * P;
+      float mloc0 = -INFINITY, mloc1 = -INFINITY;  // a warp has at most two units (eight rows, four warps)
+      for (int u = warp, k = 0; u < units; u += kConsumerWarps, ++k) {
+        const int r = u / P, part = u - r * P;
+        const int c_lo = (n_cols * part) / P, c_hi = (n_cols * (part + 1)) / P;
+        const float* srow = S + r * s_stride;
         float m = -INFINITY;
-        for (int c = c_lo + lane; c < c_hi; c += 32) m = fmaxf(m, S[r * s_stride + c]);
+#pragma unroll 4
+        for (int c = c_lo + lane; c < c_hi; c += 32) m = fmaxf(m, srow[c]);
         for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (lane == 0) red_s[r * kConsumerWarps + warp] = m;
+        if (k == 0) mloc0 = m; else mloc1 = m;
+        if (P > 1 && lane == 0) red_s[r * kConsumerWarps + part] = m;
       }
-      consumer_sync();
-      for (int r = 0; r < rows; ++r) {
-        const float4 mm = *reinterpret_cast<const float4*>(red_s + r * kConsumerWarps);
-        const float m = fmaxf(fmaxf(mm.x, mm.y), fmaxf(mm.z, mm.w));
+      if (P > 1) consumer_sync();
+      for (int u = warp, k = 0; u < units; u += kConsumerWarps, ++k) {
+        const int r = u / P, part = u - r * P;
+        const int c_lo = (n_cols * part) / P, c_hi = (n_cols * (part + 1)) / P;
+        float* srow = S + r * s_stride;
+        float m = k == 0 ? mloc0 : mloc1;
+        if (P > 1) {
+          m = red_s[r * kConsumerWarps];
+          for (int q = 1; q < P; ++q) m = fmaxf(m, red_s[r * kConsumerWarps + q]);
+        }
         float l = 0.f;
+#pragma unroll 4
         for (int c = c_lo + lane; c < c_hi; c += 32) {
-          const float e = exp2f(S[r * s_stride + c] - m);
-          S[r * s_stride + c] = e;
+          const float e = exp2f(srow[c] - m);
+          srow[c] = e;
           l += e;
         }
         for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
         if (lane == 0) {
-          l_s[r * kConsumerWarps + warp] = l;
-          if (warp == 0) m_s[r] = m;
+          l_s[r * kConsumerWarps + part] = l;
+          if (part == 0) {
+            m_s[r] = m;
+            for (int q = P; q < kConsumerWarps; ++q) l_s[r * kConsumerWarps + q] = 0.f;
+          }
         }
       }
       consumer_sync();
@@ -626,29 +645,74 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 }
 
 // Log-sum-exp merge of the split partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
+// One block per output row; eight groups of 32 lanes share the splits (a lane owns four channels),
+// so a row with many splits is a few loads deep, not one load per split.
+constexpr int kCombineThreads = 256;
+constexpr int kCombineGroups = kCombineThreads / 32;
 template <int DT>
-__global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
+__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
   grid_dep_wait();
   grid_dep_launch();
+  __shared__ float red[kCombineGroups];
+  __shared__ float4 acc_s[kCombineGroups][32];
   const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
+  const int tid = threadIdx.x, grp = tid >> 5, lane = tid & 31;
   const int n = p.g.seq_lens[b];
   const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
   const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.n_splits;
+  const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
+  // M = max_j m_j
   float M = -INFINITY;
-  for (int j = 0; j < nsp; ++j) M = fmaxf(M, p.part_ml[(prow0 + j) * 2]);
-  float L = 0.f, o = 0.f;
-  for (int j = 0; j < nsp; ++j) {
-    const float m = p.part_ml[(prow0 + j) * 2];
-    const float w = m == -INFINITY ? 0.f : exp2f(m - M);
-    L = fmaf(w, p.part_ml[(prow0 + j) * 2 + 1], L);
-    o = fmaf(w, p.part_o[(prow0 + j) * kHeadDim + threadIdx.x], o);
+  for (int j = tid; j < nsp; j += kCombineThreads) M = fmaxf(M, ml[j].x);
+  for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  if (lane == 0) red[grp] = M;
+  __syncthreads();
+  M = red[0];
+#pragma unroll
+  for (int g = 1; g < kCombineGroups; ++g) M = fmaxf(M, red[g]);
+  __syncthreads();
+  // L = sum_j w_j l_j
+  float L = 0.f;
+  for (int j = tid; j < nsp; j += kCombineThreads) {
+    const float2 v = ml[j];
+    L = fmaf(v.x == -INFINITY ? 0.f : exp2f(v.x - M), v.y, L);
   }
-  const float res = L > 0.f ? o / L : 0.f;
-  const size_t orow = ((size_t)set * p.g.batch + b) * p.n_q_heads + hq;
-  const uint32_t packed = Elem<DT>::pack(res, 0.f);
-  out[orow * kHeadDim + threadIdx.x] = (unsigned short)(packed & 0xffffu);
-  if (lse != nullptr && threadIdx.x == 0)
-    lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
+  for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+  if (lane == 0) red[grp] = L;
+  // o = sum_j w_j o_j: group grp takes the splits grp, grp + 8, ...
+  float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+  const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
+#pragma unroll 4
+  for (int j = grp; j < nsp; j += kCombineGroups) {
+    const float m = ml[j].x;
+    const float w = m == -INFINITY ? 0.f : exp2f(m - M);
+    const float4 v = po[(size_t)j * (kHeadDim / 4)];
+    o.x = fmaf(w, v.x, o.x);
+    o.y = fmaf(w, v.y, o.y);
+    o.z = fmaf(w, v.z, o.z);
+    o.w = fmaf(w, v.w, o.w);
+  }
+  acc_s[grp][lane] = o;
+  __syncthreads();
+  if (grp == 0) {
+    L = red[0];
+#pragma unroll
+    for (int g = 1; g < kCombineGroups; ++g) {
+      L += red[g];
+      const float4 v = acc_s[g][lane];
+      o.x += v.x;
+      o.y += v.y;
+      o.z += v.z;
+      o.w += v.w;
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const size_t orow = ((size_t)set * p.g.batch + b) * p.n_q_heads + hq;
+    uint2 packed;
+    packed.x = Elem<DT>::pack(o.x * inv, o.y * inv);
+    packed.y = Elem<DT>::pack(o.z * inv, o.w * inv);
+    *reinterpret_cast<uint2*>(out + orow * kHeadDim + lane * 4) = packed;
+    if (lse != nullptr && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
+  }
 }
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -731,12 +795,12 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_F16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_F16>, dim3(cgrid), dim3(128), 0, stream, ap, (unsigned short*)out, lse));
+    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_F16>, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
   } else {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_BF16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_BF16>, dim3(cgrid), dim3(128), 0, stream, ap, (unsigned short*)out, lse));
+    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_BF16>, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
   }
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;

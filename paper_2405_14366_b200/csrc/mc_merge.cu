@@ -332,6 +332,8 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
   }
 
   const int quad = tid >> 2, k = tid & 3;
+  long long run_seg = -1;  // segment of the warp's running distance extremes
+  float run_min = 0.f, run_max = 0.f;
   for (int it = 0; i < total; ++it) {
     if (warp == 0) {
       // item it + 2 goes into the stage that item it - 1 has just left
@@ -416,12 +418,29 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
       dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
     }
-    if (lane == 0 && dmin != __int_as_float(0x7f800000)) {  // the warp's 8 rows belong to one head
-      const size_t seg = ((size_t)m.tensor * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
-      atomicMin(&p.seg_minmax[seg * 2], __float_as_uint(dmin));
-      atomicMax(&p.seg_minmax[seg * 2 + 1], __float_as_uint(dmax));
+    if (dmin != __int_as_float(0x7f800000)) {  // the warp's 8 rows belong to one head
+      // Running extremes stay in registers while the warp's items keep falling into the same segment
+      // (consecutive items of a CTA usually do): all CTAs work on one sequence at a time, and one
+      // atomic pair per warp and item on its few addresses queues up in the memory system.
+      const long long seg = ((long long)m.tensor * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
+      if (seg != run_seg) {
+        if (lane == 0 && run_seg >= 0) {
+          atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));
+          atomicMax(&p.seg_minmax[run_seg * 2 + 1], __float_as_uint(run_max));
+        }
+        run_seg = seg;
+        run_min = dmin;
+        run_max = dmax;
+      } else {
+        run_min = fminf(run_min, dmin);
+        run_max = fmaxf(run_max, dmax);
+      }
     }
     i = next_valid(i + stride, m);
+  }
+  if (lane == 0 && run_seg >= 0) {
+    atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));
+    atomicMax(&p.seg_minmax[run_seg * 2 + 1], __float_as_uint(run_max));
   }
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
