@@ -41,6 +41,7 @@ constexpr int kMaxSplit = 512;
 constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
 constexpr int kCtasPerSm = 2;
+constexpr int kSlabStride = 132;  // floats per row of a warp's partial output in shared memory (4 mod 32: no bank conflicts)
 
 struct AttnParams {
   Geom g;
@@ -95,6 +96,24 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
         : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
   }
 }
+// D(16x8) += A(16x16) * B(16x8), all of A used: the cached rows are the A operand (16 tokens x 16
+// channels for the scores, 16 channels x 16 tokens for the output), the query rows / probabilities
+// the 8-wide B operand, so that every accumulator register holds a wanted number.
+template <int DT>
+__device__ __forceinline__ void mma_rows(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  if (DT == MC_F16) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+}
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
 
 // Shared-memory address of 16-byte chunk `chunk` (0..15) of token row `tk` (0..63) of a stage.
@@ -103,6 +122,13 @@ __device__ __forceinline__ uint32_t tile_addr(uint32_t stage, int tk, int chunk,
   const int j = tk >> page_shift;
   const int r = tk & ((1 << page_shift) - 1);
   return stage + (uint32_t)(j * tbytes + r * kRowBytes + (chunk_pos(r, chunk) << 4));
+}
+
+// Floats of the score buffer S [kMaxRows][split_len + 8]; the same memory later holds the four
+// warps' partial outputs [4][rows][kSlabStride].
+__host__ __device__ __forceinline__ int s_region_floats(int split_len) {
+  const int a = split_len + 8, b = kConsumerWarps * kSlabStride;
+  return kMaxRows * (a > b ? a : b);
 }
 
 // One work item.
@@ -187,7 +213,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
   float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);     // [kMaxRows][s_stride]
-  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kMaxRows * s_stride);  // [2][kMaxRows][64] packed pairs
+  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + s_region_floats(p.split_len));  // [2][kMaxRows][64] packed pairs
   float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
@@ -311,6 +337,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   const int set_row = (nslots == 2 && row < rows) ? row / p.nq : 0;  // which layer this row attends (pair mode)
   const int slot_row = nslots == 2 ? set_row : p.layer_sel;          // which of the tile's two scales it uses
   const int mi = lane >> 3, mr = lane & 7;
+  // the two query rows whose results this thread holds when the rows are the n dimension
+  const int slot0 = nslots == 2 ? min(colp / p.nq, 1) : p.layer_sel;
+  const int slot1 = nslots == 2 ? min((colp + 1) / p.nq, 1) : p.layer_sel;
   int it = 0, n_item = 0;
 
   auto load_q_words = [&](const Item& w, uint32_t (&qw)[4]) {
@@ -359,37 +388,44 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         const int valid = min(kTile, w.n_tok - t * kTile);
         xk = info_s[2 * s + 1];
         if (tk_w < valid) {
-          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-          const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
+          // A = the warp's 16 token rows (k step: 16 channels), B = the query rows: D[token][row]
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};  // even / odd k steps
+          const int tk_m = tk_w + (mi & 1) * 8 + mr;  // token row this lane addresses for ldmatrix
           const uint32_t rowaddr = sbase + (uint32_t)((tk_m >> shift) * tbytes + (tk_m & (ps - 1)) * kRowBytes);
-          const int rsw = tk_m & 7;
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t r0, r1, r2, r3;
-            const int c = ks * 2 + (mi & 1);
-            ldsm_x4(rowaddr + ((uint32_t)((c & 8) | ((c & 7) ^ rsw)) << 4), r0, r1, r2, r3);
-            mma_16816<DT>(acc0, qa0[ks], qa2[ks], r0, r1);
-            mma_16816<DT>(acc1, qa0[ks], qa2[ks], r2, r3);
+          for (int ks = 0; ks < 8; ks += 2) {
+            uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
+            const int c = ks * 2 + (mi >> 1);
+            ldsm_x4(rowaddr + ((uint32_t)((c & 8) | ((c & 7) ^ mr)) << 4), r0, r1, r2, r3);
+            ldsm_x4(rowaddr + ((uint32_t)(((c + 2) & 8) | (((c + 2) & 7) ^ mr)) << 4), r4, r5, r6, r7);
+            mma_rows<DT>(acc0, r0, r1, r2, r3, qa0[ks], qa2[ks]);
+            mma_rows<DT>(acc1, r4, r5, r6, r7, qa0[ks + 1], qa2[ks + 1]);
           }
-          if (row < rows) {
-            const int j = tk_w >> shift, r = tk_w & (ps - 1);
-            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + j * tbytes + ps * kRowBytes) +
-                               slot_row * ps + r;
-            float* srow = S + row * s_stride + t * kTile + tk_w;
-            const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
-            const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
-            *reinterpret_cast<float2*>(srow + colp) =
-                make_float2(acc0[0] * g0.x * p.scale_log2, acc0[1] * g0.y * p.scale_log2);
-            *reinterpret_cast<float2*>(srow + 8 + colp) =
-                make_float2(acc1[0] * g1.x * p.scale_log2, acc1[1] * g1.y * p.scale_log2);
+          // this thread: tokens tk_w + row and + 8, query rows colp and colp + 1
+          if (colp < rows) {
+            const int tk = tk_w + row;
+            const float* sc = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk >> shift) * tbytes + ps * kRowBytes) +
+                              (tk & (ps - 1));
+            const float* sc8 = reinterpret_cast<const float*>(stages + s * kStageBytes + ((tk + 8) >> shift) * tbytes +
+                                                              ps * kRowBytes) + ((tk + 8) & (ps - 1));
+            float* scol = S + t * kTile + tk;
+            const float g0 = sc[slot0 * ps] * p.scale_log2, g8 = sc8[slot0 * ps] * p.scale_log2;
+            scol[colp * s_stride] = (acc0[0] + acc1[0]) * g0;
+            scol[colp * s_stride + 8] = (acc0[2] + acc1[2]) * g8;
+            if (colp + 1 < rows) {
+              const float h0 = sc[slot1 * ps] * p.scale_log2, h8 = sc8[slot1 * ps] * p.scale_log2;
+              scol[(colp + 1) * s_stride] = (acc0[1] + acc1[1]) * h0;
+              scol[(colp + 1) * s_stride + 8] = (acc0[3] + acc1[3]) * h8;
+            }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
       // ---- retained K rows and the new token: their scores replace / add single columns of S.
-      // (A barrier first: the tile that wrote a column may have been handled by another warp.)
-      if (xk > 0) consumer_sync();
+      // (A barrier first: the tile that wrote a column may have been handled by another warp.
+      // Unconditional, so that every warp passes the same barriers whatever it has seen.)
+      consumer_sync();
       for (int x = 0; x < xk && ok; ++x, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
@@ -477,137 +513,106 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     load_q_words(get_item(i + stride, total_items, pre_s, len_s, p), qnext);
 
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
-    float acc[4][4];
+    // A = the warp's 16 token rows transposed (16 channels x 16 tokens per m tile), B = the rows'
+    // probabilities times the V scale: D[channel][row], eight m tiles = all 128 channels.  Every
+    // warp sums its own tokens; the four partial sums meet in shared memory at the end of the item.
+    float acc[8][4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 8; ++a)
 #pragma unroll
       for (int k = 0; k < 4; ++k) acc[a][k] = 0.f;
+    const int tk_w = warp * 16;
+    // chunk position of m tile j for this lane: chunk 2 j + (mi & 1) of a row whose index is mr (mod 8)
+    const uint32_t vsw_lo = (uint32_t)(((mi & 1) ^ (mr & 1)) | (mr & 6));
     if (ok) {
-      const int chunk0 = warp * 4;  // this warp owns channels [32 warp, 32 warp + 32)
       int xv = n_new;
       for (int t = 0; t < w.T; ++t, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const uint32_t sbase = stage0 + s * kStageBytes;
         const int valid = min(kTile, w.n_tok - t * kTile);
-        const int ksteps = (valid + 15) >> 4;
         xv = info_s[2 * s + 1];
         bool wrote = false;
-        if (valid == kTile) {
-          // full tile: all four 16-token steps unrolled, loads first, no masks
-          uint32_t a0[4], a2[4];
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            a0[kk] = a2[kk] = 0u;
-            if (row < rows) {
-              const int tk = kk * 16;
-              const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk >> shift) * tbytes +
-                                                                ps * kRowBytes) + slot_row * ps + (tk & (ps - 1));
-              const float* srow = S + row * s_stride + t * kTile + tk;
-              const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
-              const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
-              const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
-              const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
-              a0[kk] = Elem<DT>::pack(p0.x * g0.x, p0.y * g0.y);
-              a2[kk] = Elem<DT>::pack(p1.x * g1.x, p1.y * g1.y);
+        if (tk_w < valid) {
+          if (valid < tk_w + 16) {
+            // rows past the last cached token may hold anything (page tail, page not copied): zero
+            // them so that 0 * x stays 0 in the contraction
+            for (int i = lane; i < (tk_w + 16 - valid) * 16; i += 32) {
+              const uint32_t a = tile_addr(sbase, valid + (i >> 4), i & 15, shift, tbytes);
+              asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
             }
+            wrote = true;
+            __syncwarp();
           }
-          // token row (kk * 16 + (mi & 1) * 8 + mr): its swizzle term is mr for every kk
-          const uint32_t lane_base = sbase + (uint32_t)(((mi & 1) * 8 + mr) * kRowBytes);
-          const uint32_t pos0 = (uint32_t)chunk_pos(mr, chunk0 + (mi >> 1)) << 4;
-          const uint32_t pos1 = (uint32_t)chunk_pos(mr, chunk0 + 2 + (mi >> 1)) << 4;
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const int tk = kk * 16;
-            const uint32_t rowa = lane_base + (uint32_t)((tk >> shift) * tbytes + (tk & (ps - 1)) * kRowBytes);
-            uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
-            ldsm_x4_t(rowa + pos0, r0, r1, r2, r3);
-            ldsm_x4_t(rowa + pos1, r4, r5, r6, r7);
-            mma_16816<DT>(acc[0], a0[kk], a2[kk], r0, r1);
-            mma_16816<DT>(acc[1], a0[kk], a2[kk], r2, r3);
-            mma_16816<DT>(acc[2], a0[kk], a2[kk], r4, r5);
-            mma_16816<DT>(acc[3], a0[kk], a2[kk], r6, r7);
-          }
-        } else {
-        // rows past the last cached token may hold anything (page tail, page not copied): zero this
-        // warp's channels there so that 0 * x stays 0 in the contraction
-        for (int rz = valid + (lane >> 2); rz < ksteps * 16; rz += 8) {
-          const uint32_t a = tile_addr(sbase, rz, chunk0 + (lane & 3), shift, tbytes);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
-          wrote = true;
-        }
-        __syncwarp();
-        for (int kk = 0; kk < ksteps; ++kk) {
-          // A fragment: probabilities times the V scale, rounded to the storage type
-          uint32_t a0 = 0u, a2 = 0u;
+          // B fragment: row `row`, tokens tk_w + colp, + 1, + 8, + 9
+          uint32_t b0 = 0u, b1 = 0u;
           if (row < rows) {
-            const int tk = kk * 16;
-            const int j = tk >> shift, r = tk & (ps - 1);
-            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + j * tbytes + ps * kRowBytes) +
-                               slot_row * ps + r;
-            const float* srow = S + row * s_stride + t * kTile + tk;
+            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk_w >> shift) * tbytes +
+                                                              ps * kRowBytes) + slot_row * ps + (tk_w & (ps - 1));
+            const float* srow = S + row * s_stride + t * kTile + tk_w;
             const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
             const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
             const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
             const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
-            const int c0 = tk + colp;
-            a0 = Elem<DT>::pack(c0 < valid ? p0.x * g0.x : 0.f, c0 + 1 < valid ? p0.y * g0.y : 0.f);
-            a2 = Elem<DT>::pack(c0 + 8 < valid ? p1.x * g1.x : 0.f, c0 + 9 < valid ? p1.y * g1.y : 0.f);
+            const int c0 = tk_w + colp;
+            b0 = Elem<DT>::pack(c0 < valid ? p0.x * g0.x : 0.f, c0 + 1 < valid ? p0.y * g0.y : 0.f);
+            b1 = Elem<DT>::pack(c0 + 8 < valid ? p1.x * g1.x : 0.f, c0 + 9 < valid ? p1.y * g1.y : 0.f);
           }
-          const int tk_m = kk * 16 + (mi & 1) * 8 + mr;
+          const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
+          const uint32_t rowaddr = sbase + (uint32_t)((tk_m >> shift) * tbytes + (tk_m & (ps - 1)) * kRowBytes);
 #pragma unroll
-          for (int np = 0; np < 2; ++np) {
-            uint32_t r0, r1, r2, r3;
-            ldsm_x4_t(tile_addr(sbase, tk_m, chunk0 + np * 2 + (mi >> 1), shift, tbytes), r0, r1, r2, r3);
-            mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
-            mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
+          for (int j = 0; j < 8; ++j) {
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4_t(rowaddr + (((uint32_t)((j >> 2) << 3) | ((uint32_t)(2 * (j & 3)) ^ vsw_lo)) << 4), a0, a1, a2, a3);
+            mma_rows<DT>(acc[j], a0, a1, a2, a3, b0, b1);
           }
-        }
         }
         if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
-      // ---- retained V rows and the new token: raw rows weighted by their tokens' probabilities
+      // ---- retained V rows and the new token: raw rows weighted by their tokens' probabilities.
+      // Single layer: warp w takes entries 16 w .. 16 w + 15; pair mode (16 entries per layer):
+      // warp 0 layer l-1, warp 2 layer l.
       for (int x = 0; x < xv && ok; ++x, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const int cnt = info_s[2 * s];
-        const int ksteps = (cnt + 15) >> 4;
+        const int set = nslots == 2 ? (warp >> 1) : 0;
+        const int e_w = nslots == 2 ? (warp & 1) * 16 : warp * 16;
         bool wrote = false;
-        for (int set = 0; set < nslots; ++set) {
+        if (e_w < cnt) {
           const unsigned char* sb = stages + s * kStageBytes + set * set_bytes;
           const uint32_t sba = smem_u32(sb);
-          for (int rz = cnt + (lane >> 2); rz < ksteps * 16; rz += 8) {  // entries past the last one: zero our channels
-            const uint32_t a = sba + (uint32_t)(rz * kEntryBytes + ((chunk0 + (lane & 3)) << 4));
-            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+          if (cnt < e_w + 16) {  // entries past the last one: zero
+            for (int i = lane; i < (e_w + 16 - cnt) * 16; i += 32) {
+              const uint32_t a = sba + (uint32_t)((cnt + (i >> 4)) * kEntryBytes + ((i & 15) << 4));
+              asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+            }
             wrote = true;
+            __syncwarp();
           }
-          __syncwarp();
-          for (int kk = 0; kk < ksteps; ++kk) {
-            uint32_t a0 = 0u, a2 = 0u;
-            if (row < rows && set_row == set) {
-              float pv[4];
+          uint32_t b0 = 0u, b1 = 0u;
+          if (row < rows && set_row == set) {
+            float pv[4];
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const int e = kk * 16 + colp + (k & 1) + (k >> 1) * 8;
-                pv[k] = 0.f;
-                if (e < cnt) {
-                  const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
-                  pv[k] = S[row * s_stride + col];
-                }
+            for (int k = 0; k < 4; ++k) {
+              const int e = e_w + colp + (k & 1) + (k >> 1) * 8;
+              pv[k] = 0.f;
+              if (e < cnt) {
+                const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
+                pv[k] = S[row * s_stride + col];
               }
-              a0 = Elem<DT>::pack(pv[0], pv[1]);
-              a2 = Elem<DT>::pack(pv[2], pv[3]);
             }
-            const int e_m = kk * 16 + (mi & 1) * 8 + mr;
+            b0 = Elem<DT>::pack(pv[0], pv[1]);
+            b1 = Elem<DT>::pack(pv[2], pv[3]);
+          }
+          const uint32_t rowaddr = sba + (uint32_t)((e_w + (mi >> 1) * 8 + mr) * kEntryBytes + ((mi & 1) << 4));
 #pragma unroll
-            for (int np = 0; np < 2; ++np) {
-              uint32_t r0, r1, r2, r3;
-              ldsm_x4_t(sba + (uint32_t)(e_m * kEntryBytes + ((chunk0 + np * 2 + (mi >> 1)) << 4)), r0, r1, r2, r3);
-              mma_16816<DT>(acc[np * 2], a0, a2, r0, r1);
-              mma_16816<DT>(acc[np * 2 + 1], a0, a2, r2, r3);
-            }
+          for (int j = 0; j < 8; ++j) {
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4_t(rowaddr + (uint32_t)(j << 5), a0, a1, a2, a3);
+            mma_rows<DT>(acc[j], a0, a1, a2, a3, b0, b1);
           }
         }
         if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -616,16 +621,35 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       }
     }
 
-    // ---- partial results of this split ---------------------------------------------------------------
-    if (row < rows) {
-      const int rq = row - set_row * p.nq;
-      const size_t prow = (((size_t)set_row * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
-      float* dst = p.part_o + prow * kHeadDim + warp * 32 + colp;
+    // ---- partial results of this split: the four warps' sums meet in shared memory (the score
+    // buffer, free once every warp has left the V phase) ---------------------------------------------
+    consumer_sync();
+    {
+      float* slab = S + warp * rows * kSlabStride;  // [rows][kSlabStride]
 #pragma unroll
-      for (int nt = 0; nt < 4; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(acc[nt][0], acc[nt][1]);
-      if (warp == 0 && (lane & 3) == 0) {
-        const float4 ll = *reinterpret_cast<const float4*>(l_s + row * kConsumerWarps);
-        p.part_ml[prow * 2] = m_s[row];
+      for (int j = 0; j < 8; ++j) {
+        const int ch = j * 16 + row;
+        if (colp < rows) {
+          slab[colp * kSlabStride + ch] = acc[j][0];
+          slab[colp * kSlabStride + ch + 8] = acc[j][2];
+        }
+        if (colp + 1 < rows) {
+          slab[(colp + 1) * kSlabStride + ch] = acc[j][1];
+          slab[(colp + 1) * kSlabStride + ch + 8] = acc[j][3];
+        }
+      }
+    }
+    consumer_sync();
+    for (int r = 0; r < rows; ++r) {
+      const int set_r = nslots == 2 ? r / p.nq : 0;
+      const int rq = r - set_r * p.nq;
+      const size_t prow = (((size_t)set_r * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
+      const float* sl = S + r * kSlabStride + tid;
+      const int ws = rows * kSlabStride;
+      p.part_o[prow * kHeadDim + tid] = (sl[0] + sl[ws]) + (sl[2 * ws] + sl[3 * ws]);
+      if (tid == 0) {
+        const float4 ll = *reinterpret_cast<const float4*>(l_s + r * kConsumerWarps);
+        p.part_ml[prow * 2] = m_s[r];
         p.part_ml[prow * 2 + 1] = (ll.x + ll.y) + (ll.z + ll.w);
       }
     }
@@ -735,7 +759,7 @@ static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
 }
 
 static size_t attn_smem_bytes(int split_len) {
-  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kMaxRows * (split_len + 8) * 4;  // stages, S
+  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)s_region_floats(split_len) * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                                // q_s
   b += kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;                                     // m, l, red
   b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + 2 * kStages * 8 + 64;
