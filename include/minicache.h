@@ -138,7 +138,8 @@ typedef struct mc_layer_q4 {
  *            (c & 8) | ((c & 7) ^ (r & 7)), the order the attention kernel wants in shared memory.
  *            A scale is |x| / |e_stored|, the magnitude of Eq. 2 already divided by the length of
  *            the rounded direction, so that restore is one multiply: x_hat = e_stored * scale.
- *            The scales of a retained token are zero (its rows are kept raw in ret_rows).
+ *            The scales of a retained token are -0.0f (its rows are kept raw in ret_rows): a zero,
+ *            so that the shared direction contributes nothing for it, whose sign marks the token.
  * dist       [n_pages][n_kv_heads][2][page_size] fp32 angular distance d = Omega / pi; slot 0: K, 1: V.
  * Retention, per segment seg = (tensor * batch + b) * n_kv_heads + head (tensor 0 = K, 1 = V):
  * ret_count  [2 * batch * n_kv_heads] retained tokens of the segment

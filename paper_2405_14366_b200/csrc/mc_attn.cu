@@ -18,9 +18,11 @@
 //     while the copy engine saturates the memory system, so nothing irregular is left on any
 //     critical path);
 //   - four consumer warps run every contraction on the tensor cores, the query rows of the kv
-//     head's group (and of both layers in pair mode) being the padded M tile: scores x K scale
-//     -> shared memory, scores of retained rows scattered over them -> split-local softmax ->
-//     (P x V scale) V, plus gathered P times the retained V rows.
+//     head's group (and of both layers in pair mode) being the 8-wide N tile and the cached rows
+//     the M tile: scores x K scale -> shared memory (the scores of retained rows, from their raw
+//     rows, fill the columns the tiles leave out), row maxima tracked on the way -> V phase: each
+//     warp takes 16 tokens of every tile, P = 2^(score - max) x V scale formed where it is used,
+//     plus gathered P times the retained V rows; the warps' partial sums meet in shared memory.
 // Partial (m, l, o) per split are merged by attn_combine_kernel.  Every wait is bounded.
 #include <algorithm>
 
@@ -131,6 +133,11 @@ __host__ __device__ __forceinline__ int s_region_floats(int split_len) {
   return kMaxRows * (a > b ? a : b);
 }
 
+// The merge marks a retained token by the scale -0: the shared direction then contributes nothing
+// wherever scales are applied blindly, and a token whose rows are genuinely zero (scale +0, score 0)
+// stays distinguishable.
+__device__ __forceinline__ bool is_retained_scale(float g) { return __float_as_uint(g) == 0x80000000u; }
+
 // One work item.
 struct Item {
   int b, g, split;
@@ -217,7 +224,8 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
-  int* info_s = reinterpret_cast<int*>(red_s + kMaxRows * kConsumerWarps);  // [kStages][2]: entries, extra stages of the phase
+  float* red2_s = red_s + kMaxRows * kConsumerWarps;                     // [kMaxRows][kConsumerWarps]
+  int* info_s = reinterpret_cast<int*>(red2_s + kMaxRows * kConsumerWarps);  // [kStages][2]: entries, extra stages of the phase
   int* pre_s = info_s + 2 * kStages;                                     // [batch + 1] split-count prefix
   int* len_s = pre_s + kMaxBatchSmem + 1;                                // [batch] sequence lengths
   volatile int* s_abort = len_s + kMaxBatchSmem;
@@ -368,9 +376,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     const Item w = get_item(i, total_items, pre_s, len_s, p);
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
     const int n_new = w.has_new ? 1 : 0;
-    const int n_cols = w.n_tok + n_new;
     bool ok = true;
 
+    float mx0 = -INFINITY, mx1 = -INFINITY, mxe = -INFINITY;  // running maxima of the scores this thread stores
     // ---- K phase: S[r][i] = log2e * sm_scale * g_i * (q_r . e_i) ---------------------------------
     {
       uint32_t qa0[8], qa2[8];
@@ -392,16 +400,20 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};  // even / odd k steps
           const int tk_m = tk_w + (mi & 1) * 8 + mr;  // token row this lane addresses for ldmatrix
           const uint32_t rowaddr = sbase + (uint32_t)((tk_m >> shift) * tbytes + (tk_m & (ps - 1)) * kRowBytes);
+          // all eight loads first, then the contractions: the loads' latencies overlap
+          uint32_t ra[8][4];
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const int c = ks * 2 + (mi >> 1);
+            ldsm_x4(rowaddr + ((uint32_t)((c & 8) | ((c & 7) ^ mr)) << 4), ra[ks][0], ra[ks][1], ra[ks][2], ra[ks][3]);
+          }
 #pragma unroll
           for (int ks = 0; ks < 8; ks += 2) {
-            uint32_t r0, r1, r2, r3, r4, r5, r6, r7;
-            const int c = ks * 2 + (mi >> 1);
-            ldsm_x4(rowaddr + ((uint32_t)((c & 8) | ((c & 7) ^ mr)) << 4), r0, r1, r2, r3);
-            ldsm_x4(rowaddr + ((uint32_t)(((c + 2) & 8) | (((c + 2) & 7) ^ mr)) << 4), r4, r5, r6, r7);
-            mma_rows<DT>(acc0, r0, r1, r2, r3, qa0[ks], qa2[ks]);
-            mma_rows<DT>(acc1, r4, r5, r6, r7, qa0[ks + 1], qa2[ks + 1]);
+            mma_rows<DT>(acc0, ra[ks][0], ra[ks][1], ra[ks][2], ra[ks][3], qa0[ks], qa2[ks]);
+            mma_rows<DT>(acc1, ra[ks + 1][0], ra[ks + 1][1], ra[ks + 1][2], ra[ks + 1][3], qa0[ks + 1], qa2[ks + 1]);
           }
-          // this thread: tokens tk_w + row and + 8, query rows colp and colp + 1
+          // this thread: tokens tk_w + row and + 8, query rows colp and colp + 1.  A retained token
+          // (scale = -0) gets its score from its raw row further down; past the last token nothing is stored.
           if (colp < rows) {
             const int tk = tk_w + row;
             const float* sc = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk >> shift) * tbytes + ps * kRowBytes) +
@@ -409,23 +421,35 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             const float* sc8 = reinterpret_cast<const float*>(stages + s * kStageBytes + ((tk + 8) >> shift) * tbytes +
                                                               ps * kRowBytes) + ((tk + 8) & (ps - 1));
             float* scol = S + t * kTile + tk;
-            const float g0 = sc[slot0 * ps] * p.scale_log2, g8 = sc8[slot0 * ps] * p.scale_log2;
-            scol[colp * s_stride] = (acc0[0] + acc1[0]) * g0;
-            scol[colp * s_stride + 8] = (acc0[2] + acc1[2]) * g8;
+            const float g0 = sc[slot0 * ps], g8 = sc8[slot0 * ps];
+            const bool u0 = tk < valid && !is_retained_scale(g0), u8 = tk + 8 < valid && !is_retained_scale(g8);
+            const float s00 = (acc0[0] + acc1[0]) * (g0 * p.scale_log2), s08 = (acc0[2] + acc1[2]) * (g8 * p.scale_log2);
+            if (u0) {
+              scol[colp * s_stride] = s00;
+              mx0 = fmaxf(mx0, s00);
+            }
+            if (u8) {
+              scol[colp * s_stride + 8] = s08;
+              mx0 = fmaxf(mx0, s08);
+            }
             if (colp + 1 < rows) {
-              const float h0 = sc[slot1 * ps] * p.scale_log2, h8 = sc8[slot1 * ps] * p.scale_log2;
-              scol[(colp + 1) * s_stride] = (acc0[1] + acc1[1]) * h0;
-              scol[(colp + 1) * s_stride + 8] = (acc0[3] + acc1[3]) * h8;
+              const float h0 = sc[slot1 * ps], h8 = sc8[slot1 * ps];
+              const float s10 = (acc0[1] + acc1[1]) * (h0 * p.scale_log2), s18 = (acc0[3] + acc1[3]) * (h8 * p.scale_log2);
+              if (tk < valid && !is_retained_scale(h0)) {
+                scol[(colp + 1) * s_stride] = s10;
+                mx1 = fmaxf(mx1, s10);
+              }
+              if (tk + 8 < valid && !is_retained_scale(h8)) {
+                scol[(colp + 1) * s_stride + 8] = s18;
+                mx1 = fmaxf(mx1, s18);
+              }
             }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
-      // ---- retained K rows and the new token: their scores replace / add single columns of S.
-      // (A barrier first: the tile that wrote a column may have been handled by another warp.
-      // Unconditional, so that every warp passes the same barriers whatever it has seen.)
-      consumer_sync();
+      // ---- retained K rows and the new token: their scores fill the columns the tiles left out.
       for (int x = 0; x < xk && ok; ++x, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
@@ -450,7 +474,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               const int e = e_w + colp + k;
               if (e < cnt) {
                 const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
-                S[row * s_stride + col] = acc0[k] * p.scale_log2;
+                const float sc = acc0[k] * p.scale_log2;
+                S[row * s_stride + col] = sc;
+                mxe = fmaxf(mxe, sc);
               }
             }
           }
@@ -459,54 +485,29 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
     }
-    consumer_sync();
-
-    // ---- split-local softmax: S <- 2^(S - m), row sums ----------------------------------------------
-    // A unit of work = (row, part of the columns): one row is cut into four parts (one per warp), two
-    // rows into two parts each, more rows are taken whole (no exchange between warps then).
-    {
-      const int P = rows == 1 ? 4 : (rows == 2 ? 2 : 1);
-      const int units = rows * P;
-      float mloc0 = -INFINITY, mloc1 = -INFINITY;  // a warp has at most two units (eight rows, four warps)
-      for (int u = warp, k = 0; u < units; u += kConsumerWarps, ++k) {
-        const int r = u / P, part = u - r * P;
-        const int c_lo = (n_cols * part) / P, c_hi = (n_cols * (part + 1)) / P;
-        const float* srow = S + r * s_stride;
-        float m = -INFINITY;
-#pragma unroll 4
-        for (int c = c_lo + lane; c < c_hi; c += 32) m = fmaxf(m, srow[c]);
-        for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (k == 0) mloc0 = m; else mloc1 = m;
-        if (P > 1 && lane == 0) red_s[r * kConsumerWarps + part] = m;
-      }
-      if (P > 1) consumer_sync();
-      for (int u = warp, k = 0; u < units; u += kConsumerWarps, ++k) {
-        const int r = u / P, part = u - r * P;
-        const int c_lo = (n_cols * part) / P, c_hi = (n_cols * (part + 1)) / P;
-        float* srow = S + r * s_stride;
-        float m = k == 0 ? mloc0 : mloc1;
-        if (P > 1) {
-          m = red_s[r * kConsumerWarps];
-          for (int q = 1; q < P; ++q) m = fmaxf(m, red_s[r * kConsumerWarps + q]);
-        }
-        float l = 0.f;
-#pragma unroll 4
-        for (int c = c_lo + lane; c < c_hi; c += 32) {
-          const float e = exp2f(srow[c] - m);
-          srow[c] = e;
-          l += e;
-        }
-        for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-        if (lane == 0) {
-          l_s[r * kConsumerWarps + part] = l;
-          if (part == 0) {
-            m_s[r] = m;
-            for (int q = P; q < kConsumerWarps; ++q) l_s[r * kConsumerWarps + q] = 0.f;
-          }
-        }
-      }
-      consumer_sync();
+    // ---- row maxima: every thread has tracked the scores it stored; the exponentials are taken
+    // where the probabilities are used (V phase), so the scores are not passed over again ----------
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
     }
+    mxe = fmaxf(mxe, __shfl_xor_sync(0xffffffffu, mxe, 1));
+    mxe = fmaxf(mxe, __shfl_xor_sync(0xffffffffu, mxe, 2));
+    if (lane < 4) {
+      red_s[colp * kConsumerWarps + warp] = mx0;        // rows colp, colp + 1 (tiles)
+      red_s[(colp + 1) * kConsumerWarps + warp] = mx1;
+    }
+    if ((lane & 3) == 0) red2_s[row * kConsumerWarps + warp] = mxe;  // row `row` (raw rows)
+    consumer_sync();
+    float m_row;
+    {
+      const float4 ma = *reinterpret_cast<const float4*>(red_s + row * kConsumerWarps);
+      const float4 mb = *reinterpret_cast<const float4*>(red2_s + row * kConsumerWarps);
+      m_row = fmaxf(fmaxf(fmaxf(ma.x, ma.y), fmaxf(ma.z, ma.w)), fmaxf(fmaxf(mb.x, mb.y), fmaxf(mb.z, mb.w)));
+      if (warp == 0 && (lane & 3) == 0) m_s[row] = m_row;
+    }
+    float l_acc = 0.f;  // sum of this thread's probabilities of row `row`
 
     // query rows of the next item travel while the V tiles stream
     uint32_t qnext[4];
@@ -555,17 +556,21 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
             const float2 g1 = *reinterpret_cast<const float2*>(scj + 8 + colp);
             const int c0 = tk_w + colp;
-            b0 = Elem<DT>::pack(c0 < valid ? p0.x * g0.x : 0.f, c0 + 1 < valid ? p0.y * g0.y : 0.f);
-            b1 = Elem<DT>::pack(c0 + 8 < valid ? p1.x * g1.x : 0.f, c0 + 9 < valid ? p1.y * g1.y : 0.f);
+            const float e0 = c0 < valid ? exp2f(p0.x - m_row) : 0.f, e1 = c0 + 1 < valid ? exp2f(p0.y - m_row) : 0.f;
+            const float e2 = c0 + 8 < valid ? exp2f(p1.x - m_row) : 0.f, e3 = c0 + 9 < valid ? exp2f(p1.y - m_row) : 0.f;
+            l_acc += (e0 + e1) + (e2 + e3);
+            b0 = Elem<DT>::pack(e0 * g0.x, e1 * g0.y);
+            b1 = Elem<DT>::pack(e2 * g1.x, e3 * g1.y);
           }
           const int tk_m = tk_w + (mi >> 1) * 8 + mr;  // token row this lane addresses for ldmatrix
           const uint32_t rowaddr = sbase + (uint32_t)((tk_m >> shift) * tbytes + (tk_m & (ps - 1)) * kRowBytes);
+          uint32_t ra[8][4];  // all eight loads first, then the contractions
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            uint32_t a0, a1, a2, a3;
-            ldsm_x4_t(rowaddr + (((uint32_t)((j >> 2) << 3) | ((uint32_t)(2 * (j & 3)) ^ vsw_lo)) << 4), a0, a1, a2, a3);
-            mma_rows<DT>(acc[j], a0, a1, a2, a3, b0, b1);
-          }
+          for (int j = 0; j < 8; ++j)
+            ldsm_x4_t(rowaddr + (((uint32_t)((j >> 2) << 3) | ((uint32_t)(2 * (j & 3)) ^ vsw_lo)) << 4), ra[j][0], ra[j][1],
+                      ra[j][2], ra[j][3]);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) mma_rows<DT>(acc[j], ra[j][0], ra[j][1], ra[j][2], ra[j][3], b0, b1);
         }
         if (__any_sync(0xffffffffu, wrote)) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -601,7 +606,8 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               pv[k] = 0.f;
               if (e < cnt) {
                 const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
-                pv[k] = S[row * s_stride + col];
+                pv[k] = exp2f(S[row * s_stride + col] - m_row);
+                if (col >= w.n_tok) l_acc += pv[k];  // the new token: no tile has counted it
               }
             }
             b0 = Elem<DT>::pack(pv[0], pv[1]);
@@ -623,6 +629,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
     // ---- partial results of this split: the four warps' sums meet in shared memory (the score
     // buffer, free once every warp has left the V phase) ---------------------------------------------
+    l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
+    l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
+    if ((lane & 3) == 0) l_s[row * kConsumerWarps + warp] = l_acc;
     consumer_sync();
     {
       float* slab = S + warp * rows * kSlabStride;  // [rows][kSlabStride]
@@ -761,7 +770,7 @@ static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
 static size_t attn_smem_bytes(int split_len) {
   size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)s_region_floats(split_len) * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                                // q_s
-  b += kMaxRows * 4 + 2 * kMaxRows * kConsumerWarps * 4;                                     // m, l, red
+  b += kMaxRows * 4 + 3 * kMaxRows * kConsumerWarps * 4;                                     // m, l, red, red2
   b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + 2 * kStages * 8 + 64;
   return b;
 }

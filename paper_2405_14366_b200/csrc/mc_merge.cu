@@ -762,10 +762,11 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
     for (int j = 0; j < 4; ++j) {
       if (m & (1u << j)) {
         p.ret_index[pos++] = tok0 + j;
-        // a retained token is served from its raw rows: its scales are never read again, and zero
-        // makes the shared direction contribute nothing for it wherever scales are applied blindly
-        sc[j] = 0.f;
-        sc[p.g.page_size + j] = 0.f;
+        // a retained token is served from its raw rows: the scale -0 makes the shared direction
+        // contribute nothing for it wherever scales are applied blindly, and tells the attention
+        // kernel that the token's score comes from its raw key row
+        sc[j] = -0.f;
+        sc[p.g.page_size + j] = -0.f;
       }
     }
   }
