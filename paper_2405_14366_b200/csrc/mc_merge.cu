@@ -138,18 +138,21 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
   const float aa = sum4((aa2.x + aa2.y) + (aa3.x + aa3.y)), cc = sum4((cc2.x + cc2.y) + (cc3.x + cc3.y));
   const float ia = aa > 0.f ? rsqrtf(aa) : 0.f;
   const float ic = cc > 0.f ? rsqrtf(cc) : 0.f;
-  // |u - v|^2 formed channel by channel (no cancellation at small angles); |u + v|^2 = 4 - |u - v|^2
-  // is as good until the two directions come close to opposite, where it is formed the same way
-  const float2 ia2 = make_float2(ia, ia), nic2 = make_float2(-ic, -ic);
+  // |u - v|^2 = |a - (|a| / |c|) c|^2 / |a|^2, formed channel by channel (no cancellation at small
+  // angles); |u + v|^2 = 4 - |u - v|^2 is as good until the two directions come close to opposite,
+  // where it is formed the same way
+  const float ia_sq = ia * ia;
+  const float nr = -(aa * ia) * ic;  // -|a| / |c|
+  const float2 ia2 = make_float2(ia, ia), nr2 = make_float2(nr, nr);
   float2 sm2 = make_float2(0.f, 0.f), sm3 = sm2;
 #pragma unroll
   for (int i = 0; i < 16; i += 2) {
-    const float2 dm = __ffma2_rn(c[i], nic2, __fmul2_rn(a[i], ia2));
-    const float2 dn = __ffma2_rn(c[i + 1], nic2, __fmul2_rn(a[i + 1], ia2));
+    const float2 dm = __ffma2_rn(c[i], nr2, a[i]);
+    const float2 dn = __ffma2_rn(c[i + 1], nr2, a[i + 1]);
     sm2 = __ffma2_rn(dm, dm, sm2);
     sm3 = __ffma2_rn(dn, dn, sm3);
   }
-  const float sm = sum4((sm2.x + sm2.y) + (sm3.x + sm3.y));
+  const float sm = sum4((sm2.x + sm2.y) + (sm3.x + sm3.y)) * ia_sq;
   float sp = 4.0f - sm;
   if (__any_sync(0xffffffffu, sm > 3.5f)) {
     const float2 ic2 = make_float2(ic, ic);
