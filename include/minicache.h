@@ -47,7 +47,8 @@ extern "C" {
 typedef enum {
   MC_OK = 0,
   MC_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum value */
-  MC_ERR_SHAPE = 2,       /* head_dim != 128, page_size not 16/32/64, head ratio not supported */
+  MC_ERR_SHAPE = 2,       /* head_dim != 128, page_size not 16/32/64, head ratio not supported,
+                             batch above 1024 (merge) or 512 (decode attention) */
   MC_ERR_DTYPE = 3,
   MC_ERR_ALIGN = 4,       /* a pool base is not 256-byte aligned */
   MC_ERR_CAPACITY = 5,    /* workspace too small / retained pool overflowed (from mc_read_status) */

@@ -33,8 +33,6 @@ struct MergeParams {
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
   float ta, tc;
   int items_per_page;
-  int pages_used;   // page slots per sequence that can hold tokens
-  int total_items;  // 2 * batch * pages_used * items_per_page
   int32_t* status;
 };
 
@@ -189,15 +187,40 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
 // slot, row group -- row group fastest.
 struct MergeItem {
   int tensor, b, pslot, grp;
+  int pg;  // page slot counted over the used pages of all sequences
 };
-__device__ __forceinline__ bool merge_item(int i, const MergeParams& p, const int* lens, MergeItem& m) {
-  m.grp = i % p.items_per_page;
-  i /= p.items_per_page;
-  m.pslot = i % p.pages_used;
-  i /= p.pages_used;
-  m.b = i % p.g.batch;
-  m.tensor = i / p.g.batch;
-  return m.pslot * p.g.page_size < lens[m.b];
+// Only pages that hold tokens are enumerated: `pre` is the exclusive prefix of the sequences' page
+// counts (pre[batch] = P, all of them), an item index is ((tensor * P) + pg) * items_per_page + grp.
+// A CTA walks its items with a fixed stride, so the decomposition is kept incrementally (no
+// divisions per item) and the sequence is found by stepping forward in `pre`.
+__device__ __forceinline__ void merge_item_init(MergeItem& m, long long i, int ipp, int P, const int* pre) {
+  const long long per_tensor = (long long)P * ipp;
+  if (P == 0 || i >= 2 * per_tensor) {
+    m.tensor = 2;
+    m.b = m.pslot = m.grp = m.pg = 0;
+    return;
+  }
+  m.tensor = (int)(i / per_tensor);
+  const int rem = (int)(i - m.tensor * per_tensor);
+  m.pg = rem / ipp;
+  m.grp = rem - m.pg * ipp;
+  m.b = 0;
+  while (m.pg >= pre[m.b + 1]) ++m.b;
+  m.pslot = m.pg - pre[m.b];
+}
+__device__ __forceinline__ void merge_item_advance(MergeItem& m, int s_pg, int s_grp, int ipp, int P, const int* pre) {
+  if (m.tensor >= 2) return;
+  m.grp += s_grp;
+  const int carry = m.grp >= ipp ? 1 : 0;
+  m.grp -= carry * ipp;
+  m.pg += s_pg + carry;
+  while (m.pg >= P) {
+    m.pg -= P;
+    m.b = 0;
+    if (++m.tensor >= 2) return;
+  }
+  while (m.pg >= pre[m.b + 1]) ++m.b;
+  m.pslot = m.pg - pre[m.b];
 }
 
 // Persistent merge kernel.  The items' rows of both layers are streamed into a ring of shared-memory
@@ -253,8 +276,9 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
   int* page_s = reinterpret_cast<int*>(smem + kMergeStages * kMergeStageBytes);  // [kMergeStages] page id of the staged item
-  int* len_s = page_s + kMergeStages;                                            // [min(batch, kMergeMaxBatchSmem)]
-  volatile int* s_abort = len_s + kMergeMaxBatchSmem;
+  int* len_s = page_s + kMergeStages;                                            // [batch]
+  int* pre_s = len_s + kMergeMaxBatchSmem;                                       // [batch + 1] pages before each sequence
+  volatile int* s_abort = pre_s + kMergeMaxBatchSmem + 1;
   uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kMergeStages;
   const uint32_t stage0 = smem_u32(stages);
@@ -270,20 +294,37 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const bool lens_in_smem = p.g.batch <= kMergeMaxBatchSmem;
-  if (lens_in_smem)
-    for (int b = tid; b < p.g.batch; b += kMergeThreads) len_s[b] = p.g.seq_lens[b];
+  for (int b = tid; b < p.g.batch; b += kMergeThreads) len_s[b] = p.g.seq_lens[b];
   __syncthreads();
-  const int* lens = lens_in_smem ? len_s : p.g.seq_lens;
-  const int total = p.total_items;
+  if (warp == 0) {
+    // exclusive prefix of the sequences' page counts: a lane sums a run of sequences, the runs are
+    // scanned with shuffles
+    const int per = (p.g.batch + 31) / 32;
+    const int b0 = min(lane * per, p.g.batch), b1 = min(b0 + per, p.g.batch);
+    int sum = 0;
+    for (int b = b0; b < b1; ++b) sum += (len_s[b] + ps - 1) >> p.g.page_shift;
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    int acc = incl - sum;
+    for (int b = b0; b < b1; ++b) {
+      pre_s[b] = acc;
+      acc += (len_s[b] + ps - 1) >> p.g.page_shift;
+    }
+    if (lane == 31) pre_s[p.g.batch] = incl;
+  }
+  __syncthreads();
+  const int* lens = len_s;
+  const int P = pre_s[p.g.batch];
+  const int ipp = p.items_per_page;
   const int stride = gridDim.x;
+  const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
 
-  auto next_valid = [&](int i, MergeItem& m) {
-    while (i < total && !merge_item(i, p, lens, m)) i += stride;
-    return i;
-  };
-  auto page_of = [&](int i, const MergeItem& m) {
-    return i < total ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
+  auto page_of = [&](const MergeItem& m) {
+    return m.tensor < 2 ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
   };
   // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kMergeStages
   auto issue = [&](int j, const MergeItem& m, int page) -> bool {
@@ -316,39 +357,40 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
   };
 
   MergeItem m;
-  int i = next_valid(blockIdx.x, m);
+  merge_item_init(m, blockIdx.x, ipp, P, pre_s);
   // warp 0 looks two items ahead (and loads page ids three ahead: a demand load takes microseconds
   // while the copies saturate the memory system)
   MergeItem m1 = m, m2 = m, m3 = m;
-  int i1 = total, i2 = total, i3 = total, pg2 = 0, pg3 = 0;
+  int pg2 = 0, pg3 = 0;
   if (warp == 0) {
-    i1 = i < total ? next_valid(i + stride, m1) : total;
-    i2 = i1 < total ? next_valid(i1 + stride, m2) : total;
-    i3 = i2 < total ? next_valid(i2 + stride, m3) : total;
-    const int pg0 = page_of(i, m), pg1 = page_of(i1, m1);
-    pg2 = page_of(i2, m2);
-    pg3 = page_of(i3, m3);
+    merge_item_advance(m1, s_pg, s_grp, ipp, P, pre_s);
+    m2 = m1;
+    merge_item_advance(m2, s_pg, s_grp, ipp, P, pre_s);
+    m3 = m2;
+    merge_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+    const int pg0 = page_of(m), pg1 = page_of(m1);
+    pg2 = page_of(m2);
+    pg3 = page_of(m3);
     if (lane == 0) {
-      if (i < total) issue(0, m, pg0);
-      if (i1 < total) issue(1, m1, pg1);
+      if (m.tensor < 2) issue(0, m, pg0);
+      if (m1.tensor < 2) issue(1, m1, pg1);
     }
   }
 
   const int quad = tid >> 2, k = tid & 3;
   long long run_seg = -1;  // segment of the warp's running distance extremes
   float run_min = 0.f, run_max = 0.f;
-  for (int it = 0; i < total; ++it) {
+  for (int it = 0; m.tensor < 2; ++it) {
     if (warp == 0) {
       // item it + 2 goes into the stage that item it - 1 has just left
       int good = 1;
-      if (lane == 0 && i2 < total) good = issue(it + 2, m2, pg2) ? 1 : 0;
+      if (lane == 0 && m2.tensor < 2) good = issue(it + 2, m2, pg2) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
-      i2 = i3;
       m2 = m3;
       pg2 = pg3;
-      i3 = i2 < total ? next_valid(i2 + stride, m3) : total;
-      pg3 = page_of(i3, m3);
+      merge_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+      pg3 = page_of(m3);
     }
     const int s = it % kMergeStages;
     if (!mbar_wait(full0 + 8 * s, (it / kMergeStages) & 1, s_abort, p.status)) break;
@@ -439,7 +481,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
         run_max = fmaxf(run_max, dmax);
       }
     }
-    i = next_valid(i + stride, m);
+    merge_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
   }
   if (lane == 0 && run_seg >= 0) {
     atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));
@@ -903,10 +945,10 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
-  mp.pages_used = (bt->max_seq_len + cfg->page_size - 1) / cfg->page_size;
-  const long long total = 2LL * bt->batch * mp.pages_used * mp.items_per_page;
+  if (bt->batch > kMergeMaxBatchSmem) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
+  // upper bound of the item count (the kernel enumerates the pages that hold tokens)
+  const long long total = 2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
   if (total > 0x7fffffffLL) return MC_ERR_SHAPE;
-  mp.total_items = (int)total;
   mp.status = out->status;
   if (total > 0) {
     static int n_sm = 0;
@@ -916,7 +958,7 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
       MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     }
     const int grid = (int)std::min<long long>((long long)n_sm * kMergeCtasPerSm, total);
-    const size_t smem = 128 + (size_t)kMergeStages * kMergeStageBytes + (kMergeStages + kMergeMaxBatchSmem + 2) * 4 + 8 +
+    const size_t smem = 128 + (size_t)kMergeStages * kMergeStageBytes + (kMergeStages + 2 * kMergeMaxBatchSmem + 3) * 4 + 8 +
                         2 * kMergeStages * 8 + 64;
     void (*kern)(const MergeParams) =
         cfg->dtype == MC_F16 ? (q4 ? merge_kernel<MC_F16, true> : merge_kernel<MC_F16, false>)
