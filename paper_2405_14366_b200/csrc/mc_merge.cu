@@ -7,6 +7,7 @@
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
+#include "mc_items.cuh"
 #include "mc_pipe.cuh"
 
 namespace mc {
@@ -17,7 +18,7 @@ constexpr int kMergeStageBytes = 2 * kRowsPerItem * kRowBytes;  // the item's ro
 constexpr int kMergeWarps = 8;
 constexpr int kMergeThreads = kMergeWarps * 32;
 constexpr int kMergeCtasPerSm = 2;
-constexpr int kMergeMaxBatchSmem = 1024;
+constexpr int kMergeMaxBatchSmem = kMaxBatchPages;
 constexpr int kQ4RowBytes = 64;                              // 128 four-bit codes
 constexpr int kQ4CodesBytes = kRowsPerItem * kQ4RowBytes;    // one layer's codes of an item
 constexpr int kQ4MetaBytes = kRowsPerItem * 16;              // one layer's (scale, zero) pairs of an item
@@ -185,44 +186,6 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
 // Work item of the merge: 64 consecutive rows of one page (rows of a page are [head][token], so an
 // item is a contiguous 16 KB block in each layer's pool).  Flattened order: tensor, sequence, page
 // slot, row group -- row group fastest.
-struct MergeItem {
-  int tensor, b, pslot, grp;
-  int pg;  // page slot counted over the used pages of all sequences
-};
-// Only pages that hold tokens are enumerated: `pre` is the exclusive prefix of the sequences' page
-// counts (pre[batch] = P, all of them), an item index is ((tensor * P) + pg) * items_per_page + grp.
-// A CTA walks its items with a fixed stride, so the decomposition is kept incrementally (no
-// divisions per item) and the sequence is found by stepping forward in `pre`.
-__device__ __forceinline__ void merge_item_init(MergeItem& m, long long i, int ipp, int P, const int* pre) {
-  const long long per_tensor = (long long)P * ipp;
-  if (P == 0 || i >= 2 * per_tensor) {
-    m.tensor = 2;
-    m.b = m.pslot = m.grp = m.pg = 0;
-    return;
-  }
-  m.tensor = (int)(i / per_tensor);
-  const int rem = (int)(i - m.tensor * per_tensor);
-  m.pg = rem / ipp;
-  m.grp = rem - m.pg * ipp;
-  m.b = 0;
-  while (m.pg >= pre[m.b + 1]) ++m.b;
-  m.pslot = m.pg - pre[m.b];
-}
-__device__ __forceinline__ void merge_item_advance(MergeItem& m, int s_pg, int s_grp, int ipp, int P, const int* pre) {
-  if (m.tensor >= 2) return;
-  m.grp += s_grp;
-  const int carry = m.grp >= ipp ? 1 : 0;
-  m.grp -= carry * ipp;
-  m.pg += s_pg + carry;
-  while (m.pg >= P) {
-    m.pg -= P;
-    m.b = 0;
-    if (++m.tensor >= 2) return;
-  }
-  while (m.pg >= pre[m.b + 1]) ++m.b;
-  m.pslot = m.pg - pre[m.b];
-}
-
 // Persistent merge kernel.  The items' rows of both layers are streamed into a ring of shared-memory
 // stages with bulk asynchronous copies (two 16 KB copies per stage), issued two items ahead by lane 0
 // of warp 0; the eight warps take a row per quad of lanes out of shared memory, release the stage,
@@ -294,40 +257,18 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int b = tid; b < p.g.batch; b += kMergeThreads) len_s[b] = p.g.seq_lens[b];
-  __syncthreads();
-  if (warp == 0) {
-    // exclusive prefix of the sequences' page counts: a lane sums a run of sequences, the runs are
-    // scanned with shuffles
-    const int per = (p.g.batch + 31) / 32;
-    const int b0 = min(lane * per, p.g.batch), b1 = min(b0 + per, p.g.batch);
-    int sum = 0;
-    for (int b = b0; b < b1; ++b) sum += (len_s[b] + ps - 1) >> p.g.page_shift;
-    int incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
-    }
-    int acc = incl - sum;
-    for (int b = b0; b < b1; ++b) {
-      pre_s[b] = acc;
-      acc += (len_s[b] + ps - 1) >> p.g.page_shift;
-    }
-    if (lane == 31) pre_s[p.g.batch] = incl;
-  }
-  __syncthreads();
+  page_prefix(p.g, len_s, pre_s, kMergeThreads);
   const int* lens = len_s;
   const int P = pre_s[p.g.batch];
   const int ipp = p.items_per_page;
   const int stride = gridDim.x;
   const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
 
-  auto page_of = [&](const MergeItem& m) {
+  auto page_of = [&](const PageItem& m) {
     return m.tensor < 2 ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
   };
   // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kMergeStages
-  auto issue = [&](int j, const MergeItem& m, int page) -> bool {
+  auto issue = [&](int j, const PageItem& m, int page) -> bool {
     const int s = j % kMergeStages;
     if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, p.status)) return false;
     const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
@@ -356,18 +297,18 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     return true;
   };
 
-  MergeItem m;
-  merge_item_init(m, blockIdx.x, ipp, P, pre_s);
+  PageItem m;
+  page_item_init(m, blockIdx.x, ipp, P, pre_s);
   // warp 0 looks two items ahead (and loads page ids three ahead: a demand load takes microseconds
   // while the copies saturate the memory system)
-  MergeItem m1 = m, m2 = m, m3 = m;
+  PageItem m1 = m, m2 = m, m3 = m;
   int pg2 = 0, pg3 = 0;
   if (warp == 0) {
-    merge_item_advance(m1, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m1, s_pg, s_grp, ipp, P, pre_s);
     m2 = m1;
-    merge_item_advance(m2, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m2, s_pg, s_grp, ipp, P, pre_s);
     m3 = m2;
-    merge_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
     const int pg0 = page_of(m), pg1 = page_of(m1);
     pg2 = page_of(m2);
     pg3 = page_of(m3);
@@ -389,7 +330,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       if (!good) break;
       m2 = m3;
       pg2 = pg3;
-      merge_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+      page_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
       pg3 = page_of(m3);
     }
     const int s = it % kMergeStages;
@@ -481,7 +422,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
         run_max = fmaxf(run_max, dmax);
       }
     }
-    merge_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
   }
   if (lane == 0 && run_seg >= 0) {
     atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));

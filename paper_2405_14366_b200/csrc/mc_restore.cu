@@ -1,14 +1,23 @@
 // Materialising restore of one layer (Eq. 2; Sec. 4.2 "Cache restoration"):
 //   restore_scale_kernel    x_hat = e_stored * (|x| / |e_stored|) for every cached row
 //   restore_scatter_kernel  retained rows overwritten with their raw copies (x_hat[I] = R)
+#include <algorithm>
+
 #include "mc_common.cuh"
+#include "mc_items.cuh"
 #include "mc_kernels.h"
+#include "mc_pipe.cuh"
 
 namespace mc {
 
 constexpr int kRestoreThreads = 256;
+constexpr int kRestoreWarps = kRestoreThreads / 32;
+constexpr int kRestoreCtasPerSm = 2;
 constexpr int kRowsPerItem = 64;
-constexpr int kRowsPerHalfWarp = 4;
+constexpr int kRestoreStages = 6;
+// 64 rows of tiles: 64 / page_size whole (page, head) tiles, 16896 bytes for every page size
+constexpr int kRestoreStageBytes = (kRowsPerItem / 16) * (16 * kRowBytes + 2 * 16 * 4);
+constexpr int kRestoreAhead = kRestoreStages - 1;  // items in flight beyond the one being consumed
 
 struct RestoreParams {
   Geom g;
@@ -21,56 +30,141 @@ struct RestoreParams {
   int64_t ret_capacity;
   int layer;  // 0: l-1, 1: l
   int items_per_page;
+  int32_t* status;
 };
 
+// Persistent: two CTAs per SM walk the items (64 rows of a page that holds tokens) with a fixed
+// stride.  An item's tiles are one contiguous block of the pair cache; lane 0 of warp 0 streams
+// them into a ring of shared-memory stages with one bulk asynchronous copy per item, five items
+// ahead, so the bytes in flight are set by the ring.  A half-warp takes a row out of shared memory
+// (undoing the chunk permutation), the stage is released as soon as the rows are in registers, and
+// the scaled rows leave with streaming stores.
 template <int DT>
-__global__ void __launch_bounds__(kRestoreThreads) restore_scale_kernel(const RestoreParams p) {
+__global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_scale_kernel(const RestoreParams p) {
   grid_dep_wait();
   grid_dep_launch();
-  const int ipp = p.items_per_page;
-  int bid = blockIdx.x;
-  const int item = bid % ipp;
-  bid /= ipp;
-  const int pslot = bid % p.g.max_pages_per_seq;
-  bid /= p.g.max_pages_per_seq;
-  const int b = bid % p.g.batch;
-  const int tensor = bid / p.g.batch;
-  const int n = p.g.seq_lens[b];
-  const int ps = p.g.page_size;
-  if (pslot * ps >= n) return;
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + pslot];
-  const int H = p.g.n_kv_heads;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  unsigned char* stages = smem;
+  int* page_s = reinterpret_cast<int*>(smem + kRestoreStages * kRestoreStageBytes);  // [kRestoreStages]
+  int* len_s = page_s + kRestoreStages;                                               // [batch]
+  int* pre_s = len_s + kMaxBatchPages;                                                // [batch + 1]
+  volatile int* s_abort = pre_s + kMaxBatchPages + 1;
+  uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kRestoreStages;
+  const uint32_t stage0 = smem_u32(stages);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ps = p.g.page_size, shift = p.g.page_shift, H = p.g.n_kv_heads;
   const int rows_in_page = H * ps;
-  const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-  const int row0 = item * kRowsPerItem + hw * kRowsPerHalfWarp;
-  if (row0 >= rows_in_page) return;
-  const int head = row0 >> p.g.page_shift;
-  const int tk0 = row0 & (ps - 1);
-  const int tok0 = pslot * ps + tk0;
-  const size_t page_off = (size_t)page * rows_in_page;
-  const char* tile = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
-  char* pd = p.dst_pool[tensor] + (page_off + row0) * kRowBytes + l16 * 16;
-  const float* sc = reinterpret_cast<const float*>(tile + ps * kRowBytes) + p.layer * ps + tk0;
-  uint4 v[kRowsPerHalfWarp];
-  float g[kRowsPerHalfWarp];
-#pragma unroll
-  for (int j = 0; j < kRowsPerHalfWarp; ++j)
-    if (tok0 + j < n) {
-      v[j] = ld_stream16(tile + (tk0 + j) * kRowBytes + chunk_pos(tk0 + j, l16) * 16);
-      g[j] = __ldg(sc + j);
+  const int tbytes = tile_bytes(ps);
+
+  if (tid == 0) {
+    for (int s = 0; s < kRestoreStages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, kRestoreWarps);
     }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  page_prefix(p.g, len_s, pre_s, kRestoreThreads);
+  const int P = pre_s[p.g.batch];
+  const int ipp = p.items_per_page;
+  const int stride = gridDim.x;
+  const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
+
+  auto page_of = [&](const PageItem& m) {
+    return m.tensor < 2 ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
+  };
+  // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kRestoreStages
+  auto issue = [&](int j, const PageItem& m, int page) -> bool {
+    const int s = j % kRestoreStages;
+    if (j >= kRestoreStages && !mbar_wait(empty0 + 8 * s, ((j / kRestoreStages) - 1) & 1, s_abort, p.status)) return false;
+    const int h0 = (m.grp * kRowsPerItem) >> shift;
+    const int n_tiles = min(kRowsPerItem >> shift, H - h0);
+    const uint32_t bytes = (uint32_t)(n_tiles * tbytes);
+    const uint32_t bar = full0 + 8 * s;
+    page_s[s] = page;
+    mbar_expect_tx(bar, bytes);
+    bulk_load(stage0 + s * kRestoreStageBytes, (m.tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + h0) * tbytes, bytes, bar);
+    return true;
+  };
+
+  PageItem m;
+  page_item_init(m, blockIdx.x, ipp, P, pre_s);
+  // warp 0 keeps the issue point kRestoreAhead items ahead, and the page ids two items further (a
+  // demand load takes microseconds while the copies saturate the memory system)
+  PageItem mi = m, mn = m;
+  int pg_i = 0, pg_n = 0;
+  if (warp == 0) {
+    pg_i = page_of(mi);
+    page_item_advance(mn, s_pg, s_grp, ipp, P, pre_s);
+    pg_n = page_of(mn);
 #pragma unroll
-  for (int j = 0; j < kRowsPerHalfWarp; ++j)
-    if (tok0 + j < n) {
-      const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-      uint32_t o[4];
+    for (int j = 0; j < kRestoreAhead; ++j) {
+      if (lane == 0 && mi.tensor < 2) issue(j, mi, pg_i);
+      mi = mn;
+      pg_i = pg_n;
+      page_item_advance(mn, s_pg, s_grp, ipp, P, pre_s);
+      pg_n = page_of(mn);
+    }
+  }
+
+  const int hw = lane >> 4, l16 = lane & 15;
+  for (int it = 0; m.tensor < 2; ++it) {
+    if (warp == 0) {
+      // item it + kRestoreAhead goes into the stage that item it - 1 has just left
+      int good = 1;
+      if (lane == 0 && mi.tensor < 2) good = issue(it + kRestoreAhead, mi, pg_i) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      mi = mn;
+      pg_i = pg_n;
+      page_item_advance(mn, s_pg, s_grp, ipp, P, pre_s);
+      pg_n = page_of(mn);
+    }
+    const int s = it % kRestoreStages;
+    if (!mbar_wait(full0 + 8 * s, (it / kRestoreStages) & 1, s_abort, p.status)) break;
+    const int page = page_s[s];
+    const int n = len_s[m.b];
+    // warp w: rows 8 w .. 8 w + 7 of the item, four per half-warp
+    const int r0 = warp * 8 + hw * 4;
+    const unsigned char* sb = stages + s * kRestoreStageBytes;
+    uint4 v[4];
+    float g[4];
+    bool ok[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = Elem<DT>::unpack(w[i]);
-        o[i] = Elem<DT>::pack(f.x * g[j], f.y * g[j]);
+    for (int j = 0; j < 4; ++j) {
+      const int r = r0 + j, rp = m.grp * kRowsPerItem + r;
+      const int tk = r & (ps - 1);
+      const unsigned char* tile = sb + (r >> shift) * tbytes;
+      ok[j] = rp < rows_in_page && m.pslot * ps + tk < n;
+      v[j] = make_uint4(0u, 0u, 0u, 0u);
+      g[j] = 0.f;
+      if (ok[j]) {
+        v[j] = *reinterpret_cast<const uint4*>(tile + tk * kRowBytes + chunk_pos(tk, l16) * 16);
+        g[j] = reinterpret_cast<const float*>(tile + ps * kRowBytes)[p.layer * ps + tk];
       }
-      st_stream16(pd + j * kRowBytes, make_uint4(o[0], o[1], o[2], o[3]));
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
+    char* pd = (m.tensor ? p.dst_pool[1] : p.dst_pool[0]) + ((size_t)page * rows_in_page + m.grp * kRowsPerItem + r0) * kRowBytes + l16 * 16;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (ok[j]) {
+        const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = Elem<DT>::unpack(w[i]);
+          o[i] = Elem<DT>::pack(f.x * g[j], f.y * g[j]);
+        }
+        st_stream16(pd + j * kRowBytes, make_uint4(o[0], o[1], o[2], o[3]));
+      }
+    page_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
+  }
+  if (*s_abort) {
+    for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
+  }
 }
 
 __global__ void __launch_bounds__(kRestoreThreads) restore_scatter_kernel(const RestoreParams p) {
@@ -110,13 +204,24 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
   rp.ret_capacity = pair->ret_capacity;
   rp.layer = layer;
   rp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
-  const long long blocks = 2LL * bt->batch * bt->max_pages_per_seq * rp.items_per_page;
+  rp.status = pair->status;
+  if (bt->batch > kMaxBatchPages) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
+  // upper bound of the item count (the kernel enumerates the pages that hold tokens)
+  const long long blocks = 2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * rp.items_per_page;
   if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
   if (blocks > 0) {
-    if (cfg->dtype == MC_F16)
-      MC_CUDA_CHECK(launch_pdl(restore_scale_kernel<MC_F16>, dim3((unsigned)blocks), dim3(kRestoreThreads), 0, stream, rp));
-    else
-      MC_CUDA_CHECK(launch_pdl(restore_scale_kernel<MC_BF16>, dim3((unsigned)blocks), dim3(kRestoreThreads), 0, stream, rp));
+    static int n_sm = 0;
+    if (n_sm == 0) {
+      int dev = 0;
+      MC_CUDA_CHECK(cudaGetDevice(&dev));
+      MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    }
+    const int grid = (int)std::min<long long>((long long)n_sm * kRestoreCtasPerSm, blocks);
+    const size_t smem = 128 + (size_t)kRestoreStages * kRestoreStageBytes + (kRestoreStages + 2 * kMaxBatchPages + 3) * 4 + 8 +
+                        2 * kRestoreStages * 8 + 64;
+    void (*kern)(const RestoreParams) = cfg->dtype == MC_F16 ? restore_scale_kernel<MC_F16> : restore_scale_kernel<MC_BF16>;
+    MC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MC_CUDA_CHECK(launch_pdl(kern, dim3(grid), dim3(kRestoreThreads), smem, stream, rp));
     MC_CUDA_CHECK(cudaGetLastError());
   }
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
