@@ -183,10 +183,15 @@ struct Ranges {
 };
 
 // Two table entries per list: split boundaries are multiples of 128 and no retained token lies
-// past the length the pair was merged at.
-__device__ __forceinline__ Ranges load_ranges(const Item& w, const AttnParams& p) {
-  Ranges r;
-  r.k_lo = r.n_k = r.v_lo = r.n_v = 0;
+// past the length the pair was merged at.  The loads are issued one item ahead and only combined
+// (ranges_of) when that item starts: arithmetic on a loaded value would stall the producer warp for
+// the load's whole latency, microseconds while the copy engine saturates the memory system.
+struct RawRanges {
+  int off_k, off_v, k0, k1, v0, v1;
+};
+__device__ __forceinline__ RawRanges load_ranges(const Item& w, const AttnParams& p) {
+  RawRanges r;
+  r.off_k = r.off_v = r.k0 = r.k1 = r.v0 = r.v1 = 0;
   if (!w.valid) return r;
   const int H = p.g.n_kv_heads;
   const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
@@ -194,12 +199,20 @@ __device__ __forceinline__ Ranges load_ranges(const Item& w, const AttnParams& p
   const int pj1 = min((w.split_start + w.n_tok + 127) >> 7, p.ret_prefix_stride - 1);
   const int32_t* pk = p.ret_prefix + (size_t)seg_k * p.ret_prefix_stride;
   const int32_t* pv = p.ret_prefix + (size_t)seg_v * p.ret_prefix_stride;
-  const int off_k = __ldg(p.ret_offset + seg_k), off_v = __ldg(p.ret_offset + seg_v);
-  const int k0 = __ldg(pk + pj0), k1 = __ldg(pk + pj1), v0 = __ldg(pv + pj0), v1 = __ldg(pv + pj1);
-  r.k_lo = off_k + k0;
-  r.n_k = k1 - k0;
-  r.v_lo = off_v + v0;
-  r.n_v = v1 - v0;
+  r.off_k = __ldg(p.ret_offset + seg_k);
+  r.off_v = __ldg(p.ret_offset + seg_v);
+  r.k0 = __ldg(pk + pj0);
+  r.k1 = __ldg(pk + pj1);
+  r.v0 = __ldg(pv + pj0);
+  r.v1 = __ldg(pv + pj1);
+  return r;
+}
+__device__ __forceinline__ Ranges ranges_of(const RawRanges& q) {
+  Ranges r;
+  r.k_lo = q.off_k + q.k0;
+  r.n_k = q.k1 - q.k0;
+  r.v_lo = q.off_v + q.v0;
+  r.n_v = q.v1 - q.v0;
   return r;
 }
 
@@ -264,14 +277,15 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     // engine saturates the memory system.
     int it = 0;  // running stage counter, same sequence as the consumers'
     Item w = get_item(first, total_items, pre_s, len_s, p);
-    Ranges rg = load_ranges(w, p);
+    RawRanges raw = load_ranges(w, p);
     int my_page = 0;
     if (w.valid && lane < ((w.n_tok + ps - 1) >> shift))
       my_page = p.g.block_table[(size_t)w.b * p.g.max_pages_per_seq + (w.split_start >> shift) + lane];
     bool ok = true;
     for (int i = first; i < total_items && ok; i += stride) {
       const Item wn = get_item(i + stride, total_items, pre_s, len_s, p);
-      const Ranges rgn = load_ranges(wn, p);
+      const Ranges rg = ranges_of(raw);  // loaded one item ago
+      const RawRanges rawn = load_ranges(wn, p);
       int next_page = 0;
       if (wn.valid && lane < ((wn.n_tok + ps - 1) >> shift))
         next_page = p.g.block_table[(size_t)wn.b * p.g.max_pages_per_seq + (wn.split_start >> shift) + lane];
@@ -333,7 +347,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         }
       }
       w = wn;
-      rg = rgn;
+      raw = rawn;
       my_page = next_page;
     }
     return;
