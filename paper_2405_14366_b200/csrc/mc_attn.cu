@@ -39,7 +39,6 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
 constexpr int kMaxRows = 8;                          // query rows per work item (M tile rows used)
 constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
-constexpr int kMaxSplit = 512;
 constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
 constexpr int kCtasPerSm = 2;
@@ -58,8 +57,9 @@ struct AttnParams {
   const char* q;
   const char* k_new;
   const char* v_new;
-  float* part_o;   // [n_sets][batch][Hq][n_splits][128]
-  float* part_ml;  // [n_sets][batch][Hq][n_splits][2]
+  float* part_o;   // [n_sets][batch][Hq][slots][128]: a piece's partial sits in the slot of its first unit
+  float* part_ml;  // [n_sets][batch][Hq][slots][2]
+  int32_t* part_meta;  // [batch + 2]: prefix of the sequences' unit counts, then the split kernel's grid size
   int32_t* status;
   float scale_log2;  // sm_scale * log2(e)
   int layer_sel;
@@ -67,8 +67,9 @@ struct AttnParams {
   int nq;    // query heads per kv head
   int rows;  // n_sets * nq
   int n_q_heads;
-  int split_len;
-  int n_splits;
+  int cap_units;  // longest piece, in units of 128 tokens (what the score buffer holds for `rows` rows)
+  int slots;      // partial slots per output row = units of the longest sequence
+  int team_size;  // CTAs per team (one or more kv heads each)
 };
 
 // ---- PTX wrappers (tensor-core side; the copy/barrier wrappers live in mc_pipe.cuh) ---------------
@@ -126,55 +127,80 @@ __device__ __forceinline__ uint32_t tile_addr(uint32_t stage, int tk, int chunk,
   return stage + (uint32_t)(j * tbytes + r * kRowBytes + (chunk_pos(r, chunk) << 4));
 }
 
-// Floats of the score buffer S [kMaxRows][split_len + 8]; the same memory later holds the four
-// warps' partial outputs [4][rows][kSlabStride].
-__host__ __device__ __forceinline__ int s_region_floats(int split_len) {
-  const int a = split_len + 8, b = kConsumerWarps * kSlabStride;
-  return kMaxRows * (a > b ? a : b);
+constexpr int kUnit = 128;            // tokens per unit of work: pieces start and end on unit boundaries
+constexpr int kScoreFloats = 4224;    // floats of the score buffer S [rows][piece tokens + 8] (16.5 KB)
+constexpr int kMaxPiecePages = 256;   // pages of the longest piece (4096 tokens of 16-token pages)
+
+// Longest piece for `rows` query rows: rows x (tokens + 8) floats must fit the score buffer.
+__host__ __device__ __forceinline__ int piece_cap_units(int rows) {
+  const int u = (kScoreFloats / rows - 8) / kUnit;
+  return u > 32 ? 32 : u;  // 32 units (rows = 1) ... 4 units (rows = 8)
 }
+// The same memory later holds the four warps' partial outputs [4][rows][kSlabStride].
+static_assert(kMaxRows * ((kScoreFloats / kMaxRows - 8) / kUnit * kUnit + 8) <= kScoreFloats, "score buffer");
+static_assert(kConsumerWarps * kMaxRows * kSlabStride <= kScoreFloats, "slabs fit the score buffer");
 
 // The merge marks a retained token by the scale -0: the shared direction then contributes nothing
 // wherever scales are applied blindly, and a token whose rows are genuinely zero (scale +0, score 0)
 // stays distinguishable.
 __device__ __forceinline__ bool is_retained_scale(float g) { return __float_as_uint(g) == 0x80000000u; }
 
-// One work item.
+// One work item = a piece: a run of units of one (sequence, kv head).
 struct Item {
-  int b, g, split;
+  int b, g, split;  // split = the piece's first unit inside its sequence (also its partial slot)
   int split_start;
-  int n_tok;    // cached tokens of this split
+  int n_tok;    // cached tokens of this piece
   int T;        // 64-token tiles
+  int units;
   bool has_new;
   bool valid;
 };
 
-// Item `i` of the flattened list (sequence-major, then split, then kv head) from the per-sequence
-// prefix of split counts in shared memory.
-__device__ __forceinline__ Item get_item(int i, int total, const int* pre_s, const int* len_s, const AttnParams& p) {
+// Work is cut along the token axis only.  A sequence owns max(1, ceil(n / 128)) units (pre_s =
+// exclusive prefix over sequences, U units in all).  The grid is T teams of S CTAs: team t takes
+// the units [t U / T, (t + 1) U / T) -- the same share for every team whatever the lengths are --
+// and its member j takes them for the kv heads j, j + S, ...  The members of a team stream the
+// same pages at about the same time (neighbouring tiles of a page: whole DRAM rows get used), and
+// nobody waits for a last round of items.  A piece = a run of units of one (sequence, head): it
+// stops at the end of the sequence, at the end of the team's range and at the capacity of the
+// score buffer.
+struct Cursor {
+  int g, x;  // kv head, unit
+};
+__device__ __forceinline__ Item piece_at(const Cursor& c, int x_end, const int* pre_s, const int* len_s, const AttnParams& p) {
   Item it;
-  it.valid = i < total;
+  it.valid = c.g < p.g.n_kv_heads && c.x < x_end;
   if (!it.valid) {
-    it.b = it.g = it.split = it.split_start = it.n_tok = it.T = 0;
+    it.b = it.g = it.split = it.split_start = it.n_tok = it.T = it.units = 0;
     it.has_new = false;
     return it;
   }
-  const int H = p.g.n_kv_heads;
-  int lo = 0, hi = p.g.batch - 1;  // last b with pre_s[b] * H <= i
+  int lo = 0, hi = p.g.batch - 1;  // last b with pre_s[b] <= x
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if (pre_s[mid] * H <= i) lo = mid; else hi = mid - 1;
+    if (pre_s[mid] <= c.x) lo = mid; else hi = mid - 1;
   }
   it.b = lo;
-  const int local = i - pre_s[lo] * H;
-  it.split = local / H;
-  it.g = local - it.split * H;
+  it.g = c.g;
+  const int u_b = pre_s[lo + 1] - pre_s[lo];
+  it.split = c.x - pre_s[lo];
+  it.units = min(min(u_b - it.split, x_end - c.x), p.cap_units);
   const int n = len_s[lo];
-  const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
-  it.split_start = it.split * p.split_len;
-  it.n_tok = max(0, min(n, it.split_start + p.split_len) - it.split_start);
+  it.split_start = it.split * kUnit;
+  it.n_tok = max(0, min(n, (it.split + it.units) * kUnit) - it.split_start);
   it.T = (it.n_tok + kTile - 1) / kTile;
-  it.has_new = (p.k_new != nullptr) && (it.split == nsp - 1);
+  it.has_new = (p.k_new != nullptr) && (it.split + it.units == u_b);
   return it;
+}
+// The cursor after piece `it`: on through the team's range, then the member's next head.
+__device__ __forceinline__ Cursor next_cursor(const Cursor& c, const Item& it, int x_begin, int x_end, int team_size) {
+  Cursor n = c;
+  n.x += it.units;
+  if (n.x >= x_end) {
+    n.x = x_begin;
+    n.g += team_size;
+  }
+  return n;
 }
 
 // Where an item's retained entries sit in the pair's lists (first entry, count) for K and V.
@@ -218,14 +244,17 @@ __device__ __forceinline__ Ranges ranges_of(const RawRanges& q) {
 
 template <int DT>
 __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(const AttnParams p) {
-  grid_dep_wait();
+  // The batch description (lengths, block table) and the queries belong to the caller: no kernel of
+  // this library writes them, so they are read before the wait on the previous kernel in the
+  // stream (whose tail this prologue then overlaps).  The pair cache and the workspace are touched
+  // only after the wait.
   grid_dep_launch();
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
   const int tbytes = tile_bytes(ps);
   const int nslots = p.n_sets;
   const int rows = p.rows;
-  const int s_stride = p.split_len + 8;
+  const int s_stride = p.cap_units * kUnit + 8;
   const int cap_e = nslots == 2 ? 16 : 32;  // retained entries (per layer) in one extra stage
   const int set_bytes = cap_e * kEntryBytes;
 
@@ -233,15 +262,16 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
   float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);     // [kMaxRows][s_stride]
-  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + s_region_floats(p.split_len));  // [2][kMaxRows][64] packed pairs
+  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kScoreFloats);         // [2][kMaxRows][64] packed pairs
   float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
   float* red2_s = red_s + kMaxRows * kConsumerWarps;                     // [kMaxRows][kConsumerWarps]
   int* info_s = reinterpret_cast<int*>(red2_s + kMaxRows * kConsumerWarps);  // [kStages][2]: entries, extra stages of the phase
-  int* pre_s = info_s + 2 * kStages;                                     // [batch + 1] split-count prefix
+  int* pre_s = info_s + 2 * kStages;                                     // [batch + 1] unit-count prefix
   int* len_s = pre_s + kMaxBatchSmem + 1;                                // [batch] sequence lengths
-  volatile int* s_abort = len_s + kMaxBatchSmem;
+  int* pages_s = len_s + kMaxBatchSmem;                                  // [2][kMaxPiecePages] page ids of a piece
+  volatile int* s_abort = pages_s + 2 * kMaxPiecePages;
   uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
   const uint32_t stage0 = smem_u32(stages);
@@ -256,19 +286,24 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // prefix of per-sequence split counts (a sequence always owns at least one split)
+  }
+  for (int b = tid; b < p.g.batch; b += kAttnThreads) len_s[b] = p.g.seq_lens[b];
+  __syncthreads();
+  if (tid == 0) {
+    // prefix of the sequences' unit counts (a sequence always owns at least one unit)
     int acc = 0;
     for (int b = 0; b < p.g.batch; ++b) {
-      const int n = p.g.seq_lens[b];
-      len_s[b] = n;
       pre_s[b] = acc;
-      acc += max(1, (n + p.split_len - 1) / p.split_len);
+      acc += max(1, (len_s[b] + kUnit - 1) / kUnit);
     }
     pre_s[p.g.batch] = acc;
   }
   __syncthreads();
-  const int total_items = pre_s[p.g.batch] * H;
-  const int first = blockIdx.x, stride = gridDim.x;
+  const int n_teams = gridDim.x / p.team_size;
+  const int team = blockIdx.x / p.team_size;
+  const long long n_units = pre_s[p.g.batch];
+  const int x_begin = (int)(n_units * team / n_teams), x_end = (int)(n_units * (team + 1) / n_teams);
+  const Cursor c_first = {(int)(blockIdx.x % p.team_size), x_begin};
 
   if (warp == kConsumerWarps) {
     // ===================== producer =====================
@@ -276,19 +311,36 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     // retained ranges) is loaded one item ahead: such loads take microseconds while the copy
     // engine saturates the memory system.
     int it = 0;  // running stage counter, same sequence as the consumers'
-    Item w = get_item(first, total_items, pre_s, len_s, p);
-    RawRanges raw = load_ranges(w, p);
-    int my_page = 0;
-    if (w.valid && lane < ((w.n_tok + ps - 1) >> shift))
-      my_page = p.g.block_table[(size_t)w.b * p.g.max_pages_per_seq + (w.split_start >> shift) + lane];
+    Cursor cur = c_first;
+    Item w = piece_at(cur, x_end, pre_s, len_s, p);
+    RawRanges raw;
+    // page ids of a piece: lane l holds pages l, l + 32, ... (registers, loaded one piece ahead),
+    // handed over to shared memory when the piece starts
+    int pg_reg[kMaxPiecePages / 32];
+    auto load_pages = [&](const Item& it) {
+      const int np = (it.n_tok + ps - 1) >> shift;
+      const int32_t* row = p.g.block_table + (size_t)it.b * p.g.max_pages_per_seq + (it.split_start >> shift);
+#pragma unroll
+      for (int r = 0; r < kMaxPiecePages / 32; ++r) {
+        pg_reg[r] = 0;
+        if (it.valid && lane + 32 * r < np) pg_reg[r] = row[lane + 32 * r];
+      }
+    };
+    load_pages(w);
+    grid_dep_wait();
+    raw = load_ranges(w, p);
     bool ok = true;
-    for (int i = first; i < total_items && ok; i += stride) {
-      const Item wn = get_item(i + stride, total_items, pre_s, len_s, p);
-      const Ranges rg = ranges_of(raw);  // loaded one item ago
+    int n_piece = 0;
+    for (; w.valid && ok; ++n_piece) {
+      int* pages = pages_s + (n_piece & 1) * kMaxPiecePages;
+#pragma unroll
+      for (int r = 0; r < kMaxPiecePages / 32; ++r) pages[lane + 32 * r] = pg_reg[r];
+      __syncwarp();
+      cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
+      const Item wn = piece_at(cur, x_end, pre_s, len_s, p);
+      const Ranges rg = ranges_of(raw);  // loaded one piece ago
       const RawRanges rawn = load_ranges(wn, p);
-      int next_page = 0;
-      if (wn.valid && lane < ((wn.n_tok + ps - 1) >> shift))
-        next_page = p.g.block_table[(size_t)wn.b * p.g.max_pages_per_seq + (wn.split_start >> shift) + lane];
+      load_pages(wn);
       const int n_pages_item = (w.n_tok + ps - 1) >> shift;
       const int n_new = w.has_new ? 1 : 0;
       for (int ph = 0; ph < 2 && ok; ++ph) {
@@ -314,9 +366,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               mbar_expect_tx(bar, (uint32_t)(n_pg * tbytes));
             }
             __syncwarp();
-            const int j = lane - pg0;  // lane pg0 + j holds the id of the stage's page j
-            if (j >= 0 && j < n_pg)
-              bulk_load(sbase + j * tbytes, p.e_pool[ph] + ((size_t)my_page * H + w.g) * tbytes, (uint32_t)tbytes, bar);
+            if (lane < n_pg)
+              bulk_load(sbase + lane * tbytes, p.e_pool[ph] + ((size_t)pages[pg0 + lane] * H + w.g) * tbytes, (uint32_t)tbytes,
+                        bar);
           } else {
             // ---- an extra stage: up to cap_e retained entries per layer, the new token last
             const int x0 = (t - w.T) * cap_e;
@@ -348,7 +400,6 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       }
       w = wn;
       raw = rawn;
-      my_page = next_page;
     }
     return;
   }
@@ -380,14 +431,22 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   };
   {
     uint32_t qw[4];
-    load_q_words(get_item(first, total_items, pre_s, len_s, p), qw);
+    load_q_words(piece_at(c_first, x_end, pre_s, len_s, p), qw);
 #pragma unroll
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
+  grid_dep_wait();
+  if (blockIdx.x == 0) {  // the combine kernel finds the pieces from the same numbers
+    for (int b = tid; b <= p.g.batch; b += kConsumerThreads) p.part_meta[b] = pre_s[b];
+    if (tid == 0) p.part_meta[p.g.batch + 1] = (int)(gridDim.x / p.team_size);
+  }
   consumer_sync();
 
-  for (int i = first; i < total_items; i += stride, ++n_item) {
-    const Item w = get_item(i, total_items, pre_s, len_s, p);
+  Cursor cur = c_first;
+  for (;; ++n_item) {
+    const Item w = piece_at(cur, x_end, pre_s, len_s, p);
+    if (!w.valid) break;
+    cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
     const int n_new = w.has_new ? 1 : 0;
     bool ok = true;
@@ -525,7 +584,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
     // query rows of the next item travel while the V tiles stream
     uint32_t qnext[4];
-    load_q_words(get_item(i + stride, total_items, pre_s, len_s, p), qnext);
+    load_q_words(piece_at(cur, x_end, pre_s, len_s, p), qnext);
 
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
     // A = the warp's 16 token rows transposed (16 channels x 16 tokens per m tile), B = the rows'
@@ -666,7 +725,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     for (int r = 0; r < rows; ++r) {
       const int set_r = nslots == 2 ? r / p.nq : 0;
       const int rq = r - set_r * p.nq;
-      const size_t prow = (((size_t)set_r * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.n_splits + w.split;
+      const size_t prow = (((size_t)set_r * p.g.batch + w.b) * p.n_q_heads + w.g * p.nq + rq) * p.slots + w.split;
       const float* sl = S + r * kSlabStride + tid;
       const int ws = rows * kSlabStride;
       p.part_o[prow * kHeadDim + tid] = (sl[0] + sl[ws]) + (sl[2 * ws] + sl[3 * ws]);
@@ -691,11 +750,28 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   }
 }
 
-// Log-sum-exp merge of the split partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
-// One block per output row; eight groups of 32 lanes share the splits (a lane owns four channels),
-// so a row with many splits is a few loads deep, not one load per split.
+// Log-sum-exp merge of the pieces' partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
+// One block per output row.  The pieces of its (sequence, kv head) are found from the numbers the
+// split kernel left in part_meta (unit prefix, number of teams): they start where the sequence
+// starts, at every team boundary inside it, and every cap_units from there.  Eight groups of 32
+// lanes share the pieces (a lane owns four channels).
 constexpr int kCombineThreads = 256;
 constexpr int kCombineGroups = kCombineThreads / 32;
+
+// Calls f(slot, ordinal) for every piece of the units [x0, x0 + u) in order.
+template <typename F>
+__device__ __forceinline__ void for_each_piece(long long x0, int u, long long n_units, int grid, int cap, F f) {
+  long long c = ((x0 + 1) * grid - 1) / n_units;  // the team whose range holds unit x0
+  long long s = x0;
+  int ord = 0;
+  while (s < x0 + u) {
+    const long long e = min(x0 + u, n_units * (c + 1) / grid);
+    for (long long x = s; x < e; x += cap) f((int)(x - x0), ord++);
+    s = e;
+    ++c;
+  }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
   grid_dep_wait();
@@ -704,13 +780,18 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   __shared__ float4 acc_s[kCombineGroups][32];
   const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
   const int tid = threadIdx.x, grp = tid >> 5, lane = tid & 31;
-  const int n = p.g.seq_lens[b];
-  const int nsp = max(1, (n + p.split_len - 1) / p.split_len);
-  const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.n_splits;
+  const int pre_b = p.part_meta[b], u = p.part_meta[b + 1] - pre_b;
+  const long long n_units = p.part_meta[p.g.batch];
+  const int grid = p.part_meta[p.g.batch + 1];  // teams
+  const long long x0 = pre_b;
+  const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.slots;
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
-  // M = max_j m_j
+  const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
+  // M = max_j m_j (every thread walks the piece list; it is short)
   float M = -INFINITY;
-  for (int j = tid; j < nsp; j += kCombineThreads) M = fmaxf(M, ml[j].x);
+  for_each_piece(x0, u, n_units, grid, p.cap_units, [&](int slot, int ord) {
+    if ((ord & (kCombineThreads - 1)) == tid) M = fmaxf(M, ml[slot].x);
+  });
   for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   if (lane == 0) red[grp] = M;
   __syncthreads();
@@ -718,27 +799,22 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
 #pragma unroll
   for (int g = 1; g < kCombineGroups; ++g) M = fmaxf(M, red[g]);
   __syncthreads();
-  // L = sum_j w_j l_j
+  // L = sum_j w_j l_j and o = sum_j w_j o_j: group grp takes the pieces grp, grp + 8, ...
   float L = 0.f;
-  for (int j = tid; j < nsp; j += kCombineThreads) {
-    const float2 v = ml[j];
-    L = fmaf(v.x == -INFINITY ? 0.f : exp2f(v.x - M), v.y, L);
-  }
-  for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-  if (lane == 0) red[grp] = L;
-  // o = sum_j w_j o_j: group grp takes the splits grp, grp + 8, ...
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-  const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
-#pragma unroll 4
-  for (int j = grp; j < nsp; j += kCombineGroups) {
-    const float m = ml[j].x;
-    const float w = m == -INFINITY ? 0.f : exp2f(m - M);
-    const float4 v = po[(size_t)j * (kHeadDim / 4)];
-    o.x = fmaf(w, v.x, o.x);
-    o.y = fmaf(w, v.y, o.y);
-    o.z = fmaf(w, v.z, o.z);
-    o.w = fmaf(w, v.w, o.w);
-  }
+  for_each_piece(x0, u, n_units, grid, p.cap_units, [&](int slot, int ord) {
+    if ((ord & (kCombineGroups - 1)) == grp) {
+      const float2 v2 = ml[slot];
+      const float w = v2.x == -INFINITY ? 0.f : exp2f(v2.x - M);
+      const float4 v = po[(size_t)slot * (kHeadDim / 4)];
+      L = fmaf(w, v2.y, L);
+      o.x = fmaf(w, v.x, o.x);
+      o.y = fmaf(w, v.y, o.y);
+      o.z = fmaf(w, v.z, o.z);
+      o.w = fmaf(w, v.w, o.w);
+    }
+  });
+  if (lane == 0) red[grp] = L;
   acc_s[grp][lane] = o;
   __syncthreads();
   if (grp == 0) {
@@ -763,37 +839,20 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-// Split length: the candidate that minimises rounds of the persistent grid x (tokens + fixed cost).
-static int pick_split_len(const mc_config* cfg, const mc_batch* bt) {
-  const long long per_split = (long long)bt->batch * cfg->n_kv_heads;
-  const int slots = 148 * kCtasPerSm;
-  int best = 128;
-  double best_cost = 1e300;
-  for (int len = 128; len <= kMaxSplit; len <<= 1) {
-    const long long items = per_split * std::max(1, (bt->max_seq_len + len - 1) / len);
-    const double rounds = (double)((items + slots - 1) / slots);
-    const double cost = rounds * (std::min(len, std::max(bt->max_seq_len, 1)) + 40.0);
-    if (cost < best_cost * 0.999) {
-      best_cost = cost;
-      best = len;
-    }
-  }
-  return best;
-}
-
-static size_t attn_smem_bytes(int split_len) {
-  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)s_region_floats(split_len) * 4;  // stages, S
-  b += 2 * kMaxRows * 64 * 4;                                                                // q_s
-  b += kMaxRows * 4 + 3 * kMaxRows * kConsumerWarps * 4;                                     // m, l, red, red2
-  b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 4 + 8 + 2 * kStages * 8 + 64;
+static size_t attn_smem_bytes() {
+  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kScoreFloats * 4;  // stages, S
+  b += 2 * kMaxRows * 64 * 4;                                                  // q_s
+  b += kMaxRows * 4 + 3 * kMaxRows * kConsumerWarps * 4;                       // m, l, red, red2
+  b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 2 * kMaxPiecePages * 4 + 4 + 8 + 2 * kStages * 8 + 64;
   return b;
 }
 
+// Partial slots per output row: the units of the longest sequence.
+static size_t attn_slots(const mc_batch* bt) { return (size_t)std::max(1, (bt->max_seq_len + kUnit - 1) / kUnit); }
+
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets) {
-  const int split_len = pick_split_len(cfg, bt);
-  const size_t n_splits = (size_t)std::max(1, (bt->max_seq_len + split_len - 1) / split_len);
-  const size_t prow = (size_t)n_sets * bt->batch * cfg->n_q_heads * n_splits;
-  return align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256);
+  const size_t prow = (size_t)n_sets * bt->batch * cfg->n_q_heads * attn_slots(bt);
+  return align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256) + align_up(((size_t)bt->batch + 2) * 4, 256);
 }
 
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
@@ -822,11 +881,12 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.nq = cfg->n_q_heads / cfg->n_kv_heads;
   ap.rows = ap.n_sets * ap.nq;
   ap.n_q_heads = cfg->n_q_heads;
-  ap.split_len = pick_split_len(cfg, bt);
-  ap.n_splits = std::max(1, (bt->max_seq_len + ap.split_len - 1) / ap.split_len);
-  const size_t prow = (size_t)ap.n_sets * bt->batch * cfg->n_q_heads * ap.n_splits;
+  ap.cap_units = piece_cap_units(ap.rows);
+  ap.slots = (int)attn_slots(bt);
+  const size_t prow = (size_t)ap.n_sets * bt->batch * cfg->n_q_heads * ap.slots;
   ap.part_o = reinterpret_cast<float*>(workspace);
   ap.part_ml = reinterpret_cast<float*>((char*)workspace + align_up(prow * kHeadDim * 4, 256));
+  ap.part_meta = reinterpret_cast<int32_t*>((char*)workspace + align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256));
 
   static int n_sm = 0;  // persistent grid: kCtasPerSm CTAs per SM of the current device
   if (n_sm == 0) {
@@ -834,9 +894,15 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
     MC_CUDA_CHECK(cudaGetDevice(&dev));
     MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
   }
-  const long long max_items = (long long)bt->batch * ap.n_splits * cfg->n_kv_heads;
-  const int grid = (int)std::min<long long>((long long)n_sm * kCtasPerSm, std::max<long long>(max_items, 1));
-  const size_t smem = attn_smem_bytes(ap.split_len);
+  // teams: S CTAs, each with ceil(H / S) kv heads; as many whole teams as fit two CTAs per SM,
+  // and no more teams than there can be units
+  const int slots_gpu = n_sm * kCtasPerSm;
+  const int heads_per_cta = (cfg->n_kv_heads + std::min(slots_gpu, 32) - 1) / std::min(slots_gpu, 32);
+  ap.team_size = (cfg->n_kv_heads + heads_per_cta - 1) / heads_per_cta;
+  const long long max_units = (long long)bt->batch * ap.slots;
+  const int n_teams = (int)std::max<long long>(1, std::min<long long>(slots_gpu / ap.team_size, max_units));
+  const int grid = n_teams * ap.team_size;
+  const size_t smem = attn_smem_bytes();
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
