@@ -751,47 +751,66 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 }
 
 // Log-sum-exp merge of the pieces' partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
-// One block per output row.  The pieces of its (sequence, kv head) are found from the numbers the
-// split kernel left in part_meta (unit prefix, number of teams): they start where the sequence
-// starts, at every team boundary inside it, and every cap_units from there.  Eight groups of 32
-// lanes share the pieces (a lane owns four channels).
+// One block per output row.  The pieces of its sequence are found from the numbers the split kernel
+// left in part_meta (unit prefix, number of teams): they start where the sequence starts, at every
+// team boundary inside it, and every cap_units from there.  A thread per team that touches the
+// sequence counts that team's pieces, a scan turns the counts into a list of slots in shared memory;
+// then eight groups of 32 lanes share the pieces (a lane owns four channels), four loads in flight.
 constexpr int kCombineThreads = 256;
 constexpr int kCombineGroups = kCombineThreads / 32;
-
-// Calls f(slot, ordinal) for every piece of the units [x0, x0 + u) in order.
-template <typename F>
-__device__ __forceinline__ void for_each_piece(long long x0, int u, long long n_units, int grid, int cap, F f) {
-  long long c = ((x0 + 1) * grid - 1) / n_units;  // the team whose range holds unit x0
-  long long s = x0;
-  int ord = 0;
-  while (s < x0 + u) {
-    const long long e = min(x0 + u, n_units * (c + 1) / grid);
-    for (long long x = s; x < e; x += cap) f((int)(x - x0), ord++);
-    s = e;
-    ++c;
-  }
-}
+constexpr int kMaxPieces = 2048;  // pieces of one sequence (checked on the host)
 
 template <int DT>
 __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
-  grid_dep_wait();
   grid_dep_launch();
   __shared__ float red[kCombineGroups];
+  __shared__ int scan_s[kCombineGroups];
+  __shared__ int total_s;
   __shared__ float4 acc_s[kCombineGroups][32];
+  __shared__ int list_s[kMaxPieces];
   const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
   const int tid = threadIdx.x, grp = tid >> 5, lane = tid & 31;
+  grid_dep_wait();
   const int pre_b = p.part_meta[b], u = p.part_meta[b + 1] - pre_b;
   const long long n_units = p.part_meta[p.g.batch];
-  const int grid = p.part_meta[p.g.batch + 1];  // teams
+  const int n_teams = p.part_meta[p.g.batch + 1];
   const long long x0 = pre_b;
+  // ---- the list of slots
+  const int c_first = (int)(((x0 + 1) * n_teams - 1) / n_units);  // the team whose range holds the first unit
+  const int c_last = (int)(((x0 + u) * n_teams - 1) / n_units);   // ... the last unit
+  const int cap = p.cap_units;
+  int base = 0;
+  for (int c0 = c_first; c0 <= c_last; c0 += kCombineThreads) {  // (more teams than threads: one more round)
+    const int c = c0 + tid;
+    int s = 0, cnt = 0;
+    if (c <= c_last) {
+      const long long lo = max(x0, n_units * c / n_teams), hi = min(x0 + u, n_units * (c + 1) / n_teams);
+      s = (int)(lo - x0);
+      cnt = hi > lo ? (int)((hi - lo + cap - 1) / cap) : 0;
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) scan_s[grp] = incl;
+    __syncthreads();
+    int off = base + incl - cnt;
+    for (int g = 0; g < grp; ++g) off += scan_s[g];
+    for (int k = 0; k < cnt; ++k)
+      if (off + k < kMaxPieces) list_s[off + k] = s + k * cap;
+    if (tid == kCombineThreads - 1) total_s = off + cnt;
+    __syncthreads();
+    base = total_s;
+  }
+  const int n = min(base, kMaxPieces);
   const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.slots;
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
   const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
-  // M = max_j m_j (every thread walks the piece list; it is short)
+  // ---- M = max_j m_j
   float M = -INFINITY;
-  for_each_piece(x0, u, n_units, grid, p.cap_units, [&](int slot, int ord) {
-    if ((ord & (kCombineThreads - 1)) == tid) M = fmaxf(M, ml[slot].x);
-  });
+  for (int j = tid; j < n; j += kCombineThreads) M = fmaxf(M, ml[list_s[j]].x);
   for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   if (lane == 0) red[grp] = M;
   __syncthreads();
@@ -799,21 +818,33 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
 #pragma unroll
   for (int g = 1; g < kCombineGroups; ++g) M = fmaxf(M, red[g]);
   __syncthreads();
-  // L = sum_j w_j l_j and o = sum_j w_j o_j: group grp takes the pieces grp, grp + 8, ...
+  // ---- L = sum_j w_j l_j and o = sum_j w_j o_j: group grp takes the pieces grp, grp + 8, ...
   float L = 0.f;
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-  for_each_piece(x0, u, n_units, grid, p.cap_units, [&](int slot, int ord) {
-    if ((ord & (kCombineGroups - 1)) == grp) {
-      const float2 v2 = ml[slot];
-      const float w = v2.x == -INFINITY ? 0.f : exp2f(v2.x - M);
-      const float4 v = po[(size_t)slot * (kHeadDim / 4)];
-      L = fmaf(w, v2.y, L);
-      o.x = fmaf(w, v.x, o.x);
-      o.y = fmaf(w, v.y, o.y);
-      o.z = fmaf(w, v.z, o.z);
-      o.w = fmaf(w, v.w, o.w);
+  for (int j0 = grp; j0 < n; j0 += 4 * kCombineGroups) {
+    float2 v2[4];
+    float4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int j = j0 + k * kCombineGroups;
+      v2[k] = make_float2(-INFINITY, 0.f);
+      v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j < n) {
+        const int slot = list_s[j];
+        v2[k] = ml[slot];
+        v[k] = po[(size_t)slot * (kHeadDim / 4)];
+      }
     }
-  });
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float w = v2[k].x == -INFINITY ? 0.f : exp2f(v2[k].x - M);
+      L = fmaf(w, v2[k].y, L);
+      o.x = fmaf(w, v[k].x, o.x);
+      o.y = fmaf(w, v[k].y, o.y);
+      o.z = fmaf(w, v[k].z, o.z);
+      o.w = fmaf(w, v[k].w, o.w);
+    }
+  }
   if (lane == 0) red[grp] = L;
   acc_s[grp][lane] = o;
   __syncthreads();
@@ -902,6 +933,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const long long max_units = (long long)bt->batch * ap.slots;
   const int n_teams = (int)std::max<long long>(1, std::min<long long>(slots_gpu / ap.team_size, max_units));
   const int grid = n_teams * ap.team_size;
+  if ((ap.slots + ap.cap_units - 1) / ap.cap_units + n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
   const size_t smem = attn_smem_bytes();
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
