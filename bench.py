@@ -211,7 +211,7 @@ class Job:
 
     def decode_pair_all(self, steps):
         """Pair mode: both layers of a pair in one call (two query sets, one pass over the directions)."""
-        if not hasattr(self, "ws_attn2"):
+        if steps == 0 or not hasattr(self, "ws_attn2"):  # steps == 0: set up the buffers only (outside any timed region)
             bd = self.batch(True)
             self.ws_attn2 = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bd, 1, 2), dtype=torch.uint8, device=self.dev)
             self.out2 = torch.empty(2, self.B, self.Hq, 128, dtype=self.cfg.torch_dtype, device=self.dev)
@@ -416,8 +416,11 @@ def main():
     if 2 * (wl.n_q_heads // wl.n_kv_heads) <= 8:
         # pair mode (both layers' queries known up front: a replay or speculative setting, not a real
         # model's layer-by-layer decode): the shared directions are read once for two layers
+        job.decode_pair_all(0)
         job.merge_all()
         psteps = min(job.steps, 64)
+        job.decode_pair_all(min(2, psteps))  # warm-up
+        job.merge_all()
         t_p = timed(lambda: job.decode_pair_all(psteps))
         th_steps = psteps * job.tok_heads + job.B * job.H * psteps * (psteps - 1) // 2
         pair_bytes = wl.n_pairs * th_steps * (2 * ROW + 16 + 4 * rho * (ROW + 4)) + by["append"] * psteps / job.steps

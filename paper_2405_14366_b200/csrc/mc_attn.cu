@@ -59,7 +59,6 @@ struct AttnParams {
   const char* v_new;
   float* part_o;   // [n_sets][batch][Hq][slots][128]: a piece's partial sits in the slot of its first unit
   float* part_ml;  // [n_sets][batch][Hq][slots][2]
-  int32_t* part_meta;  // [batch + 2]: prefix of the sequences' unit counts, then the split kernel's grid size
   int32_t* status;
   float scale_log2;  // sm_scale * log2(e)
   int layer_sel;
@@ -70,6 +69,7 @@ struct AttnParams {
   int cap_units;  // longest piece, in units of 128 tokens (what the score buffer holds for `rows` rows)
   int slots;      // partial slots per output row = units of the longest sequence
   int team_size;  // CTAs per team (one or more kv heads each)
+  int n_teams;
 };
 
 // ---- PTX wrappers (tensor-core side; the copy/barrier wrappers live in mc_pipe.cuh) ---------------
@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     pre_s[p.g.batch] = acc;
   }
   __syncthreads();
-  const int n_teams = gridDim.x / p.team_size;
+  const int n_teams = p.n_teams;
   const int team = blockIdx.x / p.team_size;
   const long long n_units = pre_s[p.g.batch];
   const int x_begin = (int)(n_units * team / n_teams), x_end = (int)(n_units * (team + 1) / n_teams);
@@ -436,10 +436,6 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
   grid_dep_wait();
-  if (blockIdx.x == 0) {  // the combine kernel finds the pieces from the same numbers
-    for (int b = tid; b <= p.g.batch; b += kConsumerThreads) p.part_meta[b] = pre_s[b];
-    if (tid == 0) p.part_meta[p.g.batch + 1] = (int)(gridDim.x / p.team_size);
-  }
   consumer_sync();
 
   Cursor cur = c_first;
@@ -751,9 +747,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 }
 
 // Log-sum-exp merge of the pieces' partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
-// One block per output row.  The pieces of its sequence are found from the numbers the split kernel
-// left in part_meta (unit prefix, number of teams): they start where the sequence starts, at every
-// team boundary inside it, and every cap_units from there.  A thread per team that touches the
+// One block per output row.  The pieces of its sequence follow from the lengths and the number of
+// teams: they start where the sequence starts, at every team boundary inside it, and every
+// cap_units from there.  A thread per team that touches the
 // sequence counts that team's pieces, a scan turns the counts into a list of slots in shared memory;
 // then eight groups of 32 lanes share the pieces (a lane owns four channels), four loads in flight.
 constexpr int kCombineThreads = 256;
@@ -770,10 +766,34 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   __shared__ int list_s[kMaxPieces];
   const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
   const int tid = threadIdx.x, grp = tid >> 5, lane = tid & 31;
-  grid_dep_wait();
-  const int pre_b = p.part_meta[b], u = p.part_meta[b + 1] - pre_b;
-  const long long n_units = p.part_meta[p.g.batch];
-  const int n_teams = p.part_meta[p.g.batch + 1];
+  // The lengths belong to the caller (no kernel of this library writes them): the piece list is
+  // built before the wait on the split kernel, whose tail it overlaps.
+  int before = 0, all = 0;  // units of the sequences before this one, of all sequences
+  for (int bb = tid; bb < p.g.batch; bb += kCombineThreads) {
+    const int ub = max(1, (p.g.seq_lens[bb] + kUnit - 1) / kUnit);
+    all += ub;
+    if (bb < b) before += ub;
+  }
+  for (int o = 16; o; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    all += __shfl_xor_sync(0xffffffffu, all, o);
+  }
+  if (lane == 0) {
+    scan_s[grp] = before;
+    red[grp] = __int_as_float(all);
+  }
+  __syncthreads();
+  before = 0;
+  all = 0;
+#pragma unroll
+  for (int g = 0; g < kCombineGroups; ++g) {
+    before += scan_s[g];
+    all += __float_as_int(red[g]);
+  }
+  __syncthreads();
+  const int pre_b = before, u = max(1, (p.g.seq_lens[b] + kUnit - 1) / kUnit);
+  const long long n_units = all;
+  const int n_teams = p.n_teams;
   const long long x0 = pre_b;
   // ---- the list of slots
   const int c_first = (int)(((x0 + 1) * n_teams - 1) / n_units);  // the team whose range holds the first unit
@@ -805,6 +825,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
     base = total_s;
   }
   const int n = min(base, kMaxPieces);
+  grid_dep_wait();
   const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.slots;
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
   const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
@@ -883,7 +904,7 @@ static size_t attn_slots(const mc_batch* bt) { return (size_t)std::max(1, (bt->m
 
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets) {
   const size_t prow = (size_t)n_sets * bt->batch * cfg->n_q_heads * attn_slots(bt);
-  return align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256) + align_up(((size_t)bt->batch + 2) * 4, 256);
+  return align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256);
 }
 
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
@@ -917,7 +938,6 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const size_t prow = (size_t)ap.n_sets * bt->batch * cfg->n_q_heads * ap.slots;
   ap.part_o = reinterpret_cast<float*>(workspace);
   ap.part_ml = reinterpret_cast<float*>((char*)workspace + align_up(prow * kHeadDim * 4, 256));
-  ap.part_meta = reinterpret_cast<int32_t*>((char*)workspace + align_up(prow * kHeadDim * 4, 256) + align_up(prow * 2 * 4, 256));
 
   static int n_sm = 0;  // persistent grid: kCtasPerSm CTAs per SM of the current device
   if (n_sm == 0) {
@@ -933,6 +953,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const long long max_units = (long long)bt->batch * ap.slots;
   const int n_teams = (int)std::max<long long>(1, std::min<long long>(slots_gpu / ap.team_size, max_units));
   const int grid = n_teams * ap.team_size;
+  ap.n_teams = n_teams;
   if ((ap.slots + ap.cap_units - 1) / ap.cap_units + n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
   const size_t smem = attn_smem_bytes();
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
