@@ -34,9 +34,9 @@ import gen  # noqa: E402
 
 ROW = 256  # bytes of one 16-bit row of 128 channels
 # DRAM bytes (read + written) per algorithmic byte of the split attention kernel, from the ncu capture
-# summarised in profiles/attn_split_kernel_c2_one_pair.md (563.3 MB for 547.8 MB).  Set to None when
+# summarised in profiles/attn_split_kernel_c2_one_pair.md (565.4 MB for 547.4 MB).  Set to None when
 # the kernel changes until it is captured again.
-ATTN_TRAFFIC_RATIO = 1.028
+ATTN_TRAFFIC_RATIO = 1.033
 
 
 # ---------------------------------------------------------------------------------------------
@@ -253,6 +253,21 @@ class Job:
         return th * (2 * ROW + 8 + 2 * rho * (ROW + 4))
 
 
+def max_over_ranks(seconds: float, dist, device) -> float:
+    """The slowest rank's time: what a job of independent replicas takes (`dist` None = one rank)."""
+    if dist is None:
+        return seconds
+    tt = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_gbps(bytes_per_step_per_rank: float, steps: int, seconds: float, world: int) -> float:
+    """Weak scaling: every rank runs the same workload on its own data; all ranks' bytes over the
+    slowest rank's time."""
+    return world * bytes_per_step_per_rank * steps / seconds / 1e9
+
+
 def timed(fn, stream_sync=True):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -380,15 +395,12 @@ def main():
     if dist is not None:
         dist.barrier()
     t_total = timed(lambda: [job.step(sample_events=True) for _ in range(args.steps)])
-    if dist is not None:
-        tt = torch.tensor([t_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_total = float(tt.item())
+    t_total = max_over_ranks(t_total, dist, dev)
     clocks = sampler.stop() if sampler else None
     launches = job.launches
     by = job.bytes_per_step(rho)
     bytes_step = sum(by.values())
-    value = world * bytes_step * args.steps / t_total / 1e9
+    value = whole_job_gbps(bytes_step, args.steps, t_total, world)
 
     # dominant kernel: split attention (+ its small combine), sampled with CUDA events in the timed region
     ev_ms = [(e0.elapsed_time(e1), s) for e0, e1, s in job.attn_events]
@@ -514,13 +526,10 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
         dist.barrier()
     n = max(1, min(args.steps, 2))
     t = timed(lambda: [e2e_step() for _ in range(n)])
-    if dist is not None:
-        tt = torch.tensor([t], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t = float(tt.item())
+    t = max_over_ranks(t, dist, dev)
     by = job.bytes_per_step(rho)
     calls = job.steps * wl.n_pairs * 2
-    return {"value": world * sum(by.values()) * n / t / 1e9, "unit": "GB/s", "steps": n, "ms_per_step": t / n * 1e3,
+    return {"value": whole_job_gbps(sum(by.values()), n, t, world), "unit": "GB/s", "steps": n, "ms_per_step": t / n * 1e3,
             "h2d_bytes_per_step": wl.n_pairs * pool_bytes + calls * (q_bytes + 2 * n_bytes),
             "d2h_bytes_per_step": calls * q_bytes,
             "api": "mc_merge_pair_host + mc_restore + mc_decode_attn_host + mc_append_pair, pinned host buffers"}
