@@ -73,6 +73,15 @@ typedef enum { MC_LAYER_LM1 = 0, MC_LAYER_L = 1, MC_LAYER_BOTH = 2 } mc_layer_se
 /* Operations whose scratch need mc_workspace_bytes reports. */
 typedef enum { MC_OP_MERGE = 0, MC_OP_DECODE_ATTN = 1 } mc_op;
 
+/* The merge function.  MC_MERGE_SLERP is the method (Eq. 3, both magnitudes kept).  The other two
+ * are the alternatives the paper compares it with: they merge the two rows into ONE vector that
+ * stands for both layers -- MC_MERGE_FMAX the direction of the mean times the larger of the two
+ * magnitudes (Appendix, "maximum norm-preserving interpolation"), MC_MERGE_MEAN the plain average
+ * (Sec. 3.1) -- stored in the same format (direction, the one magnitude for both layers), so restore
+ * and attention do not change.  The angular distance and the retention are the same for all three;
+ * t is used by MC_MERGE_SLERP only. */
+typedef enum mc_merge_fn { MC_MERGE_SLERP = 0, MC_MERGE_FMAX = 1, MC_MERGE_MEAN = 2 } mc_merge_fn;
+
 /* Status word indices (mc_read_status). */
 enum {
   MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out */
@@ -94,6 +103,8 @@ typedef struct mc_config {
   int32_t retain_mode; /* mc_retain_mode */
   double t;            /* interpolation parameter of Eq. 3: 0 -> direction of layer l-1, 1 -> of layer l */
   double gamma;        /* retention threshold of Eq. 4 */
+  int32_t merge_fn;    /* mc_merge_fn: how the two rows of a token become the shared row */
+  int32_t reserved;    /* must be 0 */
 } mc_config;
 
 /* Batch geometry shared by the layer pools and the pair cache. */

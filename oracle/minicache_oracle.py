@@ -200,7 +200,7 @@ def retention_indices(d: np.ndarray, gamma: float, mode: str = "distinct") -> np
 # --------------------------------------------------------------------------
 def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[int], dtype: str,
                t: float, gamma: float, mode: str = "distinct", convention: str = "eq3",
-               do_retention: bool = True) -> Dict[str, object]:
+               do_retention: bool = True, merge_fn: str = "slerp") -> Dict[str, object]:
     """Compress one tensor (K or V) of a layer pair.
 
     x_*_bits: uint16 [B][S][H][D] logical rows (layer l-1, layer l).
@@ -208,14 +208,26 @@ def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[
     n_l, d [B][S][H] (float64), ``retained``: dict (b, h) -> ascending indices.
     The retained raw rows are the input bits at those indices."""
     return merge_pair_values(decode_bits(x_lm1_bits, dtype), decode_bits(x_l_bits, dtype), seq_lens, dtype, t, gamma,
-                             mode, convention, do_retention)
+                             mode, convention, do_retention, merge_fn)
 
 
 def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dtype: str, t: float, gamma: float,
-                      mode: str = "distinct", convention: str = "eq3", do_retention: bool = True) -> Dict[str, object]:
+                      mode: str = "distinct", convention: str = "eq3", do_retention: bool = True,
+                      merge_fn: str = "slerp") -> Dict[str, object]:
     """``merge_pair`` on rows given as float64 values (e.g. de-quantised 4-bit layers); `dtype` is
-    the storage type of the merged direction."""
+    the storage type of the merged direction.
+
+    merge_fn "slerp" is Eq. 3 with both magnitudes kept.  "fmax" (Eq. A) and "mean" (the averaging
+    baseline of Sec. 3.1) merge the two rows into ONE vector M that stands for both layers: the
+    stored direction is M / |M| and both layers' magnitudes are |M|.  The angular distance that
+    drives the retention (Eq. 4) is the same in all three."""
     m = merge_rows(a, c, t, convention)
+    if merge_fn != "slerp":
+        M = {"fmax": merge_rows_fmax, "mean": merge_rows_mean}[merge_fn](a, c)
+        n_m = np.sqrt(np.sum(M * M, axis=-1))
+        m["e"] = M / np.where(n_m == 0.0, 1.0, n_m)[..., None]
+        m["n_a"] = n_m
+        m["n_c"] = n_m
     e_bits = store_direction(m["e"], dtype)
     B, S, H, _ = a.shape
     retained = {}
@@ -231,9 +243,16 @@ def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dty
 
 
 def append_rows(a_bits: np.ndarray, c_bits: np.ndarray, dtype: str, t: float,
-                convention: str = "eq3") -> Dict[str, np.ndarray]:
+                convention: str = "eq3", merge_fn: str = "slerp") -> Dict[str, np.ndarray]:
     """Merge the decode step's new token pair (no retention decision for it)."""
-    m = merge_rows(decode_bits(a_bits, dtype), decode_bits(c_bits, dtype), t, convention)
+    a, c = decode_bits(a_bits, dtype), decode_bits(c_bits, dtype)
+    m = merge_rows(a, c, t, convention)
+    if merge_fn != "slerp":  # see merge_pair_values
+        M = {"fmax": merge_rows_fmax, "mean": merge_rows_mean}[merge_fn](a, c)
+        n_m = np.sqrt(np.sum(M * M, axis=-1))
+        m["e"] = M / np.where(n_m == 0.0, 1.0, n_m)[..., None]
+        m["n_a"] = n_m
+        m["n_c"] = n_m
     m["e_bits"] = store_direction(m["e"], dtype)
     return m
 

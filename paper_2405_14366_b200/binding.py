@@ -32,7 +32,7 @@ class McError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("page_size", C.c_int32), ("dtype", C.c_int32), ("retain_mode", C.c_int32),
-                ("t", C.c_double), ("gamma", C.c_double)]
+                ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _Batch(C.Structure):
@@ -82,10 +82,12 @@ class McConfig:
     gamma: float = 0.05
     retain_mode: int = MC_RETAIN_DISTINCT
     head_dim: int = 128
+    merge_fn: int = 0  # MC_MERGE_SLERP (Eq. 3) | MC_MERGE_FMAX = 1 | MC_MERGE_MEAN = 2
 
     def c(self) -> _Config:
         return _Config(self.n_kv_heads, self.n_q_heads, self.head_dim, self.page_size,
-                       {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma))
+                       {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma),
+                       int(self.merge_fn), 0)
 
     @property
     def torch_dtype(self):

@@ -25,6 +25,7 @@ static mc_status check_config(const mc_config* cfg) {
   if (nq != 1 && nq != 2 && nq != 4 && nq != 8) return MC_ERR_SHAPE;
   if (cfg->dtype != MC_F16 && cfg->dtype != MC_BF16) return MC_ERR_DTYPE;
   if (cfg->retain_mode < MC_RETAIN_DISTINCT || cfg->retain_mode > MC_RETAIN_TOPK) return MC_ERR_INVALID_ARG;
+  if (cfg->merge_fn < MC_MERGE_SLERP || cfg->merge_fn > MC_MERGE_MEAN || cfg->reserved != 0) return MC_ERR_INVALID_ARG;
   if (!(cfg->t >= 0.0 && cfg->t <= 1.0) || !(cfg->gamma >= 0.0 && cfg->gamma <= 1.0)) return MC_ERR_INVALID_ARG;
   return MC_OK;
 }

@@ -33,13 +33,14 @@ struct MergeParams {
   float* dist;
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
   float ta, tc;
+  int merge_fn;
   int items_per_page;
   int32_t* status;
 };
 
 // One merged row: 16 lanes hold 8 channels each of a (layer l-1) and c (layer l).
 template <int DT>
-__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, uint4& e_out,
+__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, int fn, uint4& e_out,
                                           float& g_a, float& g_c, float& d_out) {
   float a[8], c[8];
   {
@@ -77,7 +78,19 @@ __device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, floa
   }
   sm = sum16(sm);
   sp = sum16(sp);
-  const RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
+  RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
+  if (fn != MC_MERGE_SLERP) {  // one vector for both layers: direction of the mean, one magnitude
+    float m2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float h = a[i] + c[i];
+      m2 = fmaf(h, h, m2);
+    }
+    m2 = 0.25f * sum16(m2);
+    const float im = m2 > 0.f ? rsqrtf(m2) : 0.f;
+    s.fa = s.fc = 0.5f * im;
+    s.na = s.nc = fn == MC_MERGE_FMAX ? fmaxf(s.na, s.nc) : m2 * im;
+  }
   uint32_t w[4];
   float ee = 0.f;
 #pragma unroll
@@ -124,7 +137,7 @@ __device__ __forceinline__ float sum4(float v) {
 // a (layer l-1) and c (layer l), 32 channels each.  Arithmetic in fp32, two channels per
 // instruction (packed f32x2).  Every lane of the quad returns the row's scalars.
 template <int DT>
-__device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const float2 (&c)[16], float ta, float tc,
+__device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const float2 (&c)[16], float ta, float tc, int fn,
                                                uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
   float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2, aa3 = aa2, cc3 = aa2;
 #pragma unroll
@@ -164,7 +177,19 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
     const float spx = sum4(sp2.x + sp2.y);
     if (sm > 3.5f) sp = spx;
   }
-  const RowScalars s = slerp_scalars(aa, cc, sm, fmaxf(sp, 0.f), ta, tc);
+  RowScalars s = slerp_scalars(aa, cc, sm, fmaxf(sp, 0.f), ta, tc);
+  if (fn != MC_MERGE_SLERP) {  // one vector for both layers: direction of the mean, one magnitude
+    float2 m2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float2 h = make_float2(a[i].x + c[i].x, a[i].y + c[i].y);
+      m2 = __ffma2_rn(h, h, m2);
+    }
+    const float mm = 0.25f * sum4(m2.x + m2.y);
+    const float im = mm > 0.f ? rsqrtf(mm) : 0.f;
+    s.fa = s.fc = 0.5f * im;
+    s.na = s.nc = fn == MC_MERGE_FMAX ? fmaxf(s.na, s.nc) : mm * im;
+  }
   const float2 fa2 = make_float2(s.fa, s.fa), fc2 = make_float2(s.fc, s.fc);
   float ee4[4] = {0.f, 0.f, 0.f, 0.f};
   uint32_t w[16];
@@ -193,7 +218,7 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
 // occupancy.  (Eight warps, not nine with a dedicated producer: two CTAs of nine warps do not fit
 // the register file of an SM sub-partition.)
 template <int DT>
-__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc,
+__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc, int fn,
                                                uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
   float2 a[16], c[16];
 #pragma unroll
@@ -207,7 +232,7 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
     c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
     c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
   }
-  merge_row_core<DT>(a, c, ta, tc, e_out, g_a, g_c, d_out);
+  merge_row_core<DT>(a, c, ta, tc, fn, e_out, g_a, g_c, d_out);
 }
 
 // 32 consecutive 4-bit codes (16 bytes; channel 2i in the low nibble of byte i) to values
@@ -362,7 +387,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
-      merge_row_quad<DT>(va, vc, p.ta, p.tc, e, g_a, g_c, d);
+      merge_row_quad<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, g_a, g_c, d);
     } else {
       // lane k owns channels [32 k, 32 k + 32): 16 bytes of codes = the 16-byte chunks 4 k .. 4 k + 3 of the output row
       const unsigned char* sb = stages + s * kMergeStageBytes;
@@ -383,7 +408,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       for (int x = 0; x < 4; ++x) ci[x] = 4 * k + x;
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
-      merge_row_core<DT>(a, c, p.ta, p.tc, e, g_a, g_c, d);
+      merge_row_core<DT>(a, c, p.ta, p.tc, p.merge_fn, e, g_a, g_c, d);
     }
     float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
@@ -811,6 +836,7 @@ struct AppendParams {
   char* e_pool[2];
   float* dist;
   float ta, tc;
+  int merge_fn;
   int total_rows;  // 2 * batch * H
 };
 
@@ -834,7 +860,7 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   }
   uint4 e;
   float ga, gc, d;
-  merge_row<DT>(va, vc, p.ta, p.tc, e, ga, gc, d);
+  merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, ga, gc, d);
   if (!ok) return;
   const int tok = p.g.seq_lens[b];
   const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
@@ -883,6 +909,7 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   mp.e_pool[1] = (char*)out->e_v;
   mp.dist = out->dist;
   mp.seg_minmax = reinterpret_cast<unsigned*>(out->seg_minmax);
+  mp.merge_fn = cfg->merge_fn;
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
@@ -962,6 +989,7 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   ap.e_pool[0] = (char*)pair->e_k;
   ap.e_pool[1] = (char*)pair->e_v;
   ap.dist = pair->dist;
+  ap.merge_fn = cfg->merge_fn;
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;
   ap.total_rows = 2 * bt->batch * cfg->n_kv_heads;

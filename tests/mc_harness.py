@@ -23,7 +23,7 @@ class Problem:
     def __init__(self, cfg: WorkloadConfig, pair: int = 0, device="cuda", seq_lens=None, gamma=None, t=None,
                  retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
                  tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None,
-                 q4: bool = False):
+                 q4: bool = False, merge_fn: str = "slerp"):
         import paper_2405_14366_b200 as mc
         self.mc = mc
         self.lib = mc.lib()
@@ -48,7 +48,9 @@ class Problem:
         self.block_table = torch.from_numpy(bt).to(device)
         self.seq_lens = torch.from_numpy(self.seq_lens_host.copy()).to(device)
         self.max_seq_len = int(self.seq_lens_host.max()) if B else 0
-        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode)
+        self.merge_fn = merge_fn
+        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode,
+                               merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn])
         self.pools = {}
         self.q4 = q4
         self.q4_pools: Dict[str, Dict[str, torch.Tensor]] = {}
@@ -162,10 +164,11 @@ class Problem:
         for ti, tn in enumerate(("k", "v")):
             if self.q4:
                 out[tn] = orc.merge_pair_values(self.values[tn + "_lm1"], self.values[tn + "_l"], self.seq_lens_host,
-                                                self.dtype, self.t, self.gamma, mode=mode, do_retention=do_retention)
+                                                self.dtype, self.t, self.gamma, mode=mode, do_retention=do_retention,
+                                                merge_fn=self.merge_fn)
                 continue
             out[tn] = orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype,
-                                     self.t, self.gamma, mode=mode, do_retention=do_retention)
+                                     self.t, self.gamma, mode=mode, do_retention=do_retention, merge_fn=self.merge_fn)
         return out
 
 

@@ -171,7 +171,8 @@ def test_append_then_attend(H):
         torch.cuda.synchronize()
         # oracle: append to its own logical cache
         for tn in ("k", "v"):
-            m = orc.append_rows(gen.as_bits(nt[tn + "_lm1"][:, 0]), gen.as_bits(nt[tn + "_l"][:, 0]), p.dtype, p.t)
+            m = orc.append_rows(gen.as_bits(nt[tn + "_lm1"][:, 0]), gen.as_bits(nt[tn + "_l"][:, 0]), p.dtype, p.t,
+                                merge_fn=p.merge_fn)
             o = om[tn]
             if o["e_bits"].shape[1] < p.S + step + 1:
                 padn = p.S + 8 - o["e_bits"].shape[1]
@@ -258,3 +259,31 @@ def test_q4_rejects_other_page_sizes(H):
     dummy = {k: ws for k in ("k_codes", "k_meta", "v_codes", "v_meta")}
     with pytest.raises(Exception):
         p.lib.mc_merge_pair_q4(p.cfg, p.batch(), dummy, dummy, p.pair, True, ws)
+
+
+@pytest.mark.parametrize("merge_fn", ["fmax", "mean"])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_merge_function_variants(H, merge_fn, dtype):
+    """The two merge functions the paper compares SLERP with (Appendix Eq. A; the averaging baseline of
+    Sec. 3.1), through the same kernels and the same cache format: merge, restore of both layers,
+    attention and an appended token against the oracle's variant."""
+    wl = dataclasses.replace(CONFIGS["c1"], dtype=dtype, n_kv_heads=4, n_q_heads=8, seq_len=336)
+    lens = np.array([333], np.int32)
+    p = H.Problem(wl, seq_lens=lens, merge_fn=merge_fn)
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge()
+    dc = p.device_cache()
+    stats = H.compare_merge(p, om, dc)
+    # one magnitude for both layers
+    assert np.array_equal(dc["scale"][..., 0], dc["scale"][..., 1]) and np.array_equal(dc["scale"][..., 2], dc["scale"][..., 3])
+    for layer in (0, 1):
+        dk, dv = p.run_restore(layer)
+        stats.update(H.compare_restore(p, om, dc, layer, dk, dv))
+    q = gen.make_queries(dataclasses.replace(wl, batch=p.B), 0, n_sets=2)
+    nt = gen.make_new_tokens(dataclasses.replace(wl, batch=p.B), 0, 0)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    out, lse = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
+    stats.update(H.compare_attention(p, om, 2, q, out.cpu(), lse.cpu(), kn, vn))
+    print(merge_fn, dtype, stats)

@@ -449,3 +449,58 @@ def test_input_quantiser_matches_oracle_quantiser():
         assert np.array_equal(full, codes)
         m = q["meta"].double().numpy()
         assert np.array_equal(m[..., 0], scale) and np.array_equal(m[..., 1], zero)
+
+
+def test_merge_function_variants_closed_forms():
+    """F_max (Appendix Eq. A) and the averaging baseline (Sec. 3.1) inside merge_pair: one vector M for
+    both layers, stored as direction and magnitude.  Closed forms for two rows of equal length r at an
+    angle w: mean = r cos(w/2) along the bisector, F_max = r along the bisector; and for parallel rows of
+    lengths 1 and 3: mean = 2, F_max = 3.  The distance (retention) does not depend on the merge function."""
+    D = 128
+    rs = np.random.RandomState(11)
+    g1 = rs.standard_normal(D); g1 /= np.linalg.norm(g1)
+    g2 = rs.standard_normal(D); g2 -= g1 * (g1 @ g2); g2 /= np.linalg.norm(g2)
+    w, r = 0.8, 2.5
+    a = r * g1
+    c = r * (math.cos(w) * g1 + math.sin(w) * g2)
+    bis = (g1 + math.cos(w) * g1 + math.sin(w) * g2); bis /= np.linalg.norm(bis)
+    A = np.stack([a, g1])[None, :, None, :]        # [B=1][S=2][H=1][D]
+    Cc = np.stack([c, 3.0 * g1])[None, :, None, :]
+    ref = orc.merge_pair_values(A, Cc, [2], "f16", 0.6, 0.05)
+    for fn, n0, n1 in (("mean", r * math.cos(w / 2), 2.0), ("fmax", r, 3.0)):
+        m = orc.merge_pair_values(A, Cc, [2], "f16", 0.6, 0.05, merge_fn=fn)
+        assert np.allclose(m["e"][0, 0, 0], bis, atol=1e-12) and np.allclose(m["e"][0, 1, 0], g1, atol=1e-12)
+        assert np.allclose(m["n_lm1"][0, :, 0], [n0, n1], atol=1e-12) and np.array_equal(m["n_lm1"], m["n_l"])
+        assert np.array_equal(m["d"], ref["d"]) and np.allclose(m["d"][0, 0, 0], w / math.pi, atol=1e-12)
+        # restore gives M itself for both layers (up to the 16-bit storage of the direction)
+        x = orc.restore(m["e_bits"][0, :, 0], m["n_l"][0, :, 0], "f16")
+        assert np.allclose(x[0], n0 * bis, atol=2e-3 * n0) and np.allclose(x[1], n1 * g1, atol=2e-3 * n1)
+    # SLERP keeps both magnitudes, the variants one
+    assert not np.array_equal(ref["n_lm1"], ref["n_l"])
+    # antipodal rows: the mean vanishes, nothing to restore
+    z = orc.merge_pair_values(a[None, None, None, :], -a[None, None, None, :], [1], "f16", 0.6, 0.05, merge_fn="fmax")
+    assert np.all(z["e"] == 0) and np.all(z["n_l"] == 0)
+
+
+def test_restore_error_of_the_merge_functions_on_the_synthetic_pair():
+    """The paper's comparison axis (Sec. 3.1, Appendix): how far the restored rows are from the original
+    ones for SLERP, F_max and the plain average, on the generator's row model (independent magnitudes,
+    planted angles), without retention.  Keeping both magnitudes and splitting the angle must beat one
+    shared vector."""
+    import dataclasses
+    from gen import workload as W
+    wl = dataclasses.replace(W.CONFIGS["c1"], seq_len=128, n_kv_heads=4, n_q_heads=4)
+    t = W.make_pair_tensors(wl, 0)
+    a, c = orc.decode_bits(W.as_bits(t["k_lm1"]), "f16"), orc.decode_bits(W.as_bits(t["k_l"]), "f16")
+    err = {}
+    for fn in ("slerp", "fmax", "mean"):
+        m = orc.merge_pair_values(a, c, [128], "f16", 0.6, 0.0, merge_fn=fn)
+        tot = []
+        for layer, (x, nm) in enumerate(((a, "n_lm1"), (c, "n_l"))):
+            for h in range(4):
+                xh = orc.restore(m["e_bits"][0, :, h], m[nm][0, :, h], "f16")
+                tot.append(np.linalg.norm(xh - x[0, :, h], axis=-1) / np.linalg.norm(x[0, :, h], axis=-1))
+        err[fn] = float(np.mean(tot))
+    print("mean relative restore error:", err)
+    assert err["slerp"] < err["fmax"] and err["slerp"] < err["mean"]
+    assert err["slerp"] < 0.25  # about half the mean planted angle (0.3 rad) plus outliers
