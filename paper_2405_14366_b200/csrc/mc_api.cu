@@ -218,6 +218,17 @@ mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const 
   return mc_merge_pair(cfg, batch, dev_lm1, dev_l, out, do_retention, workspace, workspace_bytes, stream);
 }
 
+// The device's address of pinned, device-addressable host memory; nullptr for anything else.
+static const void* device_view(const void* host_ptr) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) {
+    cudaGetLastError();  // pageable memory is reported as an error by older runtimes: not an error here
+    return nullptr;
+  }
+  if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return nullptr;
+  return a.devicePointer;
+}
+
 static void decode_io_layout(const mc_config* cfg, const mc_batch* bt, int n_sets, size_t off[6]) {
   const size_t qb = align_up((size_t)n_sets * bt->batch * cfg->n_q_heads * kRowBytes, 256);
   const size_t nb = align_up((size_t)n_sets * bt->batch * cfg->n_kv_heads * kRowBytes, 256);
@@ -260,6 +271,27 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
   cudaStream_t s = (cudaStream_t)stream;
   const size_t qb = (size_t)n_sets * batch->batch * cfg->n_q_heads * kRowBytes;
   const size_t nb = (size_t)n_sets * batch->batch * cfg->n_kv_heads * kRowBytes;
+  // Pinned host memory that the device can address (what cudaHostAlloc / cudaHostRegister give on a
+  // unified address space) is read and written by the kernels themselves: the queries by the
+  // attention kernel (prefetched a piece ahead), the new rows by one small copy kernel into the
+  // staging buffer, the result by the combine kernel.  No copy engine is involved, so these small
+  // transfers do not queue behind large uploads that may be running on another stream.  Any other
+  // host memory goes through asynchronous copies.
+  const void* q_dev = device_view(q_host);
+  const void* kn_dev = k_new_host ? device_view(k_new_host) : nullptr;
+  const void* vn_dev = v_new_host ? device_view(v_new_host) : nullptr;
+  void* out_dev = const_cast<void*>(device_view(out_host));
+  float* lse_dev = lse_host ? (float*)const_cast<void*>(device_view(lse_host)) : nullptr;
+  const bool direct = q_dev && out_dev && aligned256(q_dev) && aligned256(out_dev) && (!k_new_host || (kn_dev && vn_dev)) &&
+                      (!lse_host || lse_dev) && (nb % 16 == 0);
+  if (direct) {
+    if (k_new_host) {
+      st = launch_fetch_rows(kn_dev, vn_dev, io + off[1], io + off[2], nb, s);
+      if (st != MC_OK) return st;
+    }
+    return mc_decode_attn(cfg, batch, pair, layer_sel, q_dev, k_new_host ? io + off[1] : nullptr,
+                          k_new_host ? io + off[2] : nullptr, sm_scale, out_dev, lse_dev, workspace, workspace_bytes, stream);
+  }
   MC_CUDA_CHECK(cudaMemcpyAsync(io + off[0], q_host, qb, cudaMemcpyHostToDevice, s));
   if (k_new_host) {
     MC_CUDA_CHECK(cudaMemcpyAsync(io + off[1], k_new_host, nb, cudaMemcpyHostToDevice, s));

@@ -972,6 +972,32 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   return MC_OK;
 }
 
+// ---- new-token rows from device-addressable host memory ------------------------------------------
+__global__ void __launch_bounds__(256) fetch_rows_kernel(const uint4* k_src, const uint4* v_src, uint4* k_dst, uint4* v_dst,
+                                                         int n16) {
+  grid_dep_launch();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+  if (i < n16) {  // the caller's rows are read before the wait, the staging buffer written after it
+    a = k_src[i];
+    b = v_src[i];
+  }
+  grid_dep_wait();
+  if (i < n16) {
+    k_dst[i] = a;
+    v_dst[i] = b;
+  }
+}
+
+mc_status launch_fetch_rows(const void* k_src, const void* v_src, void* k_dst, void* v_dst, size_t n, cudaStream_t stream) {
+  const int n16 = (int)(n / 16);
+  if (n16 == 0) return MC_OK;
+  MC_CUDA_CHECK(launch_pdl(fetch_rows_kernel, dim3((n16 + 255) / 256), dim3(256), 0, stream, (const uint4*)k_src,
+                           (const uint4*)v_src, (uint4*)k_dst, (uint4*)v_dst, n16));
+  MC_CUDA_CHECK(cudaGetLastError());
+  return MC_OK;
+}
+
 }  // namespace mc
 
 // ---------------------------------------------------------------------------------------------------

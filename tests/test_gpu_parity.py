@@ -287,3 +287,48 @@ def test_merge_function_variants(H, merge_fn, dtype):
     out, lse = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
     stats.update(H.compare_attention(p, om, 2, q, out.cpu(), lse.cpu(), kn, vn))
     print(merge_fn, dtype, stats)
+
+
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned", "pageable"])
+def test_host_buffer_entry_points_equal_the_device_ones(H, pinned):
+    """mc_merge_pair_host / mc_decode_attn_host run the same kernels as the device-buffer calls: the
+    same bits must come back, whether the host buffers are pinned (the kernels read and write them
+    directly) or pageable (asynchronous copies through the staging buffer)."""
+    wl = dataclasses.replace(CONFIGS["c1"], seq_len=208, n_kv_heads=4, n_q_heads=8)
+    p = H.Problem(wl, seq_lens=np.array([200], np.int32))
+    words, code = p.run_merge()
+    assert code == 0, words
+    ref_dirs = p.pair.e_k.clone(), p.pair.e_v.clone(), p.pair.ret_rows.clone(), p.pair.ret_count.clone()
+    host = lambda t: (torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) if pinned else t.cpu().clone())
+    # merge from host pools into fresh staging pools and a fresh pair cache
+    hp = {k: host(v) for k, v in p.pools.items()}
+    stage = {k: torch.zeros_like(v) for k, v in p.pools.items()}
+    pair2 = p.mc.PairCache(p.cfg, p.B, p.n_pages, p.ret_capacity, device=p.device)
+    p.lib.mc_merge_pair_host(p.cfg, p.batch(), hp, stage, pair2, True, p.workspace(0))
+    torch.cuda.synchronize()
+    assert torch.equal(pair2.e_k, ref_dirs[0]) and torch.equal(pair2.e_v, ref_dirs[1])
+    assert torch.equal(pair2.ret_rows, ref_dirs[2]) and torch.equal(pair2.ret_count, ref_dirs[3])
+    # decode, pair mode with new tokens
+    wlb = dataclasses.replace(wl, batch=p.B)
+    q = gen.make_queries(wlb, 3, n_sets=2)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    ref, ref_lse = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
+    qh, knh, vnh = host(q), host(kn), host(vn)
+    out_h = host(torch.full_like(ref.cpu(), float("nan")))
+    lse_h = host(torch.full_like(ref_lse.cpu(), float("nan")))
+    io = torch.empty(p.lib.mc_decode_io_bytes(p.cfg, p.batch(), 2), dtype=torch.uint8, device=p.device)
+    for _ in range(2):  # twice: the staging buffer and the workspace are reused
+        p.lib.mc_decode_attn_host(p.cfg, p.batch(), p.pair, 2, qh, knh, vnh, 1.0 / math.sqrt(128.0), out_h, lse_h, io,
+                                  p.workspace(1, 2))
+        torch.cuda.synchronize()
+        assert torch.equal(out_h, ref.cpu()) and torch.equal(lse_h, ref_lse.cpu())
+    # without a new token and without the log-sum-exp
+    ref1, _ = p.run_attn(1, q[1:2].contiguous().to(p.device), None, None, want_lse=False)
+    q1 = host(q[1:2].contiguous())
+    out1 = host(torch.zeros_like(ref1.cpu()))
+    p.lib.mc_decode_attn_host(p.cfg, p.batch(), p.pair, 1, q1, None, None, 1.0 / math.sqrt(128.0), out1, None, io,
+                              p.workspace(1, 1))
+    torch.cuda.synchronize()
+    assert torch.equal(out1, ref1.cpu())
