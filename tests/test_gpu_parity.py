@@ -332,3 +332,36 @@ def test_host_buffer_entry_points_equal_the_device_ones(H, pinned):
                               p.workspace(1, 1))
     torch.cuda.synchronize()
     assert torch.equal(out1, ref1.cpu())
+
+
+@pytest.mark.parametrize("hkv,hq,lens,ps", [
+    (2, 2, [9000, 130, 4097], 16),     # one query row: pieces up to 4096 tokens, cut by the score buffer and by team ranges
+    (3, 6, [700, 5, 1300, 0, 260], 32),  # three kv heads (a team of three), an empty sequence
+    (64, 64, [300, 77], 16),           # more kv heads than CTAs in a team: two heads per CTA
+    (1, 8, [2500], 64),                # eight query rows on one kv head: pieces of 512 tokens
+])
+def test_attention_work_split_shapes(H, hkv, hq, lens, ps):
+    """Decode attention where the cut into teams, heads per CTA and pieces matters: sequences longer than
+    one piece, team boundaries inside sequences, head counts that are no power of two or exceed a team.
+    Merge without retention check here (covered elsewhere); attention of layer l with a new token,
+    sampled (sequence, head) pairs against the oracle, and pair mode where the head ratio allows it."""
+    S = max(lens) + (-max(lens)) % ps
+    wl = CONFIGS["c1"].scaled("split", n_kv_heads=hkv, n_q_heads=hq, batch=len(lens), seq_len=S, page_size=ps, index=77)
+    p = H.Problem(wl, seq_lens=np.array(lens, np.int32))
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge()
+    wlb = dataclasses.replace(wl, batch=p.B)
+    q = gen.make_queries(wlb, 1, n_sets=2)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    rs = np.random.RandomState(3)
+    sample = [(b, int(rs.randint(hq))) for b in range(p.B) for _ in range(2)]
+    out, lse = p.run_attn(1, q[1:2].contiguous().to(p.device), kn[1:2].contiguous().to(p.device), vn[1:2].contiguous().to(p.device))
+    H.compare_attention(p, om, 1, q[1:2].contiguous(), out.cpu(), lse.cpu(), kn[1:2].contiguous(), vn[1:2].contiguous(), sample=sample)
+    out0, lse0 = p.run_attn(0, q[0:1].contiguous().to(p.device))  # no new token: an empty sequence gives zeros
+    H.compare_attention(p, om, 0, q[0:1].contiguous(), out0.cpu(), lse0.cpu(), sample=sample)
+    if 2 * (hq // hkv) <= 8:
+        out2, lse2 = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
+        H.compare_attention(p, om, 2, q, out2.cpu(), lse2.cpu(), kn, vn, sample=sample)
