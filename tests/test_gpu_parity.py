@@ -365,3 +365,65 @@ def test_attention_work_split_shapes(H, hkv, hq, lens, ps):
     if 2 * (hq // hkv) <= 8:
         out2, lse2 = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
         H.compare_attention(p, om, 2, q, out2.cpu(), lse2.cpu(), kn, vn, sample=sample)
+
+
+class _Segment:
+    """One (sequence, kv head) of a full-size problem, shaped like a Problem for the comparison helpers."""
+
+    def __init__(self, p, b, h):
+        self.p, self.b0, self.h0 = p, b, h
+        self.B, self.H, self.Hq, self.S = 1, 1, p.Hq // p.H, p.S
+        self.dtype, self.gamma, self.t = p.dtype, p.gamma, p.t
+        self.seq_lens_host = p.seq_lens_host[b:b + 1]
+        self.bits = {k: v[b:b + 1, :, h:h + 1] for k, v in p.bits.items()}
+
+    def retained(self, dc, tensor, b, h):
+        return self.p.retained(dc["full"], tensor, self.b0, self.h0)
+
+    def logical_of(self, rows, seq_len=None):  # the test hands over logical rows of this segment already
+        return rows
+
+    def slice_cache(self, dc):
+        b, h = self.b0, self.h0
+        out = {k: dc[k][b:b + 1, :, h:h + 1] for k in ("e_k", "e_v", "scale", "dist")}
+        out["seg_minmax"] = dc["seg_minmax"][:, b:b + 1, h:h + 1]
+        out["full"] = dc
+        return out
+
+
+def test_full_size_config2_sampled(H):
+    """Config 2 at its full size (batch 8 x 4096 tokens, 32 heads, fp16, page 16; the last layer pair), in
+    the launch configuration the benchmark times: merge, restore and decode attention with a new token
+    and room for the decode steps; sampled (sequence, head) segments are compared against the oracle
+    with the same bars as everywhere else, and the retained totals must agree with the status word."""
+    from oracle import minicache_oracle as orc
+    wl = CONFIGS["c2"]
+    p = H.Problem(wl, pair=wl.n_pairs - 1, decode_room=wl.decode_steps + 1)
+    words, code = p.run_merge()
+    assert code == 0, words
+    dc = p.device_cache()
+    assert int(dc["ret_count"].sum()) == int(words[1])
+    rs = np.random.RandomState(17)
+    segs = [(int(rs.randint(p.B)), int(rs.randint(p.H))) for _ in range(4)]
+    dk, dv = p.run_restore(1)
+    dkl, dvl = p.logical_of(dk), p.logical_of(dv)
+    wlb = dataclasses.replace(wl, batch=p.B)
+    q = gen.make_queries(wlb, 2, n_sets=2)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    out, lse = p.run_attn(1, q[1:2].contiguous().to(p.device), kn[1:2].contiguous().to(p.device), vn[1:2].contiguous().to(p.device))
+    out2, lse2 = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
+    out, lse, out2, lse2 = out.cpu(), lse.cpu(), out2.cpu(), lse2.cpu()
+    for b, h in segs:
+        sg = _Segment(p, b, h)
+        om = {tn: orc.merge_pair(sg.bits[tn + "_lm1"], sg.bits[tn + "_l"], sg.seq_lens_host, sg.dtype, sg.t, sg.gamma)
+              for tn in ("k", "v")}
+        dcs = sg.slice_cache(dc)
+        stats = H.compare_merge(sg, om, dcs)
+        # restore of layer l: dense rows of this segment
+        stats.update(H.compare_restore(sg, om, dcs, 1, dkl[b:b + 1, :, h:h + 1], dvl[b:b + 1, :, h:h + 1]))
+        sl = lambda x, hd: x[:, b:b + 1, hd:hd + 1].contiguous()
+        stats.update(H.compare_attention(sg, om, 1, sl(q[1:2], h), sl(out, h), sl(lse, h), sl(kn[1:2], h), sl(vn[1:2], h)))
+        stats.update(H.compare_attention(sg, om, 2, sl(q, h), sl(out2, h), sl(lse2, h), sl(kn, h), sl(vn, h)))
+        print("segment", b, h, stats)
