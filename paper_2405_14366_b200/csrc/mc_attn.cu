@@ -6,15 +6,16 @@
 //   sum_i p_i (g_i e_i) = sum_i (p_i g_i) e_i  the V scale multiplies the probability
 //
 // so the shared direction rows are streamed once, untouched; a retained token (whose scales the
-// merge left at zero) only replaces one score (K) or adds one term to the sum (V).
+// merge left at -0) only replaces one score (K) or adds one term to the sum (V).
 //
-// Work item = (sequence, split of the token axis, kv head).  The kernel is persistent: two CTAs
-// per SM walk the item list with a fixed stride.  In each CTA
-//   - the producer warp streams everything the item needs through one ring of stages with bulk
+// The kernel is persistent, two CTAs per SM.  The token axis is cut into equal shares for teams of
+// CTAs, a team member takes its team's share for one kv head (see piece_at); a work item (a piece)
+// is a run of 128-token units of one (sequence, kv head).  In each CTA
+//   - the producer warp streams everything a piece needs through one ring of stages with bulk
 //     asynchronous copies (TMA engine, cp.async.bulk + mbarrier): one copy per (page, head, tensor)
-//     tile, all K tiles of an item, then "extra" stages holding the split's retained K rows and
-//     the step's new K row, then the V tiles and the V extras; it runs ahead into the next item,
-//     and loads page ids and retained ranges one item early (a demand load takes microseconds
+//     tile, all K tiles of the piece, then "extra" stages holding the piece's retained K rows and
+//     the step's new K row, then the V tiles and the V extras; it runs ahead into the next piece,
+//     and loads page ids and retained ranges one piece early (a demand load takes microseconds
 //     while the copy engine saturates the memory system, so nothing irregular is left on any
 //     critical path);
 //   - four consumer warps run every contraction on the tensor cores, the query rows of the kv
@@ -23,7 +24,7 @@
 //     rows, fill the columns the tiles leave out), row maxima tracked on the way -> V phase: each
 //     warp takes 16 tokens of every tile, P = 2^(score - max) x V scale formed where it is used,
 //     plus gathered P times the retained V rows; the warps' partial sums meet in shared memory.
-// Partial (m, l, o) per split are merged by attn_combine_kernel.  Every wait is bounded.
+// Partial (m, l, o) per piece are merged by attn_combine_kernel.  Every wait is bounded.
 #include <algorithm>
 
 #include "mc_common.cuh"
@@ -208,7 +209,7 @@ struct Ranges {
   int k_lo, n_k, v_lo, n_v;
 };
 
-// Two table entries per list: split boundaries are multiples of 128 and no retained token lies
+// Two table entries per list: piece boundaries are multiples of 128 and no retained token lies
 // past the length the pair was merged at.  The loads are issued one item ahead and only combined
 // (ranges_of) when that item starts: arithmetic on a loaded value would stall the producer warp for
 // the load's whole latency, microseconds while the copy engine saturates the memory system.
@@ -696,7 +697,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       }
     }
 
-    // ---- partial results of this split: the four warps' sums meet in shared memory (the score
+    // ---- partial results of this piece: the four warps' sums meet in shared memory (the score
     // buffer, free once every warp has left the V phase) ---------------------------------------------
     l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
     l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
@@ -1001,7 +1002,7 @@ mc_status launch_fetch_rows(const void* k_src, const void* v_src, void* k_dst, v
 }  // namespace mc
 
 // ---------------------------------------------------------------------------------------------------
-// Decode attention for callers that cannot supply scratch memory: the split partials live in a
+// Decode attention for callers that cannot supply scratch memory: the pieces' partials live in a
 // device array that is part of the library image.
 // ---------------------------------------------------------------------------------------------------
 #include <mutex>
