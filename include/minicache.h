@@ -300,6 +300,14 @@ mc_status mc_decode_attn_static(const mc_config* cfg, const mc_batch* batch, con
                                 int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
                                 float sm_scale, void* out, float* lse, void* stream);
 
+/* Self-test of the error path of the bounded waits (the paper has no counterpart): enqueues a
+ * one-warp kernel that waits, with the same bounded wait the streaming kernels use and a limit of
+ * `poll_limit` polls, on a barrier that nothing completes.  The wait gives up, sets
+ * MC_FLAG_WAIT_TIMEOUT in the pair's status words and the kernel returns normally: the context
+ * stays usable and mc_read_status reports MC_ERR_DEVICE_STATUS until the next merge into the pair
+ * clears the words. */
+mc_status mc_selftest_wait_timeout(const mc_pair_cache* pair, int32_t poll_limit, void* stream);
+
 /* Copies the pair's status words to host memory `out_words[MC_STATUS_WORDS]` after synchronising
  * `stream`.  Returns MC_ERR_CAPACITY if the overflow flag is set, MC_ERR_DEVICE_STATUS for any
  * other flag, MC_OK otherwise. */

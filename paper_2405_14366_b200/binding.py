@@ -59,7 +59,7 @@ class _PairCache(C.Structure):
 
 EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
-           "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4")
+           "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -209,6 +209,8 @@ class MiniCacheLib:
         L.mc_merge_pair_q4.argtypes = [P(_Config), P(_Batch), P(_LayerQ4), P(_LayerQ4), P(_PairCache), C.c_int32, V,
                                        C.c_size_t, V]
         L.mc_merge_pair_q4.restype = C.c_int32
+        L.mc_selftest_wait_timeout.argtypes = [P(_PairCache), C.c_int32, V]
+        L.mc_selftest_wait_timeout.restype = C.c_int32
         for f in ("mc_workspace_bytes", "mc_merge_pair", "mc_append_pair", "mc_restore", "mc_decode_attn",
                   "mc_read_status", "mc_merge_pair_host", "mc_decode_attn_host", "mc_decode_io_bytes"):
             getattr(L, f).restype = C.c_int32
@@ -308,6 +310,10 @@ class MiniCacheLib:
         if code == 5:
             raise McError(code, "MC_ERR_CAPACITY", self._lib.mc_last_cuda_error().decode())
         self._check(code)
+
+    def mc_selftest_wait_timeout(self, pair: PairCache, poll_limit: int = 20000, stream=None):
+        pc = pair.c()
+        self._check(self._lib.mc_selftest_wait_timeout(C.byref(pc), int(poll_limit), _stream(stream)))
 
     def mc_read_status(self, pair: PairCache, stream=None, check: bool = True):
         words = (C.c_int32 * MC_STATUS_WORDS)()

@@ -308,6 +308,11 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
   return MC_OK;
 }
 
+mc_status mc_selftest_wait_timeout(const mc_pair_cache* pair, int32_t poll_limit, void* stream) {
+  if (pair == nullptr || pair->status == nullptr || poll_limit <= 0) return MC_ERR_INVALID_ARG;
+  return launch_wait_timeout_probe(pair->status, (uint32_t)poll_limit, (cudaStream_t)stream);
+}
+
 mc_status mc_read_status(const mc_pair_cache* pair, void* stream, int32_t* out_words) {
   if (pair == nullptr || pair->status == nullptr || out_words == nullptr) return MC_ERR_INVALID_ARG;
   MC_CUDA_CHECK(cudaMemcpyAsync(out_words, pair->status, MC_STATUS_WORDS * sizeof(int32_t), cudaMemcpyDeviceToHost,

@@ -973,6 +973,31 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   return MC_OK;
 }
 
+// ---- self-test of the bounded wait -------------------------------------------------------------------
+// One warp waits on a barrier that nothing ever completes, with the wait the streaming kernels use
+// (a short poll limit): the wait gives up, records MC_FLAG_WAIT_TIMEOUT in the status words and the
+// kernel returns normally.
+__global__ void __launch_bounds__(32) wait_timeout_probe_kernel(int32_t* status, uint32_t limit) {
+  grid_dep_wait();
+  grid_dep_launch();
+  __shared__ uint64_t bar;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, &s_abort, status, limit);
+  __syncwarp();
+}
+
+mc_status launch_wait_timeout_probe(int32_t* status, uint32_t limit, cudaStream_t stream) {
+  MC_CUDA_CHECK(launch_pdl(wait_timeout_probe_kernel, dim3(1), dim3(32), 0, stream, status, limit));
+  MC_CUDA_CHECK(cudaGetLastError());
+  return MC_OK;
+}
+
 // ---- new-token rows from device-addressable host memory ------------------------------------------
 __global__ void __launch_bounds__(256) fetch_rows_kernel(const uint4* k_src, const uint4* v_src, uint4* k_dst, uint4* v_dst,
                                                          int n16) {

@@ -23,4 +23,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
 // memory into device staging with one small kernel.
 mc_status launch_fetch_rows(const void* k_src, const void* v_src, void* k_dst, void* v_dst, size_t n, cudaStream_t stream);
 
+// One warp runs into the bounded wait's limit (`limit` polls) and records it in `status`.
+mc_status launch_wait_timeout_probe(int32_t* status, uint32_t limit, cudaStream_t stream);
+
 }  // namespace mc

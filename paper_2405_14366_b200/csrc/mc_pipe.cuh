@@ -34,9 +34,10 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 // Bounded wait: gives up after kWaitLimit polls, records it, and makes every later wait of the
 // CTA (and of CTAs that look at the status word afterwards) return at once.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int32_t* status,
+                                          uint32_t limit = kWaitLimit) {
   if (*s_abort) return false;
-  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 64) __nanosleep(40);
     if ((it & 1023) == 1023 && (*s_abort || (*(volatile int32_t*)status & MC_FLAG_WAIT_TIMEOUT))) break;

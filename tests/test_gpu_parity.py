@@ -427,3 +427,20 @@ def test_full_size_config2_sampled(H):
         stats.update(H.compare_attention(sg, om, 1, sl(q[1:2], h), sl(out, h), sl(lse, h), sl(kn[1:2], h), sl(vn[1:2], h)))
         stats.update(H.compare_attention(sg, om, 2, sl(q, h), sl(out2, h), sl(lse2, h), sl(kn, h), sl(vn, h)))
         print("segment", b, h, stats)
+
+
+def test_bounded_wait_times_out_into_the_status_word(H):
+    """A wait that nothing ends: the kernel gives up after its poll limit, records the time-out in
+    the pair's status words and returns; the context stays usable and the next merge clears the flag."""
+    p = H.Problem(CONFIGS["c1"].scaled("wait", n_kv_heads=2, n_q_heads=2, seq_len=64, index=91))
+    words, code = p.run_merge()
+    assert code == 0
+    p.lib.mc_selftest_wait_timeout(p.pair, 20000)
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 8 and (words[0] & 2) == 2, (words, code)  # MC_ERR_DEVICE_STATUS, MC_FLAG_WAIT_TIMEOUT
+    with pytest.raises(p.mc.McError):
+        p.lib.mc_read_status(p.pair)
+    words, code = p.run_merge()  # the context works, the merge clears the words
+    assert code == 0 and words[0] == 0
+    _full_cycle(H, p)
