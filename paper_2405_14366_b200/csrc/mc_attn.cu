@@ -830,6 +830,24 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.slots;
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
   const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
+  // The group's first four pieces are requested before anything depends on a loaded value, so the
+  // maxima and these partials arrive together (one memory latency for a sequence of up to 32 pieces).
+  float2 v2[4];
+  float4 v[4];
+  auto load4 = [&](int j0) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int j = j0 + k * kCombineGroups;
+      v2[k] = make_float2(-INFINITY, 0.f);
+      v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j < n) {
+        const int slot = list_s[j];
+        v2[k] = ml[slot];
+        v[k] = po[(size_t)slot * (kHeadDim / 4)];
+      }
+    }
+  };
+  load4(grp);
   // ---- M = max_j m_j
   float M = -INFINITY;
   for (int j = tid; j < n; j += kCombineThreads) M = fmaxf(M, ml[list_s[j]].x);
@@ -844,19 +862,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   float L = 0.f;
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int j0 = grp; j0 < n; j0 += 4 * kCombineGroups) {
-    float2 v2[4];
-    float4 v[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int j = j0 + k * kCombineGroups;
-      v2[k] = make_float2(-INFINITY, 0.f);
-      v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (j < n) {
-        const int slot = list_s[j];
-        v2[k] = ml[slot];
-        v[k] = po[(size_t)slot * (kHeadDim / 4)];
-      }
-    }
+    if (j0 != grp) load4(j0);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float w = v2[k].x == -INFINITY ? 0.f : exp2f(v2[k].x - M);
