@@ -10,7 +10,7 @@
 //
 // The kernel is persistent, two CTAs per SM.  The token axis is cut into equal shares for teams of
 // CTAs, a team member takes its team's share for one kv head (see piece_at); a work item (a piece)
-// is a run of 128-token units of one (sequence, kv head).  In each CTA
+// is a chunk of a piece: a run of 128-token units of one (sequence, kv head).  In each CTA
 //   - the producer warp streams everything a piece needs through one ring of stages with bulk
 //     asynchronous copies (TMA engine, cp.async.bulk + mbarrier): one copy per (page, head, tensor)
 //     tile, all K tiles of the piece, then "extra" stages holding the piece's retained K rows and
@@ -148,11 +148,12 @@ __device__ __forceinline__ bool is_retained_scale(float g) { return __float_as_u
 
 // One work item = a piece: a run of units of one (sequence, kv head).
 struct Item {
-  int b, g, split;  // split = the piece's first unit inside its sequence (also its partial slot)
-  int split_start;
-  int n_tok;    // cached tokens of this piece
+  int b, g, split;  // split = the piece's first unit inside its sequence (its partial slot)
+  int split_start;  // first token of this chunk
+  int n_tok;    // cached tokens of this chunk
   int T;        // 64-token tiles
   int units;
+  bool first, last;  // first / last chunk of its piece
   bool has_new;
   bool valid;
 };
@@ -162,18 +163,19 @@ struct Item {
 // the units [t U / T, (t + 1) U / T) -- the same share for every team whatever the lengths are --
 // and its member j takes them for the kv heads j, j + S, ...  The members of a team stream the
 // same pages at about the same time (neighbouring tiles of a page: whole DRAM rows get used), and
-// nobody waits for a last round of items.  A piece = a run of units of one (sequence, head): it
-// stops at the end of the sequence, at the end of the team's range and at the capacity of the
-// score buffer.
+// nobody waits for a last round of items.  A piece = the units of one (sequence, head) inside a
+// team's range: one partial result.  A CTA works through a piece in chunks of as many units as the
+// score buffer holds, carrying the running maximum, sum and output from chunk to chunk.
 struct Cursor {
   int g, x;  // kv head, unit
 };
-__device__ __forceinline__ Item piece_at(const Cursor& c, int x_end, const int* pre_s, const int* len_s, const AttnParams& p) {
+__device__ __forceinline__ Item piece_at(const Cursor& c, int x_begin, int x_end, const int* pre_s, const int* len_s,
+                                         const AttnParams& p) {
   Item it;
   it.valid = c.g < p.g.n_kv_heads && c.x < x_end;
   if (!it.valid) {
     it.b = it.g = it.split = it.split_start = it.n_tok = it.T = it.units = 0;
-    it.has_new = false;
+    it.has_new = it.first = it.last = false;
     return it;
   }
   int lo = 0, hi = p.g.batch - 1;  // last b with pre_s[b] <= x
@@ -184,13 +186,18 @@ __device__ __forceinline__ Item piece_at(const Cursor& c, int x_end, const int* 
   it.b = lo;
   it.g = c.g;
   const int u_b = pre_s[lo + 1] - pre_s[lo];
-  it.split = c.x - pre_s[lo];
-  it.units = min(min(u_b - it.split, x_end - c.x), p.cap_units);
+  const int k = c.x - pre_s[lo];                        // this chunk's first unit inside the sequence
+  const int k_lo = max(0, x_begin - pre_s[lo]);         // the piece's first unit
+  const int k_hi = min(u_b, x_end - pre_s[lo]);         // one past the piece's last unit
+  it.split = k_lo;
+  it.units = min(k_hi - k, p.cap_units);
+  it.first = k == k_lo;
+  it.last = k + it.units == k_hi;
   const int n = len_s[lo];
-  it.split_start = it.split * kUnit;
-  it.n_tok = max(0, min(n, (it.split + it.units) * kUnit) - it.split_start);
+  it.split_start = k * kUnit;
+  it.n_tok = max(0, min(n, (k + it.units) * kUnit) - it.split_start);
   it.T = (it.n_tok + kTile - 1) / kTile;
-  it.has_new = (p.k_new != nullptr) && (it.split + it.units == u_b);
+  it.has_new = (p.k_new != nullptr) && (k + it.units == u_b);
   return it;
 }
 // The cursor after piece `it`: on through the team's range, then the member's next head.
@@ -313,7 +320,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     // engine saturates the memory system.
     int it = 0;  // running stage counter, same sequence as the consumers'
     Cursor cur = c_first;
-    Item w = piece_at(cur, x_end, pre_s, len_s, p);
+    Item w = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
     RawRanges raw;
     // page ids of a piece: lane l holds pages l, l + 32, ... (registers, loaded one piece ahead),
     // handed over to shared memory when the piece starts
@@ -338,7 +345,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       for (int r = 0; r < kMaxPiecePages / 32; ++r) pages[lane + 32 * r] = pg_reg[r];
       __syncwarp();
       cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
-      const Item wn = piece_at(cur, x_end, pre_s, len_s, p);
+      const Item wn = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
       const Ranges rg = ranges_of(raw);  // loaded one piece ago
       const RawRanges rawn = load_ranges(wn, p);
       load_pages(wn);
@@ -432,16 +439,21 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   };
   {
     uint32_t qw[4];
-    load_q_words(piece_at(c_first, x_end, pre_s, len_s, p), qw);
+    load_q_words(piece_at(c_first, x_begin, x_end, pre_s, len_s, p), qw);
 #pragma unroll
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
   grid_dep_wait();
   consumer_sync();
 
+  // carried from chunk to chunk of a piece: the output sums, this thread's part of the row sum, and
+  // the running maxima of the rows this thread meets (row `row` in the V phase, rows colp and
+  // colp + 1 in its accumulators)
+  float acc[8][4];
+  float l_acc = 0.f, m_run = -INFINITY, m_run0 = -INFINITY, m_run1 = -INFINITY;
   Cursor cur = c_first;
   for (;; ++n_item) {
-    const Item w = piece_at(cur, x_end, pre_s, len_s, p);
+    const Item w = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
     if (!w.valid) break;
     cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
@@ -570,28 +582,51 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     }
     if ((lane & 3) == 0) red2_s[row * kConsumerWarps + warp] = mxe;  // row `row` (raw rows)
     consumer_sync();
-    float m_row;
-    {
-      const float4 ma = *reinterpret_cast<const float4*>(red_s + row * kConsumerWarps);
-      const float4 mb = *reinterpret_cast<const float4*>(red2_s + row * kConsumerWarps);
-      m_row = fmaxf(fmaxf(fmaxf(ma.x, ma.y), fmaxf(ma.z, ma.w)), fmaxf(fmaxf(mb.x, mb.y), fmaxf(mb.z, mb.w)));
-      if (warp == 0 && (lane & 3) == 0) m_s[row] = m_row;
+    auto row_max = [&](int r) {
+      const float4 ma = *reinterpret_cast<const float4*>(red_s + r * kConsumerWarps);
+      const float4 mb = *reinterpret_cast<const float4*>(red2_s + r * kConsumerWarps);
+      return fmaxf(fmaxf(fmaxf(ma.x, ma.y), fmaxf(ma.z, ma.w)), fmaxf(fmaxf(mb.x, mb.y), fmaxf(mb.z, mb.w)));
+    };
+    // this chunk's maxima joined with the piece's so far; what was summed under the old maximum is
+    // rescaled by 2^(old - new)
+    auto rescale = [](float m_old, float m_new) { return m_old == -INFINITY ? 0.f : exp2f(m_old - m_new); };
+    if (w.first) {
+      m_run = m_run0 = m_run1 = -INFINITY;
+      l_acc = 0.f;
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[a][k] = 0.f;
     }
-    float l_acc = 0.f;  // sum of this thread's probabilities of row `row`
+    const float m_row = fmaxf(m_run, row_max(row));
+    if (!w.first) {
+      const float m0 = fmaxf(m_run0, row_max(colp)), m1 = fmaxf(m_run1, row_max(colp + 1));
+      const float f = rescale(m_run, m_row), f0 = rescale(m_run0, m0), f1 = rescale(m_run1, m1);
+      l_acc *= f;
+#pragma unroll
+      for (int a = 0; a < 8; ++a) {
+        acc[a][0] *= f0;
+        acc[a][2] *= f0;
+        acc[a][1] *= f1;
+        acc[a][3] *= f1;
+      }
+      m_run0 = m0;
+      m_run1 = m1;
+    } else {
+      m_run0 = row_max(colp);
+      m_run1 = row_max(colp + 1);
+    }
+    m_run = m_row;
+    if (w.last && warp == 0 && (lane & 3) == 0) m_s[row] = m_row;
 
     // query rows of the next item travel while the V tiles stream
     uint32_t qnext[4];
-    load_q_words(piece_at(cur, x_end, pre_s, len_s, p), qnext);
+    load_q_words(piece_at(cur, x_begin, x_end, pre_s, len_s, p), qnext);
 
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
     // A = the warp's 16 token rows transposed (16 channels x 16 tokens per m tile), B = the rows'
     // probabilities times the V scale: D[channel][row], eight m tiles = all 128 channels.  Every
     // warp sums its own tokens; the four partial sums meet in shared memory at the end of the item.
-    float acc[8][4];
-#pragma unroll
-    for (int a = 0; a < 8; ++a)
-#pragma unroll
-      for (int k = 0; k < 4; ++k) acc[a][k] = 0.f;
     const int tk_w = warp * 16;
     // chunk position of m tile j for this lane: chunk 2 j + (mi & 1) of a row whose index is mr (mod 8)
     const uint32_t vsw_lo = (uint32_t)(((mi & 1) ^ (mr & 1)) | (mr & 6));
@@ -697,8 +732,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       }
     }
 
-    // ---- partial results of this piece: the four warps' sums meet in shared memory (the score
-    // buffer, free once every warp has left the V phase) ---------------------------------------------
+    // ---- the piece's partial result after its last chunk: the four warps' sums meet in shared
+    // memory (the score buffer, free once every warp has left the V phase) ----------------------------
+    if (w.last) {
     l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 1);
     l_acc += __shfl_xor_sync(0xffffffffu, l_acc, 2);
     if ((lane & 3) == 0) l_s[row * kConsumerWarps + warp] = l_acc;
@@ -732,6 +768,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         p.part_ml[prow * 2 + 1] = (ll.x + ll.y) + (ll.z + ll.w);
       }
     }
+    }
     // next item's query rows into the other buffer (nobody reads that buffer any more)
     {
       uint32_t* qn = q_s + ((n_item + 1) & 1) * kMaxRows * 64;
@@ -749,8 +786,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
 // Log-sum-exp merge of the pieces' partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
 // One block per output row.  The pieces of its sequence follow from the lengths and the number of
-// teams: they start where the sequence starts, at every team boundary inside it, and every
-// cap_units from there.  A thread per team that touches the
+// teams: one per team range that touches the sequence, stored in the slot of its first unit.  A thread per team that touches the
 // sequence counts that team's pieces, a scan turns the counts into a list of slots in shared memory;
 // then eight groups of 32 lanes share the pieces (a lane owns four channels), four loads in flight.
 constexpr int kCombineThreads = 256;
@@ -799,7 +835,6 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   // ---- the list of slots
   const int c_first = (int)(((x0 + 1) * n_teams - 1) / n_units);  // the team whose range holds the first unit
   const int c_last = (int)(((x0 + u) * n_teams - 1) / n_units);   // ... the last unit
-  const int cap = p.cap_units;
   int base = 0;
   for (int c0 = c_first; c0 <= c_last; c0 += kCombineThreads) {  // (more teams than threads: one more round)
     const int c = c0 + tid;
@@ -807,7 +842,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
     if (c <= c_last) {
       const long long lo = max(x0, n_units * c / n_teams), hi = min(x0 + u, n_units * (c + 1) / n_teams);
       s = (int)(lo - x0);
-      cnt = hi > lo ? (int)((hi - lo + cap - 1) / cap) : 0;
+      cnt = hi > lo ? 1 : 0;  // one piece (one partial) per team range that touches the sequence
     }
     int incl = cnt;
 #pragma unroll
@@ -820,7 +855,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
     int off = base + incl - cnt;
     for (int g = 0; g < grp; ++g) off += scan_s[g];
     for (int k = 0; k < cnt; ++k)
-      if (off + k < kMaxPieces) list_s[off + k] = s + k * cap;
+      if (off + k < kMaxPieces) list_s[off + k] = s;
     if (tid == kCombineThreads - 1) total_s = off + cnt;
     __syncthreads();
     base = total_s;
@@ -961,7 +996,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const int n_teams = (int)std::max<long long>(1, std::min<long long>(slots_gpu / ap.team_size, max_units));
   const int grid = n_teams * ap.team_size;
   ap.n_teams = n_teams;
-  if ((ap.slots + ap.cap_units - 1) / ap.cap_units + n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
+  if (n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
   const size_t smem = attn_smem_bytes();
   dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
