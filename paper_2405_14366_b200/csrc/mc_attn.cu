@@ -785,26 +785,28 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 }
 
 // Log-sum-exp merge of the pieces' partials: out = sum_j 2^(m_j - M) o_j / sum_j 2^(m_j - M) l_j.
-// One block per output row.  The pieces of its sequence follow from the lengths and the number of
-// teams: one per team range that touches the sequence, stored in the slot of its first unit.  A thread per team that touches the
-// sequence counts that team's pieces, a scan turns the counts into a list of slots in shared memory;
-// then eight groups of 32 lanes share the pieces (a lane owns four channels), four loads in flight.
+// A block serves R query heads of one sequence (R = 8: a warp per output row, for batches with many
+// rows; R = 1: the eight warps share the pieces of one row, for few rows with many pieces); a lane
+// owns four channels.  The pieces of the sequence follow from the lengths and the number of teams: one per
+// team range that touches the sequence, stored in the slot of its first unit; a thread per such team
+// writes the list into shared memory, before the wait on the split kernel (the lengths belong to the
+// caller), whose tail this overlaps.
 constexpr int kCombineThreads = 256;
-constexpr int kCombineGroups = kCombineThreads / 32;
-constexpr int kMaxPieces = 2048;  // pieces of one sequence (checked on the host)
+constexpr int kCombineWarps = kCombineThreads / 32;
+constexpr int kMaxPieces = 2048;  // pieces of one sequence = teams (checked on the host)
 
-template <int DT>
+template <int DT, int R>
 __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
   grid_dep_launch();
-  __shared__ float red[kCombineGroups];
-  __shared__ int scan_s[kCombineGroups];
-  __shared__ int total_s;
-  __shared__ float4 acc_s[kCombineGroups][32];
+  constexpr int GP = kCombineWarps / R;  // warps per output row
+  __shared__ int sum_s[2][kCombineWarps];
   __shared__ int list_s[kMaxPieces];
-  const int hq = blockIdx.x, b = blockIdx.y, set = blockIdx.z;
-  const int tid = threadIdx.x, grp = tid >> 5, lane = tid & 31;
-  // The lengths belong to the caller (no kernel of this library writes them): the piece list is
-  // built before the wait on the split kernel, whose tail it overlaps.
+  __shared__ float red_s[kCombineWarps];
+  __shared__ float4 acc_s[GP > 1 ? kCombineWarps : 1][32];
+  const int b = blockIdx.y, set = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int grp = warp % GP;  // this warp takes the pieces grp, grp + GP, ... of its row
+  const int hq = blockIdx.x * R + warp / GP;
   int before = 0, all = 0;  // units of the sequences before this one, of all sequences
   for (int bb = tid; bb < p.g.batch; bb += kCombineThreads) {
     const int ub = max(1, (p.g.seq_lens[bb] + kUnit - 1) / kUnit);
@@ -816,33 +818,32 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
     all += __shfl_xor_sync(0xffffffffu, all, o);
   }
   if (lane == 0) {
-    scan_s[grp] = before;
-    red[grp] = __int_as_float(all);
+    sum_s[0][warp] = before;
+    sum_s[1][warp] = all;
   }
   __syncthreads();
   before = 0;
   all = 0;
 #pragma unroll
-  for (int g = 0; g < kCombineGroups; ++g) {
-    before += scan_s[g];
-    all += __float_as_int(red[g]);
+  for (int g = 0; g < kCombineWarps; ++g) {
+    before += sum_s[0][g];
+    all += sum_s[1][g];
   }
-  __syncthreads();
-  const int pre_b = before, u = max(1, (p.g.seq_lens[b] + kUnit - 1) / kUnit);
-  const long long n_units = all;
+  const int u = max(1, (p.g.seq_lens[b] + kUnit - 1) / kUnit);
+  const long long n_units = all, x0 = before;
   const int n_teams = p.n_teams;
-  const long long x0 = pre_b;
-  // ---- the list of slots
-  const int c_first = (int)(((x0 + 1) * n_teams - 1) / n_units);  // the team whose range holds the first unit
-  const int c_last = (int)(((x0 + u) * n_teams - 1) / n_units);   // ... the last unit
+  // teams whose range [n_units c / T, n_units (c + 1) / T) meets [x0, x0 + u): consecutive, each with one piece
+  const int c_first = (int)(((x0 + 1) * n_teams - 1) / n_units);
+  const int c_last = (int)(((x0 + u) * n_teams - 1) / n_units);
+  // (a team's range can be empty when there are fewer units than teams: count, scan, then write)
   int base = 0;
   for (int c0 = c_first; c0 <= c_last; c0 += kCombineThreads) {  // (more teams than threads: one more round)
     const int c = c0 + tid;
-    int s = 0, cnt = 0;
+    int s0 = 0, cnt = 0;
     if (c <= c_last) {
       const long long lo = max(x0, n_units * c / n_teams), hi = min(x0 + u, n_units * (c + 1) / n_teams);
-      s = (int)(lo - x0);
-      cnt = hi > lo ? 1 : 0;  // one piece (one partial) per team range that touches the sequence
+      s0 = (int)(lo - x0);
+      cnt = hi > lo ? 1 : 0;
     }
     int incl = cnt;
 #pragma unroll
@@ -850,53 +851,47 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
       const int v = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += v;
     }
-    if (lane == 31) scan_s[grp] = incl;
+    __syncthreads();  // sum_s is free again
+    if (lane == 31) sum_s[0][warp] = incl;
     __syncthreads();
     int off = base + incl - cnt;
-    for (int g = 0; g < grp; ++g) off += scan_s[g];
-    for (int k = 0; k < cnt; ++k)
-      if (off + k < kMaxPieces) list_s[off + k] = s;
-    if (tid == kCombineThreads - 1) total_s = off + cnt;
-    __syncthreads();
-    base = total_s;
+    for (int g = 0; g < warp; ++g) off += sum_s[0][g];
+    if (cnt && off < kMaxPieces) list_s[off] = s0;
+#pragma unroll
+    for (int g = 0; g < kCombineWarps; ++g) base += sum_s[0][g];
   }
   const int n = min(base, kMaxPieces);
+  __syncthreads();
   grid_dep_wait();
+  const bool active = hq < p.n_q_heads;
+  if (GP == 1 && !active) return;
   const size_t prow0 = (((size_t)set * p.g.batch + b) * p.n_q_heads + hq) * p.slots;
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + prow0;
   const float4* po = reinterpret_cast<const float4*>(p.part_o + prow0 * kHeadDim) + lane;
-  // The group's first four pieces are requested before anything depends on a loaded value, so the
-  // maxima and these partials arrive together (one memory latency for a sequence of up to 32 pieces).
+  // The first four pieces are requested before anything depends on a loaded value, so the maxima
+  // and these partials arrive together.
   float2 v2[4];
   float4 v[4];
   auto load4 = [&](int j0) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const int j = j0 + k * kCombineGroups;
       v2[k] = make_float2(-INFINITY, 0.f);
       v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (j < n) {
-        const int slot = list_s[j];
+      if (active && j0 + k * GP < n) {
+        const int slot = list_s[j0 + k * GP];
         v2[k] = ml[slot];
         v[k] = po[(size_t)slot * (kHeadDim / 4)];
       }
     }
   };
   load4(grp);
-  // ---- M = max_j m_j
   float M = -INFINITY;
-  for (int j = tid; j < n; j += kCombineThreads) M = fmaxf(M, ml[list_s[j]].x);
+  if (active)
+    for (int j = lane; j < n; j += 32) M = fmaxf(M, ml[list_s[j]].x);
   for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  if (lane == 0) red[grp] = M;
-  __syncthreads();
-  M = red[0];
-#pragma unroll
-  for (int g = 1; g < kCombineGroups; ++g) M = fmaxf(M, red[g]);
-  __syncthreads();
-  // ---- L = sum_j w_j l_j and o = sum_j w_j o_j: group grp takes the pieces grp, grp + 8, ...
   float L = 0.f;
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j0 = grp; j0 < n; j0 += 4 * kCombineGroups) {
+  for (int j0 = grp; j0 < n; j0 += 4 * GP) {
     if (j0 != grp) load4(j0);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -908,28 +903,27 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
       o.w = fmaf(w, v[k].w, o.w);
     }
   }
-  if (lane == 0) red[grp] = L;
-  acc_s[grp][lane] = o;
-  __syncthreads();
-  if (grp == 0) {
-    L = red[0];
-#pragma unroll
-    for (int g = 1; g < kCombineGroups; ++g) {
-      L += red[g];
-      const float4 v = acc_s[g][lane];
-      o.x += v.x;
-      o.y += v.y;
-      o.z += v.z;
-      o.w += v.w;
+  if (GP > 1) {  // the row's warps meet in shared memory
+    acc_s[GP > 1 ? warp : 0][lane] = o;
+    if (lane == 0) red_s[warp] = L;
+    __syncthreads();
+    if (grp != 0 || !active) return;
+    for (int g = 1; g < GP; ++g) {
+      const float4 t = acc_s[GP > 1 ? warp + g : 0][lane];
+      L += red_s[warp + g];
+      o.x += t.x;
+      o.y += t.y;
+      o.z += t.z;
+      o.w += t.w;
     }
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    const size_t orow = ((size_t)set * p.g.batch + b) * p.n_q_heads + hq;
-    uint2 packed;
-    packed.x = Elem<DT>::pack(o.x * inv, o.y * inv);
-    packed.y = Elem<DT>::pack(o.z * inv, o.w * inv);
-    *reinterpret_cast<uint2*>(out + orow * kHeadDim + lane * 4) = packed;
-    if (lse != nullptr && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
   }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  const size_t orow = ((size_t)set * p.g.batch + b) * p.n_q_heads + hq;
+  uint2 packed;
+  packed.x = Elem<DT>::pack(o.x * inv, o.y * inv);
+  packed.y = Elem<DT>::pack(o.z * inv, o.w * inv);
+  *reinterpret_cast<uint2*>(out + orow * kHeadDim + lane * 4) = packed;
+  if (lse != nullptr && lane == 0) lse[orow] = L > 0.f ? (M + log2f(L)) * 0.69314718055994530942f : -INFINITY;
 }
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -998,17 +992,21 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.n_teams = n_teams;
   if (n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
   const size_t smem = attn_smem_bytes();
-  dim3 cgrid(cfg->n_q_heads, bt->batch, ap.n_sets);
+  // many output rows: a warp per row; few: a block per row
+  const bool warp_rows = (long long)ap.n_sets * bt->batch * cfg->n_q_heads >= 1024;
+  dim3 cgrid(warp_rows ? (cfg->n_q_heads + kCombineWarps - 1) / kCombineWarps : cfg->n_q_heads, bt->batch, ap.n_sets);
   if (cfg->dtype == MC_F16) {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_F16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_F16>, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
+    MC_CUDA_CHECK(launch_pdl(warp_rows ? attn_combine_kernel<MC_F16, kCombineWarps> : attn_combine_kernel<MC_F16, 1>, dim3(cgrid),
+                             dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
   } else {
     MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_BF16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
     MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(attn_combine_kernel<MC_BF16>, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
+    MC_CUDA_CHECK(launch_pdl(warp_rows ? attn_combine_kernel<MC_BF16, kCombineWarps> : attn_combine_kernel<MC_BF16, 1>, dim3(cgrid),
+                             dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
   }
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;

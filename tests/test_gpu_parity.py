@@ -338,7 +338,8 @@ def test_host_buffer_entry_points_equal_the_device_ones(H, pinned):
     (2, 2, [9000, 130, 4097], 16),     # one query row: pieces up to 4096 tokens, cut by the score buffer and by team ranges
     (3, 6, [700, 5, 1300, 0, 260], 32),  # three kv heads (a team of three), an empty sequence
     (64, 64, [300, 77], 16),           # more kv heads than CTAs in a team: two heads per CTA
-    (1, 8, [2500], 64),                # eight query rows on one kv head: pieces of 512 tokens
+    (1, 8, [2500], 64),                # eight query rows on one kv head: chunks of 512 tokens
+    (16, 32, [7 + 13 * (i % 11) for i in range(40)], 16),  # 1280 output rows: the combine kernel's warp-per-row form
 ])
 def test_attention_work_split_shapes(H, hkv, hq, lens, ps):
     """Decode attention where the cut into teams, heads per CTA and pieces matters: sequences longer than
