@@ -346,15 +346,24 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       __syncwarp();
       cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
       const Item wn = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
-      const Ranges rg = ranges_of(raw);  // loaded one piece ago
       const RawRanges rawn = load_ranges(wn, p);
       load_pages(wn);
       const int n_pages_item = (w.n_tok + ps - 1) >> shift;
       const int n_new = w.has_new ? 1 : 0;
       for (int ph = 0; ph < 2 && ok; ++ph) {
-        const int n_r = ph ? rg.n_v : rg.n_k, r_lo = ph ? rg.v_lo : rg.k_lo;
-        const int X = (n_r + n_new + cap_e - 1) / cap_e;  // extra stages: retained rows and the new token
-        for (int t = 0; t < w.T + X; ++t, ++it) {
+        // The retained ranges (loaded one piece ago; for a CTA's first piece just now) are looked at
+        // only when the last tile goes out: the consumers take the number of extra stages from the
+        // last tile's stage, so the tiles before it need not wait for those loads.
+        int n_r = 0, r_lo = 0;
+        int X = -1;  // extra stages: retained rows and the new token
+        for (int t = 0;; ++t, ++it) {
+          if (X < 0 && t >= w.T - 1) {
+            const Ranges rg = ranges_of(raw);
+            n_r = ph ? rg.n_v : rg.n_k;
+            r_lo = ph ? rg.v_lo : rg.k_lo;
+            X = (n_r + n_new + cap_e - 1) / cap_e;
+          }
+          if (X >= 0 && t >= w.T + X) break;
           const int s = it % kStages;
           if (it >= kStages) {
             int good = 1;
