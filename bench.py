@@ -34,9 +34,9 @@ import gen  # noqa: E402
 
 ROW = 256  # bytes of one 16-bit row of 128 channels
 # DRAM bytes (read + written) per algorithmic byte of the split attention kernel, from the ncu capture
-# summarised in profiles/attn_split_kernel_c2_one_pair.md (564.2 MB for 547.6 MB).  Set to None when
+# summarised in profiles/attn_split_kernel_c2_one_pair.md (562.5 MB for 547.6 MB).  Set to None when
 # the kernel changes until it is captured again.
-ATTN_TRAFFIC_RATIO = 1.030
+ATTN_TRAFFIC_RATIO = 1.027
 
 
 # ---------------------------------------------------------------------------------------------
