@@ -9,7 +9,7 @@
 // merge left at -0) only replaces one score (K) or adds one term to the sum (V).
 //
 // The kernel is persistent, two CTAs per SM.  The token axis is cut into equal shares for teams of
-// CTAs, a team member takes its team's share for one kv head (see piece_at); a work item (a piece)
+// CTAs, a team member takes its team's share for one kv head (see piece_at); a work item
 // is a chunk of a piece: a run of 128-token units of one (sequence, kv head).  In each CTA
 //   - the producer warp streams everything a piece needs through one ring of stages with bulk
 //     asynchronous copies (TMA engine, cp.async.bulk + mbarrier): one copy per (page, head, tensor)
@@ -38,7 +38,7 @@ constexpr int kStages = 5;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
-constexpr int kMaxRows = 8;                          // query rows per work item (M tile rows used)
+constexpr int kMaxRows = 8;                          // query rows per (sequence, kv head): the 8-wide N tile
 constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
 constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
@@ -48,9 +48,7 @@ constexpr int kSlabStride = 132;  // floats per row of a warp's partial output i
 struct AttnParams {
   Geom g;
   const char* e_pool[2];  // compressed tiles: K, V
-  const int32_t* ret_count;
   const int32_t* ret_offset;
-  const int32_t* ret_index;
   const int32_t* ret_prefix;
   int ret_prefix_stride;
   const char* ret_rows;  // [2 layers][ret_capacity][kEntryBytes]
@@ -67,7 +65,7 @@ struct AttnParams {
   int nq;    // query heads per kv head
   int rows;  // n_sets * nq
   int n_q_heads;
-  int cap_units;  // longest piece, in units of 128 tokens (what the score buffer holds for `rows` rows)
+  int cap_units;  // longest chunk, in units of 128 tokens (what the score buffer holds for `rows` rows)
   int slots;      // partial slots per output row = units of the longest sequence
   int team_size;  // CTAs per team (one or more kv heads each)
   int n_teams;
@@ -132,7 +130,7 @@ constexpr int kUnit = 128;            // tokens per unit of work: pieces start a
 constexpr int kScoreFloats = 4224;    // floats of the score buffer S [rows][piece tokens + 8] (16.5 KB)
 constexpr int kMaxPiecePages = 256;   // pages of the longest piece (4096 tokens of 16-token pages)
 
-// Longest piece for `rows` query rows: rows x (tokens + 8) floats must fit the score buffer.
+// Longest chunk for `rows` query rows: rows x (tokens + 8) floats must fit the score buffer.
 __host__ __device__ __forceinline__ int piece_cap_units(int rows) {
   const int u = (kScoreFloats / rows - 8) / kUnit;
   return u > 32 ? 32 : u;  // 32 units (rows = 1) ... 4 units (rows = 8)
@@ -146,7 +144,7 @@ static_assert(kConsumerWarps * kMaxRows * kSlabStride <= kScoreFloats, "slabs fi
 // stays distinguishable.
 __device__ __forceinline__ bool is_retained_scale(float g) { return __float_as_uint(g) == 0x80000000u; }
 
-// One work item = a piece: a run of units of one (sequence, kv head).
+// One work item = a chunk of a piece: a run of units of one (sequence, kv head).
 struct Item {
   int b, g, split;  // split = the piece's first unit inside its sequence (its partial slot)
   int split_start;  // first token of this chunk
@@ -635,7 +633,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
     // A = the warp's 16 token rows transposed (16 channels x 16 tokens per m tile), B = the rows'
     // probabilities times the V scale: D[channel][row], eight m tiles = all 128 channels.  Every
-    // warp sums its own tokens; the four partial sums meet in shared memory at the end of the item.
+    // warp sums its own tokens; the four partial sums meet in shared memory after the piece's last chunk.
     const int tk_w = warp * 16;
     // chunk position of m tile j for this lane: chunk 2 j + (mi & 1) of a row whose index is mr (mod 8)
     const uint32_t vsw_lo = (uint32_t)(((mi & 1) ^ (mr & 1)) | (mr & 6));
@@ -961,9 +959,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.g = g;
   ap.e_pool[0] = (const char*)pair->e_k;
   ap.e_pool[1] = (const char*)pair->e_v;
-  ap.ret_count = pair->ret_count;
   ap.ret_offset = pair->ret_offset;
-  ap.ret_index = pair->ret_index;
   ap.ret_prefix = pair->ret_prefix;
   ap.ret_prefix_stride = (int)pair->ret_prefix_stride;
   ap.ret_rows = (const char*)pair->ret_rows;
