@@ -211,6 +211,20 @@ class Job:
             self.seq_lens += 1
         self.launches += steps * self.wl.n_pairs * 5
 
+    def capture_decode_step(self):
+        """One decode step (every pair: attention of both layers, append; then the lengths grow by one)
+        as a CUDA graph: the kernels' programmatic dependencies become graph edges and the host issues
+        one launch per step."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):  # once outside capture: lazy one-time set-up must not be captured
+            self.decode_all(steps=1)
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.decode_all(steps=1)
+        return g
+
     def decode_pair_all(self, steps):
         """Pair mode: both layers of a pair in one call (two query sets, one pass over the directions)."""
         if steps == 0 or not hasattr(self, "ws_attn2"):  # steps == 0: set up the buffers only (outside any timed region)
@@ -427,6 +441,17 @@ def main():
     tok_steps = job.steps * float(job.prompt.sum()) + job.B * job.steps * (job.steps - 1) / 2
     phases["decode"] = {"ms": t_d * 1e3, "GB/s": (by["attn"] + by["append"]) / t_d / 1e9,
                         "kv_tokens_per_s": tok_steps * 2 * wl.n_pairs / t_d, "ms_per_decode_step": t_d * 1e3 / job.steps}
+    # the same decode phase replayed from a CUDA graph of one decode step (valid for any step: the
+    # lengths live on the device and grow inside the graph)
+    job.merge_all()
+    graph = job.capture_decode_step()
+    job.merge_all()
+    for _ in range(2):
+        graph.replay()
+    job.merge_all()
+    t_g = timed(lambda: [graph.replay() for _ in range(job.steps)])
+    phases["decode_cuda_graph"] = {"ms": t_g * 1e3, "GB/s": (by["attn"] + by["append"]) / t_g / 1e9,
+                                   "kv_tokens_per_s": tok_steps * 2 * wl.n_pairs / t_g, "ms_per_decode_step": t_g * 1e3 / job.steps}
     if 2 * (wl.n_q_heads // wl.n_kv_heads) <= 8:
         # pair mode (both layers' queries known up front: a replay or speculative setting, not a real
         # model's layer-by-layer decode): the shared directions are read once for two layers

@@ -445,3 +445,49 @@ def test_bounded_wait_times_out_into_the_status_word(H):
     words, code = p.run_merge()  # the context works, the merge clears the words
     assert code == 0 and words[0] == 0
     _full_cycle(H, p)
+
+
+def test_decode_step_replayed_from_a_cuda_graph(H):
+    """A decode step (attention of both layers with the new token, append, lengths + 1) captured in a
+    CUDA graph and replayed gives the same bits as the same calls issued one by one."""
+    wl = CONFIGS["c1"].scaled("graph", n_kv_heads=4, n_q_heads=8, batch=2, seq_len=320, index=93)
+    lens = np.array([300, 129], np.int32)
+    wlb = dataclasses.replace(wl, batch=2)
+    q = gen.make_queries(wlb, 0, n_sets=2)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    dev = {k: v[:, 0].contiguous().cuda() for k, v in nt.items()}
+    qd = q.cuda()
+    sm = 1.0 / math.sqrt(128.0)
+
+    def run(use_graph):
+        p = H.Problem(wl, seq_lens=lens.copy(), decode_room=8)
+        words, code = p.run_merge()
+        assert code == 0
+        outs = [torch.zeros(1, 2, 8, 128, dtype=torch.float16, device="cuda") for _ in range(2)]
+        b = p.mc.Batch(p.block_table, p.seq_lens, p.max_seq_len + 4, p.n_pages)
+        ws = torch.empty(p.lib.mc_workspace_bytes(p.cfg, b, 1, 1), dtype=torch.uint8, device="cuda")
+
+        def step():
+            for layer in (0, 1):
+                p.lib.mc_decode_attn(p.cfg, b, p.pair, layer, qd[layer], dev["k_lm1" if layer == 0 else "k_l"],
+                                     dev["v_lm1" if layer == 0 else "v_l"], sm, outs[layer], None, ws)
+            p.lib.mc_append_pair(p.cfg, b, p.pair, dev["k_lm1"], dev["v_lm1"], dev["k_l"], dev["v_l"])
+            p.seq_lens += 1
+
+        results = []
+        if use_graph:
+            g = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g):
+                step()
+        for _ in range(3):
+            g.replay() if use_graph else step()
+            torch.cuda.synchronize()
+            results.append([o.clone() for o in outs])
+        return results, p.pair.e_k.clone(), p.seq_lens.clone()
+
+    eager, ek_e, len_e = run(False)
+    graph, ek_g, len_g = run(True)
+    assert torch.equal(len_e, len_g) and torch.equal(ek_e, ek_g)
+    for a, b in zip(eager, graph):
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
