@@ -28,6 +28,10 @@
  *   batch: page id p names slot p of the layer pools and of the pair cache
  *   alike.  Token i of sequence b lives in page block_table[b][i / page_size]
  *   at row i % page_size.
+ * - The kernels are chained with programmatic dependent launch.  The batch description
+ *   (block_table, seq_lens) and the queries are never written by this library, so
+ *   mc_decode_attn reads them before it waits for the kernel ahead of it in the stream; a
+ *   caller whose own kernels let dependents start early must have them written before that.
  * - Argument errors are reported synchronously through the return code and
  *   launch nothing.  Data-dependent conditions (retained-row pool too small,
  *   a bounded wait inside a kernel running out) are recorded in the pair
