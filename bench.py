@@ -184,7 +184,7 @@ class Job:
         for pr in range(self.wl.n_pairs):
             for layer in (0, 1):
                 self.lib.mc_restore(self.cfg, b, self.pairs[pr], layer, self.dst_k, self.dst_v)
-        self.launches += 4 * self.wl.n_pairs
+        self.launches += 2 * self.wl.n_pairs  # one kernel per layer
 
     def decode_all(self, sample_events: bool = False, steps=None):
         b = self.batch(True)

@@ -1,6 +1,6 @@
 // Materialising restore of one layer (Eq. 2; Sec. 4.2 "Cache restoration"):
-//   restore_scale_kernel    x_hat = e_stored * (|x| / |e_stored|) for every cached row
-//   restore_scatter_kernel  retained rows overwritten with their raw copies (x_hat[I] = R)
+//   restore_scale_kernel    x_hat = e_stored * (|x| / |e_stored|) for every cached row that was merged,
+//                           then the retained rows from their raw copies (x_hat[I] = R)
 #include <algorithm>
 
 #include "mc_common.cuh"
@@ -147,6 +147,9 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
+#pragma unroll
+    for (int j = 0; j < 4; ++j)  // a retained token (scale -0) is written from its raw row below, by whichever CTA gets there
+      ok[j] = ok[j] && __float_as_uint(g[j]) != 0x80000000u;
     char* pd = (m.tensor ? p.dst_pool[1] : p.dst_pool[0]) + ((size_t)page * rows_in_page + m.grp * kRowsPerItem + r0) * kRowBytes + l16 * 16;
 #pragma unroll
     for (int j = 0; j < 4; ++j)
@@ -162,29 +165,27 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
       }
     page_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
   }
+  // ---- x_hat[I] = R: the raw rows of the retained tokens, segments dealt round-robin to the CTAs,
+  // a half-warp per row.  (The scaled rows above leave these tokens out, so the order is free.)
+  {
+    const int nseg = 2 * p.g.batch * H;
+    const int hw16 = tid >> 4;
+    for (int seg = blockIdx.x; seg < nseg; seg += gridDim.x) {
+      const int cnt = p.ret_count[seg], off = p.ret_offset[seg];
+      const int h = seg % H, b = (seg / H) % p.g.batch, tensor = seg / (H * p.g.batch);
+      char* dst_pool = tensor ? p.dst_pool[1] : p.dst_pool[0];
+      for (int e = hw16; e < cnt; e += kRestoreThreads / 16) {
+        const int tok = p.ret_index[off + e];
+        const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> shift)];
+        const size_t row = ((size_t)page * H + h) * ps + (tok & (ps - 1));
+        const uint4 v = *reinterpret_cast<const uint4*>(p.ret_rows + ((size_t)p.layer * p.ret_capacity + off + e) * kRetEntryBytes +
+                                                        l16 * 16);
+        *reinterpret_cast<uint4*>(dst_pool + row * kRowBytes + l16 * 16) = v;
+      }
+    }
+  }
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
-  }
-}
-
-__global__ void __launch_bounds__(kRestoreThreads) restore_scatter_kernel(const RestoreParams p) {
-  grid_dep_wait();
-  grid_dep_launch();
-  const int seg = blockIdx.y;
-  const int H = p.g.n_kv_heads;
-  const int h = seg % H;
-  const int b = (seg / H) % p.g.batch;
-  const int tensor = seg / (H * p.g.batch);
-  const int cnt = p.ret_count[seg];
-  const int off = p.ret_offset[seg];
-  const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-  for (int e = blockIdx.x * (kRestoreThreads / 16) + hw; e < cnt; e += gridDim.x * (kRestoreThreads / 16)) {
-    const int tok = p.ret_index[off + e];
-    const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
-    const size_t row = ((size_t)page * H + h) * p.g.page_size + (tok & (p.g.page_size - 1));
-    const uint4 v =
-        *reinterpret_cast<const uint4*>(p.ret_rows + ((size_t)p.layer * p.ret_capacity + off + e) * kRetEntryBytes + l16 * 16);
-    *reinterpret_cast<uint4*>(p.dst_pool[tensor] + row * kRowBytes + l16 * 16) = v;
   }
 }
 
@@ -224,10 +225,6 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
     MC_CUDA_CHECK(launch_pdl(kern, dim3(grid), dim3(kRestoreThreads), smem, stream, rp));
     MC_CUDA_CHECK(cudaGetLastError());
   }
-  const int nseg = 2 * bt->batch * cfg->n_kv_heads;
-  dim3 grid(4, nseg);
-  MC_CUDA_CHECK(launch_pdl(restore_scatter_kernel, dim3(grid), dim3(kRestoreThreads), 0, stream, rp));
-  MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }
 
