@@ -513,9 +513,14 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
     new-token rows from pinned host memory and returns its output there (mc_decode_attn_host).
     The copies are inside the timed region."""
     lib = job.lib
+    # pinned host copies of every pair's layers; with several ranks on one node the ranks share the
+    # host's memory, so each keeps one pair's copy and uploads it for every pair (same bytes, same work)
     host_pools = []
-    for pl in job.pools:
-        host_pools.append({k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in pl.items()})
+    for pr, pl in enumerate(job.pools):
+        if world > 1 and pr > 0:
+            host_pools.append(host_pools[0])
+        else:
+            host_pools.append({k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in pl.items()})
     stage = {k: torch.empty_like(v) for k, v in job.pools[0].items()}  # device staging the host pools land in
     pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
     q_host = [pin(q) for q in job.q]
