@@ -100,13 +100,18 @@ class Job:
         self.mc, self.lib, self.wl, self.dev, self.q4 = mc, mc.lib(), wl, device, q4
         self.B, self.S, self.H, self.Hq, self.ps = wl.batch, wl.seq_len, wl.n_kv_heads, wl.n_q_heads, wl.page_size
         self.steps = wl.decode_steps
-        prompt, _ = gen.make_lengths(wl)
+        prompt, gen_len = gen.make_lengths(wl)
         self.prompt = prompt
+        # the serving mix drains: a sequence leaves the batch after its own number of generated tokens
+        # (its length is set to 0: an empty sequence costs one empty work unit per head and nothing else)
+        self.gen_len = np.minimum(gen_len, self.steps) if wl.ragged else np.full(wl.batch, self.steps, np.int64)
         cap = prompt + self.steps + 1
         bt, self.n_pages = gen.make_block_table(cap, self.ps, seed=4321 + wl.index)
         self.block_table = torch.from_numpy(bt).to(device)
         self.seq0 = torch.from_numpy(prompt.copy()).to(device)
         self.seq_lens = self.seq0.clone()
+        self.gen_dev = torch.from_numpy(np.asarray(self.gen_len, np.int32)).to(device)
+        self.step_dev = torch.zeros(1, dtype=torch.int32, device=device)  # decode steps done since the merge
         self.cfg = mc.McConfig(self.H, self.Hq, self.ps, wl.dtype, t=wl.t, gamma=wl.gamma)
         self.max_prefill = int(prompt.max())
         self.tok_heads = int(prompt.sum()) * self.H  # (token, kv head) rows per layer and tensor
@@ -169,6 +174,7 @@ class Job:
     # -- phases ---------------------------------------------------------------------------------
     def merge_all(self):
         self.seq_lens.copy_(self.seq0)
+        self.step_dev.zero_()
         b = self.batch(False)
         for pr in range(self.wl.n_pairs):
             pl = self.pools[pr]
@@ -208,7 +214,7 @@ class Job:
                     e1.record()
                     self.attn_events.append((e0, e1, s))
                 self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
-            self.seq_lens += 1
+            self._advance()
         self.launches += steps * self.wl.n_pairs * 5
 
     def capture_decode_step(self):
@@ -241,7 +247,20 @@ class Job:
                 self.lib.mc_decode_attn(self.cfg, b, pc, 2, q, n2["k"], n2["v"], self.sm_scale, self.out2, None,
                                         self.ws_attn2)
                 self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
-            self.seq_lens += 1
+            self._advance()
+
+    def _advance(self):
+        """End of a decode step, on the device: every live sequence grows by one token, a sequence that
+        has generated its share leaves (length 0)."""
+        self.seq_lens += 1
+        if self.wl.ragged:
+            self.step_dev += 1
+            self.seq_lens.mul_((self.gen_dev > self.step_dev).to(torch.int32))
+
+    def live_token_heads(self, s: int) -> int:
+        """(token, kv head) rows attended at decode step s (0-based): the live sequences' prompt + s."""
+        live = self.gen_len > s
+        return int((self.prompt[live].astype(np.int64) + s).sum()) * self.H
 
     def step(self, sample_events=False):
         self.merge_all()
@@ -258,15 +277,14 @@ class Job:
         in_row = 64 + 16 if self.q4 else ROW  # 4-bit codes + the row's share of the group meta
         merge = npairs * 2 * th * (2 * in_row + ROW + 12 + 4 + rho * (2 * in_row + 2 * ROW + 4))
         restore = npairs * 2 * 2 * th * (2 * ROW + 4 + rho * 2 * ROW)
-        # decode: token-heads grow by batch*H per step
-        th_steps = steps * th + self.B * self.H * steps * (steps - 1) // 2
+        # decode: every live sequence grows by one token per step
+        th_steps = sum(self.live_token_heads(s) for s in range(steps))
         attn = npairs * 2 * th_steps * (2 * ROW + 8 + 2 * rho * (ROW + 4))
-        append = npairs * steps * 2 * self.B * self.H * (3 * ROW + 12)
+        append = npairs * 2 * int(np.minimum(self.gen_len, steps).sum()) * self.H * (3 * ROW + 12)
         return {"merge": merge, "restore": restore, "attn": attn, "append": append}
 
     def attn_bytes_at(self, s: int, rho: float):
-        th = self.tok_heads + self.B * self.H * s
-        return th * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+        return self.live_token_heads(s) * (2 * ROW + 8 + 2 * rho * (ROW + 4))
 
 
 def max_over_ranks(seconds: float, dist, device) -> float:
@@ -438,7 +456,7 @@ def main():
     t_r = timed(job.restore_all)
     phases["restore"] = {"ms": t_r * 1e3, "GB/s": by["restore"] / t_r / 1e9}
     t_d = timed(job.decode_all)
-    tok_steps = job.steps * float(job.prompt.sum()) + job.B * job.steps * (job.steps - 1) / 2
+    tok_steps = sum(job.live_token_heads(s) for s in range(job.steps)) / job.H
     phases["decode"] = {"ms": t_d * 1e3, "GB/s": (by["attn"] + by["append"]) / t_d / 1e9,
                         "kv_tokens_per_s": tok_steps * 2 * wl.n_pairs / t_d, "ms_per_decode_step": t_d * 1e3 / job.steps}
     # the same decode phase replayed from a CUDA graph of one decode step (valid for any step: the
@@ -461,10 +479,10 @@ def main():
         job.decode_pair_all(min(2, psteps))  # warm-up
         job.merge_all()
         t_p = timed(lambda: job.decode_pair_all(psteps))
-        th_steps = psteps * job.tok_heads + job.B * job.H * psteps * (psteps - 1) // 2
+        th_steps = sum(job.live_token_heads(s) for s in range(psteps))
         pair_bytes = wl.n_pairs * th_steps * (2 * ROW + 16 + 4 * rho * (ROW + 4)) + by["append"] * psteps / job.steps
         phases["decode_pair_mode"] = {"ms_per_decode_step": t_p * 1e3 / psteps, "GB/s": pair_bytes / t_p / 1e9,
-                                      "kv_tokens_per_s": (psteps * float(job.prompt.sum()) + job.B * psteps * (psteps - 1) / 2)
+                                      "kv_tokens_per_s": (th_steps / job.H)
                                       * 2 * wl.n_pairs / t_p, "steps": psteps}
     peak0, _ = measured_hbm_peak()
     for ph in phases.values():
@@ -562,6 +580,7 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
         cs = pair_sets[k % 2]
         main_s.wait_event(merged[k % 2])
         job.seq_lens.copy_(job.seq0)
+        job.step_dev.zero_()
         for s in range(job.steps):
             q, nt = q_host[s % len(q_host)], new_host[s % len(new_host)]
             ntd = job.new[s % len(job.new)]
@@ -573,7 +592,7 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
                     lib.mc_decode_attn_host(job.cfg, bd, pc, layer, q[layer], kn, vn, job.sm_scale, out_host, None,
                                             io, job.ws_attn)
                 lib.mc_append_pair(job.cfg, bd, pc, ntd["k_lm1"], ntd["v_lm1"], ntd["k_l"], ntd["v_l"])
-            job.seq_lens += 1
+            job._advance()
         ev = torch.cuda.Event()
         ev.record(main_s)
         decoded[k % 2] = ev
