@@ -30,7 +30,7 @@
  *   at row i % page_size.
  * - The kernels are chained with programmatic dependent launch.  The batch description
  *   (block_table, seq_lens) and the queries are never written by this library, so
- *   mc_decode_attn reads them before it waits for the kernel ahead of it in the stream; a
+ *   mc_decode_attn and mc_append_pair read them before they wait for the kernel ahead in the stream; a
  *   caller whose own kernels let dependents start early must have them written before that.
  * - Argument errors are reported synchronously through the return code and
  *   launch nothing.  Data-dependent conditions (retained-row pool too small,

@@ -842,7 +842,6 @@ struct AppendParams {
 
 template <int DT>
 __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
-  grid_dep_wait();
   grid_dep_launch();
   const int r = blockIdx.x * (128 / 16) + (threadIdx.x >> 4);
   const int l16 = threadIdx.x & 15;
@@ -852,6 +851,11 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   const int h = rr % H;
   const int b = (rr / H) % p.g.batch;
   const int tensor = rr / (H * p.g.batch);
+  // the batch description belongs to the caller (no kernel of this library writes it): where the row
+  // goes is looked up before the wait on the kernel ahead in the stream
+  const int tok = p.g.seq_lens[b];
+  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+  grid_dep_wait();
   uint4 va = make_uint4(0, 0, 0, 0), vc = va;
   if (ok) {
     const size_t off = ((size_t)b * H + h) * kRowBytes + l16 * 16;
@@ -862,8 +866,6 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   float ga, gc, d;
   merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, ga, gc, d);
   if (!ok) return;
-  const int tok = p.g.seq_lens[b];
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
   const int tk = tok & (p.g.page_size - 1);
   const size_t ph = (size_t)page * H + h;
   char* tile = p.e_pool[tensor] + ph * tile_bytes(p.g.page_size);
