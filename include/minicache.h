@@ -16,6 +16,8 @@
  *
  * General conventions
  * -------------------
+ * - The device that is current when a call is made must be the one that owns `stream` and the
+ *   buffers.
  * - Every pointer inside the structs below is DEVICE memory owned by the caller
  *   unless a comment says "host".  The library never allocates or frees device
  *   memory.  Struct arguments themselves live in host memory and are read
@@ -52,7 +54,8 @@ typedef enum {
   MC_OK = 0,
   MC_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum value */
   MC_ERR_SHAPE = 2,       /* head_dim != 128, page_size not 16/32/64, head ratio not supported,
-                             batch above 1024 (merge) or 512 (decode attention) */
+                             batch above 1024 (merge, restore) or 512 (decode attention), or more than
+                             65535 segments (2 * batch * n_kv_heads) */
   MC_ERR_DTYPE = 3,
   MC_ERR_ALIGN = 4,       /* a pool base is not 256-byte aligned */
   MC_ERR_CAPACITY = 5,    /* workspace too small / retained pool overflowed (from mc_read_status) */
@@ -88,14 +91,22 @@ typedef enum mc_merge_fn { MC_MERGE_SLERP = 0, MC_MERGE_FMAX = 1, MC_MERGE_MEAN 
 
 /* Status word indices (mc_read_status). */
 enum {
-  MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out */
+  MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out;
+                                   bit 2: a length or page id outside the declared bounds was met */
   MC_STATUS_RETAINED_TOTAL = 1, /* retained entries the last merge selected (K and V segments together) */
-  MC_STATUS_RESERVED0 = 2,
+  MC_STATUS_NEAR_THRESHOLD = 2, /* tokens of the last merge whose distance lies within 1e-6 of their segment's
+                                   retention threshold (a differently rounded d could have decided them the
+                                   other way) */
   MC_STATUS_RESERVED1 = 3,
   MC_STATUS_WORDS = 4
 };
 #define MC_FLAG_RETAIN_OVERFLOW 1
 #define MC_FLAG_WAIT_TIMEOUT 2
+/* A kernel met a seq_lens entry outside [0, max_seq_len] or a page id outside [0, n_pages) (or a
+ * token position past max_pages_per_seq pages).  Such a value is never turned into an address: the
+ * length is clamped, the page's rows are not written (merge, restore, append) or page 0 is read in
+ * its place (decode attention: the result of that sequence is then meaningless). */
+#define MC_FLAG_BAD_METADATA 4
 
 /* Method parameters and tensor geometry (Sec. 4.1-4.2, Sec. 5 defaults t = 0.6, gamma = 0.05). */
 typedef struct mc_config {
@@ -185,6 +196,49 @@ typedef struct mc_pair_cache {
   int32_t* status;
 } mc_pair_cache;
 
+/* Byte sizes of the buffers of one mc_pair_cache (Sec. 4.2: the shared cache C of a layer pair) for
+ * cfg, batch->batch, batch->n_pages, batch->max_seq_len (the longest sequence at merge time) and a
+ * retained-row pool of ret_capacity entries.  e_bytes is the size of e_k and of e_v alike. */
+typedef struct mc_pair_sizes {
+  size_t tile_bytes;        /* one (page, head) tile of e_k / e_v */
+  size_t e_bytes;
+  size_t dist_bytes;
+  size_t ret_count_bytes;
+  size_t ret_offset_bytes;
+  size_t ret_index_bytes;
+  size_t ret_rows_bytes;
+  size_t ret_prefix_bytes;
+  size_t seg_minmax_bytes;
+  size_t status_bytes;
+  int64_t ret_prefix_stride; /* value for mc_pair_cache.ret_prefix_stride */
+  size_t total_bytes;        /* all buffers, each rounded up to 256 bytes */
+} mc_pair_sizes;
+
+/* What the last merge into a pair did (Sec. 4.2 retention, Sec. 4.3 footprint). */
+typedef struct mc_stats {
+  int32_t flags;            /* MC_STATUS_FLAGS */
+  int32_t reserved;
+  int64_t retained_total;   /* retained entries, K and V segments together */
+  int64_t near_threshold;   /* tokens with |d - threshold| < 1e-6 (MC_STATUS_NEAR_THRESHOLD) */
+  int64_t token_heads;      /* (token, kv head) rows per layer and tensor = sum(seq_lens) * n_kv_heads */
+  int64_t full_bytes;       /* the two layers' K and V uncompressed: 4 * token_heads * 256 */
+  int64_t compressed_bytes; /* first-principles size of the shared cache: per (token, head, tensor) one
+                               direction row, two magnitudes and the distance; per retained entry both raw
+                               rows and the index (Sec. 4.3 counts the same items) */
+  int64_t stored_bytes;     /* what the pair occupies in this library's layout: whole tiles of the pages in
+                               use, padded retained entries, per-segment tables */
+} mc_stats;
+
+/* Pure host arithmetic; no device work.  (The paper has no counterpart: buffer planning.) */
+mc_status mc_pair_bytes(const mc_config* cfg, const mc_batch* batch, int64_t ret_capacity, mc_pair_sizes* out);
+
+/* Reads the pair's status words and the batch's lengths after synchronising `stream` and fills `out`.
+ * Returns like mc_read_status (MC_ERR_CAPACITY / MC_ERR_DEVICE_STATUS when a flag is set; `out` is
+ * filled either way).  batch->seq_lens must be the lengths the pair was merged at for the byte
+ * counts to describe that merge. */
+mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, void* stream,
+                       mc_stats* out);
+
 /* Library version (major * 10000 + minor * 100 + patch). No device work. */
 int32_t mc_version(void);
 
@@ -231,10 +285,13 @@ mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_p
                          const void* v_new_l, void* stream);
 
 /* Eq. 2 + Sec. 4.2 "Cache restoration": writes the dense restored K and V of one layer
- * (layer_sel = MC_LAYER_LM1 or MC_LAYER_L) into dst pools of the same paged layout and type:
- * x_hat = e * scale, then retained rows overwritten with their raw copies. */
+ * (layer_sel = MC_LAYER_LM1 or MC_LAYER_L) into dst pools of the same paged layout:
+ * x_hat = e * scale, then retained rows overwritten with their raw copies.
+ * dst_fp32 == 0: dst pools hold cfg->dtype (the product is rounded once to it).
+ * dst_fp32 != 0: dst pools are [n_pages][n_kv_heads][page_size][128] binary32: the product as
+ *                computed, raw rows converted exactly. */
 mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
-                     int32_t layer_sel, const mc_layer_kv* dst, void* stream);
+                     int32_t layer_sel, const mc_layer_kv* dst, int32_t dst_fp32, void* stream);
 
 /* Algorithm 2 "MiniCache Decoding": single-query attention of every sequence over the restored
  * cache of one layer, computed straight from the compressed pair (restore fused; the dense K/V
@@ -294,7 +351,8 @@ mc_status mc_decode_io_bytes(const mc_config* cfg, const mc_batch* batch, int32_
  *   mc_workspace_bytes(MC_OP_DECODE_ATTN) reports) is refused with MC_ERR_CAPACITY before anything
  *   is launched; mc_last_cuda_error() then names both sizes.
  * - The first call on each device looks up the array's device address (one runtime query, no
- *   allocation).  Make that first call outside any stream capture.
+ *   allocation).  Make that first call outside any stream capture.  The array used is the one of
+ *   the device that is current when the call is made: `stream` must belong to that device.
  * - All calls on a device share the one array.  Nothing in it has to start at zero: every slot a
  *   call reads was written earlier by the same call.  But two calls that may run at the same time
  *   on the GPU (different streams, no ordering between them) overwrite each other's partials:

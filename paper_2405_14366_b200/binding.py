@@ -17,7 +17,8 @@ MC_RETAIN_DISTINCT, MC_RETAIN_LITERAL, MC_RETAIN_TOPK = 0, 1, 2
 MC_LAYER_LM1, MC_LAYER_L, MC_LAYER_BOTH = 0, 1, 2
 MC_OP_MERGE, MC_OP_DECODE_ATTN = 0, 1
 MC_STATUS_WORDS = 4
-MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT = 1, 2
+MC_STATUS_FLAGS, MC_STATUS_RETAINED_TOTAL, MC_STATUS_NEAR_THRESHOLD = 0, 1, 2
+MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT, MC_FLAG_BAD_METADATA = 1, 2, 4
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libminicache.so")
 
@@ -57,7 +58,20 @@ class _PairCache(C.Structure):
                 ("status", C.c_void_p)]
 
 
-EXPORTS = ("mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+class _PairSizes(C.Structure):
+    _fields_ = [("tile_bytes", C.c_size_t), ("e_bytes", C.c_size_t), ("dist_bytes", C.c_size_t),
+                ("ret_count_bytes", C.c_size_t), ("ret_offset_bytes", C.c_size_t), ("ret_index_bytes", C.c_size_t),
+                ("ret_rows_bytes", C.c_size_t), ("ret_prefix_bytes", C.c_size_t), ("seg_minmax_bytes", C.c_size_t),
+                ("status_bytes", C.c_size_t), ("ret_prefix_stride", C.c_int64), ("total_bytes", C.c_size_t)]
+
+
+class _Stats(C.Structure):
+    _fields_ = [("flags", C.c_int32), ("reserved", C.c_int32), ("retained_total", C.c_int64),
+                ("near_threshold", C.c_int64), ("token_heads", C.c_int64), ("full_bytes", C.c_int64),
+                ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
+
+
+EXPORTS = ("mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -116,24 +130,27 @@ class PairCache:
     def __init__(self, cfg: McConfig, batch: int, n_pages: int, ret_capacity: int, device="cuda",
                  max_merge_len: Optional[int] = None):
         H, ps = cfg.n_kv_heads, cfg.page_size
-        dt = cfg.torch_dtype
         self.cfg = cfg
-        self.tile_bytes = ps * 256 + 2 * ps * 4
-        self.e_k = torch.zeros(n_pages, H, self.tile_bytes, dtype=torch.uint8, device=device)
-        self.e_v = torch.zeros(n_pages, H, self.tile_bytes, dtype=torch.uint8, device=device)
-        self.dist = torch.zeros(n_pages, H, 2, ps, dtype=torch.float32, device=device)
-        nseg = 2 * batch * H
-        self.ret_count = torch.zeros(nseg, dtype=torch.int32, device=device)
-        self.ret_offset = torch.zeros(nseg + 1, dtype=torch.int32, device=device)
-        self.ret_index = torch.zeros(max(ret_capacity, 1), dtype=torch.int32, device=device)
-        self.ret_rows = torch.zeros(2, max(ret_capacity, 1), 272, dtype=torch.uint8, device=device)
-        self.ret_capacity = int(ret_capacity)
         if max_merge_len is None:  # bound of the sequence length at merge time: what the pages can hold at most
             max_merge_len = n_pages * ps
-        self.ret_prefix_stride = (int(max_merge_len) + 127) // 128 + 1
-        self.ret_prefix = torch.zeros(nseg, self.ret_prefix_stride, dtype=torch.int32, device=device)
-        self.seg_minmax = torch.zeros(nseg, 2, dtype=torch.float32, device=device)
-        self.status = torch.zeros(MC_STATUS_WORDS, dtype=torch.int32, device=device)
+        cap = max(int(ret_capacity), 1)
+        sz = lib().mc_pair_bytes(cfg, batch, n_pages, int(max_merge_len), cap)  # every size comes from the library
+        self.sizes = sz
+        self.tile_bytes = sz.tile_bytes
+        nseg = 2 * batch * H
+        z = lambda nbytes: torch.zeros(nbytes, dtype=torch.uint8, device=device)
+        self.e_k = z(sz.e_bytes).view(n_pages, H, self.tile_bytes)
+        self.e_v = z(sz.e_bytes).view(n_pages, H, self.tile_bytes)
+        self.dist = z(sz.dist_bytes).view(torch.float32).view(n_pages, H, 2, ps)
+        self.ret_count = z(sz.ret_count_bytes).view(torch.int32)
+        self.ret_offset = z(sz.ret_offset_bytes).view(torch.int32)
+        self.ret_index = z(sz.ret_index_bytes).view(torch.int32)
+        self.ret_rows = z(sz.ret_rows_bytes).view(2, cap, 272)
+        self.ret_capacity = int(ret_capacity)
+        self.ret_prefix_stride = int(sz.ret_prefix_stride)
+        self.ret_prefix = z(sz.ret_prefix_bytes).view(torch.int32).view(nseg, self.ret_prefix_stride)
+        self.seg_minmax = z(sz.seg_minmax_bytes).view(torch.float32).view(nseg, 2)
+        self.status = z(sz.status_bytes).view(torch.int32)
 
     def c(self) -> _PairCache:
         return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.dist), _ptr(self.ret_count),
@@ -195,7 +212,11 @@ class MiniCacheLib:
         L.mc_merge_pair.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_PairCache), C.c_int32, V,
                                     C.c_size_t, V]
         L.mc_append_pair.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, V, V, V, V]
-        L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), V]
+        L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), C.c_int32, V]
+        L.mc_pair_bytes.argtypes = [P(_Config), P(_Batch), C.c_int64, P(_PairSizes)]
+        L.mc_pair_bytes.restype = C.c_int32
+        L.mc_get_stats.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, P(_Stats)]
+        L.mc_get_stats.restype = C.c_int32
         L.mc_decode_attn.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V,
                                      C.c_size_t, V]
         L.mc_read_status.argtypes = [P(_PairCache), V, P(C.c_int32)]
@@ -263,9 +284,28 @@ class MiniCacheLib:
                                              _ptr(k_new_l), _ptr(v_new_l), _stream(stream)))
 
     def mc_restore(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, dst_k, dst_v, stream=None):
+        """dst_k / dst_v: pools in the storage type, or float32 pools (then the unrounded products are written)."""
         c, b, pc = cfg.c(), batch.c(), pair.c()
         d = _LayerKV(_ptr(dst_k), _ptr(dst_v))
-        self._check(self._lib.mc_restore(C.byref(c), C.byref(b), C.byref(pc), layer_sel, C.byref(d), _stream(stream)))
+        assert dst_k.dtype == dst_v.dtype and dst_k.dtype in (torch.float32, cfg.torch_dtype)
+        f32 = 1 if dst_k.dtype == torch.float32 else 0
+        self._check(self._lib.mc_restore(C.byref(c), C.byref(b), C.byref(pc), layer_sel, C.byref(d), f32, _stream(stream)))
+
+    def mc_pair_bytes(self, cfg: McConfig, batch: int, n_pages: int, max_seq_len: int, ret_capacity: int) -> _PairSizes:
+        c = cfg.c()
+        b = _Batch(None, None, int(batch), 0, int(max_seq_len), 0, int(n_pages))
+        out = _PairSizes()
+        self._check(self._lib.mc_pair_bytes(C.byref(c), C.byref(b), int(ret_capacity), C.byref(out)))
+        return out
+
+    def mc_get_stats(self, cfg: McConfig, batch: Batch, pair: PairCache, stream=None, check: bool = True):
+        """(dict of the mc_stats fields, return code); synchronises the stream."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        out = _Stats()
+        code = self._lib.mc_get_stats(C.byref(c), C.byref(b), C.byref(pc), _stream(stream), C.byref(out))
+        if check:
+            self._check(code)
+        return {f: getattr(out, f) for f, _ in _Stats._fields_ if f != "reserved"}, code
 
     def mc_decode_attn(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q, k_new, v_new,
                        sm_scale: float, out, lse, workspace: torch.Tensor, stream=None):

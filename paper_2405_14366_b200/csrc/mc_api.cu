@@ -2,7 +2,11 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+#include <vector>
+
 #include "mc_common.cuh"
+#include "mc_items.cuh"
 #include "mc_kernels.h"
 
 namespace mc {
@@ -12,6 +16,20 @@ static thread_local char g_cuda_error[256] = "";
 void set_cuda_error(cudaError_t e, const char* where) {
   snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
   (void)cudaGetLastError();  // clear the sticky-free error state
+}
+
+mc_status sm_count(int* n_sm) {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cache[kMaxDev];  // zero-initialised; 0 = not looked up yet
+  int dev = 0;
+  MC_CUDA_CHECK(cudaGetDevice(&dev));
+  int v = (dev >= 0 && dev < kMaxDev) ? cache[dev].load(std::memory_order_relaxed) : 0;
+  if (v == 0) {
+    MC_CUDA_CHECK(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+    if (dev >= 0 && dev < kMaxDev) cache[dev].store(v, std::memory_order_relaxed);
+  }
+  *n_sm = v;
+  return MC_OK;
 }
 
 static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -61,6 +79,8 @@ static Geom make_geom(const mc_config* cfg, const mc_batch* bt) {
   g.n_kv_heads = cfg->n_kv_heads;
   g.page_size = cfg->page_size;
   g.page_shift = cfg->page_size == 16 ? 4 : (cfg->page_size == 32 ? 5 : 6);
+  g.max_seq_len = bt->max_seq_len;
+  g.n_pages = (int)bt->n_pages;
   return g;
 }
 
@@ -70,7 +90,7 @@ using namespace mc;
 
 extern "C" {
 
-int32_t mc_version(void) { return 100; }
+int32_t mc_version(void) { return 200; }
 
 const char* mc_status_str(int32_t s) {
   switch (s) {
@@ -106,6 +126,86 @@ mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_
   return MC_OK;
 }
 
+// What every form of the merge call checks about the output pair and the scratch memory.
+static mc_status check_merge_common(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* out, void* workspace,
+                                    size_t workspace_bytes) {
+  mc_status st = check_pair(out);
+  if (st != MC_OK) return st;
+  if (batch->batch > kMaxBatchPages) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
+  if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
+  return MC_OK;
+}
+
+mc_status mc_pair_bytes(const mc_config* cfg, const mc_batch* batch, int64_t ret_capacity, mc_pair_sizes* out) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (batch == nullptr || out == nullptr) return MC_ERR_INVALID_ARG;
+  if (batch->batch < 0 || batch->max_seq_len < 0 || batch->n_pages < 0 || ret_capacity < 0) return MC_ERR_INVALID_ARG;
+  const size_t nseg = (size_t)2 * batch->batch * cfg->n_kv_heads;
+  const size_t ph = (size_t)batch->n_pages * cfg->n_kv_heads;
+  memset(out, 0, sizeof(*out));
+  out->tile_bytes = (size_t)tile_bytes(cfg->page_size);
+  out->e_bytes = ph * out->tile_bytes;
+  out->dist_bytes = ph * 2 * cfg->page_size * sizeof(float);
+  out->ret_count_bytes = nseg * sizeof(int32_t);
+  out->ret_offset_bytes = (nseg + 1) * sizeof(int32_t);
+  out->ret_index_bytes = (size_t)ret_capacity * sizeof(int32_t);
+  out->ret_rows_bytes = (size_t)2 * ret_capacity * kRetEntryBytes;
+  out->ret_prefix_stride = (batch->max_seq_len + 127) / 128 + 1;
+  out->ret_prefix_bytes = nseg * (size_t)out->ret_prefix_stride * sizeof(int32_t);
+  out->seg_minmax_bytes = nseg * 2 * sizeof(float);
+  out->status_bytes = MC_STATUS_WORDS * sizeof(int32_t);
+  const size_t parts[] = {out->e_bytes, out->e_bytes, out->dist_bytes, out->ret_count_bytes, out->ret_offset_bytes,
+                          out->ret_index_bytes, out->ret_rows_bytes, out->ret_prefix_bytes, out->seg_minmax_bytes,
+                          out->status_bytes};
+  for (size_t b : parts) out->total_bytes += align_up(b, 256);
+  return MC_OK;
+}
+
+mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, void* stream,
+                       mc_stats* out) {
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  if (pair == nullptr || pair->status == nullptr || out == nullptr) return MC_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t words[MC_STATUS_WORDS];
+  std::vector<int32_t> lens_v((size_t)batch->batch + 1);
+  int32_t* lens = lens_v.data();
+  MC_CUDA_CHECK(cudaMemcpyAsync(words, pair->status, sizeof(words), cudaMemcpyDeviceToHost, s));
+  if (batch->batch > 0)
+    MC_CUDA_CHECK(cudaMemcpyAsync(lens, batch->seq_lens, (size_t)batch->batch * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  MC_CUDA_CHECK(cudaStreamSynchronize(s));
+  int64_t tokens = 0, pages = 0;
+  for (int b = 0; b < batch->batch; ++b) {
+    const int64_t n = lens[b] < 0 ? 0 : lens[b];
+    tokens += n;
+    pages += (n + cfg->page_size - 1) / cfg->page_size;
+  }
+  const int64_t th = tokens * cfg->n_kv_heads;  // (token, kv head) rows per layer and tensor
+  out->flags = words[MC_STATUS_FLAGS];
+  out->retained_total = words[MC_STATUS_RETAINED_TOTAL];
+  out->near_threshold = words[MC_STATUS_NEAR_THRESHOLD];
+  out->token_heads = th;
+  out->full_bytes = 2 * 2 * th * kRowBytes;  // two layers, K and V
+  // the shared direction row, both magnitudes and the distance per (token, head, tensor); both raw rows
+  // and the index per retained entry
+  out->compressed_bytes = 2 * th * (kRowBytes + 3 * 4) + out->retained_total * (2 * kRowBytes + 4);
+  // what the pair occupies in the caller's buffers: whole tiles of the pages in use, the distances, the
+  // padded retained entries, the per-segment tables
+  const int64_t nseg = 2LL * batch->batch * cfg->n_kv_heads;
+  out->stored_bytes = 2 * pages * cfg->n_kv_heads * ((int64_t)tile_bytes(cfg->page_size) + cfg->page_size * 4) +
+                      out->retained_total * (2 * kRetEntryBytes + 4) +
+                      nseg * (4 + 4 + 8 + 4 * pair->ret_prefix_stride) + 4 + MC_STATUS_WORDS * 4;
+  if (out->flags & MC_FLAG_RETAIN_OVERFLOW) return MC_ERR_CAPACITY;
+  if (out->flags != 0) return MC_ERR_DEVICE_STATUS;
+  return MC_OK;
+}
+
 mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1, const mc_layer_kv* l,
                         const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
                         void* stream) {
@@ -113,14 +213,11 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
   if (st != MC_OK) return st;
-  st = check_pair(out);
-  if (st != MC_OK) return st;
   if (!lm1 || !l || !lm1->k_pool || !lm1->v_pool || !l->k_pool || !l->v_pool) return MC_ERR_INVALID_ARG;
   if (!aligned256(lm1->k_pool) || !aligned256(lm1->v_pool) || !aligned256(l->k_pool) || !aligned256(l->v_pool))
     return MC_ERR_ALIGN;
-  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
-  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
-  if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
+  st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
+  if (st != MC_OK) return st;
   return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, nullptr, nullptr, out, do_retention ? 1 : 0, workspace,
                       (cudaStream_t)stream);
 }
@@ -133,17 +230,14 @@ mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc
   if (cfg->page_size != 32) return MC_ERR_SHAPE;
   st = check_batch(cfg, batch);
   if (st != MC_OK) return st;
-  st = check_pair(out);
-  if (st != MC_OK) return st;
   if (!lm1 || !l) return MC_ERR_INVALID_ARG;
   const void* ptrs[8] = {lm1->k_codes, lm1->k_meta, lm1->v_codes, lm1->v_meta, l->k_codes, l->k_meta, l->v_codes, l->v_meta};
   for (const void* q : ptrs) {
     if (q == nullptr) return MC_ERR_INVALID_ARG;
     if (!aligned256(q)) return MC_ERR_ALIGN;
   }
-  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
-  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
-  if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
+  st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
+  if (st != MC_OK) return st;
   return launch_merge(cfg, batch, make_geom(cfg, batch), nullptr, nullptr, lm1, l, out, do_retention ? 1 : 0, workspace,
                       (cudaStream_t)stream);
 }
@@ -164,7 +258,7 @@ mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_p
 }
 
 mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
-                     const mc_layer_kv* dst, void* stream) {
+                     const mc_layer_kv* dst, int32_t dst_fp32, void* stream) {
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -174,7 +268,8 @@ mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_
   if (layer_sel != MC_LAYER_LM1 && layer_sel != MC_LAYER_L) return MC_ERR_INVALID_ARG;
   if (!dst || !dst->k_pool || !dst->v_pool) return MC_ERR_INVALID_ARG;
   if (!aligned256(dst->k_pool) || !aligned256(dst->v_pool)) return MC_ERR_ALIGN;
-  return launch_restore(cfg, batch, make_geom(cfg, batch), pair, layer_sel, dst, (cudaStream_t)stream);
+  if (batch->batch > kMaxBatchPages) return MC_ERR_SHAPE;
+  return launch_restore(cfg, batch, make_geom(cfg, batch), pair, layer_sel, dst, dst_fp32 ? 1 : 0, (cudaStream_t)stream);
 }
 
 mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
@@ -209,6 +304,11 @@ mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const 
   if (!host_lm1 || !host_l || !dev_lm1 || !dev_l) return MC_ERR_INVALID_ARG;
   if (!host_lm1->k_pool || !host_lm1->v_pool || !host_l->k_pool || !host_l->v_pool) return MC_ERR_INVALID_ARG;
   if (!dev_lm1->k_pool || !dev_lm1->v_pool || !dev_l->k_pool || !dev_l->v_pool) return MC_ERR_INVALID_ARG;
+  // every check of mc_merge_pair before the first copy: an argument error enqueues nothing
+  st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
+  if (st != MC_OK) return st;
+  if (!aligned256(dev_lm1->k_pool) || !aligned256(dev_lm1->v_pool) || !aligned256(dev_l->k_pool) || !aligned256(dev_l->v_pool))
+    return MC_ERR_ALIGN;
   const size_t pool_bytes = (size_t)batch->n_pages * cfg->n_kv_heads * cfg->page_size * kRowBytes;
   cudaStream_t s = (cudaStream_t)stream;
   MC_CUDA_CHECK(cudaMemcpyAsync(dev_lm1->k_pool, host_lm1->k_pool, pool_bytes, cudaMemcpyHostToDevice, s));

@@ -293,7 +293,14 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int b = tid; b < p.g.batch; b += kAttnThreads) len_s[b] = p.g.seq_lens[b];
+  // (a length above the declared bound is clamped here, so that a sequence never owns more units than
+  // it has partial slots, and flagged once the status words may be touched)
+  int bad_meta = 0;
+  for (int b = tid; b < p.g.batch; b += kAttnThreads) {
+    const int n = p.g.seq_lens[b];
+    bad_meta |= (n < 0 || n > p.g.max_seq_len) ? 1 : 0;
+    len_s[b] = min(max(n, 0), p.g.max_seq_len);
+  }
   __syncthreads();
   if (tid == 0) {
     // prefix of the sequences' unit counts (a sequence always owns at least one unit)
@@ -330,10 +337,20 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       for (int r = 0; r < kMaxPiecePages / 32; ++r) {
         pg_reg[r] = 0;
         if (it.valid && lane + 32 * r < np) pg_reg[r] = row[lane + 32 * r];
+        // a page id outside the pools never becomes a copy's source address: page 0 is streamed
+        // instead and the call is flagged (its result for that sequence means nothing)
+        if (!page_ok(p.g, pg_reg[r])) {
+          pg_reg[r] = 0;
+          bad_meta = 1;
+        }
       }
     };
     load_pages(w);
     grid_dep_wait();
+    if (bad_meta) {
+      atomicOr(p.status, MC_FLAG_BAD_METADATA);
+      bad_meta = 0;
+    }
     raw = load_ranges(w, p);
     bool ok = true;
     int n_piece = 0;
@@ -346,6 +363,10 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       const Item wn = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
       const RawRanges rawn = load_ranges(wn, p);
       load_pages(wn);
+      if (bad_meta) {
+        atomicOr(p.status, MC_FLAG_BAD_METADATA);
+        bad_meta = 0;
+      }
       const int n_pages_item = (w.n_tok + ps - 1) >> shift;
       const int n_new = w.has_new ? 1 : 0;
       for (int ph = 0; ph < 2 && ok; ++ph) {
@@ -451,6 +472,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
   grid_dep_wait();
+  if (bad_meta) atomicOr(p.status, MC_FLAG_BAD_METADATA);
   consumer_sync();
 
   // carried from chunk to chunk of a piece: the output sums, this thread's part of the row sum, and
@@ -816,7 +838,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
   const int hq = blockIdx.x * R + warp / GP;
   int before = 0, all = 0;  // units of the sequences before this one, of all sequences
   for (int bb = tid; bb < p.g.batch; bb += kCombineThreads) {
-    const int ub = max(1, (p.g.seq_lens[bb] + kUnit - 1) / kUnit);
+    const int ub = max(1, (min(max(p.g.seq_lens[bb], 0), p.g.max_seq_len) + kUnit - 1) / kUnit);
     all += ub;
     if (bb < b) before += ub;
   }
@@ -836,7 +858,7 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
     before += sum_s[0][g];
     all += sum_s[1][g];
   }
-  const int u = max(1, (p.g.seq_lens[b] + kUnit - 1) / kUnit);
+  const int u = max(1, (min(max(p.g.seq_lens[b], 0), p.g.max_seq_len) + kUnit - 1) / kUnit);
   const long long n_units = all, x0 = before;
   const int n_teams = p.n_teams;
   // teams whose range [n_units c / T, n_units (c + 1) / T) meets [x0, x0 + u): consecutive, each with one piece
@@ -980,12 +1002,8 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.part_o = reinterpret_cast<float*>(workspace);
   ap.part_ml = reinterpret_cast<float*>((char*)workspace + align_up(prow * kHeadDim * 4, 256));
 
-  static int n_sm = 0;  // persistent grid: kCtasPerSm CTAs per SM of the current device
-  if (n_sm == 0) {
-    int dev = 0;
-    MC_CUDA_CHECK(cudaGetDevice(&dev));
-    MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-  }
+  int n_sm = 0;  // persistent grid: kCtasPerSm CTAs per SM of the current device
+  if (mc_status st = sm_count(&n_sm)) return st;
   // teams: S CTAs, each with ceil(H / S) kv heads; as many whole teams as fit two CTAs per SM,
   // and no more teams than there can be units
   const int slots_gpu = n_sm * kCtasPerSm;

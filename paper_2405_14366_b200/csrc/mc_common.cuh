@@ -60,7 +60,34 @@ struct Geom {
   int n_kv_heads;
   int page_size;
   int page_shift;  // log2(page_size)
+  int max_seq_len;  // the caller's bound of seq_lens: longer lengths are clamped to it and flagged
+  int n_pages;      // pages in every pool: page ids outside [0, n_pages) are never used as addresses
 };
+
+#if defined(__CUDACC__)
+// The batch description is the caller's and may be stale or wrong.  No kernel ever turns an
+// unchecked length or page id into an address: a length above the declared bound is clamped, a page
+// id outside the pools is replaced by page 0 for reads and skips the write, and either sets
+// MC_FLAG_BAD_METADATA in the pair's status words.
+__device__ __forceinline__ int checked_len(const Geom& g, int b, int32_t* status) {
+  const int n = g.seq_lens[b];
+  if (n < 0 || n > g.max_seq_len) {
+    atomicOr(status, MC_FLAG_BAD_METADATA);
+    return n < 0 ? 0 : g.max_seq_len;
+  }
+  return n;
+}
+__device__ __forceinline__ bool page_ok(const Geom& g, int page) { return (unsigned)page < (unsigned)g.n_pages; }
+// Page id of page slot `slot` of sequence `b`; -1 (and the flag) if the slot or the id is out of range.
+__device__ __forceinline__ int checked_page(const Geom& g, int b, int slot, int32_t* status) {
+  if ((unsigned)slot < (unsigned)g.max_pages_per_seq) {
+    const int page = g.block_table[(size_t)b * g.max_pages_per_seq + slot];
+    if (page_ok(g, page)) return page;
+  }
+  atomicOr(status, MC_FLAG_BAD_METADATA);
+  return -1;
+}
+#endif
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -15,9 +15,10 @@ struct PageItem {
 
 // Sequence lengths and the exclusive prefix of the sequences' page counts into shared memory
 // (len_s [batch], pre_s [batch + 1]); called by every thread of the CTA, ends with a barrier.
-__device__ __forceinline__ void page_prefix(const Geom& g, int* len_s, int* pre_s, int n_threads) {
+// Lengths above the declared bound are clamped to it (and flagged in `status`).
+__device__ __forceinline__ void page_prefix(const Geom& g, int* len_s, int* pre_s, int n_threads, int32_t* status) {
   const int tid = threadIdx.x, lane = tid & 31;
-  for (int b = tid; b < g.batch; b += n_threads) len_s[b] = g.seq_lens[b];
+  for (int b = tid; b < g.batch; b += n_threads) len_s[b] = checked_len(g, b, status);
   __syncthreads();
   if (tid < 32) {
     // a lane sums a run of sequences, the runs are scanned with shuffles

@@ -4,6 +4,9 @@
 
 namespace mc {
 
+// Multiprocessors of the current device (looked up once per device; the persistent grids are sized by it).
+mc_status sm_count(int* n_sm);
+
 size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt);
 mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
                        const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
@@ -12,7 +15,7 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
                         const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
                         cudaStream_t stream);
 mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
-                         int layer, const mc_layer_kv* dst, cudaStream_t stream);
+                         int layer, const mc_layer_kv* dst, int dst_fp32, cudaStream_t stream);
 
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets);
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,

@@ -282,23 +282,24 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  page_prefix(p.g, len_s, pre_s, kMergeThreads);
+  page_prefix(p.g, len_s, pre_s, kMergeThreads, p.status);
   const int* lens = len_s;
   const int P = pre_s[p.g.batch];
   const int ipp = p.items_per_page;
   const int stride = gridDim.x;
   const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
 
-  auto page_of = [&](const PageItem& m) {
-    return m.tensor < 2 ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
-  };
+  // a page id outside the pools comes back as -1: its item streams page 0 instead (any valid
+  // memory) and writes nothing
+  auto page_of = [&](const PageItem& m) { return m.tensor < 2 ? checked_page(p.g, m.b, m.pslot, p.status) : 0; };
   // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kMergeStages
-  auto issue = [&](int j, const PageItem& m, int page) -> bool {
+  auto issue = [&](int j, const PageItem& m, int page_id) -> bool {
     const int s = j % kMergeStages;
     if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, p.status)) return false;
     const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
     const uint32_t bar = full0 + 8 * s;
-    page_s[s] = page;
+    page_s[s] = page_id;
+    const int page = max(page_id, 0);
     const size_t row0 = (size_t)page * rows_in_page + m.grp * kRowsPerItem;
     if (!Q4IN) {
       const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     const int row = m.grp * kRowsPerItem + quad;  // one row per quad of lanes; a warp = 8 consecutive rows of one head
     const int head = row >> p.g.page_shift;
     const int tk = row & (ps - 1);
-    const bool valid = row < rows_in_page && m.pslot * ps + tk < n;
+    const bool valid = page >= 0 && row < rows_in_page && m.pslot * ps + tk < n;
     uint4 e[4];
     float g_a, g_c, d;
     int ci[4];
@@ -513,19 +514,25 @@ __device__ __forceinline__ bool keep_token(float d, float dmin, float dmax, doub
 }
 
 // The four consecutive distances of thread `t` of a chunk (tokens tok0 .. tok0 + 3 lie in one page).
-__device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, int b, int h, int tok0) {
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
+__device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, int b, int h, int tok0, bool& ok) {
+  const int page = checked_page(p.g, b, tok0 >> p.g.page_shift, p.status);
+  ok = page >= 0;
+  if (!ok) return make_float4(0.f, 0.f, 0.f, 0.f);  // a page id outside the pools: its tokens are never kept
   return *reinterpret_cast<const float4*>(
       p.dist + (((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok0 & (p.g.page_size - 1)));
 }
 
 // Masks over the thread's four tokens: `sure` = kept whatever the ties do, `eq` = kept only while the
 // segment's quota of ties lasts (top-k mode: d equal to the k-th largest; ties go to lower indices).
+// `near` counts the tokens whose distance lies within 1e-6 of the decision threshold: the ones a
+// different rounding of d could have decided the other way.
 __device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
-                                            unsigned& sure, unsigned& eq) {
+                                            unsigned& sure, unsigned& eq, int* near = nullptr) {
   sure = eq = 0u;
   if (tok0 >= n) return;
-  const float4 d4 = load_dist4(p, tensor, b, h, tok0);
+  bool ok;
+  const float4 d4 = load_dist4(p, tensor, b, h, tok0, ok);
+  if (!ok) return;
   const float d[4] = {d4.x, d4.y, d4.z, d4.w};
   if (p.mode == MC_RETAIN_TOPK) {
     const uint32_t v = p.seg_sel[2 * seg];
@@ -535,13 +542,19 @@ __device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int 
         const uint32_t key = __float_as_uint(d[j]);
         if (key > v) sure |= 1u << j;
         if (key == v) eq |= 1u << j;
+        if (near && v != 0xffffffffu && fabs((double)d[j] - (double)__uint_as_float(v)) < 1e-6) ++*near;
       }
     }
   } else {
     const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
+    const double lo = dmin, hi = dmax;
+    const double thr = p.mode == MC_RETAIN_DISTINCT ? hi - (hi - lo) * p.gamma : lo + (hi - lo) * p.gamma;
 #pragma unroll
     for (int j = 0; j < 4; ++j)
-      if (tok0 + j < n && keep_token(d[j], dmin, dmax, p.gamma, p.mode)) sure |= 1u << j;
+      if (tok0 + j < n) {
+        if (keep_token(d[j], dmin, dmax, p.gamma, p.mode)) sure |= 1u << j;
+        if (near && fabs((double)d[j] - thr) < 1e-6) ++*near;
+      }
   }
 }
 
@@ -558,7 +571,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const Retain
   const int h = seg % p.g.n_kv_heads;
   const int b = (seg / p.g.n_kv_heads) % p.g.batch;
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
-  const int n = p.g.seq_lens[b];
+  const int n = checked_len(p.g, b, p.status);
   const int k = min(n, (int)ceil(p.gamma * (double)n - 1e-12));
   if (k <= 0 || !p.do_retention) {
     if (threadIdx.x == 0) {
@@ -578,7 +591,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const Retain
     __syncthreads();
     const uint32_t prefix = s_prefix, mask = s_mask;
     for (int tok0 = 4 * threadIdx.x; tok0 < n; tok0 += 4 * kRetThreads) {
-      const float4 d4 = load_dist4(p, tensor, b, h, tok0);
+      bool ok;
+      const float4 d4 = load_dist4(p, tensor, b, h, tok0, ok);
       const float d[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -617,19 +631,21 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainP
   const int h = seg % p.g.n_kv_heads;
   const int b = (seg / p.g.n_kv_heads) % p.g.batch;
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
-  const int n = p.g.seq_lens[b];
+  const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int cnt = 0, cnt_eq = 0;
+  int cnt = 0, cnt_eq = 0, cnt_near = 0;
   if (p.do_retention && chunk * kChunk < n) {
     unsigned sure, eq;
-    keep_masks4(p, seg, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, sure, eq);
+    keep_masks4(p, seg, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, sure, eq, &cnt_near);
     cnt = __popc(sure);
     cnt_eq = __popc(eq);
   }
   for (int o = 16; o; o >>= 1) {
     cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, o);
+    cnt_near += __shfl_xor_sync(0xffffffffu, cnt_near, o);
   }
+  if (lane == 0 && cnt_near) atomicAdd(&p.status[MC_STATUS_NEAR_THRESHOLD], cnt_near);
   if (lane == 0) {
     s_cnt[warp] = cnt;
     s_eq[warp] = cnt_eq;
@@ -711,7 +727,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   const int h = seg % p.g.n_kv_heads;
   const int b = (seg / p.g.n_kv_heads) % p.g.batch;
   const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
-  const int n = p.g.seq_lens[b];
+  const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool overflow = (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
   const int seg_off = p.ret_offset[seg];
@@ -765,7 +781,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   for (int w = 0; w < warp; ++w) before += s_warp[w];
   if (lane == 0 && pj < p.ret_prefix_stride) prefix[pj] = out0 - seg_off + before;
   int pos = out0 + before + x - c;
-  if (m) {
+  if (m) {  // (kept tokens lie in a page that keep_masks4 has checked)
     const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
     float* sc = reinterpret_cast<float*>(p.e_pool[tensor] + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
                                          p.g.page_size * kRowBytes) + (tok0 & (p.g.page_size - 1));
@@ -787,7 +803,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
     const int ent = r >> 1, layer = r & 1;
     const int tok = p.ret_index[out0 + ent];
-    const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+    const int page = checked_page(p.g, b, tok >> p.g.page_shift, p.status);
+    if (page < 0) continue;
     const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
     char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
     if (!p.q4) {
@@ -838,6 +855,7 @@ struct AppendParams {
   float ta, tc;
   int merge_fn;
   int total_rows;  // 2 * batch * H
+  int32_t* status;
 };
 
 template <int DT>
@@ -853,9 +871,16 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   const int tensor = rr / (H * p.g.batch);
   // the batch description belongs to the caller (no kernel of this library writes it): where the row
   // goes is looked up before the wait on the kernel ahead in the stream
+  // (a length or page id that does not fit the declared bounds is flagged after the wait -- the
+  // status words belong to the pair cache -- and the row is not written)
   const int tok = p.g.seq_lens[b];
-  const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
+  int page = -1;
+  if (tok >= 0 && tok <= p.g.max_seq_len && (tok >> p.g.page_shift) < p.g.max_pages_per_seq)
+    page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> p.g.page_shift)];
   grid_dep_wait();
+  if (ok && !page_ok(p.g, page)) {
+    if (l16 == 0) atomicOr(p.status, MC_FLAG_BAD_METADATA);
+  }
   uint4 va = make_uint4(0, 0, 0, 0), vc = va;
   if (ok) {
     const size_t off = ((size_t)b * H + h) * kRowBytes + l16 * 16;
@@ -865,7 +890,7 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   uint4 e;
   float ga, gc, d;
   merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, ga, gc, d);
-  if (!ok) return;
+  if (!ok || !page_ok(p.g, page)) return;
   const int tk = tok & (p.g.page_size - 1);
   const size_t ph = (size_t)page * H + h;
   char* tile = p.e_pool[tensor] + ph * tile_bytes(p.g.page_size);
@@ -893,6 +918,11 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
                        int do_retention, void* workspace, cudaStream_t stream) {
   const bool q4 = q_lm1 != nullptr;
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
+  // every shape limit before the first launch
+  if (bt->batch > kMergeMaxBatchSmem) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
+  if (2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) *
+          ((cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem) > 0x7fffffffLL)
+    return MC_ERR_SHAPE;
   MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256), dim3(256), 0, stream, reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status));
   MC_CUDA_CHECK(cudaGetLastError());
   if (bt->batch == 0) return MC_OK;
@@ -915,18 +945,12 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
-  if (bt->batch > kMergeMaxBatchSmem) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
   // upper bound of the item count (the kernel enumerates the pages that hold tokens)
   const long long total = 2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
-  if (total > 0x7fffffffLL) return MC_ERR_SHAPE;
   mp.status = out->status;
   if (total > 0) {
-    static int n_sm = 0;
-    if (n_sm == 0) {
-      int dev = 0;
-      MC_CUDA_CHECK(cudaGetDevice(&dev));
-      MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-    }
+    int n_sm = 0;
+    if (mc_status st = sm_count(&n_sm)) return st;
     const int grid = (int)std::min<long long>((long long)n_sm * kMergeCtasPerSm, total);
     const size_t smem = 128 + (size_t)kMergeStages * kMergeStageBytes + (kMergeStages + 2 * kMergeMaxBatchSmem + 3) * 4 + 8 +
                         2 * kMergeStages * 8 + 64;
@@ -995,6 +1019,7 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;
   ap.total_rows = 2 * bt->batch * cfg->n_kv_heads;
+  ap.status = pair->status;
   if (ap.total_rows == 0) return MC_OK;
   const int blocks = (ap.total_rows + 7) / 8;
   if (cfg->dtype == MC_F16)

@@ -39,8 +39,11 @@ struct RestoreParams {
 // ahead, so the bytes in flight are set by the ring.  A half-warp takes a row out of shared memory
 // (undoing the chunk permutation), the stage is released as soon as the rows are in registers, and
 // the scaled rows leave with streaming stores.
-template <int DT>
+// F32: the dense rows are written as binary32 (the products e * scale unrounded, the raw rows of
+// retained tokens converted exactly) instead of the 16-bit storage type.
+template <int DT, bool F32>
 __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_scale_kernel(const RestoreParams p) {
+  constexpr int kOutRow = F32 ? 2 * kRowBytes : kRowBytes;  // bytes of a dense output row
   grid_dep_wait();
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];
@@ -66,24 +69,24 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  page_prefix(p.g, len_s, pre_s, kRestoreThreads);
+  page_prefix(p.g, len_s, pre_s, kRestoreThreads, p.status);
   const int P = pre_s[p.g.batch];
   const int ipp = p.items_per_page;
   const int stride = gridDim.x;
   const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
 
-  auto page_of = [&](const PageItem& m) {
-    return m.tensor < 2 ? p.g.block_table[(size_t)m.b * p.g.max_pages_per_seq + m.pslot] : 0;
-  };
+  // a page id outside the pools comes back as -1: its item streams page 0 instead and writes nothing
+  auto page_of = [&](const PageItem& m) { return m.tensor < 2 ? checked_page(p.g, m.b, m.pslot, p.status) : 0; };
   // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kRestoreStages
-  auto issue = [&](int j, const PageItem& m, int page) -> bool {
+  auto issue = [&](int j, const PageItem& m, int page_id) -> bool {
+    const int page = max(page_id, 0);
     const int s = j % kRestoreStages;
     if (j >= kRestoreStages && !mbar_wait(empty0 + 8 * s, ((j / kRestoreStages) - 1) & 1, s_abort, p.status)) return false;
     const int h0 = (m.grp * kRowsPerItem) >> shift;
     const int n_tiles = min(kRowsPerItem >> shift, H - h0);
     const uint32_t bytes = (uint32_t)(n_tiles * tbytes);
     const uint32_t bar = full0 + 8 * s;
-    page_s[s] = page;
+    page_s[s] = page_id;
     mbar_expect_tx(bar, bytes);
     bulk_load(stage0 + s * kRestoreStageBytes, (m.tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + h0) * tbytes, bytes, bar);
     return true;
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
       const int r = r0 + j, rp = m.grp * kRowsPerItem + r;
       const int tk = r & (ps - 1);
       const unsigned char* tile = sb + (r >> shift) * tbytes;
-      ok[j] = rp < rows_in_page && m.pslot * ps + tk < n;
+      ok[j] = page >= 0 && rp < rows_in_page && m.pslot * ps + tk < n;
       v[j] = make_uint4(0u, 0u, 0u, 0u);
       g[j] = 0.f;
       if (ok[j]) {
@@ -150,18 +153,27 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
 #pragma unroll
     for (int j = 0; j < 4; ++j)  // a retained token (scale -0) is written from its raw row below, by whichever CTA gets there
       ok[j] = ok[j] && __float_as_uint(g[j]) != 0x80000000u;
-    char* pd = (m.tensor ? p.dst_pool[1] : p.dst_pool[0]) + ((size_t)page * rows_in_page + m.grp * kRowsPerItem + r0) * kRowBytes + l16 * 16;
+    char* pd = (m.tensor ? p.dst_pool[1] : p.dst_pool[0]) +
+               ((size_t)max(page, 0) * rows_in_page + m.grp * kRowsPerItem + r0) * kOutRow + l16 * (kOutRow / 16);
 #pragma unroll
     for (int j = 0; j < 4; ++j)
       if (ok[j]) {
         const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
         uint32_t o[4];
+        float2 f[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float2 f = Elem<DT>::unpack(w[i]);
-          o[i] = Elem<DT>::pack(f.x * g[j], f.y * g[j]);
+          f[i] = Elem<DT>::unpack(w[i]);
+          f[i].x *= g[j];
+          f[i].y *= g[j];
+          o[i] = Elem<DT>::pack(f[i].x, f[i].y);
         }
-        st_stream16(pd + j * kRowBytes, make_uint4(o[0], o[1], o[2], o[3]));
+        if (F32) {
+          st_stream16(pd + j * kOutRow, make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x), __float_as_uint(f[1].y)));
+          st_stream16(pd + j * kOutRow + 16, make_uint4(__float_as_uint(f[2].x), __float_as_uint(f[2].y), __float_as_uint(f[3].x), __float_as_uint(f[3].y)));
+        } else {
+          st_stream16(pd + j * kOutRow, make_uint4(o[0], o[1], o[2], o[3]));
+        }
       }
     page_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
   }
@@ -176,11 +188,19 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
       char* dst_pool = tensor ? p.dst_pool[1] : p.dst_pool[0];
       for (int e = hw16; e < cnt; e += kRestoreThreads / 16) {
         const int tok = p.ret_index[off + e];
-        const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok >> shift)];
+        const int page = checked_page(p.g, b, tok >> shift, p.status);
+        if (page < 0) continue;
         const size_t row = ((size_t)page * H + h) * ps + (tok & (ps - 1));
         const uint4 v = *reinterpret_cast<const uint4*>(p.ret_rows + ((size_t)p.layer * p.ret_capacity + off + e) * kRetEntryBytes +
                                                         l16 * 16);
-        *reinterpret_cast<uint4*>(dst_pool + row * kRowBytes + l16 * 16) = v;
+        if (F32) {
+          const float2 f0 = Elem<DT>::unpack(v.x), f1 = Elem<DT>::unpack(v.y), f2 = Elem<DT>::unpack(v.z), f3 = Elem<DT>::unpack(v.w);
+          float4* d4 = reinterpret_cast<float4*>(dst_pool + row * kOutRow + l16 * 32);
+          d4[0] = make_float4(f0.x, f0.y, f1.x, f1.y);
+          d4[1] = make_float4(f2.x, f2.y, f3.x, f3.y);
+        } else {
+          *reinterpret_cast<uint4*>(dst_pool + row * kRowBytes + l16 * 16) = v;
+        }
       }
     }
   }
@@ -190,7 +210,7 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
 }
 
 mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
-                         int layer, const mc_layer_kv* dst, cudaStream_t stream) {
+                         int layer, const mc_layer_kv* dst, int dst_fp32, cudaStream_t stream) {
   if (bt->batch == 0) return MC_OK;
   RestoreParams rp;
   rp.g = g;
@@ -211,16 +231,14 @@ mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g
   const long long blocks = 2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * rp.items_per_page;
   if (blocks > 0x7fffffffLL) return MC_ERR_SHAPE;
   if (blocks > 0) {
-    static int n_sm = 0;
-    if (n_sm == 0) {
-      int dev = 0;
-      MC_CUDA_CHECK(cudaGetDevice(&dev));
-      MC_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-    }
+    int n_sm = 0;
+    if (mc_status st = sm_count(&n_sm)) return st;
     const int grid = (int)std::min<long long>((long long)n_sm * kRestoreCtasPerSm, blocks);
     const size_t smem = 128 + (size_t)kRestoreStages * kRestoreStageBytes + (kRestoreStages + 2 * kMaxBatchPages + 3) * 4 + 8 +
                         2 * kRestoreStages * 8 + 64;
-    void (*kern)(const RestoreParams) = cfg->dtype == MC_F16 ? restore_scale_kernel<MC_F16> : restore_scale_kernel<MC_BF16>;
+    void (*kern)(const RestoreParams) =
+        cfg->dtype == MC_F16 ? (dst_fp32 ? restore_scale_kernel<MC_F16, true> : restore_scale_kernel<MC_F16, false>)
+                             : (dst_fp32 ? restore_scale_kernel<MC_BF16, true> : restore_scale_kernel<MC_BF16, false>);
     MC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MC_CUDA_CHECK(launch_pdl(kern, dim3(grid), dim3(kRestoreThreads), smem, stream, rp));
     MC_CUDA_CHECK(cudaGetLastError());

@@ -96,8 +96,8 @@ def test_attn_and_restore_reject_bad_arguments(lib):
     c, b = _cfg(), _batch()
     pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
     d = B._LayerKV(0x10000, 0x20000)
-    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 2, C.byref(d), None) == 1  # BOTH is not a restore target
-    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 0, None, None) == 1
+    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 2, C.byref(d), 0, None) == 1  # BOTH is not a restore target
+    assert L.mc_restore(C.byref(c), C.byref(b), C.byref(pc), 0, None, 1, None) == 1
     ws = 0x100000
     # pair mode with 4 query heads per kv head needs 8 rows: allowed; with 8 per kv head it does not fit
     c8 = _cfg(n_kv_heads=4, n_q_heads=32)
@@ -108,6 +108,53 @@ def test_attn_and_restore_reject_bad_arguments(lib):
     assert L.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), 0, None, None, None, 1.0, 0x2000, None, ws, 1 << 24, None) == 1
     # workspace too small
     assert L.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), 0, 0x1000, None, None, 1.0, 0x2000, None, ws, 8, None) == 5
+
+
+def test_pair_bytes_is_host_arithmetic(lib):
+    """Every buffer size of a pair cache comes from the library; the tile is page_size rows of 256 bytes
+    plus two fp32 scales per token, the prefix table has one entry per 128 tokens plus one."""
+    cfg = mc.McConfig(8, 32, 16, "bf16")
+    sz = lib.mc_pair_bytes(cfg, batch=4, n_pages=100, max_seq_len=1000, ret_capacity=77)
+    assert sz.tile_bytes == 16 * 256 + 2 * 16 * 4 and sz.e_bytes == 100 * 8 * sz.tile_bytes
+    assert sz.dist_bytes == 100 * 8 * 2 * 16 * 4
+    nseg = 2 * 4 * 8
+    assert sz.ret_count_bytes == nseg * 4 and sz.ret_offset_bytes == (nseg + 1) * 4
+    assert sz.ret_index_bytes == 77 * 4 and sz.ret_rows_bytes == 2 * 77 * 272
+    assert sz.ret_prefix_stride == 8 + 1 and sz.ret_prefix_bytes == nseg * 9 * 4
+    assert sz.seg_minmax_bytes == nseg * 8 and sz.status_bytes == 16
+    assert sz.total_bytes >= 2 * sz.e_bytes + sz.dist_bytes and sz.total_bytes % 256 == 0
+    L = lib._lib
+    c, b, out = _cfg(), _batch(), B._PairSizes()
+    assert L.mc_pair_bytes(C.byref(c), C.byref(b), -1, C.byref(out)) == 1
+    assert L.mc_pair_bytes(C.byref(c), C.byref(b), 4, None) == 1
+    assert L.mc_pair_bytes(C.byref(_cfg(page_size=8)), C.byref(b), 4, C.byref(out)) == 2
+
+
+def test_get_stats_rejects_bad_arguments(lib):
+    L = lib._lib
+    c, b, out = _cfg(), _batch(), B._Stats()
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    assert L.mc_get_stats(C.byref(c), C.byref(b), None, None, C.byref(out)) == 1
+    assert L.mc_get_stats(C.byref(c), C.byref(b), C.byref(pc), None, None) == 1
+    assert L.mc_get_stats(C.byref(_cfg(head_dim=64)), C.byref(b), C.byref(pc), None, C.byref(out)) == 2
+
+
+def test_host_buffer_merge_checks_everything_before_the_first_copy(lib):
+    """An argument error must enqueue nothing: a too-small workspace is reported as such (without a GPU
+    the first copy would have failed with a CUDA error instead)."""
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    a = B._LayerKV(0x10000, 0x20000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    args = lambda pcx, ws, n: (C.byref(c), C.byref(b), C.byref(a), C.byref(a), C.byref(a), C.byref(a), C.byref(pcx), 1, ws, n, None)
+    assert L.mc_merge_pair_host(*args(pc, 0x100000, 16)) == 5
+    assert L.mc_merge_pair_host(*args(pc, 0x100010, 1 << 20)) == 4
+    pc2 = B._PairCache(0x30000, 0, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    assert L.mc_merge_pair_host(*args(pc2, 0x100000, 1 << 20)) == 1
+    # more sequences than the kernels' shared-memory prefix holds: refused before the status words are cleared
+    big = _batch(batch=1025, mpps=4, max_len=64, n_pages=5000)
+    a2 = B._LayerKV(0x10000, 0x20000)
+    assert L.mc_merge_pair(C.byref(c), C.byref(big), C.byref(a2), C.byref(a2), C.byref(pc), 1, 0x100000, 1 << 30, None) == 2
 
 
 def test_binding_fails_loudly_without_library(tmp_path):

@@ -34,13 +34,16 @@ def _full_cycle(H, p, mode="distinct", do_retention=True, new_token=True, pair_m
     for layer in (0, 1):
         dk, dv = p.run_restore(layer)
         stats.update({f"l{layer}_{k}": v for k, v in H.compare_restore(p, om, dc, layer, dk, dv).items()})
+        # binary32 output: the 2e-3 bar with no allowance for the output type's own rounding
+        dk, dv = p.run_restore(layer, fp32=True)
+        stats.update({f"l{layer}f_{k}": v for k, v in H.compare_restore(p, om, dc, layer, dk, dv).items()})
     wl = dataclasses.replace(p.wl, batch=p.B)
     q = gen.make_queries(wl, 0, device="cpu", n_sets=2).to(p.device)
     nt = gen.make_new_tokens(wl, 0, 0, device="cpu")
     for layer in (0, 1):
         out, lse = p.run_attn(layer, q[layer:layer + 1].contiguous())
         stats.update({f"a{layer}_{k}": v for k, v in
-                      H.compare_attention(p, om, layer, q[layer:layer + 1].cpu(), out.cpu(), lse.cpu()).items()})
+                      H.compare_attention(p, om, layer, q[layer:layer + 1].cpu(), out.cpu(), lse.cpu(), dc=dc).items()})
     if new_token:
         kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()  # [2][B][H][128]
         vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
@@ -50,9 +53,23 @@ def _full_cycle(H, p, mode="distinct", do_retention=True, new_token=True, pair_m
         if pair_mode and 2 * (p.Hq // p.H) <= 8:
             out, lse = p.run_attn(2, q.contiguous(), kn.to(p.device), vn.to(p.device))
             stats.update({f"apair_{k}": v for k, v in
-                          H.compare_attention(p, om, 2, q.cpu(), out.cpu(), lse.cpu(), kn, vn).items()})
+                          H.compare_attention(p, om, 2, q.cpu(), out.cpu(), lse.cpu(), kn, vn, dc=dc).items()})
     words, code = p.lib.mc_read_status(p.pair, check=False)
     assert code == 0, words
+    # the counts the library reports: retained entries, tokens within 1e-6 of their threshold (the oracle's
+    # count, from fp64 distances, may differ by the few tokens that sit within fp32 rounding of 1e-6
+    # itself), and the first-principles footprint of Sec. 4.3
+    st, code = p.lib.mc_get_stats(p.cfg, p.batch(), p.pair)
+    assert code == 0 and st["retained_total"] == int(dc["ret_count"].sum())
+    near = stats.get("k_near_threshold", 0) + stats.get("v_near_threshold", 0)
+    assert abs(st["near_threshold"] - near) <= 2 + near // 4, (st, near)
+    th = int(p.seq_lens_host.sum()) * p.H
+    assert st["token_heads"] == th
+    from oracle import minicache_oracle as orc
+    fp = orc.footprint_bytes(2, 0, th, 128, st["retained_total"])
+    assert st["full_bytes"] == fp["full"] and st["compressed_bytes"] == fp["compressed"]
+    assert st["stored_bytes"] >= st["compressed_bytes"]
+    stats["near_threshold_reported"] = st["near_threshold"]
     return stats
 
 
@@ -215,13 +232,16 @@ def test_scaled_configs_sampled(H, name):
     stats = H.compare_merge(p, om, dc)
     dk, dv = p.run_restore(1)
     stats.update(H.compare_restore(p, om, dc, 1, dk, dv))
+    dk, dv = p.run_restore(0, fp32=True)
+    stats.update({"f32_" + k: v for k, v in H.compare_restore(p, om, dc, 0, dk, dv).items()})
+    del dk, dv
     rs = np.random.RandomState(5)
     sample = [(int(rs.randint(p.B)), int(rs.randint(p.Hq))) for _ in range(6)]
     q = gen.make_queries(dataclasses.replace(wl, batch=p.B), 0, n_sets=2)
     for sel in ((0, 1, 2) if 2 * (p.Hq // p.H) <= 8 else (0, 1)):
         qq = q if sel == 2 else q[sel:sel + 1].contiguous()
         out, lse = p.run_attn(sel, qq.to(p.device))
-        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample))
+        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample, dc=dc))
     print(name, stats)
 
 
@@ -248,7 +268,7 @@ def test_serving_mix_ragged(H, q4):
     for sel in (0, 1, 2):
         qq = q if sel == 2 else q[sel:sel + 1].contiguous()
         out, lse = p.run_attn(sel, qq.to(p.device))
-        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample))
+        stats.update(H.compare_attention(p, om, sel, qq, out.cpu(), lse.cpu(), sample=sample, dc=dc))
     print("c4_s", "q4" if q4 else "f16", stats)
 
 
@@ -376,7 +396,7 @@ class _Segment:
         self.B, self.H, self.Hq, self.S = 1, 1, p.Hq // p.H, p.S
         self.dtype, self.gamma, self.t = p.dtype, p.gamma, p.t
         self.seq_lens_host = p.seq_lens_host[b:b + 1]
-        self.bits = {k: v[b:b + 1, :, h:h + 1] for k, v in p.bits.items()}
+        self.bits = {k: p.segment_bits(k, b, h) for k in ("k_lm1", "k_l", "v_lm1", "v_l")}
 
     def retained(self, dc, tensor, b, h):
         return self.p.retained(dc["full"], tensor, self.b0, self.h0)
@@ -391,43 +411,109 @@ class _Segment:
         out["full"] = dc
         return out
 
+    def oracle_merge(self, orc):
+        p, b, h = self.p, self.b0, self.h0
+        if p.q4:  # the oracle merges the exact de-quantised values of this segment
+            return {tn: orc.merge_pair_values(p.seg_values[(tn + "_lm1", b, h)], p.seg_values[(tn + "_l", b, h)],
+                                              self.seq_lens_host, self.dtype, self.t, self.gamma) for tn in ("k", "v")}
+        return {tn: orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype, self.t, self.gamma)
+                for tn in ("k", "v")}
 
-def test_full_size_config2_sampled(H):
-    """Config 2 at its full size (batch 8 x 4096 tokens, 32 heads, fp16, page 16; the last layer pair), in
-    the launch configuration the benchmark times: merge, restore and decode attention with a new token
-    and room for the decode steps; sampled (sequence, head) segments are compared against the oracle
-    with the same bars as everywhere else, and the retained totals must agree with the status word."""
+
+_FULL_TENSORS = {}
+
+
+def _full_tensors(name, pair):
+    """Host tensors of one pair of a full-size workload, generated once per test session."""
+    key = (name, pair)
+    if key not in _FULL_TENSORS:
+        _FULL_TENSORS.clear()  # one workload at a time: these are gigabytes
+        _FULL_TENSORS[key] = gen.make_pair_tensors(CONFIGS[name], pair, device="cpu")
+    return _FULL_TENSORS[key]
+
+
+@pytest.mark.parametrize("name,gamma,q4", [
+    ("c2", 0.05, False),
+    ("c3", 0.0, False), ("c3", 0.05, False), ("c3", 0.2, False),
+    ("c5", 0.05, False),
+    ("c4", 0.05, False), ("c4", 0.05, True),
+], ids=["c2", "c3_g0", "c3_g005", "c3_g02", "c5", "c4_f16", "c4_q4in"])
+def test_full_size_configs_sampled(H, name, gamma, q4):
+    """Every throughput workload at its full size (the last layer pair), in the launch configuration the
+    benchmark times: merge, restore and decode attention (single layer with a new token; pair mode where
+    the head ratio allows it) with room for the decode steps; sampled (sequence, head) segments are
+    compared against the oracle with the same bars as everywhere else, and the retained totals must agree
+    with the status word.  Config 3 runs at gamma 0 (nothing retained: the path without extra stages),
+    0.05 and 0.2 (several extra stages per piece); config 5 has 32768-token sequences (many pieces per
+    sequence, accumulators carried from chunk to chunk); config 4 is the ragged batch of 64 with pages of
+    32 tokens, with 16-bit and with 4-bit layers."""
     from oracle import minicache_oracle as orc
-    wl = CONFIGS["c2"]
-    p = H.Problem(wl, pair=wl.n_pairs - 1, decode_room=wl.decode_steps + 1)
+    wl = CONFIGS[name]
+    pair = wl.n_pairs - 1
+    rs = np.random.RandomState(17)
+    lens = gen.make_lengths(wl)[0] if wl.ragged else None
+    segs = [(int(rs.randint(wl.batch)), int(rs.randint(wl.n_kv_heads))) for _ in range(4 if wl.seq_len <= 8192 else 2)]
+    if wl.ragged:  # the longest and the shortest sequence are always among the samples
+        segs[0] = (int(np.argmax(lens)), segs[0][1])
+        segs[1] = (int(np.argmin(lens)), segs[1][1])
+    th2 = int((lens.sum() if lens is not None else wl.batch * wl.seq_len)) * wl.n_kv_heads * 2
+    p = H.Problem(wl, pair=pair, decode_room=wl.decode_steps + 1, tensors=_full_tensors(name, pair), gamma=gamma,
+                  seq_lens=lens, q4=q4, segments=segs if q4 else None, ret_capacity=int(0.12 * th2) + 1024)
     words, code = p.run_merge()
     assert code == 0, words
     dc = p.device_cache()
     assert int(dc["ret_count"].sum()) == int(words[1])
-    rs = np.random.RandomState(17)
-    segs = [(int(rs.randint(p.B)), int(rs.randint(p.H))) for _ in range(4)]
+    if gamma == 0.0:
+        assert int(words[1]) == 0
+    st, _ = p.lib.mc_get_stats(p.cfg, p.batch(), p.pair)
+    print(name, gamma, "retained fraction", words[1] / th2, "near threshold", st["near_threshold"])
     dk, dv = p.run_restore(1)
     dkl, dvl = p.logical_of(dk), p.logical_of(dv)
+    dk, dv = p.run_restore(0, fp32=True)
+    dkf, dvf = p.logical_of(dk), p.logical_of(dv)
+    del dk, dv
     wlb = dataclasses.replace(wl, batch=p.B)
     q = gen.make_queries(wlb, 2, n_sets=2)
     nt = gen.make_new_tokens(wlb, 0, 0)
     kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
     vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
-    out, lse = p.run_attn(1, q[1:2].contiguous().to(p.device), kn[1:2].contiguous().to(p.device), vn[1:2].contiguous().to(p.device))
-    out2, lse2 = p.run_attn(2, q.to(p.device), kn.to(p.device), vn.to(p.device))
-    out, lse, out2, lse2 = out.cpu(), lse.cpu(), out2.cpu(), lse2.cpu()
+    # the batch bound the benchmark's decode phase declares: prompt + decode steps + 1
+    extra = wl.decode_steps + 1
+    def attn(layer_sel, qq, kk, vv):
+        n_sets = 2 if layer_sel == 2 else 1
+        out = torch.zeros(n_sets, p.B, p.Hq, 128, dtype=p.cfg.torch_dtype, device=p.device)
+        lse = torch.zeros(n_sets, p.B, p.Hq, dtype=torch.float32, device=p.device)
+        p.lib.mc_decode_attn(p.cfg, p.batch(extra), p.pair, layer_sel, qq.to(p.device), kk.to(p.device), vv.to(p.device),
+                             1.0 / math.sqrt(128.0), out, lse, p.workspace(1, n_sets, extra))
+        torch.cuda.synchronize()
+        return out.cpu(), lse.cpu()
+    out, lse = attn(1, q[1:2].contiguous(), kn[1:2].contiguous(), vn[1:2].contiguous())
+    pair_mode = 2 * (p.Hq // p.H) <= 8
+    if pair_mode:
+        out2, lse2 = attn(2, q, kn, vn)
+    else:  # layer l-1 as a single-layer call instead
+        out0, lse0 = attn(0, q[0:1].contiguous(), kn[0:1].contiguous(), vn[0:1].contiguous())
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 0, words
+    nq = p.Hq // p.H
     for b, h in segs:
         sg = _Segment(p, b, h)
-        om = {tn: orc.merge_pair(sg.bits[tn + "_lm1"], sg.bits[tn + "_l"], sg.seq_lens_host, sg.dtype, sg.t, sg.gamma)
-              for tn in ("k", "v")}
+        om = sg.oracle_merge(orc)
         dcs = sg.slice_cache(dc)
         stats = H.compare_merge(sg, om, dcs)
-        # restore of layer l: dense rows of this segment
         stats.update(H.compare_restore(sg, om, dcs, 1, dkl[b:b + 1, :, h:h + 1], dvl[b:b + 1, :, h:h + 1]))
-        sl = lambda x, hd: x[:, b:b + 1, hd:hd + 1].contiguous()
-        stats.update(H.compare_attention(sg, om, 1, sl(q[1:2], h), sl(out, h), sl(lse, h), sl(kn[1:2], h), sl(vn[1:2], h)))
-        stats.update(H.compare_attention(sg, om, 2, sl(q, h), sl(out2, h), sl(lse2, h), sl(kn, h), sl(vn, h)))
-        print("segment", b, h, stats)
+        stats.update({"f32_" + k: v for k, v in
+                      H.compare_restore(sg, om, dcs, 0, dkf[b:b + 1, :, h:h + 1], dvf[b:b + 1, :, h:h + 1]).items()})
+        slq = lambda x: x[:, b:b + 1, h * nq:(h + 1) * nq].contiguous()  # the kv head's query heads
+        slk = lambda x: x[:, b:b + 1, h:h + 1].contiguous()
+        stats.update(H.compare_attention(sg, om, 1, slq(q[1:2]), slq(out), slq(lse), slk(kn[1:2]), slk(vn[1:2]), dc=dcs))
+        if pair_mode:
+            stats.update({"pair_" + k: v for k, v in
+                          H.compare_attention(sg, om, 2, slq(q), slq(out2), slq(lse2), slk(kn), slk(vn), dc=dcs).items()})
+        else:
+            stats.update({"l0_" + k: v for k, v in
+                          H.compare_attention(sg, om, 0, slq(q[0:1]), slq(out0), slq(lse0), slk(kn[0:1]), slk(vn[0:1]), dc=dcs).items()})
+        print(name, "segment", b, h, "len", int(p.seq_lens_host[b]), stats)
 
 
 def test_bounded_wait_times_out_into_the_status_word(H):
@@ -491,3 +577,207 @@ def test_decode_step_replayed_from_a_cuda_graph(H):
     assert torch.equal(len_e, len_g) and torch.equal(ek_e, ek_g)
     for a, b in zip(eager, graph):
         assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("use_graph", [False, True], ids=["eager", "graph"])
+def test_decode_loop_without_host_sync(H, use_graph):
+    """The loop the benchmark times, checked against the oracle: 18 decode steps of (attention of layer
+    l-1, attention of layer l, append-merge, lengths + 1 on the device) enqueued back to back with no
+    host synchronisation in between, issued call by call or replayed from a CUDA graph.  The kernel
+    right ahead of every step's first attention is the caller's `seq_lens += 1`; attention and append
+    read the lengths before their dependency wait, so a stale length would show here as an output over
+    n - 1 tokens or a row appended one position early.  Compared at the end: every step's outputs
+    and log-sum-exps and the appended directions and scales."""
+    import mc_harness as M
+    from oracle import minicache_oracle as orc
+    steps = 18
+    wl = CONFIGS["c1"].scaled("loop", n_kv_heads=4, n_q_heads=8, dtype="bf16", batch=3, seq_len=304, index=97)
+    lens = np.array([300, 129, 47], np.int32)
+    p = H.Problem(wl, seq_lens=lens, decode_room=steps + 2)
+    words, code = p.run_merge()
+    assert code == 0, words
+    om = p.oracle_merge()
+    wlb = dataclasses.replace(wl, batch=3)
+    nts = [gen.make_new_tokens(wlb, 0, s) for s in range(steps)]
+    qs = [gen.make_queries(wlb, 30 + s, n_sets=2) for s in range(steps)]
+    dev = "cuda"
+    all_new = {k: torch.stack([nt[k][:, 0] for nt in nts]).contiguous().to(dev) for k in ("k_lm1", "v_lm1", "k_l", "v_l")}
+    all_q = torch.stack(qs).contiguous().to(dev)  # [steps][2][B][Hq][128]
+    cur = {k: v[0].clone() for k, v in all_new.items()}
+    cur_q = all_q[0].clone()
+    step_dev = torch.zeros(1, dtype=torch.long, device=dev)
+    outs = torch.zeros(steps, 2, 1, 3, 8, 128, dtype=torch.bfloat16, device=dev)
+    lses = torch.zeros(steps, 2, 1, 3, 8, dtype=torch.float32, device=dev)
+    out_cur = torch.zeros(2, 1, 3, 8, 128, dtype=torch.bfloat16, device=dev)
+    lse_cur = torch.zeros(2, 1, 3, 8, dtype=torch.float32, device=dev)
+    b = p.mc.Batch(p.block_table, p.seq_lens, p.max_seq_len + steps, p.n_pages)
+    ws = torch.empty(p.lib.mc_workspace_bytes(p.cfg, b, 1, 1), dtype=torch.uint8, device=dev)
+    sm = 1.0 / math.sqrt(128.0)
+
+    def step():
+        for layer in (0, 1):
+            p.lib.mc_decode_attn(p.cfg, b, p.pair, layer, cur_q[layer], cur["k_lm1" if layer == 0 else "k_l"],
+                                 cur["v_lm1" if layer == 0 else "v_l"], sm, out_cur[layer], lse_cur[layer], ws)
+        p.lib.mc_append_pair(p.cfg, b, p.pair, cur["k_lm1"], cur["v_lm1"], cur["k_l"], cur["v_l"])
+        # results out, the next step's inputs in (device-side indexing: nothing here waits for the host)
+        outs.index_copy_(0, step_dev, out_cur[None])
+        lses.index_copy_(0, step_dev, lse_cur[None])
+        step_dev.add_(1).clamp_(max=steps - 1)
+        for k in cur:
+            cur[k].copy_(all_new[k].index_select(0, step_dev)[0])
+        cur_q.copy_(all_q.index_select(0, step_dev)[0])
+        p.seq_lens += 1  # last: the next step's first attention follows it directly
+
+    p.run_attn(0, cur_q[0:1].contiguous())  # one call outside any capture: one-time set-up of the kernels
+    if use_graph:
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            step()
+        for _ in range(steps):
+            g.replay()
+    else:
+        for _ in range(steps):
+            step()
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 0, words
+    assert np.array_equal(p.seq_lens.cpu().numpy(), lens + steps)
+    outs_h, lses_h = outs.cpu(), lses.cpu()
+    # the oracle walks the same steps: attend over what is cached plus the step's raw token, then append
+    room = steps + 2
+    for tn in ("k", "v"):
+        o = om[tn]
+        for key in ("e_bits", "n_lm1", "n_l", "d", "e"):
+            shp = list(o[key].shape)
+            shp[1] = room
+            o[key] = np.concatenate([o[key], np.zeros(shp, o[key].dtype)], axis=1)
+    stats = {}
+    appended = {tn: [] for tn in ("k", "v")}
+    for s in range(steps):
+        nt = nts[s]
+        kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+        vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+        for layer in (0, 1):
+            st = M.compare_attention(p, om, layer, qs[s][layer:layer + 1].contiguous(), outs_h[s, layer], lses_h[s, layer],
+                                     kn[layer:layer + 1].contiguous(), vn[layer:layer + 1].contiguous())
+            for k2, v2 in st.items():
+                stats[k2] = max(stats.get(k2, 0.0), v2)
+        for tn in ("k", "v"):
+            m = orc.append_rows(gen.as_bits(nt[tn + "_lm1"][:, 0]), gen.as_bits(nt[tn + "_l"][:, 0]), p.dtype, p.t)
+            appended[tn].append(m)
+            for bb in range(3):
+                pos = int(p.seq_lens_host[bb])
+                om[tn]["e_bits"][bb, pos] = m["e_bits"][bb]
+                om[tn]["n_lm1"][bb, pos] = m["n_a"][bb]
+                om[tn]["n_l"][bb, pos] = m["n_c"][bb]
+        p.seq_lens_host = p.seq_lens_host + 1
+    # the appended rows: stored directions equal the oracle's up to boundary flips, scales = |x| / |e_stored|
+    dc = p.device_cache(extra_tokens=16)  # 320 positions = the 20 pages of the longest sequence
+    ulp = M.ULP_REL[p.dtype]
+    for ti, tn in enumerate(("k", "v")):
+        for s in range(steps):
+            m = appended[tn][s]
+            for bb in range(3):
+                pos = int(lens[bb]) + s
+                e_gpu = orc.decode_bits(dc["e_" + tn][bb, pos], p.dtype)
+                e_orc = orc.decode_bits(m["e_bits"][bb], p.dtype)
+                assert np.all(np.abs(e_gpu - e_orc) <= np.maximum(np.abs(e_orc), 2.0 ** -14) * ulp * 1.01)
+                len_e = np.sqrt(np.sum(e_gpu * e_gpu, -1))
+                for li, nm in enumerate(("n_a", "n_c")):
+                    got = dc["scale"][bb, pos, :, ti * 2 + li]
+                    assert np.all(np.abs(got * len_e - m[nm][bb]) <= 4e-6 * m[nm][bb] + 1e-30)
+                assert np.all(np.abs(dc["dist"][bb, pos, :, ti] - m["d"][bb]) < 5e-7)
+    print("decode loop", "graph" if use_graph else "eager", stats)
+
+
+def test_metadata_outside_the_declared_bounds_is_flagged_not_followed(H):
+    """A stale length or page id must never become an address.  Every case here declares a bound that is
+    SMALLER than what is really allocated, so an id the check has to refuse still points into memory this
+    test owns: a length above max_seq_len is clamped (attention), a page id at or above n_pages is
+    neither written (merge, restore, append) nor read (attention reads page 0 instead), and the status
+    words carry MC_FLAG_BAD_METADATA until the next merge clears them."""
+    wl = CONFIGS["c1"].scaled("guard", n_kv_heads=2, n_q_heads=4, batch=3, seq_len=320, index=98)
+    lens = np.array([304, 200, 64], np.int32)
+    p = H.Problem(wl, seq_lens=lens, decode_room=40)
+    mc = p.mc
+    words, code = p.run_merge()
+    assert code == 0, words
+    wlb = dataclasses.replace(wl, batch=3)
+    q = gen.make_queries(wlb, 0, n_sets=1).to(p.device)
+    ref, ref_lse = p.run_attn(1, q)
+    sm = 1.0 / math.sqrt(128.0)
+
+    # (1) a length above the declared bound: sequence 1 claims 330 tokens (its pages hold 240: the
+    # clamp to max_seq_len = 200 keeps it inside them), workspace sized for the real geometry
+    ws = p.workspace(1, 1, extra=40)
+    bad_lens = p.seq_lens.clone()
+    bad_lens[1] = 330
+    small = mc.Batch(p.block_table, bad_lens, 200, p.n_pages)
+    out = torch.zeros_like(ref)
+    lse = torch.zeros_like(ref_lse)
+    p.lib.mc_decode_attn(p.cfg, small, p.pair, 1, q, None, None, sm, out, lse, ws)
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 8 and (words[0] & mc.binding.MC_FLAG_BAD_METADATA), (words, code)
+    # the sequence inside the bounds is served as ever, and so is the one clamped to 200 = its true length
+    # (the work split differs from the reference call's, so the last bits may)
+    assert (out[0, 1:].float() - ref[0, 1:].float()).abs().max().item() < 1e-2
+
+    # (2) page ids at or above the declared pool size: merge leaves their tiles alone
+    cut = int(p.block_table[p.block_table >= 0].max().item())  # declare the pools one page shorter than they are
+    used = p.block_table[0, : (304 + p.ps - 1) // p.ps].cpu().numpy()
+    short = mc.Batch(p.block_table, p.seq_lens, p.max_seq_len, cut)
+    p.pair.e_k.fill_(0xEE)
+    p.pair.e_v.fill_(0xEE)
+    p.lib.mc_merge_pair(p.cfg, short, p.pools["k_lm1"], p.pools["v_lm1"], p.pools["k_l"], p.pools["v_l"], p.pair, True,
+                        p.workspace(0))
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert (words[0] & mc.binding.MC_FLAG_BAD_METADATA), words
+    holds_tokens = bool(((p.block_table == cut) & (torch.arange(p.block_table.shape[1], device=p.device)[None, :] * p.ps <
+                                                   p.seq_lens[:, None])).any().item())
+    if holds_tokens:
+        assert torch.all(p.pair.e_k[cut] == 0xEE) and torch.all(p.pair.e_v[cut] == 0xEE)
+    assert not torch.all(p.pair.e_k[int(used[0])] == 0xEE)
+    # restore with the same short declaration: that page's dense rows stay as they were
+    dk = torch.full((p.n_pages, p.H, p.ps, 128), 7.0, dtype=p.cfg.torch_dtype, device=p.device)
+    dv = dk.clone()
+    p.lib.mc_restore(p.cfg, short, p.pair, 1, dk, dv)
+    torch.cuda.synchronize()
+    if holds_tokens:
+        assert torch.all(dk[cut] == 7.0) and torch.all(dv[cut] == 7.0)
+    # attention with the short declaration: flagged, finite, nothing followed
+    out2 = torch.zeros_like(ref)
+    p.lib.mc_decode_attn(p.cfg, short, p.pair, 1, q, None, None, sm, out2, None, ws)
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert (words[0] & mc.binding.MC_FLAG_BAD_METADATA), words
+
+    # (3) append where the new token's position has no page inside the declared table width
+    words, code = p.run_merge()  # clears the words
+    assert code == 0 and words[0] == 0
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    dev = {k: v[:, 0].contiguous().to(p.device) for k, v in nt.items()}
+    before = p.pair.e_k.clone()
+    assert 304 % p.ps == 0
+    narrow_tbl = p.block_table[:, : 304 // p.ps].contiguous()  # sequence 0 fills its pages: no slot for token 304
+    narrow = mc.Batch(narrow_tbl, p.seq_lens, 304, p.n_pages)
+    p.lib.mc_append_pair(p.cfg, narrow, p.pair, dev["k_lm1"], dev["v_lm1"], dev["k_l"], dev["v_l"])
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert (words[0] & mc.binding.MC_FLAG_BAD_METADATA), words
+    pg0 = p.block_table[0].cpu().long()
+    assert torch.equal(p.pair.e_k[pg0], before[pg0])  # none of sequence 0's pages (spare ones included) was written
+    # a length above the bound: nothing of that sequence is written
+    words, code = p.run_merge()
+    before = p.pair.e_k.clone()
+    bad_lens = p.seq_lens.clone()
+    bad_lens[2] = 90  # declared bound 80 below; its pages hold 104 tokens
+    over = mc.Batch(p.block_table, bad_lens, 80, p.n_pages)
+    p.lib.mc_append_pair(p.cfg, over, p.pair, dev["k_lm1"], dev["v_lm1"], dev["k_l"], dev["v_l"])
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert (words[0] & mc.binding.MC_FLAG_BAD_METADATA), words
+    pg2 = p.block_table[2, : (104 + p.ps - 1) // p.ps].cpu().long()
+    assert torch.equal(p.pair.e_k[pg2], before[pg2])
