@@ -357,18 +357,18 @@ def lse_combine(parts: List):
 Q4_GROUP = 32
 
 
-def q4_quantise(x: np.ndarray, axis: int):
+def q4_quantise(x: np.ndarray, axis: int, meta_dtype: str = "f16"):
     """Quantise float64 x along `axis` in groups of 32 (its length must be a multiple of 32).
 
     Returns (codes uint8, same shape; scale, zero: float64 values that are exactly representable in
-    binary16, shape of x with `axis` divided by 32)."""
+    `meta_dtype` (binary16 unless stated), shape of x with `axis` divided by 32)."""
     x = np.moveaxis(np.asarray(x, F64), axis, -1)
     shp = x.shape
     assert shp[-1] % Q4_GROUP == 0
     g = x.reshape(shp[:-1] + (shp[-1] // Q4_GROUP, Q4_GROUP))
     lo, hi = g.min(-1), g.max(-1)
-    scale = decode_bits(encode_bits((hi - lo) / 15.0, "f16"), "f16")
-    zero = decode_bits(encode_bits(lo, "f16"), "f16")
+    scale = decode_bits(encode_bits((hi - lo) / 15.0, meta_dtype), meta_dtype)
+    zero = decode_bits(encode_bits(lo, meta_dtype), meta_dtype)
     scale = np.where(scale == 0.0, 1.0, scale)
     codes = np.clip(np.rint((g - zero[..., None]) / scale[..., None]), 0, 15).astype(np.uint8)
     codes = np.moveaxis(codes.reshape(shp), -1, axis)
@@ -381,6 +381,54 @@ def q4_dequantise(codes: np.ndarray, scale: np.ndarray, zero: np.ndarray, axis: 
     s = np.repeat(np.moveaxis(np.asarray(scale, F64), axis, -1), Q4_GROUP, axis=-1)
     z = np.repeat(np.moveaxis(np.asarray(zero, F64), axis, -1), Q4_GROUP, axis=-1)
     return np.moveaxis(c * s + z, -1, axis)
+
+
+def q4_cache_quantise(e_bits: np.ndarray, n: int, kind: str, dtype: str) -> Dict[str, np.ndarray]:
+    """The shared directions of one (sequence, kv head) held in a 4-bit cache (Sec. 5: MiniCache
+    "on top of 4-bit KIVI"; the paper states no more than that, the reading is the following).
+
+    e_bits [S][D]: the merged directions already rounded to the 16-bit cache type (`store_direction`);
+    n: cached tokens.  The quantiser is the KIVI scheme above applied to that 16-bit cache, in the
+    cache's own page structure (pages of 32 tokens): keys (`kind` "k") per channel, a group = the 32
+    tokens of a page; values ("v") per token, a group = 32 channels.  Only complete pages are
+    quantised: the tokens [32 floor(n / 32), n) of the last, incomplete page stay in 16 bits (KIVI
+    keeps such a full-precision residual until a group is complete).  Scale and zero are kept in the
+    cache's 16-bit type, and a de-quantised element is code * scale + zero rounded ONCE to that
+    type: the value a 16-bit tensor-core operand carries, and the stored direction e of Eq. 2.
+
+    Returns codes [n_q][D] uint8, scale / zero (K: [n_q / 32][D], V: [n_q][D / 32]; float64 holding
+    values of the 16-bit type), e_bits [S][D] (the stored directions: de-quantised ones for the
+    first n_q = 32 floor(n / 32) tokens, the input bits for the rest) and n_q."""
+    e_bits = np.asarray(e_bits, np.uint16)
+    n_q = (int(n) // Q4_GROUP) * Q4_GROUP
+    out_bits = e_bits.copy()
+    axis = 0 if kind == "k" else 1
+    if n_q == 0:
+        d = e_bits.shape[1]
+        empty = np.zeros((0, d) if kind == "k" else (0, d // Q4_GROUP), F64)
+        return {"codes": np.zeros((0, d), np.uint8), "scale": empty, "zero": empty.copy(), "e_bits": out_bits, "n_q": 0}
+    x = decode_bits(e_bits[:n_q], dtype)
+    codes, scale, zero = q4_quantise(x, axis, meta_dtype=dtype)
+    out_bits[:n_q] = encode_bits(q4_dequantise(codes, scale, zero, axis), dtype)
+    return {"codes": codes, "scale": scale, "zero": zero, "e_bits": out_bits, "n_q": n_q}
+
+
+def q4_cache_pair(m: Dict[str, object], seq_lens: Sequence[int], kind: str, dtype: str) -> Dict[str, object]:
+    """A merged pair (the dict `merge_pair` returns for one tensor) as the 4-bit cache holds it:
+    "e_bits" becomes the stored (de-quantised, 16-bit rounded) directions, "e16_bits" keeps the
+    directions before quantisation, "q4" maps (b, h) to the codes and group parameters."""
+    out = dict(m)
+    e16 = m["e_bits"]
+    eb = e16.copy()
+    q4 = {}
+    B, S, H, _ = e16.shape
+    for b in range(B):
+        for h in range(H):
+            r = q4_cache_quantise(e16[b, :, h], int(seq_lens[b]), kind, dtype)
+            eb[b, :, h] = r["e_bits"]
+            q4[(b, h)] = r
+    out["e16_bits"], out["e_bits"], out["q4"] = e16, eb, q4
+    return out
 
 
 # --------------------------------------------------------------------------

@@ -504,3 +504,82 @@ def test_restore_error_of_the_merge_functions_on_the_synthetic_pair():
     print("mean relative restore error:", err)
     assert err["slerp"] < err["fmax"] and err["slerp"] < err["mean"]
     assert err["slerp"] < 0.25  # about half the mean planted angle (0.3 rad) plus outliers
+
+
+# --------------------------------------------------------------------------
+# 4-bit shared cache (Sec. 5: MiniCache on top of 4-bit KIVI)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+def test_q4_cache_constant_groups_survive_exactly(dt):
+    """Closed form: a group whose members are all equal has scale 1, code 0 and zero = the value, so the
+    stored direction is the input, bit for bit.  Keys: the same direction in all 32 tokens of a page (every
+    channel group is constant).  Values: a row that is constant inside each 32-channel group."""
+    rs = np.random.RandomState(3)
+    row = rs.standard_normal(128)
+    row /= np.linalg.norm(row)
+    same = np.tile(orc.encode_bits(row, dt)[None, :], (64, 1))
+    r = orc.q4_cache_quantise(same, 64, "k", dt)
+    assert np.array_equal(r["e_bits"], same) and np.all(r["codes"] == 0) and np.all(r["scale"] == 1.0)
+    steps = np.repeat(rs.standard_normal((64, 4)) * 0.1, 32, axis=1)  # constant per (token, 32-channel group)
+    sb = orc.encode_bits(steps, dt)
+    r = orc.q4_cache_quantise(sb, 64, "v", dt)
+    assert np.array_equal(r["e_bits"], sb) and np.all(r["codes"] == 0)
+
+
+@pytest.mark.parametrize("kind", ["k", "v"])
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+def test_q4_cache_error_bound_tail_and_brute_force(kind, dt):
+    """Quantised tokens are within half a step (plus the 16-bit roundings) of the 16-bit direction, the
+    extremes of a group get codes 0 and 15, the tokens of the incomplete last page are untouched, and a
+    pure-Python loop over one group reproduces codes and stored values."""
+    rs = np.random.RandomState(11)
+    n, S = 77, 96  # two complete pages, 13 tokens in the residual, padding behind
+    e = rs.standard_normal((S, 128))
+    e /= np.linalg.norm(e, axis=1, keepdims=True)
+    eb = orc.encode_bits(e, dt)
+    r = orc.q4_cache_quantise(eb, n, kind, dt)
+    assert r["n_q"] == 64 and r["codes"].shape == (64, 128) and r["codes"].max() == 15 and r["codes"].min() == 0
+    assert np.array_equal(r["e_bits"][64:], eb[64:])  # residual and padding stay as they were
+    x = orc.decode_bits(eb[:64], dt)
+    y = orc.decode_bits(r["e_bits"][:64], dt)
+    ulp = 2.0 ** -10 if dt == "f16" else 2.0 ** -7
+    step = np.repeat(r["scale"], 32, axis=0 if kind == "k" else 1)
+    # half a step, plus the rounding of zero (|zero| ulp / 2), of scale (15 |scale| ulp / 2) and of the result
+    assert np.all(np.abs(y - x) <= 0.5 * step + ulp * (0.5 * 0.4 + 7.5 * step + 0.5 * np.abs(y)) + 1e-12)
+    # brute force of one group
+    if kind == "k":
+        g = [float(v) for v in x[32:64, 5]]
+        sc, ze = float(r["scale"][1, 5]), float(r["zero"][1, 5])
+        got_codes, got_vals = r["codes"][32:64, 5], y[32:64, 5]
+    else:
+        g = [float(v) for v in x[40, 64:96]]
+        sc, ze = float(r["scale"][40, 2]), float(r["zero"][40, 2])
+        got_codes, got_vals = r["codes"][40, 64:96], y[40, 64:96]
+    one = lambda v: float(orc.decode_bits(orc.encode_bits(np.array([v]), dt), dt)[0])
+    lo, hi = min(g), max(g)
+    assert ze == one(lo) and sc == one((hi - lo) / 15.0)
+    for v, c, w in zip(g, got_codes, got_vals):
+        q = min(15, max(0, round((v - ze) / sc)))  # Python's round is ties-to-even, like rint
+        assert q == int(c) and w == one(q * sc + ze)
+    assert got_codes.min() == 0 and got_codes.max() == 15  # the group's minimum and maximum
+
+
+def test_q4_cache_restore_keeps_the_magnitudes():
+    """Eq. 2 with the 4-bit cache: the restored row still has exactly the stored magnitude, because the
+    division is by the length of the stored (de-quantised) direction; and the angle between the restored
+    row and the 16-bit cache's restored row is small (a 4-bit step is 1/15 of the group's range)."""
+    import gen
+    cfg = gen.CONFIGS["c1"].scaled("q4c", n_kv_heads=2, n_q_heads=2, batch=1, seq_len=96, index=61)
+    t = gen.make_pair_tensors(cfg, 0)
+    lens = [80]
+    for kind in ("k", "v"):
+        m = orc.merge_pair(gen.as_bits(t[kind + "_lm1"]), gen.as_bits(t[kind + "_l"]), lens, "f16", 0.6, 0.05)
+        mq = orc.q4_cache_pair(m, lens, kind, "f16")
+        assert np.array_equal(mq["e_bits"][0, 64:80], m["e_bits"][0, 64:80])
+        assert not np.array_equal(mq["e_bits"][0, :64], m["e_bits"][0, :64])
+        for h in range(2):
+            x16 = orc.restore(m["e_bits"][0, :80, h], m["n_l"][0, :80, h], "f16")
+            x4 = orc.restore(mq["e_bits"][0, :80, h], m["n_l"][0, :80, h], "f16")
+            assert np.allclose(np.linalg.norm(x4, axis=1), m["n_l"][0, :80, h], rtol=1e-12)
+            cos = np.sum(x16 * x4, 1) / (np.linalg.norm(x16, axis=1) * np.linalg.norm(x4, axis=1))
+            assert np.all(cos > 0.97) and np.all(cos[64:] > 1 - 1e-12)
