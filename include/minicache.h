@@ -119,7 +119,8 @@ typedef struct mc_config {
   double t;            /* interpolation parameter of Eq. 3: 0 -> direction of layer l-1, 1 -> of layer l */
   double gamma;        /* retention threshold of Eq. 4 */
   int32_t merge_fn;    /* mc_merge_fn: how the two rows of a token become the shared row */
-  int32_t reserved;    /* must be 0 */
+  int32_t cache_bits;  /* storage of the shared directions E: 0 or 16 = the 16-bit type `dtype`; 4 = the 4-bit
+                          shared cache described at mc_pair_cache (page_size must then be 32) */
 } mc_config;
 
 /* Batch geometry shared by the layer pools and the pair cache. */
@@ -182,7 +183,7 @@ typedef struct mc_layer_q4 {
  * seg_minmax [2 * batch * n_kv_heads][2] fp32 d_min, d_max of the prefill tokens
  * status     [MC_STATUS_WORDS] int32 */
 typedef struct mc_pair_cache {
-  void* e_k;
+  void* e_k;  /* cache_bits = 4: the 4-bit tile pools, see below */
   void* e_v;
   float* dist;
   int32_t* ret_count;
@@ -194,7 +195,38 @@ typedef struct mc_pair_cache {
   int64_t ret_prefix_stride;
   float* seg_minmax;
   int32_t* status;
+  void* res_k; /* cache_bits = 4 only (else ignored, may be NULL): residual tiles, see below */
+  void* res_v;
 } mc_pair_cache;
+
+/* The 4-bit shared cache (cfg->cache_bits = 4; Sec. 5: MiniCache on top of 4-bit KIVI quantisation --
+ * the paper names the scheme only; the reading and the layout are ours).  The merged directions,
+ * already rounded to the 16-bit type, are quantised page by page (page_size = 32 = the group size):
+ * keys per channel (a group = the page's 32 tokens of one channel), values per token (a group = 32
+ * consecutive channels), asymmetric round-to-nearest: scale = (max - min) / 15 and zero = min, both
+ * kept in the 16-bit type (a constant group stores scale 1), code = clamp(rint((x - zero) / scale), 0, 15).
+ * A stored direction element is code * scale + zero rounded ONCE to the 16-bit type; the scales of
+ * Eq. 2 are |x| / |that stored direction|.  Only complete pages are quantised: the tokens of a
+ * sequence's last, incomplete page stay in 16 bits (KIVI's full-precision residual) in the residual
+ * tile of their (sequence, head) until mc_append_pair completes the page and quantises it.
+ *
+ * e_k / e_v  [n_pages][n_kv_heads][2816 bytes]; a tile = 2048 bytes of codes, 512 of group parameters,
+ *            then the two layers' scales [2][32] fp32 as in the 16-bit tile.
+ *   K codes  token row r at byte 64 r; in 32-bit word w of a row, bits [4p, 4p+4) hold channel 8w + 2p
+ *            and bits [16 + 4p, 16 + 4p + 4) channel 8w + 2p + 1 (p = 0..3).
+ *   K groups sixteen 16-byte chunks of scales, then sixteen of zeros (16-bit type); the chunk of the
+ *            channels [8 o, 8 o + 8) sits at chunk position 4 (o & 3) + (o >> 2).
+ *   V codes  sixteen 128-byte blocks, block i = tokens 2i and 2i+1; its 16-byte chunk c (0..7) sits at
+ *            chunk position c ^ ((i & 3) << 1); in word k (0..3) of chunk c the low 16 bits belong to
+ *            token 2i, the high 16 bits to token 2i+1, and bits [4n, 4n+4) of a half hold channel
+ *            32 k + 16 (n >> 1) + 8 (n & 1) + c (n = 0..3).
+ *   V groups per token pair i 32 bytes: four words (scale of token 2i, scale of token 2i+1) for the
+ *            channel groups 0..3, then four such words of zeros.
+ *            (These orders are the ones in which the attention kernel builds tensor-core fragments
+ *            straight from the codes.)
+ * res_k / res_v  [batch][n_kv_heads][8448 bytes]: one 16-bit tile (the format of cfg->cache_bits = 16,
+ *            page_size 32) per (sequence, head) holding the tokens [32 floor(n / 32), n).
+ * dist, the retention fields and status are as for the 16-bit cache. */
 
 /* Byte sizes of the buffers of one mc_pair_cache (Sec. 4.2: the shared cache C of a layer pair) for
  * cfg, batch->batch, batch->n_pages, batch->max_seq_len (the longest sequence at merge time) and a
@@ -212,6 +244,7 @@ typedef struct mc_pair_sizes {
   size_t status_bytes;
   int64_t ret_prefix_stride; /* value for mc_pair_cache.ret_prefix_stride */
   size_t total_bytes;        /* all buffers, each rounded up to 256 bytes */
+  size_t res_bytes;          /* res_k and res_v alike; 0 unless cfg->cache_bits = 4 */
 } mc_pair_sizes;
 
 /* What the last merge into a pair did (Sec. 4.2 retention, Sec. 4.3 footprint). */

@@ -33,7 +33,7 @@ class McError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("page_size", C.c_int32), ("dtype", C.c_int32), ("retain_mode", C.c_int32),
-                ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("reserved", C.c_int32)]
+                ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("cache_bits", C.c_int32)]
 
 
 class _Batch(C.Structure):
@@ -55,14 +55,15 @@ class _PairCache(C.Structure):
                 ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
                 ("ret_rows", C.c_void_p), ("ret_capacity", C.c_int64), ("ret_prefix", C.c_void_p),
                 ("ret_prefix_stride", C.c_int64), ("seg_minmax", C.c_void_p),
-                ("status", C.c_void_p)]
+                ("status", C.c_void_p), ("res_k", C.c_void_p), ("res_v", C.c_void_p)]
 
 
 class _PairSizes(C.Structure):
     _fields_ = [("tile_bytes", C.c_size_t), ("e_bytes", C.c_size_t), ("dist_bytes", C.c_size_t),
                 ("ret_count_bytes", C.c_size_t), ("ret_offset_bytes", C.c_size_t), ("ret_index_bytes", C.c_size_t),
                 ("ret_rows_bytes", C.c_size_t), ("ret_prefix_bytes", C.c_size_t), ("seg_minmax_bytes", C.c_size_t),
-                ("status_bytes", C.c_size_t), ("ret_prefix_stride", C.c_int64), ("total_bytes", C.c_size_t)]
+                ("status_bytes", C.c_size_t), ("ret_prefix_stride", C.c_int64), ("total_bytes", C.c_size_t),
+                ("res_bytes", C.c_size_t)]
 
 
 class _Stats(C.Structure):
@@ -97,11 +98,12 @@ class McConfig:
     retain_mode: int = MC_RETAIN_DISTINCT
     head_dim: int = 128
     merge_fn: int = 0  # MC_MERGE_SLERP (Eq. 3) | MC_MERGE_FMAX = 1 | MC_MERGE_MEAN = 2
+    cache_bits: int = 16  # storage of the shared directions: 16 (the 16-bit type) or 4 (4-bit shared cache, pages of 32)
 
     def c(self) -> _Config:
         return _Config(self.n_kv_heads, self.n_q_heads, self.head_dim, self.page_size,
                        {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma),
-                       int(self.merge_fn), 0)
+                       int(self.merge_fn), int(self.cache_bits))
 
     @property
     def torch_dtype(self):
@@ -151,33 +153,103 @@ class PairCache:
         self.ret_prefix = z(sz.ret_prefix_bytes).view(torch.int32).view(nseg, self.ret_prefix_stride)
         self.seg_minmax = z(sz.seg_minmax_bytes).view(torch.float32).view(nseg, 2)
         self.status = z(sz.status_bytes).view(torch.int32)
+        self.q4 = cfg.cache_bits == 4
+        self.res_k = self.res_v = None
+        if self.q4:  # one 16-bit tile of 32 tokens per (sequence, head): the last, incomplete page
+            self.res_k = z(sz.res_bytes).view(batch, H, sz.res_bytes // max(batch * H, 1))
+            self.res_v = z(sz.res_bytes).view(batch, H, sz.res_bytes // max(batch * H, 1))
 
     def c(self) -> _PairCache:
         return _PairCache(_ptr(self.e_k), _ptr(self.e_v), _ptr(self.dist), _ptr(self.ret_count),
                           _ptr(self.ret_offset), _ptr(self.ret_index), _ptr(self.ret_rows), self.ret_capacity,
-                          _ptr(self.ret_prefix), self.ret_prefix_stride, _ptr(self.seg_minmax), _ptr(self.status))
+                          _ptr(self.ret_prefix), self.ret_prefix_stride, _ptr(self.seg_minmax), _ptr(self.status),
+                          _ptr(self.res_k), _ptr(self.res_v))
 
     # -- decoding the tile layout (pure re-indexing, no arithmetic) ------------------------------
-    def directions(self, tensor: str) -> torch.Tensor:
-        """Stored directions of "k" or "v" as [n_pages][H][page_size][128] in the storage type
-        (the 16-byte chunk permutation of the tile format undone)."""
-        pool = self.e_k if tensor == "k" else self.e_v
+    def _rows16(self, pool: torch.Tensor) -> torch.Tensor:
+        """16-bit tiles [n][H][tile] -> direction rows [n][H][page_size][128] (chunk permutation undone)."""
         ps = self.cfg.page_size
-        n_pages, H = pool.shape[:2]
-        rows = pool[:, :, :ps * 256].reshape(n_pages, H, ps, 16, 16)  # [..][row][chunk position][16 bytes]
+        n, H = pool.shape[:2]
+        rows = pool[:, :, :ps * 256].reshape(n, H, ps, 16, 16)  # [..][row][chunk position][16 bytes]
         r = torch.arange(ps, device=pool.device)[:, None]
         c = torch.arange(16, device=pool.device)[None, :]
         pos = (c & 8) | ((c & 7) ^ (r & 7))  # where chunk c of row r is stored
-        idx = pos[None, None, :, :, None].expand(n_pages, H, ps, 16, 16)
-        plain = torch.gather(rows, 3, idx).reshape(n_pages, H, ps, 256)
+        idx = pos[None, None, :, :, None].expand(n, H, ps, 16, 16)
+        plain = torch.gather(rows, 3, idx).reshape(n, H, ps, 256)
         return plain.view(self.cfg.torch_dtype)
+
+    def directions(self, tensor: str) -> torch.Tensor:
+        """Stored directions of "k" or "v" as [n_pages][H][page_size][128] in the storage type
+        (the 16-byte chunk permutation of the tile format undone).  16-bit cache only."""
+        assert not self.q4, "a 4-bit cache holds codes: see q4_codes / q4_groups / residual_directions"
+        return self._rows16(self.e_k if tensor == "k" else self.e_v)
 
     def scales(self, tensor: str) -> torch.Tensor:
         """Scales of "k" or "v" as [n_pages][H][2][page_size] fp32 ([..][0]: layer l-1, [1]: layer l)."""
         pool = self.e_k if tensor == "k" else self.e_v
         ps = self.cfg.page_size
         n_pages, H = pool.shape[:2]
-        return pool[:, :, ps * 256:].contiguous().view(torch.float32).reshape(n_pages, H, 2, ps)
+        off = 2560 if self.q4 else ps * 256
+        return pool[:, :, off:].contiguous().view(torch.float32).reshape(n_pages, H, 2, ps)
+
+    # -- 4-bit shared cache: the tile's orders undone (pure re-indexing) -------------------------
+    def q4_codes(self, tensor: str) -> torch.Tensor:
+        """Codes of "k" or "v" as [n_pages][H][32][128] uint8, channels in natural order."""
+        assert self.q4
+        pool = self.e_k if tensor == "k" else self.e_v
+        n_pages, H = pool.shape[:2]
+        dev = pool.device
+        words = pool[:, :, :2048].contiguous().view(torch.int32).reshape(n_pages, H, 512).long() & 0xFFFFFFFF
+        nib = torch.stack([(words >> (4 * j)) & 15 for j in range(8)], dim=-1).to(torch.uint8)  # [..][word][nibble]
+        out = torch.zeros(n_pages, H, 32, 128, dtype=torch.uint8, device=dev)
+        if tensor == "k":
+            # row r, word w, nibble j: channel 8 w + 2 (j % 4) + j // 4
+            nib = nib.reshape(n_pages, H, 32, 16, 8)
+            w = torch.arange(16, device=dev)[:, None]
+            j = torch.arange(8, device=dev)[None, :]
+            ch = (8 * w + 2 * (j % 4) + j // 4).reshape(-1)
+            out[:, :, :, ch] = nib.reshape(n_pages, H, 32, 128)
+        else:
+            # block i (tokens 2i, 2i+1), chunk position cp, word k, nibble j: token 2i + j // 4,
+            # channel 32 k + 16 ((j % 4) // 2) + 8 (j % 2) + (cp ^ ((i % 4) * 2))
+            nib = nib.reshape(n_pages, H, 16, 8, 4, 8)
+            i = torch.arange(16, device=dev)[:, None, None, None]
+            cp = torch.arange(8, device=dev)[None, :, None, None]
+            k = torch.arange(4, device=dev)[None, None, :, None]
+            j = torch.arange(8, device=dev)[None, None, None, :]
+            tok = (2 * i + j // 4).expand(16, 8, 4, 8).reshape(-1)
+            ch = (32 * k + 16 * ((j % 4) // 2) + 8 * (j % 2) + (cp ^ ((i % 4) * 2))).expand(16, 8, 4, 8).reshape(-1)
+            out[:, :, tok, ch] = nib.reshape(n_pages, H, -1)
+        return out
+
+    def q4_groups(self, tensor: str):
+        """(scale, zero) of "k" ([n_pages][H][128], per channel) or "v" ([n_pages][H][32][4], per token and
+        channel group) in the storage type."""
+        assert self.q4
+        pool = self.e_k if tensor == "k" else self.e_v
+        n_pages, H = pool.shape[:2]
+        dev = pool.device
+        m = pool[:, :, 2048:2560].contiguous().view(self.cfg.torch_dtype)  # 256 values
+        if tensor == "k":
+            m = m.reshape(n_pages, H, 2, 16, 8)  # [scale|zero][chunk position][8 channels]
+            o = torch.arange(16, device=dev)
+            pos = 4 * (o & 3) + (o >> 2)  # where the chunk of channels [8 o, 8 o + 8) is stored
+            m = m[:, :, :, pos].reshape(n_pages, H, 2, 128)
+            return m[:, :, 0].contiguous(), m[:, :, 1].contiguous()
+        m = m.reshape(n_pages, H, 16, 2, 4, 2)  # [token pair][scale|zero][group][token of the pair]
+        m = m.permute(0, 1, 3, 2, 5, 4).reshape(n_pages, H, 2, 32, 4)
+        return m[:, :, 0].contiguous(), m[:, :, 1].contiguous()
+
+    def residual_directions(self, tensor: str) -> torch.Tensor:
+        """The residual tiles' rows [batch][H][32][128] in the storage type (tokens of the last, incomplete page)."""
+        assert self.q4
+        return self._rows16(self.res_k if tensor == "k" else self.res_v)
+
+    def residual_scales(self, tensor: str) -> torch.Tensor:
+        """The residual tiles' scales [batch][H][2][32] fp32."""
+        assert self.q4
+        pool = self.res_k if tensor == "k" else self.res_v
+        return pool[:, :, 32 * 256:].contiguous().view(torch.float32).reshape(pool.shape[0], pool.shape[1], 2, 32)
 
     def retained_rows(self, layer: int) -> torch.Tensor:
         """Raw retained rows of one layer (0: l-1, 1: l) as [ret_capacity][128] in the storage type."""
@@ -189,7 +261,7 @@ class PairCache:
 
     def nbytes(self) -> int:
         ts = (self.e_k, self.e_v, self.dist, self.ret_count, self.ret_offset, self.ret_index,
-              self.ret_rows, self.ret_prefix, self.seg_minmax, self.status)
+              self.ret_rows, self.ret_prefix, self.seg_minmax, self.status) + ((self.res_k, self.res_v) if self.q4 else ())
         return sum(t.numel() * t.element_size() for t in ts)
 
 

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libminicache.so")
-SOURCES = ["mc_api.cu", "mc_merge.cu", "mc_restore.cu", "mc_attn.cu"]
+SOURCES = ["mc_api.cu", "mc_merge.cu", "mc_restore.cu", "mc_attn.cu", "mc_q4cache.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

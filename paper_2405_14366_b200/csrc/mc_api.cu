@@ -8,6 +8,7 @@
 #include "mc_common.cuh"
 #include "mc_items.cuh"
 #include "mc_kernels.h"
+#include "mc_q4.cuh"
 
 namespace mc {
 
@@ -43,7 +44,9 @@ static mc_status check_config(const mc_config* cfg) {
   if (nq != 1 && nq != 2 && nq != 4 && nq != 8) return MC_ERR_SHAPE;
   if (cfg->dtype != MC_F16 && cfg->dtype != MC_BF16) return MC_ERR_DTYPE;
   if (cfg->retain_mode < MC_RETAIN_DISTINCT || cfg->retain_mode > MC_RETAIN_TOPK) return MC_ERR_INVALID_ARG;
-  if (cfg->merge_fn < MC_MERGE_SLERP || cfg->merge_fn > MC_MERGE_MEAN || cfg->reserved != 0) return MC_ERR_INVALID_ARG;
+  if (cfg->merge_fn < MC_MERGE_SLERP || cfg->merge_fn > MC_MERGE_MEAN) return MC_ERR_INVALID_ARG;
+  if (cfg->cache_bits != 0 && cfg->cache_bits != 16 && cfg->cache_bits != 4) return MC_ERR_INVALID_ARG;
+  if (cfg->cache_bits == 4 && cfg->page_size != kQ4Page) return MC_ERR_SHAPE;
   if (!(cfg->t >= 0.0 && cfg->t <= 1.0) || !(cfg->gamma >= 0.0 && cfg->gamma <= 1.0)) return MC_ERR_INVALID_ARG;
   return MC_OK;
 }
@@ -58,8 +61,12 @@ static mc_status check_batch(const mc_config* cfg, const mc_batch* bt) {
   return MC_OK;
 }
 
-static mc_status check_pair(const mc_pair_cache* pc) {
+static mc_status check_pair(const mc_config* cfg, const mc_pair_cache* pc) {
   if (pc == nullptr) return MC_ERR_INVALID_ARG;
+  if (cfg->cache_bits == 4) {
+    if (!pc->res_k || !pc->res_v) return MC_ERR_INVALID_ARG;
+    if (!aligned256(pc->res_k) || !aligned256(pc->res_v)) return MC_ERR_ALIGN;
+  }
   if (!pc->e_k || !pc->e_v || !pc->dist || !pc->ret_count || !pc->ret_offset || !pc->seg_minmax ||
       !pc->status)
     return MC_ERR_INVALID_ARG;
@@ -82,6 +89,27 @@ static Geom make_geom(const mc_config* cfg, const mc_batch* bt) {
   g.max_seq_len = bt->max_seq_len;
   g.n_pages = (int)bt->n_pages;
   return g;
+}
+
+// Merge scratch: the retention tables, and for the 4-bit shared cache the 16-bit staging tiles of both tensors.
+static size_t merge_workspace_total(const mc_config* cfg, const mc_batch* bt) {
+  return merge_workspace_bytes(cfg, bt) + (cfg->cache_bits == 4 ? 2 * q4_stage_bytes(cfg, bt) : 0);
+}
+
+// Runs the merge; with a 4-bit shared cache the kernels write 16-bit tiles into the staging part of the
+// workspace (retention marks its tokens there), which then become 4-bit tiles and residual tiles.
+static mc_status run_merge(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1, const mc_layer_kv* l,
+                           const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out, int do_retention,
+                           void* workspace, cudaStream_t stream) {
+  const Geom g = make_geom(cfg, batch);
+  if (cfg->cache_bits != 4) return launch_merge(cfg, batch, g, lm1, l, q_lm1, q_l, out, do_retention, workspace, stream);
+  mc_pair_cache stg = *out;
+  char* base = (char*)workspace + merge_workspace_bytes(cfg, batch);
+  stg.e_k = base;
+  stg.e_v = base + q4_stage_bytes(cfg, batch);
+  mc_status st = launch_merge(cfg, batch, g, lm1, l, q_lm1, q_l, &stg, do_retention, workspace, stream);
+  if (st != MC_OK) return st;
+  return launch_q4_quantise(cfg, batch, g, stg.e_k, stg.e_v, out, stream);
 }
 
 }  // namespace mc
@@ -116,7 +144,8 @@ mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_
   if (batch == nullptr || bytes == nullptr) return MC_ERR_INVALID_ARG;
   if (batch->batch < 0 || batch->max_seq_len < 0) return MC_ERR_INVALID_ARG;
   if (op == MC_OP_MERGE) {
-    *bytes = merge_workspace_bytes(cfg, batch) + 256;
+    if (batch->n_pages < 0) return MC_ERR_INVALID_ARG;
+    *bytes = merge_workspace_total(cfg, batch) + 256;
   } else if (op == MC_OP_DECODE_ATTN) {
     if (n_query_sets != 1 && n_query_sets != 2) return MC_ERR_INVALID_ARG;
     *bytes = attn_workspace_bytes(cfg, batch, n_query_sets) + 256;
@@ -129,11 +158,11 @@ mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_
 // What every form of the merge call checks about the output pair and the scratch memory.
 static mc_status check_merge_common(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* out, void* workspace,
                                     size_t workspace_bytes) {
-  mc_status st = check_pair(out);
+  mc_status st = check_pair(cfg, out);
   if (st != MC_OK) return st;
   if (batch->batch > kMaxBatchPages) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
   if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
-  if (workspace_bytes < merge_workspace_bytes(cfg, batch)) return MC_ERR_CAPACITY;
+  if (workspace_bytes < merge_workspace_total(cfg, batch)) return MC_ERR_CAPACITY;
   if (out->ret_prefix_stride < (batch->max_seq_len + 127) / 128 + 1) return MC_ERR_CAPACITY;
   return MC_OK;
 }
@@ -146,8 +175,10 @@ mc_status mc_pair_bytes(const mc_config* cfg, const mc_batch* batch, int64_t ret
   const size_t nseg = (size_t)2 * batch->batch * cfg->n_kv_heads;
   const size_t ph = (size_t)batch->n_pages * cfg->n_kv_heads;
   memset(out, 0, sizeof(*out));
-  out->tile_bytes = (size_t)tile_bytes(cfg->page_size);
+  const bool q4 = cfg->cache_bits == 4;
+  out->tile_bytes = q4 ? (size_t)kQ4TileBytes : (size_t)tile_bytes(cfg->page_size);
   out->e_bytes = ph * out->tile_bytes;
+  out->res_bytes = q4 ? (size_t)batch->batch * cfg->n_kv_heads * kResTileBytes : 0;
   out->dist_bytes = ph * 2 * cfg->page_size * sizeof(float);
   out->ret_count_bytes = nseg * sizeof(int32_t);
   out->ret_offset_bytes = (nseg + 1) * sizeof(int32_t);
@@ -159,7 +190,7 @@ mc_status mc_pair_bytes(const mc_config* cfg, const mc_batch* batch, int64_t ret
   out->status_bytes = MC_STATUS_WORDS * sizeof(int32_t);
   const size_t parts[] = {out->e_bytes, out->e_bytes, out->dist_bytes, out->ret_count_bytes, out->ret_offset_bytes,
                           out->ret_index_bytes, out->ret_rows_bytes, out->ret_prefix_bytes, out->seg_minmax_bytes,
-                          out->status_bytes};
+                          out->status_bytes, out->res_bytes, out->res_bytes};
   for (size_t b : parts) out->total_bytes += align_up(b, 256);
   return MC_OK;
 }
@@ -180,11 +211,12 @@ mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pai
   if (batch->batch > 0)
     MC_CUDA_CHECK(cudaMemcpyAsync(lens, batch->seq_lens, (size_t)batch->batch * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   MC_CUDA_CHECK(cudaStreamSynchronize(s));
-  int64_t tokens = 0, pages = 0;
+  int64_t tokens = 0, pages = 0, tokens_q = 0;
   for (int b = 0; b < batch->batch; ++b) {
     const int64_t n = lens[b] < 0 ? 0 : lens[b];
     tokens += n;
     pages += (n + cfg->page_size - 1) / cfg->page_size;
+    tokens_q += n / kQ4Page * kQ4Page;  // tokens in complete pages
   }
   const int64_t th = tokens * cfg->n_kv_heads;  // (token, kv head) rows per layer and tensor
   out->flags = words[MC_STATUS_FLAGS];
@@ -195,10 +227,19 @@ mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pai
   // the shared direction row, both magnitudes and the distance per (token, head, tensor); both raw rows
   // and the index per retained entry
   out->compressed_bytes = 2 * th * (kRowBytes + 3 * 4) + out->retained_total * (2 * kRowBytes + 4);
+  if (cfg->cache_bits == 4) {
+    // a row in a complete page: 64 bytes of codes and its share of the group parameters (keys: 128 x 4
+    // bytes per 32 tokens, values: 4 x 4 bytes per token: 16 either way); the residual rows stay 16-bit
+    const int64_t thq = tokens_q * cfg->n_kv_heads;
+    out->compressed_bytes = 2 * thq * (64 + 16 + 3 * 4) + 2 * (th - thq) * (kRowBytes + 3 * 4) +
+                            out->retained_total * (2 * kRowBytes + 4);
+  }
   // what the pair occupies in the caller's buffers: whole tiles of the pages in use, the distances, the
   // padded retained entries, the per-segment tables
   const int64_t nseg = 2LL * batch->batch * cfg->n_kv_heads;
-  out->stored_bytes = 2 * pages * cfg->n_kv_heads * ((int64_t)tile_bytes(cfg->page_size) + cfg->page_size * 4) +
+  const int64_t tile_b = cfg->cache_bits == 4 ? kQ4TileBytes : tile_bytes(cfg->page_size);
+  const int64_t res_b = cfg->cache_bits == 4 ? 2LL * batch->batch * cfg->n_kv_heads * kResTileBytes : 0;
+  out->stored_bytes = res_b + 2 * pages * cfg->n_kv_heads * (tile_b + cfg->page_size * 4) +
                       out->retained_total * (2 * kRetEntryBytes + 4) +
                       nseg * (4 + 4 + 8 + 4 * pair->ret_prefix_stride) + 4 + MC_STATUS_WORDS * 4;
   if (out->flags & MC_FLAG_RETAIN_OVERFLOW) return MC_ERR_CAPACITY;
@@ -218,8 +259,7 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
     return MC_ERR_ALIGN;
   st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
   if (st != MC_OK) return st;
-  return launch_merge(cfg, batch, make_geom(cfg, batch), lm1, l, nullptr, nullptr, out, do_retention ? 1 : 0, workspace,
-                      (cudaStream_t)stream);
+  return run_merge(cfg, batch, lm1, l, nullptr, nullptr, out, do_retention ? 1 : 0, workspace, (cudaStream_t)stream);
 }
 
 mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc_layer_q4* lm1, const mc_layer_q4* l,
@@ -238,8 +278,7 @@ mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc
   }
   st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
   if (st != MC_OK) return st;
-  return launch_merge(cfg, batch, make_geom(cfg, batch), nullptr, nullptr, lm1, l, out, do_retention ? 1 : 0, workspace,
-                      (cudaStream_t)stream);
+  return run_merge(cfg, batch, nullptr, nullptr, lm1, l, out, do_retention ? 1 : 0, workspace, (cudaStream_t)stream);
 }
 
 mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, const void* k_new_lm1,
@@ -248,11 +287,13 @@ mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_p
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
   if (st != MC_OK) return st;
-  st = check_pair(pair);
+  st = check_pair(cfg, pair);
   if (st != MC_OK) return st;
   if (!k_new_lm1 || !v_new_lm1 || !k_new_l || !v_new_l) return MC_ERR_INVALID_ARG;
   const uintptr_t al = (uintptr_t)k_new_lm1 | (uintptr_t)v_new_lm1 | (uintptr_t)k_new_l | (uintptr_t)v_new_l;
   if (al & 15u) return MC_ERR_ALIGN;
+  if (cfg->cache_bits == 4)
+    return launch_append_q4(cfg, batch, make_geom(cfg, batch), pair, k_new_lm1, v_new_lm1, k_new_l, v_new_l, (cudaStream_t)stream);
   return launch_append(cfg, batch, make_geom(cfg, batch), pair, k_new_lm1, v_new_lm1, k_new_l, v_new_l,
                        (cudaStream_t)stream);
 }
@@ -263,12 +304,14 @@ mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
   if (st != MC_OK) return st;
-  st = check_pair(pair);
+  st = check_pair(cfg, pair);
   if (st != MC_OK) return st;
   if (layer_sel != MC_LAYER_LM1 && layer_sel != MC_LAYER_L) return MC_ERR_INVALID_ARG;
   if (!dst || !dst->k_pool || !dst->v_pool) return MC_ERR_INVALID_ARG;
   if (!aligned256(dst->k_pool) || !aligned256(dst->v_pool)) return MC_ERR_ALIGN;
   if (batch->batch > kMaxBatchPages) return MC_ERR_SHAPE;
+  if (cfg->cache_bits == 4)
+    return launch_restore_q4(cfg, batch, make_geom(cfg, batch), pair, layer_sel, dst, dst_fp32 ? 1 : 0, (cudaStream_t)stream);
   return launch_restore(cfg, batch, make_geom(cfg, batch), pair, layer_sel, dst, dst_fp32 ? 1 : 0, (cudaStream_t)stream);
 }
 
@@ -279,7 +322,7 @@ mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_p
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
   if (st != MC_OK) return st;
-  st = check_pair(pair);
+  st = check_pair(cfg, pair);
   if (st != MC_OK) return st;
   if (layer_sel < MC_LAYER_LM1 || layer_sel > MC_LAYER_BOTH) return MC_ERR_INVALID_ARG;
   const int n_sets = layer_sel == MC_LAYER_BOTH ? 2 : 1;

@@ -30,6 +30,7 @@
 #include "mc_common.cuh"
 #include "mc_kernels.h"
 #include "mc_pipe.cuh"
+#include "mc_q4.cuh"
 
 namespace mc {
 
@@ -48,6 +49,7 @@ constexpr int kSlabStride = 132;  // floats per row of a warp's partial output i
 struct AttnParams {
   Geom g;
   const char* e_pool[2];  // compressed tiles: K, V
+  const char* res_pool[2];  // 4-bit cache: the residual 16-bit tiles [batch][H][kResTileBytes]
   const int32_t* ret_offset;
   const int32_t* ret_prefix;
   int ret_prefix_stride;
@@ -150,6 +152,10 @@ struct Item {
   int split_start;  // first token of this chunk
   int n_tok;    // cached tokens of this chunk
   int T;        // 64-token tiles
+  int n_q;      // 4-bit cache: tokens of this chunk that live in 4-bit pages (a multiple of 32; the rest,
+                // at most 31 at the sequence's end, sit in the residual tile)
+  int Tq;       // 4-bit cache: stages of up to four 4-bit pages (128 tokens)
+  int TT;       // tile stages of a phase: T, or Tq plus one for the residual tile
   int units;
   bool first, last;  // first / last chunk of its piece
   bool has_new;
@@ -167,12 +173,13 @@ struct Item {
 struct Cursor {
   int g, x;  // kv head, unit
 };
+template <bool Q4>
 __device__ __forceinline__ Item piece_at(const Cursor& c, int x_begin, int x_end, const int* pre_s, const int* len_s,
                                          const AttnParams& p) {
   Item it;
   it.valid = c.g < p.g.n_kv_heads && c.x < x_end;
   if (!it.valid) {
-    it.b = it.g = it.split = it.split_start = it.n_tok = it.T = it.units = 0;
+    it.b = it.g = it.split = it.split_start = it.n_tok = it.T = it.units = it.n_q = it.Tq = it.TT = 0;
     it.has_new = it.first = it.last = false;
     return it;
   }
@@ -195,6 +202,9 @@ __device__ __forceinline__ Item piece_at(const Cursor& c, int x_begin, int x_end
   it.split_start = k * kUnit;
   it.n_tok = max(0, min(n, (k + it.units) * kUnit) - it.split_start);
   it.T = (it.n_tok + kTile - 1) / kTile;
+  it.n_q = Q4 ? max(0, min(it.n_tok, (n & ~(kQ4Page - 1)) - it.split_start)) : 0;
+  it.Tq = (it.n_q + kUnit - 1) / kUnit;
+  it.TT = Q4 ? it.Tq + (it.n_tok > it.n_q ? 1 : 0) : it.T;
   it.has_new = (p.k_new != nullptr) && (k + it.units == u_b);
   return it;
 }
@@ -248,7 +258,11 @@ __device__ __forceinline__ Ranges ranges_of(const RawRanges& q) {
   return r;
 }
 
-template <int DT>
+// Q4: the pair is a 4-bit shared cache (pages of 32 tokens): a tile stage holds up to four 4-bit tiles
+// (128 tokens, one page per consumer warp), whose tensor-core fragments are built in registers straight
+// from the codes (code * scale + zero in one packed 16-bit FMA, the exact stored direction); the tokens
+// of a sequence's last, incomplete page arrive as one more tile stage in the 16-bit format.
+template <int DT, bool Q4>
 __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(const AttnParams p) {
   // The batch description (lengths, block table) and the queries belong to the caller: no kernel of
   // this library writes them, so they are read before the wait on the previous kernel in the
@@ -325,7 +339,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     // engine saturates the memory system.
     int it = 0;  // running stage counter, same sequence as the consumers'
     Cursor cur = c_first;
-    Item w = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
+    Item w = piece_at<Q4>(cur, x_begin, x_end, pre_s, len_s, p);
     RawRanges raw;
     // page ids of a piece: lane l holds pages l, l + 32, ... (registers, loaded one piece ahead),
     // handed over to shared memory when the piece starts
@@ -360,7 +374,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       for (int r = 0; r < kMaxPiecePages / 32; ++r) pages[lane + 32 * r] = pg_reg[r];
       __syncwarp();
       cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
-      const Item wn = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
+      const Item wn = piece_at<Q4>(cur, x_begin, x_end, pre_s, len_s, p);
       const RawRanges rawn = load_ranges(wn, p);
       load_pages(wn);
       if (bad_meta) {
@@ -376,13 +390,13 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         int n_r = 0, r_lo = 0;
         int X = -1;  // extra stages: retained rows and the new token
         for (int t = 0;; ++t, ++it) {
-          if (X < 0 && t >= w.T - 1) {
+          if (X < 0 && t >= w.TT - 1) {
             const Ranges rg = ranges_of(raw);
             n_r = ph ? rg.n_v : rg.n_k;
             r_lo = ph ? rg.v_lo : rg.k_lo;
             X = (n_r + n_new + cap_e - 1) / cap_e;
           }
-          if (X >= 0 && t >= w.T + X) break;
+          if (X >= 0 && t >= w.TT + X) break;
           const int s = it % kStages;
           if (it >= kStages) {
             int good = 1;
@@ -392,7 +406,29 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
           }
           const uint32_t bar = full0 + 8 * s;
           const uint32_t sbase = stage0 + s * kStageBytes;
-          if (t < w.T) {
+          if (Q4 && t < w.Tq) {
+            // ---- up to four 4-bit pages (128 tokens): a bulk copy per page
+            const int n_pg = min(kUnit / kQ4Page, (w.n_q >> 5) - t * (kUnit / kQ4Page));
+            if (lane == 0) {
+              info_s[2 * s] = 0;
+              info_s[2 * s + 1] = X;
+              mbar_expect_tx(bar, (uint32_t)(n_pg * kQ4TileBytes));
+            }
+            __syncwarp();
+            if (lane < n_pg)
+              bulk_load(sbase + lane * kQ4TileBytes,
+                        p.e_pool[ph] + ((size_t)pages[t * (kUnit / kQ4Page) + lane] * H + w.g) * kQ4TileBytes,
+                        (uint32_t)kQ4TileBytes, bar);
+          } else if (Q4 && t < w.TT) {
+            // ---- the residual tile: the sequence's last, incomplete page in 16 bits
+            if (lane == 0) {
+              info_s[2 * s] = 0;
+              info_s[2 * s + 1] = X;
+              mbar_expect_tx(bar, (uint32_t)kResTileBytes);
+              bulk_load(sbase, p.res_pool[ph] + ((size_t)w.b * H + w.g) * kResTileBytes, (uint32_t)kResTileBytes, bar);
+            }
+            __syncwarp();
+          } else if (t < w.TT) {
             // ---- one 64-token tile: a bulk copy per page
             const int pg0 = (t * kTile) >> shift;
             const int n_pg = min(kTile >> shift, n_pages_item - pg0);
@@ -407,7 +443,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
                         bar);
           } else {
             // ---- an extra stage: up to cap_e retained entries per layer, the new token last
-            const int x0 = (t - w.T) * cap_e;
+            const int x0 = (t - w.TT) * cap_e;
             const int cnt_ret = max(0, min(n_r, x0 + cap_e) - x0);
             const bool add_new = n_new && n_r >= x0 && n_r < x0 + cap_e;
             if (lane == 0) {
@@ -467,7 +503,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   };
   {
     uint32_t qw[4];
-    load_q_words(piece_at(c_first, x_begin, x_end, pre_s, len_s, p), qw);
+    load_q_words(piece_at<Q4>(c_first, x_begin, x_end, pre_s, len_s, p), qw);
 #pragma unroll
     for (int k = 0; k < 4; ++k) q_s[tid + k * kConsumerThreads] = qw[k];
   }
@@ -482,7 +518,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   float l_acc = 0.f, m_run = -INFINITY, m_run0 = -INFINITY, m_run1 = -INFINITY;
   Cursor cur = c_first;
   for (;; ++n_item) {
-    const Item w = piece_at(cur, x_begin, x_end, pre_s, len_s, p);
+    const Item w = piece_at<Q4>(cur, x_begin, x_end, pre_s, len_s, p);
     if (!w.valid) break;
     cur = next_cursor(cur, w, x_begin, x_end, p.team_size);
     const uint32_t* qcur = q_s + (n_item & 1) * kMaxRows * 64;
@@ -498,14 +534,88 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         qa0[ks] = qcur[row * 64 + ks * 8 + (lane & 3)];
         qa2[ks] = qcur[row * 64 + ks * 8 + 4 + (lane & 3)];
       }
+      // 4-bit tiles: lane (row, t4) owns the channels [32 t4, 32 t4 + 32) of its token rows (16 bytes of
+      // codes); k step ks pairs the channels 32 t4 + 4 ks + {0, 1} and + {2, 3} with the matching query words
+      uint32_t qk0[8], qk2[8];
+      if (Q4) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          qk0[ks] = qcur[row * 64 + 16 * (lane & 3) + 2 * ks];
+          qk2[ks] = qcur[row * 64 + 16 * (lane & 3) + 2 * ks + 1];
+        }
+      }
       const int tk_w = warp * 16;  // this warp's 16 tokens of every tile
       int xk = n_new;              // extra stages after the tiles (an item without tiles has no retained rows)
-      for (int t = 0; t < w.T; ++t, ++it) {
+      for (int t = 0; t < w.TT; ++t, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const uint32_t sbase = stage0 + s * kStageBytes;
-        const int valid = min(kTile, w.n_tok - t * kTile);
         xk = info_s[2 * s + 1];
+        if (Q4 && t < w.Tq) {
+          // ---- four 4-bit pages, one per warp
+          if (warp < (w.n_q >> 5) - t * (kUnit / kQ4Page)) {
+            const unsigned char* tb = stages + s * kStageBytes + warp * kQ4TileBytes;
+            const int t4 = lane & 3;
+            uint4 sK[4], zK[4];  // the group parameters of this lane's 32 channels, word k = channels 8 (4 t4 + k) + ...
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              sK[k] = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + (4 * k + t4) * 16);
+              zK[k] = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + 256 + (4 * k + t4) * 16);
+            }
+            const float* gq = reinterpret_cast<const float*>(tb + kQ4ScaleOff);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              const int ra_ = 16 * hf + row;  // this lane's token rows inside the page: ra_, ra_ + 8
+              const uint4 wA = *reinterpret_cast<const uint4*>(tb + ra_ * 64 + t4 * 16);
+              const uint4 wB = *reinterpret_cast<const uint4*>(tb + (ra_ + 8) * 64 + t4 * 16);
+              const uint32_t wa[4] = {wA.x, wA.y, wA.z, wA.w}, wb[4] = {wB.x, wB.y, wB.z, wB.w};
+              float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                uint32_t cA[4], cB[4];
+                code_pairs<DT>(wa[k], cA);
+                code_pairs<DT>(wb[k], cB);
+                const uint32_t sk[4] = {sK[k].x, sK[k].y, sK[k].z, sK[k].w}, zk[4] = {zK[k].x, zK[k].y, zK[k].z, zK[k].w};
+                mma_rows<DT>(acc0, deq_pair<DT>(cA[0], sk[0], zk[0]), deq_pair<DT>(cB[0], sk[0], zk[0]),
+                             deq_pair<DT>(cA[1], sk[1], zk[1]), deq_pair<DT>(cB[1], sk[1], zk[1]), qk0[2 * k], qk2[2 * k]);
+                mma_rows<DT>(acc1, deq_pair<DT>(cA[2], sk[2], zk[2]), deq_pair<DT>(cB[2], sk[2], zk[2]),
+                             deq_pair<DT>(cA[3], sk[3], zk[3]), deq_pair<DT>(cB[3], sk[3], zk[3]), qk0[2 * k + 1], qk2[2 * k + 1]);
+              }
+              // this thread: tokens ra_ and ra_ + 8 of the page, query rows colp and colp + 1
+              if (colp < rows) {
+                float* scol = S + t * kUnit + warp * kQ4Page + ra_;
+                const float g0 = gq[slot0 * kQ4Page + ra_], g8 = gq[slot0 * kQ4Page + ra_ + 8];
+                const float s00 = (acc0[0] + acc1[0]) * (g0 * p.scale_log2), s08 = (acc0[2] + acc1[2]) * (g8 * p.scale_log2);
+                if (!is_retained_scale(g0)) {
+                  scol[colp * s_stride] = s00;
+                  mx0 = fmaxf(mx0, s00);
+                }
+                if (!is_retained_scale(g8)) {
+                  scol[colp * s_stride + 8] = s08;
+                  mx0 = fmaxf(mx0, s08);
+                }
+                if (colp + 1 < rows) {
+                  const float h0 = gq[slot1 * kQ4Page + ra_], h8 = gq[slot1 * kQ4Page + ra_ + 8];
+                  const float s10 = (acc0[1] + acc1[1]) * (h0 * p.scale_log2), s18 = (acc0[3] + acc1[3]) * (h8 * p.scale_log2);
+                  if (!is_retained_scale(h0)) {
+                    scol[(colp + 1) * s_stride] = s10;
+                    mx1 = fmaxf(mx1, s10);
+                  }
+                  if (!is_retained_scale(h8)) {
+                    scol[(colp + 1) * s_stride + 8] = s18;
+                    mx1 = fmaxf(mx1, s18);
+                  }
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty0 + 8 * s);
+          continue;
+        }
+        // a 16-bit tile stage: 64 tokens of pages, or (4-bit cache) the residual tile behind the 4-bit pages
+        const int s_off = Q4 ? w.n_q : t * kTile;
+        const int valid = Q4 ? w.n_tok - w.n_q : min(kTile, w.n_tok - t * kTile);
         if (tk_w < valid) {
           // A = the warp's 16 token rows (k step: 16 channels), B = the query rows: D[token][row]
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};  // even / odd k steps
@@ -531,7 +641,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
                               (tk & (ps - 1));
             const float* sc8 = reinterpret_cast<const float*>(stages + s * kStageBytes + ((tk + 8) >> shift) * tbytes +
                                                               ps * kRowBytes) + ((tk + 8) & (ps - 1));
-            float* scol = S + t * kTile + tk;
+            float* scol = S + s_off + tk;
             const float g0 = sc[slot0 * ps], g8 = sc8[slot0 * ps];
             const bool u0 = tk < valid && !is_retained_scale(g0), u8 = tk + 8 < valid && !is_retained_scale(g8);
             const float s00 = (acc0[0] + acc1[0]) * (g0 * p.scale_log2), s08 = (acc0[2] + acc1[2]) * (g8 * p.scale_log2);
@@ -650,7 +760,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
 
     // query rows of the next item travel while the V tiles stream
     uint32_t qnext[4];
-    load_q_words(piece_at(cur, x_begin, x_end, pre_s, len_s, p), qnext);
+    load_q_words(piece_at<Q4>(cur, x_begin, x_end, pre_s, len_s, p), qnext);
 
     // ---- V phase: O[r][:] = sum_i (P[r][i] g_i) e_i -----------------------------------------------
     // A = the warp's 16 token rows transposed (16 channels x 16 tokens per m tile), B = the rows'
@@ -661,12 +771,64 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     const uint32_t vsw_lo = (uint32_t)(((mi & 1) ^ (mr & 1)) | (mr & 6));
     if (ok) {
       int xv = n_new;
-      for (int t = 0; t < w.T; ++t, ++it) {
+      for (int t = 0; t < w.TT; ++t, ++it) {
         const int s = it % kStages;
         if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
         const uint32_t sbase = stage0 + s * kStageBytes;
-        const int valid = min(kTile, w.n_tok - t * kTile);
         xv = info_s[2 * s + 1];
+        if (Q4 && t < w.Tq) {
+          // ---- four 4-bit pages, one per warp: lane (row, t4) owns the channels row, row + 8 (mod 16)
+          // of the token pairs t4, t4 + 4 of each half page: one 16-byte chunk of codes per pair
+          if (warp < (w.n_q >> 5) - t * (kUnit / kQ4Page)) {
+            const unsigned char* tb = stages + s * kStageBytes + warp * kQ4TileBytes;
+            const int t4 = lane & 3;
+            const float* gq = reinterpret_cast<const float*>(tb + kQ4ScaleOff) + slot_row * kQ4Page;
+            const float* srow = S + row * s_stride + t * kUnit + warp * kQ4Page;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              // B fragment: row `row`, tokens 16 hf + colp, + 1, + 8, + 9 of the page
+              uint32_t b0 = 0u, b1 = 0u;
+              if (row < rows) {
+                const float2 p0 = *reinterpret_cast<const float2*>(srow + 16 * hf + colp);
+                const float2 p1 = *reinterpret_cast<const float2*>(srow + 16 * hf + 8 + colp);
+                const float2 g0 = *reinterpret_cast<const float2*>(gq + 16 * hf + colp);
+                const float2 g1 = *reinterpret_cast<const float2*>(gq + 16 * hf + 8 + colp);
+                // (a retained token's column holds the score of its raw row; its scale -0 removes it here)
+                const float e0 = exp2f(p0.x - m_row), e1 = exp2f(p0.y - m_row);
+                const float e2 = exp2f(p1.x - m_row), e3 = exp2f(p1.y - m_row);
+                l_acc += (e0 + e1) + (e2 + e3);
+                b0 = Elem<DT>::pack(e0 * g0.x, e1 * g0.y);
+                b1 = Elem<DT>::pack(e2 * g1.x, e3 * g1.y);
+              }
+              const int i0 = 8 * hf + t4, i1 = i0 + 4;  // token pairs (2 i0, 2 i0 + 1), (2 i1, 2 i1 + 1)
+              const uint32_t cpos = (uint32_t)(row ^ (t4 << 1)) << 4;
+              const uint4 w0 = *reinterpret_cast<const uint4*>(tb + i0 * 128 + cpos);
+              const uint4 w1 = *reinterpret_cast<const uint4*>(tb + i1 * 128 + cpos);
+              const uint4 s0 = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + i0 * 32);
+              const uint4 z0 = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + i0 * 32 + 16);
+              const uint4 s1 = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + i1 * 32);
+              const uint4 z1 = *reinterpret_cast<const uint4*>(tb + kQ4CodeBytes + i1 * 32 + 16);
+              const uint32_t w0a[4] = {w0.x, w0.y, w0.z, w0.w}, w1a[4] = {w1.x, w1.y, w1.z, w1.w};
+              const uint32_t s0a[4] = {s0.x, s0.y, s0.z, s0.w}, z0a[4] = {z0.x, z0.y, z0.z, z0.w};
+              const uint32_t s1a[4] = {s1.x, s1.y, s1.z, s1.w}, z1a[4] = {z1.x, z1.y, z1.z, z1.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {  // word k = channel group k: m tiles 2 k and 2 k + 1
+                uint32_t c0[4], c1[4];
+                code_pairs<DT>(w0a[k], c0);
+                code_pairs<DT>(w1a[k], c1);
+                mma_rows<DT>(acc[2 * k], deq_pair<DT>(c0[0], s0a[k], z0a[k]), deq_pair<DT>(c0[1], s0a[k], z0a[k]),
+                             deq_pair<DT>(c1[0], s1a[k], z1a[k]), deq_pair<DT>(c1[1], s1a[k], z1a[k]), b0, b1);
+                mma_rows<DT>(acc[2 * k + 1], deq_pair<DT>(c0[2], s0a[k], z0a[k]), deq_pair<DT>(c0[3], s0a[k], z0a[k]),
+                             deq_pair<DT>(c1[2], s1a[k], z1a[k]), deq_pair<DT>(c1[3], s1a[k], z1a[k]), b0, b1);
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty0 + 8 * s);
+          continue;
+        }
+        const int s_off = Q4 ? w.n_q : t * kTile;
+        const int valid = Q4 ? w.n_tok - w.n_q : min(kTile, w.n_tok - t * kTile);
         bool wrote = false;
         if (tk_w < valid) {
           if (valid < tk_w + 16) {
@@ -684,7 +846,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
           if (row < rows) {
             const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk_w >> shift) * tbytes +
                                                               ps * kRowBytes) + slot_row * ps + (tk_w & (ps - 1));
-            const float* srow = S + row * s_stride + t * kTile + tk_w;
+            const float* srow = S + row * s_stride + s_off + tk_w;
             const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
             const float2 p1 = *reinterpret_cast<const float2*>(srow + 8 + colp);
             const float2 g0 = *reinterpret_cast<const float2*>(scj + colp);
@@ -981,6 +1143,9 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.g = g;
   ap.e_pool[0] = (const char*)pair->e_k;
   ap.e_pool[1] = (const char*)pair->e_v;
+  const bool q4 = cfg->cache_bits == 4;
+  ap.res_pool[0] = q4 ? (const char*)pair->res_k : nullptr;
+  ap.res_pool[1] = q4 ? (const char*)pair->res_v : nullptr;
   ap.ret_offset = pair->ret_offset;
   ap.ret_prefix = pair->ret_prefix;
   ap.ret_prefix_stride = (int)pair->ret_prefix_stride;
@@ -1018,19 +1183,16 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   // many output rows: a warp per row; few: a block per row
   const bool warp_rows = (long long)ap.n_sets * bt->batch * cfg->n_q_heads >= 1024;
   dim3 cgrid(warp_rows ? (cfg->n_q_heads + kCombineWarps - 1) / kCombineWarps : cfg->n_q_heads, bt->batch, ap.n_sets);
-  if (cfg->dtype == MC_F16) {
-    MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_F16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
-    MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(warp_rows ? attn_combine_kernel<MC_F16, kCombineWarps> : attn_combine_kernel<MC_F16, 1>, dim3(cgrid),
-                             dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
-  } else {
-    MC_CUDA_CHECK(cudaFuncSetAttribute(attn_split_kernel<MC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    MC_CUDA_CHECK(launch_pdl(attn_split_kernel<MC_BF16>, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
-    MC_CUDA_CHECK(cudaGetLastError());
-    MC_CUDA_CHECK(launch_pdl(warp_rows ? attn_combine_kernel<MC_BF16, kCombineWarps> : attn_combine_kernel<MC_BF16, 1>, dim3(cgrid),
-                             dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
-  }
+  void (*split)(const AttnParams) =
+      cfg->dtype == MC_F16 ? (q4 ? attn_split_kernel<MC_F16, true> : attn_split_kernel<MC_F16, false>)
+                           : (q4 ? attn_split_kernel<MC_BF16, true> : attn_split_kernel<MC_BF16, false>);
+  void (*combine)(const AttnParams, unsigned short*, float*) =
+      cfg->dtype == MC_F16 ? (warp_rows ? attn_combine_kernel<MC_F16, kCombineWarps> : attn_combine_kernel<MC_F16, 1>)
+                           : (warp_rows ? attn_combine_kernel<MC_BF16, kCombineWarps> : attn_combine_kernel<MC_BF16, 1>);
+  MC_CUDA_CHECK(cudaFuncSetAttribute(split, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  MC_CUDA_CHECK(launch_pdl(split, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
+  MC_CUDA_CHECK(cudaGetLastError());
+  MC_CUDA_CHECK(launch_pdl(combine, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }

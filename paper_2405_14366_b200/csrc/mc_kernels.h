@@ -17,6 +17,18 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
 mc_status launch_restore(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                          int layer, const mc_layer_kv* dst, int dst_fp32, cudaStream_t stream);
 
+// The 4-bit shared cache (cfg->cache_bits = 4).  The merge writes 16-bit tiles into a staging area
+// (q4_stage_bytes per tensor, part of the merge workspace), which launch_q4_quantise turns into 4-bit
+// tiles and residual tiles.
+size_t q4_stage_bytes(const mc_config* cfg, const mc_batch* bt);
+mc_status launch_q4_quantise(const mc_config* cfg, const mc_batch* bt, const Geom& g, const void* stage_k, const void* stage_v,
+                             const mc_pair_cache* out, cudaStream_t stream);
+mc_status launch_append_q4(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
+                           const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
+                           cudaStream_t stream);
+mc_status launch_restore_q4(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair, int layer,
+                            const mc_layer_kv* dst, int dst_fp32, cudaStream_t stream);
+
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets);
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                              int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,

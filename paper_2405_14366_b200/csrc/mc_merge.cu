@@ -38,78 +38,6 @@ struct MergeParams {
   int32_t* status;
 };
 
-// One merged row: 16 lanes hold 8 channels each of a (layer l-1) and c (layer l).
-template <int DT>
-__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, int fn, uint4& e_out,
-                                          float& g_a, float& g_c, float& d_out) {
-  float a[8], c[8];
-  {
-    const uint32_t wa[4] = {ra.x, ra.y, ra.z, ra.w};
-    const uint32_t wc[4] = {rc.x, rc.y, rc.z, rc.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float2 fa = Elem<DT>::unpack(wa[i]);
-      float2 fc = Elem<DT>::unpack(wc[i]);
-      a[2 * i] = fa.x;
-      a[2 * i + 1] = fa.y;
-      c[2 * i] = fc.x;
-      c[2 * i + 1] = fc.y;
-    }
-  }
-  float aa = 0.f, cc = 0.f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    aa = fmaf(a[i], a[i], aa);
-    cc = fmaf(c[i], c[i], cc);
-  }
-  aa = sum16(aa);
-  cc = sum16(cc);
-  const float ia = aa > 0.f ? rsqrtf(aa) : 0.f;
-  const float ic = cc > 0.f ? rsqrtf(cc) : 0.f;
-  // |u - v|^2 and |u + v|^2 formed channel by channel: no cancellation at small or large angles
-  float sm = 0.f, sp = 0.f;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const float u = a[i] * ia;
-    const float dm = fmaf(-c[i], ic, u);
-    const float dp = fmaf(c[i], ic, u);
-    sm = fmaf(dm, dm, sm);
-    sp = fmaf(dp, dp, sp);
-  }
-  sm = sum16(sm);
-  sp = sum16(sp);
-  RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
-  if (fn != MC_MERGE_SLERP) {  // one vector for both layers: direction of the mean, one magnitude
-    float m2 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float h = a[i] + c[i];
-      m2 = fmaf(h, h, m2);
-    }
-    m2 = 0.25f * sum16(m2);
-    const float im = m2 > 0.f ? rsqrtf(m2) : 0.f;
-    s.fa = s.fc = 0.5f * im;
-    s.na = s.nc = fn == MC_MERGE_FMAX ? fmaxf(s.na, s.nc) : m2 * im;
-  }
-  uint32_t w[4];
-  float ee = 0.f;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float x = fmaf(s.fa, a[2 * i], s.fc * c[2 * i]);
-    const float y = fmaf(s.fa, a[2 * i + 1], s.fc * c[2 * i + 1]);
-    w[i] = Elem<DT>::pack(x, y);
-    const float2 r = Elem<DT>::unpack(w[i]);  // the stored value: Eq. 2 divides by its length
-    ee = fmaf(r.x, r.x, ee);
-    ee = fmaf(r.y, r.y, ee);
-  }
-  ee = sum16(ee);
-  const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
-  e_out = make_uint4(w[0], w[1], w[2], w[3]);
-  g_a = s.na * il;
-  g_c = s.nc * il;
-  d_out = s.d;
-}
-
 // Sum of squares of the two 16-bit values of a packed word, accumulated in fp32 by the
 // mixed-precision FMA of sm_100 (no conversion instructions).
 template <int DT>

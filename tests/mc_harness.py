@@ -23,7 +23,7 @@ class Problem:
     def __init__(self, cfg: WorkloadConfig, pair: int = 0, device="cuda", seq_lens=None, gamma=None, t=None,
                  retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
                  tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None,
-                 q4: bool = False, merge_fn: str = "slerp", segments=None):
+                 q4: bool = False, merge_fn: str = "slerp", segments=None, cache_bits: int = 16):
         """segments: list of (sequence, kv head) the oracle will look at; given, the host copies of 4-bit
         layers (exact de-quantised values, fp64) are kept for those segments only (full-size workloads)."""
         import paper_2405_14366_b200 as mc
@@ -52,7 +52,8 @@ class Problem:
         self.max_seq_len = int(self.seq_lens_host.max()) if B else 0
         self.merge_fn = merge_fn
         self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode,
-                               merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn])
+                               merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn], cache_bits=cache_bits)
+        self.cache_bits = cache_bits
         self.pools = {}
         self.q4 = q4
         self.q4_pools: Dict[str, Dict[str, torch.Tensor]] = {}
@@ -155,9 +156,12 @@ class Problem:
         """The compressed pair read back into logical numpy arrays."""
         S = self.S + extra_tokens
         pc = self.pair
-        out = {"e_k": as_bits(self.logical_of(pc.directions("k"), S)), "e_v": as_bits(self.logical_of(pc.directions("v"), S))}
         scale = torch.cat([pc.scales("k"), pc.scales("v")], dim=2)  # [n_pages][H][4][ps]: K l-1, K l, V l-1, V l
         sc = gen.from_paged(scale.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()  # [B][S][H][4]
+        if self.cache_bits == 4:
+            out = self._q4_cache_bits(S, extra_tokens, sc)
+        else:
+            out = {"e_k": as_bits(self.logical_of(pc.directions("k"), S)), "e_v": as_bits(self.logical_of(pc.directions("v"), S))}
         ds = gen.from_paged(pc.dist.permute(0, 1, 3, 2).contiguous(), self.block_table, S).cpu().numpy()   # [B][S][H][2]
         out["scale"], out["dist"] = sc.astype(np.float64), ds.astype(np.float64)
         out["ret_count"] = pc.ret_count.cpu().numpy().reshape(2, self.B, self.H)
@@ -166,6 +170,45 @@ class Problem:
         out["ret_rows"] = np.stack([as_bits(pc.retained_rows(0).cpu()), as_bits(pc.retained_rows(1).cpu())], axis=1)  # [cap][2][128]
         out["ret_tokens"] = np.stack([pc.retained_tokens(0).cpu().numpy(), pc.retained_tokens(1).cpu().numpy()], axis=1)
         out["seg_minmax"] = pc.seg_minmax.cpu().numpy().reshape(2, self.B, self.H, 2).astype(np.float64)
+        return out
+
+    def _q4_cache_bits(self, S: int, extra_tokens: int, sc: np.ndarray) -> Dict[str, np.ndarray]:
+        """The stored directions of a 4-bit shared cache as 16-bit patterns [B][S][H][128]: for the tokens in
+        complete pages code * scale + zero rounded once to the storage type (formed here with the oracle's
+        de-quantiser from the device's codes and group parameters), for the tokens of the last, incomplete
+        page the residual tile's rows; `sc` gets the residual tokens' scales.  Also returns the codes and
+        group parameters per (sequence, head).  With `self.segments` only those (sequence, head) are filled."""
+        pc = self.pair
+        S32 = (S + 31) // 32 * 32
+        npg = S32 // 32
+        segs = self.segments if self.segments is not None else [(b, h) for b in range(self.B) for h in range(self.H)]
+        out = {"q4": {}}
+        for ti, tn in enumerate(("k", "v")):
+            codes_dev = pc.q4_codes(tn)
+            sg, zg = pc.q4_groups(tn)
+            res = pc.residual_directions(tn)  # [B][H][32][128]
+            rsc = pc.residual_scales(tn)      # [B][H][2][32]
+            e = np.zeros((self.B, S, self.H, 128), np.uint16)
+            for (b, h) in segs:
+                n = int(self.seq_lens_host[b]) + extra_tokens
+                nq = n // 32 * 32
+                btl = self.block_table[b, :npg].long().clamp(min=0)
+                codes = codes_dev[btl, h].reshape(S32, 128).cpu().numpy()[:nq]
+                if tn == "k":  # per (page, channel)
+                    scale = orc.decode_bits(as_bits(sg[btl, h].cpu()), self.dtype)[:nq // 32]
+                    zero = orc.decode_bits(as_bits(zg[btl, h].cpu()), self.dtype)[:nq // 32]
+                    axis = 0
+                else:  # per (token, channel group)
+                    scale = orc.decode_bits(as_bits(sg[btl, h].reshape(S32, 4).cpu()), self.dtype)[:nq]
+                    zero = orc.decode_bits(as_bits(zg[btl, h].reshape(S32, 4).cpu()), self.dtype)[:nq]
+                    axis = 1
+                if nq:
+                    e[b, :nq, h] = orc.encode_bits(orc.q4_dequantise(codes, scale, zero, axis), self.dtype)
+                if n > nq:
+                    e[b, nq:n, h] = as_bits(res[b, h, :n - nq].cpu())
+                    sc[b, nq:n, h, 2 * ti:2 * ti + 2] = rsc[b, h, :, :n - nq].cpu().numpy().T
+                out["q4"][(tn, b, h)] = {"codes": codes, "scale": scale, "zero": zero, "n_q": nq}
+            out["e_" + tn] = e
         return out
 
     def retained(self, dc, tensor: int, b: int, h: int):
@@ -187,6 +230,8 @@ class Problem:
                 continue
             out[tn] = orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype,
                                      self.t, self.gamma, mode=mode, do_retention=do_retention, merge_fn=self.merge_fn)
+        if self.cache_bits == 4:  # the merged directions as the 4-bit shared cache stores them
+            out = {tn: orc.q4_cache_pair(out[tn], self.seq_lens_host, tn, self.dtype) for tn in out}
         return out
 
 
@@ -379,6 +424,13 @@ def oracle_attention_from_device(p: Problem, dc, layer: int, q_bits, b: int, hq:
 # bar (same stored cache on both sides, so no flips) is 1e-4 for both types.
 LSE_E2E_BAR = {"f16": 1e-3, "bf16": 8e-3}
 LSE_STAGE_BAR = 1e-4
+# 4-bit shared cache, end to end: a flipped 16-bit element that is the minimum or maximum of its group
+# moves the group's scale or zero by one unit in the last place of the 16-bit type, and with it up to 32
+# stored values of that group by as much as the group's range (about 0.3 for unit directions) times that
+# unit: |q_c| x 0.3 x 2^-11 x scale x sm_scale = 113 x 0.3 x 2^-11 x 4 x 0.088 = 5.8e-3 at worst in binary16,
+# eight times that in bfloat16 (typical: 28 x 0.3 x 2^-8 x 1 x 0.088 = 2.9e-3).  The stage-wise bar (the
+# device's own codes and group parameters on both sides) stays 1e-4.
+LSE_E2E_BAR_Q4 = {"f16": 6e-3, "bf16": 5e-2}
 
 
 def compare_attention(p: Problem, om, layer_sel: int, q: torch.Tensor, out: torch.Tensor, lse, k_new=None, v_new=None,
@@ -413,7 +465,8 @@ def compare_attention(p: Problem, om, layer_sel: int, q: torch.Tensor, out: torc
                 if lse is not None:
                     slerr = max(slerr, abs(float(lse[si, b, hq]) - l2))
     assert err < 1e-2, f"attention output off by {err} (max-abs)"
-    assert lerr < LSE_E2E_BAR[p.dtype], f"log-sum-exp off by {lerr}"
+    bar = LSE_E2E_BAR_Q4 if getattr(p, "cache_bits", 16) == 4 else LSE_E2E_BAR
+    assert lerr < bar[p.dtype], f"log-sum-exp off by {lerr}"
     stats = {"attn_abs": err, "lse_abs": lerr}
     if dc is not None:
         # stage-wise: the probabilities enter the tensor cores rounded to the storage type (relative
@@ -421,4 +474,48 @@ def compare_attention(p: Problem, om, layer_sel: int, q: torch.Tensor, out: torc
         assert serr < (1e-3 if p.dtype == "f16" else 4e-3), f"attention over the device's cache off by {serr}"
         assert slerr < LSE_STAGE_BAR, f"log-sum-exp over the device's cache off by {slerr}"
         stats.update({"attn_stage_abs": serr, "lse_stage_abs": slerr})
+    return stats
+
+
+def compare_q4_cache(p4: Problem, dc4, dc16, om4) -> Dict[str, float]:
+    """The 4-bit shared cache, stage by stage.  `dc16` is the 16-bit cache the same merge kernels wrote for
+    the same inputs (compared with the oracle by compare_merge); the quantiser is deterministic integer
+    work on those bits, so the oracle's quantiser fed with them must give the device's codes, group
+    parameters and stored (de-quantised) directions exactly.  The scales refer to the stored direction:
+    |x| / |e_q|, checked against the 16-bit scale times |e_16| / |e_q| (stage-wise) and against the oracle's
+    own 4-bit cache `om4` on rows whose stored bits agree (end to end)."""
+    stats = {"q4_groups": 0, "q4_scale_stage": 0.0, "q4_scale_e2e": 0.0, "q4_rows_differ": 0}
+    for (tn, b, h), dev in dc4["q4"].items():
+        ti = 0 if tn == "k" else 1
+        n = int(p4.seq_lens_host[b])
+        r = orc.q4_cache_quantise(dc16["e_" + tn][b, :, h], n, tn, p4.dtype)
+        assert r["n_q"] == dev["n_q"]
+        assert np.array_equal(r["codes"], dev["codes"]), f"codes differ {tn} {b} {h}"
+        assert np.array_equal(r["scale"], dev["scale"]) and np.array_equal(r["zero"], dev["zero"]), f"group parameters differ {tn} {b} {h}"
+        assert np.array_equal(r["e_bits"][:n], dc4["e_" + tn][b, :n, h]), f"stored directions differ {tn} {b} {h}"
+        stats["q4_groups"] += r["scale"].size
+        if n == 0:
+            continue
+        e16 = orc.decode_bits(dc16["e_" + tn][b, :n, h], p4.dtype)
+        eq = orc.decode_bits(dc4["e_" + tn][b, :n, h], p4.dtype)
+        l16, lq = np.sqrt(np.sum(e16 * e16, -1)), np.sqrt(np.sum(eq * eq, -1))
+        lq = np.where(lq == 0, 1.0, lq)
+        eo = orc.decode_bits(om4[tn]["e_bits"][b, :n, h], p4.dtype)
+        lo = np.sqrt(np.sum(eo * eo, -1))
+        lo = np.where(lo == 0, 1.0, lo)
+        same = np.all(om4[tn]["e_bits"][b, :n, h] == dc4["e_" + tn][b, :n, h], axis=-1)
+        stats["q4_rows_differ"] += int((~same).sum())
+        for li, nm in enumerate(("n_lm1", "n_l")):
+            g16, g4 = dc16["scale"][b, :n, h, 2 * ti + li], dc4["scale"][b, :n, h, 2 * ti + li]
+            # a retained token keeps its mark (-0), a zero row its zero
+            assert np.array_equal(np.signbit(g16) & (g16 == 0), np.signbit(g4) & (g4 == 0))
+            want = g16 * l16 / lq
+            rel = np.abs(g4 - want) / np.maximum(np.abs(want), 1e-30) * (g16 != 0)
+            stats["q4_scale_stage"] = max(stats["q4_scale_stage"], float(rel.max(initial=0.0)))
+            want2 = om4[tn][nm][b, :n, h] / lo
+            rel2 = np.abs(g4 - want2) / np.maximum(np.abs(want2), 1e-30) * (g4 != 0) * same
+            stats["q4_scale_e2e"] = max(stats["q4_scale_e2e"], float(rel2.max(initial=0.0)))
+    # one fp32 rounding of the product on top of the 16-bit scale's own arithmetic
+    assert stats["q4_scale_stage"] < 2e-7, stats
+    assert stats["q4_scale_e2e"] < 3e-6, stats
     return stats
