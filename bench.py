@@ -26,9 +26,8 @@ import numpy as np
 import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
-for _p in (ROOT, os.path.join(ROOT, "tests")):
-    if _p not in sys.path:
-        sys.path.insert(0, _p)
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
 
 import gen  # noqa: E402
 
@@ -95,9 +94,10 @@ class ClockSampler:
 class Job:
     """All device state of one rank's workload."""
 
-    def __init__(self, wl: gen.WorkloadConfig, device, q4: bool = False):
+    def __init__(self, wl: gen.WorkloadConfig, device, q4: bool = False, q4cache: bool = False):
         import paper_2405_14366_b200 as mc
         self.mc, self.lib, self.wl, self.dev, self.q4 = mc, mc.lib(), wl, device, q4
+        self.q4cache = q4cache  # the shared cache itself is 4-bit (pages of 32 tokens)
         self.B, self.S, self.H, self.Hq, self.ps = wl.batch, wl.seq_len, wl.n_kv_heads, wl.n_q_heads, wl.page_size
         self.steps = wl.decode_steps
         prompt, gen_len = gen.make_lengths(wl)
@@ -112,7 +112,7 @@ class Job:
         self.seq_lens = self.seq0.clone()
         self.gen_dev = torch.from_numpy(np.asarray(self.gen_len, np.int32)).to(device)
         self.step_dev = torch.zeros(1, dtype=torch.int32, device=device)  # decode steps done since the merge
-        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, wl.dtype, t=wl.t, gamma=wl.gamma)
+        self.cfg = mc.McConfig(self.H, self.Hq, self.ps, wl.dtype, t=wl.t, gamma=wl.gamma, cache_bits=4 if q4cache else 16)
         self.max_prefill = int(prompt.max())
         self.tok_heads = int(prompt.sum()) * self.H  # (token, kv head) rows per layer and tensor
         self.pools, self.pairs = [], []
@@ -140,7 +140,8 @@ class Job:
             self.new.append({k: v[:, 0].contiguous() for k, v in nt.items()})
         self.out = torch.empty(1, self.B, self.Hq, 128, dtype=dt, device=device)
         bm, bd = self.batch(False), self.batch(True)
-        self.ws_merge = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bm, 0, 1), dtype=torch.uint8, device=device)
+        n_ws = wl.n_pairs if not (q4 or q4cache) else 1  # mc_merge_pairs: one scratch area per pair
+        self.ws_merge = torch.empty(n_ws * self.lib.mc_workspace_bytes(self.cfg, bm, 0, 1), dtype=torch.uint8, device=device)
         self.ws_attn = torch.empty(self.lib.mc_workspace_bytes(self.cfg, bd, 1, 1), dtype=torch.uint8, device=device)
         self.sm_scale = 1.0 / math.sqrt(128.0)
         self.launches = 0
@@ -176,6 +177,11 @@ class Job:
         self.seq_lens.copy_(self.seq0)
         self.step_dev.zero_()
         b = self.batch(False)
+        if not self.q4 and not self.q4cache:
+            # Algorithm 1's loop over the merged layers as one call: the pairs share four launches per group of 8
+            self.lib.mc_merge_pairs(self.cfg, b, self.pools, self.pairs, True, self.ws_merge)
+            self.launches += 4 * ((self.wl.n_pairs + 7) // 8)  # init, merge, count(+scan), compact
+            return
         for pr in range(self.wl.n_pairs):
             pl = self.pools[pr]
             if self.q4:
@@ -183,7 +189,7 @@ class Job:
                 continue
             self.lib.mc_merge_pair(self.cfg, b, pl["k_lm1"], pl["v_lm1"], pl["k_l"], pl["v_l"], self.pairs[pr], True,
                                    self.ws_merge)
-        self.launches += 4 * self.wl.n_pairs  # init, merge, count(+scan), compact
+        self.launches += (5 if self.q4cache else 4) * self.wl.n_pairs  # init, merge, count(+scan), compact (, quantise)
 
     def restore_all(self):
         b = self.batch(False)
@@ -262,6 +268,18 @@ class Job:
         live = self.gen_len > s
         return int((self.prompt[live].astype(np.int64) + s).sum()) * self.H
 
+    def live_residual_heads(self, s: int) -> int:
+        """4-bit cache: the rows of step s that still sit in 16 bits (the last, incomplete page of each live sequence)."""
+        live = self.gen_len > s
+        return int(((self.prompt[live].astype(np.int64) + s) % 32).sum()) * self.H
+
+    def attn_row_bytes(self, th: int, th_res: int, rho: float) -> float:
+        """Algorithmic bytes of one layer's attention over th (token, head) rows, th_res of them residual."""
+        if not self.q4cache:
+            return th * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+        q4row = 64 + 16  # codes + the row's share of the group parameters
+        return (th - th_res) * (2 * q4row + 8) + th_res * (2 * ROW + 8) + th * 2 * rho * (ROW + 4)
+
     def step(self, sample_events=False):
         self.merge_all()
         self.restore_all()
@@ -275,16 +293,17 @@ class Job:
     def bytes_per_step(self, rho: float):
         th, npairs, steps = self.tok_heads, self.wl.n_pairs, self.steps
         in_row = 64 + 16 if self.q4 else ROW  # 4-bit codes + the row's share of the group meta
-        merge = npairs * 2 * th * (2 * in_row + ROW + 12 + 4 + rho * (2 * in_row + 2 * ROW + 4))
-        restore = npairs * 2 * 2 * th * (2 * ROW + 4 + rho * 2 * ROW)
+        e_row = 64 + 16 if self.q4cache else ROW  # what a direction row occupies in the shared cache
+        merge = npairs * 2 * th * (2 * in_row + e_row + 12 + 4 + rho * (2 * in_row + 2 * ROW + 4))
+        restore = npairs * 2 * 2 * th * (e_row + ROW + 4 + rho * 2 * ROW)
         # decode: every live sequence grows by one token per step
-        th_steps = sum(self.live_token_heads(s) for s in range(steps))
-        attn = npairs * 2 * th_steps * (2 * ROW + 8 + 2 * rho * (ROW + 4))
-        append = npairs * 2 * int(np.minimum(self.gen_len, steps).sum()) * self.H * (3 * ROW + 12)
+        attn = npairs * 2 * sum(self.attn_row_bytes(self.live_token_heads(s), self.live_residual_heads(s), rho) for s in range(steps))
+        # 4-bit cache: a row is read once more (16 bits) and written in 4 bits when its page completes
+        append = npairs * 2 * int(np.minimum(self.gen_len, steps).sum()) * self.H * (3 * ROW + 12 + ((ROW + 80) if self.q4cache else 0))
         return {"merge": merge, "restore": restore, "attn": attn, "append": append}
 
     def attn_bytes_at(self, s: int, rho: float):
-        return self.live_token_heads(s) * (2 * ROW + 8 + 2 * rho * (ROW + 4))
+        return self.attn_row_bytes(self.live_token_heads(s), self.live_residual_heads(s), rho)
 
 
 def max_over_ranks(seconds: float, dist, device) -> float:
@@ -380,6 +399,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--q4", action="store_true", help="the layers arrive in 4 bits (page size 32; no host-buffer leg)")
+    ap.add_argument("--q4cache", action="store_true", help="the shared cache is 4-bit (page size 32): restore and attention read codes")
     args = ap.parse_args()
     wl = gen.CONFIGS[args.workload]
     if args.decode_steps is not None:
@@ -407,7 +427,7 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    job = Job(wl, dev, q4=args.q4)
+    job = Job(wl, dev, q4=args.q4, q4cache=args.q4cache)
     if args.q4:
         args.no_e2e = True  # the host-buffer entry points take 16-bit layers only
     warm = max(3, args.warmup)
@@ -442,10 +462,10 @@ def main():
     attn_ms = float(np.mean([m for m, _ in ev_ms]))
     peak, peak_src = measured_hbm_peak()
     achieved = attn_bytes / (attn_ms * 1e-3) / 1e9
-    roofline = {"kernel": "attn_split_kernel (+attn_combine_kernel)", "bound": "hbm", "achieved": achieved,
+    roofline = {"kernel": ("attn_split_kernel<4-bit tiles>" if args.q4cache else "attn_split_kernel") + " (+attn_combine_kernel)", "bound": "hbm", "achieved": achieved,
                 "peak": peak, "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0,
                 "peak_source": peak_src,
-                "traffic": (float(attn_bytes) * ATTN_TRAFFIC_RATIO if ATTN_TRAFFIC_RATIO and wl.name.startswith("c2") else None), "launch_ms": attn_ms, "launches_timed": 2 * len(ev_ms),
+                "traffic": (float(attn_bytes) * ATTN_TRAFFIC_RATIO if ATTN_TRAFFIC_RATIO and wl.name.startswith("c2") and not args.q4cache else None), "launch_ms": attn_ms, "launches_timed": 2 * len(ev_ms),
                 "algorithmic_bytes_per_launch": float(attn_bytes)}
 
     # ---- per-phase breakdown (outside the headline region) ----------------------------------------
@@ -480,13 +500,18 @@ def main():
         job.merge_all()
         t_p = timed(lambda: job.decode_pair_all(psteps))
         th_steps = sum(job.live_token_heads(s) for s in range(psteps))
-        pair_bytes = wl.n_pairs * th_steps * (2 * ROW + 16 + 4 * rho * (ROW + 4)) + by["append"] * psteps / job.steps
+        if args.q4cache:
+            pair_bytes = wl.n_pairs * sum(job.attn_row_bytes(job.live_token_heads(s), job.live_residual_heads(s), 2 * rho) + 8 * job.live_token_heads(s)
+                                          for s in range(psteps)) + by["append"] * psteps / job.steps
+        else:
+            pair_bytes = wl.n_pairs * th_steps * (2 * ROW + 16 + 4 * rho * (ROW + 4)) + by["append"] * psteps / job.steps
         phases["decode_pair_mode"] = {"ms_per_decode_step": t_p * 1e3 / psteps, "GB/s": pair_bytes / t_p / 1e9,
                                       "kv_tokens_per_s": (th_steps / job.H)
                                       * 2 * wl.n_pairs / t_p, "steps": psteps}
     peak0, _ = measured_hbm_peak()
     for ph in phases.values():
         ph["frac_of_measured_hbm"] = ph["GB/s"] / peak0
+        ph["frac_of_nominal_8000"] = ph["GB/s"] / 8000.0
 
     # ---- end to end: host buffers, copies inside the timed region ----------------------------------
     e2e = None
@@ -512,7 +537,7 @@ def main():
                 "steps": args.steps, "warmup": warm, "ms_per_step": t_total / args.steps * 1e3,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": wl.name, "batch": wl.batch, "seq_len": wl.seq_len, "kv_heads": wl.n_kv_heads,
-                           "q_heads": wl.n_q_heads, "storage": wl.dtype, "input_layers": "4-bit, de-quantised in the merge" if args.q4 else wl.dtype, "page_size": wl.page_size,
+                           "q_heads": wl.n_q_heads, "storage": wl.dtype, "shared_cache": "4-bit (groups of 32) + 16-bit residual page" if args.q4cache else wl.dtype, "input_layers": "4-bit, de-quantised in the merge" if args.q4 else wl.dtype, "page_size": wl.page_size,
                            "pairs": wl.n_pairs, "decode_steps": wl.decode_steps, "t": wl.t, "gamma": wl.gamma,
                            "retained_fraction": rho, "attention_mode": "single-layer calls (2 per pair per step)",
                            "l2": "inputs larger than L2: every launch streams >= 0.5 GB"},

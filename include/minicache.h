@@ -92,7 +92,8 @@ typedef enum mc_merge_fn { MC_MERGE_SLERP = 0, MC_MERGE_FMAX = 1, MC_MERGE_MEAN 
 /* Status word indices (mc_read_status). */
 enum {
   MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out;
-                                   bit 2: a length or page id outside the declared bounds was met */
+                                   bit 2: a length or page id outside the declared bounds was met;
+                                   bit 3: a range check of the range-checked build failed */
   MC_STATUS_RETAINED_TOTAL = 1, /* retained entries the last merge selected (K and V segments together) */
   MC_STATUS_NEAR_THRESHOLD = 2, /* tokens of the last merge whose distance lies within 1e-6 of their segment's
                                    retention threshold (a differently rounded d could have decided them the
@@ -107,6 +108,11 @@ enum {
  * length is clamped, the page's rows are not written (merge, restore, append) or page 0 is read in
  * its place (decode attention: the result of that sequence is then meaningless). */
 #define MC_FLAG_BAD_METADATA 4
+/* Range-checked build only (mc_build_flags() & MC_BUILD_BOUNDS): an index the library derived from the
+ * pair cache's own contents -- a retained entry's token index, a retained range against the pool's
+ * capacity, a compaction slot -- fell outside its bounds.  The access is skipped, the kernel carries
+ * on, results that depended on it are meaningless. */
+#define MC_FLAG_BOUNDS 8
 
 /* Method parameters and tensor geometry (Sec. 4.1-4.2, Sec. 5 defaults t = 0.6, gamma = 0.05). */
 typedef struct mc_config {
@@ -275,6 +281,13 @@ mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pai
 /* Library version (major * 10000 + minor * 100 + patch). No device work. */
 int32_t mc_version(void);
 
+/* How the library was built (the paper has no counterpart).  MC_BUILD_BOUNDS: compiled with -DMC_BOUNDS=1,
+ * the debugging build in which the kernels also range-check every index they derive from the pair cache's
+ * contents (see MC_FLAG_BOUNDS); it stands in for a memory checker where none can be run.  Checks of the
+ * caller's batch description (MC_FLAG_BAD_METADATA) are part of every build. */
+#define MC_BUILD_BOUNDS 1
+int32_t mc_build_flags(void);
+
 /* Human-readable name of a status code (static string). */
 const char* mc_status_str(int32_t status);
 
@@ -282,7 +295,9 @@ const char* mc_status_str(int32_t status);
 const char* mc_last_cuda_error(void);
 
 /* Scratch bytes `op` needs for this geometry (a multiple of 256).  Pure host arithmetic.
- * `n_query_sets` is 2 for MC_LAYER_BOTH decode attention, else 1 (ignored for MC_OP_MERGE). */
+ * `n_query_sets` is 2 for MC_LAYER_BOTH decode attention, else 1 (ignored for MC_OP_MERGE).
+ * With cfg->cache_bits = 4 the merge scratch also holds the 16-bit direction tiles of both tensors
+ * before they are quantised (2 * n_pages * n_kv_heads * 8448 bytes: batch->n_pages must be set). */
 mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_t op,
                              int32_t n_query_sets, size_t* bytes);
 
@@ -295,10 +310,28 @@ mc_status mc_workspace_bytes(const mc_config* cfg, const mc_batch* batch, int32_
  * If the selection needs more than ret_capacity entries the overflow flag is set, no retained
  * entry is written and every ret_count is 0 (the merged directions are still valid).
  * workspace: at least mc_workspace_bytes(MC_OP_MERGE) bytes, 256-byte aligned, contents
- * irrelevant on entry, must stay untouched until the call has run on the stream. */
+ * irrelevant on entry, must stay untouched until the call has run on the stream.
+ * cfg->cache_bits = 4: the merged directions are formed and rounded to cfg->dtype exactly as for the
+ * 16-bit cache (in the workspace), retention marks its tokens, then every complete page is quantised
+ * into out->e_k / e_v and each sequence's last, incomplete page is copied to out->res_k / res_v. */
 mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1,
                         const mc_layer_kv* l, const mc_pair_cache* out, int32_t do_retention,
                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 1's prefill loop over the merged half of the model ("for l = S .. L-1: if l is odd, merge
+ * layers l and l-1"): mc_merge_pair for n_pairs layer pairs of one batch at once.  lm1[i], l[i], out[i]
+ * are pair i's layers and pair cache (host arrays of pointers, read before the call returns; every pair
+ * needs its own pair cache).  The pairs are independent, so their rows are streamed by one persistent grid
+ * and their segments go through one retention pass: four launches for up to 8 pairs instead of four per
+ * pair.  Results are bit-identical to n_pairs calls of mc_merge_pair.
+ * workspace: n_pairs * mc_workspace_bytes(MC_OP_MERGE) bytes, 256-byte aligned.
+ * A length outside its declared bound or a wait that ran out is recorded in the status words of the first
+ * pair of its group of 8; everything else in the pair's own.  cfg->cache_bits = 4 is not supported here
+ * (MC_ERR_UNSUPPORTED): merge such pairs one by one. */
+mc_status mc_merge_pairs(const mc_config* cfg, const mc_batch* batch, int32_t n_pairs,
+                         const mc_layer_kv* const* lm1, const mc_layer_kv* const* l,
+                         const mc_pair_cache* const* out, int32_t do_retention, void* workspace,
+                         size_t workspace_bytes, void* stream);
 
 /* mc_merge_pair for layers stored in 4 bits: the rows are de-quantised inside the merge kernel
  * (code * scale + zero in fp32) and merged exactly as in mc_merge_pair; the pair cache it writes is
@@ -312,7 +345,9 @@ mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc
  * merges k/v_new_lm1 with k/v_new_l ([batch][n_kv_heads][128], 16-bit) by Eq. 3 and writes
  * direction, scales and distance at token position seq_lens[b] of every sequence (the block
  * table must already hold a page for it).  No retention decision is taken for new tokens.
- * seq_lens is not modified: the caller advances it once all layers of the step are done. */
+ * seq_lens is not modified: the caller advances it once all layers of the step are done.
+ * cfg->cache_bits = 4: the row goes to slot seq_lens[b] % 32 of the sequence's residual tile; when
+ * that fills the page (slot 31) the same kernel quantises the 32 rows into the page's 4-bit tile. */
 mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
                          const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l,
                          const void* v_new_l, void* stream);
@@ -322,7 +357,9 @@ mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_p
  * x_hat = e * scale, then retained rows overwritten with their raw copies.
  * dst_fp32 == 0: dst pools hold cfg->dtype (the product is rounded once to it).
  * dst_fp32 != 0: dst pools are [n_pages][n_kv_heads][page_size][128] binary32: the product as
- *                computed, raw rows converted exactly. */
+ *                computed, raw rows converted exactly.
+ * cfg->cache_bits = 4: e is the stored direction of the 4-bit cache (code * scale + zero rounded once
+ * to cfg->dtype) for tokens in complete pages and the residual tile's row for the others. */
 mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
                      int32_t layer_sel, const mc_layer_kv* dst, int32_t dst_fp32, void* stream);
 
@@ -338,7 +375,10 @@ mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_
  * out         [n_sets][batch][n_q_heads][128] 16-bit
  * lse         [n_sets][batch][n_q_heads] fp32 natural-log sum of exponentials, or NULL
  * workspace   at least mc_workspace_bytes(MC_OP_DECODE_ATTN, n_sets) bytes, 256-byte aligned.
- * A sequence with seq_lens[b] == 0 and no new token yields zeros (lse = -inf). */
+ * A sequence with seq_lens[b] == 0 and no new token yields zeros (lse = -inf).
+ * cfg->cache_bits = 4: the 4-bit tiles are streamed as they are and de-quantised in registers (one
+ * packed 16-bit FMA per element pair gives the stored direction exactly); the residual tile of a
+ * sequence's last page is attended in 16 bits.  Same arguments, same workspace size. */
 mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
                          int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
                          float sm_scale, void* out, float* lse, void* workspace,

@@ -18,9 +18,11 @@ MC_LAYER_LM1, MC_LAYER_L, MC_LAYER_BOTH = 0, 1, 2
 MC_OP_MERGE, MC_OP_DECODE_ATTN = 0, 1
 MC_STATUS_WORDS = 4
 MC_STATUS_FLAGS, MC_STATUS_RETAINED_TOTAL, MC_STATUS_NEAR_THRESHOLD = 0, 1, 2
-MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT, MC_FLAG_BAD_METADATA = 1, 2, 4
+MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT, MC_FLAG_BAD_METADATA, MC_FLAG_BOUNDS = 1, 2, 4, 8
+MC_BUILD_BOUNDS = 1
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libminicache.so")
+# MINICACHE_LIBRARY selects another build of the same library (the range-checked one, for instance)
+_LIB_PATH = os.environ.get("MINICACHE_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libminicache.so")
 
 
 class McError(RuntimeError):
@@ -72,7 +74,7 @@ class _Stats(C.Structure):
                 ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
 
 
-EXPORTS = ("mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+EXPORTS = ("mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -276,6 +278,7 @@ class MiniCacheLib:
         self._lib = C.CDLL(path)
         L = self._lib
         L.mc_version.restype = C.c_int32
+        L.mc_build_flags.restype = C.c_int32
         L.mc_status_str.restype = C.c_char_p
         L.mc_status_str.argtypes = [C.c_int32]
         L.mc_last_cuda_error.restype = C.c_char_p
@@ -283,6 +286,9 @@ class MiniCacheLib:
         L.mc_workspace_bytes.argtypes = [P(_Config), P(_Batch), C.c_int32, C.c_int32, P(C.c_size_t)]
         L.mc_merge_pair.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_PairCache), C.c_int32, V,
                                     C.c_size_t, V]
+        L.mc_merge_pairs.argtypes = [P(_Config), P(_Batch), C.c_int32, P(P(_LayerKV)), P(P(_LayerKV)), P(P(_PairCache)),
+                                     C.c_int32, V, C.c_size_t, V]
+        L.mc_merge_pairs.restype = C.c_int32
         L.mc_append_pair.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, V, V, V, V]
         L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), C.c_int32, V]
         L.mc_pair_bytes.argtypes = [P(_Config), P(_Batch), C.c_int64, P(_PairSizes)]
@@ -322,6 +328,9 @@ class MiniCacheLib:
     def mc_version(self) -> int:
         return self._lib.mc_version()
 
+    def mc_build_flags(self) -> int:
+        return self._lib.mc_build_flags()
+
     def mc_status_str(self, code: int) -> str:
         return self._lib.mc_status_str(code).decode()
 
@@ -338,6 +347,20 @@ class MiniCacheLib:
         self._check(self._lib.mc_merge_pair(C.byref(c), C.byref(b), C.byref(a), C.byref(l), C.byref(pc),
                                             1 if do_retention else 0, _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_merge_pairs(self, cfg: McConfig, batch: Batch, layers, pairs, do_retention: bool, workspace: torch.Tensor,
+                       stream=None):
+        """layers: per pair a dict with k_lm1, v_lm1, k_l, v_l pools; pairs: the PairCache of each.
+        workspace: len(pairs) * mc_workspace_bytes(MC_OP_MERGE) bytes."""
+        n = len(pairs)
+        c, b = cfg.c(), batch.c()
+        a = [_LayerKV(_ptr(x["k_lm1"]), _ptr(x["v_lm1"])) for x in layers]
+        l = [_LayerKV(_ptr(x["k_l"]), _ptr(x["v_l"])) for x in layers]
+        pcs = [pc.c() for pc in pairs]
+        arr = lambda items, T: (C.POINTER(T) * n)(*[C.pointer(x) for x in items])
+        self._check(self._lib.mc_merge_pairs(C.byref(c), C.byref(b), n, arr(a, _LayerKV), arr(l, _LayerKV),
+                                             arr(pcs, _PairCache), 1 if do_retention else 0, _ptr(workspace),
+                                             workspace.numel() * workspace.element_size(), _stream(stream)))
 
     def mc_merge_pair_q4(self, cfg: McConfig, batch: Batch, q_lm1, q_l, pair: PairCache, do_retention: bool,
                          workspace: torch.Tensor, stream=None):

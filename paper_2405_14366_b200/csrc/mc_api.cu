@@ -5,6 +5,8 @@
 #include <atomic>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "mc_common.cuh"
 #include "mc_items.cuh"
 #include "mc_kernels.h"
@@ -32,6 +34,13 @@ mc_status sm_count(int* n_sm) {
   *n_sm = v;
   return MC_OK;
 }
+
+// A named range around every compute entry point: visible on a profiler's timeline, a no-op (one
+// indirect call) when no tool is attached.
+struct ApiRange {
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
+};
 
 static bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
@@ -118,7 +127,15 @@ using namespace mc;
 
 extern "C" {
 
-int32_t mc_version(void) { return 200; }
+int32_t mc_version(void) { return 210; }
+
+int32_t mc_build_flags(void) {
+#if defined(MC_BOUNDS) && MC_BOUNDS
+  return MC_BUILD_BOUNDS;
+#else
+  return 0;
+#endif
+}
 
 const char* mc_status_str(int32_t s) {
   switch (s) {
@@ -197,6 +214,7 @@ mc_status mc_pair_bytes(const mc_config* cfg, const mc_batch* batch, int64_t ret
 
 mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, void* stream,
                        mc_stats* out) {
+  ApiRange range_("mc_get_stats");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -250,6 +268,7 @@ mc_status mc_get_stats(const mc_config* cfg, const mc_batch* batch, const mc_pai
 mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* lm1, const mc_layer_kv* l,
                         const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
                         void* stream) {
+  ApiRange range_("mc_merge_pair");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -262,9 +281,43 @@ mc_status mc_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_la
   return run_merge(cfg, batch, lm1, l, nullptr, nullptr, out, do_retention ? 1 : 0, workspace, (cudaStream_t)stream);
 }
 
+mc_status mc_merge_pairs(const mc_config* cfg, const mc_batch* batch, int32_t n_pairs, const mc_layer_kv* const* lm1,
+                         const mc_layer_kv* const* l, const mc_pair_cache* const* out, int32_t do_retention, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_merge_pairs");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  if (n_pairs < 0 || !lm1 || !l || !out) return MC_ERR_INVALID_ARG;
+  if (cfg->cache_bits == 4) return MC_ERR_UNSUPPORTED;  // the 4-bit cache is merged pair by pair (mc_merge_pair)
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  const size_t ws_pair = merge_workspace_bytes(cfg, batch);
+  if (workspace_bytes < (size_t)n_pairs * ws_pair) return MC_ERR_CAPACITY;
+  // every pair is checked before anything is launched
+  for (int i = 0; i < n_pairs; ++i) {
+    if (!lm1[i] || !l[i] || !lm1[i]->k_pool || !lm1[i]->v_pool || !l[i]->k_pool || !l[i]->v_pool) return MC_ERR_INVALID_ARG;
+    if (!aligned256(lm1[i]->k_pool) || !aligned256(lm1[i]->v_pool) || !aligned256(l[i]->k_pool) || !aligned256(l[i]->v_pool))
+      return MC_ERR_ALIGN;
+    st = check_merge_common(cfg, batch, out[i], workspace, ws_pair);
+    if (st != MC_OK) return st;
+    for (int j = 0; j < i; ++j)
+      if (out[j] == out[i] || out[j]->status == out[i]->status) return MC_ERR_INVALID_ARG;  // one pair cache per pair
+  }
+  const Geom g = make_geom(cfg, batch);
+  for (int i0 = 0; i0 < n_pairs; i0 += kMergePairsPerLaunch) {
+    const int n = n_pairs - i0 < kMergePairsPerLaunch ? n_pairs - i0 : kMergePairsPerLaunch;
+    st = launch_merge_pairs(cfg, batch, g, n, lm1 + i0, l + i0, nullptr, nullptr, out + i0, do_retention ? 1 : 0,
+                            (char*)workspace + (size_t)i0 * ws_pair, (cudaStream_t)stream);
+    if (st != MC_OK) return st;
+  }
+  return MC_OK;
+}
+
 mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc_layer_q4* lm1, const mc_layer_q4* l,
                            const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
                            void* stream) {
+  ApiRange range_("mc_merge_pair_q4");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   if (cfg->page_size != 32) return MC_ERR_SHAPE;
@@ -283,6 +336,7 @@ mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc
 
 mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, const void* k_new_lm1,
                          const void* v_new_lm1, const void* k_new_l, const void* v_new_l, void* stream) {
+  ApiRange range_("mc_append_pair");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -300,6 +354,7 @@ mc_status mc_append_pair(const mc_config* cfg, const mc_batch* batch, const mc_p
 
 mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
                      const mc_layer_kv* dst, int32_t dst_fp32, void* stream) {
+  ApiRange range_("mc_restore");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -318,6 +373,7 @@ mc_status mc_restore(const mc_config* cfg, const mc_batch* batch, const mc_pair_
 mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
                          const void* q, const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
                          void* workspace, size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_decode_attn");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -340,6 +396,7 @@ mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const 
                              const mc_layer_kv* host_l, const mc_layer_kv* dev_lm1, const mc_layer_kv* dev_l,
                              const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
                              void* stream) {
+  ApiRange range_("mc_merge_pair_host");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);
@@ -398,6 +455,7 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
                               int32_t layer_sel, const void* q_host, const void* k_new_host, const void* v_new_host,
                               float sm_scale, void* out_host, float* lse_host, void* dev_io, size_t dev_io_bytes,
                               void* workspace, size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_decode_attn_host");
   mc_status st = check_config(cfg);
   if (st != MC_OK) return st;
   st = check_batch(cfg, batch);

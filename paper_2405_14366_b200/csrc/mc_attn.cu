@@ -394,6 +394,8 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             const Ranges rg = ranges_of(raw);
             n_r = ph ? rg.n_v : rg.n_k;
             r_lo = ph ? rg.v_lo : rg.k_lo;
+            // (range-checked build: a retained range that does not fit the pool or the chunk is not followed)
+            if (!MC_IN_BOUNDS(n_r >= 0 && r_lo >= 0 && n_r <= w.n_tok && (int64_t)r_lo + n_r <= p.ret_capacity, p.status)) n_r = 0;
             X = (n_r + n_new + cap_e - 1) / cap_e;
           }
           if (X >= 0 && t >= w.TT + X) break;
@@ -696,8 +698,10 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               if (e < cnt) {
                 const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
                 const float sc = acc0[k] * p.scale_log2;
-                S[row * s_stride + col] = sc;
-                mxe = fmaxf(mxe, sc);
+                if (MC_IN_BOUNDS(col >= 0 && col <= w.n_tok, p.status)) {  // (the step's new token sits at column n_tok)
+                  S[row * s_stride + col] = sc;
+                  mxe = fmaxf(mxe, sc);
+                }
               }
             }
           }
@@ -902,8 +906,10 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               pv[k] = 0.f;
               if (e < cnt) {
                 const int col = *reinterpret_cast<const int*>(sb + e * kEntryBytes + kRowBytes) - w.split_start;
-                pv[k] = exp2f(S[row * s_stride + col] - m_row);
-                if (col >= w.n_tok) l_acc += pv[k];  // the new token: no tile has counted it
+                if (MC_IN_BOUNDS(col >= 0 && col <= w.n_tok, p.status)) {
+                  pv[k] = exp2f(S[row * s_stride + col] - m_row);
+                  if (col >= w.n_tok) l_acc += pv[k];  // the new token: no tile has counted it
+                }
               }
             }
             b0 = Elem<DT>::pack(pv[0], pv[1]);

@@ -89,6 +89,15 @@ __device__ __forceinline__ int checked_page(const Geom& g, int b, int slot, int3
 }
 #endif
 
+// Range-checked build (-DMC_BOUNDS=1): indices derived from the pair cache's own contents are checked
+// where they are used; a failed check records MC_FLAG_BOUNDS and the access is skipped.  In the normal
+// build the check is the constant `true`.
+#if defined(MC_BOUNDS) && MC_BOUNDS
+#define MC_IN_BOUNDS(cond, status) ((cond) ? true : (atomicOr((status), MC_FLAG_BOUNDS), false))
+#else
+#define MC_IN_BOUNDS(cond, status) true
+#endif
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Compressed tile of one (page, kv head, tensor) in the pair cache: page_size direction rows of

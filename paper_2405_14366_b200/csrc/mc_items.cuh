@@ -47,11 +47,12 @@ __device__ __forceinline__ void page_prefix(const Geom& g, int* len_s, int* pre_
 // counts (pre[batch] = P, all of them), an item index is ((tensor * P) + pg) * items_per_page + grp
 // -- row group fastest, then page, sequence, tensor.  A CTA walks its items with a fixed stride, so
 // the decomposition is kept incrementally (no divisions per item) and the sequence is found by
-// stepping forward in `pre`.  tensor == 2 marks the end.
-__device__ __forceinline__ void page_item_init(PageItem& m, long long i, int ipp, int P, const int* pre) {
+// stepping forward in `pre`.  `tensor` runs over n_slots tensors (K and V of one pair, or of several
+// pairs one after the other: slot = 2 * pair + tensor); tensor == n_slots marks the end.
+__device__ __forceinline__ void page_item_init(PageItem& m, long long i, int ipp, int P, const int* pre, int n_slots = 2) {
   const long long per_tensor = (long long)P * ipp;
-  if (P == 0 || i >= 2 * per_tensor) {
-    m.tensor = 2;
+  if (P == 0 || i >= n_slots * per_tensor) {
+    m.tensor = n_slots;
     m.b = m.pslot = m.grp = m.pg = 0;
     return;
   }
@@ -63,8 +64,9 @@ __device__ __forceinline__ void page_item_init(PageItem& m, long long i, int ipp
   while (m.pg >= pre[m.b + 1]) ++m.b;
   m.pslot = m.pg - pre[m.b];
 }
-__device__ __forceinline__ void page_item_advance(PageItem& m, int s_pg, int s_grp, int ipp, int P, const int* pre) {
-  if (m.tensor >= 2) return;
+__device__ __forceinline__ void page_item_advance(PageItem& m, int s_pg, int s_grp, int ipp, int P, const int* pre,
+                                                  int n_slots = 2) {
+  if (m.tensor >= n_slots) return;
   m.grp += s_grp;
   const int carry = m.grp >= ipp ? 1 : 0;
   m.grp -= carry * ipp;
@@ -72,7 +74,7 @@ __device__ __forceinline__ void page_item_advance(PageItem& m, int s_pg, int s_g
   while (m.pg >= P) {
     m.pg -= P;
     m.b = 0;
-    if (++m.tensor >= 2) return;
+    if (++m.tensor >= n_slots) return;
   }
   while (m.pg >= pre[m.b + 1]) ++m.b;
   m.pslot = m.pg - pre[m.b];

@@ -23,8 +23,9 @@ constexpr int kQ4RowBytes = 64;                              // 128 four-bit cod
 constexpr int kQ4CodesBytes = kRowsPerItem * kQ4RowBytes;    // one layer's codes of an item
 constexpr int kQ4MetaBytes = kRowsPerItem * 16;              // one layer's (scale, zero) pairs of an item
 
-struct MergeParams {
-  Geom g;
+constexpr int kMaxMergePairs = 8;  // layer pairs one launch sequence can merge (they share the batch geometry)
+
+struct MergePair {
   const char* a_pool[2];  // layer l-1: K, V
   const char* c_pool[2];  // layer l:   K, V
   const char* a_meta[2];  // 4-bit layers: (scale, zero) pairs; a_pool / c_pool then hold the codes
@@ -32,10 +33,16 @@ struct MergeParams {
   char* e_pool[2];  // compressed tiles (see tile_bytes)
   float* dist;
   unsigned* seg_minmax;  // [seg][2] float bits (d >= 0, so unsigned order = float order)
+  int32_t* status;
+};
+
+struct MergeParams {
+  Geom g;
+  MergePair pr[kMaxMergePairs];
+  int n_pairs;
   float ta, tc;
   int merge_fn;
   int items_per_page;
-  int32_t* status;
 };
 
 // Sum of squares of the two 16-bit values of a packed word, accumulated in fp32 by the
@@ -185,7 +192,7 @@ __device__ __forceinline__ void dequant32(const uint4& codes, const uint32_t* me
 }
 
 template <int DT, bool Q4IN>
-__global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(const __grid_constant__ MergeParams p) {
   grid_dep_wait();
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];
@@ -210,20 +217,26 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  page_prefix(p.g, len_s, pre_s, kMergeThreads, p.status);
+  // (what concerns the batch as a whole -- a length outside its bound, a wait that ran out -- is
+  // recorded in the first pair's status words)
+  int32_t* const status0 = p.pr[0].status;
+  const int n_slots = 2 * p.n_pairs;  // item order: pair, tensor, page, row group
+  page_prefix(p.g, len_s, pre_s, kMergeThreads, status0);
   const int* lens = len_s;
-  const int P = pre_s[p.g.batch];
+  const int P_all = pre_s[p.g.batch];
   const int ipp = p.items_per_page;
   const int stride = gridDim.x;
   const int s_pg = stride / ipp, s_grp = stride - s_pg * ipp;
 
   // a page id outside the pools comes back as -1: its item streams page 0 instead (any valid
   // memory) and writes nothing
-  auto page_of = [&](const PageItem& m) { return m.tensor < 2 ? checked_page(p.g, m.b, m.pslot, p.status) : 0; };
+  auto page_of = [&](const PageItem& m) { return m.tensor < n_slots ? checked_page(p.g, m.b, m.pslot, p.pr[m.tensor >> 1].status) : 0; };
   // lane 0 of warp 0: copy item j (the j-th item of this CTA) into stage j % kMergeStages
   auto issue = [&](int j, const PageItem& m, int page_id) -> bool {
     const int s = j % kMergeStages;
-    if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, p.status)) return false;
+    if (j >= kMergeStages && !mbar_wait(empty0 + 8 * s, ((j / kMergeStages) - 1) & 1, s_abort, status0)) return false;
+    const MergePair& P = p.pr[m.tensor >> 1];
+    const int ts = m.tensor & 1;
     const int rows_item = min(kRowsPerItem, rows_in_page - m.grp * kRowsPerItem);
     const uint32_t bar = full0 + 8 * s;
     page_s[s] = page_id;
@@ -232,63 +245,65 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     if (!Q4IN) {
       const uint32_t bytes = (uint32_t)rows_item * kRowBytes;
       mbar_expect_tx(bar, 2 * bytes);
-      bulk_load(stage0 + s * kMergeStageBytes, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + row0 * kRowBytes, bytes, bar);
-      bulk_load(stage0 + s * kMergeStageBytes + kRowsPerItem * kRowBytes,
-                (m.tensor ? p.c_pool[1] : p.c_pool[0]) + row0 * kRowBytes, bytes, bar);
+      bulk_load(stage0 + s * kMergeStageBytes, P.a_pool[ts] + row0 * kRowBytes, bytes, bar);
+      bulk_load(stage0 + s * kMergeStageBytes + kRowsPerItem * kRowBytes, P.c_pool[ts] + row0 * kRowBytes, bytes, bar);
     } else {
       // 4-bit layers: 64 bytes of codes per row; (scale, zero) pairs per channel and head (keys, a
       // group = the page's 32 tokens) or per token and 32 channels (values)
       const uint32_t cbytes = (uint32_t)rows_item * kQ4RowBytes;
-      const uint32_t mbytes = m.tensor ? (uint32_t)rows_item * 16u : (uint32_t)(rows_item / 32) * 512u;
-      const size_t moff = m.tensor ? row0 * 16 : (row0 / 32) * 512;
+      const uint32_t mbytes = ts ? (uint32_t)rows_item * 16u : (uint32_t)(rows_item / 32) * 512u;
+      const size_t moff = ts ? row0 * 16 : (row0 / 32) * 512;
       mbar_expect_tx(bar, 2 * (cbytes + mbytes));
       const uint32_t sb = stage0 + s * kMergeStageBytes;
-      bulk_load(sb, (m.tensor ? p.a_pool[1] : p.a_pool[0]) + row0 * kQ4RowBytes, cbytes, bar);
-      bulk_load(sb + kQ4CodesBytes, (m.tensor ? p.c_pool[1] : p.c_pool[0]) + row0 * kQ4RowBytes, cbytes, bar);
-      bulk_load(sb + 2 * kQ4CodesBytes, (m.tensor ? p.a_meta[1] : p.a_meta[0]) + moff, mbytes, bar);
-      bulk_load(sb + 2 * kQ4CodesBytes + kQ4MetaBytes, (m.tensor ? p.c_meta[1] : p.c_meta[0]) + moff, mbytes, bar);
+      bulk_load(sb, P.a_pool[ts] + row0 * kQ4RowBytes, cbytes, bar);
+      bulk_load(sb + kQ4CodesBytes, P.c_pool[ts] + row0 * kQ4RowBytes, cbytes, bar);
+      bulk_load(sb + 2 * kQ4CodesBytes, P.a_meta[ts] + moff, mbytes, bar);
+      bulk_load(sb + 2 * kQ4CodesBytes + kQ4MetaBytes, P.c_meta[ts] + moff, mbytes, bar);
     }
     return true;
   };
 
   PageItem m;
-  page_item_init(m, blockIdx.x, ipp, P, pre_s);
+  page_item_init(m, blockIdx.x, ipp, P_all, pre_s, n_slots);
   // warp 0 looks two items ahead (and loads page ids three ahead: a demand load takes microseconds
   // while the copies saturate the memory system)
   PageItem m1 = m, m2 = m, m3 = m;
   int pg2 = 0, pg3 = 0;
   if (warp == 0) {
-    page_item_advance(m1, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m1, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
     m2 = m1;
-    page_item_advance(m2, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m2, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
     m3 = m2;
-    page_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m3, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
     const int pg0 = page_of(m), pg1 = page_of(m1);
     pg2 = page_of(m2);
     pg3 = page_of(m3);
     if (lane == 0) {
-      if (m.tensor < 2) issue(0, m, pg0);
-      if (m1.tensor < 2) issue(1, m1, pg1);
+      if (m.tensor < n_slots) issue(0, m, pg0);
+      if (m1.tensor < n_slots) issue(1, m1, pg1);
     }
   }
 
   const int quad = tid >> 2, k = tid & 3;
-  long long run_seg = -1;  // segment of the warp's running distance extremes
+  long long run_seg = -1;  // segment of the warp's running distance extremes (pairs counted through)
+  unsigned* run_ptr = nullptr;  // its d_min / d_max words
   float run_min = 0.f, run_max = 0.f;
-  for (int it = 0; m.tensor < 2; ++it) {
+  for (int it = 0; m.tensor < n_slots; ++it) {
     if (warp == 0) {
       // item it + 2 goes into the stage that item it - 1 has just left
       int good = 1;
-      if (lane == 0 && m2.tensor < 2) good = issue(it + 2, m2, pg2) ? 1 : 0;
+      if (lane == 0 && m2.tensor < n_slots) good = issue(it + 2, m2, pg2) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
       m2 = m3;
       pg2 = pg3;
-      page_item_advance(m3, s_pg, s_grp, ipp, P, pre_s);
+      page_item_advance(m3, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
       pg3 = page_of(m3);
     }
     const int s = it % kMergeStages;
-    if (!mbar_wait(full0 + 8 * s, (it / kMergeStages) & 1, s_abort, p.status)) break;
+    if (!mbar_wait(full0 + 8 * s, (it / kMergeStages) & 1, s_abort, status0)) break;
+    const MergePair& P = p.pr[m.tensor >> 1];
+    const int ts = m.tensor & 1;
     const int page = page_s[s];
     const int n = lens[m.b];
     const int row = m.grp * kRowsPerItem + quad;  // one row per quad of lanes; a warp = 8 consecutive rows of one head
@@ -322,7 +337,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       const unsigned char* sb = stages + s * kMergeStageBytes;
       const uint4 qa = *reinterpret_cast<const uint4*>(sb + quad * kQ4RowBytes + k * 16);
       const uint4 qc = *reinterpret_cast<const uint4*>(sb + kQ4CodesBytes + quad * kQ4RowBytes + k * 16);
-      const bool per_channel = m.tensor == 0;
+      const bool per_channel = ts == 0;
       const int mo = per_channel ? ((quad >> 5) * 128 + 32 * k) : (quad * 4 + k);  // in (scale, zero) pairs
       const uint32_t* ma = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes) + mo;
       const uint32_t* mc = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes + kQ4MetaBytes) + mo;
@@ -341,14 +356,14 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
     }
     float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
-      char* tile = (m.tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * H + head) * tile_bytes(ps);
+      char* tile = P.e_pool[ts] + ((size_t)page * H + head) * tile_bytes(ps);
 #pragma unroll
       for (int x = 0; x < 4; ++x) st_stream16(tile + tk * kRowBytes + chunk_pos(tk, ci[x]) * 16, e[x]);
       if (k == 0) {
         float* scp = reinterpret_cast<float*>(tile + ps * kRowBytes) + tk;
         scp[0] = g_a;
         scp[ps] = g_c;
-        p.dist[(((size_t)page * H + head) * 2 + m.tensor) * ps + tk] = d;
+        P.dist[(((size_t)page * H + head) * 2 + ts) * ps + tk] = d;
       }
       dmin = d;
       dmax = d;
@@ -362,13 +377,15 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       // Running extremes stay in registers while the warp's items keep falling into the same segment
       // (consecutive items of a CTA usually do): all CTAs work on one sequence at a time, and one
       // atomic pair per warp and item on its few addresses queues up in the memory system.
-      const long long seg = ((long long)m.tensor * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
+      const int seg_local = (ts * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
+      const long long seg = (long long)(m.tensor >> 1) * (2LL * p.g.batch * H) + seg_local;
       if (seg != run_seg) {
         if (lane == 0 && run_seg >= 0) {
-          atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));
-          atomicMax(&p.seg_minmax[run_seg * 2 + 1], __float_as_uint(run_max));
+          atomicMin(run_ptr, __float_as_uint(run_min));
+          atomicMax(run_ptr + 1, __float_as_uint(run_max));
         }
         run_seg = seg;
+        run_ptr = P.seg_minmax + 2 * seg_local;
         run_min = dmin;
         run_max = dmax;
       } else {
@@ -376,11 +393,11 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
         run_max = fmaxf(run_max, dmax);
       }
     }
-    page_item_advance(m, s_pg, s_grp, ipp, P, pre_s);
+    page_item_advance(m, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
   }
   if (lane == 0 && run_seg >= 0) {
-    atomicMin(&p.seg_minmax[run_seg * 2], __float_as_uint(run_min));
-    atomicMax(&p.seg_minmax[run_seg * 2 + 1], __float_as_uint(run_max));
+    atomicMin(run_ptr, __float_as_uint(run_min));
+    atomicMax(run_ptr + 1, __float_as_uint(run_max));
   }
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
@@ -423,15 +440,85 @@ struct RetainParams {
   double gamma;
 };
 
-__global__ void merge_init_kernel(unsigned* seg_minmax, int nseg, int32_t* status) {
+// The part of RetainParams that differs from pair to pair when several pairs are merged at once.
+struct RetainPair {
+  const char* a_pool[2];
+  const char* c_pool[2];
+  const char* a_meta[2];
+  const char* c_meta[2];
+  char* e_pool[2];
+  const float* dist;
+  const float* seg_minmax;
+  int32_t* chunk_count;
+  int32_t* chunk_offset;
+  int32_t* chunk_eq;
+  uint32_t* seg_sel;
+  int32_t* ret_count;
+  int32_t* ret_offset;
+  int32_t* ret_index;
+  char* ret_rows;
+  int64_t ret_capacity;
+  int32_t* status;
+  int32_t* ret_prefix;
+  int ret_prefix_stride;
+};
+struct RetainBatch {
+  Geom g;
+  RetainPair pr[kMaxMergePairs];  // blockIdx.z selects the pair
+  int q4, dtype, chunks_per_seg, nseg, mode, do_retention;
+  double gamma;
+};
+__device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int pair) {
+  const RetainPair& r = bp.pr[pair];
+  RetainParams p;
+  p.g = bp.g;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    p.a_pool[i] = r.a_pool[i];
+    p.c_pool[i] = r.c_pool[i];
+    p.a_meta[i] = r.a_meta[i];
+    p.c_meta[i] = r.c_meta[i];
+    p.e_pool[i] = r.e_pool[i];
+  }
+  p.q4 = bp.q4;
+  p.dtype = bp.dtype;
+  p.dist = r.dist;
+  p.seg_minmax = r.seg_minmax;
+  p.chunk_count = r.chunk_count;
+  p.chunk_offset = r.chunk_offset;
+  p.chunk_eq = r.chunk_eq;
+  p.seg_sel = r.seg_sel;
+  p.ret_count = r.ret_count;
+  p.ret_offset = r.ret_offset;
+  p.ret_index = r.ret_index;
+  p.ret_rows = r.ret_rows;
+  p.ret_capacity = r.ret_capacity;
+  p.status = r.status;
+  p.ret_prefix = r.ret_prefix;
+  p.ret_prefix_stride = r.ret_prefix_stride;
+  p.chunks_per_seg = bp.chunks_per_seg;
+  p.nseg = bp.nseg;
+  p.mode = bp.mode;
+  p.do_retention = bp.do_retention;
+  p.gamma = bp.gamma;
+  return p;
+}
+
+struct InitParams {
+  unsigned* seg_minmax[kMaxMergePairs];
+  int32_t* status[kMaxMergePairs];
+  int nseg;
+};
+__global__ void merge_init_kernel(const __grid_constant__ InitParams ip) {
   grid_dep_wait();
   grid_dep_launch();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < nseg) {
+  unsigned* seg_minmax = ip.seg_minmax[blockIdx.y];
+  if (i < ip.nseg) {
     seg_minmax[2 * i] = 0x7f800000u;
     seg_minmax[2 * i + 1] = 0u;
   }
-  if (i < MC_STATUS_WORDS) status[i] = 0;
+  if (i < MC_STATUS_WORDS) ip.status[blockIdx.y][i] = 0;
 }
 
 // Retention decision of one token; the threshold is formed in double from the fp32 extremes.
@@ -489,9 +576,10 @@ __device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int 
 // Top-k reading of the retention rule: per segment, the k-th largest distance (k = ceil(gamma n)) by a
 // radix select over the float bits (d >= 0, so unsigned order is float order), and how many of the
 // tokens equal to it belong to the k largest.
-__global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const RetainParams p) {
+__global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const __grid_constant__ RetainBatch bp) {
   grid_dep_wait();
   grid_dep_launch();
+  const RetainParams p = retain_view(bp, blockIdx.z);
   __shared__ int hist[256];
   __shared__ uint32_t s_prefix, s_mask;
   __shared__ int s_remaining;
@@ -549,9 +637,10 @@ __global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const Retain
 
 // Per (segment, 1024-token chunk): how many tokens Eq. 4 keeps.  The block that finishes last
 // (ticket in a status word) turns the counts into offsets: exclusive scan in (segment, chunk) order.
-__global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainParams p) {
+__global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_constant__ RetainBatch bp) {
   grid_dep_wait();
   grid_dep_launch();
+  const RetainParams p = retain_view(bp, blockIdx.z);
   __shared__ int s_cnt[kRetThreads / 32], s_eq[kRetThreads / 32];
   __shared__ int s_last;
   __shared__ int s_carry;
@@ -647,9 +736,10 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const RetainP
 // Per (segment, chunk): ordered compaction of the kept token indices, their scales zeroed, bit copies
 // of both layers' rows, and the chunk's eight entries of the prefix table (one per 128 tokens =
 // one warp).  Writes ret_count per segment.
-__global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const RetainParams p) {
+__global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __grid_constant__ RetainBatch bp) {
   grid_dep_wait();
   grid_dep_launch();
+  const RetainParams p = retain_view(bp, blockIdx.z);
   __shared__ int s_warp[kRetThreads / 32];
   const int seg = blockIdx.y, chunk = blockIdx.x;
   const int h = seg % p.g.n_kv_heads;
@@ -711,11 +801,12 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   int pos = out0 + before + x - c;
   if (m) {  // (kept tokens lie in a page that keep_masks4 has checked)
     const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
-    float* sc = reinterpret_cast<float*>(p.e_pool[tensor] + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
+    float* sc = reinterpret_cast<float*>((tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
                                          p.g.page_size * kRowBytes) + (tok0 & (p.g.page_size - 1));
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (m & (1u << j)) {
+        if (!MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) continue;  // (range-checked build)
         p.ret_index[pos++] = tok0 + j;
         // a retained token is served from its raw rows: the scale -0 makes the shared direction
         // contribute nothing for it wherever scales are applied blindly, and tells the attention
@@ -730,19 +821,20 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const Retai
   const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
   for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
     const int ent = r >> 1, layer = r & 1;
+    if (!MC_IN_BOUNDS(out0 >= 0 && (int64_t)out0 + ent < p.ret_capacity, p.status)) continue;  // (range-checked build)
     const int tok = p.ret_index[out0 + ent];
     const int page = checked_page(p.g, b, tok >> p.g.page_shift, p.status);
     if (page < 0) continue;
     const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
     char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
     if (!p.q4) {
-      const char* src = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kRowBytes + l16 * 16;
+      const char* src = (layer ? (tensor ? p.c_pool[1] : p.c_pool[0]) : (tensor ? p.a_pool[1] : p.a_pool[0])) + row * kRowBytes + l16 * 16;
       *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
     } else {
       // lane l16: channels [8 l16, 8 l16 + 8).  code * scale + zero is formed in double (exact) and
       // rounded once to the storage type, so the row is the same bits on any machine.
-      const char* codes = (layer ? p.c_pool[tensor] : p.a_pool[tensor]) + row * kQ4RowBytes;
-      const char* meta = layer ? p.c_meta[tensor] : p.a_meta[tensor];
+      const char* codes = (layer ? (tensor ? p.c_pool[1] : p.c_pool[0]) : (tensor ? p.a_pool[1] : p.a_pool[0])) + row * kQ4RowBytes;
+      const char* meta = layer ? (tensor ? p.c_meta[1] : p.c_meta[0]) : (tensor ? p.a_meta[1] : p.a_meta[0]);
       const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + l16 * 4);
       const __half2* mp = tensor == 0 ? reinterpret_cast<const __half2*>(meta) + (row / p.g.page_size) * 128 + 8 * l16
                                       : reinterpret_cast<const __half2*>(meta) + row * 4 + (l16 >> 2);
@@ -841,41 +933,80 @@ size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
   return align_up(nseg * chunks_per_seg(bt->max_seq_len) * sizeof(int32_t), 256) * 3 + align_up(nseg * 2 * sizeof(uint32_t), 256);
 }
 
-mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
-                       const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
-                       int do_retention, void* workspace, cudaStream_t stream) {
+mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geom& g, int n_pairs, const mc_layer_kv* const* lm1,
+                             const mc_layer_kv* const* l, const mc_layer_q4* const* q_lm1, const mc_layer_q4* const* q_l,
+                             const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream) {
   const bool q4 = q_lm1 != nullptr;
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
   // every shape limit before the first launch
+  if (n_pairs < 1 || n_pairs > kMaxMergePairs) return MC_ERR_SHAPE;
   if (bt->batch > kMergeMaxBatchSmem) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
-  if (2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) *
+  if (2LL * n_pairs * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) *
           ((cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem) > 0x7fffffffLL)
     return MC_ERR_SHAPE;
-  MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256), dim3(256), 0, stream, reinterpret_cast<unsigned*>(out->seg_minmax), nseg, out->status));
+  InitParams ip;
+  for (int i = 0; i < kMaxMergePairs; ++i) {
+    ip.seg_minmax[i] = reinterpret_cast<unsigned*>(out[std::min(i, n_pairs - 1)]->seg_minmax);
+    ip.status[i] = out[std::min(i, n_pairs - 1)]->status;
+  }
+  ip.nseg = nseg;
+  MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256, n_pairs), dim3(256), 0, stream, ip));
   MC_CUDA_CHECK(cudaGetLastError());
   if (bt->batch == 0) return MC_OK;
 
   MergeParams mp;
+  RetainBatch rb;
   mp.g = g;
-  mp.a_pool[0] = (const char*)(q4 ? q_lm1->k_codes : lm1->k_pool);
-  mp.a_pool[1] = (const char*)(q4 ? q_lm1->v_codes : lm1->v_pool);
-  mp.c_pool[0] = (const char*)(q4 ? q_l->k_codes : l->k_pool);
-  mp.c_pool[1] = (const char*)(q4 ? q_l->v_codes : l->v_pool);
-  mp.a_meta[0] = (const char*)(q4 ? q_lm1->k_meta : nullptr);
-  mp.a_meta[1] = (const char*)(q4 ? q_lm1->v_meta : nullptr);
-  mp.c_meta[0] = (const char*)(q4 ? q_l->k_meta : nullptr);
-  mp.c_meta[1] = (const char*)(q4 ? q_l->v_meta : nullptr);
-  mp.e_pool[0] = (char*)out->e_k;
-  mp.e_pool[1] = (char*)out->e_v;
-  mp.dist = out->dist;
-  mp.seg_minmax = reinterpret_cast<unsigned*>(out->seg_minmax);
+  rb.g = g;
+  const size_t arr = align_up((size_t)nseg * chunks_per_seg(bt->max_seq_len) * sizeof(int32_t), 256);
+  const size_t ws_pair = merge_workspace_bytes(cfg, bt);
+  for (int i = 0; i < kMaxMergePairs; ++i) {
+    const int j = std::min(i, n_pairs - 1);  // (unused slots repeat the last pair: no null pointers in the parameters)
+    MergePair& m = mp.pr[i];
+    m.a_pool[0] = (const char*)(q4 ? q_lm1[j]->k_codes : lm1[j]->k_pool);
+    m.a_pool[1] = (const char*)(q4 ? q_lm1[j]->v_codes : lm1[j]->v_pool);
+    m.c_pool[0] = (const char*)(q4 ? q_l[j]->k_codes : l[j]->k_pool);
+    m.c_pool[1] = (const char*)(q4 ? q_l[j]->v_codes : l[j]->v_pool);
+    m.a_meta[0] = (const char*)(q4 ? q_lm1[j]->k_meta : nullptr);
+    m.a_meta[1] = (const char*)(q4 ? q_lm1[j]->v_meta : nullptr);
+    m.c_meta[0] = (const char*)(q4 ? q_l[j]->k_meta : nullptr);
+    m.c_meta[1] = (const char*)(q4 ? q_l[j]->v_meta : nullptr);
+    m.e_pool[0] = (char*)out[j]->e_k;
+    m.e_pool[1] = (char*)out[j]->e_v;
+    m.dist = out[j]->dist;
+    m.seg_minmax = reinterpret_cast<unsigned*>(out[j]->seg_minmax);
+    m.status = out[j]->status;
+    RetainPair& r = rb.pr[i];
+    for (int t = 0; t < 2; ++t) {
+      r.a_pool[t] = m.a_pool[t];
+      r.c_pool[t] = m.c_pool[t];
+      r.a_meta[t] = m.a_meta[t];
+      r.c_meta[t] = m.c_meta[t];
+      r.e_pool[t] = m.e_pool[t];
+    }
+    r.dist = out[j]->dist;
+    r.seg_minmax = out[j]->seg_minmax;
+    char* ws = (char*)workspace + (size_t)j * ws_pair;
+    r.chunk_count = reinterpret_cast<int32_t*>(ws);
+    r.chunk_offset = reinterpret_cast<int32_t*>(ws + arr);
+    r.chunk_eq = reinterpret_cast<int32_t*>(ws + 2 * arr);
+    r.seg_sel = reinterpret_cast<uint32_t*>(ws + 3 * arr);
+    r.ret_count = out[j]->ret_count;
+    r.ret_offset = out[j]->ret_offset;
+    r.ret_index = out[j]->ret_index;
+    r.ret_rows = (char*)out[j]->ret_rows;
+    r.ret_capacity = out[j]->ret_capacity;
+    r.status = out[j]->status;
+    r.ret_prefix = out[j]->ret_prefix;
+    r.ret_prefix_stride = (int)out[j]->ret_prefix_stride;
+  }
+  mp.n_pairs = n_pairs;
   mp.merge_fn = cfg->merge_fn;
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
   // upper bound of the item count (the kernel enumerates the pages that hold tokens)
-  const long long total = 2LL * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
-  mp.status = out->status;
+  const long long total = 2LL * n_pairs * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
   if (total > 0) {
     int n_sm = 0;
     if (mc_status st = sm_count(&n_sm)) return st;
@@ -889,46 +1020,26 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
     MC_CUDA_CHECK(launch_pdl(kern, dim3(grid), dim3(kMergeThreads), smem, stream, mp));
   }
 
-  RetainParams rp;
-  rp.g = g;
-  rp.a_pool[0] = mp.a_pool[0];
-  rp.a_pool[1] = mp.a_pool[1];
-  rp.c_pool[0] = mp.c_pool[0];
-  rp.c_pool[1] = mp.c_pool[1];
-  rp.a_meta[0] = mp.a_meta[0];
-  rp.a_meta[1] = mp.a_meta[1];
-  rp.c_meta[0] = mp.c_meta[0];
-  rp.c_meta[1] = mp.c_meta[1];
-  rp.q4 = q4 ? 1 : 0;
-  rp.dtype = cfg->dtype;
-  rp.e_pool[0] = mp.e_pool[0];
-  rp.e_pool[1] = mp.e_pool[1];
-  rp.dist = out->dist;
-  rp.seg_minmax = out->seg_minmax;
-  rp.chunks_per_seg = chunks_per_seg(bt->max_seq_len);
-  rp.nseg = nseg;
-  rp.chunk_count = reinterpret_cast<int32_t*>(workspace);
-  const size_t arr = align_up((size_t)nseg * rp.chunks_per_seg * sizeof(int32_t), 256);
-  rp.chunk_offset = reinterpret_cast<int32_t*>((char*)workspace + arr);
-  rp.chunk_eq = reinterpret_cast<int32_t*>((char*)workspace + 2 * arr);
-  rp.seg_sel = reinterpret_cast<uint32_t*>((char*)workspace + 3 * arr);
-  rp.ret_count = out->ret_count;
-  rp.ret_offset = out->ret_offset;
-  rp.ret_index = out->ret_index;
-  rp.ret_rows = (char*)out->ret_rows;
-  rp.ret_capacity = out->ret_capacity;
-  rp.status = out->status;
-  rp.ret_prefix = out->ret_prefix;
-  rp.ret_prefix_stride = (int)out->ret_prefix_stride;
-  rp.mode = cfg->retain_mode;
-  rp.do_retention = do_retention;
-  rp.gamma = cfg->gamma;
-  dim3 grid(rp.chunks_per_seg, nseg);
+  rb.q4 = q4 ? 1 : 0;
+  rb.dtype = cfg->dtype;
+  rb.chunks_per_seg = chunks_per_seg(bt->max_seq_len);
+  rb.nseg = nseg;
+  rb.mode = cfg->retain_mode;
+  rb.do_retention = do_retention;
+  rb.gamma = cfg->gamma;
+  dim3 grid(rb.chunks_per_seg, nseg, n_pairs);
   if (cfg->retain_mode == MC_RETAIN_TOPK)
-    MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg), dim3(kRetThreads), 0, stream, rp));
-  MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
-  MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rp));
+    MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg, 1, n_pairs), dim3(kRetThreads), 0, stream, rb));
+  MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rb));
+  MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rb));
   return MC_OK;
+}
+
+mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_layer_kv* lm1,
+                       const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
+                       int do_retention, void* workspace, cudaStream_t stream) {
+  return launch_merge_pairs(cfg, bt, g, 1, lm1 ? &lm1 : nullptr, l ? &l : nullptr, q_lm1 ? &q_lm1 : nullptr, q_l ? &q_l : nullptr,
+                            &out, do_retention, workspace, stream);
 }
 
 mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,

@@ -369,7 +369,9 @@ __global__ void __launch_bounds__(kQThreads) restore_q4_kernel(const RestoreQ4Pa
   const int cnt = p.ret_count[seg], off = p.ret_offset[seg];
   const int l16 = tid & 15;
   for (int e = tid >> 4; e < cnt; e += kQThreads / 16) {
+    if (!MC_IN_BOUNDS(off >= 0 && (int64_t)off + e < p.ret_capacity, p.status)) continue;  // (range-checked build)
     const int tok = p.ret_index[off + e];
+    if (!MC_IN_BOUNDS(tok >= 0 && tok < n, p.status)) continue;
     const int pg = checked_page(p.g, b, tok >> 5, p.status);
     if (pg < 0) continue;
     const size_t row = ((size_t)pg * H + h) * kQ4Page + (tok & (kQ4Page - 1));

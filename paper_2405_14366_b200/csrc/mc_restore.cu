@@ -187,7 +187,9 @@ __global__ void __launch_bounds__(kRestoreThreads, kRestoreCtasPerSm) restore_sc
       const int h = seg % H, b = (seg / H) % p.g.batch, tensor = seg / (H * p.g.batch);
       char* dst_pool = tensor ? p.dst_pool[1] : p.dst_pool[0];
       for (int e = hw16; e < cnt; e += kRestoreThreads / 16) {
+        if (!MC_IN_BOUNDS(off >= 0 && (int64_t)off + e < p.ret_capacity, p.status)) continue;  // (range-checked build)
         const int tok = p.ret_index[off + e];
+        if (!MC_IN_BOUNDS(tok >= 0 && tok < len_s[b], p.status)) continue;
         const int page = checked_page(p.g, b, tok >> shift, p.status);
         if (page < 0) continue;
         const size_t row = ((size_t)page * H + h) * ps + (tok & (ps - 1));

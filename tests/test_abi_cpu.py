@@ -35,10 +35,11 @@ def test_status_strings(lib):
 
 
 def _cfg(**kw):
-    d = dict(n_kv_heads=8, n_q_heads=32, head_dim=128, page_size=16, dtype=0, retain_mode=0, t=0.6, gamma=0.05)
+    d = dict(n_kv_heads=8, n_q_heads=32, head_dim=128, page_size=16, dtype=0, retain_mode=0, t=0.6, gamma=0.05,
+             merge_fn=0, cache_bits=0)
     d.update(kw)
     return B._Config(d["n_kv_heads"], d["n_q_heads"], d["head_dim"], d["page_size"], d["dtype"], d["retain_mode"],
-                     d["t"], d["gamma"])
+                     d["t"], d["gamma"], d["merge_fn"], d["cache_bits"])
 
 
 def _batch(batch=2, mpps=4, max_len=64, n_pages=10, bt=0x1000, sl=0x2000):
@@ -62,6 +63,7 @@ def test_workspace_bytes_is_host_arithmetic(lib):
 @pytest.mark.parametrize("kw,code", [
     (dict(head_dim=64), 2), (dict(page_size=8), 2), (dict(n_q_heads=12), 2), (dict(n_q_heads=24), 2),
     (dict(dtype=5), 3), (dict(retain_mode=9), 1), (dict(t=1.5), 1), (dict(gamma=-0.1), 1),
+    (dict(cache_bits=8), 1), (dict(cache_bits=4, page_size=16), 2), (dict(merge_fn=3), 1),
 ])
 def test_bad_config_rejected(lib, kw, code):
     out = C.c_size_t(0)
@@ -128,6 +130,56 @@ def test_pair_bytes_is_host_arithmetic(lib):
     assert L.mc_pair_bytes(C.byref(c), C.byref(b), -1, C.byref(out)) == 1
     assert L.mc_pair_bytes(C.byref(c), C.byref(b), 4, None) == 1
     assert L.mc_pair_bytes(C.byref(_cfg(page_size=8)), C.byref(b), 4, C.byref(out)) == 2
+
+
+def test_q4_cache_sizes_and_argument_checks(lib):
+    """The 4-bit shared cache: tiles of 2816 bytes (2048 of codes, 512 of group parameters, 256 of scales), one
+    16-bit residual tile of 32 tokens per (sequence, head), a merge workspace that also holds the 16-bit
+    staging tiles, and residual pools that must be given."""
+    cfg = mc.McConfig(8, 32, 32, "f16", cache_bits=4)
+    sz = lib.mc_pair_bytes(cfg, batch=4, n_pages=100, max_seq_len=1000, ret_capacity=77)
+    assert sz.tile_bytes == 2816 and sz.e_bytes == 100 * 8 * 2816
+    assert sz.res_bytes == 4 * 8 * (32 * 256 + 2 * 32 * 4)
+    assert sz.total_bytes >= 2 * sz.e_bytes + 2 * sz.res_bytes + sz.dist_bytes and sz.total_bytes % 256 == 0
+    sz16 = lib.mc_pair_bytes(mc.McConfig(8, 32, 32, "f16"), batch=4, n_pages=100, max_seq_len=1000, ret_capacity=77)
+    assert sz16.res_bytes == 0 and sz16.tile_bytes == 3 * 2816
+    L = lib._lib
+    out = C.c_size_t(0)
+    c4, c16, b = _cfg(page_size=32, cache_bits=4), _cfg(page_size=32), _batch(max_len=64, mpps=4, n_pages=10)
+    assert L.mc_workspace_bytes(C.byref(c16), C.byref(b), 0, 1, C.byref(out)) == 0
+    w16 = out.value
+    assert L.mc_workspace_bytes(C.byref(c4), C.byref(b), 0, 1, C.byref(out)) == 0
+    assert out.value == w16 + 2 * 10 * 8 * 8448  # the staging tiles of both tensors (already a multiple of 256)
+    # a 4-bit pair without residual pools is refused; with them the next check (workspace size) answers
+    a = B._LayerKV(0x10000, 0x20000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    assert L.mc_merge_pair(C.byref(c4), C.byref(b), C.byref(a), C.byref(a), C.byref(pc), 1, 0x100000, 1 << 30, None) == 1
+    pcr = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000,
+                       0xE0000, 0xF0000)
+    assert L.mc_merge_pair(C.byref(c4), C.byref(b), C.byref(a), C.byref(a), C.byref(pcr), 1, 0x100000, w16, None) == 5
+    pcm = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000,
+                       0xE0010, 0xF0000)
+    assert L.mc_decode_attn(C.byref(c4), C.byref(b), C.byref(pcm), 0, 0x1000, None, None, 1.0, 0x2000, None, 0x100000, 1 << 24, None) == 4
+
+
+def test_merge_pairs_checks_every_pair_before_launching(lib):
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    a = B._LayerKV(0x10000, 0x20000)
+    mk = lambda st: B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, st)
+    pcs = [mk(0xC0000), mk(0xC1000)]
+    arr = lambda items, T: (C.POINTER(T) * len(items))(*[C.pointer(x) for x in items])
+    out = C.c_size_t(0)
+    assert L.mc_workspace_bytes(C.byref(c), C.byref(b), 0, 1, C.byref(out)) == 0
+    call = lambda lay, pc, n, wsb: L.mc_merge_pairs(C.byref(c), C.byref(b), n, arr(lay, B._LayerKV), arr(lay, B._LayerKV),
+                                                    arr(pc, B._PairCache), 1, 0x100000, wsb, None)
+    assert call([a, a], pcs, 2, out.value) == 5                      # one pair's worth of scratch for two pairs
+    assert call([a, B._LayerKV(0, 0x20000)], pcs, 2, 1 << 30) == 1   # the second pair has a null pool
+    assert call([a, a], [pcs[0], pcs[0]], 2, 1 << 30) == 1           # the same pair cache twice
+    assert call([a, a], pcs, -1, 1 << 30) == 1
+    c4 = _cfg(page_size=32, cache_bits=4)
+    assert L.mc_merge_pairs(C.byref(c4), C.byref(b), 1, arr([a], B._LayerKV), arr([a], B._LayerKV), arr(pcs[:1], B._PairCache),
+                            1, 0x100000, 1 << 30, None) == 6
 
 
 def test_get_stats_rejects_bad_arguments(lib):

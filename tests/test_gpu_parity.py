@@ -516,6 +516,36 @@ def test_full_size_configs_sampled(H, name, gamma, q4):
         print(name, "segment", b, h, "len", int(p.seq_lens_host[b]), stats)
 
 
+@pytest.mark.parametrize("name,n_pairs", [("c4_s", 1), ("c3_s", 2), ("c2_s", 2)])
+def test_merging_several_pairs_at_once_equals_one_by_one(H, name, n_pairs):
+    """mc_merge_pairs (Algorithm 1's loop over the merged layers in one launch sequence): every buffer of
+    every pair cache is bit-identical to what mc_merge_pair writes for that pair alone (which the other
+    tests compare with the oracle)."""
+    wl = CONFIGS[name]
+    lens = gen.make_lengths(wl)[0] if wl.ragged else None
+    n_pairs = min(n_pairs, wl.n_pairs)
+    ps = [H.Problem(wl, pair=i, seq_lens=lens) for i in range(n_pairs)]
+    for p in ps:  # same lengths, same block-table seed: one batch description serves all pairs
+        assert torch.equal(p.block_table, ps[0].block_table) and p.n_pages == ps[0].n_pages
+        words, code = p.run_merge()
+        assert code == 0, words
+    p0 = ps[0]
+    import paper_2405_14366_b200 as mc
+    twins = [mc.PairCache(p0.cfg, p0.B, p0.n_pages, p0.ret_capacity, device=p0.device) for _ in ps]
+    ws1 = p0.lib.mc_workspace_bytes(p0.cfg, p0.batch(), 0)
+    ws = torch.empty(n_pairs * ws1, dtype=torch.uint8, device=p0.device)
+    p0.lib.mc_merge_pairs(p0.cfg, p0.batch(), [p.pools for p in ps], twins, True, ws)
+    torch.cuda.synchronize()
+    for p, tw in zip(ps, twins):
+        words, code = p0.lib.mc_read_status(tw, check=False)
+        assert code == 0, words
+        ref = p.pair
+        for f in ("e_k", "e_v", "dist", "ret_count", "ret_offset", "ret_prefix", "seg_minmax", "status"):
+            assert torch.equal(getattr(tw, f), getattr(ref, f)), f
+        n = int(ref.ret_offset[-1].item())
+        assert torch.equal(tw.ret_index[:n], ref.ret_index[:n]) and torch.equal(tw.ret_rows[:, :n], ref.ret_rows[:, :n])
+
+
 def test_bounded_wait_times_out_into_the_status_word(H):
     """A wait that nothing ends: the kernel gives up after its poll limit, records the time-out in
     the pair's status words and returns; the context stays usable and the next merge clears the flag."""

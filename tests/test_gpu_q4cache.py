@@ -160,3 +160,73 @@ def test_q4_cache_decode_loop(H, dtype):
             differ += int((dc["e_" + tn][b, :n] != om4[tn]["e_bits"][b, :n]).any(-1).sum())
         print(dtype, tn, "rows whose stored bits differ from the oracle's", differ)
         assert differ <= 0.05 * int(p.seq_lens_host.sum()) * hkv
+
+
+def test_full_size_serving_mix_q4_cache(H):
+    """Config 4 as the paper's efficiency setting has it (Sec. 5): the ragged batch of 64 at full size, the
+    layers arriving in 4 bits and the shared cache kept in 4 bits, in the launch configuration the benchmark
+    times.  Sampled (sequence, head) segments -- the longest and the shortest sequence among them -- go
+    through all three stages."""
+    from oracle import minicache_oracle as orc
+    from test_gpu_parity import _Segment, _full_tensors
+    wl = CONFIGS["c4"]
+    pair = wl.n_pairs - 1
+    rs = np.random.RandomState(23)
+    lens = gen.make_lengths(wl)[0]
+    segs = [(int(rs.randint(wl.batch)), int(rs.randint(wl.n_kv_heads))) for _ in range(4)]
+    segs[0] = (int(np.argmax(lens)), segs[0][1])
+    segs[1] = (int(np.argmin(lens)), segs[1][1])
+    th2 = int(lens.sum()) * wl.n_kv_heads * 2
+    kw = dict(pair=pair, decode_room=wl.decode_steps + 1, tensors=_full_tensors("c4", pair), seq_lens=lens, q4=True,
+              segments=segs, ret_capacity=int(0.12 * th2) + 1024)
+    p16 = H.Problem(wl, **kw)
+    words, code = p16.run_merge()
+    assert code == 0, words
+    dc16 = p16.device_cache()
+    del p16.pair, p16.q4_pools
+    p4 = H.Problem(wl, cache_bits=4, **kw)
+    words, code = p4.run_merge()
+    assert code == 0, words
+    dc4 = p4.device_cache()
+    assert np.array_equal(dc4["ret_index"], dc16["ret_index"])
+    dk, dv = p4.run_restore(1)
+    dkl, dvl = p4.logical_of(dk), p4.logical_of(dv)
+    dk, dv = p4.run_restore(0, fp32=True)
+    dkf, dvf = p4.logical_of(dk), p4.logical_of(dv)
+    del dk, dv
+    wlb = dataclasses.replace(wl, batch=p4.B)
+    q = gen.make_queries(wlb, 2, n_sets=2)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    extra = wl.decode_steps + 1
+
+    def attn(layer_sel, qq, kk, vv):
+        n_sets = 2 if layer_sel == 2 else 1
+        out = torch.zeros(n_sets, p4.B, p4.Hq, 128, dtype=p4.cfg.torch_dtype, device=p4.device)
+        lse = torch.zeros(n_sets, p4.B, p4.Hq, dtype=torch.float32, device=p4.device)
+        p4.lib.mc_decode_attn(p4.cfg, p4.batch(extra), p4.pair, layer_sel, qq.to(p4.device), kk.to(p4.device), vv.to(p4.device),
+                              1.0 / math.sqrt(128.0), out, lse, p4.workspace(1, n_sets, extra))
+        torch.cuda.synchronize()
+        return out.cpu(), lse.cpu()
+    out, lse = attn(1, q[1:2].contiguous(), kn[1:2].contiguous(), vn[1:2].contiguous())
+    out2, lse2 = attn(2, q, kn, vn)
+    words, code = p4.lib.mc_read_status(p4.pair, check=False)
+    assert code == 0, words
+    for b, h in segs:
+        sg = _Segment(p4, b, h)
+        sg.cache_bits = 4
+        om16 = sg.oracle_merge(orc)
+        dcs16, dcs4 = sg.slice_cache(dc16), sg.slice_cache(dc4)
+        stats = H.compare_merge(sg, om16, dcs16)
+        om4 = {tn: orc.q4_cache_pair(om16[tn], sg.seq_lens_host, tn, sg.dtype) for tn in ("k", "v")}
+        dcs4["q4"] = {(tn, 0, 0): dc4["q4"][(tn, b, h)] for tn in ("k", "v")}
+        stats.update(H.compare_q4_cache(sg, dcs4, dcs16, om4))
+        stats.update(H.compare_restore(sg, om4, dcs4, 1, dkl[b:b + 1, :, h:h + 1], dvl[b:b + 1, :, h:h + 1]))
+        stats.update({"f32_" + k: v for k, v in
+                      H.compare_restore(sg, om4, dcs4, 0, dkf[b:b + 1, :, h:h + 1], dvf[b:b + 1, :, h:h + 1]).items()})
+        slq = lambda x: x[:, b:b + 1, h:h + 1].contiguous()  # one query head per kv head in this workload
+        stats.update(H.compare_attention(sg, om4, 1, slq(q[1:2]), slq(out), slq(lse), slq(kn[1:2]), slq(vn[1:2]), dc=dcs4))
+        stats.update({"pair_" + k: v for k, v in
+                      H.compare_attention(sg, om4, 2, slq(q), slq(out2), slq(lse2), slq(kn), slq(vn), dc=dcs4).items()})
+        print("c4 4-bit cache, segment", b, h, "len", int(p4.seq_lens_host[b]), stats)
