@@ -26,6 +26,11 @@ What each function follows (MiniCache, arXiv 2405.14366):
 * ``merge_rows_fmax`` / ``merge_rows_mean``
                             Eq. A (Sec. "Alternative merging function") and the
                             averaging baseline of Sec. 3.1.
+* ``dynamic_t``             Sec. 5, ablation of t: the interpolation parameter taken per
+                            token from the relative magnitude ratio of the two layers.
+* ``retention_union``       Sec. 4.2 writes ONE index set I for the pair cache while
+                            Algorithm 2 computes one per tensor: the reading with one
+                            set, the union of the keys' and the values' sets.
 
 Readings taken where the paper is silent or inconsistent (each is a keyword
 argument so the other reading can be run):
@@ -45,6 +50,12 @@ argument so the other reading can be run):
   layer l-1's.  A zero row has angle 0 and contributes no direction.
 * restore divides by the length of the *stored* (16-bit rounded) direction,
   exactly as Eq. 2 is written.
+* ``t="ratio"`` (not the default): the paper observes that the best t follows the
+  relative magnitude ratio of adjacent layers, whose histogram clusters at 0.4 and
+  0.6 (the same scale as t), and suggests taking t from it; it gives no formula.
+  Reading: per token t_i = |x^l_i| / (|x^{l-1}_i| + |x^l_i|), so the layer with the
+  larger magnitude pulls the direction its way and equal magnitudes give the
+  geodesic midpoint; 0.5 if both rows are zero.
 
 Parity unpinned: none of the functions here.  What stays unpinned is outside
 this file: whether merging preserves a real model's accuracy needs trained
@@ -99,8 +110,19 @@ def encode_bits(x: np.ndarray, dtype: str) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Merge (Eq. 3), distance, alternative merge functions
 # --------------------------------------------------------------------------
-def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") -> Dict[str, np.ndarray]:
+def dynamic_t(n_a: np.ndarray, n_c: np.ndarray) -> np.ndarray:
+    """Per-token interpolation parameter from the relative magnitude ratio (Sec. 5, ablation of t):
+    t = |x^l| / (|x^{l-1}| + |x^l|); 0.5 where both magnitudes are zero."""
+    n_a = np.asarray(n_a, F64)
+    n_c = np.asarray(n_c, F64)
+    tot = n_a + n_c
+    return np.where(tot > 0.0, n_c / np.where(tot > 0.0, tot, 1.0), 0.5)
+
+
+def merge_rows(a: np.ndarray, c: np.ndarray, t, convention: str = "eq3") -> Dict[str, np.ndarray]:
     """SLERP-merge rows a (layer l-1) and c (layer l); both [..., D] float64.
+    t: the interpolation parameter of Eq. 3, a number, an array with one value per row, or
+    "ratio" (``dynamic_t`` of the two magnitudes).
 
     Returns e (unit direction, float64, not yet rounded for storage), n_a, n_c
     (the two magnitudes), omega (angle in [0, pi]) and d = omega / pi."""
@@ -108,6 +130,11 @@ def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") 
     c = np.asarray(c, F64)
     n_a = np.sqrt(np.sum(a * a, axis=-1))
     n_c = np.sqrt(np.sum(c * c, axis=-1))
+    if isinstance(t, str):
+        if t != "ratio":
+            raise ValueError(t)
+        t = dynamic_t(n_a, n_c)
+    t = np.asarray(t, F64)
     za = n_a == 0.0
     zc = n_c == 0.0
     u = a / np.where(za, 1.0, n_a)[..., None]
@@ -122,6 +149,7 @@ def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") 
         ta, tc = t, 1.0 - t
     else:
         raise ValueError(convention)
+    ta, tc = np.broadcast_to(ta, omega.shape), np.broadcast_to(tc, omega.shape)
     safe = np.where(sinw < SIN_GUARD, 1.0, sinw)
     w_a = np.sin(ta * omega) / safe
     w_c = np.sin(tc * omega) / safe
@@ -129,14 +157,14 @@ def merge_rows(a: np.ndarray, c: np.ndarray, t: float, convention: str = "eq3") 
     # sin(Omega) -> 0 with the same direction: limit of Eq. 3, renormalised.
     same = (sinw < SIN_GUARD) & (cosw > 0.0) & ~(za | zc)
     if np.any(same):
-        lin = ta * u + tc * v
+        lin = ta[..., None] * u + tc[..., None] * v
         len_lin = np.sqrt(np.sum(lin * lin, axis=-1))
         lin = lin / np.where(same, len_lin, 1.0)[..., None]
         e = np.where(same[..., None], lin, e)
     # opposite directions: Eq. 3 is undefined; take the endpoint t is closer to.
     opp = (sinw < SIN_GUARD) & (cosw <= 0.0) & ~(za | zc)
     if np.any(opp):
-        pick = v if tc >= 0.5 else u
+        pick = np.where((tc >= 0.5)[..., None], v, u)
         e = np.where(opp[..., None], pick, e)
     # zero rows carry no direction: use the other row's (zero vector if both).
     e = np.where((za & ~zc)[..., None], v, e)
@@ -198,8 +226,15 @@ def retention_indices(d: np.ndarray, gamma: float, mode: str = "distinct") -> np
 # --------------------------------------------------------------------------
 # One layer pair (Algorithm 2, "MiniCache Prefill")
 # --------------------------------------------------------------------------
+def retention_union(retained_k: Dict, retained_v: Dict) -> Dict:
+    """One index set per (sequence, kv head) for keys and values alike -- Sec. 4.2 writes the pair cache with
+    a single I, Algorithm 2 computes one per tensor --: a token either tensor's rule (Eq. 4) keeps is kept
+    unmerged in both."""
+    return {key: np.union1d(retained_k[key], retained_v[key]).astype(np.int64) for key in retained_k}
+
+
 def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[int], dtype: str,
-               t: float, gamma: float, mode: str = "distinct", convention: str = "eq3",
+               t, gamma: float, mode: str = "distinct", convention: str = "eq3",
                do_retention: bool = True, merge_fn: str = "slerp") -> Dict[str, object]:
     """Compress one tensor (K or V) of a layer pair.
 
@@ -211,7 +246,7 @@ def merge_pair(x_lm1_bits: np.ndarray, x_l_bits: np.ndarray, seq_lens: Sequence[
                              mode, convention, do_retention, merge_fn)
 
 
-def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dtype: str, t: float, gamma: float,
+def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dtype: str, t, gamma: float,
                       mode: str = "distinct", convention: str = "eq3", do_retention: bool = True,
                       merge_fn: str = "slerp") -> Dict[str, object]:
     """``merge_pair`` on rows given as float64 values (e.g. de-quantised 4-bit layers); `dtype` is
@@ -242,7 +277,7 @@ def merge_pair_values(a: np.ndarray, c: np.ndarray, seq_lens: Sequence[int], dty
             "omega": m["omega"], "retained": retained}
 
 
-def append_rows(a_bits: np.ndarray, c_bits: np.ndarray, dtype: str, t: float,
+def append_rows(a_bits: np.ndarray, c_bits: np.ndarray, dtype: str, t,
                 convention: str = "eq3", merge_fn: str = "slerp") -> Dict[str, np.ndarray]:
     """Merge the decode step's new token pair (no retention decision for it)."""
     a, c = decode_bits(a_bits, dtype), decode_bits(c_bits, dtype)

@@ -35,12 +35,15 @@
 namespace mc {
 
 constexpr int kTile = 64;  // tokens per pipeline stage
+constexpr int kUnit_ = 128;  // (= kUnit below) tokens per stage of 4-bit tiles
 constexpr int kStages = 5;
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
 constexpr int kMaxRows = 8;                          // query rows per (sequence, kv head): the 8-wide N tile
 constexpr int kStageBytes = (kTile / 16) * (16 * kRowBytes + 2 * 16 * 4);  // 64 tokens of tiles: 16896 for any page size
+constexpr int kQ4StageBytes = (kUnit_ / kQ4Page) * kQ4TileBytes;  // four 4-bit tiles: 11264
+constexpr int kQ4Stages = 5;
 constexpr int kEntryBytes = 272;  // a retained entry: 256-byte raw row, int32 token index, padding
 constexpr int kMaxBatchSmem = 512;
 constexpr int kCtasPerSm = 2;
@@ -268,6 +271,10 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   // this library writes them, so they are read before the wait on the previous kernel in the
   // stream (whose tail this prologue then overlaps).  The pair cache and the workspace are touched
   // only after the wait.
+  // stage ring: five slots of 64 tokens of 16-bit tiles, or (4-bit cache) four slots of four 4-bit tiles,
+  // which also hold the residual tile or a stage of retained entries
+  constexpr int STAGE_BYTES = Q4 ? kQ4StageBytes : kStageBytes;
+  constexpr int N_STAGES = Q4 ? kQ4Stages : kStages;
   grid_dep_launch();
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
@@ -281,26 +288,26 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
-  float* S = reinterpret_cast<float*>(smem + kStages * kStageBytes);     // [kMaxRows][s_stride]
+  float* S = reinterpret_cast<float*>(smem + N_STAGES * STAGE_BYTES);     // [kMaxRows][s_stride]
   uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kScoreFloats);         // [2][kMaxRows][64] packed pairs
   float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
   float* red2_s = red_s + kMaxRows * kConsumerWarps;                     // [kMaxRows][kConsumerWarps]
-  int* info_s = reinterpret_cast<int*>(red2_s + kMaxRows * kConsumerWarps);  // [kStages][2]: entries, extra stages of the phase
-  int* pre_s = info_s + 2 * kStages;                                     // [batch + 1] unit-count prefix
+  int* info_s = reinterpret_cast<int*>(red2_s + kMaxRows * kConsumerWarps);  // [N_STAGES][2]: entries, extra stages of the phase
+  int* pre_s = info_s + 2 * N_STAGES;                                     // [batch + 1] unit-count prefix
   int* len_s = pre_s + kMaxBatchSmem + 1;                                // [batch] sequence lengths
   int* pages_s = len_s + kMaxBatchSmem;                                  // [2][kMaxPiecePages] page ids of a piece
   volatile int* s_abort = pages_s + 2 * kMaxPiecePages;
   uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(s_abort + 1) + 7) & ~uintptr_t(7));
-  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * N_STAGES;
   const uint32_t stage0 = smem_u32(stages);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- prologue -----------------------------------------------------------------------------------
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < N_STAGES; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, kConsumerWarps);
     }
@@ -399,15 +406,15 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
             X = (n_r + n_new + cap_e - 1) / cap_e;
           }
           if (X >= 0 && t >= w.TT + X) break;
-          const int s = it % kStages;
-          if (it >= kStages) {
+          const int s = it % N_STAGES;
+          if (it >= N_STAGES) {
             int good = 1;
-            if (lane == 0) good = mbar_wait(empty0 + 8 * s, ((it / kStages) - 1) & 1, s_abort, p.status) ? 1 : 0;
+            if (lane == 0) good = mbar_wait(empty0 + 8 * s, ((it / N_STAGES) - 1) & 1, s_abort, p.status) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) { ok = false; break; }
           }
           const uint32_t bar = full0 + 8 * s;
-          const uint32_t sbase = stage0 + s * kStageBytes;
+          const uint32_t sbase = stage0 + s * STAGE_BYTES;
           if (Q4 && t < w.Tq) {
             // ---- up to four 4-bit pages (128 tokens): a bulk copy per page
             const int n_pg = min(kUnit / kQ4Page, (w.n_q >> 5) - t * (kUnit / kQ4Page));
@@ -453,7 +460,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
               info_s[2 * s + 1] = X;
               if (add_new) {
                 for (int set = 0; set < nslots; ++set)
-                  *reinterpret_cast<int*>(stages + s * kStageBytes + set * set_bytes + cnt_ret * kEntryBytes + kRowBytes) =
+                  *reinterpret_cast<int*>(stages + s * STAGE_BYTES + set * set_bytes + cnt_ret * kEntryBytes + kRowBytes) =
                       w.split_start + w.n_tok;  // the new token's index
               }
               mbar_expect_tx(bar, (uint32_t)(nslots * (cnt_ret * kEntryBytes + (add_new ? kRowBytes : 0))));
@@ -530,12 +537,17 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     float mx0 = -INFINITY, mx1 = -INFINITY, mxe = -INFINITY;  // running maxima of the scores this thread stores
     // ---- K phase: S[r][i] = log2e * sm_scale * g_i * (q_r . e_i) ---------------------------------
     {
+      // query fragments for 16-bit rows (k step ks: channels 16 ks + 2 t4 + {0, 1} and + {8, 9}); with a
+      // 4-bit cache they are fetched only where a 16-bit stage needs them (residual tile, raw rows)
       uint32_t qa0[8], qa2[8];
+      auto load_qa = [&]() {
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        qa0[ks] = qcur[row * 64 + ks * 8 + (lane & 3)];
-        qa2[ks] = qcur[row * 64 + ks * 8 + 4 + (lane & 3)];
-      }
+        for (int ks = 0; ks < 8; ++ks) {
+          qa0[ks] = qcur[row * 64 + ks * 8 + (lane & 3)];
+          qa2[ks] = qcur[row * 64 + ks * 8 + 4 + (lane & 3)];
+        }
+      };
+      if (!Q4) load_qa();
       // 4-bit tiles: lane (row, t4) owns the channels [32 t4, 32 t4 + 32) of its token rows (16 bytes of
       // codes); k step ks pairs the channels 32 t4 + 4 ks + {0, 1} and + {2, 3} with the matching query words
       uint32_t qk0[8], qk2[8];
@@ -549,14 +561,14 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       const int tk_w = warp * 16;  // this warp's 16 tokens of every tile
       int xk = n_new;              // extra stages after the tiles (an item without tiles has no retained rows)
       for (int t = 0; t < w.TT; ++t, ++it) {
-        const int s = it % kStages;
-        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
-        const uint32_t sbase = stage0 + s * kStageBytes;
+        const int s = it % N_STAGES;
+        if (!mbar_wait(full0 + 8 * s, (it / N_STAGES) & 1, s_abort, p.status)) { ok = false; break; }
+        const uint32_t sbase = stage0 + s * STAGE_BYTES;
         xk = info_s[2 * s + 1];
         if (Q4 && t < w.Tq) {
           // ---- four 4-bit pages, one per warp
           if (warp < (w.n_q >> 5) - t * (kUnit / kQ4Page)) {
-            const unsigned char* tb = stages + s * kStageBytes + warp * kQ4TileBytes;
+            const unsigned char* tb = stages + s * STAGE_BYTES + warp * kQ4TileBytes;
             const int t4 = lane & 3;
             uint4 sK[4], zK[4];  // the group parameters of this lane's 32 channels, word k = channels 8 (4 t4 + k) + ...
 #pragma unroll
@@ -618,6 +630,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         // a 16-bit tile stage: 64 tokens of pages, or (4-bit cache) the residual tile behind the 4-bit pages
         const int s_off = Q4 ? w.n_q : t * kTile;
         const int valid = Q4 ? w.n_tok - w.n_q : min(kTile, w.n_tok - t * kTile);
+        if (Q4) load_qa();
         if (tk_w < valid) {
           // A = the warp's 16 token rows (k step: 16 channels), B = the query rows: D[token][row]
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};  // even / odd k steps
@@ -639,9 +652,9 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
           // (scale = -0) gets its score from its raw row further down; past the last token nothing is stored.
           if (colp < rows) {
             const int tk = tk_w + row;
-            const float* sc = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk >> shift) * tbytes + ps * kRowBytes) +
+            const float* sc = reinterpret_cast<const float*>(stages + s * STAGE_BYTES + (tk >> shift) * tbytes + ps * kRowBytes) +
                               (tk & (ps - 1));
-            const float* sc8 = reinterpret_cast<const float*>(stages + s * kStageBytes + ((tk + 8) >> shift) * tbytes +
+            const float* sc8 = reinterpret_cast<const float*>(stages + s * STAGE_BYTES + ((tk + 8) >> shift) * tbytes +
                                                               ps * kRowBytes) + ((tk + 8) & (ps - 1));
             float* scol = S + s_off + tk;
             const float g0 = sc[slot0 * ps], g8 = sc8[slot0 * ps];
@@ -673,16 +686,17 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
       }
       // ---- retained K rows and the new token: their scores fill the columns the tiles left out.
+      if (Q4 && xk > 0) load_qa();
       for (int x = 0; x < xk && ok; ++x, ++it) {
-        const int s = it % kStages;
-        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const int s = it % N_STAGES;
+        if (!mbar_wait(full0 + 8 * s, (it / N_STAGES) & 1, s_abort, p.status)) { ok = false; break; }
         const int cnt = info_s[2 * s];
         // single layer: warp w takes entries 8w..8w+7; pair mode: warps 0,1 layer l-1, warps 2,3 layer l
         const int set = nslots == 2 ? (warp >> 1) : 0;
         const int e_w = nslots == 2 ? (warp & 1) * 8 : warp * 8;
         if (e_w < cnt) {
           float acc0[4] = {0.f, 0.f, 0.f, 0.f};
-          const unsigned char* sb = stages + s * kStageBytes + set * set_bytes;
+          const unsigned char* sb = stages + s * STAGE_BYTES + set * set_bytes;
           const uint32_t rowaddr = smem_u32(sb) + (uint32_t)((e_w + mr) * kEntryBytes);
 #pragma unroll
           for (int k2 = 0; k2 < 4; ++k2) {
@@ -776,15 +790,15 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
     if (ok) {
       int xv = n_new;
       for (int t = 0; t < w.TT; ++t, ++it) {
-        const int s = it % kStages;
-        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
-        const uint32_t sbase = stage0 + s * kStageBytes;
+        const int s = it % N_STAGES;
+        if (!mbar_wait(full0 + 8 * s, (it / N_STAGES) & 1, s_abort, p.status)) { ok = false; break; }
+        const uint32_t sbase = stage0 + s * STAGE_BYTES;
         xv = info_s[2 * s + 1];
         if (Q4 && t < w.Tq) {
           // ---- four 4-bit pages, one per warp: lane (row, t4) owns the channels row, row + 8 (mod 16)
           // of the token pairs t4, t4 + 4 of each half page: one 16-byte chunk of codes per pair
           if (warp < (w.n_q >> 5) - t * (kUnit / kQ4Page)) {
-            const unsigned char* tb = stages + s * kStageBytes + warp * kQ4TileBytes;
+            const unsigned char* tb = stages + s * STAGE_BYTES + warp * kQ4TileBytes;
             const int t4 = lane & 3;
             const float* gq = reinterpret_cast<const float*>(tb + kQ4ScaleOff) + slot_row * kQ4Page;
             const float* srow = S + row * s_stride + t * kUnit + warp * kQ4Page;
@@ -848,7 +862,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
           // B fragment: row `row`, tokens tk_w + colp, + 1, + 8, + 9
           uint32_t b0 = 0u, b1 = 0u;
           if (row < rows) {
-            const float* scj = reinterpret_cast<const float*>(stages + s * kStageBytes + (tk_w >> shift) * tbytes +
+            const float* scj = reinterpret_cast<const float*>(stages + s * STAGE_BYTES + (tk_w >> shift) * tbytes +
                                                               ps * kRowBytes) + slot_row * ps + (tk_w & (ps - 1));
             const float* srow = S + row * s_stride + s_off + tk_w;
             const float2 p0 = *reinterpret_cast<const float2*>(srow + colp);
@@ -880,14 +894,14 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
       // Single layer: warp w takes entries 16 w .. 16 w + 15; pair mode (16 entries per layer):
       // warp 0 layer l-1, warp 2 layer l.
       for (int x = 0; x < xv && ok; ++x, ++it) {
-        const int s = it % kStages;
-        if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1, s_abort, p.status)) { ok = false; break; }
+        const int s = it % N_STAGES;
+        if (!mbar_wait(full0 + 8 * s, (it / N_STAGES) & 1, s_abort, p.status)) { ok = false; break; }
         const int cnt = info_s[2 * s];
         const int set = nslots == 2 ? (warp >> 1) : 0;
         const int e_w = nslots == 2 ? (warp & 1) * 16 : warp * 16;
         bool wrote = false;
         if (e_w < cnt) {
-          const unsigned char* sb = stages + s * kStageBytes + set * set_bytes;
+          const unsigned char* sb = stages + s * STAGE_BYTES + set * set_bytes;
           const uint32_t sba = smem_u32(sb);
           if (cnt < e_w + 16) {  // entries past the last one: zero
             for (int i = lane; i < (e_w + 16 - cnt) * 16; i += 32) {
@@ -1124,8 +1138,8 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static size_t attn_smem_bytes() {
-  size_t b = 128 + (size_t)kStages * kStageBytes + (size_t)kScoreFloats * 4;  // stages, S
+static size_t attn_smem_bytes(bool q4) {
+  size_t b = 128 + (q4 ? (size_t)kQ4Stages * kQ4StageBytes : (size_t)kStages * kStageBytes) + (size_t)kScoreFloats * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                  // q_s
   b += kMaxRows * 4 + 3 * kMaxRows * kConsumerWarps * 4;                       // m, l, red, red2
   b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 2 * kMaxPiecePages * 4 + 4 + 8 + 2 * kStages * 8 + 64;
@@ -1185,7 +1199,7 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const int grid = n_teams * ap.team_size;
   ap.n_teams = n_teams;
   if (n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
-  const size_t smem = attn_smem_bytes();
+  const size_t smem = attn_smem_bytes(q4);
   // many output rows: a warp per row; few: a block per row
   const bool warp_rows = (long long)ap.n_sets * bt->batch * cfg->n_q_heads >= 1024;
   dim3 cgrid(warp_rows ? (cfg->n_q_heads + kCombineWarps - 1) / kCombineWarps : cfg->n_q_heads, bt->batch, ap.n_sets);

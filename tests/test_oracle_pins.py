@@ -583,3 +583,82 @@ def test_q4_cache_restore_keeps_the_magnitudes():
             assert np.allclose(np.linalg.norm(x4, axis=1), m["n_l"][0, :80, h], rtol=1e-12)
             cos = np.sum(x16 * x4, 1) / (np.linalg.norm(x16, axis=1) * np.linalg.norm(x4, axis=1))
             assert np.all(cos > 0.97) and np.all(cos[64:] > 1 - 1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# Variants the paper points at: dynamic t (Sec. 5, ablation of t), one retention set for K and V
+# ---------------------------------------------------------------------------------------------
+def _angle(x, y):
+    """Angle between two vectors by the atan2 formula (no arccos)."""
+    x, y = x / np.linalg.norm(x), y / np.linalg.norm(y)
+    return 2.0 * math.atan2(np.linalg.norm(x - y), np.linalg.norm(x + y))
+
+
+def test_dynamic_t_is_the_relative_magnitude_ratio():
+    assert orc.dynamic_t(1.0, 1.0) == 0.5
+    assert orc.dynamic_t(1.0, 3.0) == 0.75 and orc.dynamic_t(3.0, 1.0) == 0.25
+    assert orc.dynamic_t(0.0, 0.0) == 0.5 and orc.dynamic_t(0.0, 2.0) == 1.0
+    rs = np.random.RandomState(3)
+    na, nc = rs.rand(100) + 0.1, rs.rand(100) + 0.1
+    t = orc.dynamic_t(na, nc)
+    assert np.all((t > 0) & (t < 1)) and np.allclose(t + orc.dynamic_t(nc, na), 1.0)
+
+
+def test_dynamic_t_splits_the_angle_by_the_magnitudes():
+    """With t = |c| / (|a| + |c|) the merged direction sits at t * Omega from layer l-1's direction: three
+    times closer to the row that is three times longer; equal lengths give the geodesic midpoint."""
+    rs = np.random.RandomState(4)
+    u = rs.randn(128)
+    u /= np.linalg.norm(u)
+    g = rs.randn(128)
+    g -= (g @ u) * u
+    g /= np.linalg.norm(g)
+    for omega, la, lc in ((0.5, 1.0, 3.0), (1.3, 2.0, 2.0), (2.0, 5.0, 1.0)):
+        a = la * u
+        c = lc * (math.cos(omega) * u + math.sin(omega) * g)
+        m = orc.merge_rows(a[None], c[None], "ratio")
+        t = lc / (la + lc)
+        assert abs(np.linalg.norm(m["e"][0]) - 1.0) < 1e-12
+        assert abs(_angle(m["e"][0], a) - t * omega) < 1e-9 and abs(_angle(m["e"][0], c) - (1 - t) * omega) < 1e-9
+        # the same number as Eq. 3 with that t given explicitly, and per-row arrays of t are honoured
+        assert np.allclose(m["e"], orc.merge_rows(a[None], c[None], t)["e"], atol=1e-15)
+    rows_a = np.stack([1.0 * u, 2.0 * u])
+    rows_c = np.stack([3.0 * g, 2.0 * g])
+    m = orc.merge_rows(rows_a, rows_c, "ratio")  # orthogonal rows: e = cos(t pi/2) u + sin(t pi/2) g
+    for i, t in enumerate((0.75, 0.5)):
+        assert np.allclose(m["e"][i], math.cos(t * math.pi / 2) * u + math.sin(t * math.pi / 2) * g, atol=1e-12)
+    # a fixed t is unchanged by the array handling
+    assert np.array_equal(orc.merge_rows(rows_a, rows_c, 0.6)["e"], orc.merge_rows(rows_a, rows_c, np.array([0.6, 0.6]))["e"])
+
+
+def test_dynamic_t_through_the_pair_merge_and_restore():
+    import gen
+    wl = gen.CONFIGS["c1"].scaled("dyn", n_kv_heads=2, n_q_heads=2, batch=1, seq_len=40, index=61)
+    t = gen.make_pair_tensors(wl, 0)
+    bits = {k: gen.as_bits(v) for k, v in t.items()}
+    m = orc.merge_pair(bits["k_lm1"], bits["k_l"], [40], "f16", "ratio", 0.05)
+    a, c = orc.decode_bits(bits["k_lm1"], "f16"), orc.decode_bits(bits["k_l"], "f16")
+    tt = m["n_l"] / (m["n_lm1"] + m["n_l"])
+    for i in (0, 7, 39):
+        for h in (0, 1):
+            om = _angle(a[0, i, h], c[0, i, h])
+            assert abs(_angle(m["e"][0, i, h], a[0, i, h]) - tt[0, i, h] * om) < 1e-9
+    # restore keeps both magnitudes whatever t was
+    x = orc.restore(m["e_bits"][0, :, 0], m["n_l"][0, :, 0], "f16")
+    assert np.allclose(np.linalg.norm(x, axis=-1), m["n_l"][0, :, 0], rtol=1e-12)
+
+
+def test_retention_union_brute_force():
+    rs = np.random.RandomState(9)
+    dk, dv = rs.rand(3, 50), rs.rand(3, 50)
+    rk = {(b, 0): orc.retention_indices(dk[b], 0.2) for b in range(3)}
+    rv = {(b, 0): orc.retention_indices(dv[b], 0.2) for b in range(3)}
+    un = orc.retention_union(rk, rv)
+    for b in range(3):
+        want = sorted(i for i in range(50) if i in set(rk[(b, 0)].tolist()) or i in set(rv[(b, 0)].tolist()))
+        assert un[(b, 0)].tolist() == want
+        assert set(rk[(b, 0)].tolist()) <= set(want) and set(rv[(b, 0)].tolist()) <= set(want)
+    # nothing kept for the values: the union is the keys' set; same sets: unchanged
+    empty = {k: np.zeros(0, np.int64) for k in rk}
+    assert all(np.array_equal(orc.retention_union(rk, empty)[k], rk[k]) for k in rk)
+    assert all(np.array_equal(orc.retention_union(rk, rk)[k], rk[k]) for k in rk)
