@@ -94,13 +94,15 @@ class ClockSampler:
 class Job:
     """All device state of one rank's workload."""
 
-    def __init__(self, wl: gen.WorkloadConfig, device, q4: bool = False, q4cache: bool = False):
+    def __init__(self, wl: gen.WorkloadConfig, device, q4: bool = False, q4cache: bool = False, serving: bool = False):
         import paper_2405_14366_b200 as mc
         self.mc, self.lib, self.wl, self.dev, self.q4 = mc, mc.lib(), wl, device, q4
         self.q4cache = q4cache  # the shared cache itself is 4-bit (pages of 32 tokens)
         self.B, self.S, self.H, self.Hq, self.ps = wl.batch, wl.seq_len, wl.n_kv_heads, wl.n_q_heads, wl.page_size
         self.steps = wl.decode_steps
         prompt, gen_len = gen.make_lengths(wl)
+        if serving:  # slots that are refilled: every slot gets pages for the longest prompt and the longest generation
+            prompt = np.full(wl.batch, wl.seq_len, prompt.dtype)
         self.prompt = prompt
         # the serving mix drains: a sequence leaves the batch after its own number of generated tokens
         # (its length is set to 0: an empty sequence costs one empty work unit per head and nothing else)
@@ -117,9 +119,12 @@ class Job:
         self.tok_heads = int(prompt.sum()) * self.H  # (token, kv head) rows per layer and tensor
         self.pools, self.pairs = [], []
         cap_rows = int(0.10 * 2 * self.tok_heads) + 1024
+        if serving:  # one region of the retained pool per slot
+            self.rows_per_seq = int(0.10 * 2 * wl.seq_len * self.H) + 64
+            cap_rows = self.B * self.rows_per_seq
         for pr in range(wl.n_pairs):
             t = gen.make_pair_tensors(wl, pr, device=device)
-            if wl.ragged:
+            if wl.ragged and not serving:
                 for b in range(self.B):
                     for v in t.values():
                         v[b, prompt[b]:] = 0
@@ -400,6 +405,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--q4", action="store_true", help="the layers arrive in 4 bits (page size 32; no host-buffer leg)")
     ap.add_argument("--q4cache", action="store_true", help="the shared cache is 4-bit (page size 32): restore and attention read codes")
+    ap.add_argument("--refill", action="store_true",
+                    help="serving trace: a seeded list of 4 x batch sequences, a slot is refilled when its sequence leaves, "
+                         "the admitted sequence is merged on a second stream while the others decode")
     args = ap.parse_args()
     wl = gen.CONFIGS[args.workload]
     if args.decode_steps is not None:
@@ -427,6 +435,9 @@ def main():
     if dist is not None:
         dist.barrier()
 
+    if args.refill:
+        run_refill(args, wl, dev, rank, world, dist)
+        return
     job = Job(wl, dev, q4=args.q4, q4cache=args.q4cache)
     if args.q4:
         args.no_e2e = True  # the host-buffer entry points take 16-bit layers only
@@ -544,6 +555,160 @@ def main():
                 "kv_tokens_per_s": {"merge": phases["merge"]["kv_tokens_per_s"], "decode": phases["decode"]["kv_tokens_per_s"]},
                 "phases": phases, "bytes_per_step": by, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches, "clocks": clocks}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_refill(args, wl, dev, rank, world, dist):
+    """The serving mix with slot refill (the paper's efficiency experiment, Sec. 5, gets its throughput from
+    the live batch): 4 x batch sequences with seeded prompt and generation lengths wait in a list; the
+    batch's slots start with the first ones; every decode step attends both layers of every pair for every
+    live slot and appends the new token; a slot whose sequence has generated its share is handed the next
+    sequence of the list, whose pairs are merged by mc_admit_sequences on a second stream while the decode
+    steps go on, and joins the batch (its length becomes visible to the decode calls) once that merge has run.
+    The decode step is replayed from a CUDA graph; the host never waits for the device inside the loop."""
+    n_list = 4 * wl.batch
+    prompts, gens = gen.make_lengths(dataclasses.replace(wl, batch=n_list))
+    job = Job(wl, dev, q4=args.q4, q4cache=args.q4cache, serving=True)
+    lib, B, H = job.lib, job.B, job.H
+    max_len = wl.seq_len + wl.decode_steps + 1
+    bd = job.mc.Batch(job.block_table, job.seq_lens, max_len, job.n_pages)
+    adm_lens = torch.zeros(B, dtype=torch.int32, device=dev)
+    badm = job.mc.Batch(job.block_table, adm_lens, wl.seq_len, job.n_pages)
+    ws1 = lib.mc_workspace_bytes(job.cfg, badm, 0, 1)
+    ws16 = lib.mc_workspace_bytes(dataclasses.replace(job.cfg, cache_bits=16), badm, 0, 1)
+    # per pair the retention tables; the 16-bit staging tiles of a 4-bit cache once (the pairs take turns)
+    ws_adm = torch.empty(wl.n_pairs * ws16 + (ws1 - ws16), dtype=torch.uint8, device=dev)
+    main_s, side_s = torch.cuda.current_stream(), torch.cuda.Stream()
+    remaining = torch.zeros(B, dtype=torch.int32, device=dev)  # tokens each slot's sequence has still to generate
+
+    def admit(slots, seqs, stream):
+        """Merge sequence seqs[i] into slot slots[i] (a run of neighbouring slots) on `stream`."""
+        with torch.cuda.stream(stream):
+            adm_lens[slots[0]:slots[0] + len(slots)] = torch.from_numpy(prompts[seqs].astype(np.int32)).to(dev, non_blocking=True)
+            lib.mc_admit_sequences(job.cfg, badm, slots[0], len(slots), job.pools, job.pairs, job.rows_per_seq, True, ws_adm,
+                                   stream=stream, q4=args.q4)
+
+    def decode_step():
+        q, nt = job.q[0], job.new[0]
+        for pr in range(wl.n_pairs):
+            pc = job.pairs[pr]
+            for layer in (0, 1):
+                lib.mc_decode_attn(job.cfg, bd, pc, layer, q[layer], nt["k_lm1" if layer == 0 else "k_l"],
+                                   nt["v_lm1" if layer == 0 else "v_l"], job.sm_scale, job.out, None, job.ws_attn)
+            lib.mc_append_pair(job.cfg, bd, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
+        # end of the step, on the device: live slots grow by one token; a slot that has generated its share empties
+        live = (remaining > 0).to(torch.int32)
+        job.seq_lens.add_(live)
+        remaining.sub_(live)
+        job.seq_lens.mul_((remaining > 0).to(torch.int32))
+
+    def serve(max_steps):
+        """Returns (steps, generated tokens, sum over steps of live (token, head) rows, steps at full batch, residual rows)."""
+        job.seq_lens.zero_()
+        remaining.zero_()
+        side_s.wait_stream(main_s)
+        admit(list(range(B)), np.arange(B), main_s)
+        job.seq_lens.copy_(adm_lens)
+        remaining.copy_(torch.from_numpy(gens[:B].astype(np.int32)).to(dev))
+        h_len = prompts[:B].astype(np.int64).copy()      # host mirror of the slots
+        h_rem = gens[:B].astype(np.int64).copy()
+        nxt, pending = B, []                              # next sequence of the list; admissions in flight
+        steps = tokens = th_sum = full = th_res = 0
+        while steps < max_steps and (h_rem.max() > 0 or pending):
+            # admissions that have run join the batch
+            still = []
+            for slot, j, ev in pending:
+                if ev.query():
+                    main_s.wait_event(ev)
+                    job.seq_lens[slot:slot + 1].fill_(int(prompts[j]))
+                    remaining[slot:slot + 1].fill_(int(gens[j]))
+                    h_len[slot], h_rem[slot] = prompts[j], gens[j]
+                else:
+                    still.append((slot, j, ev))
+            pending = still
+            livem = h_rem > 0
+            if livem.any():
+                graph.replay()
+                steps += 1
+                tokens += int(livem.sum())
+                th_sum += int(h_len[livem].sum()) * H
+                th_res += int((h_len[livem] % 32).sum()) * H
+                full += int(livem.all())
+                h_len[livem] += 1
+                h_rem[livem] -= 1
+                done = livem & (h_rem == 0)
+                h_len[done] = 0
+                if done.any() and nxt < n_list:
+                    ev_step = torch.cuda.Event()
+                    ev_step.record(main_s)
+                    for slot in np.nonzero(done)[0]:
+                        if nxt >= n_list:
+                            break
+                        side_s.wait_event(ev_step)  # the slot's last decode step has run
+                        admit([int(slot)], np.array([nxt]), side_s)
+                        ev = torch.cuda.Event()
+                        ev.record(side_s)
+                        pending.append((int(slot), nxt, ev))
+                        nxt += 1
+            else:
+                pending[0][2].synchronize()  # nothing to decode until an admission lands
+        main_s.wait_stream(side_s)
+        return steps, tokens, th_sum, full, th_res, nxt
+
+    # warm-up: set-up calls outside capture, then the decode step as a graph
+    admit(list(range(B)), np.arange(B), main_s)
+    job.seq_lens.copy_(adm_lens)
+    remaining.fill_(4)
+    side = torch.cuda.Stream()
+    side.wait_stream(main_s)
+    with torch.cuda.stream(side):
+        decode_step()
+    main_s.wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        decode_step()
+    torch.cuda.synchronize()
+    max_steps = args.decode_steps if args.decode_steps is not None else 10 ** 9
+    serve(min(max_steps, 32))
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if dist is not None:
+        dist.barrier()
+    res = []
+    t = timed(lambda: res.append(serve(max_steps)))
+    t = max_over_ranks(t, dist, dev)
+    clocks = sampler.stop() if sampler else None
+    steps, tokens, th_sum, full, th_res, admitted = res[0]
+    for pc in job.pairs:
+        words, code = lib.mc_read_status(pc, check=False)
+        if code != 0:
+            raise SystemExit(f"device status {words} after the serving trace")
+    rho = 0.004  # retained fraction of this workload's recipe (measured by the drained runs)
+    attn_bytes = wl.n_pairs * 2 * job.attn_row_bytes(th_sum, th_res, rho)
+    append_bytes = wl.n_pairs * 2 * tokens * H * (3 * ROW + 12 + ((ROW + 80) if args.q4cache else 0))
+    in_row = 64 + 16 if args.q4 else ROW
+    e_row = 64 + 16 if args.q4cache else ROW
+    adm_th = int(prompts[:admitted].sum()) * H
+    merge_bytes = wl.n_pairs * 2 * adm_th * (2 * in_row + e_row + 16)
+    value = world * (attn_bytes + append_bytes + merge_bytes) / t / 1e9
+    peak, peak_src = measured_hbm_peak()
+    if rank == 0:
+        line = {"metric": "hbm_gbps_merge_restore_decode_attn", "value": value, "unit": "GB/s", "n_gpus": world, "steps": 1,
+                "warmup": 1, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": wl.name + " serving trace with slot refill", "slots": B, "sequences_in_list": n_list,
+                           "sequences_admitted": admitted, "kv_heads": H, "storage": wl.dtype,
+                           "shared_cache": "4-bit" if args.q4cache else wl.dtype,
+                           "input_layers": "4-bit" if args.q4 else wl.dtype, "page_size": wl.page_size, "pairs": wl.n_pairs},
+                "serving": {"decode_steps": steps, "generated_tokens": world * tokens, "served_tokens_per_s": world * tokens / t,
+                            "ms_per_decode_step": t * 1e3 / max(steps, 1), "mean_live_slots": tokens / max(steps, 1),
+                            "fraction_of_steps_at_full_batch": full / max(steps, 1),
+                            "decode_GB/s": world * (attn_bytes + append_bytes) / t / 1e9,
+                            "frac_of_measured_hbm": value / world / peak, "admission_merge_bytes": merge_bytes},
+                "gpu_launches": steps * wl.n_pairs * 5 + (admitted - B + 1) * 4, "clocks": clocks}
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

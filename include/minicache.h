@@ -89,6 +89,13 @@ typedef enum { MC_OP_MERGE = 0, MC_OP_DECODE_ATTN = 1 } mc_op;
  * t is used by MC_MERGE_SLERP only. */
 typedef enum mc_merge_fn { MC_MERGE_SLERP = 0, MC_MERGE_FMAX = 1, MC_MERGE_MEAN = 2 } mc_merge_fn;
 
+/* Where the interpolation parameter of Eq. 3 comes from.  MC_T_FIXED: cfg->t for every token (the paper's
+ * setting, t = 0.6).  MC_T_MAGNITUDE_RATIO: per token t_i = |x^l_i| / (|x^{l-1}_i| + |x^l_i|) -- Sec. 5's
+ * ablation of t observes that the best t follows the relative magnitude ratio of adjacent layers and
+ * suggests determining t from it; the formula is our reading (the longer row pulls the direction its
+ * way, equal lengths give the geodesic midpoint).  cfg->t is then ignored. */
+typedef enum mc_t_mode { MC_T_FIXED = 0, MC_T_MAGNITUDE_RATIO = 1 } mc_t_mode;
+
 /* Status word indices (mc_read_status). */
 enum {
   MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out;
@@ -127,6 +134,11 @@ typedef struct mc_config {
   int32_t merge_fn;    /* mc_merge_fn: how the two rows of a token become the shared row */
   int32_t cache_bits;  /* storage of the shared directions E: 0 or 16 = the 16-bit type `dtype`; 4 = the 4-bit
                           shared cache described at mc_pair_cache (page_size must then be 32) */
+  int32_t t_mode;      /* mc_t_mode: where Eq. 3's t comes from */
+  int32_t retain_union; /* 0: Eq. 4 applied to keys and values separately (Algorithm 2 computes I_k and I_v);
+                           1: one set per (sequence, head), the union of the two (Sec. 4.2 writes the pair cache
+                           with a single I): a token either rule keeps is kept unmerged in both tensors.
+                           Not with MC_RETAIN_TOPK. */
 } mc_config;
 
 /* Batch geometry shared by the layer pools and the pair cache. */
@@ -332,6 +344,29 @@ mc_status mc_merge_pairs(const mc_config* cfg, const mc_batch* batch, int32_t n_
                          const mc_layer_kv* const* lm1, const mc_layer_kv* const* l,
                          const mc_pair_cache* const* out, int32_t do_retention, void* workspace,
                          size_t workspace_bytes, void* stream);
+
+/* Admission of new sequences into a running batch (Algorithm 1's prefill branch for sequences that arrive
+ * while others decode; the paper's serving experiment, Sec. 5, gets its throughput from the larger live
+ * batch): Algorithm 2 "MiniCache Prefill" for the sequences [seq_begin, seq_begin + seq_count) of the batch
+ * only, for n_pairs layer pairs in one launch sequence.  The other sequences' tiles, tables and retained
+ * entries are not touched, so the call may run on a second stream while decode steps attend them -- as
+ * long as the admitted sequences' seq_lens entries read 0 for those decode calls (give this call a
+ * mc_batch whose seq_lens holds the new lengths, and copy them into the decode batch's seq_lens once this
+ * call has run).
+ * lm1 / l            16-bit layers per pair, or both NULL with q4_lm1 / q4_l given (4-bit layers, page 32)
+ * rows_per_seq       the retained pool is used as one region per sequence: sequence b owns the entries
+ *                    [b * rows_per_seq, (b + 1) * rows_per_seq) (batch->batch * rows_per_seq <= ret_capacity).
+ *                    A sequence whose retention needs more keeps nothing and MC_FLAG_RETAIN_OVERFLOW is set.
+ *                    A pair cache filled this way must be filled this way for all its sequences (never mix
+ *                    with mc_merge_pair, whose retained lists are one compact run for the whole batch).
+ * Status words are not cleared (flags accumulate); MC_STATUS_RETAINED_TOTAL / NEAR_THRESHOLD are not kept.
+ * workspace          n_pairs * mc_workspace_bytes(MC_OP_MERGE) bytes (with cfg->cache_bits = 4: the part
+ *                    without the staging tiles per pair, plus the staging tiles once), 256-byte aligned. */
+mc_status mc_admit_sequences(const mc_config* cfg, const mc_batch* batch, int32_t seq_begin, int32_t seq_count,
+                             int32_t n_pairs, const mc_layer_kv* const* lm1, const mc_layer_kv* const* l,
+                             const mc_layer_q4* const* q4_lm1, const mc_layer_q4* const* q4_l,
+                             const mc_pair_cache* const* out, int64_t rows_per_seq, int32_t do_retention,
+                             void* workspace, size_t workspace_bytes, void* stream);
 
 /* mc_merge_pair for layers stored in 4 bits: the rows are de-quantised inside the merge kernel
  * (code * scale + zero in fp32) and merged exactly as in mc_merge_pair; the pair cache it writes is

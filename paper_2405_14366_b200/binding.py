@@ -35,7 +35,8 @@ class McError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("page_size", C.c_int32), ("dtype", C.c_int32), ("retain_mode", C.c_int32),
-                ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("cache_bits", C.c_int32)]
+                ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("cache_bits", C.c_int32),
+                ("t_mode", C.c_int32), ("retain_union", C.c_int32)]
 
 
 class _Batch(C.Structure):
@@ -74,7 +75,7 @@ class _Stats(C.Structure):
                 ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
 
 
-EXPORTS = ("mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+EXPORTS = ("mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -101,11 +102,13 @@ class McConfig:
     head_dim: int = 128
     merge_fn: int = 0  # MC_MERGE_SLERP (Eq. 3) | MC_MERGE_FMAX = 1 | MC_MERGE_MEAN = 2
     cache_bits: int = 16  # storage of the shared directions: 16 (the 16-bit type) or 4 (4-bit shared cache, pages of 32)
+    t_mode: int = 0  # MC_T_FIXED | MC_T_MAGNITUDE_RATIO = 1 (per-token t from the two magnitudes)
+    retain_union: int = 0  # 1: one retention set for keys and values (the union of Eq. 4's two sets)
 
     def c(self) -> _Config:
         return _Config(self.n_kv_heads, self.n_q_heads, self.head_dim, self.page_size,
                        {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma),
-                       int(self.merge_fn), int(self.cache_bits))
+                       int(self.merge_fn), int(self.cache_bits), int(self.t_mode), int(self.retain_union))
 
     @property
     def torch_dtype(self):
@@ -289,6 +292,9 @@ class MiniCacheLib:
         L.mc_merge_pairs.argtypes = [P(_Config), P(_Batch), C.c_int32, P(P(_LayerKV)), P(P(_LayerKV)), P(P(_PairCache)),
                                      C.c_int32, V, C.c_size_t, V]
         L.mc_merge_pairs.restype = C.c_int32
+        L.mc_admit_sequences.argtypes = [P(_Config), P(_Batch), C.c_int32, C.c_int32, C.c_int32, P(P(_LayerKV)), P(P(_LayerKV)),
+                                         P(P(_LayerQ4)), P(P(_LayerQ4)), P(P(_PairCache)), C.c_int64, C.c_int32, V, C.c_size_t, V]
+        L.mc_admit_sequences.restype = C.c_int32
         L.mc_append_pair.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, V, V, V, V]
         L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), C.c_int32, V]
         L.mc_pair_bytes.argtypes = [P(_Config), P(_Batch), C.c_int64, P(_PairSizes)]
@@ -361,6 +367,26 @@ class MiniCacheLib:
         self._check(self._lib.mc_merge_pairs(C.byref(c), C.byref(b), n, arr(a, _LayerKV), arr(l, _LayerKV),
                                              arr(pcs, _PairCache), 1 if do_retention else 0, _ptr(workspace),
                                              workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_admit_sequences(self, cfg: McConfig, batch: Batch, seq_begin: int, seq_count: int, layers, pairs, rows_per_seq: int,
+                           do_retention: bool, workspace: torch.Tensor, stream=None, q4: bool = False):
+        """layers: per pair a dict with k_lm1, v_lm1, k_l, v_l pools, or (q4) with "_lm1" / "_l" dicts of
+        k_codes, k_meta, v_codes, v_meta; pairs: the PairCache of each pair."""
+        n = len(pairs)
+        c, b = cfg.c(), batch.c()
+        pcs = [pc.c() for pc in pairs]
+        arr = lambda items, T: (C.POINTER(T) * n)(*[C.pointer(x) for x in items])
+        if q4:
+            mk = lambda d: _LayerQ4(_ptr(d["k_codes"]), _ptr(d["k_meta"]), _ptr(d["v_codes"]), _ptr(d["v_meta"]))
+            a, l = [mk(x["_lm1"]) for x in layers], [mk(x["_l"]) for x in layers]
+            args = (None, None, arr(a, _LayerQ4), arr(l, _LayerQ4))
+        else:
+            a = [_LayerKV(_ptr(x["k_lm1"]), _ptr(x["v_lm1"])) for x in layers]
+            l = [_LayerKV(_ptr(x["k_l"]), _ptr(x["v_l"])) for x in layers]
+            args = (arr(a, _LayerKV), arr(l, _LayerKV), None, None)
+        self._check(self._lib.mc_admit_sequences(C.byref(c), C.byref(b), int(seq_begin), int(seq_count), n, *args,
+                                                 arr(pcs, _PairCache), int(rows_per_seq), 1 if do_retention else 0,
+                                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
     def mc_merge_pair_q4(self, cfg: McConfig, batch: Batch, q_lm1, q_l, pair: PairCache, do_retention: bool,
                          workspace: torch.Tensor, stream=None):

@@ -56,6 +56,9 @@ static mc_status check_config(const mc_config* cfg) {
   if (cfg->merge_fn < MC_MERGE_SLERP || cfg->merge_fn > MC_MERGE_MEAN) return MC_ERR_INVALID_ARG;
   if (cfg->cache_bits != 0 && cfg->cache_bits != 16 && cfg->cache_bits != 4) return MC_ERR_INVALID_ARG;
   if (cfg->cache_bits == 4 && cfg->page_size != kQ4Page) return MC_ERR_SHAPE;
+  if (cfg->t_mode != MC_T_FIXED && cfg->t_mode != MC_T_MAGNITUDE_RATIO) return MC_ERR_INVALID_ARG;
+  if (cfg->retain_union != 0 && cfg->retain_union != 1) return MC_ERR_INVALID_ARG;
+  if (cfg->retain_union && cfg->retain_mode == MC_RETAIN_TOPK) return MC_ERR_UNSUPPORTED;
   if (!(cfg->t >= 0.0 && cfg->t <= 1.0) || !(cfg->gamma >= 0.0 && cfg->gamma <= 1.0)) return MC_ERR_INVALID_ARG;
   return MC_OK;
 }
@@ -97,6 +100,8 @@ static Geom make_geom(const mc_config* cfg, const mc_batch* bt) {
   g.page_shift = cfg->page_size == 16 ? 4 : (cfg->page_size == 32 ? 5 : 6);
   g.max_seq_len = bt->max_seq_len;
   g.n_pages = (int)bt->n_pages;
+  g.seq_begin = 0;
+  g.seq_count = bt->batch;
   return g;
 }
 
@@ -309,6 +314,77 @@ mc_status mc_merge_pairs(const mc_config* cfg, const mc_batch* batch, int32_t n_
     const int n = n_pairs - i0 < kMergePairsPerLaunch ? n_pairs - i0 : kMergePairsPerLaunch;
     st = launch_merge_pairs(cfg, batch, g, n, lm1 + i0, l + i0, nullptr, nullptr, out + i0, do_retention ? 1 : 0,
                             (char*)workspace + (size_t)i0 * ws_pair, (cudaStream_t)stream);
+    if (st != MC_OK) return st;
+  }
+  return MC_OK;
+}
+
+mc_status mc_admit_sequences(const mc_config* cfg, const mc_batch* batch, int32_t seq_begin, int32_t seq_count, int32_t n_pairs,
+                             const mc_layer_kv* const* lm1, const mc_layer_kv* const* l, const mc_layer_q4* const* q4_lm1,
+                             const mc_layer_q4* const* q4_l, const mc_pair_cache* const* out, int64_t rows_per_seq,
+                             int32_t do_retention, void* workspace, size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_admit_sequences");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  const bool q4 = q4_lm1 != nullptr;
+  if (n_pairs < 0 || !out || (q4 ? (!q4_l || lm1 || l) : (!lm1 || !l || q4_l))) return MC_ERR_INVALID_ARG;
+  if (seq_begin < 0 || seq_count < 0 || seq_begin + (int64_t)seq_count > batch->batch) return MC_ERR_INVALID_ARG;
+  if (rows_per_seq <= 0 || rows_per_seq > 0x7fffffff / (batch->batch > 0 ? batch->batch : 1)) return MC_ERR_INVALID_ARG;
+  if (q4 && cfg->page_size != kQ4Page) return MC_ERR_SHAPE;
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  const size_t ws_pair = merge_workspace_bytes(cfg, batch);
+  const size_t ws_stage = cfg->cache_bits == 4 ? 2 * q4_stage_bytes(cfg, batch) : 0;
+  if (workspace_bytes < (size_t)n_pairs * ws_pair + ws_stage) return MC_ERR_CAPACITY;
+  for (int i = 0; i < n_pairs; ++i) {
+    const void* ptrs[8];
+    if (q4) {
+      if (!q4_lm1[i] || !q4_l[i]) return MC_ERR_INVALID_ARG;
+      const void* pp[8] = {q4_lm1[i]->k_codes, q4_lm1[i]->k_meta, q4_lm1[i]->v_codes, q4_lm1[i]->v_meta,
+                           q4_l[i]->k_codes,   q4_l[i]->k_meta,   q4_l[i]->v_codes,   q4_l[i]->v_meta};
+      memcpy(ptrs, pp, sizeof(pp));
+    } else {
+      if (!lm1[i] || !l[i]) return MC_ERR_INVALID_ARG;
+      const void* pp[8] = {lm1[i]->k_pool, lm1[i]->v_pool, l[i]->k_pool, l[i]->v_pool, lm1[i]->k_pool, lm1[i]->v_pool, l[i]->k_pool, l[i]->v_pool};
+      memcpy(ptrs, pp, sizeof(pp));
+    }
+    for (const void* q : ptrs) {
+      if (q == nullptr) return MC_ERR_INVALID_ARG;
+      if (!aligned256(q)) return MC_ERR_ALIGN;
+    }
+    st = check_merge_common(cfg, batch, out[i], workspace, ws_pair + ws_stage);
+    if (st != MC_OK) return st;
+    if ((int64_t)batch->batch * rows_per_seq > out[i]->ret_capacity) return MC_ERR_CAPACITY;
+    for (int j = 0; j < i; ++j)
+      if (out[j] == out[i] || out[j]->status == out[i]->status) return MC_ERR_INVALID_ARG;
+  }
+  Geom g = make_geom(cfg, batch);
+  g.seq_begin = seq_begin;
+  g.seq_count = seq_count;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cfg->cache_bits == 4) {
+    // one pair after the other through the one staging area: merge into 16-bit tiles, then quantise
+    char* stage = (char*)workspace + (size_t)n_pairs * ws_pair;
+    for (int i = 0; i < n_pairs; ++i) {
+      mc_pair_cache stg = *out[i];
+      stg.e_k = stage;
+      stg.e_v = stage + q4_stage_bytes(cfg, batch);
+      const mc_pair_cache* sp = &stg;
+      st = launch_merge_pairs(cfg, batch, g, 1, q4 ? nullptr : lm1 + i, q4 ? nullptr : l + i, q4 ? q4_lm1 + i : nullptr,
+                              q4 ? q4_l + i : nullptr, &sp, do_retention ? 1 : 0, (char*)workspace + (size_t)i * ws_pair, s,
+                              (int)rows_per_seq);
+      if (st != MC_OK) return st;
+      st = launch_q4_quantise(cfg, batch, g, stg.e_k, stg.e_v, out[i], s);
+      if (st != MC_OK) return st;
+    }
+    return MC_OK;
+  }
+  for (int i0 = 0; i0 < n_pairs; i0 += kMergePairsPerLaunch) {
+    const int n = n_pairs - i0 < kMergePairsPerLaunch ? n_pairs - i0 : kMergePairsPerLaunch;
+    st = launch_merge_pairs(cfg, batch, g, n, q4 ? nullptr : lm1 + i0, q4 ? nullptr : l + i0, q4 ? q4_lm1 + i0 : nullptr,
+                            q4 ? q4_l + i0 : nullptr, out + i0, do_retention ? 1 : 0, (char*)workspace + (size_t)i0 * ws_pair, s,
+                            (int)rows_per_seq);
     if (st != MC_OK) return st;
   }
   return MC_OK;

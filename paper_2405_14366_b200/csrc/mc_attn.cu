@@ -237,7 +237,8 @@ struct RawRanges {
 __device__ __forceinline__ RawRanges load_ranges(const Item& w, const AttnParams& p) {
   RawRanges r;
   r.off_k = r.off_v = r.k0 = r.k1 = r.v0 = r.v1 = 0;
-  if (!w.valid) return r;
+  // (an empty sequence has no retained tokens; its tables may be being rewritten by an admission)
+  if (!w.valid || w.n_tok == 0) return r;
   const int H = p.g.n_kv_heads;
   const int seg_k = w.b * H + w.g, seg_v = (p.g.batch + w.b) * H + w.g;
   const int pj0 = min(w.split_start >> 7, p.ret_prefix_stride - 1);

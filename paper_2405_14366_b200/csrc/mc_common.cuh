@@ -62,6 +62,9 @@ struct Geom {
   int page_shift;  // log2(page_size)
   int max_seq_len;  // the caller's bound of seq_lens: longer lengths are clamped to it and flagged
   int n_pages;      // pages in every pool: page ids outside [0, n_pages) are never used as addresses
+  // the sequences a merge works on: all of them, or (admission of new sequences into free slots) a
+  // range; the others count as empty for that call
+  int seq_begin, seq_count;
 };
 
 #if defined(__CUDACC__)
@@ -70,6 +73,7 @@ struct Geom {
 // id outside the pools is replaced by page 0 for reads and skips the write, and either sets
 // MC_FLAG_BAD_METADATA in the pair's status words.
 __device__ __forceinline__ int checked_len(const Geom& g, int b, int32_t* status) {
+  if ((unsigned)(b - g.seq_begin) >= (unsigned)g.seq_count) return 0;  // not part of this call
   const int n = g.seq_lens[b];
   if (n < 0 || n > g.max_seq_len) {
     atomicOr(status, MC_FLAG_BAD_METADATA);
@@ -240,9 +244,19 @@ __device__ __forceinline__ RowScalars slerp_scalars(float aa, float cc, float sm
 }
 
 #if defined(__CUDACC__)
+// Eq. 3's (1 - t, t) for one row: the configured pair, or (MC_T_MAGNITUDE_RATIO) t = |c| / (|a| + |c|)
+// from the two squared lengths; 0.5 if both rows are zero.
+__device__ __forceinline__ void row_t(int t_mode, float aa, float cc, float& ta, float& tc) {
+  if (t_mode == MC_T_MAGNITUDE_RATIO) {
+    const float na = aa > 0.f ? aa * rsqrtf(aa) : 0.f, nc = cc > 0.f ? cc * rsqrtf(cc) : 0.f;
+    tc = na + nc > 0.f ? __fdividef(nc, na + nc) : 0.5f;
+    ta = 1.0f - tc;
+  }
+}
+
 // One merged row: 16 lanes hold 8 channels each of a (layer l-1) and c (layer l).
 template <int DT>
-__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, int fn, uint4& e_out,
+__device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, float ta, float tc, int fn, int t_mode, uint4& e_out,
                                           float& g_a, float& g_c, float& d_out) {
   float a[8], c[8];
   {
@@ -280,6 +294,7 @@ __device__ __forceinline__ void merge_row(const uint4& ra, const uint4& rc, floa
   }
   sm = sum16(sm);
   sp = sum16(sp);
+  row_t(t_mode, aa, cc, ta, tc);
   RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
   if (fn != MC_MERGE_SLERP) {  // one vector for both layers: direction of the mean, one magnitude
     float m2 = 0.f;

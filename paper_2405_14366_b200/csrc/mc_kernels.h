@@ -14,10 +14,14 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
 // Up to kMergePairsPerLaunch pairs that share the batch geometry in one launch sequence (one persistent
 // merge grid over all pairs' rows, one retention pass each over all pairs' segments); the workspace
 // holds merge_workspace_bytes per pair, one after the other.
+// g.seq_begin / g.seq_count select the sequences the call works on.  region_rows > 0 (admission of new
+// sequences): sequence b's retained entries go to the entries [b * region_rows, (b + 1) * region_rows) of the
+// pool instead of one compact list for the batch, and the status words are not cleared.
 constexpr int kMergePairsPerLaunch = 8;
 mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geom& g, int n_pairs, const mc_layer_kv* const* lm1,
                              const mc_layer_kv* const* l, const mc_layer_q4* const* q_lm1, const mc_layer_q4* const* q_l,
-                             const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream);
+                             const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream,
+                             int region_rows = 0);
 mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                         const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
                         cudaStream_t stream);

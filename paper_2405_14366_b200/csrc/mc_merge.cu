@@ -42,6 +42,7 @@ struct MergeParams {
   int n_pairs;
   float ta, tc;
   int merge_fn;
+  int t_mode;
   int items_per_page;
 };
 
@@ -72,7 +73,7 @@ __device__ __forceinline__ float sum4(float v) {
 // a (layer l-1) and c (layer l), 32 channels each.  Arithmetic in fp32, two channels per
 // instruction (packed f32x2).  Every lane of the quad returns the row's scalars.
 template <int DT>
-__device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const float2 (&c)[16], float ta, float tc, int fn,
+__device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const float2 (&c)[16], float ta, float tc, int fn, int t_mode,
                                                uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
   float2 aa2 = make_float2(0.f, 0.f), cc2 = aa2, aa3 = aa2, cc3 = aa2;
 #pragma unroll
@@ -112,6 +113,7 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
     const float spx = sum4(sp2.x + sp2.y);
     if (sm > 3.5f) sp = spx;
   }
+  row_t(t_mode, aa, cc, ta, tc);
   RowScalars s = slerp_scalars(aa, cc, sm, fmaxf(sp, 0.f), ta, tc);
   if (fn != MC_MERGE_SLERP) {  // one vector for both layers: direction of the mean, one magnitude
     float2 m2 = make_float2(0.f, 0.f);
@@ -153,7 +155,7 @@ __device__ __forceinline__ void merge_row_core(const float2 (&a)[16], const floa
 // occupancy.  (Eight warps, not nine with a dedicated producer: two CTAs of nine warps do not fit
 // the register file of an SM sub-partition.)
 template <int DT>
-__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc, int fn,
+__device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4 (&rc)[4], float ta, float tc, int fn, int t_mode,
                                                uint4 (&e_out)[4], float& g_a, float& g_c, float& d_out) {
   float2 a[16], c[16];
 #pragma unroll
@@ -167,7 +169,7 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
     c[4 * i + 2] = Elem<DT>::unpack(rc[i].z);
     c[4 * i + 3] = Elem<DT>::unpack(rc[i].w);
   }
-  merge_row_core<DT>(a, c, ta, tc, fn, e_out, g_a, g_c, d_out);
+  merge_row_core<DT>(a, c, ta, tc, fn, t_mode, e_out, g_a, g_c, d_out);
 }
 
 // 32 consecutive 4-bit codes (16 bytes; channel 2i in the low nibble of byte i) to values
@@ -331,7 +333,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);  // the stage is in registers now
-      merge_row_quad<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, g_a, g_c, d);
+      merge_row_quad<DT>(va, vc, p.ta, p.tc, p.merge_fn, p.t_mode, e, g_a, g_c, d);
     } else {
       // lane k owns channels [32 k, 32 k + 32): 16 bytes of codes = the 16-byte chunks 4 k .. 4 k + 3 of the output row
       const unsigned char* sb = stages + s * kMergeStageBytes;
@@ -352,7 +354,7 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       for (int x = 0; x < 4; ++x) ci[x] = 4 * k + x;
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
-      merge_row_core<DT>(a, c, p.ta, p.tc, p.merge_fn, e, g_a, g_c, d);
+      merge_row_core<DT>(a, c, p.ta, p.tc, p.merge_fn, p.t_mode, e, g_a, g_c, d);
     }
     float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
@@ -437,6 +439,8 @@ struct RetainParams {
   int nseg;
   int mode;
   int do_retention;
+  int union_kv;  // one set for keys and values: a token the other tensor's rule keeps is kept here too
+  int region_rows;  // admission: entries of the retained pool each sequence owns (0: one compact list for the batch)
   double gamma;
 };
 
@@ -465,7 +469,7 @@ struct RetainPair {
 struct RetainBatch {
   Geom g;
   RetainPair pr[kMaxMergePairs];  // blockIdx.z selects the pair
-  int q4, dtype, chunks_per_seg, nseg, mode, do_retention;
+  int q4, dtype, chunks_per_seg, nseg, mode, do_retention, union_kv, region_rows;
   double gamma;
 };
 __device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int pair) {
@@ -500,25 +504,40 @@ __device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int p
   p.nseg = bp.nseg;
   p.mode = bp.mode;
   p.do_retention = bp.do_retention;
+  p.union_kv = bp.union_kv;
+  p.region_rows = bp.region_rows;
   p.gamma = bp.gamma;
   return p;
 }
 
+// Segment (tensor, b, h) number `ls` of the call's sequences [seq_begin, seq_begin + seq_count):
+// ls = (tensor * seq_count + (b - seq_begin)) * H + h; returns its index in the pair's tables.
+__device__ __forceinline__ int call_segment(const Geom& g, int ls, int& tensor, int& b, int& h) {
+  h = ls % g.n_kv_heads;
+  const int r = ls / g.n_kv_heads;
+  b = g.seq_begin + r % g.seq_count;
+  tensor = r / g.seq_count;
+  return (tensor * g.batch + b) * g.n_kv_heads + h;
+}
+
 struct InitParams {
+  Geom g;
   unsigned* seg_minmax[kMaxMergePairs];
   int32_t* status[kMaxMergePairs];
-  int nseg;
+  int clear_status;  // a merge of the whole batch starts from clean status words; an admission keeps them
 };
 __global__ void merge_init_kernel(const __grid_constant__ InitParams ip) {
   grid_dep_wait();
   grid_dep_launch();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   unsigned* seg_minmax = ip.seg_minmax[blockIdx.y];
-  if (i < ip.nseg) {
-    seg_minmax[2 * i] = 0x7f800000u;
-    seg_minmax[2 * i + 1] = 0u;
+  if (i < 2 * ip.g.seq_count * ip.g.n_kv_heads) {
+    int tensor, b, h;
+    const int seg = call_segment(ip.g, i, tensor, b, h);
+    seg_minmax[2 * seg] = 0x7f800000u;
+    seg_minmax[2 * seg + 1] = 0u;
   }
-  if (i < MC_STATUS_WORDS) ip.status[blockIdx.y][i] = 0;
+  if (ip.clear_status && i < MC_STATUS_WORDS) ip.status[blockIdx.y][i] = 0;
 }
 
 // Retention decision of one token; the threshold is formed in double from the fp32 extremes.
@@ -541,8 +560,8 @@ __device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, 
 // segment's quota of ties lasts (top-k mode: d equal to the k-th largest; ties go to lower indices).
 // `near` counts the tokens whose distance lies within 1e-6 of the decision threshold: the ones a
 // different rounding of d could have decided the other way.
-__device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
-                                            unsigned& sure, unsigned& eq, int* near = nullptr) {
+__device__ __forceinline__ void keep_masks4_one(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
+                                                unsigned& sure, unsigned& eq, int* near) {
   sure = eq = 0u;
   if (tok0 >= n) return;
   bool ok;
@@ -573,6 +592,20 @@ __device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int 
   }
 }
 
+// The decision for the thread's four tokens of segment (tensor, b, h).  With one set for keys and values
+// (union_kv; threshold modes only) the other tensor's rule is applied to its own distances as well and
+// the two masks are joined; `near` counts this tensor's own near-threshold tokens either way.
+__device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
+                                            unsigned& sure, unsigned& eq, int* near = nullptr) {
+  keep_masks4_one(p, seg, tensor, b, h, tok0, n, sure, eq, near);
+  if (p.union_kv && p.mode != MC_RETAIN_TOPK) {
+    const int seg_o = tensor ? seg - p.g.batch * p.g.n_kv_heads : seg + p.g.batch * p.g.n_kv_heads;
+    unsigned sure_o, eq_o;
+    keep_masks4_one(p, seg_o, 1 - tensor, b, h, tok0, n, sure_o, eq_o, nullptr);
+    sure |= sure_o;
+  }
+}
+
 // Top-k reading of the retention rule: per segment, the k-th largest distance (k = ceil(gamma n)) by a
 // radix select over the float bits (d >= 0, so unsigned order is float order), and how many of the
 // tokens equal to it belong to the k largest.
@@ -583,10 +616,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const __grid
   __shared__ int hist[256];
   __shared__ uint32_t s_prefix, s_mask;
   __shared__ int s_remaining;
-  const int seg = blockIdx.x;
-  const int h = seg % p.g.n_kv_heads;
-  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
-  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  int tensor, b, h;
+  const int seg = call_segment(p.g, blockIdx.x, tensor, b, h);
   const int n = checked_len(p.g, b, p.status);
   const int k = min(n, (int)ceil(p.gamma * (double)n - 1e-12));
   if (k <= 0 || !p.do_retention) {
@@ -644,10 +675,9 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
   __shared__ int s_cnt[kRetThreads / 32], s_eq[kRetThreads / 32];
   __shared__ int s_last;
   __shared__ int s_carry;
-  const int seg = blockIdx.y, chunk = blockIdx.x;
-  const int h = seg % p.g.n_kv_heads;
-  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
-  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  const int chunk = blockIdx.x;
+  int tensor, b, h;
+  const int seg = call_segment(p.g, blockIdx.y, tensor, b, h);
   const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int cnt = 0, cnt_eq = 0, cnt_near = 0;
@@ -687,7 +717,9 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
   // ---- last block.  Top-k mode first: the ties are handed out in token order, so per segment the
   // chunks take from the quota one after the other; chunk_eq becomes "ties before this chunk".
   if (p.mode == MC_RETAIN_TOPK) {
-    for (int sg = threadIdx.x; sg < p.nseg; sg += kRetThreads) {
+    for (int ls = threadIdx.x; ls < 2 * p.g.seq_count * p.g.n_kv_heads; ls += kRetThreads) {
+      int t_, b_, h_;
+      const int sg = call_segment(p.g, ls, t_, b_, h_);
       const int quota = (int)p.seg_sel[2 * sg + 1];
       int eq_run = 0;
       for (int c = 0; c < p.chunks_per_seg; ++c) {
@@ -700,6 +732,50 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
     }
     __threadfence();
     __syncthreads();
+  }
+  if (p.region_rows > 0) {
+    // ---- admission: every sequence of the call owns the entries [b R, (b + 1) R) of the pool, its
+    // segments in (tensor, head) order inside them.  A sequence that needs more keeps nothing
+    // (offset -1) and the overflow flag is set.
+    const int per_seq = 2 * p.g.n_kv_heads * p.chunks_per_seg;
+    for (int sq = 0; sq < p.g.seq_count; ++sq) {
+      const int bq = p.g.seq_begin + sq;
+      __syncthreads();
+      if (threadIdx.x == 0) s_carry = 0;
+      __syncthreads();
+      for (int base = 0; base < per_seq; base += kRetThreads) {
+        const int j = base + threadIdx.x;  // (tensor, head, chunk), chunk fastest
+        const int sg = j < per_seq ? ((j / p.chunks_per_seg / p.g.n_kv_heads) * p.g.batch + bq) * p.g.n_kv_heads +
+                                         (j / p.chunks_per_seg) % p.g.n_kv_heads : 0;
+        const size_t ci = (size_t)sg * p.chunks_per_seg + (j % p.chunks_per_seg);
+        const int v = j < per_seq ? __ldcg(p.chunk_count + ci) : 0;
+        int x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, x, o);
+          if (lane >= o) x += y;
+        }
+        if (lane == 31) s_cnt[warp] = x;
+        __syncthreads();
+        int warp_excl = 0;
+        for (int w = 0; w < warp; ++w) warp_excl += s_cnt[w];
+        const int excl = s_carry + warp_excl + x - v;
+        if (j < per_seq) p.chunk_offset[ci] = bq * p.region_rows + excl;
+        __syncthreads();
+        if (threadIdx.x == kRetThreads - 1) s_carry = excl + v;
+        __syncthreads();
+      }
+      const bool fits = s_carry <= p.region_rows;
+      for (int sj = threadIdx.x; sj < 2 * p.g.n_kv_heads; sj += kRetThreads) {
+        const int sg = ((sj / p.g.n_kv_heads) * p.g.batch + bq) * p.g.n_kv_heads + sj % p.g.n_kv_heads;
+        int cnt_seg = 0;
+        for (int c = 0; c < p.chunks_per_seg; ++c) cnt_seg += __ldcg(p.chunk_count + (size_t)sg * p.chunks_per_seg + c);
+        p.ret_offset[sg] = fits ? p.chunk_offset[(size_t)sg * p.chunks_per_seg] : -1;
+        p.ret_count[sg] = fits ? cnt_seg : 0;
+      }
+      if (threadIdx.x == 0 && !fits) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_RETAIN_OVERFLOW);
+    }
+    if (threadIdx.x == 0) p.status[MC_STATUS_RESERVED1] = 0;
+    return;
   }
   // exclusive scan of all chunk counts
   const int total = p.nseg * p.chunks_per_seg;
@@ -741,15 +817,15 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __gri
   grid_dep_launch();
   const RetainParams p = retain_view(bp, blockIdx.z);
   __shared__ int s_warp[kRetThreads / 32];
-  const int seg = blockIdx.y, chunk = blockIdx.x;
-  const int h = seg % p.g.n_kv_heads;
-  const int b = (seg / p.g.n_kv_heads) % p.g.batch;
-  const int tensor = seg / (p.g.n_kv_heads * p.g.batch);
+  const int chunk = blockIdx.x;
+  int tensor, b, h;
+  const int seg = call_segment(p.g, blockIdx.y, tensor, b, h);
   const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const bool overflow = (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
   const int seg_off = p.ret_offset[seg];
-  const int seg_cnt = overflow ? 0 : p.ret_offset[seg + 1] - seg_off;
+  // (admission: the scan has written the segment's count, and -1 as the offset of a sequence that did not fit)
+  const bool overflow = p.region_rows > 0 ? seg_off < 0 : (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
+  const int seg_cnt = overflow ? 0 : (p.region_rows > 0 ? p.ret_count[seg] : p.ret_offset[seg + 1] - seg_off);
   if (chunk == 0 && threadIdx.x == 0) p.ret_count[seg] = seg_cnt;
   int32_t* prefix = p.ret_prefix + (size_t)seg * p.ret_prefix_stride;
   if (chunk == 0)  // table entries past the last chunk: everything lies before them
@@ -874,6 +950,7 @@ struct AppendParams {
   float* dist;
   float ta, tc;
   int merge_fn;
+  int t_mode;
   int total_rows;  // 2 * batch * H
   int32_t* status;
 };
@@ -909,7 +986,7 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   }
   uint4 e;
   float ga, gc, d;
-  merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, ga, gc, d);
+  merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, p.t_mode, e, ga, gc, d);
   if (!ok || !page_ok(p.g, page)) return;
   const int tk = tok & (p.g.page_size - 1);
   const size_t ph = (size_t)page * H + h;
@@ -935,9 +1012,11 @@ size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
 
 mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geom& g, int n_pairs, const mc_layer_kv* const* lm1,
                              const mc_layer_kv* const* l, const mc_layer_q4* const* q_lm1, const mc_layer_q4* const* q_l,
-                             const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream) {
+                             const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream,
+                             int region_rows) {
   const bool q4 = q_lm1 != nullptr;
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
+  const int nseg_call = 2 * g.seq_count * cfg->n_kv_heads;  // segments of the sequences this call works on
   // every shape limit before the first launch
   if (n_pairs < 1 || n_pairs > kMaxMergePairs) return MC_ERR_SHAPE;
   if (bt->batch > kMergeMaxBatchSmem) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
@@ -949,10 +1028,11 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
     ip.seg_minmax[i] = reinterpret_cast<unsigned*>(out[std::min(i, n_pairs - 1)]->seg_minmax);
     ip.status[i] = out[std::min(i, n_pairs - 1)]->status;
   }
-  ip.nseg = nseg;
-  MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg, (int)MC_STATUS_WORDS) + 255) / 256, n_pairs), dim3(256), 0, stream, ip));
+  ip.g = g;
+  ip.clear_status = region_rows > 0 ? 0 : 1;
+  MC_CUDA_CHECK(launch_pdl(merge_init_kernel, dim3((std::max(nseg_call, (int)MC_STATUS_WORDS) + 255) / 256, n_pairs), dim3(256), 0, stream, ip));
   MC_CUDA_CHECK(cudaGetLastError());
-  if (bt->batch == 0) return MC_OK;
+  if (bt->batch == 0 || g.seq_count == 0) return MC_OK;
 
   MergeParams mp;
   RetainBatch rb;
@@ -1002,11 +1082,12 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   }
   mp.n_pairs = n_pairs;
   mp.merge_fn = cfg->merge_fn;
+  mp.t_mode = cfg->t_mode;
   mp.ta = (float)(1.0 - cfg->t);
   mp.tc = (float)cfg->t;
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
   // upper bound of the item count (the kernel enumerates the pages that hold tokens)
-  const long long total = 2LL * n_pairs * bt->batch * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
+  const long long total = 2LL * n_pairs * g.seq_count * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
   if (total > 0) {
     int n_sm = 0;
     if (mc_status st = sm_count(&n_sm)) return st;
@@ -1026,10 +1107,12 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   rb.nseg = nseg;
   rb.mode = cfg->retain_mode;
   rb.do_retention = do_retention;
+  rb.union_kv = cfg->retain_union;
+  rb.region_rows = region_rows;
   rb.gamma = cfg->gamma;
-  dim3 grid(rb.chunks_per_seg, nseg, n_pairs);
+  dim3 grid(rb.chunks_per_seg, nseg_call, n_pairs);
   if (cfg->retain_mode == MC_RETAIN_TOPK)
-    MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg, 1, n_pairs), dim3(kRetThreads), 0, stream, rb));
+    MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg_call, 1, n_pairs), dim3(kRetThreads), 0, stream, rb));
   MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rb));
   MC_CUDA_CHECK(launch_pdl(retain_compact_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rb));
   return MC_OK;
@@ -1039,7 +1122,7 @@ mc_status launch_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, 
                        const mc_layer_kv* l, const mc_layer_q4* q_lm1, const mc_layer_q4* q_l, const mc_pair_cache* out,
                        int do_retention, void* workspace, cudaStream_t stream) {
   return launch_merge_pairs(cfg, bt, g, 1, lm1 ? &lm1 : nullptr, l ? &l : nullptr, q_lm1 ? &q_lm1 : nullptr, q_l ? &q_l : nullptr,
-                            &out, do_retention, workspace, stream);
+                            &out, do_retention, workspace, stream, 0);
 }
 
 mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
@@ -1055,6 +1138,7 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   ap.e_pool[1] = (char*)pair->e_v;
   ap.dist = pair->dist;
   ap.merge_fn = cfg->merge_fn;
+  ap.t_mode = cfg->t_mode;
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;
   ap.total_rows = 2 * bt->batch * cfg->n_kv_heads;

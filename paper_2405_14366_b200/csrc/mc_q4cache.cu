@@ -206,6 +206,7 @@ struct AppendQ4Params {
   float* dist;
   float ta, tc;
   int merge_fn;
+  int t_mode;
   int32_t* status;
 };
 
@@ -235,7 +236,7 @@ __global__ void __launch_bounds__(kQThreads) append_q4_kernel(const AppendQ4Para
     const uint4 vc = *reinterpret_cast<const uint4*>(p.c_new[tensor] + off);
     uint4 e;
     float ga, gc, d;
-    merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, e, ga, gc, d);
+    merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, p.t_mode, e, ga, gc, d);
     if (threadIdx.x < 16) {
       *reinterpret_cast<uint4*>(res + slot * kRowBytes + chunk_pos(slot, l16) * 16) = e;
       if (l16 == 0) {
@@ -434,6 +435,7 @@ mc_status launch_append_q4(const mc_config* cfg, const mc_batch* bt, const Geom&
   ap.res[1] = (char*)pair->res_v;
   ap.dist = pair->dist;
   ap.merge_fn = cfg->merge_fn;
+  ap.t_mode = cfg->t_mode;
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;
   ap.status = pair->status;

@@ -23,7 +23,8 @@ class Problem:
     def __init__(self, cfg: WorkloadConfig, pair: int = 0, device="cuda", seq_lens=None, gamma=None, t=None,
                  retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
                  tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None,
-                 q4: bool = False, merge_fn: str = "slerp", segments=None, cache_bits: int = 16):
+                 q4: bool = False, merge_fn: str = "slerp", segments=None, cache_bits: int = 16,
+                 t_mode: int = 0, retain_union: int = 0):
         """segments: list of (sequence, kv head) the oracle will look at; given, the host copies of 4-bit
         layers (exact de-quantised values, fp64) are kept for those segments only (full-size workloads)."""
         import paper_2405_14366_b200 as mc
@@ -52,8 +53,9 @@ class Problem:
         self.max_seq_len = int(self.seq_lens_host.max()) if B else 0
         self.merge_fn = merge_fn
         self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode,
-                               merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn], cache_bits=cache_bits)
-        self.cache_bits = cache_bits
+                               merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn], cache_bits=cache_bits,
+                               t_mode=t_mode, retain_union=retain_union)
+        self.cache_bits, self.t_mode, self.retain_union = cache_bits, t_mode, retain_union
         self.pools = {}
         self.q4 = q4
         self.q4_pools: Dict[str, Dict[str, torch.Tensor]] = {}
@@ -220,16 +222,24 @@ class Problem:
         return idx, dc["ret_rows"][off:off + cnt]
 
     # ------------------------------------------------------------------ oracle side
+    @property
+    def oracle_t(self):
+        """The oracle's t argument: the number, or "ratio" for the per-token magnitude ratio."""
+        return "ratio" if self.t_mode == 1 else self.t
+
     def oracle_merge(self, mode: str = "distinct", do_retention: bool = True):
         out = {}
         for ti, tn in enumerate(("k", "v")):
             if self.q4:
                 out[tn] = orc.merge_pair_values(self.values[tn + "_lm1"], self.values[tn + "_l"], self.seq_lens_host,
-                                                self.dtype, self.t, self.gamma, mode=mode, do_retention=do_retention,
+                                                self.dtype, self.oracle_t, self.gamma, mode=mode, do_retention=do_retention,
                                                 merge_fn=self.merge_fn)
                 continue
             out[tn] = orc.merge_pair(self.bits[tn + "_lm1"], self.bits[tn + "_l"], self.seq_lens_host, self.dtype,
-                                     self.t, self.gamma, mode=mode, do_retention=do_retention, merge_fn=self.merge_fn)
+                                     self.oracle_t, self.gamma, mode=mode, do_retention=do_retention, merge_fn=self.merge_fn)
+        if self.retain_union:  # one set for keys and values
+            un = orc.retention_union(out["k"]["retained"], out["v"]["retained"])
+            out["k"]["retained"], out["v"]["retained"] = un, dict(un)
         if self.cache_bits == 4:  # the merged directions as the 4-bit shared cache stores them
             out = {tn: orc.q4_cache_pair(out[tn], self.seq_lens_host, tn, self.dtype) for tn in out}
         return out
@@ -315,7 +325,11 @@ def compare_merge(p: Problem, om, dc, mode: str = "distinct", do_retention: bool
                     thr = orc.retention_threshold(d, p.gamma, mode)
                 sym = np.setxor1d(want, got)
                 # exact, except tokens whose distance lies within 1e-6 of the threshold
-                assert np.all(np.abs(d[sym] - thr) < 1e-6), f"retained set differs away from the threshold: {sym}"
+                close = np.abs(d[sym] - thr) < 1e-6
+                if getattr(p, "retain_union", 0):  # ... or of the other tensor's threshold, whose rule also decides
+                    d_o = om["v" if tn == "k" else "k"]["d"][b, :n, h]
+                    close |= np.abs(d_o[sym] - orc.retention_threshold(d_o, p.gamma, mode)) < 1e-6
+                assert np.all(close), f"retained set differs away from the threshold: {sym}"
                 mism += len(sym)
                 near += int(np.sum(np.abs(d - thr) < 1e-6))
                 # raw rows are bit copies of both layers' inputs

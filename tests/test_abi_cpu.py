@@ -36,10 +36,10 @@ def test_status_strings(lib):
 
 def _cfg(**kw):
     d = dict(n_kv_heads=8, n_q_heads=32, head_dim=128, page_size=16, dtype=0, retain_mode=0, t=0.6, gamma=0.05,
-             merge_fn=0, cache_bits=0)
+             merge_fn=0, cache_bits=0, t_mode=0, retain_union=0)
     d.update(kw)
     return B._Config(d["n_kv_heads"], d["n_q_heads"], d["head_dim"], d["page_size"], d["dtype"], d["retain_mode"],
-                     d["t"], d["gamma"], d["merge_fn"], d["cache_bits"])
+                     d["t"], d["gamma"], d["merge_fn"], d["cache_bits"], d["t_mode"], d["retain_union"])
 
 
 def _batch(batch=2, mpps=4, max_len=64, n_pages=10, bt=0x1000, sl=0x2000):
@@ -64,6 +64,7 @@ def test_workspace_bytes_is_host_arithmetic(lib):
     (dict(head_dim=64), 2), (dict(page_size=8), 2), (dict(n_q_heads=12), 2), (dict(n_q_heads=24), 2),
     (dict(dtype=5), 3), (dict(retain_mode=9), 1), (dict(t=1.5), 1), (dict(gamma=-0.1), 1),
     (dict(cache_bits=8), 1), (dict(cache_bits=4, page_size=16), 2), (dict(merge_fn=3), 1),
+    (dict(t_mode=2), 1), (dict(retain_union=2), 1), (dict(retain_union=1, retain_mode=2), 6),
 ])
 def test_bad_config_rejected(lib, kw, code):
     out = C.c_size_t(0)
@@ -180,6 +181,22 @@ def test_merge_pairs_checks_every_pair_before_launching(lib):
     c4 = _cfg(page_size=32, cache_bits=4)
     assert L.mc_merge_pairs(C.byref(c4), C.byref(b), 1, arr([a], B._LayerKV), arr([a], B._LayerKV), arr(pcs[:1], B._PairCache),
                             1, 0x100000, 1 << 30, None) == 6
+
+
+def test_admit_sequences_argument_checks(lib):
+    L = lib._lib
+    c, b = _cfg(), _batch()
+    a = B._LayerKV(0x10000, 0x20000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    arr = lambda items, T: (C.POINTER(T) * len(items))(*[C.pointer(x) for x in items])
+    call = lambda sb, sc, rows, wsb: L.mc_admit_sequences(C.byref(c), C.byref(b), sb, sc, 1, arr([a], B._LayerKV), arr([a], B._LayerKV),
+                                                          None, None, arr([pc], B._PairCache), rows, 1, 0x100000, wsb, None)
+    assert call(1, 2, 8, 1 << 30) == 1      # sequences 1..2 of a batch of 2
+    assert call(0, 1, 0, 1 << 30) == 1      # no room per sequence
+    assert call(0, 1, 9, 1 << 30) == 5      # 2 sequences x 9 entries > the pool's 16
+    assert call(0, 1, 8, 16) == 5           # workspace too small
+    # both kinds of layers given, or neither
+    assert L.mc_admit_sequences(C.byref(c), C.byref(b), 0, 1, 1, None, None, None, None, arr([pc], B._PairCache), 8, 1, 0x100000, 1 << 30, None) == 1
 
 
 def test_get_stats_rejects_bad_arguments(lib):
