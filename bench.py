@@ -118,7 +118,7 @@ class Job:
         self.max_prefill = int(prompt.max())
         self.tok_heads = int(prompt.sum()) * self.H  # (token, kv head) rows per layer and tensor
         self.pools, self.pairs = [], []
-        cap_rows = int(max(0.10, 2.5 * wl.outlier_frac) * 2 * self.tok_heads) + 1024
+        cap_rows = int(max(0.10, 4.0 * wl.outlier_frac, 1.5 * wl.gamma) * 2 * self.tok_heads) + 1024
         if serving:  # one region of the retained pool per slot
             self.rows_per_seq = int(0.10 * 2 * wl.seq_len * self.H) + 64
             cap_rows = self.B * self.rows_per_seq

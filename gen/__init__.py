@@ -10,6 +10,7 @@ from .workload import (  # noqa: F401
     CONFIGS,
     WorkloadConfig,
     make_pair_tensors,
+    make_projection_case,
     make_queries,
     make_new_tokens,
     make_lengths,

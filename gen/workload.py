@@ -268,3 +268,36 @@ def quantise_q4(x: torch.Tensor, kind: str) -> Dict[str, torch.Tensor]:
     q = q.to(torch.uint8)
     codes = (q[..., 0::2] | (q[..., 1::2] << 4)).contiguous()
     return {"codes": codes, "meta": torch.stack([scale, zero], dim=-1).contiguous()}
+
+
+def make_projection_case(cfg: WorkloadConfig, pair: int, d_model: int, x_seq_stride: int, device="cpu") -> Dict[str, torch.Tensor]:
+    """Inputs of the merge fused into layer l's K/V projection: hidden states ``x`` [batch][x_seq_stride][d_model]
+    and transposed weights ``w_k, w_v`` [n_kv_heads * 128][d_model] in the storage dtype, scaled so that the rows
+    x W^T follow the row model (random directions, log-normal lengths), and layer l-1's rows ``k_lm1, v_lm1``
+    [batch][x_seq_stride][n_kv_heads][128] planted at the row model's angles from those products (the same recipe
+    as make_pair_tensors, with layer l's rows given by the projection instead of drawn)."""
+    B, S, H, D = cfg.batch, x_seq_stride, cfg.n_kv_heads, cfg.head_dim
+    dt = torch_dtype(cfg.dtype)
+    mu = cfg.theta_mean(pair)
+    gm = _rng(device, _seed(cfg, pair, 40))
+    outlier = torch.rand(B, S, generator=gm, device=device) < cfg.outlier_frac
+    x = torch.randn(B, S, d_model, generator=gm, device=device, dtype=torch.float32)
+    x *= torch.exp(0.5 * torch.randn(B, S, 1, generator=gm, device=device, dtype=torch.float32))  # per-token length
+    x = x.to(dt)
+    out: Dict[str, torch.Tensor] = {"x": x}
+    for ti, name in enumerate(("k", "v")):
+        g = _rng(device, _seed(cfg, pair, 41 + ti))
+        w = (torch.randn(H * D, d_model, generator=g, device=device, dtype=torch.float32) / math.sqrt(d_model * D)).to(dt)
+        out["w_" + name] = w
+        c = (x.float().reshape(B * S, d_model) @ w.float().T).reshape(B, S, H, D)  # layer l's rows, before storage rounding
+        cn = c / c.norm(dim=-1, keepdim=True).clamp_min(1e-20)
+        nz = torch.randn(B, S, H, D, generator=g, device=device, dtype=torch.float32)
+        nz -= (nz * cn).sum(-1, keepdim=True) * cn
+        nz /= nz.norm(dim=-1, keepdim=True)
+        u = torch.rand(B, S, H, generator=g, device=device, dtype=torch.float32)
+        theta = torch.where(outlier[:, :, None], 1.2 + 0.8 * u, 2.0 * mu * u)
+        len_lm1 = torch.exp(0.5 * torch.randn(B, S, H, generator=g, device=device, dtype=torch.float32))
+        y = torch.cos(theta)[..., None] * cn + torch.sin(theta)[..., None] * nz
+        out[name + "_lm1"] = (y * len_lm1[..., None]).to(dt)
+        out[name + "_ref"] = c
+    return out

@@ -100,7 +100,8 @@ typedef enum mc_t_mode { MC_T_FIXED = 0, MC_T_MAGNITUDE_RATIO = 1 } mc_t_mode;
 enum {
   MC_STATUS_FLAGS = 0,          /* bit 0: retained pool overflow; bit 1: a bounded wait ran out;
                                    bit 2: a length or page id outside the declared bounds was met;
-                                   bit 3: a range check of the range-checked build failed */
+                                   bit 3: a range check of the range-checked build failed;
+                                   bit 4: mc_prefill_merge_pair's distance hint was too high */
   MC_STATUS_RETAINED_TOTAL = 1, /* retained entries the last merge selected (K and V segments together) */
   MC_STATUS_NEAR_THRESHOLD = 2, /* tokens of the last merge whose distance lies within 1e-6 of their segment's
                                    retention threshold (a differently rounded d could have decided them the
@@ -120,6 +121,9 @@ enum {
  * capacity, a compaction slot -- fell outside its bounds.  The access is skipped, the kernel carries
  * on, results that depended on it are meaningless. */
 #define MC_FLAG_BOUNDS 8
+/* mc_prefill_merge_pair: a segment's retention threshold fell below the caller's distance hint, so the raw
+ * layer-l row of some retained token may not have been stored; merge that pair again with a lower hint. */
+#define MC_FLAG_HINT_TOO_HIGH 16
 
 /* Method parameters and tensor geometry (Sec. 4.1-4.2, Sec. 5 defaults t = 0.6, gamma = 0.05). */
 typedef struct mc_config {
@@ -367,6 +371,39 @@ mc_status mc_admit_sequences(const mc_config* cfg, const mc_batch* batch, int32_
                              const mc_layer_q4* const* q4_lm1, const mc_layer_q4* const* q4_l,
                              const mc_pair_cache* const* out, int64_t rows_per_seq, int32_t do_retention,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* The K/V projection of layer l (the stand-in for the model's own: the library computes K^l = X W_k^T and
+ * V^l = X W_v^T itself so that it can merge in the projection's epilogue).
+ * x        [batch * x_seq_stride][d_model] hidden states entering layer l's K/V projection, cfg->dtype;
+ *          token i of sequence b is row b * x_seq_stride + i; x_seq_stride a multiple of 128, >= max_seq_len
+ * w_k, w_v [n_kv_heads * 128][d_model] cfg->dtype: row (head * 128 + channel) holds that output channel's
+ *          weights (the transposed weight matrix, contiguous along d_model)
+ * d_model  a multiple of 64.  All three base addresses 256-byte aligned. */
+typedef struct mc_projection {
+  const void* x;
+  const void* w_k;
+  const void* w_v;
+  int32_t d_model;
+  int32_t x_seq_stride;
+} mc_projection;
+
+/* Algorithm 1's prefill branch with the merge fused into layer l's projection ("merge at odd layers during
+ * prefill"): layer l's K and V rows are formed on chip (tensor cores, fp32 accumulation, rounded once to
+ * cfg->dtype -- the rows the model would have cached) and merged with layer l-1's cached rows (lm1) by
+ * Eq. 2 / Eq. 3 right there, so they are never written to and read back from device memory; `out` receives
+ * exactly what mc_merge_pair would have written for those rows.
+ * Retention (Eq. 4) needs the raw layer-l rows of the tokens it keeps, and which tokens those are is known
+ * only once every distance of a segment is: the rows of tokens with distance d > d_hint are therefore also
+ * stored, at their places in the pools `l` (everything else in `l` is left untouched), and the retention
+ * pass gathers from there.  d_hint < 0 stores every row (`l` then holds the whole layer, e.g. for checking).
+ * If a segment's threshold turns out below d_hint, MC_FLAG_HINT_TOO_HIGH is set: merge that pair again with
+ * a lower hint.  With do_retention == 0 nothing needs to be stored (pass d_hint = 2).
+ * Limits: cfg->merge_fn = MC_MERGE_SLERP, cfg->retain_mode = MC_RETAIN_DISTINCT (or d_hint < 0), 16-bit
+ * shared cache, d_model % 64 == 0.  workspace as for mc_merge_pair. */
+mc_status mc_prefill_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_projection* proj,
+                                const mc_layer_kv* lm1, const mc_layer_kv* l, const mc_pair_cache* out,
+                                float d_hint, int32_t do_retention, void* workspace, size_t workspace_bytes,
+                                void* stream);
 
 /* mc_merge_pair for layers stored in 4 bits: the rows are de-quantised inside the merge kernel
  * (code * scale + zero in fp32) and merged exactly as in mc_merge_pair; the pair cache it writes is

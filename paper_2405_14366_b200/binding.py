@@ -19,6 +19,7 @@ MC_OP_MERGE, MC_OP_DECODE_ATTN = 0, 1
 MC_STATUS_WORDS = 4
 MC_STATUS_FLAGS, MC_STATUS_RETAINED_TOTAL, MC_STATUS_NEAR_THRESHOLD = 0, 1, 2
 MC_FLAG_RETAIN_OVERFLOW, MC_FLAG_WAIT_TIMEOUT, MC_FLAG_BAD_METADATA, MC_FLAG_BOUNDS = 1, 2, 4, 8
+MC_FLAG_HINT_TOO_HIGH = 16
 MC_BUILD_BOUNDS = 1
 
 # MINICACHE_LIBRARY selects another build of the same library (the range-checked one, for instance)
@@ -53,6 +54,10 @@ class _LayerQ4(C.Structure):
     _fields_ = [("k_codes", C.c_void_p), ("k_meta", C.c_void_p), ("v_codes", C.c_void_p), ("v_meta", C.c_void_p)]
 
 
+class _Projection(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("w_k", C.c_void_p), ("w_v", C.c_void_p), ("d_model", C.c_int32), ("x_seq_stride", C.c_int32)]
+
+
 class _PairCache(C.Structure):
     _fields_ = [("e_k", C.c_void_p), ("e_v", C.c_void_p), ("dist", C.c_void_p),
                 ("ret_count", C.c_void_p), ("ret_offset", C.c_void_p), ("ret_index", C.c_void_p),
@@ -75,7 +80,7 @@ class _Stats(C.Structure):
                 ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
 
 
-EXPORTS = ("mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+EXPORTS = ("mc_prefill_merge_pair", "mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -295,6 +300,9 @@ class MiniCacheLib:
         L.mc_admit_sequences.argtypes = [P(_Config), P(_Batch), C.c_int32, C.c_int32, C.c_int32, P(P(_LayerKV)), P(P(_LayerKV)),
                                          P(P(_LayerQ4)), P(P(_LayerQ4)), P(P(_PairCache)), C.c_int64, C.c_int32, V, C.c_size_t, V]
         L.mc_admit_sequences.restype = C.c_int32
+        L.mc_prefill_merge_pair.argtypes = [P(_Config), P(_Batch), P(_Projection), P(_LayerKV), P(_LayerKV), P(_PairCache),
+                                            C.c_float, C.c_int32, V, C.c_size_t, V]
+        L.mc_prefill_merge_pair.restype = C.c_int32
         L.mc_append_pair.argtypes = [P(_Config), P(_Batch), P(_PairCache), V, V, V, V, V]
         L.mc_restore.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, P(_LayerKV), C.c_int32, V]
         L.mc_pair_bytes.argtypes = [P(_Config), P(_Batch), C.c_int64, P(_PairSizes)]
@@ -387,6 +395,17 @@ class MiniCacheLib:
         self._check(self._lib.mc_admit_sequences(C.byref(c), C.byref(b), int(seq_begin), int(seq_count), n, *args,
                                                  arr(pcs, _PairCache), int(rows_per_seq), 1 if do_retention else 0,
                                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_prefill_merge_pair(self, cfg: McConfig, batch: Batch, x, w_k, w_v, k_lm1, v_lm1, k_l, v_l, pair: PairCache,
+                              d_hint: float, do_retention: bool, workspace: torch.Tensor, stream=None):
+        """x [batch][x_seq_stride][d_model], w_k / w_v [n_kv_heads * 128][d_model]: layer l's projection;
+        k_l / v_l: pools that receive the raw rows of tokens with distance above d_hint."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        pj = _Projection(_ptr(x), _ptr(w_k), _ptr(w_v), int(x.shape[-1]), int(x.shape[1]))
+        a, l = _LayerKV(_ptr(k_lm1), _ptr(v_lm1)), _LayerKV(_ptr(k_l), _ptr(v_l))
+        self._check(self._lib.mc_prefill_merge_pair(C.byref(c), C.byref(b), C.byref(pj), C.byref(a), C.byref(l), C.byref(pc),
+                                                    float(d_hint), 1 if do_retention else 0, _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(), _stream(stream)))
 
     def mc_merge_pair_q4(self, cfg: McConfig, batch: Batch, q_lm1, q_l, pair: PairCache, do_retention: bool,
                          workspace: torch.Tensor, stream=None):

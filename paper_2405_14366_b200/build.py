@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libminicache.so")
 BOUNDS_LIB_PATH = os.path.join(PKG_DIR, "libminicache_bounds.so")  # the range-checked build (-DMC_BOUNDS=1)
-SOURCES = ["mc_api.cu", "mc_merge.cu", "mc_restore.cu", "mc_attn.cu", "mc_q4cache.cu"]
+SOURCES = ["mc_api.cu", "mc_merge.cu", "mc_restore.cu", "mc_attn.cu", "mc_q4cache.cu", "mc_prefill.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

@@ -390,6 +390,32 @@ mc_status mc_admit_sequences(const mc_config* cfg, const mc_batch* batch, int32_
   return MC_OK;
 }
 
+mc_status mc_prefill_merge_pair(const mc_config* cfg, const mc_batch* batch, const mc_projection* proj, const mc_layer_kv* lm1,
+                                const mc_layer_kv* l, const mc_pair_cache* out, float d_hint, int32_t do_retention,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_prefill_merge_pair");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  if (!proj || !proj->x || !proj->w_k || !proj->w_v || !lm1 || !l || !lm1->k_pool || !lm1->v_pool || !l->k_pool || !l->v_pool)
+    return MC_ERR_INVALID_ARG;
+  if (proj->d_model <= 0 || proj->d_model % 64 != 0 || proj->x_seq_stride <= 0 || proj->x_seq_stride % 128 != 0 ||
+      proj->x_seq_stride < batch->max_seq_len)
+    return MC_ERR_SHAPE;
+  if (cfg->merge_fn != MC_MERGE_SLERP || cfg->cache_bits == 4) return MC_ERR_UNSUPPORTED;
+  if (do_retention && cfg->retain_mode != MC_RETAIN_DISTINCT && d_hint >= 0.f) return MC_ERR_UNSUPPORTED;
+  if (do_retention && cfg->retain_union && d_hint >= 0.f) return MC_ERR_UNSUPPORTED;  // the other tensor's rule may keep a token below the hint
+  if (!aligned256(proj->x) || !aligned256(proj->w_k) || !aligned256(proj->w_v) || !aligned256(lm1->k_pool) ||
+      !aligned256(lm1->v_pool) || !aligned256(l->k_pool) || !aligned256(l->v_pool))
+    return MC_ERR_ALIGN;
+  st = check_merge_common(cfg, batch, out, workspace, workspace_bytes);
+  if (st != MC_OK) return st;
+  PrefillHook hook = {proj, d_hint};
+  return launch_merge_pairs(cfg, batch, make_geom(cfg, batch), 1, &lm1, &l, nullptr, nullptr, &out, do_retention ? 1 : 0, workspace,
+                            (cudaStream_t)stream, 0, &hook);
+}
+
 mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc_layer_q4* lm1, const mc_layer_q4* l,
                            const mc_pair_cache* out, int32_t do_retention, void* workspace, size_t workspace_bytes,
                            void* stream) {

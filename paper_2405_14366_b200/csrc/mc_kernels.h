@@ -21,7 +21,16 @@ constexpr int kMergePairsPerLaunch = 8;
 mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geom& g, int n_pairs, const mc_layer_kv* const* lm1,
                              const mc_layer_kv* const* l, const mc_layer_q4* const* q_lm1, const mc_layer_q4* const* q_l,
                              const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream,
-                             int region_rows = 0);
+                             int region_rows = 0, const struct PrefillHook* hook = nullptr);
+// With a hook (one pair), the rows of layer l come out of its projection inside launch_prefill_merge instead of
+// from pools; `l` then names the pools that receive the raw rows of tokens with d > d_hint.
+struct PrefillHook {
+  const mc_projection* proj;
+  float d_hint;
+};
+mc_status launch_prefill_merge(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_projection* proj,
+                               const mc_layer_kv* lm1, const mc_layer_kv* l, const mc_pair_cache* out, float d_hint,
+                               cudaStream_t stream);
 mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                         const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
                         cudaStream_t stream);

@@ -441,6 +441,7 @@ struct RetainParams {
   int do_retention;
   int union_kv;  // one set for keys and values: a token the other tensor's rule keeps is kept here too
   int region_rows;  // admission: entries of the retained pool each sequence owns (0: one compact list for the batch)
+  float d_hint;     // fused prefill: raw layer-l rows exist only for tokens with d > d_hint (< 0: for all)
   double gamma;
 };
 
@@ -470,6 +471,7 @@ struct RetainBatch {
   Geom g;
   RetainPair pr[kMaxMergePairs];  // blockIdx.z selects the pair
   int q4, dtype, chunks_per_seg, nseg, mode, do_retention, union_kv, region_rows;
+  float d_hint;  // fused prefill: raw layer-l rows exist only for tokens with d > d_hint (< 0: for all)
   double gamma;
 };
 __device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int pair) {
@@ -506,6 +508,7 @@ __device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int p
   p.do_retention = bp.do_retention;
   p.union_kv = bp.union_kv;
   p.region_rows = bp.region_rows;
+  p.d_hint = bp.d_hint;
   p.gamma = bp.gamma;
   return p;
 }
@@ -693,6 +696,11 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
     cnt_near += __shfl_xor_sync(0xffffffffu, cnt_near, o);
   }
   if (lane == 0 && cnt_near) atomicAdd(&p.status[MC_STATUS_NEAR_THRESHOLD], cnt_near);
+  if (chunk == 0 && threadIdx.x == 0 && p.do_retention && p.d_hint >= 0.f && n > 0 && p.mode == MC_RETAIN_DISTINCT) {
+    // fused prefill: every token this segment keeps must be one whose raw row was stored (d > d_hint)
+    const double lo = p.seg_minmax[2 * seg], hi = p.seg_minmax[2 * seg + 1];
+    if (hi - (hi - lo) * p.gamma < (double)p.d_hint && hi > lo && p.gamma > 0.0) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_HINT_TOO_HIGH);
+  }
   if (lane == 0) {
     s_cnt[warp] = cnt;
     s_eq[warp] = cnt_eq;
@@ -1013,8 +1021,9 @@ size_t merge_workspace_bytes(const mc_config* cfg, const mc_batch* bt) {
 mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geom& g, int n_pairs, const mc_layer_kv* const* lm1,
                              const mc_layer_kv* const* l, const mc_layer_q4* const* q_lm1, const mc_layer_q4* const* q_l,
                              const mc_pair_cache* const* out, int do_retention, void* workspace, cudaStream_t stream,
-                             int region_rows) {
+                             int region_rows, const PrefillHook* hook) {
   const bool q4 = q_lm1 != nullptr;
+  if (hook != nullptr && (n_pairs != 1 || q4)) return MC_ERR_UNSUPPORTED;
   const int nseg = 2 * bt->batch * cfg->n_kv_heads;
   const int nseg_call = 2 * g.seq_count * cfg->n_kv_heads;  // segments of the sequences this call works on
   // every shape limit before the first launch
@@ -1088,7 +1097,9 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   mp.items_per_page = (cfg->n_kv_heads * cfg->page_size + kRowsPerItem - 1) / kRowsPerItem;
   // upper bound of the item count (the kernel enumerates the pages that hold tokens)
   const long long total = 2LL * n_pairs * g.seq_count * ((bt->max_seq_len + cfg->page_size - 1) / cfg->page_size) * mp.items_per_page;
-  if (total > 0) {
+  if (hook != nullptr) {
+    if (mc_status st = launch_prefill_merge(cfg, bt, g, hook->proj, lm1[0], l[0], out[0], hook->d_hint, stream)) return st;
+  } else if (total > 0) {
     int n_sm = 0;
     if (mc_status st = sm_count(&n_sm)) return st;
     const int grid = (int)std::min<long long>((long long)n_sm * kMergeCtasPerSm, total);
@@ -1109,6 +1120,7 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   rb.do_retention = do_retention;
   rb.union_kv = cfg->retain_union;
   rb.region_rows = region_rows;
+  rb.d_hint = hook != nullptr ? hook->d_hint : -1.f;
   rb.gamma = cfg->gamma;
   dim3 grid(rb.chunks_per_seg, nseg_call, n_pairs);
   if (cfg->retain_mode == MC_RETAIN_TOPK)

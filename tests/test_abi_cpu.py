@@ -199,6 +199,24 @@ def test_admit_sequences_argument_checks(lib):
     assert L.mc_admit_sequences(C.byref(c), C.byref(b), 0, 1, 1, None, None, None, None, arr([pc], B._PairCache), 8, 1, 0x100000, 1 << 30, None) == 1
 
 
+def test_prefill_merge_argument_checks(lib):
+    L = lib._lib
+    c, b = _cfg(), _batch(max_len=64, mpps=4)
+    a = B._LayerKV(0x10000, 0x20000)
+    pc = B._PairCache(0x30000, 0x40000, 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 16, 0xD0000, 64, 0xB0000, 0xC0000)
+    pj = lambda **kw: B._Projection(kw.get("x", 0x200000), 0x300000, 0x400000, kw.get("d_model", 512), kw.get("stride", 128))
+    call = lambda cfg, proj, hint=0.3: L.mc_prefill_merge_pair(C.byref(cfg), C.byref(b), C.byref(proj), C.byref(a), C.byref(a), C.byref(pc),
+                                                               C.c_float(hint), 1, 0x100000, 1 << 30, None)
+    assert call(c, pj(d_model=500)) == 2           # d_model not a multiple of 64
+    assert call(c, pj(stride=100)) == 2            # rows per sequence not a multiple of 128
+    assert call(c, pj(stride=0)) == 2
+    assert call(c, pj(x=0)) == 1
+    assert call(c, pj(x=0x200010)) == 4
+    assert call(_cfg(merge_fn=1), pj()) == 6       # only the SLERP merge is fused
+    assert call(_cfg(retain_mode=1), pj()) == 6    # a distance hint needs the "most distinct" rule
+    assert call(_cfg(page_size=32, cache_bits=4), pj()) == 6
+
+
 def test_get_stats_rejects_bad_arguments(lib):
     L = lib._lib
     c, b, out = _cfg(), _batch(), B._Stats()
