@@ -407,6 +407,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--q4", action="store_true", help="the layers arrive in 4 bits (page size 32; no host-buffer leg)")
     ap.add_argument("--q4cache", action="store_true", help="the shared cache is 4-bit (page size 32): restore and attention read codes")
+    ap.add_argument("--prefill-fused", action="store_true",
+                    help="one pair: the merge fused into layer l's K/V projection (tensor cores) against projection + merge")
+    ap.add_argument("--d-model", type=int, default=4096, help="hidden size of the stand-in projection (--prefill-fused)")
     ap.add_argument("--refill", action="store_true",
                     help="serving trace: a seeded list of 8 x batch sequences, a slot is refilled when its sequence leaves, "
                          "the admitted sequence is merged on a second stream while the others decode")
@@ -443,6 +446,9 @@ def main():
 
     if args.refill:
         run_refill(args, wl, dev, rank, world, dist)
+        return
+    if args.prefill_fused:
+        run_prefill_fused(args, wl, dev)
         return
     job = Job(wl, dev, q4=args.q4, q4cache=args.q4cache)
     if args.q4:
@@ -568,6 +574,68 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_prefill_fused(args, wl, dev):
+    """One layer pair: layer l's K/V come out of a projection X W^T.  Fused: mc_prefill_merge_pair (the rows are
+    merged in the projection's epilogue and never stored, except those above the distance hint).  Unfused: a
+    library GEMM writes layer l's rows, mc_merge_pair reads them back.  Reports both times and the cache traffic."""
+    import paper_2405_14366_b200 as mc
+    lib = mc.lib()
+    B, S, H = wl.batch, wl.seq_len, wl.n_kv_heads
+    stride = (S + 127) // 128 * 128
+    case = gen.make_projection_case(wl, 0, args.d_model, stride, device=dev)
+    bt, n_pages = gen.make_block_table(np.full(B, S + 1), wl.page_size, seed=4321 + wl.index)
+    block_table = torch.from_numpy(bt).to(dev)
+    seq_lens = torch.full((B,), S, dtype=torch.int32, device=dev)
+    cfg = mc.McConfig(H, wl.n_q_heads, wl.page_size, wl.dtype, t=wl.t, gamma=wl.gamma)
+    batch = mc.Batch(block_table, seq_lens, S, n_pages)
+    pools = {k: gen.to_paged(case[k][:, :S], block_table, wl.page_size, n_pages) for k in ("k_lm1", "v_lm1")}
+    pools["k_l"] = torch.zeros_like(pools["k_lm1"])
+    pools["v_l"] = torch.zeros_like(pools["k_lm1"])
+    del case["k_lm1"], case["v_lm1"], case["k_ref"], case["v_ref"]
+    th = B * S * H
+    pair = mc.PairCache(cfg, B, n_pages, int(0.2 * th) + 1024, device=dev)
+    ws = torch.empty(lib.mc_workspace_bytes(cfg, batch, 0, 1), dtype=torch.uint8, device=dev)
+    hint = 0.3
+    fused = lambda: lib.mc_prefill_merge_pair(cfg, batch, case["x"], case["w_k"], case["w_v"], pools["k_lm1"], pools["v_lm1"],
+                                              pools["k_l"], pools["v_l"], pair, hint, True, ws)
+    x2 = case["x"].reshape(B * stride, args.d_model)
+    ck = torch.empty(B * stride, H * 128, dtype=x2.dtype, device=dev)
+    cv = torch.empty_like(ck)
+    gemms = lambda: (torch.matmul(x2, case["w_k"].T, out=ck), torch.matmul(x2, case["w_v"].T, out=cv))
+    merge = lambda: lib.mc_merge_pair(cfg, batch, pools["k_lm1"], pools["v_lm1"], pools["k_l"], pools["v_l"], pair, True, ws)
+    for _ in range(3):
+        fused()
+        gemms()
+    torch.cuda.synchronize()
+    med = lambda fn: float(np.median([timed(fn) for _ in range(5)]))
+    t_f = med(fused)
+    words, code = lib.mc_read_status(pair, check=False)
+    if code != 0:
+        raise SystemExit(f"device status {words}")
+    rho = int(pair.ret_count.sum().item()) / (2.0 * th)
+    stored = float((pair.dist > hint).float().sum().item()) / (2.0 * th)  # layer l's rows that were stored raw
+    t_g = med(gemms)
+    # the unfused merge needs all of layer l's rows in the pools: the fused call with a negative hint puts them there
+    lib.mc_prefill_merge_pair(cfg, batch, case["x"], case["w_k"], case["w_v"], pools["k_lm1"], pools["v_lm1"], pools["k_l"],
+                              pools["v_l"], pair, -1.0, True, ws)
+    merge()
+    t_m = med(merge)
+    flops = 2.0 * B * stride * args.d_model * (2 * H * 128)
+    kv_bytes_fused = 2 * th * (ROW + ROW + 12 + 4 + stored * ROW + rho * (4 * ROW + 4))   # layer l-1 read, E written (+ stored rows)
+    kv_bytes_unfused = 2 * th * (ROW + 2 * ROW + ROW + 12 + 4 + rho * (4 * ROW + 4))         # + layer l written, then read
+    line = {"metric": "hbm_gbps_merge_restore_decode_attn", "value": kv_bytes_fused / t_f / 1e9, "unit": "GB/s", "n_gpus": 1, "steps": 5,
+            "warmup": 3, "ms_per_step": t_f * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": wl.name + " one pair, merge fused into the K/V projection", "batch": B, "seq_len": S, "kv_heads": H,
+                       "d_model": args.d_model, "storage": wl.dtype, "distance_hint": hint},
+            "prefill_fused": {"fused_ms": t_f * 1e3, "gemm_tflops_fused": flops / t_f / 1e12,
+                              "library_gemm_ms": t_g * 1e3, "library_gemm_tflops": flops / t_g / 1e12, "merge_ms": t_m * 1e3,
+                              "unfused_ms": (t_g + t_m) * 1e3, "retained_fraction": rho, "rows_stored_fraction": stored,
+                              "cache_bytes_per_unit_fused": kv_bytes_fused / (2 * th), "cache_bytes_per_unit_unfused": kv_bytes_unfused / (2 * th)},
+            "gpu_launches": 4}
+    print(json.dumps(line))
 
 
 def run_refill(args, wl, dev, rank, world, dist):
