@@ -93,6 +93,7 @@ def _mk() -> Dict[str, WorkloadConfig]:
     # one pair of config 2 / 3 at full batch and length (larger than L2, ~2 GB): profiler captures
     c["c2_p1"] = c["c2"].scaled("c2_p1", n_layers=18, decode_steps=2)
     c["c3_p1"] = c["c3"].scaled("c3_p1", n_layers=18, decode_steps=2)
+    c["c4_p1"] = c["c4"].scaled("c4_p1", n_layers=18, decode_steps=2)
     return c
 
 
