@@ -173,22 +173,57 @@ __device__ __forceinline__ void merge_row_quad(const uint4 (&ra)[4], const uint4
 }
 
 // 32 consecutive 4-bit codes (16 bytes; channel 2i in the low nibble of byte i) to values
-// code * scale + zero.  `meta` points at the (scale, zero) binary16 pairs: one pair per channel
-// (keys, per_channel) or a single pair for all 32 (values, one group per token).  The nibble becomes a
-// float through the 2^23 trick on the integer pipe (the integer-to-float conversion unit is slow).
-__device__ __forceinline__ void dequant32(const uint4& codes, const uint32_t* meta, bool per_channel, float2 (&out)[16]) {
-  const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
-  float2 sz = Elem<MC_F16>::unpack(meta[0]);
+// code * scale + zero, four channels at a time.  `meta` points at the lane's (scale, zero) binary16 pairs in
+// shared memory: one pair per channel (keys, per_channel) or a single pair for all 32 (values, one group
+// per token).  Position j of the output holds the channels [4 c, 4 c + 4) of the lane's 32 with
+// c = (j + rot) & 7: for the keys the four lanes of a quad read their 32 parameter words from addresses a
+// multiple of 32 words apart, so each lane starts at a different chunk (rot = 2 * lane-in-quad) and the
+// 16-byte loads of a quad fall into different banks; the arithmetic that follows does not care about the
+// order, only the store addresses do.
+// A group of four nibbles becomes two pairs of exact binary16 integers on the way (nibble OR-ed into
+// the mantissa of 1024, 1024 subtracted), and value = code * scale + zero is ONE mixed-precision FMA
+// (binary16 x binary16 + binary32 -> binary32: exact product, one rounding).
+__device__ __forceinline__ float h2f(unsigned short h) {
+  float r;
+  asm("{\n\t.reg .b16 one;\n\tmov.b16 one, 0x3C00;\n\tfma.rn.f32.f16 %0, %1, one, 0f00000000;\n\t}" : "=f"(r) : "h"(h));
+  return r;
+}
+__device__ __forceinline__ float fma_hhf(unsigned short a, unsigned short b, float c) {
+  float r;
+  asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(r) : "h"(a), "h"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ void dequant32(const uint4& codes, const uint32_t* meta, bool per_channel, int rot, float2 (&out)[16]) {
+  const __half2 k1024 = __half2half2(__ushort_as_half((unsigned short)0x6400));
+  unsigned short s_one = 0;
+  float z_one = 0.f;
+  if (!per_channel) {
+    const uint32_t m = meta[0];
+    s_one = (unsigned short)(m & 0xffffu);
+    z_one = h2f((unsigned short)(m >> 16));
+  }
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const uint32_t two = w[i >> 2] >> (8 * (i & 3));
-    const float c0 = __uint_as_float(0x4B000000u | (two & 15u)) - 8388608.0f;
-    const float c1 = __uint_as_float(0x4B000000u | ((two >> 4) & 15u)) - 8388608.0f;
+  for (int j = 0; j < 8; ++j) {
+    const int c = (j + rot) & 7;
+    // the 16 bits of codes of chunk c: half (c & 1) of word (c >> 1)
+    const uint32_t wd = (c & 4) ? ((c & 2) ? codes.w : codes.z) : ((c & 2) ? codes.y : codes.x);
+    const uint32_t h16 = (wd >> ((c & 1) << 4)) & 0xffffu;
+    // nibbles 0, 1 at bits 0 and 16; nibbles 2, 3 at bits 8 and 24: the low half as it is, the high half from a copy
+    // shifted up by 12 bits
+    const uint32_t t = __byte_perm(h16, h16 << 12, 0x7610);
+    uint32_t p01 = (t & 0x000F000Fu) | 0x64006400u, p23 = ((t >> 8) & 0x000F000Fu) | 0x64006400u;
+    const __half2 c01 = __hsub2(*reinterpret_cast<__half2*>(&p01), k1024), c23 = __hsub2(*reinterpret_cast<__half2*>(&p23), k1024);
+    const unsigned short n0 = __half_as_ushort(__low2half(c01)), n1 = __half_as_ushort(__high2half(c01));
+    const unsigned short n2 = __half_as_ushort(__low2half(c23)), n3 = __half_as_ushort(__high2half(c23));
     if (per_channel) {
-      const float2 s0 = Elem<MC_F16>::unpack(meta[2 * i]), s1 = Elem<MC_F16>::unpack(meta[2 * i + 1]);
-      out[i] = make_float2(fmaf(c0, s0.x, s0.y), fmaf(c1, s1.x, s1.y));
+      const uint4 m = *reinterpret_cast<const uint4*>(meta + 4 * c);  // (scale, zero) of the chunk's four channels
+      out[2 * j] = make_float2(fma_hhf(n0, (unsigned short)(m.x & 0xffffu), h2f((unsigned short)(m.x >> 16))),
+                               fma_hhf(n1, (unsigned short)(m.y & 0xffffu), h2f((unsigned short)(m.y >> 16))));
+      out[2 * j + 1] = make_float2(fma_hhf(n2, (unsigned short)(m.z & 0xffffu), h2f((unsigned short)(m.z >> 16))),
+                                   fma_hhf(n3, (unsigned short)(m.w & 0xffffu), h2f((unsigned short)(m.w >> 16))));
     } else {
-      out[i] = make_float2(fmaf(c0, sz.x, sz.y), fmaf(c1, sz.x, sz.y));
+      out[2 * j] = make_float2(fma_hhf(n0, s_one, z_one), fma_hhf(n1, s_one, z_one));
+      out[2 * j + 1] = make_float2(fma_hhf(n2, s_one, z_one), fma_hhf(n3, s_one, z_one));
     }
   }
 }
@@ -344,14 +379,15 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       const uint32_t* ma = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes) + mo;
       const uint32_t* mc = reinterpret_cast<const uint32_t*>(sb + 2 * kQ4CodesBytes + kQ4MetaBytes) + mo;
       float2 a[16], c[16];
-      dequant32(qa, ma, per_channel, a);
-      dequant32(qc, mc, per_channel, c);
+      const int rot = per_channel ? 2 * k : 0;
+      dequant32(qa, ma, per_channel, rot, a);
+      dequant32(qc, mc, per_channel, rot, c);
       if (!valid) {
 #pragma unroll
         for (int x = 0; x < 16; ++x) a[x] = c[x] = make_float2(0.f, 0.f);
       }
 #pragma unroll
-      for (int x = 0; x < 4; ++x) ci[x] = 4 * k + x;
+      for (int x = 0; x < 4; ++x) ci[x] = 4 * k + ((x + (rot >> 1)) & 3);  // output chunk x holds the 8 channels of these two groups
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
       merge_row_core<DT>(a, c, p.ta, p.tc, p.merge_fn, p.t_mode, e, g_a, g_c, d);
