@@ -31,6 +31,8 @@ constexpr int kPfStages = 4;
 constexpr int kPfStageBytes = (kPfTileM + kPfTileN) * kPfTileK * 2;  // X tile, then W tile: 32 KB
 constexpr int kPfThreads = 192;
 constexpr int kPfTmemCols = 128;
+constexpr int kPfEpiRow = kRowBytes + 16;           // a staged row, padded: 32 rows fall into different banks
+constexpr int kPfEpiWarp = 32 * kPfEpiRow;          // staging of one epilogue warp's 32 rows: 8704 bytes
 
 struct PrefillParams {
   Geom g;
@@ -42,6 +44,8 @@ struct PrefillParams {
   int32_t* status;
   int x_seq_stride;  // rows of X per sequence (a multiple of 128)
   int d_model;
+  int n_mtiles;      // token tiles in all: batch * x_seq_stride / 128
+  int mt_group, ht_group, n_htg;  // tile order, see below
   float ta, tc;
   int t_mode;
   float d_hint;
@@ -112,14 +116,25 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kPfStages * kPfStageBytes);  // full[4], empty[4], accum
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPfStages + 1);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned char* epi = smem + kPfStages * kPfStageBytes + 256;  // [4 warps][32 rows][kPfEpiRow]: row staging of the epilogue
   const uint32_t stage0 = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kPfStages, accum_bar = empty0 + 8 * kPfStages;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   const int H = p.g.n_kv_heads;
-  const int tensor = blockIdx.x / H, head = blockIdx.x % H;
+  // Tile order: the CTAs that run at the same time should share operands in L2.  CTAs are numbered in
+  // groups of mt_group token tiles x ht_group (tensor, head) columns -- inside a group the token tile runs
+  // fastest, the groups of one band of token tiles follow each other -- so a group touches mt_group X
+  // tiles and ht_group W slices (a few tens of MB), each used by many of its CTAs, and the X tiles of a
+  // band stay resident while the W slices cycle.
+  const int per_group = p.mt_group * p.ht_group;
+  const int grp = blockIdx.x / per_group, within = blockIdx.x % per_group;
+  const int mt = (grp / p.n_htg) * p.mt_group + within % p.mt_group;
+  const int ht = (grp % p.n_htg) * p.ht_group + within / p.mt_group;
+  if (mt >= p.n_mtiles) return;
+  const int tensor = ht / H, head = ht % H;
   const int tiles_per_seq = p.x_seq_stride / kPfTileM;
-  const int b = blockIdx.y / tiles_per_seq, tile = blockIdx.y % tiles_per_seq;
+  const int b = mt / tiles_per_seq, tile = mt % tiles_per_seq;
   const int tok0 = tile * kPfTileM;
   const int n = checked_len(p.g, b, p.status);
   if (tok0 >= n) return;  // (the whole CTA: nothing has been set up yet)
@@ -173,17 +188,31 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
     }
   } else {
     // ===================== epilogue: one token row per thread =====================
+    // Global memory is touched a row at a time by sixteen lanes (whole 256-byte rows), the arithmetic
+    // wants a row per thread: the rows pass through a padded staging area in shared memory.
     const int q = warp & 3;            // the quarter of the tensor memory's lanes this warp may read
     const int m = q * 32 + lane;       // row of the tile
     const int tok = tok0 + m;
-    const bool ok_wait = mbar_wait(accum_bar, 0, s_abort, p.status);
-    tc_fence_after();
-    const bool live = ok_wait && !*s_abort && tok < n;
     const int ps = p.g.page_size, shift = p.g.page_shift;
     int page = -1;
-    if (live) page = checked_page(p.g, b, tok >> shift, p.status);
+    if (tok < n) page = checked_page(p.g, b, tok >> shift, p.status);
     const int tk = tok & (ps - 1);
-    const size_t prow = ((size_t)max(page, 0) * H + head) * ps + tk;  // row index inside a layer pool
+    const int prow = page >= 0 ? (page * H + head) * ps + tk : -1;  // row index inside a layer pool (-1: no such row)
+    unsigned char* my = epi + q * kPfEpiWarp;
+    const int r_half = lane >> 4, ch16 = lane & 15;
+    // layer l-1's rows go to the staging area while the tensor cores are still busy
+#pragma unroll 4
+    for (int i = 0; i < 16; ++i) {
+      const int r = 2 * i + r_half;
+      const int pr = __shfl_sync(0xffffffffu, prow, r);
+      if (pr >= 0)
+        *reinterpret_cast<uint4*>(my + r * kPfEpiRow + ch16 * 16) =
+            ld_stream16(p.a_pool[tensor] + (size_t)pr * kRowBytes + ch16 * 16);
+    }
+    __syncwarp();
+    const bool ok_wait = mbar_wait(accum_bar, 0, s_abort, p.status);
+    tc_fence_after();
+    const bool live = ok_wait && !*s_abort && prow >= 0;
     // layer l's row: accumulators rounded once to the storage type (what the model would have cached)
     uint32_t cw[64];
 #pragma unroll
@@ -193,18 +222,18 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
 #pragma unroll
       for (int i = 0; i < 16; ++i) cw[j * 16 + i] = Elem<DT>::pack(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
     }
-    float dmin = __int_as_float(0x7f800000), dmax = 0.f;
-    if (live && page >= 0) {
-      const uint4* ap = reinterpret_cast<const uint4*>(p.a_pool[tensor] + prow * kRowBytes);
-      uint32_t aw[64];
+    uint32_t aw[64];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const uint4 v = ap[i];
-        aw[4 * i] = v.x;
-        aw[4 * i + 1] = v.y;
-        aw[4 * i + 2] = v.z;
-        aw[4 * i + 3] = v.w;
-      }
+    for (int i = 0; i < 16; ++i) {
+      const uint4 v = *reinterpret_cast<const uint4*>(my + lane * kPfEpiRow + i * 16);
+      aw[4 * i] = v.x;
+      aw[4 * i + 1] = v.y;
+      aw[4 * i + 2] = v.z;
+      aw[4 * i + 3] = v.w;
+    }
+    __syncwarp();  // every lane holds its row: the staging area is free for the merged rows
+    float dmin = __int_as_float(0x7f800000), dmax = 0.f;
+    if (live) {
       float aa = 0.f, cc = 0.f;
 #pragma unroll
       for (int i = 0; i < 64; ++i) {
@@ -219,8 +248,8 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
       for (int i = 0; i < 64; ++i) {
         const float2 a = Elem<DT>::unpack(aw[i]), c = Elem<DT>::unpack(cw[i]);
         const float ux = a.x * ia, uy = a.y * ia;
-        const float mx = fmaf(-c.x, ic, ux), my = fmaf(-c.y, ic, uy), px = fmaf(c.x, ic, ux), py = fmaf(c.y, ic, uy);
-        sm = fmaf(mx, mx, fmaf(my, my, sm));
+        const float mx = fmaf(-c.x, ic, ux), my_ = fmaf(-c.y, ic, uy), px = fmaf(c.x, ic, ux), py = fmaf(c.y, ic, uy);
+        sm = fmaf(mx, mx, fmaf(my_, my_, sm));
         sp = fmaf(px, px, fmaf(py, py, sp));
       }
       float ta = p.ta, tc = p.tc;
@@ -238,7 +267,7 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
           const float2 r = Elem<DT>::unpack(w[i]);  // the stored value: Eq. 2 divides by its length
           ee = fmaf(r.x, r.x, fmaf(r.y, r.y, ee));
         }
-        *reinterpret_cast<uint4*>(tile_p + tk * kRowBytes + chunk_pos(tk, ch) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(my + lane * kPfEpiRow + ch * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
       const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
       float* scp = reinterpret_cast<float*>(tile_p + ps * kRowBytes) + tk;
@@ -248,9 +277,23 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
       dmin = dmax = s.d;
       // a token that may end up unmerged (Eq. 4) keeps its raw row of layer l
       if (s.d > p.d_hint) {
-        uint4* cp = reinterpret_cast<uint4*>(p.c_pool[tensor] + prow * kRowBytes);
+        uint4* cp = reinterpret_cast<uint4*>(p.c_pool[tensor] + (size_t)prow * kRowBytes);
 #pragma unroll
         for (int i = 0; i < 16; ++i) cp[i] = make_uint4(cw[4 * i], cw[4 * i + 1], cw[4 * i + 2], cw[4 * i + 3]);
+      }
+    }
+    __syncwarp();
+    // the merged rows leave: sixteen lanes per row
+    const int page_live = live ? page : -1;
+#pragma unroll 4
+    for (int i = 0; i < 16; ++i) {
+      const int r = 2 * i + r_half;
+      const int pg = __shfl_sync(0xffffffffu, page_live, r);
+      if (pg >= 0) {
+        const int tk_r = (tok0 + q * 32 + r) & (ps - 1);
+        // (chunk ch16 goes to its place in the tile's chunk order: the sixteen lanes still cover the whole row)
+        st_stream16(p.e_pool[tensor] + ((size_t)pg * H + head) * tile_bytes(ps) + tk_r * kRowBytes + chunk_pos(tk_r, ch16) * 16,
+                    *reinterpret_cast<const uint4*>(my + r * kPfEpiRow + ch16 * 16));
       }
     }
 #pragma unroll
@@ -340,10 +383,17 @@ mc_status launch_prefill_merge(const mc_config* cfg, const mc_batch* bt, const G
   pp.tc = (float)cfg->t;
   pp.t_mode = cfg->t_mode;
   pp.d_hint = d_hint;
-  const size_t smem = 1024 + (size_t)kPfStages * kPfStageBytes + (2 * kPfStages + 1) * 8 + 16;
-  const int tiles = (std::min(bt->max_seq_len, proj->x_seq_stride) + kPfTileM - 1) / kPfTileM;
-  const dim3 grid(2 * cfg->n_kv_heads, bt->batch * (proj->x_seq_stride / kPfTileM));
-  (void)tiles;
+  const size_t smem = 1024 + (size_t)kPfStages * kPfStageBytes + 256 + 4 * (size_t)kPfEpiWarp;  // stages, barriers, row staging
+  pp.n_mtiles = bt->batch * (proj->x_seq_stride / kPfTileM);
+  const int n_ht = 2 * cfg->n_kv_heads;
+  pp.ht_group = 1;
+  for (int dv = 1; dv <= 16; ++dv)
+    if (n_ht % dv == 0) pp.ht_group = dv;  // the largest divisor of the column count up to 16
+  pp.n_htg = n_ht / pp.ht_group;
+  pp.mt_group = std::min(32, pp.n_mtiles);
+  const long long n_ctas = (long long)((pp.n_mtiles + pp.mt_group - 1) / pp.mt_group) * pp.n_htg * pp.mt_group * pp.ht_group;
+  if (n_ctas > 0x7fffffffLL) return MC_ERR_SHAPE;
+  const dim3 grid((unsigned)n_ctas);
   void (*kern)(const PrefillParams, const CUtensorMap, const CUtensorMap, const CUtensorMap) =
       cfg->dtype == MC_F16 ? prefill_merge_kernel<MC_F16> : prefill_merge_kernel<MC_BF16>;
   MC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
