@@ -6,9 +6,9 @@
 //                             residual tile; the page it completes is quantised on the spot
 //   restore_q4_kernel         Eq. 2 + Sec. 4.2 "Cache restoration" from 4-bit tiles and the residual tile
 // The quantiser (scale = (max - min) / 15 and zero = min kept in the 16-bit type, round to nearest,
-// groups of 32: keys per channel over a page's tokens, values per token over 32 channels) runs in
-// double precision: none of this is on a bandwidth-critical path, and the codes are then the same
-// integers on any machine.
+// groups of 32: keys per channel over a page's tokens, values per token over 32 channels) is defined in
+// double precision, so that the codes are the same integers on any machine; the kernels evaluate it in
+// single precision wherever that provably gives the same integer (q4_code) and in double elsewhere.
 #include <algorithm>
 
 #include "mc_common.cuh"
@@ -36,6 +36,16 @@ __device__ __forceinline__ unsigned short deq_one(int code, unsigned short scale
     return __half_as_ushort(__hfma(__int2half_rn(code), __ushort_as_half(scale), __ushort_as_half(zero)));
   }
   return __bfloat16_as_ushort(__hfma(__int2bfloat16_rn(code), __ushort_as_bfloat16(scale), __ushort_as_bfloat16(zero)));
+}
+
+// code = clamp(rint((x - zero) / scale), 0, 15) as the double-precision quantiser defines it, at single-precision
+// cost: the fp32 quotient is within 1e-5 of the exact one (operands of at most 11 significant bits), so it
+// rounds to the same integer unless it lies that close to a tie -- only then is the quotient formed in double.
+__device__ __forceinline__ int q4_code(float x, float z, float s, float inv_s) {
+  const float qf = (x - z) * inv_s;
+  float r = rintf(qf);
+  if (fabsf(fabsf(qf - r) - 0.5f) < 1e-3f) r = (float)rint(((double)x - (double)z) / (double)s);
+  return (int)fminf(fmaxf(r, 0.f), 15.f);
 }
 
 // Shared memory of one tile conversion.
@@ -79,11 +89,8 @@ __device__ void quantise_tile(int tensor, QTileSmem& sm, char* dst) {
     unsigned short s16 = double_to_elem<DT>(((double)hi - (double)lo) / 15.0);
     if (elem_to_float<DT>(s16) == 0.f) s16 = double_to_elem<DT>(1.0);  // a constant group
     const unsigned short z16 = double_to_elem<DT>((double)lo);
-    const double sd = (double)elem_to_float<DT>(s16), zd = (double)elem_to_float<DT>(z16);
-    for (int r = 0; r < kQ4Page; ++r) {
-      const double q = rint(((double)elem_to_float<DT>(sm.rows[r][c]) - zd) / sd);
-      sm.codes[r][c] = (unsigned char)(int)fmin(fmax(q, 0.0), 15.0);
-    }
+    const float sf = elem_to_float<DT>(s16), zf = elem_to_float<DT>(z16), inv_s = 1.0f / sf;
+    for (int r = 0; r < kQ4Page; ++r) sm.codes[r][c] = (unsigned char)q4_code(elem_to_float<DT>(sm.rows[r][c]), zf, sf, inv_s);
     sm.scale[c] = s16;
     sm.zero[c] = z16;
   } else {
@@ -97,11 +104,9 @@ __device__ void quantise_tile(int tensor, QTileSmem& sm, char* dst) {
     unsigned short s16 = double_to_elem<DT>(((double)hi - (double)lo) / 15.0);
     if (elem_to_float<DT>(s16) == 0.f) s16 = double_to_elem<DT>(1.0);
     const unsigned short z16 = double_to_elem<DT>((double)lo);
-    const double sd = (double)elem_to_float<DT>(s16), zd = (double)elem_to_float<DT>(z16);
-    for (int j = 0; j < 32; ++j) {
-      const double q = rint(((double)elem_to_float<DT>(sm.rows[r][32 * g + j]) - zd) / sd);
-      sm.codes[r][32 * g + j] = (unsigned char)(int)fmin(fmax(q, 0.0), 15.0);
-    }
+    const float sf = elem_to_float<DT>(s16), zf = elem_to_float<DT>(z16), inv_s = 1.0f / sf;
+    for (int j = 0; j < 32; ++j)
+      sm.codes[r][32 * g + j] = (unsigned char)q4_code(elem_to_float<DT>(sm.rows[r][32 * g + j]), zf, sf, inv_s);
     sm.scale[r * 4 + g] = s16;
     sm.zero[r * 4 + g] = z16;
   }
