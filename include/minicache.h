@@ -143,6 +143,13 @@ typedef struct mc_config {
                            1: one set per (sequence, head), the union of the two (Sec. 4.2 writes the pair cache
                            with a single I): a token either rule keeps is kept unmerged in both tensors.
                            Not with MC_RETAIN_TOPK. */
+  int32_t append_slack; /* retention of tokens appended during decode (Sec. 4.2 keeps "unmergeable" tokens; Algorithm 2
+                           decides only over the prefill tokens, so this is an extension).  0: an appended token is
+                           always merged.  n > 0: every segment's retained list is laid out with n free entries
+                           behind it when the pair is merged, and mc_append_pair applies Eq. 4 to the new token
+                           with the segment's stored d_min and d_max (the threshold of the prefill tokens,
+                           never recomputed): a token it keeps takes the next free entry.  Threshold modes only
+                           (with MC_RETAIN_TOPK appended tokens are always merged); gamma = 0 keeps nothing. */
 } mc_config;
 
 /* Batch geometry shared by the layer pools and the pair cache. */
@@ -193,7 +200,9 @@ typedef struct mc_layer_q4 {
  * dist       [n_pages][n_kv_heads][2][page_size] fp32 angular distance d = Omega / pi; slot 0: K, 1: V.
  * Retention, per segment seg = (tensor * batch + b) * n_kv_heads + head (tensor 0 = K, 1 = V):
  * ret_count  [2 * batch * n_kv_heads] retained tokens of the segment
- * ret_offset [2 * batch * n_kv_heads + 1] exclusive prefix of ret_count = first slot of the segment
+ * ret_offset [2 * batch * n_kv_heads + 1] first slot of the segment: the exclusive prefix of ret_count, plus
+ *            cfg->append_slack free entries behind every segment's list (their ret_index is -1 until
+ *            mc_append_pair fills them); ret_capacity must cover those too
  * ret_index  [ret_capacity] token indices, ascending inside a segment
  * ret_rows   [2][ret_capacity][272 bytes]: [0] layer l-1, [1] layer l; an entry is the raw 16-bit row
  *            (256 bytes, a bit copy of the input), the token's index (int32) and 12 bytes of padding,
@@ -416,7 +425,12 @@ mc_status mc_merge_pair_q4(const mc_config* cfg, const mc_batch* batch, const mc
 /* Algorithm 2 "MiniCache Decoding", the branch that compresses the step's new token pair:
  * merges k/v_new_lm1 with k/v_new_l ([batch][n_kv_heads][128], 16-bit) by Eq. 3 and writes
  * direction, scales and distance at token position seq_lens[b] of every sequence (the block
- * table must already hold a page for it).  No retention decision is taken for new tokens.
+ * table must already hold a page for it).  With cfg->append_slack == 0 no retention decision is taken
+ * for new tokens.  With cfg->append_slack > 0 (the value the pair was merged with) a new token whose
+ * distance passes Eq. 4 against the segment's stored d_min, d_max (both tensors' rules with
+ * cfg->retain_union) is kept unmerged: its two raw rows go to the next free entry of the segment's
+ * retained list, its scales become -0.0, ret_count, ret_prefix and the retained total are updated.  A
+ * segment whose free entries are used up sets MC_FLAG_RETAIN_OVERFLOW and the token is merged instead.
  * seq_lens is not modified: the caller advances it once all layers of the step are done.
  * cfg->cache_bits = 4: the row goes to slot seq_lens[b] % 32 of the sequence's residual tile; when
  * that fills the page (slot 31) the same kernel quantises the 32 rows into the page's 4-bit tile. */

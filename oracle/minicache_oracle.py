@@ -223,6 +223,18 @@ def retention_indices(d: np.ndarray, gamma: float, mode: str = "distinct") -> np
     raise ValueError(mode)
 
 
+def append_keep(d_new: float, d_prefill: np.ndarray, gamma: float, mode: str = "distinct") -> bool:
+    """Is a token appended during decode kept unmerged?  An extension of Eq. 4 (Algorithm 2 decides only over
+    the prefill tokens): the new token's distance is held against the threshold of its segment's PREFILL
+    distances -- d_min and d_max stay what they were when the pair was merged.  gamma = 0 keeps nothing, an
+    empty prefill segment has no threshold, and the top-k reading has none either."""
+    d_prefill = np.asarray(d_prefill, F64)
+    if not gamma > 0.0 or d_prefill.shape[0] == 0 or mode == "topk":
+        return False
+    thr = retention_threshold(d_prefill, gamma, mode)
+    return bool(d_new > thr) if mode == "distinct" else bool(d_new < thr)
+
+
 # --------------------------------------------------------------------------
 # One layer pair (Algorithm 2, "MiniCache Prefill")
 # --------------------------------------------------------------------------

@@ -37,7 +37,7 @@ class _Config(C.Structure):
     _fields_ = [("n_kv_heads", C.c_int32), ("n_q_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("page_size", C.c_int32), ("dtype", C.c_int32), ("retain_mode", C.c_int32),
                 ("t", C.c_double), ("gamma", C.c_double), ("merge_fn", C.c_int32), ("cache_bits", C.c_int32),
-                ("t_mode", C.c_int32), ("retain_union", C.c_int32)]
+                ("t_mode", C.c_int32), ("retain_union", C.c_int32), ("append_slack", C.c_int32)]
 
 
 class _Batch(C.Structure):
@@ -109,11 +109,13 @@ class McConfig:
     cache_bits: int = 16  # storage of the shared directions: 16 (the 16-bit type) or 4 (4-bit shared cache, pages of 32)
     t_mode: int = 0  # MC_T_FIXED | MC_T_MAGNITUDE_RATIO = 1 (per-token t from the two magnitudes)
     retain_union: int = 0  # 1: one retention set for keys and values (the union of Eq. 4's two sets)
+    append_slack: int = 0  # > 0: free retained entries per segment; appended tokens are held against Eq. 4's stored threshold
 
     def c(self) -> _Config:
         return _Config(self.n_kv_heads, self.n_q_heads, self.head_dim, self.page_size,
                        {"f16": MC_F16, "bf16": MC_BF16}[self.dtype], self.retain_mode, float(self.t), float(self.gamma),
-                       int(self.merge_fn), int(self.cache_bits), int(self.t_mode), int(self.retain_union))
+                       int(self.merge_fn), int(self.cache_bits), int(self.t_mode), int(self.retain_union),
+                       int(self.append_slack))
 
     @property
     def torch_dtype(self):

@@ -59,6 +59,7 @@ static mc_status check_config(const mc_config* cfg) {
   if (cfg->t_mode != MC_T_FIXED && cfg->t_mode != MC_T_MAGNITUDE_RATIO) return MC_ERR_INVALID_ARG;
   if (cfg->retain_union != 0 && cfg->retain_union != 1) return MC_ERR_INVALID_ARG;
   if (cfg->retain_union && cfg->retain_mode == MC_RETAIN_TOPK) return MC_ERR_UNSUPPORTED;
+  if (cfg->append_slack < 0 || cfg->append_slack > 65536) return MC_ERR_INVALID_ARG;
   if (!(cfg->t >= 0.0 && cfg->t <= 1.0) || !(cfg->gamma >= 0.0 && cfg->gamma <= 1.0)) return MC_ERR_INVALID_ARG;
   return MC_OK;
 }
@@ -132,7 +133,7 @@ using namespace mc;
 
 extern "C" {
 
-int32_t mc_version(void) { return 210; }
+int32_t mc_version(void) { return 220; }
 
 int32_t mc_build_flags(void) {
 #if defined(MC_BOUNDS) && MC_BOUNDS

@@ -9,6 +9,7 @@
 #include "mc_kernels.h"
 #include "mc_items.cuh"
 #include "mc_pipe.cuh"
+#include "mc_retain.cuh"
 
 namespace mc {
 
@@ -477,6 +478,7 @@ struct RetainParams {
   int do_retention;
   int union_kv;  // one set for keys and values: a token the other tensor's rule keeps is kept here too
   int region_rows;  // admission: entries of the retained pool each sequence owns (0: one compact list for the batch)
+  int slack;        // free entries behind every segment's list, for tokens kept at decode time
   float d_hint;     // fused prefill: raw layer-l rows exist only for tokens with d > d_hint (< 0: for all)
   double gamma;
 };
@@ -506,7 +508,7 @@ struct RetainPair {
 struct RetainBatch {
   Geom g;
   RetainPair pr[kMaxMergePairs];  // blockIdx.z selects the pair
-  int q4, dtype, chunks_per_seg, nseg, mode, do_retention, union_kv, region_rows;
+  int q4, dtype, chunks_per_seg, nseg, mode, do_retention, union_kv, region_rows, slack;
   float d_hint;  // fused prefill: raw layer-l rows exist only for tokens with d > d_hint (< 0: for all)
   double gamma;
 };
@@ -544,6 +546,7 @@ __device__ __forceinline__ RetainParams retain_view(const RetainBatch& bp, int p
   p.do_retention = bp.do_retention;
   p.union_kv = bp.union_kv;
   p.region_rows = bp.region_rows;
+  p.slack = bp.slack;
   p.d_hint = bp.d_hint;
   p.gamma = bp.gamma;
   return p;
@@ -577,13 +580,6 @@ __global__ void merge_init_kernel(const __grid_constant__ InitParams ip) {
     seg_minmax[2 * seg + 1] = 0u;
   }
   if (ip.clear_status && i < MC_STATUS_WORDS) ip.status[blockIdx.y][i] = 0;
-}
-
-// Retention decision of one token; the threshold is formed in double from the fp32 extremes.
-__device__ __forceinline__ bool keep_token(float d, float dmin, float dmax, double gamma, int mode) {
-  const double lo = dmin, hi = dmax;
-  if (mode == MC_RETAIN_DISTINCT) return (double)d > hi - (hi - lo) * gamma;
-  return (double)d < lo + (hi - lo) * gamma;
 }
 
 // The four consecutive distances of thread `t` of a chunk (tokens tok0 .. tok0 + 3 lie in one page).
@@ -792,7 +788,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
         const int sg = j < per_seq ? ((j / p.chunks_per_seg / p.g.n_kv_heads) * p.g.batch + bq) * p.g.n_kv_heads +
                                          (j / p.chunks_per_seg) % p.g.n_kv_heads : 0;
         const size_t ci = (size_t)sg * p.chunks_per_seg + (j % p.chunks_per_seg);
-        const int v = j < per_seq ? __ldcg(p.chunk_count + ci) : 0;
+        // (the free entries of a segment follow its last chunk's)
+        const int v = j < per_seq ? __ldcg(p.chunk_count + ci) + (j % p.chunks_per_seg == p.chunks_per_seg - 1 ? p.slack : 0) : 0;
         int x = v;
         for (int o = 1; o < 32; o <<= 1) {
           const int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -825,7 +822,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
   const int total = p.nseg * p.chunks_per_seg;
   for (int base = 0; base < total; base += kRetThreads) {
     const int i = base + threadIdx.x;
-    const int v = i < total ? __ldcg(p.chunk_count + i) : 0;
+    const int v = i < total ? __ldcg(p.chunk_count + i) + (i % p.chunks_per_seg == p.chunks_per_seg - 1 ? p.slack : 0) : 0;
     int x = v;
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -847,7 +844,7 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
   if (threadIdx.x == 0) {
     const int sum = s_carry;
     p.ret_offset[p.nseg] = sum;
-    p.status[MC_STATUS_RETAINED_TOTAL] = sum;
+    p.status[MC_STATUS_RETAINED_TOTAL] = sum - p.nseg * p.slack;
     p.status[MC_STATUS_RESERVED1] = 0;
     if ((int64_t)sum > p.ret_capacity) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_RETAIN_OVERFLOW);
   }
@@ -869,8 +866,13 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __gri
   const int seg_off = p.ret_offset[seg];
   // (admission: the scan has written the segment's count, and -1 as the offset of a sequence that did not fit)
   const bool overflow = p.region_rows > 0 ? seg_off < 0 : (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
-  const int seg_cnt = overflow ? 0 : (p.region_rows > 0 ? p.ret_count[seg] : p.ret_offset[seg + 1] - seg_off);
+  const int seg_cnt = overflow ? 0 : (p.region_rows > 0 ? p.ret_count[seg] : p.ret_offset[seg + 1] - seg_off - p.slack);
   if (chunk == 0 && threadIdx.x == 0) p.ret_count[seg] = seg_cnt;
+  if (chunk == 0 && !overflow)  // the free entries behind the list
+    for (int j = threadIdx.x; j < p.slack; j += kRetThreads) {
+      const int64_t pos = (int64_t)seg_off + seg_cnt + j;
+      if (MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) p.ret_index[pos] = -1;
+    }
   int32_t* prefix = p.ret_prefix + (size_t)seg * p.ret_prefix_stride;
   if (chunk == 0)  // table entries past the last chunk: everything lies before them
     for (int j = p.chunks_per_seg * (kChunk / 128) + threadIdx.x; j < p.ret_prefix_stride; j += kRetThreads) prefix[j] = seg_cnt;
@@ -997,6 +999,7 @@ struct AppendParams {
   int t_mode;
   int total_rows;  // 2 * batch * H
   int32_t* status;
+  AppendKeep keep;
 };
 
 template <int DT>
@@ -1031,7 +1034,29 @@ __global__ void __launch_bounds__(128) append_kernel(const AppendParams p) {
   uint4 e;
   float ga, gc, d;
   merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, p.t_mode, e, ga, gc, d);
+  const unsigned half_mask = 0xffffu << (threadIdx.x & 16);
+  bool kept = false;
+  if (p.keep.slack > 0) {  // (uniform over the block)
+    const int seg = (tensor * p.g.batch + b) * H + h;
+    bool keep = ok && page_ok(p.g, page) && append_keeps(p.keep, seg, d);
+    if (p.keep.union_kv) {
+      // one set for keys and values: the other tensor's rule, on its own new rows, counts as well
+      uint4 oa = make_uint4(0, 0, 0, 0), oc = oa;
+      if (ok) {
+        const size_t off = ((size_t)b * H + h) * kRowBytes + l16 * 16;
+        oa = *reinterpret_cast<const uint4*>(p.a_new[1 - tensor] + off);
+        oc = *reinterpret_cast<const uint4*>(p.c_new[1 - tensor] + off);
+      }
+      uint4 e_o;
+      float ga_o, gc_o, d_o;
+      merge_row<DT>(oa, oc, p.ta, p.tc, p.merge_fn, p.t_mode, e_o, ga_o, gc_o, d_o);
+      keep = keep || (ok && page_ok(p.g, page) && append_keeps(p.keep, ((1 - tensor) * p.g.batch + b) * H + h, d_o));
+    }
+    keep = __shfl_sync(half_mask, (int)keep, threadIdx.x & 16) != 0;  // (one decision per half-warp)
+    if (keep) kept = append_retain(p.keep, seg, tok, l16, va, vc, p.status);
+  }
   if (!ok || !page_ok(p.g, page)) return;
+  if (kept) ga = gc = -0.f;  // served from its raw rows (the mark retain_compact_kernel leaves as well)
   const int tk = tok & (p.g.page_size - 1);
   const size_t ph = (size_t)page * H + h;
   char* tile = p.e_pool[tensor] + ph * tile_bytes(p.g.page_size);
@@ -1156,6 +1181,7 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   rb.do_retention = do_retention;
   rb.union_kv = cfg->retain_union;
   rb.region_rows = region_rows;
+  rb.slack = cfg->append_slack;
   rb.d_hint = hook != nullptr ? hook->d_hint : -1.f;
   rb.gamma = cfg->gamma;
   dim3 grid(rb.chunks_per_seg, nseg_call, n_pairs);
@@ -1191,6 +1217,7 @@ mc_status launch_append(const mc_config* cfg, const mc_batch* bt, const Geom& g,
   ap.tc = (float)cfg->t;
   ap.total_rows = 2 * bt->batch * cfg->n_kv_heads;
   ap.status = pair->status;
+  ap.keep = make_append_keep(cfg, pair);
   if (ap.total_rows == 0) return MC_OK;
   const int blocks = (ap.total_rows + 7) / 8;
   if (cfg->dtype == MC_F16)

@@ -14,6 +14,7 @@
 #include "mc_common.cuh"
 #include "mc_kernels.h"
 #include "mc_q4.cuh"
+#include "mc_retain.cuh"
 
 namespace mc {
 
@@ -213,6 +214,7 @@ struct AppendQ4Params {
   int merge_fn;
   int t_mode;
   int32_t* status;
+  AppendKeep keep;
 };
 
 template <int DT>
@@ -242,6 +244,20 @@ __global__ void __launch_bounds__(kQThreads) append_q4_kernel(const AppendQ4Para
     uint4 e;
     float ga, gc, d;
     merge_row<DT>(va, vc, p.ta, p.tc, p.merge_fn, p.t_mode, e, ga, gc, d);
+    if (p.keep.slack > 0) {  // (uniform over the block) Eq. 4 for the new token, against the stored extremes
+      const int seg = (tensor * p.g.batch + b) * H + h;
+      bool keep = append_keeps(p.keep, seg, d);
+      if (p.keep.union_kv) {  // the other tensor's rule, on its own new rows, counts as well
+        const uint4 oa = *reinterpret_cast<const uint4*>(p.a_new[1 - tensor] + off);
+        const uint4 oc = *reinterpret_cast<const uint4*>(p.c_new[1 - tensor] + off);
+        uint4 e_o;
+        float ga_o, gc_o, d_o;
+        merge_row<DT>(oa, oc, p.ta, p.tc, p.merge_fn, p.t_mode, e_o, ga_o, gc_o, d_o);
+        keep = keep || append_keeps(p.keep, ((1 - tensor) * p.g.batch + b) * H + h, d_o);
+      }
+      keep = __shfl_sync(0xffffffffu, (int)keep, 0) != 0;
+      if (keep && threadIdx.x < 16 && append_retain(p.keep, seg, tok, l16, va, vc, p.status)) ga = gc = -0.f;
+    }
     if (threadIdx.x < 16) {
       *reinterpret_cast<uint4*>(res + slot * kRowBytes + chunk_pos(slot, l16) * 16) = e;
       if (l16 == 0) {
@@ -444,6 +460,7 @@ mc_status launch_append_q4(const mc_config* cfg, const mc_batch* bt, const Geom&
   ap.ta = (float)(1.0 - cfg->t);
   ap.tc = (float)cfg->t;
   ap.status = pair->status;
+  ap.keep = make_append_keep(cfg, pair);
   const dim3 grid(2 * cfg->n_kv_heads, bt->batch);
   if (cfg->dtype == MC_F16)
     MC_CUDA_CHECK(launch_pdl(append_q4_kernel<MC_F16>, grid, dim3(kQThreads), 0, stream, ap));

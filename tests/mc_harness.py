@@ -24,7 +24,7 @@ class Problem:
                  retain_mode: int = 0, page_size: Optional[int] = None, decode_room: int = 8,
                  tensors: Optional[Dict[str, torch.Tensor]] = None, ret_capacity: Optional[int] = None,
                  q4: bool = False, merge_fn: str = "slerp", segments=None, cache_bits: int = 16,
-                 t_mode: int = 0, retain_union: int = 0):
+                 t_mode: int = 0, retain_union: int = 0, append_slack: int = 0):
         """segments: list of (sequence, kv head) the oracle will look at; given, the host copies of 4-bit
         layers (exact de-quantised values, fp64) are kept for those segments only (full-size workloads)."""
         import paper_2405_14366_b200 as mc
@@ -54,8 +54,9 @@ class Problem:
         self.merge_fn = merge_fn
         self.cfg = mc.McConfig(self.H, self.Hq, self.ps, cfg.dtype, t=self.t, gamma=self.gamma, retain_mode=retain_mode,
                                merge_fn={"slerp": 0, "fmax": 1, "mean": 2}[merge_fn], cache_bits=cache_bits,
-                               t_mode=t_mode, retain_union=retain_union)
+                               t_mode=t_mode, retain_union=retain_union, append_slack=append_slack)
         self.cache_bits, self.t_mode, self.retain_union = cache_bits, t_mode, retain_union
+        self.append_slack = append_slack
         self.pools = {}
         self.q4 = q4
         self.q4_pools: Dict[str, Dict[str, torch.Tensor]] = {}
@@ -98,7 +99,7 @@ class Problem:
             else:
                 pm = gen.to_paged(meta.reshape(B, S, self.H, 8).to(device), self.block_table, self.ps, n_pages)
             self.q4_pools[name] = {"codes": pc, "meta": pm.contiguous()}
-        total = int(self.seq_lens_host.sum()) * self.H * 2
+        total = int(self.seq_lens_host.sum()) * self.H * 2 + 2 * B * self.H * append_slack
         self.ret_capacity = total if ret_capacity is None else ret_capacity
         self.pair = mc.PairCache(self.cfg, B, n_pages, self.ret_capacity, device=device)
         if q4:  # the rows the cache can hold: the de-quantised values rounded once to the storage type

@@ -662,3 +662,27 @@ def test_retention_union_brute_force():
     empty = {k: np.zeros(0, np.int64) for k in rk}
     assert all(np.array_equal(orc.retention_union(rk, empty)[k], rk[k]) for k in rk)
     assert all(np.array_equal(orc.retention_union(rk, rk)[k], rk[k]) for k in rk)
+
+
+def test_append_keep_hand_values_and_prefill_consistency():
+    """The decode-time retention decision: hand-applied Eq. 4 on dyadic distances (the prefill extremes are
+    0.125 and 0.875, gamma = 0.25: thresholds 0.6875 for the similarity reading and 0.3125 for the literal
+    one), and a brute-force link to the prefill rule: a new token with the distance of prefill token i is
+    kept exactly when i was."""
+    d = np.array([0.125, 0.5, 0.875, 0.25, 0.75])
+    assert orc.append_keep(0.75, d, 0.25, "distinct") and not orc.append_keep(0.6875, d, 0.25, "distinct")
+    assert not orc.append_keep(0.5, d, 0.25, "distinct")
+    assert orc.append_keep(0.25, d, 0.25, "literal") and not orc.append_keep(0.3125, d, 0.25, "literal")
+    assert not orc.append_keep(0.5, d, 0.25, "literal")
+    # beyond the prefill extremes: the stored threshold still decides, the extremes do not move
+    assert orc.append_keep(0.99, d, 0.25, "distinct") and orc.append_keep(0.01, d, 0.25, "literal")
+    # nothing is kept with gamma = 0, without prefill tokens, or under the top-k reading
+    assert not orc.append_keep(0.99, d, 0.0, "distinct") and not orc.append_keep(0.01, d, 0.0, "literal")
+    assert not orc.append_keep(0.99, np.zeros(0), 0.25, "distinct")
+    assert not orc.append_keep(0.99, d, 0.25, "topk")
+    rs = np.random.RandomState(77)
+    for mode in ("distinct", "literal"):
+        dd = rs.rand(200)
+        kept = set(orc.retention_indices(dd, 0.2, mode).tolist())
+        for i in range(200):
+            assert orc.append_keep(dd[i], dd, 0.2, mode) == (i in kept)
