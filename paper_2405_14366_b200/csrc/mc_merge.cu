@@ -323,9 +323,26 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
   }
 
   const int quad = tid >> 2, k = tid & 3;
-  long long run_seg = -1;  // segment of the warp's running distance extremes (pairs counted through)
+  // Distance extremes: every lane keeps the running d_min / d_max of its own rows while the warp's items
+  // keep falling into the same segment (consecutive items of a CTA usually do: all CTAs work on one
+  // sequence at a time); only when the segment changes are the lanes reduced and one atomic pair sent.
+  // (One atomic pair per warp and item on a segment's few addresses queues up in the memory system, and
+  // a per-item warp reduction is a chain of shuffles at the end of every item.)
+  int run_key = -1;             // (slot, sequence, head) of the running extremes
   unsigned* run_ptr = nullptr;  // its d_min / d_max words
-  float run_min = 0.f, run_max = 0.f;
+  float run_min = __int_as_float(0x7f800000), run_max = 0.f;
+  auto flush_extremes = [&]() {
+    if (run_key < 0) return;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      run_min = fminf(run_min, __shfl_xor_sync(0xffffffffu, run_min, o));
+      run_max = fmaxf(run_max, __shfl_xor_sync(0xffffffffu, run_max, o));
+    }
+    if (lane == 0 && run_min != __int_as_float(0x7f800000)) {  // (some row of the run was a cached token)
+      atomicMin(run_ptr, __float_as_uint(run_min));
+      atomicMax(run_ptr + 1, __float_as_uint(run_max));
+    }
+  };
   for (int it = 0; m.tensor < n_slots; ++it) {
     if (warp == 0) {
       // item it + 2 goes into the stage that item it - 1 has just left
@@ -393,7 +410,6 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
       merge_row_core<DT>(a, c, p.ta, p.tc, p.merge_fn, p.t_mode, e, g_a, g_c, d);
     }
-    float dmin = __int_as_float(0x7f800000), dmax = 0.f;
     if (valid) {
       char* tile = P.e_pool[ts] + ((size_t)page * H + head) * tile_bytes(ps);
 #pragma unroll
@@ -404,40 +420,26 @@ __global__ void __launch_bounds__(kMergeThreads, kMergeCtasPerSm) merge_kernel(c
         scp[ps] = g_c;
         P.dist[(((size_t)page * H + head) * 2 + ts) * ps + tk] = d;
       }
-      dmin = d;
-      dmax = d;
     }
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-      dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
-      dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
-    }
-    if (dmin != __int_as_float(0x7f800000)) {  // the warp's 8 rows belong to one head
-      // Running extremes stay in registers while the warp's items keep falling into the same segment
-      // (consecutive items of a CTA usually do): all CTAs work on one sequence at a time, and one
-      // atomic pair per warp and item on its few addresses queues up in the memory system.
-      const int seg_local = (ts * p.g.batch + m.b) * H + ((m.grp * kRowsPerItem + warp * 8) >> p.g.page_shift);
-      const long long seg = (long long)(m.tensor >> 1) * (2LL * p.g.batch * H) + seg_local;
-      if (seg != run_seg) {
-        if (lane == 0 && run_seg >= 0) {
-          atomicMin(run_ptr, __float_as_uint(run_min));
-          atomicMax(run_ptr + 1, __float_as_uint(run_max));
-        }
-        run_seg = seg;
-        run_ptr = P.seg_minmax + 2 * seg_local;
-        run_min = dmin;
-        run_max = dmax;
-      } else {
-        run_min = fminf(run_min, dmin);
-        run_max = fmaxf(run_max, dmax);
+    const int row_w = m.grp * kRowsPerItem + warp * 8;  // the warp's 8 rows lie in one head
+    if (row_w < rows_in_page) {
+      const int head_w = row_w >> p.g.page_shift;
+      const int key = (m.tensor * p.g.batch + m.b) * H + head_w;
+      if (key != run_key) {
+        flush_extremes();
+        run_key = key;
+        run_ptr = P.seg_minmax + 2 * ((ts * p.g.batch + m.b) * H + head_w);
+        run_min = __int_as_float(0x7f800000);
+        run_max = 0.f;
+      }
+      if (valid) {
+        run_min = fminf(run_min, d);
+        run_max = fmaxf(run_max, d);
       }
     }
     page_item_advance(m, s_pg, s_grp, ipp, P_all, pre_s, n_slots);
   }
-  if (lane == 0 && run_seg >= 0) {
-    atomicMin(run_ptr, __float_as_uint(run_min));
-    atomicMax(run_ptr + 1, __float_as_uint(run_max));
-  }
+  flush_extremes();
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
   }
