@@ -584,7 +584,7 @@ __global__ void merge_init_kernel(const __grid_constant__ InitParams ip) {
   if (ip.clear_status && i < MC_STATUS_WORDS) ip.status[blockIdx.y][i] = 0;
 }
 
-// The four consecutive distances of thread `t` of a chunk (tokens tok0 .. tok0 + 3 lie in one page).
+// The four consecutive distances starting at token tok0 (a multiple of 4: they lie in one page).
 __device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, int b, int h, int tok0, bool& ok) {
   const int page = checked_page(p.g, b, tok0 >> p.g.page_shift, p.status);
   ok = page >= 0;
@@ -593,52 +593,140 @@ __device__ __forceinline__ float4 load_dist4(const RetainParams& p, int tensor, 
       p.dist + (((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (tok0 & (p.g.page_size - 1)));
 }
 
-// Masks over the thread's four tokens: `sure` = kept whatever the ties do, `eq` = kept only while the
-// segment's quota of ties lasts (top-k mode: d equal to the k-th largest; ties go to lower indices).
-// `near` counts the tokens whose distance lies within 1e-6 of the decision threshold: the ones a
-// different rounding of d could have decided the other way.
-__device__ __forceinline__ void keep_masks4_one(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
-                                                unsigned& sure, unsigned& eq, int* near) {
-  sure = eq = 0u;
-  if (tok0 >= n) return;
-  bool ok;
-  const float4 d4 = load_dist4(p, tensor, b, h, tok0, ok);
-  if (!ok) return;
-  const float d[4] = {d4.x, d4.y, d4.z, d4.w};
-  if (p.mode == MC_RETAIN_TOPK) {
-    const uint32_t v = p.seg_sel[2 * seg];
+// The retention passes give a chunk of 1024 tokens to one warp: lane l owns the 32 consecutive tokens
+// [32 l, 32 l + 32) of the chunk, i.e. one or two pages' worth of distances (pages hold at least 16 tokens).
+struct Dist32 {
+  float4 d[8];
+  unsigned ok;   // bit i: d[i] was loaded (its tokens exist and their page id is valid)
+  int page[2];   // page of the lane's first and second 16 tokens (-1: none)
+};
+__device__ __forceinline__ void load_dist32(const RetainParams& p, int tensor, int b, int h, int tok0, int n, Dist32& r) {
+  r.ok = 0u;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (tok0 + j < n) {
-        const uint32_t key = __float_as_uint(d[j]);
-        if (key > v) sure |= 1u << j;
-        if (key == v) eq |= 1u << j;
-        if (near && v != 0xffffffffu && fabs((double)d[j] - (double)__uint_as_float(v)) < 1e-6) ++*near;
-      }
+  for (int hf = 0; hf < 2; ++hf) {
+    const int t = tok0 + 16 * hf;
+    r.page[hf] = t < n ? checked_page(p.g, b, t >> p.g.page_shift, p.status) : -1;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int t = tok0 + 4 * i;
+    const int page = r.page[i >> 2];
+    r.d[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (t < n && page >= 0) {
+      r.d[i] = *reinterpret_cast<const float4*>(
+          p.dist + (((size_t)page * p.g.n_kv_heads + h) * 2 + tensor) * p.g.page_size + (t & (p.g.page_size - 1)));
+      r.ok |= 1u << i;
     }
-  } else {
-    const float dmin = p.seg_minmax[2 * seg], dmax = p.seg_minmax[2 * seg + 1];
-    const double lo = dmin, hi = dmax;
-    const double thr = p.mode == MC_RETAIN_DISTINCT ? hi - (hi - lo) * p.gamma : lo + (hi - lo) * p.gamma;
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (tok0 + j < n) {
-        if (keep_token(d[j], dmin, dmax, p.gamma, p.mode)) sure |= 1u << j;
-        if (near && fabs((double)d[j] - thr) < 1e-6) ++*near;
-      }
   }
 }
 
-// The decision for the thread's four tokens of segment (tensor, b, h).  With one set for keys and values
-// (union_kv; threshold modes only) the other tensor's rule is applied to its own distances as well and
-// the two masks are joined; `near` counts this tensor's own near-threshold tokens either way.
-__device__ __forceinline__ void keep_masks4(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
-                                            unsigned& sure, unsigned& eq, int* near = nullptr) {
-  keep_masks4_one(p, seg, tensor, b, h, tok0, n, sure, eq, near);
+// Eq. 4's decision as single-precision comparisons.  The rule is defined on the double-precision
+// threshold thr formed from the fp32 extremes ((double)d > thr, or < thr as printed); for a binary32 d that
+// is the same as d > round_down(thr) (d < round_up(thr)), and |d - thr| < 1e-6 is the same as
+// round_down(thr - 1e-6) < d < round_up(thr + 1e-6).  Top-k reading: the k-th largest distance's bits
+// decide (d >= 0, so unsigned order is float order).
+struct KeepRule {
+  int kind;  // 0: d > cmp, 1: d < cmp, 2: top-k
+  float cmp, near_lo, near_hi;
+  uint32_t v;
+};
+__device__ __forceinline__ KeepRule make_rule(const RetainParams& p, int seg) {
+  KeepRule r;
+  r.v = 0u;
+  double thr;
+  if (p.mode == MC_RETAIN_TOPK) {
+    r.kind = 2;
+    r.v = p.seg_sel[2 * seg];
+    thr = (double)__uint_as_float(r.v);
+    r.cmp = 0.f;
+    if (r.v == 0xffffffffu) thr = -4.0;  // nothing is kept: nothing is near either (d lies in [0, 1])
+  } else {
+    const double lo = p.seg_minmax[2 * seg], hi = p.seg_minmax[2 * seg + 1];
+    if (p.mode == MC_RETAIN_DISTINCT) {
+      r.kind = 0;
+      thr = hi - (hi - lo) * p.gamma;
+      r.cmp = __double2float_rd(thr);
+    } else {
+      r.kind = 1;
+      thr = lo + (hi - lo) * p.gamma;
+      r.cmp = __double2float_ru(thr);
+    }
+  }
+  r.near_lo = __double2float_rd(thr - 1e-6);
+  r.near_hi = __double2float_ru(thr + 1e-6);
+  return r;
+}
+// Masks over the lane's 32 tokens (bit 4 i + j = token tok0 + 4 i + j): `sure` = kept whatever the ties do,
+// `eq` = kept only while the segment's quota of ties lasts (top-k reading: d equal to the k-th largest; ties
+// go to lower indices).  `near` counts the tokens whose distance lies within 1e-6 of the decision
+// threshold: the ones a different rounding of d could have decided the other way.
+__device__ __forceinline__ void keep_masks32_one(const KeepRule& r, const Dist32& dd, int tok0, int n, unsigned& sure, unsigned& eq,
+                                                 int* near) {
+  sure = eq = 0u;
+  unsigned nr = 0u;
+  // (one loop per rule: the rule is the same for the whole launch, the loop bodies stay a few instructions per token)
+  if (r.kind == 2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float d[4] = {dd.d[i].x, dd.d[i].y, dd.d[i].z, dd.d[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t key = __float_as_uint(d[j]);
+        sure |= (key > r.v ? 1u : 0u) << (4 * i + j);
+        eq |= (key == r.v ? 1u : 0u) << (4 * i + j);
+      }
+    }
+  } else if (r.kind == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float d[4] = {dd.d[i].x, dd.d[i].y, dd.d[i].z, dd.d[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sure |= (d[j] > r.cmp ? 1u : 0u) << (4 * i + j);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float d[4] = {dd.d[i].x, dd.d[i].y, dd.d[i].z, dd.d[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sure |= (d[j] < r.cmp ? 1u : 0u) << (4 * i + j);
+    }
+  }
+  // tokens that exist (before the sequence's end, in a page with a valid id)
+  unsigned valid = 0u;
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (dd.ok & (1u << i)) valid |= 0xFu << (4 * i);
+  const int left = n - tok0;
+  valid &= left >= 32 ? 0xffffffffu : (left > 0 ? (1u << left) - 1u : 0u);
+  sure &= valid;
+  eq &= valid;
+  if (near) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float d[4] = {dd.d[i].x, dd.d[i].y, dd.d[i].z, dd.d[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) nr |= (d[j] > r.near_lo && d[j] < r.near_hi ? 1u : 0u) << (4 * i + j);
+    }
+    *near += __popc(nr & valid);
+  }
+}
+
+// The decision for the lane's 32 tokens of segment (tensor, b, h), distances included.  With one set for keys
+// and values (union_kv; threshold modes only) the other tensor's rule is applied to its own distances as
+// well and the two masks are joined; `near` counts this tensor's own near-threshold tokens either way.
+// `page` receives the pages of the lane's first and second 16 tokens.
+__device__ __forceinline__ void keep_masks32(const RetainParams& p, int seg, int tensor, int b, int h, int tok0, int n,
+                                             unsigned& sure, unsigned& eq, int (&page)[2], int* near = nullptr) {
+  Dist32 dd;
+  load_dist32(p, tensor, b, h, tok0, n, dd);
+  page[0] = dd.page[0];
+  page[1] = dd.page[1];
+  keep_masks32_one(make_rule(p, seg), dd, tok0, n, sure, eq, near);
   if (p.union_kv && p.mode != MC_RETAIN_TOPK) {
     const int seg_o = tensor ? seg - p.g.batch * p.g.n_kv_heads : seg + p.g.batch * p.g.n_kv_heads;
     unsigned sure_o, eq_o;
-    keep_masks4_one(p, seg_o, 1 - tensor, b, h, tok0, n, sure_o, eq_o, nullptr);
+    load_dist32(p, 1 - tensor, b, h, tok0, n, dd);
+    keep_masks32_one(make_rule(p, seg_o), dd, tok0, n, sure_o, eq_o, nullptr);
     sure |= sure_o;
   }
 }
@@ -703,54 +791,54 @@ __global__ void __launch_bounds__(kRetThreads) retain_select_kernel(const __grid
   }
 }
 
-// Per (segment, 1024-token chunk): how many tokens Eq. 4 keeps.  The block that finishes last
+// Per (segment, 1024-token chunk): how many tokens Eq. 4 keeps; one warp per chunk (a lane looks at 32
+// consecutive tokens), eight chunks per block in (segment, chunk) order.  The block that finishes last
 // (ticket in a status word) turns the counts into offsets: exclusive scan in (segment, chunk) order.
 __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_constant__ RetainBatch bp) {
   grid_dep_wait();
   grid_dep_launch();
   const RetainParams p = retain_view(bp, blockIdx.z);
-  __shared__ int s_cnt[kRetThreads / 32], s_eq[kRetThreads / 32];
+  __shared__ int s_cnt[kRetThreads / 32];
   __shared__ int s_last;
   __shared__ int s_carry;
-  const int chunk = blockIdx.x;
-  int tensor, b, h;
-  const int seg = call_segment(p.g, blockIdx.y, tensor, b, h);
-  const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int cnt = 0, cnt_eq = 0, cnt_near = 0;
-  if (p.do_retention && chunk * kChunk < n) {
-    unsigned sure, eq;
-    keep_masks4(p, seg, tensor, b, h, chunk * kChunk + 4 * threadIdx.x, n, sure, eq, &cnt_near);
-    cnt = __popc(sure);
-    cnt_eq = __popc(eq);
-  }
-  for (int o = 16; o; o >>= 1) {
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, o);
-    cnt_near += __shfl_xor_sync(0xffffffffu, cnt_near, o);
-  }
-  if (lane == 0 && cnt_near) atomicAdd(&p.status[MC_STATUS_NEAR_THRESHOLD], cnt_near);
-  if (chunk == 0 && threadIdx.x == 0 && p.do_retention && p.d_hint >= 0.f && n > 0 && p.mode == MC_RETAIN_DISTINCT) {
-    // fused prefill: every token this segment keeps must be one whose raw row was stored (d > d_hint)
-    const double lo = p.seg_minmax[2 * seg], hi = p.seg_minmax[2 * seg + 1];
-    if (hi - (hi - lo) * p.gamma < (double)p.d_hint && hi > lo && p.gamma > 0.0) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_HINT_TOO_HIGH);
-  }
-  if (lane == 0) {
-    s_cnt[warp] = cnt;
-    s_eq[warp] = cnt_eq;
+  const int n_items = 2 * p.g.seq_count * p.g.n_kv_heads * p.chunks_per_seg;
+  const int item = blockIdx.x * (kRetThreads / 32) + warp;
+  if (item < n_items) {  // (warp-uniform)
+    const int chunk = item % p.chunks_per_seg;
+    int tensor, b, h;
+    const int seg = call_segment(p.g, item / p.chunks_per_seg, tensor, b, h);
+    const int n = checked_len(p.g, b, p.status);
+    int cnt = 0, cnt_eq = 0, cnt_near = 0;
+    if (p.do_retention && chunk * kChunk < n) {
+      unsigned sure, eq;
+      int page[2];
+      keep_masks32(p, seg, tensor, b, h, chunk * kChunk + 32 * lane, n, sure, eq, page, &cnt_near);
+      cnt = __popc(sure);
+      cnt_eq = __popc(eq);
+    }
+    for (int o = 16; o; o >>= 1) {
+      cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+      cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, o);
+      cnt_near += __shfl_xor_sync(0xffffffffu, cnt_near, o);
+    }
+    if (lane == 0) {
+      p.chunk_count[(size_t)seg * p.chunks_per_seg + chunk] = cnt;
+      p.chunk_eq[(size_t)seg * p.chunks_per_seg + chunk] = cnt_eq;
+      if (cnt_near) atomicAdd(&p.status[MC_STATUS_NEAR_THRESHOLD], cnt_near);
+      if (chunk == 0 && p.do_retention && p.d_hint >= 0.f && n > 0 && p.mode == MC_RETAIN_DISTINCT) {
+        // fused prefill: every token this segment keeps must be one whose raw row was stored (d > d_hint)
+        const double lo = p.seg_minmax[2 * seg], hi = p.seg_minmax[2 * seg + 1];
+        if (hi - (hi - lo) * p.gamma < (double)p.d_hint && hi > lo && p.gamma > 0.0) atomicOr(&p.status[MC_STATUS_FLAGS], MC_FLAG_HINT_TOO_HIGH);
+      }
+      __threadfence();  // the counts, before this block's ticket
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    int t = 0, te = 0;
-    for (int w = 0; w < kRetThreads / 32; ++w) {
-      t += s_cnt[w];
-      te += s_eq[w];
-    }
-    p.chunk_count[(size_t)seg * p.chunks_per_seg + chunk] = t;
-    p.chunk_eq[(size_t)seg * p.chunks_per_seg + chunk] = te;
     __threadfence();
     const int ticket = atomicAdd(&p.status[MC_STATUS_RESERVED1], 1);
-    s_last = ticket == (int)(gridDim.x * gridDim.y) - 1;
+    s_last = ticket == (int)gridDim.x - 1;
     s_carry = 0;
   }
   __syncthreads();
@@ -852,44 +940,50 @@ __global__ void __launch_bounds__(kRetThreads) retain_count_kernel(const __grid_
   }
 }
 
-// Per (segment, chunk): ordered compaction of the kept token indices, their scales zeroed, bit copies
-// of both layers' rows, and the chunk's eight entries of the prefix table (one per 128 tokens =
-// one warp).  Writes ret_count per segment.
+// Per (segment, chunk), one warp each: ordered compaction of the kept token indices, their scales zeroed,
+// bit copies of both layers' rows, and the chunk's eight entries of the prefix table (one per 128 tokens =
+// four lanes).  Writes ret_count per segment.
 __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __grid_constant__ RetainBatch bp) {
   grid_dep_wait();
   grid_dep_launch();
   const RetainParams p = retain_view(bp, blockIdx.z);
-  __shared__ int s_warp[kRetThreads / 32];
-  const int chunk = blockIdx.x;
-  int tensor, b, h;
-  const int seg = call_segment(p.g, blockIdx.y, tensor, b, h);
-  const int n = checked_len(p.g, b, p.status);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_items = 2 * p.g.seq_count * p.g.n_kv_heads * p.chunks_per_seg;
+  const int item = blockIdx.x * (kRetThreads / 32) + warp;
+  if (item >= n_items) return;  // (no block-wide barrier below)
+  const int chunk = item % p.chunks_per_seg;
+  int tensor, b, h;
+  const int seg = call_segment(p.g, item / p.chunks_per_seg, tensor, b, h);
+  const int n = checked_len(p.g, b, p.status);
   const int seg_off = p.ret_offset[seg];
   // (admission: the scan has written the segment's count, and -1 as the offset of a sequence that did not fit)
   const bool overflow = p.region_rows > 0 ? seg_off < 0 : (int64_t)p.ret_offset[p.nseg] > p.ret_capacity;
   const int seg_cnt = overflow ? 0 : (p.region_rows > 0 ? p.ret_count[seg] : p.ret_offset[seg + 1] - seg_off - p.slack);
-  if (chunk == 0 && threadIdx.x == 0) p.ret_count[seg] = seg_cnt;
-  if (chunk == 0 && !overflow)  // the free entries behind the list
-    for (int j = threadIdx.x; j < p.slack; j += kRetThreads) {
-      const int64_t pos = (int64_t)seg_off + seg_cnt + j;
-      if (MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) p.ret_index[pos] = -1;
-    }
   int32_t* prefix = p.ret_prefix + (size_t)seg * p.ret_prefix_stride;
-  if (chunk == 0)  // table entries past the last chunk: everything lies before them
-    for (int j = p.chunks_per_seg * (kChunk / 128) + threadIdx.x; j < p.ret_prefix_stride; j += kRetThreads) prefix[j] = seg_cnt;
-  const int pj = chunk * (kChunk / 128) + warp;  // this warp's 128 tokens start at table entry pj
+  if (chunk == 0) {
+    __syncwarp();  // (every lane has read ret_count)
+    if (lane == 0) p.ret_count[seg] = seg_cnt;
+    if (!overflow)  // the free entries behind the list
+      for (int j = lane; j < p.slack; j += 32) {
+        const int64_t pos = (int64_t)seg_off + seg_cnt + j;
+        if (MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) p.ret_index[pos] = -1;
+      }
+    // table entries past the last chunk: everything lies before them
+    for (int j = p.chunks_per_seg * (kChunk / 128) + lane; j < p.ret_prefix_stride; j += 32) prefix[j] = seg_cnt;
+  }
+  const int pj = chunk * (kChunk / 128) + (lane >> 2);  // the table entry of the lane's 128 tokens
   const bool active = !overflow && p.do_retention && chunk * kChunk < n;
   if (!active) {
-    if (lane == 0 && pj < p.ret_prefix_stride) prefix[pj] = seg_cnt;  // chunk past the sequence (or nothing retained)
+    if ((lane & 3) == 0 && pj < p.ret_prefix_stride) prefix[pj] = seg_cnt;  // chunk past the sequence (or nothing retained)
     return;
   }
   const size_t ci = (size_t)seg * p.chunks_per_seg + chunk;
   const int my_count = p.chunk_count[ci];
   const int out0 = p.chunk_offset[ci];
-  const int tok0 = chunk * kChunk + 4 * threadIdx.x;
+  const int tok0 = chunk * kChunk + 32 * lane;
   unsigned m, m_eq;
-  keep_masks4(p, seg, tensor, b, h, tok0, n, m, m_eq);
+  int page[2];
+  keep_masks32(p, seg, tensor, b, h, tok0, n, m, m_eq, page);
   if (p.mode == MC_RETAIN_TOPK) {
     // ties: kept while the segment's quota lasts, in token order (ordered count of the ties before each)
     const int ce = __popc(m_eq);
@@ -898,18 +992,12 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __gri
       const int y = __shfl_up_sync(0xffffffffu, xe, o);
       if (lane >= o) xe += y;
     }
-    if (lane == 31) s_warp[warp] = xe;
-    __syncthreads();
     int seen = p.chunk_eq[ci] + xe - ce;
-    for (int w = 0; w < warp; ++w) seen += s_warp[w];
     const int quota = (int)p.seg_sel[2 * seg + 1];
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (m_eq & (1u << j)) {
-        if (seen < quota) m |= 1u << j;
-        ++seen;
-      }
-    __syncthreads();
+    for (unsigned rest = m_eq; rest; rest &= rest - 1) {
+      if (seen < quota) m |= rest & (0u - rest);
+      ++seen;
+    }
   }
   const int c = __popc(m);
   int x = c;
@@ -917,47 +1005,67 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __gri
     const int y = __shfl_up_sync(0xffffffffu, x, o);
     if (lane >= o) x += y;
   }
-  if (lane == 31) s_warp[warp] = x;
-  __syncthreads();
-  int before = 0;
-  for (int w = 0; w < warp; ++w) before += s_warp[w];
-  if (lane == 0 && pj < p.ret_prefix_stride) prefix[pj] = out0 - seg_off + before;
-  int pos = out0 + before + x - c;
-  if (m) {  // (kept tokens lie in a page that keep_masks4 has checked)
-    const int page = p.g.block_table[(size_t)b * p.g.max_pages_per_seq + (tok0 >> p.g.page_shift)];
-    float* sc = reinterpret_cast<float*>((tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)page * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
-                                         p.g.page_size * kRowBytes) + (tok0 & (p.g.page_size - 1));
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (m & (1u << j)) {
-        if (!MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) continue;  // (range-checked build)
-        p.ret_index[pos++] = tok0 + j;
-        // a retained token is served from its raw rows: the scale -0 makes the shared direction
-        // contribute nothing for it wherever scales are applied blindly, and tells the attention
-        // kernel that the token's score comes from its raw key row
-        sc[j] = -0.f;
-        sc[p.g.page_size + j] = -0.f;
-      }
-    }
+  if ((lane & 3) == 0 && pj < p.ret_prefix_stride) prefix[pj] = out0 - seg_off + x - c;
+  int pos = out0 + x - c;
+  for (unsigned rest = m; rest; rest &= rest - 1) {  // (kept tokens lie in a page that keep_masks32 has checked)
+    const int j = __ffs(rest) - 1;
+    const int tok = tok0 + j;
+    float* sc = reinterpret_cast<float*>((tensor ? p.e_pool[1] : p.e_pool[0]) + ((size_t)((j >> 4) ? page[1] : page[0]) * p.g.n_kv_heads + h) * tile_bytes(p.g.page_size) +
+                                         p.g.page_size * kRowBytes) + (tok & (p.g.page_size - 1));
+    if (!MC_IN_BOUNDS(pos >= 0 && pos < p.ret_capacity, p.status)) continue;  // (range-checked build)
+    p.ret_index[pos++] = tok;
+    // a retained token is served from its raw rows: the scale -0 makes the shared direction
+    // contribute nothing for it wherever scales are applied blindly, and tells the attention
+    // kernel that the token's score comes from its raw key row
+    sc[0] = -0.f;
+    sc[p.g.page_size] = -0.f;
   }
-  __syncthreads();
-  // gather: one half-warp per (entry, layer): the raw row and the token index behind it
-  const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-  for (int r = hw; r < my_count * 2; r += kRetThreads / 16) {
-    const int ent = r >> 1, layer = r & 1;
-    if (!MC_IN_BOUNDS(out0 >= 0 && (int64_t)out0 + ent < p.ret_capacity, p.status)) continue;  // (range-checked build)
-    const int tok = p.ret_index[out0 + ent];
-    const int page = checked_page(p.g, b, tok >> p.g.page_shift, p.status);
-    if (page < 0) continue;
-    const size_t row = ((size_t)page * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
-    char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + ent) * kRetEntryBytes;
+  // gather: the warp copies both layers' raw rows of one entry at a time (a half-warp per layer), four
+  // entries in flight.  Which token an entry is comes from the lane that kept it (its mask and its pages),
+  // not from memory: the copies of different entries do not wait on one another.
+  const int layer = lane >> 4, l16 = lane & 15;
+  const int excl = x - c;
+  const char* pool = layer ? (tensor ? p.c_pool[1] : p.c_pool[0]) : (tensor ? p.a_pool[1] : p.a_pool[0]);
+  for (int e0 = 0; e0 < my_count; e0 += 4) {
+    int tok_u[4];
+    size_t row_u[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + u;
+      const bool mine = e >= excl && e < excl + c;
+      const unsigned own = __ballot_sync(0xffffffffu, mine);
+      const int src = own ? __ffs(own) - 1 : 0;
+      const int j = __shfl_sync(0xffffffffu, mine ? (int)__fns(m, 0, e - excl + 1) : 0, src);
+      const int pg0 = __shfl_sync(0xffffffffu, page[0], src), pg1 = __shfl_sync(0xffffffffu, page[1], src);
+      const int tok = chunk * kChunk + 32 * src + j;
+      const int pg = (j >> 4) ? pg1 : pg0;
+      // (an entry past the lanes' kept tokens, or past the pool in the range-checked build, is skipped)
+      const bool ok = own != 0u && e < my_count && pg >= 0 && MC_IN_BOUNDS(out0 >= 0 && (int64_t)out0 + e < p.ret_capacity, p.status);
+      tok_u[u] = ok ? tok : -1;
+      row_u[u] = ((size_t)max(pg, 0) * p.g.n_kv_heads + h) * p.g.page_size + (tok & (p.g.page_size - 1));
+    }
     if (!p.q4) {
-      const char* src = (layer ? (tensor ? p.c_pool[1] : p.c_pool[0]) : (tensor ? p.a_pool[1] : p.a_pool[0])) + row * kRowBytes + l16 * 16;
-      *reinterpret_cast<uint4*>(dst + l16 * 16) = *reinterpret_cast<const uint4*>(src);
-    } else {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (tok_u[u] >= 0) v[u] = *reinterpret_cast<const uint4*>(pool + row_u[u] * kRowBytes + l16 * 16);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (tok_u[u] >= 0) {
+          char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + e0 + u) * kRetEntryBytes;
+          *reinterpret_cast<uint4*>(dst + l16 * 16) = v[u];
+          if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok_u[u], 0, 0, 0);
+        }
+      continue;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (tok_u[u] < 0) continue;
+      const size_t row = row_u[u];
+      char* dst = p.ret_rows + ((size_t)layer * p.ret_capacity + out0 + e0 + u) * kRetEntryBytes;
       // lane l16: channels [8 l16, 8 l16 + 8).  code * scale + zero is formed in double (exact) and
       // rounded once to the storage type, so the row is the same bits on any machine.
-      const char* codes = (layer ? (tensor ? p.c_pool[1] : p.c_pool[0]) : (tensor ? p.a_pool[1] : p.a_pool[0])) + row * kQ4RowBytes;
+      const char* codes = pool + row * kQ4RowBytes;
       const char* meta = layer ? (tensor ? p.c_meta[1] : p.c_meta[0]) : (tensor ? p.a_meta[1] : p.a_meta[0]);
       const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + l16 * 4);
       const __half2* mp = tensor == 0 ? reinterpret_cast<const __half2*>(meta) + (row / p.g.page_size) * 128 + 8 * l16
@@ -982,8 +1090,8 @@ __global__ void __launch_bounds__(kRetThreads) retain_compact_kernel(const __gri
         o[j] = (uint32_t)hb[0] | ((uint32_t)hb[1] << 16);
       }
       *reinterpret_cast<uint4*>(dst + l16 * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+      if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok_u[u], 0, 0, 0);
     }
-    if (l16 == 0) *reinterpret_cast<int4*>(dst + kRowBytes) = make_int4(tok, 0, 0, 0);
   }
 }
 
@@ -1186,7 +1294,7 @@ mc_status launch_merge_pairs(const mc_config* cfg, const mc_batch* bt, const Geo
   rb.slack = cfg->append_slack;
   rb.d_hint = hook != nullptr ? hook->d_hint : -1.f;
   rb.gamma = cfg->gamma;
-  dim3 grid(rb.chunks_per_seg, nseg_call, n_pairs);
+  dim3 grid((rb.chunks_per_seg * nseg_call + kRetThreads / 32 - 1) / (kRetThreads / 32), 1, n_pairs);  // a warp per (segment, chunk)
   if (cfg->retain_mode == MC_RETAIN_TOPK)
     MC_CUDA_CHECK(launch_pdl(retain_select_kernel, dim3(nseg_call, 1, n_pairs), dim3(kRetThreads), 0, stream, rb));
   MC_CUDA_CHECK(launch_pdl(retain_count_kernel, dim3(grid), dim3(kRetThreads), 0, stream, rb));
