@@ -13,6 +13,8 @@
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
+#include "mc_items.cuh"
+#include "mc_pipe.cuh"
 #include "mc_q4.cuh"
 #include "mc_retain.cuh"
 
@@ -41,24 +43,35 @@ __device__ __forceinline__ unsigned short deq_one(int code, unsigned short scale
 
 // code = clamp(rint((x - zero) / scale), 0, 15) as the double-precision quantiser defines it, at single-precision
 // cost: the fp32 quotient is within 1e-5 of the exact one (operands of at most 11 significant bits), so it
-// rounds to the same integer unless it lies that close to a tie -- only then is the quotient formed in double.
+// rounds to the same integer unless it lies that close to a tie -- only then is the quotient formed in double
+// (out of line: the kernels stay small enough for the instruction cache).  zero is the group's minimum, so the
+// quotient is never negative, and at most 15 plus the rounding of the scale: adding 1.5 * 2^23 leaves rint(q)
+// in the sum's last mantissa bits, with no conversion instruction.
+__device__ __noinline__ int q4_code_exact(float x, float z, float s) {
+  const double r = rint(((double)x - (double)z) / (double)s);
+  return (int)fmin(fmax(r, 0.0), 15.0);
+}
 __device__ __forceinline__ int q4_code(float x, float z, float s, float inv_s) {
   const float qf = (x - z) * inv_s;
-  float r = rintf(qf);
-  if (fabsf(fabsf(qf - r) - 0.5f) < 1e-3f) r = (float)rint(((double)x - (double)z) / (double)s);
-  return (int)fminf(fmaxf(r, 0.f), 15.f);
+  const float m = qf + 12582912.0f;
+  const float r = m - 12582912.0f;
+  if (fabsf(fabsf(qf - r) - 0.5f) < 1e-3f) return q4_code_exact(x, z, s);
+  return min(__float_as_int(m) & 31, 15);
 }
 
 // Shared memory of one tile conversion.
 struct QTileSmem {
-  unsigned short rows[kQ4Page][kHeadDim];  // the 16-bit directions, channels in natural order
-  float g[2][kQ4Page];                     // the two layers' scales of the 16-bit tile
-  unsigned char codes[kQ4Page][kHeadDim];
+  // two 16-bit tiles (one being converted, one arriving): the directions, channels in natural order, and the
+  // two layers' scales
+  unsigned short rows[2][kQ4Page][kHeadDim];
+  float g[2][2][kQ4Page];
+  unsigned char codes[kQ4Page][kHeadDim + 8];  // (rows 34 words apart: the row-wise reads of a warp's rows fall into different banks)
   unsigned short scale[kQ4Page * 4];       // K: [128] per channel; V: [32][4] per (token, channel group)
   unsigned short zero[kQ4Page * 4];
+  float4 mm[2][kHeadDim / 2];              // K: (min, max) of a channel pair over each half of the tokens
 };
 
-// A 16-bit tile (page_size 32, chunks permuted) from global memory into QTileSmem::rows / g.
+// A 16-bit tile (page_size 32, chunks permuted) from global memory into QTileSmem::rows[0] / g[0].
 // Plain loads: the tile may have been written by this very block a moment ago.
 __device__ __forceinline__ void load_tile16(const char* src, QTileSmem& sm) {
   for (int idx = threadIdx.x; idx < kResTileBytes / 16; idx += kQThreads) {
@@ -66,84 +79,177 @@ __device__ __forceinline__ void load_tile16(const char* src, QTileSmem& sm) {
     if (idx < kQ4Page * 16) {
       const int r = idx >> 4, pos = idx & 15;
       const int c = (pos & 8) | ((pos & 7) ^ (r & 7));  // the chunk stored at this position
-      *reinterpret_cast<uint4*>(&sm.rows[r][c * 8]) = v;
+      *reinterpret_cast<uint4*>(&sm.rows[0][r][c * 8]) = v;
     } else {
-      *reinterpret_cast<uint4*>(&sm.g[0][0] + (idx - kQ4Page * 16) * 4) = v;
+      *reinterpret_cast<uint4*>(&sm.g[0][0][0] + (idx - kQ4Page * 16) * 4) = v;
     }
   }
 }
 
-// Quantises the tile in `sm` (32 complete tokens) and writes the 4-bit tile to `dst`.
+// Scale and zero of a group from its extremes: (max - min) / 15 and min, kept in the 16-bit type.
 template <int DT>
-__device__ void quantise_tile(int tensor, QTileSmem& sm, char* dst) {
+__device__ __noinline__ void group_params(float lo, float hi, unsigned short& s16, unsigned short& z16) {
+  s16 = double_to_elem<DT>(((double)hi - (double)lo) / 15.0);
+  if (elem_to_float<DT>(s16) == 0.f) s16 = double_to_elem<DT>(1.0);  // a constant group
+  z16 = double_to_elem<DT>((double)lo);
+}
+// Two codes (0..15) as exact integers of the 16-bit type, packed (the magic-number conversion of code_pairs).
+template <int DT>
+__device__ __forceinline__ uint32_t int_pair(int c0, int c1) {
+  if (DT == MC_F16) {
+    uint32_t r = (uint32_t)c0 | ((uint32_t)c1 << 16) | 0x64006400u;
+    const __half2 v = __hsub2(*reinterpret_cast<__half2*>(&r), __half2half2(__ushort_as_half((unsigned short)0x6400)));
+    return *reinterpret_cast<const uint32_t*>(&v);
+  }
+  uint32_t r = (uint32_t)c0 | ((uint32_t)c1 << 16) | 0x43004300u;
+  const __nv_bfloat162 v = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&r), __bfloat162bfloat162(__ushort_as_bfloat16((unsigned short)0x4300)));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+// Sum of the squares of eight values, pairwise (each product is exact in fp32 for 16-bit inputs).
+__device__ __forceinline__ float sumsq8(const float2 (&v)[4]) {
+  const float a = fmaf(v[0].y, v[0].y, v[0].x * v[0].x), b = fmaf(v[1].y, v[1].y, v[1].x * v[1].x);
+  const float c = fmaf(v[2].y, v[2].y, v[2].x * v[2].x), d = fmaf(v[3].y, v[3].y, v[3].x * v[3].x);
+  return (a + b) + (c + d);
+}
+
+// The chunk (8 channels of the thread's 32) that thread (row r, quarter q) of the row-wise phases takes in its
+// turn jj: the rotation keeps the 16-byte shared-memory loads of a quarter-warp (two rows, four quarters) in
+// different banks (rows are 64 words apart, quarters 16).
+__device__ __forceinline__ int row_turn(int r, int q, int jj) { return (jj + (q >> 1) + 2 * (r & 1)) & 3; }
+
+// Quantises the 16-bit tile in buffer `buf` of `sm` (32 complete tokens) and writes the 4-bit tile to `dst`.
+// The two sums of squares behind a scale (|e_16|^2 and |e_q|^2 of a row) are accumulated in fp32 pairwise:
+// seven roundings deep, so each is within 7 * 2^-24 of the exact sum and the scale within 5e-7 (relative) of
+// g_16 |e_16| / |e_q|.
+template <int DT>
+__device__ void quantise_tile(int tensor, QTileSmem& sm, int buf, char* dst) {
   const int tid = threadIdx.x;
+  const int r = tid >> 2, qd = tid & 3;  // the row-wise phases: four threads per token, 32 channels each
+  const float inf = __int_as_float(0x7f800000);
   __syncthreads();
-  // ---- groups: extremes, scale, zero, codes
+  float ss16 = 0.f, ssq = 0.f;
   if (tensor == 0) {
-    const int c = tid;  // a channel over the page's 32 tokens
-    float lo = elem_to_float<DT>(sm.rows[0][c]), hi = lo;
-    for (int r = 1; r < kQ4Page; ++r) {
-      const float x = elem_to_float<DT>(sm.rows[r][c]);
-      lo = fminf(lo, x);
-      hi = fmaxf(hi, x);
+    // ---- keys: a group is a channel over the page's 32 tokens.  Two threads per channel pair (a 32-bit
+    // word of a row), 16 tokens each; the extremes of the two halves meet in shared memory.
+    const int cp = tid & 63, th = tid >> 6;
+    const uint32_t* rows32 = reinterpret_cast<const uint32_t*>(&sm.rows[buf][0][0]);
+    float2 x[16];
+    float2 lo = make_float2(inf, inf), hi = make_float2(-inf, -inf);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      x[i] = Elem<DT>::unpack(rows32[(16 * th + i) * (kHeadDim / 2) + cp]);
+      lo.x = fminf(lo.x, x[i].x);
+      lo.y = fminf(lo.y, x[i].y);
+      hi.x = fmaxf(hi.x, x[i].x);
+      hi.y = fmaxf(hi.y, x[i].y);
     }
-    unsigned short s16 = double_to_elem<DT>(((double)hi - (double)lo) / 15.0);
-    if (elem_to_float<DT>(s16) == 0.f) s16 = double_to_elem<DT>(1.0);  // a constant group
-    const unsigned short z16 = double_to_elem<DT>((double)lo);
-    const float sf = elem_to_float<DT>(s16), zf = elem_to_float<DT>(z16), inv_s = 1.0f / sf;
-    for (int r = 0; r < kQ4Page; ++r) sm.codes[r][c] = (unsigned char)q4_code(elem_to_float<DT>(sm.rows[r][c]), zf, sf, inv_s);
-    sm.scale[c] = s16;
-    sm.zero[c] = z16;
+    sm.mm[th][cp] = make_float4(lo.x, hi.x, lo.y, hi.y);
+    __syncthreads();
+    const float4 o = sm.mm[1 - th][cp];
+    unsigned short s0, z0, s1, z1;
+    group_params<DT>(fminf(lo.x, o.x), fmaxf(hi.x, o.y), s0, z0);
+    group_params<DT>(fminf(lo.y, o.z), fmaxf(hi.y, o.w), s1, z1);
+    const float sf0 = elem_to_float<DT>(s0), zf0 = elem_to_float<DT>(z0), inv0 = 1.0f / sf0;
+    const float sf1 = elem_to_float<DT>(s1), zf1 = elem_to_float<DT>(z1), inv1 = 1.0f / sf1;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int c0 = q4_code(x[i].x, zf0, sf0, inv0), c1 = q4_code(x[i].y, zf1, sf1, inv1);
+      *reinterpret_cast<unsigned short*>(&sm.codes[16 * th + i][2 * cp]) = (unsigned short)(c0 | (c1 << 8));
+    }
+    if (th == 0) {
+      reinterpret_cast<uint32_t*>(sm.scale)[cp] = (uint32_t)s0 | ((uint32_t)s1 << 16);
+      reinterpret_cast<uint32_t*>(sm.zero)[cp] = (uint32_t)z0 | ((uint32_t)z1 << 16);
+    }
+    __syncthreads();
+    // ---- row-wise: the two lengths of every token's direction
+    const uint32_t* codes32 = reinterpret_cast<const uint32_t*>(&sm.codes[r][32 * qd]);
+    const uint32_t* sc32 = reinterpret_cast<const uint32_t*>(sm.scale) + 16 * qd;
+    const uint32_t* zr32 = reinterpret_cast<const uint32_t*>(sm.zero) + 16 * qd;
+    float p16[4], pq[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int q = row_turn(r, qd, jj);
+      const uint4 v = *reinterpret_cast<const uint4*>(&sm.rows[buf][r][32 * qd + 8 * q]);
+      const float2 e[4] = {Elem<DT>::unpack(v.x), Elem<DT>::unpack(v.y), Elem<DT>::unpack(v.z), Elem<DT>::unpack(v.w)};
+      p16[jj] = sumsq8(e);
+      // the codes of the same 8 channels: two words, the (scale, zero) pairs of their channel pairs beside them
+      const uint2 cw = *reinterpret_cast<const uint2*>(codes32 + 2 * q);
+      const uint4 s4 = *reinterpret_cast<const uint4*>(sc32 + 4 * q), z4 = *reinterpret_cast<const uint4*>(zr32 + 4 * q);
+      const float2 d[4] = {Elem<DT>::unpack(deq_pair<DT>(int_pair<DT>(cw.x & 15u, (cw.x >> 8) & 15u), s4.x, z4.x)),
+                           Elem<DT>::unpack(deq_pair<DT>(int_pair<DT>((cw.x >> 16) & 15u, cw.x >> 24), s4.y, z4.y)),
+                           Elem<DT>::unpack(deq_pair<DT>(int_pair<DT>(cw.y & 15u, (cw.y >> 8) & 15u), s4.z, z4.z)),
+                           Elem<DT>::unpack(deq_pair<DT>(int_pair<DT>((cw.y >> 16) & 15u, cw.y >> 24), s4.w, z4.w))};
+      pq[jj] = sumsq8(d);
+    }
+    ss16 = (p16[0] + p16[1]) + (p16[2] + p16[3]);
+    ssq = (pq[0] + pq[1]) + (pq[2] + pq[3]);
   } else {
-    const int r = tid >> 2, g = tid & 3;  // 32 channels of one token
-    float lo = elem_to_float<DT>(sm.rows[r][32 * g]), hi = lo;
-    for (int j = 1; j < 32; ++j) {
-      const float x = elem_to_float<DT>(sm.rows[r][32 * g + j]);
-      lo = fminf(lo, x);
-      hi = fmaxf(hi, x);
+    // ---- values: a group is 32 channels of one token: the thread's own 32 values, start to finish
+    float2 x[4][4];
+    float lo = inf, hi = -inf;
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int q = row_turn(r, qd, jj);
+      const uint4 v = *reinterpret_cast<const uint4*>(&sm.rows[buf][r][32 * qd + 8 * q]);
+      x[jj][0] = Elem<DT>::unpack(v.x);
+      x[jj][1] = Elem<DT>::unpack(v.y);
+      x[jj][2] = Elem<DT>::unpack(v.z);
+      x[jj][3] = Elem<DT>::unpack(v.w);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        lo = fminf(lo, fminf(x[jj][k].x, x[jj][k].y));
+        hi = fmaxf(hi, fmaxf(x[jj][k].x, x[jj][k].y));
+      }
     }
-    unsigned short s16 = double_to_elem<DT>(((double)hi - (double)lo) / 15.0);
-    if (elem_to_float<DT>(s16) == 0.f) s16 = double_to_elem<DT>(1.0);
-    const unsigned short z16 = double_to_elem<DT>((double)lo);
+    unsigned short s16, z16;
+    group_params<DT>(lo, hi, s16, z16);
     const float sf = elem_to_float<DT>(s16), zf = elem_to_float<DT>(z16), inv_s = 1.0f / sf;
-    for (int j = 0; j < 32; ++j)
-      sm.codes[r][32 * g + j] = (unsigned char)q4_code(elem_to_float<DT>(sm.rows[r][32 * g + j]), zf, sf, inv_s);
-    sm.scale[r * 4 + g] = s16;
-    sm.zero[r * 4 + g] = z16;
+    const uint32_t s2 = (uint32_t)s16 | ((uint32_t)s16 << 16), z2 = (uint32_t)z16 | ((uint32_t)z16 << 16);
+    float p16[4], pq[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const int q = row_turn(r, qd, jj);
+      int c[8];
+      float2 d[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        c[2 * k] = q4_code(x[jj][k].x, zf, sf, inv_s);
+        c[2 * k + 1] = q4_code(x[jj][k].y, zf, sf, inv_s);
+        d[k] = Elem<DT>::unpack(deq_pair<DT>(int_pair<DT>(c[2 * k], c[2 * k + 1]), s2, z2));
+      }
+      *reinterpret_cast<uint2*>(&sm.codes[r][32 * qd + 8 * q]) =
+          make_uint2((uint32_t)c[0] | ((uint32_t)c[1] << 8) | ((uint32_t)c[2] << 16) | ((uint32_t)c[3] << 24),
+                     (uint32_t)c[4] | ((uint32_t)c[5] << 8) | ((uint32_t)c[6] << 16) | ((uint32_t)c[7] << 24));
+      p16[jj] = sumsq8(x[jj]);
+      pq[jj] = sumsq8(d);
+    }
+    ss16 = (p16[0] + p16[1]) + (p16[2] + p16[3]);
+    ssq = (pq[0] + pq[1]) + (pq[2] + pq[3]);
+    sm.scale[r * 4 + qd] = s16;
+    sm.zero[r * 4 + qd] = z16;
+  }
+  // ---- the scales of Eq. 2 refer to the stored direction: |x| / |e_q| = g16 * |e_16| / |e_q|
+  ss16 += __shfl_xor_sync(0xffffffffu, ss16, 1);
+  ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
+  ss16 += __shfl_xor_sync(0xffffffffu, ss16, 2);
+  ssq += __shfl_xor_sync(0xffffffffu, ssq, 2);
+  if (qd < 2) {
+    const float g16 = sm.g[buf][qd][r];
+    float gq = g16;  // -0 (a retained token) and 0 (a zero row) stay what they are
+    if (g16 != 0.f) gq = g16 * sqrtf(ss16 / (ssq > 0.f ? ssq : ss16));
+    reinterpret_cast<float*>(dst + kQ4ScaleOff)[qd * kQ4Page + r] = gq;
   }
   __syncthreads();
-  // ---- the scales of Eq. 2 refer to the stored direction: |x| / |e_q| = g16 * |e_16| / |e_q|
-  {
-    const int r = tid >> 2, qd = tid & 3;
-    double ss16 = 0.0, ssq = 0.0;
-    for (int j = 0; j < 32; ++j) {
-      const int c = 32 * qd + j;
-      const int mi = tensor == 0 ? c : r * 4 + qd;
-      const double e16 = (double)elem_to_float<DT>(sm.rows[r][c]);
-      const double eq = (double)elem_to_float<DT>(deq_one<DT>(sm.codes[r][c], sm.scale[mi], sm.zero[mi]));
-      ss16 += e16 * e16;
-      ssq += eq * eq;
-    }
-    ss16 += __shfl_xor_sync(0xffffffffu, ss16, 1);
-    ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
-    ss16 += __shfl_xor_sync(0xffffffffu, ss16, 2);
-    ssq += __shfl_xor_sync(0xffffffffu, ssq, 2);
-    if (qd < 2) {
-      const float g16 = sm.g[qd][r];
-      float gq = g16;  // -0 (a retained token) and 0 (a zero row) stay what they are
-      if (g16 != 0.f) gq = (float)((double)g16 * sqrt(ss16 / (ssq > 0.0 ? ssq : ss16)));
-      reinterpret_cast<float*>(dst + kQ4ScaleOff)[qd * kQ4Page + r] = gq;
-    }
-  }
   // ---- pack the codes and the group parameters in the tile's orders
   uint32_t* out_w = reinterpret_cast<uint32_t*>(dst);
   for (int wi = tid; wi < kQ4CodeBytes / 4; wi += kQThreads) {
     uint32_t w = 0;
     if (tensor == 0) {
-      const int r = wi >> 4, wd = wi & 15;
-#pragma unroll
-      for (int p = 0; p < 4; ++p)
-        w |= ((uint32_t)sm.codes[r][8 * wd + 2 * p] << (4 * p)) | ((uint32_t)sm.codes[r][8 * wd + 2 * p + 1] << (16 + 4 * p));
+      const int rr = wi >> 4, wd = wi & 15;
+      const uint2 b = *reinterpret_cast<const uint2*>(&sm.codes[rr][8 * wd]);  // codes of channels 8 wd .. 8 wd + 7
+      // even channels to the nibbles 0..3, odd ones to the nibbles 4..7
+      w = (b.x & 0xFu) | ((b.x >> 12) & 0xF0u) | ((b.y & 0xFu) << 8) | ((b.y >> 4) & 0xF000u) |
+          ((b.x << 8) & 0xF0000u) | ((b.x >> 4) & 0xF00000u) | ((b.y << 16) & 0xF000000u) | ((b.y << 4) & 0xF0000000u);
     } else {
       const int i = wi >> 5, cp = (wi >> 2) & 7, k = wi & 3;
       const int c = q4_vchunk_pos(i, cp);  // (an involution: the chunk stored at position cp)
@@ -180,26 +286,87 @@ struct Q4Params {
   int32_t* status;
 };
 
+// One 16-bit tile of the merge's staging area and where it goes.
+struct QTile {
+  int b, pslot, th;  // sequence, page slot, tensor * H + head
+  int raw_page;      // page id as read from the block table (validated when the tile's turn comes)
+  bool valid;        // false: past the last tile
+};
+
+// Persistent over the used pages of the call's sequences (tile index = page * 2 H + tensor * H + head, pages
+// counted through the sequences): while a tile is converted, the next one's 16-bit tile is already on its way
+// into registers and the page id of the one after that is being read, so the conversion of a tile does not
+// start with two dependent trips to memory.
 template <int DT>
-__global__ void __launch_bounds__(kQThreads) q4_quantise_pages_kernel(const Q4Params p) {
+__global__ void __launch_bounds__(kQThreads, 6) q4_quantise_pages_kernel(const Q4Params p) {
   grid_dep_wait();
   grid_dep_launch();
   __shared__ __align__(16) QTileSmem sm;
+  __shared__ int len_s[kMaxBatchPages];
+  __shared__ int pre_s[kMaxBatchPages + 1];
   const int H = p.g.n_kv_heads;
-  const int tensor = blockIdx.x / H, h = blockIdx.x % H, pslot = blockIdx.y, b = blockIdx.z;
-  const int n = checked_len(p.g, b, p.status);
-  if (pslot * kQ4Page >= n) return;
-  const int page = checked_page(p.g, b, pslot, p.status);
-  if (page < 0) return;
-  const char* src = p.stage[tensor] + ((size_t)page * H + h) * kResTileBytes;
-  if ((pslot + 1) * kQ4Page <= n) {
-    load_tile16(src, sm);
-    quantise_tile<DT>(tensor, sm, p.e_pool[tensor] + ((size_t)page * H + h) * kQ4TileBytes);
-  } else {
-    char* dst = p.res[tensor] + ((size_t)b * H + h) * kResTileBytes;
-    for (int idx = threadIdx.x; idx < kResTileBytes / 16; idx += kQThreads)
-      reinterpret_cast<uint4*>(dst)[idx] = reinterpret_cast<const uint4*>(src)[idx];
+  page_prefix(p.g, len_s, pre_s, kQThreads, p.status);
+  const long long total = (long long)pre_s[p.g.batch] * 2 * H;
+  int b_run = 0;  // (tile indices only grow: the sequence is found by stepping forward)
+  auto tile_at = [&](long long t) {
+    QTile q;
+    q.valid = t < total;
+    q.b = q.pslot = q.th = 0;
+    q.raw_page = -1;
+    if (!q.valid) return q;
+    const int pg = (int)(t / (2 * H));
+    q.th = (int)(t - (long long)pg * 2 * H);
+    while (pg >= pre_s[b_run + 1]) ++b_run;
+    q.b = b_run;
+    q.pslot = pg - pre_s[b_run];
+    if (q.pslot < p.g.max_pages_per_seq) q.raw_page = p.g.block_table[(size_t)q.b * p.g.max_pages_per_seq + q.pslot];
+    return q;
+  };
+  auto full_page = [&](const QTile& q) { return (q.pslot + 1) * kQ4Page <= len_s[q.b]; };
+  auto page_of = [&](const QTile& q) {  // -1 (and the flag) for an id outside the pools
+    if (page_ok(p.g, q.raw_page)) return q.raw_page;
+    if (threadIdx.x == 0) atomicOr(p.status, MC_FLAG_BAD_METADATA);
+    return -1;
+  };
+  // the tile's 16-bit rows (chunks put back in channel order) and scales, asynchronously into buffer `buf`
+  auto fetch = [&](const QTile& q, int buf) {
+    const int page = q.valid && full_page(q) ? page_of(q) : -1;
+    if (page >= 0) {
+      const char* src = p.stage[q.th / H] + ((size_t)page * H + q.th % H) * kResTileBytes;
+      for (int idx = threadIdx.x; idx < kResTileBytes / 16; idx += kQThreads) {
+        const int r = idx >> 4, pos = idx & 15;
+        const int c = (pos & 8) | ((pos & 7) ^ (r & 7));  // the chunk stored at this position
+        void* dst = idx < kQ4Page * 16 ? (void*)&sm.rows[buf][r][c * 8] : (void*)(&sm.g[buf][0][0] + (idx - kQ4Page * 16) * 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src + (size_t)idx * 16) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  const long long stride = gridDim.x;
+  QTile cur = tile_at(blockIdx.x);
+  QTile nxt = tile_at(blockIdx.x + stride);
+  fetch(cur, 0);
+  int buf = 0;
+  for (long long t = blockIdx.x; cur.valid; t += stride, buf ^= 1) {
+    const int tensor = cur.th / H, h = cur.th % H;
+    const bool full = full_page(cur);
+    const int page = full ? (page_ok(p.g, cur.raw_page) ? cur.raw_page : -1) : page_of(cur);  // (a full page was checked by fetch)
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // this tile has arrived; the other buffer's tile is converted and gone
+    fetch(nxt, buf ^ 1);
+    const QTile nxt2 = tile_at(t + 2 * stride);
+    if (full && page >= 0) {
+      quantise_tile<DT>(tensor, sm, buf, p.e_pool[tensor] + ((size_t)page * H + h) * kQ4TileBytes);
+    } else if (page >= 0) {  // the sequence's last, incomplete page: to its residual tile as it is
+      const char* src = p.stage[tensor] + ((size_t)page * H + h) * kResTileBytes;
+      char* dst = p.res[tensor] + ((size_t)cur.b * H + h) * kResTileBytes;
+      for (int idx = threadIdx.x; idx < kResTileBytes / 16; idx += kQThreads)
+        reinterpret_cast<uint4*>(dst)[idx] = reinterpret_cast<const uint4*>(src)[idx];
+    }
+    cur = nxt;
+    nxt = nxt2;
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -272,7 +439,7 @@ __global__ void __launch_bounds__(kQThreads) append_q4_kernel(const AppendQ4Para
   // the page is complete: its 32 rows leave the residual tile as a 4-bit tile
   __syncthreads();
   load_tile16(res, sm);
-  quantise_tile<DT>(tensor, sm, p.e_pool[tensor] + ((size_t)page * H + h) * kQ4TileBytes);
+  quantise_tile<DT>(tensor, sm, 0, p.e_pool[tensor] + ((size_t)page * H + h) * kQ4TileBytes);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -431,7 +598,11 @@ mc_status launch_q4_quantise(const mc_config* cfg, const mc_batch* bt, const Geo
   qp.res[0] = (char*)out->res_k;
   qp.res[1] = (char*)out->res_v;
   qp.status = out->status;
-  const dim3 grid(2 * cfg->n_kv_heads, q4_page_slots(bt), bt->batch);
+  if (bt->batch > kMaxBatchPages) return MC_ERR_SHAPE;  // the sequences' page prefix lives in shared memory
+  const long long tiles = (long long)bt->batch * q4_page_slots(bt) * 2 * cfg->n_kv_heads;  // (an upper bound)
+  int n_sm = 0;
+  if (mc_status st = sm_count(&n_sm)) return st;
+  const dim3 grid((unsigned)std::max<long long>(1, std::min<long long>(tiles, (long long)n_sm * 6)));
   if (cfg->dtype == MC_F16)
     MC_CUDA_CHECK(launch_pdl(q4_quantise_pages_kernel<MC_F16>, grid, dim3(kQThreads), 0, stream, qp));
   else

@@ -530,7 +530,9 @@ def compare_q4_cache(p4: Problem, dc4, dc16, om4) -> Dict[str, float]:
             want2 = om4[tn][nm][b, :n, h] / lo
             rel2 = np.abs(g4 - want2) / np.maximum(np.abs(want2), 1e-30) * (g4 != 0) * same
             stats["q4_scale_e2e"] = max(stats["q4_scale_e2e"], float(rel2.max(initial=0.0)))
-    # one fp32 rounding of the product on top of the 16-bit scale's own arithmetic
-    assert stats["q4_scale_stage"] < 2e-7, stats
+    # g_q = g_16 |e_16| / |e_q| on the device: the two sums of 128 exact squares are accumulated pairwise in fp32
+    # (seven roundings deep: within 7 x 2^-24 = 4.2e-7 each), then one division, one square root (which halves
+    # the relative error) and one product, one rounding each: (2 x 4.2e-7 + 6e-8) / 2 + 2 x 6e-8 < 6e-7
+    assert stats["q4_scale_stage"] < 6e-7, stats
     assert stats["q4_scale_e2e"] < 3e-6, stats
     return stats
