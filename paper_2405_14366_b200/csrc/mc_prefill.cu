@@ -12,6 +12,9 @@
 //   warps 2..5  epilogue: a thread takes one token row out of tensor memory (its 128 channels), rounds it
 //               to the storage type -- these are layer l's rows --, fetches layer l-1's row, merges, and
 //               writes the shared direction, the scales and the distance in the pair cache's tile format
+// Two CTAs share an SM (two ring stages of 32 KB and the epilogue's row staging each, 128 of the 512 tensor-memory
+// columns, under 100 registers per thread): while one is in its epilogue the other's main loop has the tensor
+// cores and the copy engine.
 // Every wait is bounded; tensor memory is released on every path.
 #include <cuda.h>
 
@@ -27,7 +30,7 @@ namespace mc {
 constexpr int kPfTileM = 128;   // tokens per tile
 constexpr int kPfTileN = 128;   // channels per tile = one head
 constexpr int kPfTileK = 64;    // elements per stage row: 128 bytes, the swizzle span
-constexpr int kPfStages = 4;
+constexpr int kPfStages = 2;
 constexpr int kPfStageBytes = (kPfTileM + kPfTileN) * kPfTileK * 2;  // X tile, then W tile: 32 KB
 constexpr int kPfThreads = 192;
 constexpr int kPfTmemCols = 128;
@@ -106,14 +109,14 @@ __device__ __forceinline__ uint32_t umma_idesc() {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv) {
   grid_dep_wait();
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kPfStages * kPfStageBytes);  // full[4], empty[4], accum
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kPfStages * kPfStageBytes);  // full[stages], empty[stages], accum
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPfStages + 1);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   unsigned char* epi = smem + kPfStages * kPfStageBytes + 256;  // [4 warps][32 rows][kPfEpiRow]: row staging of the epilogue
@@ -213,73 +216,95 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
     const bool ok_wait = mbar_wait(accum_bar, 0, s_abort, p.status);
     tc_fence_after();
     const bool live = ok_wait && !*s_abort && prow >= 0;
-    // layer l's row: accumulators rounded once to the storage type (what the model would have cached)
-    uint32_t cw[64];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    // Layer l's row = the accumulators rounded once to the storage type (what the model would have cached).
+    // Neither row is held in registers across the three passes of the merge (two 64-register copies would not
+    // leave room for two CTAs per SM): layer l's 32-channel blocks are read from tensor memory again in every
+    // pass -- the rounding is deterministic, so every pass sees the same bits --, layer l-1's row is read from
+    // the staging area, which the last pass overwrites, chunk by chunk, with the merged row.
+    // (tcgen05.ld is warp-wide: every lane runs the passes; only the stores depend on the lane having a row.)
+    const unsigned char* my_row = my + lane * kPfEpiRow;
+    auto load_c = [&](int j, uint32_t (&cj)[16]) {
       uint32_t r[32];
-      tmem_ld32(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * 32), r);  // (every lane of the warp: .sync.aligned)
+      tmem_ld32(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * 32), r);
 #pragma unroll
-      for (int i = 0; i < 16; ++i) cw[j * 16 + i] = Elem<DT>::pack(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
-    }
-    uint32_t aw[64];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const uint4 v = *reinterpret_cast<const uint4*>(my + lane * kPfEpiRow + i * 16);
-      aw[4 * i] = v.x;
-      aw[4 * i + 1] = v.y;
-      aw[4 * i + 2] = v.z;
-      aw[4 * i + 3] = v.w;
-    }
-    __syncwarp();  // every lane holds its row: the staging area is free for the merged rows
+      for (int i = 0; i < 16; ++i) cj[i] = Elem<DT>::pack(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+    };
     float dmin = __int_as_float(0x7f800000), dmax = 0.f;
-    if (live) {
+    {
       float aa = 0.f, cc = 0.f;
+#pragma unroll 1
+      for (int j = 0; j < 4; ++j) {
+        uint32_t cj[16];
+        load_c(j, cj);
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float2 a = Elem<DT>::unpack(aw[i]), c = Elem<DT>::unpack(cw[i]);
-        aa = fmaf(a.x, a.x, fmaf(a.y, a.y, aa));
-        cc = fmaf(c.x, c.x, fmaf(c.y, c.y, cc));
+        for (int cq = 0; cq < 4; ++cq) {
+          const uint4 av = *reinterpret_cast<const uint4*>(my_row + (4 * j + cq) * 16);
+          const uint32_t aw4[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 a = Elem<DT>::unpack(aw4[i]), c = Elem<DT>::unpack(cj[4 * cq + i]);
+            aa = fmaf(a.x, a.x, fmaf(a.y, a.y, aa));
+            cc = fmaf(c.x, c.x, fmaf(c.y, c.y, cc));
+          }
+        }
       }
       const float ia = aa > 0.f ? rsqrtf(aa) : 0.f, ic = cc > 0.f ? rsqrtf(cc) : 0.f;
       // |u - v|^2 and |u + v|^2 channel by channel (no cancellation at either end)
       float sm = 0.f, sp = 0.f;
+#pragma unroll 1
+      for (int j = 0; j < 4; ++j) {
+        uint32_t cj[16];
+        load_c(j, cj);
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float2 a = Elem<DT>::unpack(aw[i]), c = Elem<DT>::unpack(cw[i]);
-        const float ux = a.x * ia, uy = a.y * ia;
-        const float mx = fmaf(-c.x, ic, ux), my_ = fmaf(-c.y, ic, uy), px = fmaf(c.x, ic, ux), py = fmaf(c.y, ic, uy);
-        sm = fmaf(mx, mx, fmaf(my_, my_, sm));
-        sp = fmaf(px, px, fmaf(py, py, sp));
+        for (int cq = 0; cq < 4; ++cq) {
+          const uint4 av = *reinterpret_cast<const uint4*>(my_row + (4 * j + cq) * 16);
+          const uint32_t aw4[4] = {av.x, av.y, av.z, av.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 a = Elem<DT>::unpack(aw4[i]), c = Elem<DT>::unpack(cj[4 * cq + i]);
+            const float ux = a.x * ia, uy = a.y * ia;
+            const float mx = fmaf(-c.x, ic, ux), my_ = fmaf(-c.y, ic, uy), px = fmaf(c.x, ic, ux), py = fmaf(c.y, ic, uy);
+            sm = fmaf(mx, mx, fmaf(my_, my_, sm));
+            sp = fmaf(px, px, fmaf(py, py, sp));
+          }
+        }
       }
       float ta = p.ta, tc = p.tc;
       row_t(p.t_mode, aa, cc, ta, tc);
       const RowScalars s = slerp_scalars(aa, cc, sm, sp, ta, tc);
-      char* tile_p = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
-      float ee = 0.f;
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {  // 16-byte chunk ch of the row = channels [8 ch, 8 ch + 8)
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 a = Elem<DT>::unpack(aw[4 * ch + i]), c = Elem<DT>::unpack(cw[4 * ch + i]);
-          w[i] = Elem<DT>::pack(fmaf(s.fa, a.x, s.fc * c.x), fmaf(s.fa, a.y, s.fc * c.y));
-          const float2 r = Elem<DT>::unpack(w[i]);  // the stored value: Eq. 2 divides by its length
-          ee = fmaf(r.x, r.x, fmaf(r.y, r.y, ee));
-        }
-        *reinterpret_cast<uint4*>(my + lane * kPfEpiRow + ch * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-      }
-      const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
-      float* scp = reinterpret_cast<float*>(tile_p + ps * kRowBytes) + tk;
-      scp[0] = s.na * il;
-      scp[ps] = s.nc * il;
-      p.dist[(((size_t)page * H + head) * 2 + tensor) * ps + tk] = s.d;
-      dmin = dmax = s.d;
       // a token that may end up unmerged (Eq. 4) keeps its raw row of layer l
-      if (s.d > p.d_hint) {
-        uint4* cp = reinterpret_cast<uint4*>(p.c_pool[tensor] + (size_t)prow * kRowBytes);
+      const bool keep_raw = live && s.d > p.d_hint;
+      uint4* cp = reinterpret_cast<uint4*>(p.c_pool[tensor] + (size_t)max(prow, 0) * kRowBytes);
+      float ee = 0.f;
+#pragma unroll 1
+      for (int j = 0; j < 4; ++j) {
+        uint32_t cj[16];
+        load_c(j, cj);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) cp[i] = make_uint4(cw[4 * i], cw[4 * i + 1], cw[4 * i + 2], cw[4 * i + 3]);
+        for (int cq = 0; cq < 4; ++cq) {  // 16-byte chunk 4 j + cq of the row = channels [8 (4 j + cq), + 8)
+          const int ch = 4 * j + cq;
+          const uint4 av = *reinterpret_cast<const uint4*>(my_row + ch * 16);
+          const uint32_t aw4[4] = {av.x, av.y, av.z, av.w};
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 a = Elem<DT>::unpack(aw4[i]), c = Elem<DT>::unpack(cj[4 * cq + i]);
+            w[i] = Elem<DT>::pack(fmaf(s.fa, a.x, s.fc * c.x), fmaf(s.fa, a.y, s.fc * c.y));
+            const float2 r = Elem<DT>::unpack(w[i]);  // the stored value: Eq. 2 divides by its length
+            ee = fmaf(r.x, r.x, fmaf(r.y, r.y, ee));
+          }
+          *reinterpret_cast<uint4*>(my + lane * kPfEpiRow + ch * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          if (keep_raw) cp[ch] = make_uint4(cj[4 * cq], cj[4 * cq + 1], cj[4 * cq + 2], cj[4 * cq + 3]);
+        }
+      }
+      if (live) {
+        const float il = ee > 0.f ? 1.0f / sqrtf(ee) : 0.f;
+        char* tile_p = p.e_pool[tensor] + ((size_t)page * H + head) * tile_bytes(ps);
+        float* scp = reinterpret_cast<float*>(tile_p + ps * kRowBytes) + tk;
+        scp[0] = s.na * il;
+        scp[ps] = s.nc * il;
+        p.dist[(((size_t)page * H + head) * 2 + tensor) * ps + tk] = s.d;
+        dmin = dmax = s.d;
       }
     }
     __syncwarp();
