@@ -216,17 +216,17 @@ class Job:
                 if ev:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
-                for layer in (0, 1):
-                    kn = nt["k_lm1" if layer == 0 else "k_l"]
-                    vn = nt["v_lm1" if layer == 0 else "v_l"]
-                    self.lib.mc_decode_attn(self.cfg, b, pc, layer, q[layer], kn, vn, self.sm_scale, self.out, None,
-                                            self.ws_attn)
+                # layer l-1, then layer l with the step's append folded into the same call (it rides on the
+                # attention's combine launch; with a 4-bit cache it is a launch of its own)
+                self.lib.mc_decode_attn(self.cfg, b, pc, 0, q[0], nt["k_lm1"], nt["v_lm1"], self.sm_scale, self.out, None,
+                                        self.ws_attn)
+                self.lib.mc_decode_attn_append(self.cfg, b, pc, 1, q[1], nt["k_l"], nt["v_l"], self.sm_scale, self.out, None,
+                                               nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"], self.ws_attn)
                 if ev:
                     e1.record()
                     self.attn_events.append((e0, e1, s))
-                self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
             self._advance()
-        self.launches += steps * self.wl.n_pairs * 5
+        self.launches += steps * self.wl.n_pairs * (5 if self.q4cache else 4)
 
     def capture_decode_step(self):
         """One decode step (every pair: attention of both layers, append; then the lengths grow by one)
@@ -255,9 +255,8 @@ class Job:
             q, nt, n2 = self.q[s % len(self.q)], self.new[s % len(self.new)], self.new2[s % len(self.new)]
             for pr in range(self.wl.n_pairs):
                 pc = self.pairs[pr]
-                self.lib.mc_decode_attn(self.cfg, b, pc, 2, q, n2["k"], n2["v"], self.sm_scale, self.out2, None,
-                                        self.ws_attn2)
-                self.lib.mc_append_pair(self.cfg, b, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
+                self.lib.mc_decode_attn_append(self.cfg, b, pc, 2, q, n2["k"], n2["v"], self.sm_scale, self.out2, None,
+                                               nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"], self.ws_attn2)
             self._advance()
 
     def _advance(self):
@@ -701,10 +700,9 @@ def run_refill(args, wl, dev, rank, world, dist):
         q, nt = job.q[0], job.new[0]
         for pr in range(wl.n_pairs):
             pc = job.pairs[pr]
-            for layer in (0, 1):
-                lib.mc_decode_attn(job.cfg, bd, pc, layer, q[layer], nt["k_lm1" if layer == 0 else "k_l"],
-                                   nt["v_lm1" if layer == 0 else "v_l"], job.sm_scale, job.out, None, job.ws_attn)
-            lib.mc_append_pair(job.cfg, bd, pc, nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"])
+            lib.mc_decode_attn(job.cfg, bd, pc, 0, q[0], nt["k_lm1"], nt["v_lm1"], job.sm_scale, job.out, None, job.ws_attn)
+            lib.mc_decode_attn_append(job.cfg, bd, pc, 1, q[1], nt["k_l"], nt["v_l"], job.sm_scale, job.out, None,
+                                      nt["k_lm1"], nt["v_lm1"], nt["k_l"], nt["v_l"], job.ws_attn)
         # end of the step, on the device: live slots grow by one token; a slot that has generated its share empties
         live = (remaining > 0).to(torch.int32)
         job.seq_lens.add_(live)
@@ -822,7 +820,7 @@ def run_refill(args, wl, dev, rank, world, dist):
                             "fraction_of_steps_at_full_batch": full / max(steps, 1),
                             "decode_GB/s": world * (attn_bytes + append_bytes) / t / 1e9,
                             "frac_of_measured_hbm": value / world / peak, "admission_merge_bytes": merge_bytes},
-                "gpu_launches": steps * wl.n_pairs * 5 + (admitted - B + 1) * 4, "clocks": clocks}
+                "gpu_launches": steps * wl.n_pairs * (5 if args.q4cache else 4) + (admitted - B + 1) * 4, "clocks": clocks}
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

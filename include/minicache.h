@@ -470,6 +470,20 @@ mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_p
                          float sm_scale, void* out, float* lse, void* workspace,
                          size_t workspace_bytes, void* stream);
 
+/* One decode step of a layer pair's second layer in one call (Algorithm 2 "MiniCache Decoding": attend, then
+ * compress the step's token pair): mc_decode_attn with the first ten arguments, followed by mc_append_pair with
+ * k/v_new_lm1, k/v_new_l -- same results, bit for bit, as the two calls one after the other.  With a 16-bit
+ * shared cache the append rides on the attention's second launch (a few more blocks of the combine kernel,
+ * which run once the split kernel is complete) instead of taking a launch of its own; with cfg->cache_bits = 4
+ * it is the two calls.  Typical use: layer_sel = MC_LAYER_L with k_new = k_new_l, v_new = v_new_l (the pair's
+ * layer l-1 was attended by a plain mc_decode_attn before), or MC_LAYER_BOTH.  Every argument of both calls is
+ * checked before anything is launched. */
+mc_status mc_decode_attn_append(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair,
+                                int32_t layer_sel, const void* q, const void* k_new, const void* v_new,
+                                float sm_scale, void* out, float* lse, const void* k_new_lm1,
+                                const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* Host-buffer form of mc_merge_pair (Algorithm 2 "MiniCache Prefill" with the layers' K/V arriving
  * from the host): host_lm1 / host_l are HOST pools (pinned memory for asynchronous copies) in the
  * paged layout; they are copied into the caller's device pools dev_lm1 / dev_l on `stream`

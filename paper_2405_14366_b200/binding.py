@@ -80,7 +80,7 @@ class _Stats(C.Structure):
                 ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
 
 
-EXPORTS = ("mc_prefill_merge_pair", "mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+EXPORTS = ("mc_decode_attn_append", "mc_prefill_merge_pair", "mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -313,6 +313,9 @@ class MiniCacheLib:
         L.mc_get_stats.restype = C.c_int32
         L.mc_decode_attn.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V,
                                      C.c_size_t, V]
+        L.mc_decode_attn_append.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V, V, V, V,
+                                            V, C.c_size_t, V]
+        L.mc_decode_attn_append.restype = C.c_int32
         L.mc_read_status.argtypes = [P(_PairCache), V, P(C.c_int32)]
         L.mc_merge_pair_host.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_LayerKV), P(_LayerKV),
                                          P(_PairCache), C.c_int32, V, C.c_size_t, V]
@@ -455,6 +458,16 @@ class MiniCacheLib:
         self._check(self._lib.mc_decode_attn(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q), _ptr(k_new),
                                              _ptr(v_new), float(sm_scale), _ptr(out), _ptr(lse), _ptr(workspace),
                                              workspace.numel() * workspace.element_size(), _stream(stream)))
+
+    def mc_decode_attn_append(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q, k_new, v_new,
+                              sm_scale: float, out, lse, k_new_lm1, v_new_lm1, k_new_l, v_new_l, workspace: torch.Tensor,
+                              stream=None):
+        """mc_decode_attn followed by mc_append_pair, in one call (the append rides on the attention's second launch)."""
+        c, b, pc = cfg.c(), batch.c(), pair.c()
+        self._check(self._lib.mc_decode_attn_append(C.byref(c), C.byref(b), C.byref(pc), layer_sel, _ptr(q), _ptr(k_new),
+                                                    _ptr(v_new), float(sm_scale), _ptr(out), _ptr(lse), _ptr(k_new_lm1),
+                                                    _ptr(v_new_lm1), _ptr(k_new_l), _ptr(v_new_l), _ptr(workspace),
+                                                    workspace.numel() * workspace.element_size(), _stream(stream)))
 
     def mc_merge_pair_host(self, cfg: McConfig, batch: Batch, host, dev, pair: PairCache, do_retention: bool,
                            workspace: torch.Tensor, stream=None):

@@ -10,6 +10,7 @@
 #include "mc_common.cuh"
 #include "mc_items.cuh"
 #include "mc_kernels.h"
+#include "mc_append.cuh"
 #include "mc_q4.cuh"
 
 namespace mc {
@@ -133,7 +134,7 @@ using namespace mc;
 
 extern "C" {
 
-int32_t mc_version(void) { return 220; }
+int32_t mc_version(void) { return 230; }
 
 int32_t mc_build_flags(void) {
 #if defined(MC_BOUNDS) && MC_BOUNDS
@@ -493,6 +494,39 @@ mc_status mc_decode_attn(const mc_config* cfg, const mc_batch* batch, const mc_p
   if (workspace_bytes < attn_workspace_bytes(cfg, batch, n_sets)) return MC_ERR_CAPACITY;
   return launch_decode_attn(cfg, batch, make_geom(cfg, batch), pair, layer_sel, q, k_new, v_new, sm_scale, out, lse,
                             workspace, (cudaStream_t)stream);
+}
+
+mc_status mc_decode_attn_append(const mc_config* cfg, const mc_batch* batch, const mc_pair_cache* pair, int32_t layer_sel,
+                                const void* q, const void* k_new, const void* v_new, float sm_scale, void* out, float* lse,
+                                const void* k_new_lm1, const void* v_new_lm1, const void* k_new_l, const void* v_new_l,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  ApiRange range_("mc_decode_attn_append");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  st = check_batch(cfg, batch);
+  if (st != MC_OK) return st;
+  st = check_pair(cfg, pair);
+  if (st != MC_OK) return st;
+  // every check of both calls before the first launch
+  if (layer_sel < MC_LAYER_LM1 || layer_sel > MC_LAYER_BOTH) return MC_ERR_INVALID_ARG;
+  const int n_sets = layer_sel == MC_LAYER_BOTH ? 2 : 1;
+  if (n_sets * (cfg->n_q_heads / cfg->n_kv_heads) > 8) return MC_ERR_SHAPE;
+  if (!q || !out) return MC_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return MC_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) & 15u) return MC_ERR_ALIGN;
+  if (!k_new_lm1 || !v_new_lm1 || !k_new_l || !v_new_l) return MC_ERR_INVALID_ARG;
+  if (((uintptr_t)k_new_lm1 | (uintptr_t)v_new_lm1 | (uintptr_t)k_new_l | (uintptr_t)v_new_l) & 15u) return MC_ERR_ALIGN;
+  if (workspace == nullptr || !aligned256(workspace)) return workspace ? MC_ERR_ALIGN : MC_ERR_INVALID_ARG;
+  if (workspace_bytes < attn_workspace_bytes(cfg, batch, n_sets)) return MC_ERR_CAPACITY;
+  const Geom g = make_geom(cfg, batch);
+  if (cfg->cache_bits == 4) {  // the 4-bit cache's append quantises whole pages: a launch of its own, after the attention
+    st = launch_decode_attn(cfg, batch, g, pair, layer_sel, q, k_new, v_new, sm_scale, out, lse, workspace, (cudaStream_t)stream);
+    if (st != MC_OK) return st;
+    return launch_append_q4(cfg, batch, g, pair, k_new_lm1, v_new_lm1, k_new_l, v_new_l, (cudaStream_t)stream);
+  }
+  const AppendParams app = make_append_params(cfg, batch, g, pair, k_new_lm1, v_new_lm1, k_new_l, v_new_l);
+  return launch_decode_attn(cfg, batch, g, pair, layer_sel, q, k_new, v_new, sm_scale, out, lse, workspace, (cudaStream_t)stream,
+                            &app);
 }
 
 mc_status mc_merge_pair_host(const mc_config* cfg, const mc_batch* batch, const mc_layer_kv* host_lm1,

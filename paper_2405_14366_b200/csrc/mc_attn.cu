@@ -25,12 +25,15 @@
 //     warp takes 16 tokens of every tile, P = 2^(score - max) x V scale formed where it is used,
 //     plus gathered P times the retained V rows; the warps' partial sums meet in shared memory.
 // Partial (m, l, o) per piece are merged by attn_combine_kernel.  Every wait is bounded.
+#include <string.h>
+
 #include <algorithm>
 
 #include "mc_common.cuh"
 #include "mc_kernels.h"
 #include "mc_pipe.cuh"
 #include "mc_q4.cuh"
+#include "mc_append.cuh"
 
 namespace mc {
 
@@ -1007,9 +1010,21 @@ constexpr int kCombineThreads = 256;
 constexpr int kCombineWarps = kCombineThreads / 32;
 constexpr int kMaxPieces = 2048;  // pieces of one sequence = teams (checked on the host)
 
+// The launch can carry the decode step's append as well (mc_decode_attn_append): blocks past the combine's own
+// (blockIdx.x >= combine_x) merge the new token pair of sequence blockIdx.y into the pair cache, a row per
+// half-warp -- what append_kernel does, without a launch of its own.  The split kernel is complete by then
+// (the wait), so nothing reads the cache while the row is written.
 template <int DT, int R>
-__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse) {
+__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const AttnParams p, unsigned short* out, float* lse,
+                                                                       const __grid_constant__ AppendParams app, int combine_x) {
   grid_dep_launch();
+  if ((int)blockIdx.x >= combine_x) {
+    const int H = app.g.n_kv_heads;
+    const int j = ((int)blockIdx.x - combine_x) * (kCombineThreads / 16) + (int)(threadIdx.x >> 4);  // (tensor, head) of the sequence
+    const int r = blockIdx.z == 0 && j < 2 * H ? ((j / H) * app.g.batch + (int)blockIdx.y) * H + j % H : app.total_rows;
+    append_row<DT>(app, r, threadIdx.x & 15, [] { grid_dep_wait(); });
+    return;
+  }
   constexpr int GP = kCombineWarps / R;  // warps per output row
   __shared__ int sum_s[2][kCombineWarps];
   __shared__ int list_s[kMaxPieces];
@@ -1157,7 +1172,7 @@ size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets
 
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                              int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,
-                             void* out, float* lse, void* workspace, cudaStream_t stream) {
+                             void* out, float* lse, void* workspace, cudaStream_t stream, const AppendParams* append) {
   if (bt->batch == 0) return MC_OK;
   if (bt->batch > kMaxBatchSmem) return MC_ERR_SHAPE;
   AttnParams ap;
@@ -1207,13 +1222,21 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   void (*split)(const AttnParams) =
       cfg->dtype == MC_F16 ? (q4 ? attn_split_kernel<MC_F16, true> : attn_split_kernel<MC_F16, false>)
                            : (q4 ? attn_split_kernel<MC_BF16, true> : attn_split_kernel<MC_BF16, false>);
-  void (*combine)(const AttnParams, unsigned short*, float*) =
+  // (the append rides on the combine launch: ceil(2 H / 16) more blocks per sequence)
+  AppendParams app;
+  memset(&app, 0, sizeof(app));
+  const int combine_x = (int)cgrid.x;
+  if (append != nullptr) {
+    app = *append;
+    cgrid.x += (2 * cfg->n_kv_heads + kCombineThreads / 16 - 1) / (kCombineThreads / 16);
+  }
+  void (*combine)(const AttnParams, unsigned short*, float*, const AppendParams, int) =
       cfg->dtype == MC_F16 ? (warp_rows ? attn_combine_kernel<MC_F16, kCombineWarps> : attn_combine_kernel<MC_F16, 1>)
                            : (warp_rows ? attn_combine_kernel<MC_BF16, kCombineWarps> : attn_combine_kernel<MC_BF16, 1>);
   MC_CUDA_CHECK(cudaFuncSetAttribute(split, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MC_CUDA_CHECK(launch_pdl(split, dim3(grid), dim3(kAttnThreads), smem, stream, ap));
   MC_CUDA_CHECK(cudaGetLastError());
-  MC_CUDA_CHECK(launch_pdl(combine, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse));
+  MC_CUDA_CHECK(launch_pdl(combine, dim3(cgrid), dim3(kCombineThreads), 0, stream, ap, (unsigned short*)out, lse, app, combine_x));
   MC_CUDA_CHECK(cudaGetLastError());
   return MC_OK;
 }

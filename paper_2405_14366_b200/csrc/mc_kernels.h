@@ -50,9 +50,11 @@ mc_status launch_restore_q4(const mc_config* cfg, const mc_batch* bt, const Geom
                             const mc_layer_kv* dst, int dst_fp32, cudaStream_t stream);
 
 size_t attn_workspace_bytes(const mc_config* cfg, const mc_batch* bt, int n_sets);
+// `append` (may be null): the decode step's append for this pair, folded into the combine launch (16-bit cache).
+struct AppendParams;
 mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geom& g, const mc_pair_cache* pair,
                              int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,
-                             void* out, float* lse, void* workspace, cudaStream_t stream);
+                             void* out, float* lse, void* workspace, cudaStream_t stream, const AppendParams* append = nullptr);
 
 // Copies the new token's K and V rows (n bytes each, a multiple of 16) from device-addressable host
 // memory into device staging with one small kernel.
