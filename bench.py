@@ -843,11 +843,14 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
             host_pools.append({k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in pl.items()})
     stage = {k: torch.empty_like(v) for k, v in job.pools[0].items()}  # device staging the host pools land in
     pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+    # per decode step and pair: both layers' queries [2][B][Hq][128] and new rows [2][B][H][128], pinned
     q_host = [pin(q) for q in job.q]
-    new_host = [{k: pin(v) for k, v in nt.items()} for nt in job.new]
-    out_host = torch.empty(job.out.shape, dtype=job.out.dtype, pin_memory=True)
+    kn_host = [pin(torch.stack([nt["k_lm1"], nt["k_l"]])) for nt in job.new]
+    vn_host = [pin(torch.stack([nt["v_lm1"], nt["v_l"]])) for nt in job.new]
+    out_host = torch.empty((2,) + tuple(job.out.shape[1:]), dtype=job.out.dtype, pin_memory=True)  # a pair's two results
+    out_dev = [torch.empty((2,) + tuple(job.out.shape[1:]), dtype=job.out.dtype, device=dev) for _ in range(2)]
     bd = job.batch(True)
-    io = torch.empty(lib.mc_decode_io_bytes(job.cfg, bd, 1), dtype=torch.uint8, device=dev)
+    io = [torch.empty(lib.mc_decode_io_bytes(job.cfg, bd, 2), dtype=torch.uint8, device=dev) for _ in range(2)]
     pool_bytes = sum(v.numel() * v.element_size() for v in job.pools[0].values())
     q_bytes = job.B * job.Hq * ROW
     n_bytes = job.B * job.H * ROW
@@ -878,23 +881,60 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
             ev.record(side_s)
             merged[k % 2] = ev
 
+    # The inputs of a pair's two attention calls (both layers' queries and new rows, 384 KB here) are staged from
+    # the pinned host buffers by mc_decode_stage_host on a third stream, one pair ahead: while an upload saturates the
+    # host link such a transfer takes tens of microseconds, which a fetch inside the call would put on the critical
+    # path of every call.  The results of a pair go back the same way: mc_decode_drain_host on a fourth stream, behind
+    # the pair's second call (a result written to host memory by the attention itself waits on the busy link too).
+    stage_s, drain_s = torch.cuda.Stream(), torch.cuda.Stream()
+    staged = [torch.cuda.Event(), torch.cuda.Event()]    # io[j] holds the inputs of its pair
+    consumed = [None, None]                              # io[j]'s pair has been attended
+    drained = [None, None]                               # out_dev[j] has been copied to the host
+
+    def stage_inputs(c):  # c: running index of the (decode step, pair)
+        j = c % 2
+        s_i = (c // wl.n_pairs) % job.steps
+        with torch.cuda.stream(stage_s):
+            if consumed[j] is not None:
+                stage_s.wait_event(consumed[j])
+            views = lib.mc_decode_stage_host(job.cfg, bd, 2, q_host[s_i % len(q_host)], kn_host[s_i % len(kn_host)],
+                                             vn_host[s_i % len(vn_host)], io[j], stream=stage_s)
+            staged[j].record(stage_s)
+        return views
+
     def decode(k):  # step k's decode phase on the main stream
         cs = pair_sets[k % 2]
         main_s.wait_event(merged[k % 2])
         job.seq_lens.copy_(job.seq0)
         job.step_dev.zero_()
+        c0 = k * job.steps * wl.n_pairs
+        views = stage_inputs(c0)
         for s in range(job.steps):
-            q, nt = q_host[s % len(q_host)], new_host[s % len(new_host)]
-            ntd = job.new[s % len(job.new)]
             for pr in range(wl.n_pairs):
+                c = c0 + s * wl.n_pairs + pr
                 pc = cs[pr]
-                for layer in (0, 1):
-                    kn = nt["k_lm1" if layer == 0 else "k_l"]
-                    vn = nt["v_lm1" if layer == 0 else "v_l"]
-                    lib.mc_decode_attn_host(job.cfg, bd, pc, layer, q[layer], kn, vn, job.sm_scale, out_host, None,
-                                            io, job.ws_attn)
-                lib.mc_append_pair(job.cfg, bd, pc, ntd["k_lm1"], ntd["v_lm1"], ntd["k_l"], ntd["v_l"])
+                qd, knd, vnd = views
+                last = s == job.steps - 1 and pr == wl.n_pairs - 1
+                if not last:
+                    views = stage_inputs(c + 1)
+                main_s.wait_event(staged[c % 2])
+                if drained[c % 2] is not None:
+                    main_s.wait_event(drained[c % 2])
+                od = out_dev[c % 2]
+                lib.mc_decode_attn(job.cfg, bd, pc, 0, qd[0], knd[0], vnd[0], job.sm_scale, od[0:1], None, job.ws_attn)
+                lib.mc_decode_attn_append(job.cfg, bd, pc, 1, qd[1], knd[1], vnd[1], job.sm_scale, od[1:2], None,
+                                          knd[0], vnd[0], knd[1], vnd[1], job.ws_attn)
+                ev = torch.cuda.Event()
+                ev.record(main_s)
+                consumed[c % 2] = ev
+                with torch.cuda.stream(drain_s):
+                    drain_s.wait_event(ev)
+                    lib.mc_decode_drain_host(job.cfg, bd, 2, od, None, out_host, None, stream=drain_s)
+                    dv = torch.cuda.Event()
+                    dv.record(drain_s)
+                    drained[c % 2] = dv
             job._advance()
+        main_s.wait_stream(drain_s)  # the step's results are on the host
         ev = torch.cuda.Event()
         ev.record(main_s)
         decoded[k % 2] = ev
@@ -922,7 +962,9 @@ def run_e2e(job: Job, wl, rho, args, dist, dev, world):
     return {"value": whole_job_gbps(sum(by.values()), n, t, world), "unit": "GB/s", "steps": n, "ms_per_step": t / n * 1e3,
             "h2d_bytes_per_step": wl.n_pairs * pool_bytes + calls * (q_bytes + 2 * n_bytes),
             "d2h_bytes_per_step": calls * q_bytes,
-            "api": "mc_merge_pair_host + mc_restore + mc_decode_attn_host + mc_append_pair, pinned host buffers; "
+            "api": "mc_merge_pair_host + mc_restore + mc_decode_stage_host + mc_decode_attn + mc_decode_attn_append + "
+                   "mc_decode_drain_host, pinned host buffers (a pair's inputs staged one pair ahead on a third stream, its "
+                   "results copied back on a fourth); "
                    "two steps in flight (the next step's upload and merge on a second stream)"}
 
 

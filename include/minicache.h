@@ -504,6 +504,30 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
                               void* dev_io, size_t dev_io_bytes, void* workspace,
                               size_t workspace_bytes, void* stream);
 
+/* Stages the inputs of later mc_decode_attn / mc_decode_attn_append calls from HOST memory: copies q
+ * ([n_query_sets][batch][n_q_heads][128]) and, if given, k_new / v_new ([n_query_sets][batch][n_kv_heads][128])
+ * into `dev_io` (device memory of at least mc_decode_io_bytes(n_query_sets) bytes, 256-byte aligned) on `stream`
+ * and returns where they landed in *q_dev, *k_new_dev, *v_new_dev (device pointers into dev_io; set k of a
+ * two-set staging starts n_q_heads (n_kv_heads) * batch * 256 bytes after set 0).  Meant to be issued on a second
+ * stream, a call or a layer pair ahead of the attention that consumes the rows, so that the transfer -- slow when the
+ * host link is busy with an upload -- is off the decode loop's critical path; the caller orders the two streams
+ * (an event after the staging, one after the attention before the buffer is staged again).  Pinned,
+ * device-addressable host memory is read by a kernel, any other by asynchronous copies.  An attention call can
+ * write its result straight to pinned host memory: pass the buffer's device pointer as `out`. */
+mc_status mc_decode_stage_host(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets,
+                               const void* q_host, const void* k_new_host, const void* v_new_host,
+                               void* dev_io, size_t dev_io_bytes, void** q_dev, void** k_new_dev,
+                               void** v_new_dev, void* stream);
+
+/* The other direction: copies the result of an attention call ([n_query_sets][batch][n_q_heads][128] 16-bit, and the
+ * log-sum-exps [n_query_sets][batch][n_q_heads] fp32 if lse_dev / lse_host are given -- both or neither) from device
+ * memory to HOST memory, asynchronously on `stream` (the device-to-host copy engine: it does not compete with an
+ * upload).  Meant for a stream of its own, ordered after the attention by the caller, so that the transfer is off
+ * the decode loop's critical path. */
+mc_status mc_decode_drain_host(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets,
+                               const void* out_dev, const float* lse_dev, void* out_host, float* lse_host,
+                               void* stream);
+
 /* Bytes of device staging mc_decode_attn_host needs (q, new K/V rows, out, lse). Host arithmetic. */
 mc_status mc_decode_io_bytes(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets,
                              size_t* bytes);

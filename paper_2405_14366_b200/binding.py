@@ -80,7 +80,7 @@ class _Stats(C.Structure):
                 ("compressed_bytes", C.c_int64), ("stored_bytes", C.c_int64)]
 
 
-EXPORTS = ("mc_decode_attn_append", "mc_prefill_merge_pair", "mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
+EXPORTS = ("mc_decode_drain_host", "mc_decode_stage_host", "mc_decode_attn_append", "mc_prefill_merge_pair", "mc_admit_sequences", "mc_build_flags", "mc_merge_pairs", "mc_pair_bytes", "mc_get_stats", "mc_version", "mc_status_str", "mc_last_cuda_error", "mc_workspace_bytes", "mc_merge_pair",
            "mc_append_pair", "mc_restore", "mc_decode_attn", "mc_read_status", "mc_merge_pair_host",
            "mc_decode_attn_host", "mc_decode_io_bytes", "mc_decode_attn_static", "mc_merge_pair_q4", "mc_selftest_wait_timeout")
 
@@ -316,6 +316,10 @@ class MiniCacheLib:
         L.mc_decode_attn_append.argtypes = [P(_Config), P(_Batch), P(_PairCache), C.c_int32, V, V, V, C.c_float, V, V, V, V, V, V,
                                             V, C.c_size_t, V]
         L.mc_decode_attn_append.restype = C.c_int32
+        L.mc_decode_stage_host.argtypes = [P(_Config), P(_Batch), C.c_int32, V, V, V, V, C.c_size_t, P(V), P(V), P(V), V]
+        L.mc_decode_stage_host.restype = C.c_int32
+        L.mc_decode_drain_host.argtypes = [P(_Config), P(_Batch), C.c_int32, V, V, V, V, V]
+        L.mc_decode_drain_host.restype = C.c_int32
         L.mc_read_status.argtypes = [P(_PairCache), V, P(C.c_int32)]
         L.mc_merge_pair_host.argtypes = [P(_Config), P(_Batch), P(_LayerKV), P(_LayerKV), P(_LayerKV), P(_LayerKV),
                                          P(_PairCache), C.c_int32, V, C.c_size_t, V]
@@ -494,6 +498,33 @@ class MiniCacheLib:
                                                   _ptr(lse_host), _ptr(dev_io), dev_io.numel() * dev_io.element_size(),
                                                   _ptr(workspace), workspace.numel() * workspace.element_size(),
                                                   _stream(stream)))
+
+    def mc_decode_stage_host(self, cfg: McConfig, batch: Batch, n_query_sets: int, q_host, k_new_host, v_new_host,
+                             dev_io: torch.Tensor, stream=None):
+        """Stages q (and the new rows) from host tensors into `dev_io`; returns views of dev_io: (q, k_new, v_new)
+        shaped [n_query_sets][batch][heads][128] in the storage type (k_new / v_new None if not given)."""
+        c, b = cfg.c(), batch.c()
+        qd, kd, vd = C.c_void_p(), C.c_void_p(), C.c_void_p()
+        self._check(self._lib.mc_decode_stage_host(C.byref(c), C.byref(b), int(n_query_sets), _ptr(q_host), _ptr(k_new_host),
+                                                   _ptr(v_new_host), _ptr(dev_io), dev_io.numel() * dev_io.element_size(),
+                                                   C.byref(qd), C.byref(kd), C.byref(vd), _stream(stream)))
+        base = dev_io.data_ptr()
+        nb = batch.seq_lens.shape[0]
+
+        def view(ptr, heads):
+            if not ptr.value:
+                return None
+            n = n_query_sets * nb * heads * 256
+            off = ptr.value - base
+            return dev_io[off:off + n].view(cfg.torch_dtype).view(n_query_sets, nb, heads, 128)
+        return view(qd, cfg.n_q_heads), view(kd, cfg.n_kv_heads), view(vd, cfg.n_kv_heads)
+
+    def mc_decode_drain_host(self, cfg: McConfig, batch: Batch, n_query_sets: int, out_dev, lse_dev, out_host, lse_host,
+                             stream=None):
+        """Asynchronous copy of an attention result (and its log-sum-exps, if given) from device to host tensors."""
+        c, b = cfg.c(), batch.c()
+        self._check(self._lib.mc_decode_drain_host(C.byref(c), C.byref(b), int(n_query_sets), _ptr(out_dev), _ptr(lse_dev),
+                                                   _ptr(out_host), _ptr(lse_host), _stream(stream)))
 
     def mc_decode_attn_static(self, cfg: McConfig, batch: Batch, pair: PairCache, layer_sel: int, q, k_new, v_new,
                               sm_scale: float, out, lse, stream=None):

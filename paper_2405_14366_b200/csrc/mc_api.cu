@@ -134,7 +134,7 @@ using namespace mc;
 
 extern "C" {
 
-int32_t mc_version(void) { return 230; }
+int32_t mc_version(void) { return 240; }
 
 int32_t mc_build_flags(void) {
 #if defined(MC_BOUNDS) && MC_BOUNDS
@@ -643,6 +643,58 @@ mc_status mc_decode_attn_host(const mc_config* cfg, const mc_batch* batch, const
   if (lse_host)
     MC_CUDA_CHECK(cudaMemcpyAsync(lse_host, io + off[4], (size_t)n_sets * batch->batch * cfg->n_q_heads * sizeof(float),
                                   cudaMemcpyDeviceToHost, s));
+  return MC_OK;
+}
+
+mc_status mc_decode_stage_host(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets, const void* q_host,
+                               const void* k_new_host, const void* v_new_host, void* dev_io, size_t dev_io_bytes, void** q_dev,
+                               void** k_new_dev, void** v_new_dev, void* stream) {
+  ApiRange range_("mc_decode_stage_host");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (!batch || batch->batch < 0 || (n_query_sets != 1 && n_query_sets != 2)) return MC_ERR_INVALID_ARG;
+  if (!q_host || !dev_io || !q_dev || !k_new_dev || !v_new_dev) return MC_ERR_INVALID_ARG;
+  if ((k_new_host == nullptr) != (v_new_host == nullptr)) return MC_ERR_INVALID_ARG;
+  if (!aligned256(dev_io)) return MC_ERR_ALIGN;
+  size_t off[6];
+  decode_io_layout(cfg, batch, n_query_sets, off);
+  if (dev_io_bytes < off[5]) return MC_ERR_CAPACITY;
+  char* io = (char*)dev_io;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t qb = (size_t)n_query_sets * batch->batch * cfg->n_q_heads * kRowBytes;
+  const size_t nb = (size_t)n_query_sets * batch->batch * cfg->n_kv_heads * kRowBytes;
+  *q_dev = io + off[0];
+  *k_new_dev = k_new_host ? io + off[1] : nullptr;
+  *v_new_dev = v_new_host ? io + off[2] : nullptr;
+  // device-addressable pinned memory is fetched by a kernel (no copy engine: the transfer does not queue behind
+  // large uploads on other streams); anything else by asynchronous copies
+  const void* src[3] = {device_view(q_host), k_new_host ? device_view(k_new_host) : nullptr,
+                        v_new_host ? device_view(v_new_host) : nullptr};
+  void* dst[3] = {io + off[0], io + off[1], io + off[2]};
+  const size_t bytes[3] = {qb, nb, nb};
+  const int n = k_new_host ? 3 : 1;
+  bool direct = true;
+  for (int a = 0; a < n; ++a) direct = direct && src[a] != nullptr && (((uintptr_t)src[a]) & 15u) == 0;
+  if (direct) return launch_fetch3(src, dst, bytes, n, s);
+  MC_CUDA_CHECK(cudaMemcpyAsync(dst[0], q_host, qb, cudaMemcpyHostToDevice, s));
+  if (k_new_host) {
+    MC_CUDA_CHECK(cudaMemcpyAsync(dst[1], k_new_host, nb, cudaMemcpyHostToDevice, s));
+    MC_CUDA_CHECK(cudaMemcpyAsync(dst[2], v_new_host, nb, cudaMemcpyHostToDevice, s));
+  }
+  return MC_OK;
+}
+
+mc_status mc_decode_drain_host(const mc_config* cfg, const mc_batch* batch, int32_t n_query_sets, const void* out_dev,
+                               const float* lse_dev, void* out_host, float* lse_host, void* stream) {
+  ApiRange range_("mc_decode_drain_host");
+  mc_status st = check_config(cfg);
+  if (st != MC_OK) return st;
+  if (!batch || batch->batch < 0 || (n_query_sets != 1 && n_query_sets != 2)) return MC_ERR_INVALID_ARG;
+  if (!out_dev || !out_host || ((lse_dev == nullptr) != (lse_host == nullptr))) return MC_ERR_INVALID_ARG;
+  const size_t rows = (size_t)n_query_sets * batch->batch * cfg->n_q_heads;
+  if (rows == 0) return MC_OK;
+  MC_CUDA_CHECK(cudaMemcpyAsync(out_host, out_dev, rows * kRowBytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  if (lse_host) MC_CUDA_CHECK(cudaMemcpyAsync(lse_host, lse_dev, rows * sizeof(float), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   return MC_OK;
 }
 

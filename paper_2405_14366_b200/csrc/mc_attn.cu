@@ -1292,6 +1292,37 @@ mc_status launch_fetch_rows(const void* k_src, const void* v_src, void* k_dst, v
   return MC_OK;
 }
 
+// Up to three arrays (16-byte pieces) from device-addressable host memory into device memory, one launch.
+struct Fetch3 {
+  const uint4* src[3];
+  uint4* dst[3];
+  int n16[3];
+};
+__global__ void __launch_bounds__(256) fetch3_kernel(const Fetch3 f) {
+  grid_dep_launch();
+  const int a = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (i < f.n16[a]) v = f.src[a][i];  // the caller's rows are read before the wait, the staging buffer written after it
+  grid_dep_wait();
+  if (i < f.n16[a]) f.dst[a][i] = v;
+}
+
+mc_status launch_fetch3(const void* const* src, void* const* dst, const size_t* bytes, int n, cudaStream_t stream) {
+  Fetch3 f;
+  int most = 0;
+  for (int a = 0; a < 3; ++a) {
+    f.src[a] = a < n ? (const uint4*)src[a] : nullptr;
+    f.dst[a] = a < n ? (uint4*)dst[a] : nullptr;
+    f.n16[a] = a < n ? (int)(bytes[a] / 16) : 0;
+    most = std::max(most, f.n16[a]);
+  }
+  if (most == 0) return MC_OK;
+  MC_CUDA_CHECK(launch_pdl(fetch3_kernel, dim3((most + 255) / 256, n), dim3(256), 0, stream, f));
+  MC_CUDA_CHECK(cudaGetLastError());
+  return MC_OK;
+}
+
 }  // namespace mc
 
 // ---------------------------------------------------------------------------------------------------

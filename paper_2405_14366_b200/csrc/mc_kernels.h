@@ -56,6 +56,8 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
                              int layer_sel, const void* q, const void* k_new, const void* v_new, float sm_scale,
                              void* out, float* lse, void* workspace, cudaStream_t stream, const AppendParams* append = nullptr);
 
+// Up to three arrays (sizes multiples of 16 bytes) from device-addressable host memory into device memory, by a kernel.
+mc_status launch_fetch3(const void* const* src, void* const* dst, const size_t* bytes, int n, cudaStream_t stream);
 // Copies the new token's K and V rows (n bytes each, a multiple of 16) from device-addressable host
 // memory into device staging with one small kernel.
 mc_status launch_fetch_rows(const void* k_src, const void* v_src, void* k_dst, void* v_dst, size_t n, cudaStream_t stream);

@@ -102,3 +102,48 @@ def test_folded_append_checks_every_argument_before_launching(H):
     torch.cuda.synchronize()
     after = _pair_state(p)
     assert all(torch.equal(before[k], after[k]) for k in before) and not o.any()
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_inputs_staged_from_host_memory_give_the_same_attention(H, pinned):
+    """mc_decode_stage_host on a second stream, then the attention on the staged rows, with the result written
+    straight to pinned host memory: the same bits as the call on device tensors."""
+    wl = CONFIGS["c1"].scaled("stage", n_kv_heads=4, n_q_heads=8, dtype="bf16", batch=3, seq_len=96, page_size=16, index=99)
+    p = H.Problem(wl, seq_lens=np.array([96, 17, 40], np.int32), decode_room=2)
+    words, code = p.run_merge()
+    assert code == 0
+    wlb = dataclasses.replace(wl, batch=3)
+    nt = gen.make_new_tokens(wlb, 0, 0)
+    q = gen.make_queries(wlb, 3, n_sets=2)
+    kn = torch.stack([nt["k_lm1"][:, 0], nt["k_l"][:, 0]]).contiguous()
+    vn = torch.stack([nt["v_lm1"][:, 0], nt["v_l"][:, 0]]).contiguous()
+    host = [t.pin_memory() if pinned else t.clone() for t in (q, kn, vn)]
+    batch = p.batch(1)
+    io = torch.empty(p.lib.mc_decode_io_bytes(p.cfg, batch, 2), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        qd, knd, vnd = p.lib.mc_decode_stage_host(p.cfg, batch, 2, host[0], host[1], host[2], io, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    assert torch.equal(qd.cpu(), q) and torch.equal(knd.cpu(), kn) and torch.equal(vnd.cpu(), vn)
+    sm = 1.0 / math.sqrt(128.0)
+    ws = p.workspace(1, 1, 1)
+    out_host = torch.zeros(1, p.B, p.Hq, 128, dtype=p.cfg.torch_dtype).pin_memory()
+    lse_host = torch.zeros(1, p.B, p.Hq, dtype=torch.float32).pin_memory()
+    p.lib.mc_decode_attn(p.cfg, batch, p.pair, 1, qd[1], knd[1], vnd[1], sm, out_host, lse_host, ws)
+    ref = torch.zeros(1, p.B, p.Hq, 128, dtype=p.cfg.torch_dtype, device="cuda")
+    ref_lse = torch.zeros(1, p.B, p.Hq, dtype=torch.float32, device="cuda")
+    p.lib.mc_decode_attn(p.cfg, batch, p.pair, 1, q[1:2].contiguous().cuda(), kn[1:2].contiguous().cuda(),
+                         vn[1:2].contiguous().cuda(), sm, ref, ref_lse, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, ref.cpu()) and torch.equal(lse_host, ref_lse.cpu())
+    # ... and the result copied back by the library on a stream of its own
+    back = torch.zeros(1, p.B, p.Hq, 128, dtype=p.cfg.torch_dtype).pin_memory()
+    back_lse = torch.zeros(1, p.B, p.Hq, dtype=torch.float32).pin_memory()
+    side.wait_stream(torch.cuda.current_stream())
+    p.lib.mc_decode_drain_host(p.cfg, batch, 1, ref, ref_lse, back, back_lse, stream=side)
+    side.synchronize()
+    assert torch.equal(back, ref.cpu()) and torch.equal(back_lse, ref_lse.cpu())
+    # the staging refuses a buffer that is too small, before anything is enqueued
+    with pytest.raises(p.mc.McError):
+        p.lib.mc_decode_stage_host(p.cfg, batch, 2, host[0], host[1], host[2], io[:256])
