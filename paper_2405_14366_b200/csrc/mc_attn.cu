@@ -39,7 +39,8 @@ namespace mc {
 
 constexpr int kTile = 64;  // tokens per pipeline stage
 constexpr int kUnit_ = 128;  // (= kUnit below) tokens per stage of 4-bit tiles
-constexpr int kStages = 5;
+constexpr int kStages = 5;      // ring stages of the 16-bit kernel with one query row per kv head
+constexpr int kStagesWide = 4;  // ... with several rows: a stage is given up for a score buffer twice the size
 constexpr int kConsumerWarps = 4;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kAttnThreads = kConsumerThreads + 32;  // + producer warp
@@ -135,16 +136,21 @@ __device__ __forceinline__ uint32_t tile_addr(uint32_t stage, int tk, int chunk,
 }
 
 constexpr int kUnit = 128;            // tokens per unit of work: pieces start and end on unit boundaries
-constexpr int kScoreFloats = 4224;    // floats of the score buffer S [rows][piece tokens + 8] (16.5 KB)
+// Floats of the score buffer S [rows][piece tokens + 8]: 16.5 KB, or 33 KB (WIDE) where several query rows share
+// a kv head (grouped queries, pair mode) and for the 4-bit cache, whose stages are smaller: chunks twice as long,
+// half as many switches between the K and the V phase of a piece.
+constexpr int kScoreFloats = 4224;
+constexpr int kScoreFloatsWide = 8448;
 constexpr int kMaxPiecePages = 256;   // pages of the longest piece (4096 tokens of 16-token pages)
 
 // Longest chunk for `rows` query rows: rows x (tokens + 8) floats must fit the score buffer.
-__host__ __device__ __forceinline__ int piece_cap_units(int rows) {
-  const int u = (kScoreFloats / rows - 8) / kUnit;
-  return u > 32 ? 32 : u;  // 32 units (rows = 1) ... 4 units (rows = 8)
+__host__ __device__ __forceinline__ int piece_cap_units(int rows, bool wide) {
+  const int u = ((wide ? kScoreFloatsWide : kScoreFloats) / rows - 8) / kUnit;
+  return u > 32 ? 32 : u;  // 32 units (rows = 1) ... 4 units (rows = 8; 8 with the wide buffer)
 }
 // The same memory later holds the four warps' partial outputs [4][rows][kSlabStride].
 static_assert(kMaxRows * ((kScoreFloats / kMaxRows - 8) / kUnit * kUnit + 8) <= kScoreFloats, "score buffer");
+static_assert(kMaxRows * ((kScoreFloatsWide / kMaxRows - 8) / kUnit * kUnit + 8) <= kScoreFloatsWide, "score buffer");
 static_assert(kConsumerWarps * kMaxRows * kSlabStride <= kScoreFloats, "slabs fit the score buffer");
 
 // The merge marks a retained token by the scale -0: the shared direction then contributes nothing
@@ -269,7 +275,7 @@ __device__ __forceinline__ Ranges ranges_of(const RawRanges& q) {
 // (128 tokens, one page per consumer warp), whose tensor-core fragments are built in registers straight
 // from the codes (code * scale + zero in one packed 16-bit FMA, the exact stored direction); the tokens
 // of a sequence's last, incomplete page arrive as one more tile stage in the 16-bit format.
-template <int DT, bool Q4>
+template <int DT, bool Q4, bool WIDE>
 __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(const AttnParams p) {
   // The batch description (lengths, block table) and the queries belong to the caller: no kernel of
   // this library writes them, so they are read before the wait on the previous kernel in the
@@ -278,7 +284,8 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   // stage ring: five slots of 64 tokens of 16-bit tiles, or (4-bit cache) four slots of four 4-bit tiles,
   // which also hold the residual tile or a stage of retained entries
   constexpr int STAGE_BYTES = Q4 ? kQ4StageBytes : kStageBytes;
-  constexpr int N_STAGES = Q4 ? kQ4Stages : kStages;
+  constexpr int N_STAGES = Q4 ? kQ4Stages : (WIDE ? kStagesWide : kStages);
+  constexpr int SCORE_FLOATS = WIDE ? kScoreFloatsWide : kScoreFloats;
   grid_dep_launch();
   const int ps = p.g.page_size, shift = p.g.page_shift;
   const int H = p.g.n_kv_heads;
@@ -293,7 +300,7 @@ __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm) attn_split_kernel(co
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   unsigned char* stages = smem;
   float* S = reinterpret_cast<float*>(smem + N_STAGES * STAGE_BYTES);     // [kMaxRows][s_stride]
-  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + kScoreFloats);         // [2][kMaxRows][64] packed pairs
+  uint32_t* q_s = reinterpret_cast<uint32_t*>(S + SCORE_FLOATS);         // [2][kMaxRows][64] packed pairs
   float* m_s = reinterpret_cast<float*>(q_s + 2 * kMaxRows * 64);        // [kMaxRows]
   float* l_s = m_s + kMaxRows;                                           // [kMaxRows][kConsumerWarps]
   float* red_s = l_s + kMaxRows * kConsumerWarps;                        // [kMaxRows][kConsumerWarps]
@@ -1154,8 +1161,9 @@ __global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const Att
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static size_t attn_smem_bytes(bool q4) {
-  size_t b = 128 + (q4 ? (size_t)kQ4Stages * kQ4StageBytes : (size_t)kStages * kStageBytes) + (size_t)kScoreFloats * 4;  // stages, S
+static size_t attn_smem_bytes(bool q4, bool wide) {
+  size_t b = 128 + (q4 ? (size_t)kQ4Stages * kQ4StageBytes : (size_t)(wide ? kStagesWide : kStages) * kStageBytes) +
+             (size_t)(wide ? kScoreFloatsWide : kScoreFloats) * 4;  // stages, S
   b += 2 * kMaxRows * 64 * 4;                                                  // q_s
   b += kMaxRows * 4 + 3 * kMaxRows * kConsumerWarps * 4;                       // m, l, red, red2
   b += 2 * kStages * 4 + (2 * kMaxBatchSmem + 1) * 4 + 2 * kMaxPiecePages * 4 + 4 + 8 + 2 * kStages * 8 + 64;
@@ -1197,7 +1205,8 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   ap.nq = cfg->n_q_heads / cfg->n_kv_heads;
   ap.rows = ap.n_sets * ap.nq;
   ap.n_q_heads = cfg->n_q_heads;
-  ap.cap_units = piece_cap_units(ap.rows);
+  const bool wide = q4 || ap.rows > 1;  // (see kScoreFloatsWide)
+  ap.cap_units = piece_cap_units(ap.rows, wide);
   ap.slots = (int)attn_slots(bt);
   const size_t prow = (size_t)ap.n_sets * bt->batch * cfg->n_q_heads * ap.slots;
   ap.part_o = reinterpret_cast<float*>(workspace);
@@ -1215,13 +1224,14 @@ mc_status launch_decode_attn(const mc_config* cfg, const mc_batch* bt, const Geo
   const int grid = n_teams * ap.team_size;
   ap.n_teams = n_teams;
   if (n_teams > kMaxPieces) return MC_ERR_SHAPE;  // pieces of one sequence
-  const size_t smem = attn_smem_bytes(q4);
+  const size_t smem = attn_smem_bytes(q4, wide);
   // many output rows: a warp per row; few: a block per row
   const bool warp_rows = (long long)ap.n_sets * bt->batch * cfg->n_q_heads >= 1024;
   dim3 cgrid(warp_rows ? (cfg->n_q_heads + kCombineWarps - 1) / kCombineWarps : cfg->n_q_heads, bt->batch, ap.n_sets);
   void (*split)(const AttnParams) =
-      cfg->dtype == MC_F16 ? (q4 ? attn_split_kernel<MC_F16, true> : attn_split_kernel<MC_F16, false>)
-                           : (q4 ? attn_split_kernel<MC_BF16, true> : attn_split_kernel<MC_BF16, false>);
+      cfg->dtype == MC_F16
+          ? (q4 ? attn_split_kernel<MC_F16, true, true> : (wide ? attn_split_kernel<MC_F16, false, true> : attn_split_kernel<MC_F16, false, false>))
+          : (q4 ? attn_split_kernel<MC_BF16, true, true> : (wide ? attn_split_kernel<MC_BF16, false, true> : attn_split_kernel<MC_BF16, false, false>));
   // (the append rides on the combine launch: ceil(2 H / 16) more blocks per sequence)
   AppendParams app;
   memset(&app, 0, sizeof(app));
