@@ -33,9 +33,9 @@ import gen  # noqa: E402
 
 ROW = 256  # bytes of one 16-bit row of 128 channels
 # DRAM bytes (read + written) per algorithmic byte of the split attention kernel (16-bit cache), from the ncu
-# capture summarised in profiles/attn_split_kernel_c2_one_pair.md (560.4 MB for 547.5 MB), taken after the
-# kernel became a template over the cache format.  Set to None when the kernel changes until it is captured again.
-ATTN_TRAFFIC_RATIO = 1.024
+# capture summarised in profiles/attn_split_kernel_c2_one_pair.md (560.2 MB for 547.5 MB), taken of the kernel
+# as it is now (a template over the cache format and the score-buffer width).  Set to None when the kernel changes until it is captured again.
+ATTN_TRAFFIC_RATIO = 1.023
 
 
 # ---------------------------------------------------------------------------------------------
