@@ -205,3 +205,43 @@ def test_a_segment_without_free_entries_merges_the_token_and_says_so(H):
                 marked = np.nonzero(np.signbit(g))[0] + 96
                 assert np.array_equal(marked, [first[(ti, b, h)]] if took else [])
                 assert np.all(g[~np.signbit(g)] > 0)
+
+
+def test_free_entries_in_the_regions_of_admitted_sequences(H):
+    """Sequences admitted one by one (mc_admit_sequences: every sequence's retained entries in its own region of the
+    pool) get their free entries too; tokens appended afterwards are kept in their own segment's list."""
+    steps = 4
+    wl = CONFIGS["c1"].scaled("rethr_adm", n_kv_heads=2, n_q_heads=4, dtype="f16", batch=3, seq_len=128, page_size=16,
+                              outlier_frac=0.05, index=93)
+    lens = np.array([128, 40, 77], np.int32)
+    R = 2 * 2 * (40 + steps)  # entries per sequence
+    p = H.Problem(wl, seq_lens=lens, gamma=0.2, append_slack=steps, decode_room=steps, ret_capacity=3 * R)
+    ws = torch.empty(p.lib.mc_workspace_bytes(p.cfg, p.batch(), 0), dtype=torch.uint8, device=p.device)
+    for b in (2, 0, 1):
+        p.lib.mc_admit_sequences(p.cfg, p.batch(), b, 1, [p.pools], [p.pair], R, True, ws)
+    torch.cuda.synchronize()
+    words, code = p.lib.mc_read_status(p.pair, check=False)
+    assert code == 0, words
+    om = p.oracle_merge()
+    H.compare_merge(p, om, p.device_cache())
+    off = p.pair.ret_offset.cpu().numpy()[:-1].reshape(2, p.B, p.H)
+    cnt = p.pair.ret_count.cpu().numpy().reshape(2, p.B, p.H)
+    idx = p.pair.ret_index.cpu().numpy()
+    for ti in range(2):
+        for b in range(p.B):
+            for h in range(p.H):
+                o, c = int(off[ti, b, h]), int(cnt[ti, b, h])
+                assert o // R == b and (o + c + steps - 1) // R == b, "list and free entries inside the sequence's region"
+                assert np.all(idx[o + c:o + c + steps] == -1)
+    kept, near = _decode_with_retention(H, p, om, steps, "distinct", outlier_frac=0.5)
+    assert kept > 0
+    p.S += steps
+    dc = p.device_cache()
+    for ti, tn in enumerate(("k", "v")):
+        for b in range(p.B):
+            for h in range(p.H):
+                got, rows = p.retained(dc, ti, b, h)
+                assert np.array_equal(got, om[tn]["retained"][(b, h)])
+                assert np.array_equal(rows[:, 1], p.bits[tn + "_l"][b, got, h])
+    off2 = p.pair.ret_offset.cpu().numpy()[:-1].reshape(2, p.B, p.H)
+    assert np.array_equal(off, off2)
