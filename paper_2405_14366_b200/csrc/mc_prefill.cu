@@ -31,9 +31,9 @@ constexpr int kPfTileM = 128;   // tokens per tile
 constexpr int kPfTileN = 128;   // channels per tile = one head
 constexpr int kPfTileK = 64;    // elements per stage row: 128 bytes, the swizzle span
 constexpr int kPfStages = 2;
-constexpr int kPfStageBytes = (kPfTileM + kPfTileN) * kPfTileK * 2;  // X tile, then W tile: 32 KB
+constexpr int kPfStageBytes = (kPfTileM + kPfTileN) * kPfTileK * 2;  // X tile, then W tile of one head: 32 KB
 constexpr int kPfThreads = 192;
-constexpr int kPfTmemCols = 128;
+constexpr int kPfTmemCols = 128;  // per head
 constexpr int kPfEpiRow = kRowBytes + 16;           // a staged row, padded: 32 rows fall into different banks
 constexpr int kPfEpiWarp = 32 * kPfEpiRow;          // staging of one epilogue warp's 32 rows: 8704 bytes
 
@@ -49,6 +49,7 @@ struct PrefillParams {
   int d_model;
   int n_mtiles;      // token tiles in all: batch * x_seq_stride / 128
   int mt_group, ht_group, n_htg;  // tile order, see below
+  int n_hgroups;  // columns per tensor: kv heads / heads per CTA
   float ta, tc;
   int t_mode;
   float d_hint;
@@ -102,13 +103,17 @@ __device__ __forceinline__ uint64_t smem_desc_k128(uint32_t smem_addr) {
          ((uint64_t)2 << 61);
 }
 // Instruction descriptor: fp32 accumulate, A and B of the 16-bit type (both K-major), N = 128, M = 128.
-template <int DT>
+template <int DT, int N>
 __device__ __forceinline__ uint32_t umma_idesc() {
   const uint32_t fmt = DT == MC_F16 ? 0u : 1u;
-  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kPfTileN >> 3) << 17) | ((uint32_t)(kPfTileM >> 4) << 24);
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kPfTileM >> 4) << 24);
 }
 
-template <int DT>
+// NH = heads per CTA.  NH = 2: the tile is 128 tokens x 256 channels (one N = 256 instruction per K step, 256
+// columns of tensor memory), the X tile feeds two heads -- a quarter less operand traffic through L2 per output
+// element, which is what bounds the launch; the stages are 48 KB then, and the epilogue's row staging takes the
+// stage memory over once the main loop is done (layer l-1's rows are fetched only then, head by head).
+template <int DT, int NH>
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_constant__ CUtensorMap map_x,
                      const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv) {
@@ -116,10 +121,13 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
   grid_dep_launch();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kPfStages * kPfStageBytes);  // full[stages], empty[stages], accum
+  constexpr int STAGE_BYTES = (kPfTileM + NH * kPfTileN) * kPfTileK * 2;
+  constexpr int TMEM_COLS = NH * kPfTmemCols;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kPfStages * STAGE_BYTES);  // full[stages], empty[stages], accum
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPfStages + 1);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  unsigned char* epi = smem + kPfStages * kPfStageBytes + 256;  // [4 warps][32 rows][kPfEpiRow]: row staging of the epilogue
+  // [4 warps][32 rows][kPfEpiRow]: row staging of the epilogue (NH = 2: over the stages, after the main loop)
+  unsigned char* epi = NH == 1 ? smem + kPfStages * STAGE_BYTES + 256 : smem;
   const uint32_t stage0 = smem_u32(smem);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kPfStages, accum_bar = empty0 + 8 * kPfStages;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -135,7 +143,7 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
   const int mt = (grp / p.n_htg) * p.mt_group + within % p.mt_group;
   const int ht = (grp % p.n_htg) * p.ht_group + within / p.mt_group;
   if (mt >= p.n_mtiles) return;
-  const int tensor = ht / H, head = ht % H;
+  const int tensor = ht / p.n_hgroups, head0 = (ht % p.n_hgroups) * NH;
   const int tiles_per_seq = p.x_seq_stride / kPfTileM;
   const int b = mt / tiles_per_seq, tile = mt % tiles_per_seq;
   const int tok0 = tile * kPfTileM;
@@ -151,7 +159,7 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kPfTmemCols);
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -166,22 +174,22 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
         const int s = kb % kPfStages;
         if (kb >= kPfStages && !mbar_wait(empty0 + 8 * s, ((kb / kPfStages) - 1) & 1, s_abort, p.status)) break;
         const uint32_t bar = full0 + 8 * s;
-        mbar_expect_tx(bar, (uint32_t)kPfStageBytes);
-        tma_load_2d(stage0 + s * kPfStageBytes, &map_x, kb * kPfTileK, b * p.x_seq_stride + tok0, bar);
-        tma_load_2d(stage0 + s * kPfStageBytes + kPfTileM * kPfTileK * 2, map_w, kb * kPfTileK, head * kPfTileN, bar);
+        mbar_expect_tx(bar, (uint32_t)STAGE_BYTES);
+        tma_load_2d(stage0 + s * STAGE_BYTES, &map_x, kb * kPfTileK, b * p.x_seq_stride + tok0, bar);
+        tma_load_2d(stage0 + s * STAGE_BYTES + kPfTileM * kPfTileK * 2, map_w, kb * kPfTileK, head0 * kPfTileN, bar);
       }
     }
   } else if (warp == 1) {
     // ===================== tensor-core issue =====================
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc<DT>();
+      const uint32_t idesc = umma_idesc<DT, NH * kPfTileN>();
       bool ok = true;
       for (int kb = 0; kb < n_kb && ok; ++kb) {
         const int s = kb % kPfStages;
         if (!mbar_wait(full0 + 8 * s, (kb / kPfStages) & 1, s_abort, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint64_t da = smem_desc_k128(stage0 + s * kPfStageBytes);
-        const uint64_t db = smem_desc_k128(stage0 + s * kPfStageBytes + kPfTileM * kPfTileK * 2);
+        const uint64_t da = smem_desc_k128(stage0 + s * STAGE_BYTES);
+        const uint64_t db = smem_desc_k128(stage0 + s * STAGE_BYTES + kPfTileM * kPfTileK * 2);
 #pragma unroll
         for (int k = 0; k < kPfTileK / 16; ++k)  // 16 elements (32 bytes) per instruction along K
           umma_f16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -200,21 +208,34 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
     int page = -1;
     if (tok < n) page = checked_page(p.g, b, tok >> shift, p.status);
     const int tk = tok & (ps - 1);
-    const int prow = page >= 0 ? (page * H + head) * ps + tk : -1;  // row index inside a layer pool (-1: no such row)
-    unsigned char* my = epi + q * kPfEpiWarp;
+    unsigned char* my = epi + q * kPfEpiWarp;  // (head hh of the CTA: + hh * 4 * kPfEpiWarp)
     const int r_half = lane >> 4, ch16 = lane & 15;
-    // layer l-1's rows go to the staging area while the tensor cores are still busy
+    // layer l-1's rows of head `hd` into its staging area, sixteen lanes per row
+    auto fetch_a = [&](int hd) {
+      unsigned char* my = epi + (hd - head0) * 4 * kPfEpiWarp + q * kPfEpiWarp;
+      const int prow_h = page >= 0 ? (page * H + hd) * ps + tk : -1;
 #pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-      const int r = 2 * i + r_half;
-      const int pr = __shfl_sync(0xffffffffu, prow, r);
-      if (pr >= 0)
-        *reinterpret_cast<uint4*>(my + r * kPfEpiRow + ch16 * 16) =
-            ld_stream16(p.a_pool[tensor] + (size_t)pr * kRowBytes + ch16 * 16);
-    }
-    __syncwarp();
+      for (int i = 0; i < 16; ++i) {
+        const int r = 2 * i + r_half;
+        const int pr = __shfl_sync(0xffffffffu, prow_h, r);
+        if (pr >= 0)
+          *reinterpret_cast<uint4*>(my + r * kPfEpiRow + ch16 * 16) =
+              ld_stream16(p.a_pool[tensor] + (size_t)pr * kRowBytes + ch16 * 16);
+      }
+      __syncwarp();
+    };
+    if (NH == 1) fetch_a(head0);  // ... while the tensor cores are still busy (its own staging area)
     const bool ok_wait = mbar_wait(accum_bar, 0, s_abort, p.status);
     tc_fence_after();
+    if (NH > 1) {  // (the stages are free: every tensor-core instruction has completed; both heads' rows are
+      fetch_a(head0);  //  requested now, the second head's arrive under the first head's passes)
+      fetch_a(head0 + 1);
+    }
+#pragma unroll 1
+    for (int hh = 0; hh < NH; ++hh) {
+    const int head = head0 + hh;
+    const int prow = page >= 0 ? (page * H + head) * ps + tk : -1;  // row index inside a layer pool (-1: no such row)
+    my = epi + hh * 4 * kPfEpiWarp + q * kPfEpiWarp;
     const bool live = ok_wait && !*s_abort && prow >= 0;
     // Layer l's row = the accumulators rounded once to the storage type (what the model would have cached).
     // Neither row is held in registers across the three passes of the merge (two 64-register copies would not
@@ -225,7 +246,7 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
     const unsigned char* my_row = my + lane * kPfEpiRow;
     auto load_c = [&](int j, uint32_t (&cj)[16]) {
       uint32_t r[32];
-      tmem_ld32(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * 32), r);
+      tmem_ld32(tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)(hh * kPfTmemCols + j * 32), r);
 #pragma unroll
       for (int i = 0; i < 16; ++i) cj[i] = Elem<DT>::pack(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
     };
@@ -331,13 +352,15 @@ prefill_merge_kernel(const __grid_constant__ PrefillParams p, const __grid_const
       atomicMin(&p.seg_minmax[2 * seg], __float_as_uint(dmin));
       atomicMax(&p.seg_minmax[2 * seg + 1], __float_as_uint(dmax));
     }
+    __syncwarp();  // (the staging area is reused by the next head)
+    }
   }
   // ---- every path ends here: the accumulators are no longer needed, the tensor memory goes back
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_d, kPfTmemCols);
+    tmem_dealloc(tmem_d, TMEM_COLS);
   }
   if (*s_abort) {
     for (int x = 0; x < 2000; ++x) __nanosleep(1000);  // let copies in flight land before the CTA's memory is released
@@ -363,13 +386,13 @@ static EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// A [rows][cols] 16-bit row-major matrix, copied in boxes of 128 rows x 64 columns with the 128-byte swizzle.
-static mc_status make_map(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols) {
+// A [rows][cols] 16-bit row-major matrix, copied in boxes of box_rows rows x 64 columns with the 128-byte swizzle.
+static mc_status make_map(CUtensorMap* map, int dtype, const void* base, uint64_t rows, uint64_t cols, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return MC_ERR_UNSUPPORTED;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kPfTileK, (cuuint32_t)kPfTileM};
+  const cuuint32_t box[2] = {(cuuint32_t)kPfTileK, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, dtype == MC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -388,9 +411,10 @@ mc_status launch_prefill_merge(const mc_config* cfg, const mc_batch* bt, const G
   CUtensorMap map_x, map_wk, map_wv;
   const uint64_t x_rows = (uint64_t)bt->batch * proj->x_seq_stride;
   const uint64_t w_rows = (uint64_t)cfg->n_kv_heads * kPfTileN;
-  if (mc_status st = make_map(&map_x, cfg->dtype, proj->x, x_rows, proj->d_model)) return st;
-  if (mc_status st = make_map(&map_wk, cfg->dtype, proj->w_k, w_rows, proj->d_model)) return st;
-  if (mc_status st = make_map(&map_wv, cfg->dtype, proj->w_v, w_rows, proj->d_model)) return st;
+  const int nh = cfg->n_kv_heads % 2 == 0 ? 2 : 1;  // heads per CTA
+  if (mc_status st = make_map(&map_x, cfg->dtype, proj->x, x_rows, proj->d_model, kPfTileM)) return st;
+  if (mc_status st = make_map(&map_wk, cfg->dtype, proj->w_k, w_rows, proj->d_model, nh * kPfTileN)) return st;
+  if (mc_status st = make_map(&map_wv, cfg->dtype, proj->w_v, w_rows, proj->d_model, nh * kPfTileN)) return st;
   PrefillParams pp;
   pp.g = g;
   pp.a_pool[0] = (const char*)lm1->k_pool;
@@ -408,9 +432,12 @@ mc_status launch_prefill_merge(const mc_config* cfg, const mc_batch* bt, const G
   pp.tc = (float)cfg->t;
   pp.t_mode = cfg->t_mode;
   pp.d_hint = d_hint;
-  const size_t smem = 1024 + (size_t)kPfStages * kPfStageBytes + 256 + 4 * (size_t)kPfEpiWarp;  // stages, barriers, row staging
+  // stages, barriers, row staging (two heads per CTA: the staging lives in the stages)
+  const size_t smem = nh == 1 ? 1024 + (size_t)kPfStages * kPfStageBytes + 256 + 4 * (size_t)kPfEpiWarp
+                              : 1024 + (size_t)kPfStages * (kPfTileM + 2 * kPfTileN) * kPfTileK * 2 + 256;
   pp.n_mtiles = bt->batch * (proj->x_seq_stride / kPfTileM);
-  const int n_ht = 2 * cfg->n_kv_heads;
+  pp.n_hgroups = cfg->n_kv_heads / nh;
+  const int n_ht = 2 * pp.n_hgroups;
   pp.ht_group = 1;
   for (int dv = 1; dv <= 16; ++dv)
     if (n_ht % dv == 0) pp.ht_group = dv;  // the largest divisor of the column count up to 16
@@ -420,7 +447,8 @@ mc_status launch_prefill_merge(const mc_config* cfg, const mc_batch* bt, const G
   if (n_ctas > 0x7fffffffLL) return MC_ERR_SHAPE;
   const dim3 grid((unsigned)n_ctas);
   void (*kern)(const PrefillParams, const CUtensorMap, const CUtensorMap, const CUtensorMap) =
-      cfg->dtype == MC_F16 ? prefill_merge_kernel<MC_F16> : prefill_merge_kernel<MC_BF16>;
+      cfg->dtype == MC_F16 ? (nh == 2 ? prefill_merge_kernel<MC_F16, 2> : prefill_merge_kernel<MC_F16, 1>)
+                           : (nh == 2 ? prefill_merge_kernel<MC_BF16, 2> : prefill_merge_kernel<MC_BF16, 1>);
   MC_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MC_CUDA_CHECK(launch_pdl(kern, grid, dim3(kPfThreads), smem, stream, pp, map_x, map_wk, map_wv));
   MC_CUDA_CHECK(cudaGetLastError());
